@@ -1,0 +1,168 @@
+"""Oracle: LLaMA-family decoder forward over tree rows, greedy decoding drivers.
+
+TEST INFRASTRUCTURE ONLY (see the package docstring).  Paper Eq. 1 (the
+autoregressive greedy target), Section 2.1 (Jacobi decoding), Section 3.3
+(TR-Jacobi: one forward verifies the tree and produces the next candidates).
+"""
+from __future__ import annotations
+
+from typing import Callable, Dict, List, Sequence
+
+import numpy as np
+
+from .accept import accept_path, compact_rows, node_argmax
+from .attention import tree_attention
+from .tree import build_tree, depths, refill_window, retrieve, ahead_noise
+
+
+def rmsnorm(h: np.ndarray, gain: np.ndarray, eps: float) -> np.ndarray:
+    """x / sqrt(mean(x^2) + eps) * gain along the last axis."""
+    ms = np.mean(h * h, axis=-1, keepdims=True)
+    return h / np.sqrt(ms + eps) * gain
+
+
+def rope(x: np.ndarray, pos: np.ndarray, theta: float) -> np.ndarray:
+    """Rotary embedding, half-split pairing: (x[i], x[i + D/2]) is rotated by pos * theta^(-2i/D).
+
+    x: [M, H, D]; pos: [M].
+    """
+    d = x.shape[-1]
+    half = d // 2
+    inv_freq = theta ** (-2.0 * np.arange(half, dtype=np.float64) / d)
+    ang = np.asarray(pos, np.float64)[:, None] * inv_freq[None, :]        # [M, half]
+    c, s = np.cos(ang)[:, None, :], np.sin(ang)[:, None, :]
+    a, b = x[..., :half], x[..., half:]
+    return np.concatenate([a * c - b * s, b * c + a * s], axis=-1)
+
+
+def silu(x: np.ndarray) -> np.ndarray:
+    return x / (1.0 + np.exp(-x))
+
+
+class KVCache:
+    """K and V of every layer, [L, H, capacity, D] fp64, and the number of committed rows."""
+
+    def __init__(self, n_layers: int, n_heads: int, capacity: int, head_dim: int):
+        self.k = np.zeros((n_layers, n_heads, capacity, head_dim), np.float64)
+        self.v = np.zeros((n_layers, n_heads, capacity, head_dim), np.float64)
+        self.seq_len = 0
+
+
+class Decoder:
+    """Random-init LLaMA-shaped decoder.
+
+    ``layers`` is indexable by layer and yields the dict produced by the input
+    generator (``attn_norm``, ``wqkv``, ``wo``, ``mlp_norm``, ``w_gate_up``,
+    ``w_down``; matrices are [d_out, d_in]); ``glob`` holds ``embed``,
+    ``lm_head``, ``final_norm``.
+    """
+
+    def __init__(self, cfg, layers, glob: Dict[str, np.ndarray]):
+        self.cfg = cfg
+        self.layers = layers
+        self.glob = glob
+
+    def new_cache(self, capacity: int) -> KVCache:
+        c = self.cfg
+        return KVCache(c.n_layers, c.n_heads, capacity, c.head_dim)
+
+    def forward_rows(self, cache: KVCache, tokens: Sequence[int], parent: Sequence[int]) -> np.ndarray:
+        """Logits [M, V] of the M tree rows given the cache's first ``seq_len`` rows.
+
+        K/V of tree row i is stored at cache row seq_len + i; ``seq_len`` itself
+        is left unchanged (the caller commits rows by compaction).
+        """
+        c = self.cfg
+        m, s = len(tokens), cache.seq_len
+        n_heads, hd = c.n_heads, c.head_dim
+        pos = s + depths(parent)
+        h = np.asarray(self.glob["embed"], np.float64)[np.asarray(tokens, np.int64)]
+        for l in range(c.n_layers):
+            w = self.layers[l]
+            x = rmsnorm(h, np.asarray(w["attn_norm"], np.float64), c.rms_eps)
+            qkv = x @ np.asarray(w["wqkv"], np.float64).T
+            q, k, v = (qkv[:, j * n_heads * hd:(j + 1) * n_heads * hd].reshape(m, n_heads, hd)
+                       for j in range(3))
+            q, k = rope(q, pos, c.rope_theta), rope(k, pos, c.rope_theta)
+            cache.k[l][:, s:s + m, :] = k.transpose(1, 0, 2)
+            cache.v[l][:, s:s + m, :] = v.transpose(1, 0, 2)
+            att = tree_attention(q, cache.k[l][:, :s], cache.v[l][:, :s],
+                                 cache.k[l][:, s:s + m], cache.v[l][:, s:s + m], parent)
+            h = h + att.reshape(m, n_heads * hd) @ np.asarray(w["wo"], np.float64).T
+            x = rmsnorm(h, np.asarray(w["mlp_norm"], np.float64), c.rms_eps)
+            gu = x @ np.asarray(w["w_gate_up"], np.float64).T
+            act = silu(gu[:, :c.d_ff]) * gu[:, c.d_ff:]
+            h = h + act @ np.asarray(w["w_down"], np.float64).T
+        x = rmsnorm(h, np.asarray(self.glob["final_norm"], np.float64), c.rms_eps)
+        return x @ np.asarray(self.glob["lm_head"], np.float64).T
+
+
+def autoregressive_greedy(dec: Decoder, prompt: Sequence[int], n_new: int,
+                          capacity: int = 0) -> List[int]:
+    """Eq. 1 solved first to last: one token per forward, y_t = argmax P(y_t | y_<t, x)."""
+    cache = dec.new_cache(capacity or len(prompt) + n_new + 1)
+    out: List[int] = []
+    nxt = None
+    for t in prompt:
+        logits = dec.forward_rows(cache, [int(t)], [-1])
+        cache.seq_len += 1
+        nxt = int(node_argmax(logits)[0])
+    for _ in range(n_new):
+        out.append(nxt)
+        logits = dec.forward_rows(cache, [nxt], [-1])
+        cache.seq_len += 1
+        nxt = int(node_argmax(logits)[0])
+    return out
+
+
+def verify_step(dec: Decoder, cache: KVCache, tokens, parent):
+    """One TR-Jacobi verification step (Section 3.3): forward, arg-max, acceptance, compaction.
+
+    Returns a dict with the logits, the per-row prediction, k, path and bonus;
+    the cache afterwards holds seq_len + k + 1 committed rows.
+    """
+    s = cache.seq_len
+    logits = dec.forward_rows(cache, tokens, parent)
+    pred = node_argmax(logits)
+    k, path, bonus = accept_path(tokens, parent, pred)
+    compact_rows(cache.k, s, path)
+    cache.seq_len = compact_rows(cache.v, s, path)
+    return {"logits": logits, "pred": pred, "k": k, "path": path, "bonus": bonus, "prefix": s}
+
+
+def tr_jacobi_generate(dec: Decoder, prompt: Sequence[int], n_new: int, width: int,
+                       n_branches: int, branch_len: int,
+                       draw_fn: Callable[[int, int], Sequence[int]],
+                       capacity: int = 0, trace: List[dict] = None) -> List[int]:
+    """Greedy TR-Jacobi decoding (Section 3.3).
+
+    The prompt is scored once (a chain tree over an empty cache), which yields
+    the first committed token.  Every further step builds a tree from the
+    current Jacobi window and the retrieved branches, verifies it in one
+    forward and commits k + 1 tokens.  ``draw_fn(step, n)`` supplies the raw
+    random integers behind ahead noise: step 0 seeds the first window; step
+    t >= 1 uses slots [0, width) for the window refill after that step and
+    slots [width, width + n_branches * branch_len) for that step's retrieval.
+    When ``trace`` is a list, one record per step is appended to it.
+    """
+    n_tree = 1 + width + n_branches * branch_len
+    cache = dec.new_cache(capacity or len(prompt) + n_new + n_tree + 1)
+    p = len(prompt)
+    logits = dec.forward_rows(cache, list(prompt), list(range(-1, p - 1)))
+    cache.seq_len = p
+    committed = [int(t) for t in prompt] + [int(node_argmax(logits[-1:])[0])]
+    d0 = draw_fn(0, width)
+    window = [ahead_noise(committed, d0[i]) for i in range(width)]
+    step = 0
+    while len(committed) - p < n_new:
+        step += 1
+        draws = draw_fn(step, width + n_branches * branch_len)
+        branches = retrieve(committed, n_branches, branch_len, draws[width:])
+        tokens, parent = build_tree(committed[-1], window, branches)
+        rec = verify_step(dec, cache, tokens, parent)
+        committed += [int(tokens[r]) for r in rec["path"][1:]] + [rec["bonus"]]
+        window = refill_window(parent, rec["pred"], rec["path"][-1], width, committed, draws[:width])
+        if trace is not None:
+            rec.update(tokens=tokens, parent=parent, step=step, next_window=list(window))
+            trace.append(rec)
+    return committed[p:p + n_new]
