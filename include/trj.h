@@ -1,0 +1,270 @@
+/*
+ * trj.h -- C ABI of the TR-Jacobi verification step on one B200 (sm_100a).
+ *
+ * One verification step of tree-based retrieval-augmented Jacobi decoding
+ * (paper Section 3.3): a token tree that merges the Jacobi window with
+ * retrieved draft branches is scored by ONE model forward against the KV cache
+ * (token-tree verification, Section 2.2 / Appendix B), the greedy longest
+ * accepted root-to-leaf path is chosen (Section 3.3, Eq. 1) and the K/V of the
+ * accepted rows is kept contiguous in the cache.
+ *
+ * Conventions that hold for every entry point
+ * -------------------------------------------
+ * Pointers   "dev" pointers are CUDA device addresses of the current device,
+ *            "host" pointers are ordinary host addresses.  The caller allocates
+ *            and owns every buffer; the library borrows it for the duration of
+ *            the call (weights and workspace: for the lifetime of the context)
+ *            and frees nothing it did not allocate.  The library allocates no
+ *            device memory: all scratch comes from caller-provided workspaces.
+ * Streams    `stream` is a cudaStream_t passed as void* (NULL = default
+ *            stream).  Device entry points only enqueue work; results are in
+ *            device memory once the stream has been synchronised.  Entry
+ *            points whose name ends in _host copy to and from host buffers and
+ *            synchronise the stream before returning.
+ * Errors     Every function returns a trj_status.  Shapes, capacities and
+ *            pointers are checked on the host before anything is launched, so
+ *            an invalid call launches nothing.  Nothing aborts, throws or
+ *            prints.  trj_last_error gives a message for the calling thread's
+ *            most recent failure.
+ * Layouts    All tensors are dense, row-major, innermost dimension last.
+ *            dtype is TRJ_BF16 (bf16 storage, fp32 accumulation) or TRJ_F32.
+ *            KV cache: [L][B][H][max_seq][D]; sequence b has seq_len[b]
+ *            committed rows; during a step the M_b tree rows of sequence b
+ *            live at cache rows seq_len[b] .. seq_len[b] + M_b - 1.
+ * Trees      A tree is a parent-pointer array in topological order:
+ *            parent[0] = -1 (row 0 is the root = the last committed token,
+ *            whose K/V is not cached yet) and 0 <= parent[i] < i.  depth[i] is
+ *            the number of edges from the root.  anc is the ancestor-or-self
+ *            bitmask: bit (j % 64) of word anc[i * anc_words + j / 64] is set
+ *            iff row j is row i or one of its ancestors.  A batch of trees is
+ *            ragged: rows of sequence b are row_off[b] .. row_off[b+1] - 1 and
+ *            parent / anc bit indices are local to the sequence.
+ * Limits     At most TRJ_MAX_ROWS rows per tree, TRJ_MAX_BATCH sequences.
+ */
+#ifndef TRJ_H
+#define TRJ_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define TRJ_MAX_ROWS  128      /* tree rows per sequence, root included          */
+#define TRJ_MAX_BATCH 64       /* sequences per call                             */
+#define TRJ_PATH_STRIDE 128    /* int32 slots per sequence in `path` arrays      */
+
+typedef enum {
+    TRJ_OK = 0,
+    TRJ_EINVAL = 1,        /* bad pointer, shape, tree or enum                   */
+    TRJ_ECAPACITY = 2,     /* rows, batch, sequence length or workspace too small */
+    TRJ_ECUDA = 3,         /* a CUDA runtime call failed                          */
+    TRJ_ETIMEOUT = 4,      /* a bounded device-side wait expired                  */
+    TRJ_EUNSUPPORTED = 5   /* valid request that this build has no kernel for     */
+} trj_status;
+
+typedef enum { TRJ_F32 = 0, TRJ_BF16 = 1 } trj_dtype;
+
+typedef struct trj_ctx trj_ctx;    /* opaque model context */
+
+/* LLaMA-family decoder shape: pre-norm, RMSNorm, rotary embedding (half-split
+ * pairing, base rope_theta), multi-head attention, SwiGLU, untied LM head. */
+typedef struct {
+    int32_t n_layers, d_model, n_heads, head_dim, d_ff, vocab;
+    float   rms_eps, rope_theta;
+    int32_t dtype;                 /* trj_dtype of weights, activations and cache */
+    int32_t max_batch, max_seq, max_rows;   /* capacities the workspace is sized for */
+} trj_model_cfg;
+
+/* Device pointers to the weights, borrowed for the lifetime of the context.
+ * Every matrix is [d_out][d_in].  The per-layer members are HOST arrays of
+ * n_layers device pointers.  wqkv stacks Wq, Wk, Wv rows; w_gate_up stacks the
+ * SwiGLU gate rows over the up rows.  Norm gains are fp32 vectors [d_model]. */
+typedef struct {
+    const void*  embed;            /* [vocab][d_model]  dtype                     */
+    const void*  lm_head;          /* [vocab][d_model]  dtype                     */
+    const float* final_norm;       /* [d_model]                                   */
+    const float* const* attn_norm; /* [L] -> [d_model]                            */
+    const void*  const* wqkv;      /* [L] -> [3*H*D][d_model]                     */
+    const void*  const* wo;        /* [L] -> [d_model][H*D]                       */
+    const float* const* mlp_norm;  /* [L] -> [d_model]                            */
+    const void*  const* w_gate_up; /* [L] -> [2*d_ff][d_model]                    */
+    const void*  const* w_down;    /* [L] -> [d_model][d_ff]                      */
+} trj_weights;
+
+const char* trj_last_error(void);
+/* Library version string; also a cheap "does it load" probe. */
+const char* trj_version(void);
+
+/* ------------------------------------------------------------------------
+ * build_tree (host, integers only).  Section 3.3: every path of the tree is an
+ * ordinary Jacobi trajectory and retrieved drafts get a path of their own;
+ * Appendix B: the tree is verified through a sparse attention mask.
+ *
+ * Lays out row 0 = root, rows 1..W = the Jacobi window as a chain, then each of
+ * the R retrieved branches (branch r = branches[r*branch_len .. +branch_len))
+ * as a chain hanging off the root.  Writes tokens/parent/depth [M] and
+ * anc [M * anc_words] (anc_words >= ceil(M/64)), M = 1 + W + R*branch_len, and
+ * *n_rows = M.  All pointers host.  TRJ_ECAPACITY if M > max_rows or
+ * max_rows > TRJ_MAX_ROWS; TRJ_EINVAL on NULL or negative sizes. */
+trj_status trj_build_tree(int32_t root, const int32_t* window, int32_t W,
+                          const int32_t* branches, int32_t R, int32_t branch_len,
+                          int32_t max_rows, int32_t anc_words,
+                          int32_t* tokens, int32_t* parent, int32_t* depth,
+                          uint64_t* anc, int32_t* n_rows);
+
+/* Same derivation for an arbitrary tree given by parent pointers (host):
+ * validates parent (TRJ_EINVAL if parent[0] != -1 or parent[i] is not an
+ * earlier row; TRJ_ECAPACITY if M > TRJ_MAX_ROWS or anc_words < ceil(M/64))
+ * and writes depth [M] and anc [M * anc_words]. */
+trj_status trj_tree_from_parents(const int32_t* parent, int32_t M, int32_t anc_words,
+                                 int32_t* depth, uint64_t* anc);
+
+/* Prompt-lookup retrieval (Section 3.3, host).  Key = last 2 tokens of
+ * context[0..n) (which ends with the root), then the last 1; scanning
+ * backwards, the branch_len tokens after each of the R most recent earlier
+ * occurrences become a branch; a slot retrieval cannot fill holds ahead noise
+ * (Eq. 4) context[draws[r*branch_len + j] % n].  Writes branches [R*branch_len]. */
+trj_status trj_retrieve(const int32_t* context, int32_t n, int32_t R, int32_t branch_len,
+                        const int64_t* draws, int32_t* branches);
+
+/* Next Jacobi window (Section 3.3, host): the predictions below the winning row
+ * `best` along its branch (lowest-index child at every level), then ahead noise
+ * context[draws[i] % n] for the remaining slots i < W.  Writes window [W]. */
+trj_status trj_refill_window(const int32_t* parent, const int32_t* node_argmax, int32_t M,
+                             int32_t best, int32_t W, const int32_t* context, int32_t n,
+                             const int64_t* draws, int32_t* window);
+
+/* ------------------------------------------------------------------------
+ * Tree-masked attention (Section 2.2, Appendix B), batched and ragged.
+ *
+ *   out[r][h] = sum_j softmax_j( q[r][h] . K[b][h][j] / sqrt(D) ) V[b][h][j]
+ *
+ * for row r of sequence b (local index i = r - row_off[b]), j ranging over the
+ * cache rows 0 .. seq_len[b]-1 and those tree rows seq_len[b] + t whose bit t is
+ * set in anc[r].
+ *   q, out     dev [rows_total][H][D]   dtype
+ *   k_cache,
+ *   v_cache    dev [B][H][max_seq][D]   dtype (tree rows already stored in place)
+ *   seq_len    dev [B] int32;  row_off dev [B+1] int32;  anc dev [rows_total][anc_words]
+ *   max_rows   upper bound of rows per sequence (<= TRJ_MAX_ROWS)
+ *   max_len    upper bound of seq_len[b] + rows of b, <= max_seq (sizes the KV split)
+ *   workspace  dev, at least trj_tree_attention_workspace(...) bytes, 256-byte aligned;
+ *              holds split-KV partial results, contents undefined afterwards.
+ * TRJ_EUNSUPPORTED for a head_dim the build has no kernel for (supported: 64, 128). */
+size_t trj_tree_attention_workspace(int32_t rows_total, int32_t B, int32_t H, int32_t D, int32_t max_len);
+trj_status trj_tree_attention(const void* q, const void* k_cache, const void* v_cache,
+                              const int32_t* seq_len, const int32_t* row_off, const uint64_t* anc,
+                              int32_t anc_words, int32_t B, int32_t rows_total, int32_t max_rows,
+                              int32_t H, int32_t D, int32_t max_seq, int32_t max_len, int32_t dtype,
+                              void* out, void* workspace, size_t workspace_bytes, void* stream);
+
+/* ------------------------------------------------------------------------
+ * Per-node arg-max fused with greedy longest-path acceptance (Eq. 1; Section
+ * 3.3: candidate generation and verification share the forward, so every row's
+ * prediction is an output).
+ *
+ *   node_argmax[r] = argmax_v logits[r][v]           (ties -> smallest v)
+ *   ok[0] = 1;  ok[i] = ok[parent[i]] && tokens[i] == node_argmax[parent[i]]
+ *   best  = accepted row of largest depth (ties -> smallest row);  k = depth[best]
+ *   path  = rows root..best (k+1 entries, local indices, rest -1);  bonus = node_argmax[best]
+ *
+ *   logits     dev [rows_total][V] dtype;  tokens/parent/depth dev [rows_total] int32
+ *   node_argmax dev [rows_total];  margin dev [rows_total] fp32 or NULL (top-1 minus top-2 logit)
+ *   k_acc, bonus dev [B];  path dev [B][TRJ_PATH_STRIDE]
+ *   workspace  dev, >= trj_argmax_accept_workspace(rows_total, B) bytes, 256-byte aligned.
+ *              The library keeps tickets in it that must be zero on entry of the
+ *              FIRST call; every call leaves them zero again.
+ * Inputs must be finite. */
+size_t trj_argmax_accept_workspace(int32_t rows_total, int32_t B);
+trj_status trj_argmax_accept(const void* logits, int32_t dtype, int32_t V,
+                             const int32_t* tokens, const int32_t* parent, const int32_t* depth,
+                             const int32_t* row_off, int32_t B, int32_t rows_total,
+                             int32_t* node_argmax, float* margin,
+                             int32_t* k_acc, int32_t* path, int32_t* bonus,
+                             void* workspace, size_t workspace_bytes, void* stream);
+
+/* ------------------------------------------------------------------------
+ * KV compaction of the accepted path (implied by Section 3.3: decoding
+ * continues from the accepted tokens).  For every layer, head and both K and
+ * V, row seq_len[b] + path[b][j] moves to row seq_len[b] + j, j = 1..k_acc[b]
+ * (row 0, the root, is already in place); then seq_len[b] += k_acc[b] + 1.
+ * Bit-exact copy; source and destination ranges may overlap.
+ *   k_cache, v_cache  dev [L][B][H][max_seq][D] dtype, modified in place
+ *   seq_len dev [B] (updated);  k_acc dev [B];  path dev [B][TRJ_PATH_STRIDE] */
+trj_status trj_compact_rows(void* k_cache, void* v_cache, int32_t L, int32_t B, int32_t H,
+                            int32_t max_seq, int32_t D, int32_t dtype, int32_t* seq_len,
+                            const int32_t* k_acc, const int32_t* path, void* stream);
+
+/* ------------------------------------------------------------------------
+ * Model context: the whole verification step of a LLaMA-shaped decoder.
+ * workspace: dev, >= trj_workspace_bytes(cfg), 256-byte aligned, zero-filled by
+ * the caller before trj_create, owned by the caller, used by every call on ctx.
+ * The cache passed to the calls below is [n_layers][max_batch][H][max_seq][D]. */
+size_t     trj_workspace_bytes(const trj_model_cfg* cfg);
+trj_status trj_create(const trj_model_cfg* cfg, const trj_weights* weights,
+                      void* workspace, size_t workspace_bytes, trj_ctx** out);
+trj_status trj_destroy(trj_ctx* ctx);
+
+/* verify_step (Section 3.3): ONE forward of the decoder over all tree rows.
+ * Embeds tokens, runs every layer (RMSNorm, QKV projection, rotary embedding at
+ * position seq_len[b] + depth, K/V of the tree rows written to cache rows
+ * seq_len[b] + i, tree-masked attention, output projection, SwiGLU MLP), the
+ * final norm and the LM head, and writes node_argmax [rows_total] (Eq. 1),
+ * margin [rows_total] when not NULL and, when logits is not NULL, the fp32
+ * logits [rows_total][vocab].  seq_len is not changed.  All pointers dev.
+ * B <= cfg.max_batch, rows per sequence <= cfg.max_rows and seq_len[b] + rows
+ * <= max_len <= cfg.max_seq must hold (the caller's contract for device-held
+ * lengths; max_len is the host-known bound used for launch sizing). */
+trj_status trj_verify_step(trj_ctx* ctx, void* k_cache, void* v_cache, const int32_t* seq_len,
+                           const int32_t* tokens, const int32_t* parent, const int32_t* depth,
+                           const uint64_t* anc, int32_t anc_words, const int32_t* row_off,
+                           int32_t B, int32_t rows_total, int32_t max_rows, int32_t max_len,
+                           int32_t* node_argmax, float* margin, float* logits, void* stream);
+
+/* accept (Section 3.3): longest accepted path from node_argmax; see
+ * trj_argmax_accept for the rule and the output layout.  All pointers dev. */
+trj_status trj_accept(trj_ctx* ctx, const int32_t* tokens, const int32_t* parent, const int32_t* depth,
+                      const int32_t* row_off, int32_t B, int32_t rows_total, const int32_t* node_argmax,
+                      int32_t* k_acc, int32_t* path, int32_t* bonus, void* stream);
+
+/* compact_kv: trj_compact_rows over all layers of the context's cache shape. */
+trj_status trj_compact_kv(trj_ctx* ctx, void* k_cache, void* v_cache, int32_t* seq_len, int32_t B,
+                          const int32_t* k_acc, const int32_t* path, void* stream);
+
+/* Prefill of sequence b: scores n prompt tokens (dev int32) as chain trees of at
+ * most cfg.max_rows rows (a chain tree is causal attention), appends their K/V
+ * at seq_len[b] and advances seq_len[b] by n; *first_token (dev) receives the
+ * greedy prediction after the last prompt token (Eq. 1). */
+trj_status trj_prefill(trj_ctx* ctx, void* k_cache, void* v_cache, int32_t* seq_len, int32_t b,
+                       const int32_t* tokens, int32_t n, int32_t* first_token, void* stream);
+
+/* One whole decode step from HOST buffers for batch 1 (the call a decoding loop
+ * makes): builds the tree from root/window/branches (trj_build_tree), copies it
+ * to the device, runs verify_step + accept + compact_kv, copies the result back
+ * and synchronises `stream`.
+ *   host in : root, window [W], branches [R*branch_len]
+ *   host out: tokens/parent [M] (the tree that was scored), node_argmax [M],
+ *             *k_acc, path [TRJ_PATH_STRIDE], *bonus, *n_rows
+ *   dev     : k_cache, v_cache, seq_len [1] (advanced by k_acc + 1)
+ *   max_len : host-known bound of seq_len[0] + M */
+trj_status trj_step_host(trj_ctx* ctx, void* k_cache, void* v_cache, int32_t* seq_len, int32_t max_len,
+                         int32_t root, const int32_t* window, int32_t W,
+                         const int32_t* branches, int32_t R, int32_t branch_len,
+                         int32_t* tokens, int32_t* parent, int32_t* n_rows, int32_t* node_argmax,
+                         int32_t* k_acc, int32_t* path, int32_t* bonus, void* stream);
+
+/* ------------------------------------------------------------------------
+ * The projections as a stand-alone op: y[M][N] (fp32) = x[M][K] . w[N][K]^T,
+ * x and w of `dtype`, all dev.  Used by the model path for every projection
+ * and exposed for measurement.  workspace: dev, >= trj_gemm_workspace(M, N, K)
+ * bytes, 256-byte aligned (split-K partial sums). */
+size_t     trj_gemm_workspace(int32_t M, int32_t N, int32_t K);
+trj_status trj_gemm(const void* x, const void* w, float* y, int32_t M, int32_t N, int32_t K,
+                    int32_t dtype, void* workspace, size_t workspace_bytes, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* TRJ_H */
