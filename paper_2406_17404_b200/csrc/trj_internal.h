@@ -1,0 +1,75 @@
+// Internal declarations shared by the translation units of libtrj (not part of the ABI).
+#pragma once
+#include <cuda_runtime.h>
+#include <cuda_bf16.h>
+#include <stdint.h>
+#include <stddef.h>
+#include "trj.h"
+
+namespace trj {
+
+// ---- error plumbing (thread-local message, never throws) -------------------
+trj_status fail(trj_status code, const char* fmt, ...);
+#define TRJ_CHECK_CUDA(expr)                                                        \
+    do {                                                                            \
+        cudaError_t e__ = (expr);                                                   \
+        if (e__ != cudaSuccess)                                                     \
+            return ::trj::fail(TRJ_ECUDA, "%s: %s", #expr, cudaGetErrorString(e__)); \
+    } while (0)
+#define TRJ_REQUIRE(cond, code, ...)                         \
+    do {                                                     \
+        if (!(cond)) return ::trj::fail(code, __VA_ARGS__);  \
+    } while (0)
+
+inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+inline size_t dtype_size(int32_t dt) { return dt == TRJ_BF16 ? 2 : 4; }
+
+// ---- host-side tree helpers (host_tree.cpp) ---------------------------------
+trj_status tree_from_parents_impl(const int32_t* parent, int32_t M, int32_t anc_words,
+                                  int32_t* depth, uint64_t* anc);
+
+// ---- generic kernels (kernels_generic.cu); every launcher only enqueues ------
+// Geometry of a ragged batch of trees over a KV cache slab of one layer.
+struct Batch {
+    const int32_t* seq_len;   // [B] dev
+    const int32_t* row_off;   // [B+1] dev
+    int32_t B, rows_total, max_rows, max_len;
+};
+
+cudaError_t launch_embed(const void* embed, int32_t dtype, const int32_t* tokens, float* h,
+                         int32_t rows, int32_t d, cudaStream_t st);
+// h += add (when add != nullptr, h is updated in place); x = rmsnorm(h) * gain, stored as dtype.
+cudaError_t launch_add_rmsnorm(float* h, const float* add, const float* gain, void* x, int32_t dtype,
+                               int32_t rows, int32_t d, float eps, cudaStream_t st);
+// y[M][N] fp32 = x[M][K] . w[N][K]^T, plain shared-memory tiled FMA kernel.
+cudaError_t launch_gemm_simt(const void* x, const void* w, float* y, int32_t M, int32_t N, int32_t K,
+                             int32_t dtype, cudaStream_t st);
+// Rotary embedding of q and k at position seq_len[b] + depth[row]; q -> q_out [rows][H][D];
+// k, v -> cache rows seq_len[b] + local row of the layer slab [B][H][max_seq][D].
+cudaError_t launch_rope_kv_write(const float* qkv, const double* inv_freq, const int32_t* depth,
+                                 const Batch& bt, void* q_out, void* k_slab, void* v_slab, int32_t dtype,
+                                 int32_t H, int32_t D, int32_t max_seq, cudaStream_t st);
+cudaError_t launch_tree_attention_generic(const void* q, const void* k_slab, const void* v_slab,
+                                          const uint64_t* anc, int32_t anc_words, const Batch& bt,
+                                          int32_t H, int32_t D, int32_t max_seq, int32_t dtype,
+                                          void* out, cudaStream_t st);
+// act[M][f] (dtype) = silu(gu[:, :f]) * gu[:, f:]
+cudaError_t launch_swiglu(const float* gu, void* act, int32_t dtype, int32_t rows, int32_t f, cudaStream_t st);
+
+// Arg-max over the vocabulary and/or acceptance.  do_argmax: compute node_argmax (+margin) from
+// logits; do_accept: walk the tree and write k_acc/path/bonus.  ws: tickets + partials.
+size_t argmax_workspace_bytes(int32_t rows_total, int32_t B);
+cudaError_t launch_argmax_accept(const void* logits, int32_t dtype, int32_t V,
+                                 const int32_t* tokens, const int32_t* parent, const int32_t* depth,
+                                 const int32_t* row_off, int32_t B, int32_t rows_total,
+                                 int32_t* node_argmax, float* margin, int32_t* k_acc, int32_t* path,
+                                 int32_t* bonus, bool do_argmax, bool do_accept, void* ws, cudaStream_t st);
+
+cudaError_t launch_compact(void* k_cache, void* v_cache, int32_t L, int32_t B_cache, int32_t B, int32_t H,
+                           int32_t max_seq, int32_t D, int32_t dtype, int32_t* seq_len,
+                           const int32_t* k_acc, const int32_t* path, cudaStream_t st);
+// row_off = {0, m} and seq_len[b] += delta: small bookkeeping used by prefill.
+cudaError_t launch_set_chunk(int32_t* row_off2, int32_t m, cudaStream_t st);
+cudaError_t launch_bump_len(int32_t* seq_len_b, int32_t delta, cudaStream_t st);
+
+}  // namespace trj
