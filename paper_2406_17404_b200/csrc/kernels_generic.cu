@@ -1,0 +1,477 @@
+// Shape-generic kernels of the verification step (fp32 or bf16 storage, fp32 arithmetic).
+// They serve every shape the specialised sm_100a kernels do not cover (fp32 models, odd head
+// sizes) and all the small element-wise steps between the projections.
+#include "trj_internal.h"
+
+namespace trj {
+namespace {
+
+template <typename T> __device__ __forceinline__ float to_f(T v);
+template <> __device__ __forceinline__ float to_f<float>(float v) { return v; }
+template <> __device__ __forceinline__ float to_f<__nv_bfloat16>(__nv_bfloat16 v) { return __bfloat162float(v); }
+template <typename T> __device__ __forceinline__ T from_f(float v);
+template <> __device__ __forceinline__ float from_f<float>(float v) { return v; }
+template <> __device__ __forceinline__ __nv_bfloat16 from_f<__nv_bfloat16>(float v) { return __float2bfloat16_rn(v); }
+
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    return v;
+}
+__device__ __forceinline__ float warp_max(float v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
+    return v;
+}
+
+// Sequence that owns a global row (B is small: linear scan of the offsets).
+__device__ __forceinline__ int seq_of_row(const int32_t* row_off, int B, int row) {
+    int b = 0;
+    while (b + 1 < B && row >= row_off[b + 1]) ++b;
+    return b;
+}
+
+// ---------------------------------------------------------------- embedding
+template <typename T>
+__global__ void embed_kernel(const T* __restrict__ embed, const int32_t* __restrict__ tokens,
+                             float* __restrict__ h, int d) {
+    const int row = blockIdx.x;
+    const T* src = embed + (size_t)tokens[row] * d;
+    for (int c = threadIdx.x; c < d; c += blockDim.x) h[(size_t)row * d + c] = to_f(src[c]);
+}
+
+// ---------------------------------------------------------------- residual add + RMSNorm
+template <typename T>
+__global__ void add_rmsnorm_kernel(float* __restrict__ h, const float* __restrict__ add,
+                                   const float* __restrict__ gain, T* __restrict__ x, int d, float eps) {
+    __shared__ float red[32];
+    const int row = blockIdx.x;
+    float* hr = h + (size_t)row * d;
+    float ss = 0.f;
+    for (int c = threadIdx.x; c < d; c += blockDim.x) {
+        float v = hr[c];
+        if (add) { v += add[(size_t)row * d + c]; hr[c] = v; }
+        ss += v * v;
+    }
+    ss = warp_sum(ss);
+    if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = ss;
+    __syncthreads();
+    if (threadIdx.x < 32) {
+        float t = threadIdx.x < (blockDim.x >> 5) ? red[threadIdx.x] : 0.f;
+        t = warp_sum(t);
+        if (threadIdx.x == 0) red[0] = t;
+    }
+    __syncthreads();
+    const float inv = rsqrtf(red[0] / (float)d + eps);
+    for (int c = threadIdx.x; c < d; c += blockDim.x) x[(size_t)row * d + c] = from_f<T>(hr[c] * inv * gain[c]);
+}
+
+// ---------------------------------------------------------------- plain tiled GEMM
+// y[M][N] = x[M][K] . w[N][K]^T ; 64x64 tile, 16-deep slices, 4x4 outputs per thread.
+template <typename T>
+__global__ void __launch_bounds__(256) gemm_simt_kernel(const T* __restrict__ x, const T* __restrict__ w,
+                                                        float* __restrict__ y, int M, int N, int K) {
+    constexpr int BM = 64, BN = 64, BK = 16;
+    __shared__ float xs[BK][BM + 4];
+    __shared__ float ws[BK][BN + 4];
+    const int m0 = blockIdx.y * BM, n0 = blockIdx.x * BN;
+    const int tid = threadIdx.x, ty = tid >> 4, tx = tid & 15;
+    const int lr = tid >> 2, lk = (tid & 3) * 4;          // this thread stages row lr, k-slice lk..lk+3
+    float acc[4][4] = {};
+    for (int k0 = 0; k0 < K; k0 += BK) {
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const int k = k0 + lk + i;
+            const int xm = m0 + lr, wn = n0 + lr;
+            xs[lk + i][lr] = (xm < M && k < K) ? to_f(x[(size_t)xm * K + k]) : 0.f;
+            ws[lk + i][lr] = (wn < N && k < K) ? to_f(w[(size_t)wn * K + k]) : 0.f;
+        }
+        __syncthreads();
+#pragma unroll
+        for (int kk = 0; kk < BK; ++kk) {
+            float a[4], b[4];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) { a[i] = xs[kk][ty * 4 + i]; b[i] = ws[kk][tx * 4 + i]; }
+#pragma unroll
+            for (int i = 0; i < 4; ++i)
+#pragma unroll
+                for (int j = 0; j < 4; ++j) acc[i][j] = fmaf(a[i], b[j], acc[i][j]);
+        }
+        __syncthreads();
+    }
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const int m = m0 + ty * 4 + i;
+        if (m >= M) continue;
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const int n = n0 + tx * 4 + j;
+            if (n < N) y[(size_t)m * N + n] = acc[i][j];
+        }
+    }
+}
+
+// ---------------------------------------------------------------- rotary embedding + K/V append
+template <typename T>
+__global__ void rope_kv_write_kernel(const float* __restrict__ qkv, const double* __restrict__ inv_freq,
+                                     const int32_t* __restrict__ depth, const int32_t* __restrict__ seq_len,
+                                     const int32_t* __restrict__ row_off, int B, T* __restrict__ q_out,
+                                     T* __restrict__ k_slab, T* __restrict__ v_slab, int H, int D, int max_seq) {
+    const int row = blockIdx.x, hh = blockIdx.y;
+    const int b = seq_of_row(row_off, B, row);
+    const int local = row - row_off[b];
+    const int pos = seq_len[b] + depth[row];
+    const int half = D >> 1, HD = H * D;
+    const float* src = qkv + (size_t)row * 3 * HD + hh * D;
+    const size_t cache_row = (((size_t)b * H + hh) * max_seq + seq_len[b] + local) * D;
+    for (int i = threadIdx.x; i < half; i += blockDim.x) {
+        double s, c;
+        sincos((double)pos * inv_freq[i], &s, &c);
+        const float cs = (float)c, sn = (float)s;
+        const float qa = src[i], qb = src[i + half];
+        q_out[(size_t)row * HD + hh * D + i] = from_f<T>(qa * cs - qb * sn);
+        q_out[(size_t)row * HD + hh * D + i + half] = from_f<T>(qb * cs + qa * sn);
+        const float ka = src[HD + i], kb = src[HD + i + half];
+        k_slab[cache_row + i] = from_f<T>(ka * cs - kb * sn);
+        k_slab[cache_row + i + half] = from_f<T>(kb * cs + ka * sn);
+        v_slab[cache_row + i] = from_f<T>(src[2 * HD + i]);
+        v_slab[cache_row + i + half] = from_f<T>(src[2 * HD + i + half]);
+    }
+}
+
+// ---------------------------------------------------------------- tree attention, one CTA per (row, head)
+// 4 warps split the keys; inside a warp every lane scores one key of a 32-key chunk, the chunk's
+// statistics are merged with an online softmax, and P.V is accumulated with lanes spread over D.
+template <typename T, int D>
+__global__ void __launch_bounds__(128) tree_attention_generic_kernel(
+        const T* __restrict__ q, const T* __restrict__ k_slab, const T* __restrict__ v_slab,
+        const uint64_t* __restrict__ anc, int anc_words, const int32_t* __restrict__ seq_len,
+        const int32_t* __restrict__ row_off, int B, int H, int max_seq, T* __restrict__ out) {
+    constexpr int PER = D / 32;                  // output dims per lane
+    __shared__ float qs[D];
+    __shared__ float part_m[4], part_l[4];
+    __shared__ float part_acc[4][D];
+    const int row = blockIdx.x, hh = blockIdx.y;
+    const int b = seq_of_row(row_off, B, row);
+    const int S = seq_len[b];
+    const int rows_b = row_off[b + 1] - row_off[b];
+    const int total = S + rows_b;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const T* kb = k_slab + ((size_t)b * H + hh) * max_seq * D;
+    const T* vb = v_slab + ((size_t)b * H + hh) * max_seq * D;
+    const uint64_t* mask = anc + (size_t)row * anc_words;
+    for (int c = threadIdx.x; c < D; c += blockDim.x) qs[c] = to_f(q[((size_t)row * H + hh) * D + c]);
+    __syncthreads();
+    const float scale = rsqrtf((float)D);
+    float m_run = -INFINITY, l_run = 0.f, acc[PER];
+#pragma unroll
+    for (int i = 0; i < PER; ++i) acc[i] = 0.f;
+    for (int base = warp * 32; base < total; base += 128) {
+        const int j = base + lane;
+        bool vis = j < total;
+        if (vis && j >= S) { const int t = j - S; vis = (mask[t >> 6] >> (t & 63)) & 1ull; }
+        float s = -INFINITY;
+        if (vis) {
+            const T* kr = kb + (size_t)j * D;
+            float dot = 0.f;
+#pragma unroll 8
+            for (int c = 0; c < D; ++c) dot = fmaf(qs[c], to_f(kr[c]), dot);
+            s = dot * scale;
+        }
+        const float cmax = warp_max(s);
+        if (cmax == -INFINITY) continue;          // whole chunk masked (warp-uniform)
+        const float m_new = fmaxf(m_run, cmax);
+        const float corr = (m_run == -INFINITY) ? 0.f : expf(m_run - m_new);
+        const float p = vis ? expf(s - m_new) : 0.f;
+        l_run = l_run * corr + warp_sum(p);
+#pragma unroll
+        for (int i = 0; i < PER; ++i) acc[i] *= corr;
+        const int nk = min(32, total - base);
+        for (int jj = 0; jj < nk; ++jj) {
+            const float pj = __shfl_sync(0xffffffffu, p, jj);
+            if (pj == 0.f) continue;              // warp-uniform
+            const T* vr = vb + (size_t)(base + jj) * D + lane * PER;
+#pragma unroll
+            for (int i = 0; i < PER; ++i) acc[i] = fmaf(pj, to_f(vr[i]), acc[i]);
+        }
+        m_run = m_new;
+    }
+    if (lane == 0) { part_m[warp] = m_run; part_l[warp] = l_run; }
+#pragma unroll
+    for (int i = 0; i < PER; ++i) part_acc[warp][lane * PER + i] = acc[i];
+    __syncthreads();
+    const float m_all = fmaxf(fmaxf(part_m[0], part_m[1]), fmaxf(part_m[2], part_m[3]));
+    for (int c = threadIdx.x; c < D; c += blockDim.x) {
+        float l = 0.f, o = 0.f;
+#pragma unroll
+        for (int w = 0; w < 4; ++w) {
+            const float f = (part_m[w] == -INFINITY) ? 0.f : expf(part_m[w] - m_all);
+            l += part_l[w] * f;
+            o += part_acc[w][c] * f;
+        }
+        out[((size_t)row * H + hh) * D + c] = from_f<T>(o / l);
+    }
+}
+
+// ---------------------------------------------------------------- SwiGLU
+template <typename T>
+__global__ void swiglu_kernel(const float* __restrict__ gu, T* __restrict__ act, int rows, int f) {
+    const size_t n = (size_t)rows * f;
+    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x) {
+        const size_t r = i / f, c = i % f;
+        const float g = gu[r * 2 * f + c], u = gu[r * 2 * f + f + c];
+        act[i] = from_f<T>(g / (1.f + expf(-g)) * u);
+    }
+}
+
+// ---------------------------------------------------------------- arg-max + acceptance
+// Candidate of a (partial) row scan: best value/index and the runner-up value.
+struct Top { float v1; int i1; float v2; };
+__device__ __forceinline__ Top top_merge(const Top& a, const Top& b) {
+    const bool a_wins = (a.v1 > b.v1) || (a.v1 == b.v1 && a.i1 < b.i1);
+    Top r;
+    r.v1 = a_wins ? a.v1 : b.v1;
+    r.i1 = a_wins ? a.i1 : b.i1;
+    r.v2 = fmaxf(a_wins ? b.v1 : a.v1, fmaxf(a.v2, b.v2));
+    return r;
+}
+__device__ __forceinline__ void top_push(Top& t, float v, int i) {
+    if (v > t.v1 || (v == t.v1 && i < t.i1)) { t.v2 = fmaxf(t.v2, t.v1); t.v1 = v; t.i1 = i; }
+    else t.v2 = fmaxf(t.v2, v);
+}
+__device__ __forceinline__ Top top_shfl_xor(const Top& t, int o) {
+    Top r;
+    r.v1 = __shfl_xor_sync(0xffffffffu, t.v1, o);
+    r.i1 = __shfl_xor_sync(0xffffffffu, t.i1, o);
+    r.v2 = __shfl_xor_sync(0xffffffffu, t.v2, o);
+    return r;
+}
+
+constexpr int ARGMAX_THREADS = 256;
+constexpr int ARGMAX_CHUNKS = 4;              // vocabulary slices per row (one CTA each)
+
+// The acceptance walk of one sequence, run by one CTA after every prediction of it is known.
+__device__ void accept_sequence(const int32_t* tokens, const int32_t* parent, const int32_t* depth,
+                                const int32_t* pred, int rows, int32_t* k_acc, int32_t* path, int32_t* bonus) {
+    __shared__ unsigned char ok[TRJ_MAX_ROWS];
+    if (threadIdx.x == 0) {
+        ok[0] = 1;
+        int best = 0, best_depth = 0;
+        for (int i = 1; i < rows; ++i) {
+            const int p = parent[i];
+            const unsigned char o = ok[p] && tokens[i] == pred[p];
+            ok[i] = o;
+            if (o && depth[i] > best_depth) { best = i; best_depth = depth[i]; }
+        }
+        *k_acc = best_depth;
+        *bonus = pred[best];
+        int node = best;
+        for (int j = best_depth; j >= 0; --j) { path[j] = node; node = parent[node]; }
+        for (int j = best_depth + 1; j < TRJ_PATH_STRIDE; ++j) path[j] = -1;
+    }
+}
+
+template <typename T>
+__global__ void __launch_bounds__(ARGMAX_THREADS) argmax_accept_kernel(
+        const T* __restrict__ logits, int V, const int32_t* __restrict__ tokens,
+        const int32_t* __restrict__ parent, const int32_t* __restrict__ depth,
+        const int32_t* __restrict__ row_off, int B, int32_t* node_argmax,
+        float* __restrict__ margin, int32_t* __restrict__ k_acc, int32_t* __restrict__ path,
+        int32_t* __restrict__ bonus, int do_accept, unsigned int* tickets, Top* partial) {
+    __shared__ Top red[ARGMAX_THREADS / 32];
+    __shared__ int last_flag;
+    const int row = blockIdx.x, chunk = blockIdx.y;
+    const int per = (V + ARGMAX_CHUNKS - 1) / ARGMAX_CHUNKS;
+    const int v0 = chunk * per, v1 = min(V, v0 + per);
+    const T* lr = logits + (size_t)row * V;
+    Top t{-INFINITY, 0x7fffffff, -INFINITY};
+    for (int v = v0 + threadIdx.x; v < v1; v += ARGMAX_THREADS) top_push(t, to_f(lr[v]), v);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) t = top_merge(t, top_shfl_xor(t, o));
+    if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = t;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        Top r = red[0];
+        for (int w = 1; w < ARGMAX_THREADS / 32; ++w) r = top_merge(r, red[w]);
+        partial[(size_t)row * ARGMAX_CHUNKS + chunk] = r;
+        __threadfence();
+        const int b = seq_of_row(row_off, B, row);
+        const unsigned int need = (unsigned int)(row_off[b + 1] - row_off[b]) * ARGMAX_CHUNKS;
+        const unsigned int got = atomicAdd(&tickets[b], 1u);
+        last_flag = (got + 1 == need) ? b : -1;
+    }
+    __syncthreads();
+    const int b = last_flag;
+    if (b < 0) return;
+    // this CTA saw the last slice of sequence b: finish its rows, then walk the tree
+    __threadfence();
+    const int r0 = row_off[b], rows = row_off[b + 1] - r0;
+    for (int i = threadIdx.x; i < rows; i += ARGMAX_THREADS) {
+        const volatile Top* pp = partial + (size_t)(r0 + i) * ARGMAX_CHUNKS;
+        Top r{pp[0].v1, pp[0].i1, pp[0].v2};
+        for (int c = 1; c < ARGMAX_CHUNKS; ++c) { Top o{pp[c].v1, pp[c].i1, pp[c].v2}; r = top_merge(r, o); }
+        node_argmax[r0 + i] = r.i1;
+        if (margin) margin[r0 + i] = r.v1 - r.v2;
+    }
+    if (threadIdx.x == 0) tickets[b] = 0;       // ready for the next call
+    __syncthreads();
+    if (do_accept)
+        accept_sequence(tokens + r0, parent + r0, depth + r0, node_argmax + r0, rows,
+                        k_acc + b, path + (size_t)b * TRJ_PATH_STRIDE, bonus + b);
+}
+
+__global__ void accept_only_kernel(const int32_t* __restrict__ tokens, const int32_t* __restrict__ parent,
+                                   const int32_t* __restrict__ depth, const int32_t* __restrict__ row_off,
+                                   const int32_t* __restrict__ node_argmax, int32_t* __restrict__ k_acc,
+                                   int32_t* __restrict__ path, int32_t* __restrict__ bonus) {
+    const int b = blockIdx.x, r0 = row_off[b], rows = row_off[b + 1] - r0;
+    accept_sequence(tokens + r0, parent + r0, depth + r0, node_argmax + r0, rows,
+                    k_acc + b, path + (size_t)b * TRJ_PATH_STRIDE, bonus + b);
+}
+
+// ---------------------------------------------------------------- KV compaction
+// One CTA per (layer, sequence, head, K|V).  Rows are moved in ascending order in batches that are
+// fully loaded before they are stored; since path[j] >= j and the path is strictly increasing, a
+// destination never overwrites a row that a later batch still has to read.
+constexpr int COMPACT_BATCH = 16;
+__global__ void __launch_bounds__(256) compact_kernel(uint4* __restrict__ k_cache, uint4* __restrict__ v_cache,
+                                                      int B_cache, int B, int H, int max_seq, int row_vec,
+                                                      const int32_t* __restrict__ seq_len,
+                                                      const int32_t* __restrict__ k_acc,
+                                                      const int32_t* __restrict__ path) {
+    extern __shared__ uint4 stage[];             // [COMPACT_BATCH][row_vec]
+    int idx = blockIdx.x;
+    const int kv = idx & 1; idx >>= 1;
+    const int hh = idx % H; idx /= H;
+    const int b = idx % B; const int l = idx / B;
+    const int k = k_acc[b];
+    if (k <= 0) return;
+    const int S = seq_len[b];
+    uint4* slab = (kv ? v_cache : k_cache) + (((size_t)l * B_cache + b) * H + hh) * (size_t)max_seq * row_vec;
+    const int32_t* pb = path + (size_t)b * TRJ_PATH_STRIDE;
+    for (int j0 = 1; j0 <= k; j0 += COMPACT_BATCH) {
+        const int nj = min(COMPACT_BATCH, k - j0 + 1);
+        for (int e = threadIdx.x; e < nj * row_vec; e += blockDim.x) {
+            const int j = j0 + e / row_vec, c = e % row_vec;
+            stage[e] = slab[(size_t)(S + pb[j]) * row_vec + c];
+        }
+        __syncthreads();
+        for (int e = threadIdx.x; e < nj * row_vec; e += blockDim.x) {
+            const int j = j0 + e / row_vec, c = e % row_vec;
+            slab[(size_t)(S + j) * row_vec + c] = stage[e];
+        }
+        __syncthreads();
+    }
+}
+
+__global__ void advance_len_kernel(int32_t* seq_len, const int32_t* k_acc, int B) {
+    const int b = blockIdx.x * blockDim.x + threadIdx.x;
+    if (b < B) seq_len[b] += k_acc[b] + 1;
+}
+__global__ void set_chunk_kernel(int32_t* row_off2, int m) { row_off2[0] = 0; row_off2[1] = m; }
+__global__ void bump_len_kernel(int32_t* seq_len_b, int delta) { *seq_len_b += delta; }
+
+}  // namespace
+
+// ============================================================================ launchers
+#define DISPATCH_T(dtype, ...)                                         \
+    if ((dtype) == TRJ_BF16) { using T = __nv_bfloat16; __VA_ARGS__; } \
+    else { using T = float; __VA_ARGS__; }
+
+cudaError_t launch_embed(const void* embed, int32_t dtype, const int32_t* tokens, float* h,
+                         int32_t rows, int32_t d, cudaStream_t st) {
+    DISPATCH_T(dtype, embed_kernel<T><<<rows, 256, 0, st>>>((const T*)embed, tokens, h, d));
+    return cudaGetLastError();
+}
+
+cudaError_t launch_add_rmsnorm(float* h, const float* add, const float* gain, void* x, int32_t dtype,
+                               int32_t rows, int32_t d, float eps, cudaStream_t st) {
+    DISPATCH_T(dtype, add_rmsnorm_kernel<T><<<rows, 256, 0, st>>>(h, add, gain, (T*)x, d, eps));
+    return cudaGetLastError();
+}
+
+cudaError_t launch_gemm_simt(const void* x, const void* w, float* y, int32_t M, int32_t N, int32_t K,
+                             int32_t dtype, cudaStream_t st) {
+    dim3 grid((N + 63) / 64, (M + 63) / 64);
+    DISPATCH_T(dtype, gemm_simt_kernel<T><<<grid, 256, 0, st>>>((const T*)x, (const T*)w, y, M, N, K));
+    return cudaGetLastError();
+}
+
+cudaError_t launch_rope_kv_write(const float* qkv, const double* inv_freq, const int32_t* depth,
+                                 const Batch& bt, void* q_out, void* k_slab, void* v_slab, int32_t dtype,
+                                 int32_t H, int32_t D, int32_t max_seq, cudaStream_t st) {
+    dim3 grid(bt.rows_total, H);
+    DISPATCH_T(dtype, rope_kv_write_kernel<T><<<grid, 64, 0, st>>>(qkv, inv_freq, depth, bt.seq_len, bt.row_off,
+                                                                  bt.B, (T*)q_out, (T*)k_slab, (T*)v_slab, H, D, max_seq));
+    return cudaGetLastError();
+}
+
+cudaError_t launch_tree_attention_generic(const void* q, const void* k_slab, const void* v_slab,
+                                          const uint64_t* anc, int32_t anc_words, const Batch& bt,
+                                          int32_t H, int32_t D, int32_t max_seq, int32_t dtype,
+                                          void* out, cudaStream_t st) {
+    dim3 grid(bt.rows_total, H);
+#define ATT(DD)                                                                                          \
+    DISPATCH_T(dtype, tree_attention_generic_kernel<T, DD><<<grid, 128, 0, st>>>(                        \
+                          (const T*)q, (const T*)k_slab, (const T*)v_slab, anc, anc_words, bt.seq_len,   \
+                          bt.row_off, bt.B, H, max_seq, (T*)out))
+    if (D == 64) { ATT(64); }
+    else if (D == 128) { ATT(128); }
+    else return cudaErrorInvalidValue;
+#undef ATT
+    return cudaGetLastError();
+}
+
+cudaError_t launch_swiglu(const float* gu, void* act, int32_t dtype, int32_t rows, int32_t f, cudaStream_t st) {
+    const size_t n = (size_t)rows * f;
+    const int blocks = (int)((n + 255) / 256 < 1184 ? (n + 255) / 256 : 1184);
+    DISPATCH_T(dtype, swiglu_kernel<T><<<blocks, 256, 0, st>>>(gu, (T*)act, rows, f));
+    return cudaGetLastError();
+}
+
+size_t argmax_workspace_bytes(int32_t rows_total, int32_t B) {
+    (void)B;
+    return align_up(sizeof(unsigned int) * TRJ_MAX_BATCH, 256) + align_up(sizeof(Top) * ARGMAX_CHUNKS * (size_t)rows_total, 256);
+}
+
+cudaError_t launch_argmax_accept(const void* logits, int32_t dtype, int32_t V,
+                                 const int32_t* tokens, const int32_t* parent, const int32_t* depth,
+                                 const int32_t* row_off, int32_t B, int32_t rows_total,
+                                 int32_t* node_argmax, float* margin, int32_t* k_acc, int32_t* path,
+                                 int32_t* bonus, bool do_argmax, bool do_accept, void* ws, cudaStream_t st) {
+    if (do_argmax) {
+        unsigned int* tickets = (unsigned int*)ws;
+        Top* partial = (Top*)((char*)ws + align_up(sizeof(unsigned int) * TRJ_MAX_BATCH, 256));
+        dim3 grid(rows_total, ARGMAX_CHUNKS);
+        DISPATCH_T(dtype, argmax_accept_kernel<T><<<grid, ARGMAX_THREADS, 0, st>>>(
+                              (const T*)logits, V, tokens, parent, depth, row_off, B, node_argmax, margin, k_acc,
+                              path, bonus, do_accept ? 1 : 0, tickets, partial));
+    } else if (do_accept) {
+        accept_only_kernel<<<B, 32, 0, st>>>(tokens, parent, depth, row_off, node_argmax, k_acc, path, bonus);
+    }
+    return cudaGetLastError();
+}
+
+cudaError_t launch_compact(void* k_cache, void* v_cache, int32_t L, int32_t B_cache, int32_t B, int32_t H,
+                           int32_t max_seq, int32_t D, int32_t dtype, int32_t* seq_len,
+                           const int32_t* k_acc, const int32_t* path, cudaStream_t st) {
+    const int row_vec = (int)(D * dtype_size(dtype) / 16);
+    const size_t smem = sizeof(uint4) * COMPACT_BATCH * row_vec;
+    compact_kernel<<<L * B * H * 2, 256, smem, st>>>((uint4*)k_cache, (uint4*)v_cache, B_cache, B, H, max_seq,
+                                                     row_vec, seq_len, k_acc, path);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+    advance_len_kernel<<<(B + 63) / 64, 64, 0, st>>>(seq_len, k_acc, B);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_set_chunk(int32_t* row_off2, int32_t m, cudaStream_t st) {
+    set_chunk_kernel<<<1, 1, 0, st>>>(row_off2, m);
+    return cudaGetLastError();
+}
+cudaError_t launch_bump_len(int32_t* seq_len_b, int32_t delta, cudaStream_t st) {
+    bump_len_kernel<<<1, 1, 0, st>>>(seq_len_b, delta);
+    return cudaGetLastError();
+}
+
+}  // namespace trj
