@@ -1,0 +1,403 @@
+// C ABI of libtrj: argument checks, workspace carving and the launch sequence of a verification step.
+#include <algorithm>
+#include <cmath>
+#include <cstring>
+#include <new>
+#include <vector>
+#include "trj_internal.h"
+
+using namespace trj;
+
+namespace {
+
+bool aligned(const void* p, size_t a) { return ((uintptr_t)p % a) == 0; }
+bool dtype_ok(int32_t dt) { return dt == TRJ_F32 || dt == TRJ_BF16; }
+
+// Carves consecutive 256-byte aligned regions out of a workspace.
+struct Carver {
+    char* base; size_t off = 0;
+    explicit Carver(void* p) : base((char*)p) {}
+    template <typename T> T* take(size_t count) {
+        T* r = (T*)(base + off);
+        off += align_up(sizeof(T) * count, 256);
+        return r;
+    }
+};
+
+}  // namespace
+
+// ---------------------------------------------------------------------------- op-level entry points
+extern "C" size_t trj_tree_attention_workspace(int32_t rows_total, int32_t B, int32_t H, int32_t D, int32_t max_len) {
+    (void)rows_total; (void)B; (void)H; (void)D; (void)max_len;
+    return 256;
+}
+
+extern "C" trj_status trj_tree_attention(const void* q, const void* k_cache, const void* v_cache,
+                                         const int32_t* seq_len, const int32_t* row_off, const uint64_t* anc,
+                                         int32_t anc_words, int32_t B, int32_t rows_total, int32_t max_rows,
+                                         int32_t H, int32_t D, int32_t max_seq, int32_t max_len, int32_t dtype,
+                                         void* out, void* workspace, size_t workspace_bytes, void* stream) {
+    TRJ_REQUIRE(q && k_cache && v_cache && seq_len && row_off && anc && out, TRJ_EINVAL, "tree_attention: null pointer");
+    TRJ_REQUIRE(dtype_ok(dtype), TRJ_EINVAL, "tree_attention: unknown dtype %d", dtype);
+    TRJ_REQUIRE(B >= 1 && H >= 1 && rows_total >= 0 && max_rows >= 1, TRJ_EINVAL, "tree_attention: bad sizes");
+    TRJ_REQUIRE(B <= TRJ_MAX_BATCH, TRJ_ECAPACITY, "tree_attention: batch %d exceeds %d", B, TRJ_MAX_BATCH);
+    TRJ_REQUIRE(max_rows <= TRJ_MAX_ROWS, TRJ_ECAPACITY, "tree_attention: %d rows per tree exceed %d", max_rows, TRJ_MAX_ROWS);
+    TRJ_REQUIRE(anc_words >= (max_rows + 63) / 64, TRJ_EINVAL, "tree_attention: anc_words %d too small", anc_words);
+    TRJ_REQUIRE(max_len <= max_seq, TRJ_ECAPACITY, "tree_attention: max_len %d exceeds cache rows %d", max_len, max_seq);
+    TRJ_REQUIRE(D == 64 || D == 128, TRJ_EUNSUPPORTED, "tree_attention: head_dim %d (supported: 64, 128)", D);
+    TRJ_REQUIRE(aligned(q, 16) && aligned(k_cache, 16) && aligned(v_cache, 16) && aligned(out, 16), TRJ_EINVAL,
+                "tree_attention: tensors must be 16-byte aligned");
+    TRJ_REQUIRE(workspace && workspace_bytes >= trj_tree_attention_workspace(rows_total, B, H, D, max_len),
+                TRJ_ECAPACITY, "tree_attention: workspace too small");
+    if (rows_total == 0) return TRJ_OK;
+    Batch bt{seq_len, row_off, B, rows_total, max_rows, max_len};
+    TRJ_CHECK_CUDA(launch_tree_attention_generic(q, k_cache, v_cache, anc, anc_words, bt, H, D, max_seq, dtype, out,
+                                                 (cudaStream_t)stream));
+    return TRJ_OK;
+}
+
+extern "C" size_t trj_argmax_accept_workspace(int32_t rows_total, int32_t B) {
+    return argmax_workspace_bytes(rows_total, B);
+}
+
+extern "C" trj_status trj_argmax_accept(const void* logits, int32_t dtype, int32_t V,
+                                        const int32_t* tokens, const int32_t* parent, const int32_t* depth,
+                                        const int32_t* row_off, int32_t B, int32_t rows_total,
+                                        int32_t* node_argmax, float* margin,
+                                        int32_t* k_acc, int32_t* path, int32_t* bonus,
+                                        void* workspace, size_t workspace_bytes, void* stream) {
+    TRJ_REQUIRE(logits && tokens && parent && depth && row_off && node_argmax && k_acc && path && bonus,
+                TRJ_EINVAL, "argmax_accept: null pointer");
+    TRJ_REQUIRE(dtype_ok(dtype), TRJ_EINVAL, "argmax_accept: unknown dtype %d", dtype);
+    TRJ_REQUIRE(V >= 1 && B >= 1 && rows_total >= B, TRJ_EINVAL, "argmax_accept: bad sizes (every tree has a root)");
+    TRJ_REQUIRE(B <= TRJ_MAX_BATCH, TRJ_ECAPACITY, "argmax_accept: batch %d exceeds %d", B, TRJ_MAX_BATCH);
+    TRJ_REQUIRE(rows_total <= B * TRJ_MAX_ROWS, TRJ_ECAPACITY, "argmax_accept: too many rows");
+    TRJ_REQUIRE(workspace && aligned(workspace, 256) && workspace_bytes >= argmax_workspace_bytes(rows_total, B),
+                TRJ_ECAPACITY, "argmax_accept: workspace too small or misaligned");
+    TRJ_CHECK_CUDA(launch_argmax_accept(logits, dtype, V, tokens, parent, depth, row_off, B, rows_total, node_argmax,
+                                        margin, k_acc, path, bonus, true, true, workspace, (cudaStream_t)stream));
+    return TRJ_OK;
+}
+
+extern "C" trj_status trj_compact_rows(void* k_cache, void* v_cache, int32_t L, int32_t B, int32_t H,
+                                       int32_t max_seq, int32_t D, int32_t dtype, int32_t* seq_len,
+                                       const int32_t* k_acc, const int32_t* path, void* stream) {
+    TRJ_REQUIRE(k_cache && v_cache && seq_len && k_acc && path, TRJ_EINVAL, "compact_rows: null pointer");
+    TRJ_REQUIRE(dtype_ok(dtype), TRJ_EINVAL, "compact_rows: unknown dtype %d", dtype);
+    TRJ_REQUIRE(L >= 1 && B >= 1 && H >= 1 && max_seq >= 1 && D >= 1, TRJ_EINVAL, "compact_rows: bad sizes");
+    TRJ_REQUIRE(B <= TRJ_MAX_BATCH, TRJ_ECAPACITY, "compact_rows: batch %d exceeds %d", B, TRJ_MAX_BATCH);
+    TRJ_REQUIRE((D * dtype_size(dtype)) % 16 == 0 && aligned(k_cache, 16) && aligned(v_cache, 16), TRJ_EINVAL,
+                "compact_rows: cache rows must be multiples of 16 bytes and 16-byte aligned");
+    TRJ_CHECK_CUDA(launch_compact(k_cache, v_cache, L, B, B, H, max_seq, D, dtype, seq_len, k_acc, path,
+                                  (cudaStream_t)stream));
+    return TRJ_OK;
+}
+
+extern "C" size_t trj_gemm_workspace(int32_t M, int32_t N, int32_t K) {
+    (void)M; (void)N; (void)K;
+    return 256;
+}
+
+extern "C" trj_status trj_gemm(const void* x, const void* w, float* y, int32_t M, int32_t N, int32_t K,
+                               int32_t dtype, void* workspace, size_t workspace_bytes, void* stream) {
+    TRJ_REQUIRE(x && w && y, TRJ_EINVAL, "gemm: null pointer");
+    TRJ_REQUIRE(dtype_ok(dtype), TRJ_EINVAL, "gemm: unknown dtype %d", dtype);
+    TRJ_REQUIRE(M >= 1 && N >= 1 && K >= 1, TRJ_EINVAL, "gemm: bad sizes");
+    TRJ_REQUIRE(workspace && workspace_bytes >= trj_gemm_workspace(M, N, K), TRJ_ECAPACITY, "gemm: workspace too small");
+    TRJ_CHECK_CUDA(launch_gemm_simt(x, w, y, M, N, K, dtype, (cudaStream_t)stream));
+    return TRJ_OK;
+}
+
+// ---------------------------------------------------------------------------- model context
+struct trj_ctx {
+    trj_model_cfg cfg;
+    const void* embed; const void* lm_head; const float* final_norm;
+    std::vector<const float*> attn_norm, mlp_norm;
+    std::vector<const void*> wqkv, wo, w_gate_up, w_down;
+    // workspace regions (device)
+    float* h; float* y; float* logits;
+    void* x; void* q; void* act;
+    double* inv_freq;
+    void* argmax_ws; void* attn_ws; size_t attn_ws_bytes; void* gemm_ws; size_t gemm_ws_bytes;
+    // chain-tree tables for prefill and the staging area of trj_step_host (device)
+    int32_t* chain_depth; uint64_t* chain_anc; int32_t* chunk_row_off; int32_t* unit_row_off;
+    int32_t* step_in;      // tokens | parent | depth | row_off(2) | pad -> anc
+    int32_t* step_out;     // node_argmax | k_acc | bonus | path
+    int32_t* pin_in; int32_t* pin_out;   // pinned host mirrors
+};
+
+namespace {
+
+constexpr int STEP_IN_INTS = 3 * TRJ_MAX_ROWS + 4;                       // + anc (2 words per row) after it
+constexpr int STEP_IN_BYTES = STEP_IN_INTS * 4 + TRJ_MAX_ROWS * 2 * 8;
+constexpr int STEP_OUT_INTS = TRJ_MAX_ROWS + 2 + TRJ_PATH_STRIDE;
+
+size_t carve(const trj_model_cfg& c, void* ws, trj_ctx* ctx) {
+    const size_t es = dtype_size(c.dtype);
+    const int rows = c.max_batch * c.max_rows;
+    const int HD = c.n_heads * c.head_dim;
+    const size_t wide = (size_t)std::max(std::max(3 * HD, 2 * c.d_ff), c.d_model);
+    Carver cv(ws);
+    float* h = cv.take<float>((size_t)rows * c.d_model);
+    float* y = cv.take<float>((size_t)rows * wide);
+    float* logits = cv.take<float>((size_t)rows * c.vocab);
+    char* x = cv.take<char>((size_t)rows * std::max(c.d_model, HD) * es);
+    char* q = cv.take<char>((size_t)rows * HD * es);
+    char* act = cv.take<char>((size_t)rows * c.d_ff * es);
+    double* inv_freq = cv.take<double>(c.head_dim / 2);
+    char* argmax_ws = cv.take<char>(argmax_workspace_bytes(rows, c.max_batch));
+    const size_t attn_bytes = trj_tree_attention_workspace(rows, c.max_batch, c.n_heads, c.head_dim, c.max_seq);
+    char* attn_ws = cv.take<char>(attn_bytes);
+    const size_t gemm_bytes = trj_gemm_workspace(rows, (int32_t)std::max(wide, (size_t)c.vocab), std::max(c.d_model, c.d_ff));
+    char* gemm_ws = cv.take<char>(gemm_bytes);
+    int32_t* chain_depth = cv.take<int32_t>(TRJ_MAX_ROWS);
+    uint64_t* chain_anc = cv.take<uint64_t>(TRJ_MAX_ROWS * 2);
+    int32_t* chunk_row_off = cv.take<int32_t>(2);
+    int32_t* unit_row_off = cv.take<int32_t>(2);
+    int32_t* step_in = (int32_t*)cv.take<char>(STEP_IN_BYTES);
+    int32_t* step_out = cv.take<int32_t>(STEP_OUT_INTS);
+    if (ctx) {
+        ctx->h = h; ctx->y = y; ctx->logits = logits; ctx->x = x; ctx->q = q; ctx->act = act;
+        ctx->inv_freq = inv_freq; ctx->argmax_ws = argmax_ws; ctx->attn_ws = attn_ws; ctx->attn_ws_bytes = attn_bytes;
+        ctx->gemm_ws = gemm_ws; ctx->gemm_ws_bytes = gemm_bytes;
+        ctx->chain_depth = chain_depth; ctx->chain_anc = chain_anc;
+        ctx->chunk_row_off = chunk_row_off; ctx->unit_row_off = unit_row_off;
+        ctx->step_in = step_in; ctx->step_out = step_out;
+    }
+    return cv.off;
+}
+
+trj_status check_cfg(const trj_model_cfg* c) {
+    TRJ_REQUIRE(c, TRJ_EINVAL, "cfg: null");
+    TRJ_REQUIRE(dtype_ok(c->dtype), TRJ_EINVAL, "cfg: unknown dtype %d", c->dtype);
+    TRJ_REQUIRE(c->n_layers >= 1 && c->d_model >= 1 && c->n_heads >= 1 && c->d_ff >= 1 && c->vocab >= 1,
+                TRJ_EINVAL, "cfg: non-positive dimension");
+    TRJ_REQUIRE(c->head_dim == 64 || c->head_dim == 128, TRJ_EUNSUPPORTED, "cfg: head_dim %d (supported: 64, 128)", c->head_dim);
+    TRJ_REQUIRE(c->max_batch >= 1 && c->max_batch <= TRJ_MAX_BATCH, TRJ_ECAPACITY, "cfg: max_batch %d outside 1..%d", c->max_batch, TRJ_MAX_BATCH);
+    TRJ_REQUIRE(c->max_rows >= 1 && c->max_rows <= TRJ_MAX_ROWS, TRJ_ECAPACITY, "cfg: max_rows %d outside 1..%d", c->max_rows, TRJ_MAX_ROWS);
+    TRJ_REQUIRE(c->max_seq >= c->max_rows, TRJ_EINVAL, "cfg: max_seq smaller than a tree");
+    TRJ_REQUIRE(c->rms_eps >= 0.f && c->rope_theta > 0.f, TRJ_EINVAL, "cfg: bad eps or rope base");
+    return TRJ_OK;
+}
+
+// One forward of the decoder over the rows of `bt`.  lm_first/lm_rows select which rows reach the
+// LM head (prefill only needs its last row).  b0 = first sequence of the cache the batch maps to.
+trj_status forward(trj_ctx* ctx, void* k_cache, void* v_cache, int32_t b0, const Batch& bt,
+                   const int32_t* tokens, const int32_t* depth, const uint64_t* anc, int32_t anc_words,
+                   int32_t lm_first, int32_t lm_rows, cudaStream_t st) {
+    const trj_model_cfg& c = ctx->cfg;
+    const int M = bt.rows_total, d = c.d_model, HD = c.n_heads * c.head_dim;
+    const size_t es = dtype_size(c.dtype);
+    const size_t seq_stride = (size_t)c.n_heads * c.max_seq * c.head_dim * es;     // one sequence of one layer
+    TRJ_CHECK_CUDA(launch_embed(ctx->embed, c.dtype, tokens, ctx->h, M, d, st));
+    for (int l = 0; l < c.n_layers; ++l) {
+        char* k_slab = (char*)k_cache + ((size_t)l * c.max_batch + b0) * seq_stride;
+        char* v_slab = (char*)v_cache + ((size_t)l * c.max_batch + b0) * seq_stride;
+        TRJ_CHECK_CUDA(launch_add_rmsnorm(ctx->h, l == 0 ? nullptr : ctx->y, ctx->attn_norm[l], ctx->x, c.dtype, M, d, c.rms_eps, st));
+        TRJ_CHECK_CUDA(launch_gemm_simt(ctx->x, ctx->wqkv[l], ctx->y, M, 3 * HD, d, c.dtype, st));
+        TRJ_CHECK_CUDA(launch_rope_kv_write(ctx->y, ctx->inv_freq, depth, bt, ctx->q, k_slab, v_slab, c.dtype,
+                                            c.n_heads, c.head_dim, c.max_seq, st));
+        TRJ_CHECK_CUDA(launch_tree_attention_generic(ctx->q, k_slab, v_slab, anc, anc_words, bt, c.n_heads, c.head_dim,
+                                                     c.max_seq, c.dtype, ctx->x, st));
+        TRJ_CHECK_CUDA(launch_gemm_simt(ctx->x, ctx->wo[l], ctx->y, M, d, HD, c.dtype, st));
+        TRJ_CHECK_CUDA(launch_add_rmsnorm(ctx->h, ctx->y, ctx->mlp_norm[l], ctx->x, c.dtype, M, d, c.rms_eps, st));
+        TRJ_CHECK_CUDA(launch_gemm_simt(ctx->x, ctx->w_gate_up[l], ctx->y, M, 2 * c.d_ff, d, c.dtype, st));
+        TRJ_CHECK_CUDA(launch_swiglu(ctx->y, ctx->act, c.dtype, M, c.d_ff, st));
+        TRJ_CHECK_CUDA(launch_gemm_simt(ctx->act, ctx->w_down[l], ctx->y, M, d, c.d_ff, c.dtype, st));
+    }
+    TRJ_CHECK_CUDA(launch_add_rmsnorm(ctx->h, ctx->y, ctx->final_norm, ctx->x, c.dtype, M, d, c.rms_eps, st));
+    if (lm_rows > 0)
+        TRJ_CHECK_CUDA(launch_gemm_simt((char*)ctx->x + (size_t)lm_first * d * es, ctx->lm_head,
+                                        ctx->logits + (size_t)lm_first * c.vocab, lm_rows, c.vocab, d, c.dtype, st));
+    return TRJ_OK;
+}
+
+trj_status check_step_args(const trj_ctx* ctx, int32_t B, int32_t rows_total, int32_t max_rows, int32_t max_len,
+                           int32_t anc_words) {
+    TRJ_REQUIRE(ctx, TRJ_EINVAL, "null context");
+    const trj_model_cfg& c = ctx->cfg;
+    TRJ_REQUIRE(B >= 1 && B <= c.max_batch, TRJ_ECAPACITY, "batch %d outside 1..%d", B, c.max_batch);
+    TRJ_REQUIRE(max_rows >= 1 && max_rows <= c.max_rows, TRJ_ECAPACITY, "%d rows per tree exceed max_rows %d", max_rows, c.max_rows);
+    TRJ_REQUIRE(rows_total >= B && rows_total <= B * max_rows, TRJ_EINVAL, "rows_total %d inconsistent with batch %d x %d", rows_total, B, max_rows);
+    TRJ_REQUIRE(max_len >= max_rows && max_len <= c.max_seq, TRJ_ECAPACITY, "max_len %d outside %d..%d", max_len, max_rows, c.max_seq);
+    TRJ_REQUIRE(anc_words >= (max_rows + 63) / 64, TRJ_EINVAL, "anc_words %d too small", anc_words);
+    return TRJ_OK;
+}
+
+}  // namespace
+
+extern "C" size_t trj_workspace_bytes(const trj_model_cfg* cfg) {
+    if (check_cfg(cfg) != TRJ_OK) return 0;
+    return carve(*cfg, nullptr, nullptr);
+}
+
+extern "C" trj_status trj_create(const trj_model_cfg* cfg, const trj_weights* w,
+                                 void* workspace, size_t workspace_bytes, trj_ctx** out) {
+    TRJ_REQUIRE(out, TRJ_EINVAL, "create: null out");
+    *out = nullptr;
+    trj_status s = check_cfg(cfg);
+    if (s != TRJ_OK) return s;
+    TRJ_REQUIRE(w && w->embed && w->lm_head && w->final_norm && w->attn_norm && w->wqkv && w->wo && w->mlp_norm &&
+                w->w_gate_up && w->w_down, TRJ_EINVAL, "create: null weight table");
+    for (int l = 0; l < cfg->n_layers; ++l)
+        TRJ_REQUIRE(w->attn_norm[l] && w->wqkv[l] && w->wo[l] && w->mlp_norm[l] && w->w_gate_up[l] && w->w_down[l],
+                    TRJ_EINVAL, "create: null weight in layer %d", l);
+    TRJ_REQUIRE(workspace && aligned(workspace, 256), TRJ_EINVAL, "create: workspace must be 256-byte aligned");
+    TRJ_REQUIRE(workspace_bytes >= trj_workspace_bytes(cfg), TRJ_ECAPACITY, "create: workspace of %zu bytes, need %zu",
+                workspace_bytes, trj_workspace_bytes(cfg));
+    trj_ctx* ctx = new (std::nothrow) trj_ctx();
+    TRJ_REQUIRE(ctx, TRJ_ECUDA, "create: out of host memory");
+    ctx->cfg = *cfg;
+    ctx->embed = w->embed; ctx->lm_head = w->lm_head; ctx->final_norm = w->final_norm;
+    for (int l = 0; l < cfg->n_layers; ++l) {
+        ctx->attn_norm.push_back(w->attn_norm[l]); ctx->mlp_norm.push_back(w->mlp_norm[l]);
+        ctx->wqkv.push_back(w->wqkv[l]); ctx->wo.push_back(w->wo[l]);
+        ctx->w_gate_up.push_back(w->w_gate_up[l]); ctx->w_down.push_back(w->w_down[l]);
+    }
+    carve(*cfg, workspace, ctx);
+    ctx->pin_in = ctx->pin_out = nullptr;
+    // tables: rotary frequencies and the chain tree used by prefill
+    const int half = cfg->head_dim / 2;
+    std::vector<double> freq(half);
+    for (int i = 0; i < half; ++i) freq[i] = std::pow((double)cfg->rope_theta, -2.0 * i / cfg->head_dim);
+    std::vector<int32_t> par(TRJ_MAX_ROWS), dep(TRJ_MAX_ROWS);
+    std::vector<uint64_t> anc(TRJ_MAX_ROWS * 2);
+    for (int i = 0; i < TRJ_MAX_ROWS; ++i) par[i] = i - 1;
+    tree_from_parents_impl(par.data(), TRJ_MAX_ROWS, 2, dep.data(), anc.data());
+    const int32_t unit[2] = {0, 1};
+    cudaError_t e = cudaMemcpy(ctx->inv_freq, freq.data(), sizeof(double) * half, cudaMemcpyHostToDevice);
+    if (e == cudaSuccess) e = cudaMemcpy(ctx->chain_depth, dep.data(), sizeof(int32_t) * TRJ_MAX_ROWS, cudaMemcpyHostToDevice);
+    if (e == cudaSuccess) e = cudaMemcpy(ctx->chain_anc, anc.data(), sizeof(uint64_t) * TRJ_MAX_ROWS * 2, cudaMemcpyHostToDevice);
+    if (e == cudaSuccess) e = cudaMemcpy(ctx->unit_row_off, unit, sizeof(unit), cudaMemcpyHostToDevice);
+    if (e == cudaSuccess) e = cudaMallocHost((void**)&ctx->pin_in, STEP_IN_BYTES);
+    if (e == cudaSuccess) e = cudaMallocHost((void**)&ctx->pin_out, sizeof(int32_t) * STEP_OUT_INTS);
+    if (e != cudaSuccess) {
+        if (ctx->pin_in) cudaFreeHost(ctx->pin_in);
+        if (ctx->pin_out) cudaFreeHost(ctx->pin_out);
+        delete ctx;
+        return fail(TRJ_ECUDA, "create: %s", cudaGetErrorString(e));
+    }
+    *out = ctx;
+    return TRJ_OK;
+}
+
+extern "C" trj_status trj_destroy(trj_ctx* ctx) {
+    if (!ctx) return TRJ_OK;
+    if (ctx->pin_in) cudaFreeHost(ctx->pin_in);
+    if (ctx->pin_out) cudaFreeHost(ctx->pin_out);
+    delete ctx;
+    return TRJ_OK;
+}
+
+extern "C" trj_status trj_verify_step(trj_ctx* ctx, void* k_cache, void* v_cache, const int32_t* seq_len,
+                                      const int32_t* tokens, const int32_t* parent, const int32_t* depth,
+                                      const uint64_t* anc, int32_t anc_words, const int32_t* row_off,
+                                      int32_t B, int32_t rows_total, int32_t max_rows, int32_t max_len,
+                                      int32_t* node_argmax, float* margin, float* logits, void* stream) {
+    trj_status s = check_step_args(ctx, B, rows_total, max_rows, max_len, anc_words);
+    if (s != TRJ_OK) return s;
+    TRJ_REQUIRE(k_cache && v_cache && seq_len && tokens && parent && depth && anc && row_off && node_argmax,
+                TRJ_EINVAL, "verify_step: null pointer");
+    cudaStream_t st = (cudaStream_t)stream;
+    Batch bt{seq_len, row_off, B, rows_total, max_rows, max_len};
+    s = forward(ctx, k_cache, v_cache, 0, bt, tokens, depth, anc, anc_words, 0, rows_total, st);
+    if (s != TRJ_OK) return s;
+    TRJ_CHECK_CUDA(launch_argmax_accept(ctx->logits, TRJ_F32, ctx->cfg.vocab, tokens, parent, depth, row_off, B,
+                                        rows_total, node_argmax, margin, nullptr, nullptr, nullptr, true, false,
+                                        ctx->argmax_ws, st));
+    if (logits)
+        TRJ_CHECK_CUDA(cudaMemcpyAsync(logits, ctx->logits, sizeof(float) * (size_t)rows_total * ctx->cfg.vocab,
+                                       cudaMemcpyDeviceToDevice, st));
+    return TRJ_OK;
+}
+
+extern "C" trj_status trj_accept(trj_ctx* ctx, const int32_t* tokens, const int32_t* parent, const int32_t* depth,
+                                 const int32_t* row_off, int32_t B, int32_t rows_total, const int32_t* node_argmax,
+                                 int32_t* k_acc, int32_t* path, int32_t* bonus, void* stream) {
+    TRJ_REQUIRE(ctx, TRJ_EINVAL, "accept: null context");
+    TRJ_REQUIRE(tokens && parent && depth && row_off && node_argmax && k_acc && path && bonus, TRJ_EINVAL, "accept: null pointer");
+    TRJ_REQUIRE(B >= 1 && B <= ctx->cfg.max_batch && rows_total >= B, TRJ_ECAPACITY, "accept: bad batch");
+    TRJ_CHECK_CUDA(launch_argmax_accept(nullptr, TRJ_F32, 0, tokens, parent, depth, row_off, B, rows_total,
+                                        const_cast<int32_t*>(node_argmax), nullptr, k_acc, path, bonus, false, true,
+                                        ctx->argmax_ws, (cudaStream_t)stream));
+    return TRJ_OK;
+}
+
+extern "C" trj_status trj_compact_kv(trj_ctx* ctx, void* k_cache, void* v_cache, int32_t* seq_len, int32_t B,
+                                     const int32_t* k_acc, const int32_t* path, void* stream) {
+    TRJ_REQUIRE(ctx, TRJ_EINVAL, "compact_kv: null context");
+    TRJ_REQUIRE(k_cache && v_cache && seq_len && k_acc && path, TRJ_EINVAL, "compact_kv: null pointer");
+    const trj_model_cfg& c = ctx->cfg;
+    TRJ_REQUIRE(B >= 1 && B <= c.max_batch, TRJ_ECAPACITY, "compact_kv: batch %d outside 1..%d", B, c.max_batch);
+    TRJ_CHECK_CUDA(launch_compact(k_cache, v_cache, c.n_layers, c.max_batch, B, c.n_heads, c.max_seq, c.head_dim,
+                                  c.dtype, seq_len, k_acc, path, (cudaStream_t)stream));
+    return TRJ_OK;
+}
+
+extern "C" trj_status trj_prefill(trj_ctx* ctx, void* k_cache, void* v_cache, int32_t* seq_len, int32_t b,
+                                  const int32_t* tokens, int32_t n, int32_t* first_token, void* stream) {
+    TRJ_REQUIRE(ctx, TRJ_EINVAL, "prefill: null context");
+    const trj_model_cfg& c = ctx->cfg;
+    TRJ_REQUIRE(k_cache && v_cache && seq_len && tokens && first_token, TRJ_EINVAL, "prefill: null pointer");
+    TRJ_REQUIRE(b >= 0 && b < c.max_batch, TRJ_EINVAL, "prefill: sequence %d outside the cache", b);
+    TRJ_REQUIRE(n >= 1 && n <= c.max_seq, TRJ_ECAPACITY, "prefill: %d tokens do not fit %d cache rows", n, c.max_seq);
+    cudaStream_t st = (cudaStream_t)stream;
+    for (int32_t done = 0; done < n; done += c.max_rows) {
+        const int32_t m = std::min(c.max_rows, n - done);
+        const bool last = done + m >= n;
+        TRJ_CHECK_CUDA(launch_set_chunk(ctx->chunk_row_off, m, st));
+        Batch bt{seq_len + b, ctx->chunk_row_off, 1, m, m, c.max_seq};
+        trj_status s = forward(ctx, k_cache, v_cache, b, bt, tokens + done, ctx->chain_depth, ctx->chain_anc, 2,
+                               m - 1, last ? 1 : 0, st);
+        if (s != TRJ_OK) return s;
+        if (last)   // greedy prediction after the last prompt token: a one-row arg-max
+            TRJ_CHECK_CUDA(launch_argmax_accept(ctx->logits + (size_t)(m - 1) * c.vocab, TRJ_F32, c.vocab, nullptr, nullptr,
+                                                nullptr, ctx->unit_row_off, 1, 1, first_token, nullptr, nullptr,
+                                                nullptr, nullptr, true, false, ctx->argmax_ws, st));
+        TRJ_CHECK_CUDA(launch_bump_len(seq_len + b, m, st));
+    }
+    return TRJ_OK;
+}
+
+extern "C" trj_status trj_step_host(trj_ctx* ctx, void* k_cache, void* v_cache, int32_t* seq_len, int32_t max_len,
+                                    int32_t root, const int32_t* window, int32_t W,
+                                    const int32_t* branches, int32_t R, int32_t branch_len,
+                                    int32_t* tokens, int32_t* parent, int32_t* n_rows, int32_t* node_argmax,
+                                    int32_t* k_acc, int32_t* path, int32_t* bonus, void* stream) {
+    TRJ_REQUIRE(ctx, TRJ_EINVAL, "step_host: null context");
+    TRJ_REQUIRE(k_cache && v_cache && seq_len && tokens && parent && n_rows && node_argmax && k_acc && path && bonus,
+                TRJ_EINVAL, "step_host: null pointer");
+    const trj_model_cfg& c = ctx->cfg;
+    cudaStream_t st = (cudaStream_t)stream;
+    int32_t* in = ctx->pin_in;
+    int32_t* h_tokens = in, *h_parent = in + TRJ_MAX_ROWS, *h_depth = in + 2 * TRJ_MAX_ROWS, *h_off = in + 3 * TRJ_MAX_ROWS;
+    uint64_t* h_anc = (uint64_t*)(in + STEP_IN_INTS);
+    int32_t M = 0;
+    trj_status s = trj_build_tree(root, window, W, branches, R, branch_len, c.max_rows, 2, h_tokens, h_parent, h_depth, h_anc, &M);
+    if (s != TRJ_OK) return s;
+    s = check_step_args(ctx, 1, M, M, max_len, 2);
+    if (s != TRJ_OK) return s;
+    h_off[0] = 0; h_off[1] = M;
+    TRJ_CHECK_CUDA(cudaMemcpyAsync(ctx->step_in, in, STEP_IN_BYTES, cudaMemcpyHostToDevice, st));
+    int32_t* d_tokens = ctx->step_in, *d_parent = d_tokens + TRJ_MAX_ROWS, *d_depth = d_tokens + 2 * TRJ_MAX_ROWS;
+    int32_t* d_off = d_tokens + 3 * TRJ_MAX_ROWS;
+    uint64_t* d_anc = (uint64_t*)(d_tokens + STEP_IN_INTS);
+    int32_t* d_pred = ctx->step_out, *d_k = d_pred + TRJ_MAX_ROWS, *d_bonus = d_k + 1, *d_path = d_k + 2;
+    Batch bt{seq_len, d_off, 1, M, M, max_len};
+    s = forward(ctx, k_cache, v_cache, 0, bt, d_tokens, d_depth, d_anc, 2, 0, M, st);
+    if (s != TRJ_OK) return s;
+    TRJ_CHECK_CUDA(launch_argmax_accept(ctx->logits, TRJ_F32, c.vocab, d_tokens, d_parent, d_depth, d_off, 1, M, d_pred,
+                                        nullptr, d_k, d_path, d_bonus, true, true, ctx->argmax_ws, st));
+    TRJ_CHECK_CUDA(launch_compact(k_cache, v_cache, c.n_layers, c.max_batch, 1, c.n_heads, c.max_seq, c.head_dim,
+                                  c.dtype, seq_len, d_k, d_path, st));
+    TRJ_CHECK_CUDA(cudaMemcpyAsync(ctx->pin_out, ctx->step_out, sizeof(int32_t) * STEP_OUT_INTS, cudaMemcpyDeviceToHost, st));
+    TRJ_CHECK_CUDA(cudaStreamSynchronize(st));
+    std::memcpy(tokens, h_tokens, sizeof(int32_t) * M);
+    std::memcpy(parent, h_parent, sizeof(int32_t) * M);
+    *n_rows = M;
+    std::memcpy(node_argmax, ctx->pin_out, sizeof(int32_t) * M);
+    *k_acc = ctx->pin_out[TRJ_MAX_ROWS];
+    *bonus = ctx->pin_out[TRJ_MAX_ROWS + 1];
+    std::memcpy(path, ctx->pin_out + TRJ_MAX_ROWS + 2, sizeof(int32_t) * TRJ_PATH_STRIDE);
+    return TRJ_OK;
+}
