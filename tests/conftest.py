@@ -25,3 +25,13 @@ def pytest_collection_modifyitems(config, items):
     for item in items:
         if "gpu" in item.keywords:
             item.add_marker(skip)
+
+
+@pytest.fixture(scope="session")
+def trj():
+    """The binding with libtrj.so built (incrementally) from the sources in the tree."""
+    from paper_2406_17404_b200 import build as trj_build
+    trj_build.build()
+    import paper_2406_17404_b200 as binding
+    binding.lib()
+    return binding
