@@ -38,10 +38,12 @@ def _stale(target: str, deps) -> bool:
 
 def build(verbose: bool = False, force: bool = False) -> str:
     """Compile every source under csrc/ and link libtrj.so; returns its path."""
-    nvcc = _nvcc()
-    os.makedirs(OBJ, exist_ok=True)
     headers = [os.path.join(CSRC, f) for f in os.listdir(CSRC) if f.endswith((".h", ".cuh"))]
     headers.append(os.path.join(ROOT, "include", "trj.h"))
+    if not force and not verbose and not _stale(LIB, [os.path.join(CSRC, s) for s in sources()] + headers):
+        return LIB                      # the library is newer than every source: nothing to do
+    nvcc = _nvcc()
+    os.makedirs(OBJ, exist_ok=True)
     objs, procs = [], []
     for src in sources():
         path = os.path.join(CSRC, src)
