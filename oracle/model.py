@@ -39,6 +39,13 @@ def silu(x: np.ndarray) -> np.ndarray:
     return x / (1.0 + np.exp(-x))
 
 
+def store_bf16(x: np.ndarray) -> np.ndarray:
+    """Value a bf16 tensor holds after ``x`` is stored in it: nearest bf16, ties to even (as fp64)."""
+    u = np.ascontiguousarray(x, dtype=np.float32).view(np.uint32)
+    r = (u + (np.uint32(0x7FFF) + ((u >> np.uint32(16)) & np.uint32(1)))) & np.uint32(0xFFFF0000)
+    return r.view(np.float32).astype(np.float64)
+
+
 class KVCache:
     """K and V of every layer, [L, H, capacity, D] fp64, and the number of committed rows."""
 
@@ -76,6 +83,10 @@ class Decoder:
         m, s = len(tokens), cache.seq_len
         n_heads, hd = c.n_heads, c.head_dim
         pos = s + depths(parent)
+        # bf16 configs: q, the K/V cache rows and the attention output are bf16 tensors (they are the
+        # operands and the result of the attention op at the library boundary); what such a tensor
+        # holds is the rounded value.  Everything else, and all arithmetic, stays fp64.
+        store = store_bf16 if c.dtype == "bf16" else (lambda t: t)
         h = np.asarray(self.glob["embed"], np.float64)[np.asarray(tokens, np.int64)]
         for l in range(c.n_layers):
             w = self.layers[l]
@@ -83,11 +94,11 @@ class Decoder:
             qkv = x @ np.asarray(w["wqkv"], np.float64).T
             q, k, v = (qkv[:, j * n_heads * hd:(j + 1) * n_heads * hd].reshape(m, n_heads, hd)
                        for j in range(3))
-            q, k = rope(q, pos, c.rope_theta), rope(k, pos, c.rope_theta)
+            q, k, v = store(rope(q, pos, c.rope_theta)), store(rope(k, pos, c.rope_theta)), store(v)
             cache.k[l][:, s:s + m, :] = k.transpose(1, 0, 2)
             cache.v[l][:, s:s + m, :] = v.transpose(1, 0, 2)
-            att = tree_attention(q, cache.k[l][:, :s], cache.v[l][:, :s],
-                                 cache.k[l][:, s:s + m], cache.v[l][:, s:s + m], parent)
+            att = store(tree_attention(q, cache.k[l][:, :s], cache.v[l][:, :s],
+                                       cache.k[l][:, s:s + m], cache.v[l][:, s:s + m], parent))
             h = h + att.reshape(m, n_heads * hd) @ np.asarray(w["wo"], np.float64).T
             x = rmsnorm(h, np.asarray(w["mlp_norm"], np.float64), c.rms_eps)
             gu = x @ np.asarray(w["w_gate_up"], np.float64).T

@@ -410,3 +410,30 @@ def test_generators_are_reproducible_and_bf16_exact():
     # ties-to-even on a value exactly between two bf16 numbers
     x = np.array([1.0 + 2 ** -8, 1.0 + 3 * 2 ** -8], np.float32)
     np.testing.assert_array_equal(synth.round_bf16(x), np.array([1.0, 1.0 + 2 ** -6], np.float32))
+
+
+# ---------------------------------------------------------------- bf16 storage of the attention operands
+def test_store_bf16_matches_library_conversion_and_ties_to_even():
+    import torch
+    from oracle.model import store_bf16
+    g = np.random.default_rng(0)
+    x = g.standard_normal(50000) * np.exp(g.uniform(-20, 20, 50000))
+    ref = torch.tensor(x, dtype=torch.float32).to(torch.bfloat16).double().numpy()
+    np.testing.assert_array_equal(store_bf16(x), ref)
+    np.testing.assert_array_equal(store_bf16(np.array([1.0 + 2 ** -8, 1.0 + 3 * 2 ** -8, -1.0 - 2 ** -8])),
+                                  [1.0, 1.0 + 2 ** -6, -1.0])
+
+
+def test_bf16_model_rounds_only_the_attention_operands():
+    """In a bf16 config the cache rows and q are bf16 values; TR-Jacobi still equals greedy AR decoding."""
+    import dataclasses
+    cfg = dataclasses.replace(synth.TINY, dtype="bf16")
+    dec = tiny_decoder(3, cfg)
+    pr = synth.prompt(3, 40, cfg.vocab)
+    cache = dec.new_cache(64)
+    dec.forward_rows(cache, pr, synth.chain_parents(40))
+    np.testing.assert_array_equal(synth.round_bf16(cache.k[:, :, :40].astype(np.float32)), cache.k[:, :, :40])
+    np.testing.assert_array_equal(synth.round_bf16(cache.v[:, :, :40].astype(np.float32)), cache.v[:, :, :40])
+    ar = oracle.autoregressive_greedy(dec, pr, 30)
+    out = oracle.tr_jacobi_generate(dec, pr, 30, 4, 2, 3, lambda s, n: synth.noise_draws(5, s, n))
+    assert out == ar
