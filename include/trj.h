@@ -264,6 +264,23 @@ size_t     trj_gemm_workspace(int32_t M, int32_t N, int32_t K);
 trj_status trj_gemm(const void* x, const void* w, float* y, int32_t M, int32_t N, int32_t K,
                     int32_t dtype, void* workspace, size_t workspace_bytes, void* stream);
 
+/* ------------------------------------------------------------------------
+ * Measurement aids (no counterpart in the paper).
+ * trj_launch_count: kernel launches this process has enqueued through the
+ * library so far (every launch is counted on the host when it is enqueued).
+ * trj_profile_enable(ctx, 1): from now on every kernel launch made on behalf of
+ * ctx is bracketed by two CUDA events on its stream (cost: two event records
+ * per launch; at most 8192 launches are kept between reads).
+ * trj_profile_read: waits for the recorded events, sums the device time and
+ * the launches per category (0 element-wise/norm, 1 projections, 2 rotary +
+ * K/V append, 3 tree attention, 4 arg-max/accept, 5 compaction) into
+ * ms[TRJ_PROF_CATEGORIES] / launches[TRJ_PROF_CATEGORIES] (host) and clears
+ * the record. */
+#define TRJ_PROF_CATEGORIES 6
+uint64_t   trj_launch_count(void);
+trj_status trj_profile_enable(trj_ctx* ctx, int32_t on);
+trj_status trj_profile_read(trj_ctx* ctx, float* ms, int32_t* launches);
+
 #ifdef __cplusplus
 }
 #endif

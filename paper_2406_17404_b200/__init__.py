@@ -72,7 +72,11 @@ _SIGNATURES = {
                            _I32P, _I32P, _I32P, _VP]),
     "trj_gemm_workspace": (_SZ, [_I, _I, _I]),
     "trj_gemm": (_I, [_VP, _VP, _VP, _I, _I, _I, _I, _VP, _SZ, _VP]),
+    "trj_launch_count": (C.c_uint64, []),
+    "trj_profile_enable": (_I, [_VP, _I]),
+    "trj_profile_read": (_I, [_VP, C.POINTER(C.c_float), _I32P]),
 }
+PROF_CATEGORIES = ("elementwise", "gemm", "rope_kv", "attention", "argmax_accept", "compact")
 EXPORTS = tuple(_SIGNATURES)
 
 
@@ -98,6 +102,11 @@ def _check(status: int) -> None:
 
 def version() -> str:
     return lib().trj_version().decode()
+
+
+def launch_count() -> int:
+    """trj_launch_count: kernel launches enqueued by the library in this process."""
+    return int(lib().trj_launch_count())
 
 
 # ----------------------------------------------------------------------------- host helpers (numpy)
@@ -317,6 +326,16 @@ class Model:
             self.close()
         except Exception:
             pass
+
+    def profile_enable(self, on: bool = True) -> None:
+        _check(lib().trj_profile_enable(self._handle, 1 if on else 0))
+
+    def profile_read(self) -> Dict[str, Tuple[float, int]]:
+        """trj_profile_read: {category: (device ms, launches)} since the last read."""
+        ms = (C.c_float * len(PROF_CATEGORIES))()
+        n = (C.c_int32 * len(PROF_CATEGORIES))()
+        _check(lib().trj_profile_read(self._handle, ms, n))
+        return {c: (float(ms[i]), int(n[i])) for i, c in enumerate(PROF_CATEGORIES)}
 
     def prefill(self, tokens, b: int = 0, stream=None):
         """trj_prefill: returns the device tensor holding the first greedy token."""

@@ -104,7 +104,7 @@ extern "C" trj_status trj_gemm(const void* x, const void* w, float* y, int32_t M
     TRJ_REQUIRE(dtype_ok(dtype), TRJ_EINVAL, "gemm: unknown dtype %d", dtype);
     TRJ_REQUIRE(M >= 1 && N >= 1 && K >= 1, TRJ_EINVAL, "gemm: bad sizes");
     TRJ_REQUIRE(workspace && workspace_bytes >= trj_gemm_workspace(M, N, K), TRJ_ECAPACITY, "gemm: workspace too small");
-    TRJ_CHECK_CUDA(launch_gemm_simt(x, w, y, M, N, K, dtype, (cudaStream_t)stream));
+    TRJ_CHECK_CUDA(launch_gemm_simt(x, nullptr, w, y, M, N, K, dtype, (cudaStream_t)stream));
     return TRJ_OK;
 }
 
@@ -116,7 +116,7 @@ struct trj_ctx {
     std::vector<const void*> wqkv, wo, w_gate_up, w_down;
     // workspace regions (device)
     float* h; float* y; float* logits;
-    void* x; void* q; void* act;
+    void* x; void* x_lo; void* q; void* act; void* act_lo;   // *_lo: low halves of split bf16 activations
     double* inv_freq;
     void* argmax_ws; void* attn_ws; size_t attn_ws_bytes; void* gemm_ws; size_t gemm_ws_bytes;
     // chain-tree tables for prefill and the staging area of trj_step_host (device)
@@ -124,6 +124,8 @@ struct trj_ctx {
     int32_t* step_in;      // tokens | parent | depth | row_off(2) | pad -> anc
     int32_t* step_out;     // node_argmax | k_acc | bonus | path
     int32_t* pin_in; int32_t* pin_out;   // pinned host mirrors
+    // optional per-launch device timing (trj_profile_enable)
+    bool prof_on = false; std::vector<cudaEvent_t> prof_ev; std::vector<int> prof_cat; size_t prof_used = 0;
 };
 
 namespace {
@@ -142,8 +144,10 @@ size_t carve(const trj_model_cfg& c, void* ws, trj_ctx* ctx) {
     float* y = cv.take<float>((size_t)rows * wide);
     float* logits = cv.take<float>((size_t)rows * c.vocab);
     char* x = cv.take<char>((size_t)rows * std::max(c.d_model, HD) * es);
+    char* x_lo = cv.take<char>((size_t)rows * std::max(c.d_model, HD) * es);
     char* q = cv.take<char>((size_t)rows * HD * es);
     char* act = cv.take<char>((size_t)rows * c.d_ff * es);
+    char* act_lo = cv.take<char>((size_t)rows * c.d_ff * es);
     double* inv_freq = cv.take<double>(c.head_dim / 2);
     char* argmax_ws = cv.take<char>(argmax_workspace_bytes(rows, c.max_batch));
     const size_t attn_bytes = trj_tree_attention_workspace(rows, c.max_batch, c.n_heads, c.head_dim, c.max_seq);
@@ -158,6 +162,7 @@ size_t carve(const trj_model_cfg& c, void* ws, trj_ctx* ctx) {
     int32_t* step_out = cv.take<int32_t>(STEP_OUT_INTS);
     if (ctx) {
         ctx->h = h; ctx->y = y; ctx->logits = logits; ctx->x = x; ctx->q = q; ctx->act = act;
+        ctx->x_lo = c.dtype == TRJ_BF16 ? x_lo : nullptr; ctx->act_lo = c.dtype == TRJ_BF16 ? act_lo : nullptr;
         ctx->inv_freq = inv_freq; ctx->argmax_ws = argmax_ws; ctx->attn_ws = attn_ws; ctx->attn_ws_bytes = attn_bytes;
         ctx->gemm_ws = gemm_ws; ctx->gemm_ws_bytes = gemm_bytes;
         ctx->chain_depth = chain_depth; ctx->chain_anc = chain_anc;
@@ -180,6 +185,27 @@ trj_status check_cfg(const trj_model_cfg* c) {
     return TRJ_OK;
 }
 
+enum { PROF_ELEMENTWISE = 0, PROF_GEMM = 1, PROF_ROPE = 2, PROF_ATTENTION = 3, PROF_ARGMAX = 4, PROF_COMPACT = 5 };
+constexpr size_t PROF_MAX_LAUNCHES = 8192;
+
+void prof_begin(trj_ctx* ctx, int cat, cudaStream_t st) {
+    if (!ctx->prof_on || ctx->prof_used >= PROF_MAX_LAUNCHES) return;
+    ctx->prof_cat[ctx->prof_used] = cat;
+    cudaEventRecord(ctx->prof_ev[2 * ctx->prof_used], st);
+}
+void prof_end(trj_ctx* ctx, cudaStream_t st) {
+    if (!ctx->prof_on || ctx->prof_used >= PROF_MAX_LAUNCHES) return;
+    cudaEventRecord(ctx->prof_ev[2 * ctx->prof_used + 1], st);
+    ++ctx->prof_used;
+}
+#define LAUNCH(cat, expr)                  \
+    do {                                   \
+        prof_begin(ctx, cat, st);          \
+        cudaError_t le__ = (expr);         \
+        prof_end(ctx, st);                 \
+        if (le__ != cudaSuccess) return fail(TRJ_ECUDA, "%s: %s", #expr, cudaGetErrorString(le__)); \
+    } while (0)
+
 // One forward of the decoder over the rows of `bt`.  lm_first/lm_rows select which rows reach the
 // LM head (prefill only needs its last row).  b0 = first sequence of the cache the batch maps to.
 trj_status forward(trj_ctx* ctx, void* k_cache, void* v_cache, int32_t b0, const Batch& bt,
@@ -189,26 +215,32 @@ trj_status forward(trj_ctx* ctx, void* k_cache, void* v_cache, int32_t b0, const
     const int M = bt.rows_total, d = c.d_model, HD = c.n_heads * c.head_dim;
     const size_t es = dtype_size(c.dtype);
     const size_t seq_stride = (size_t)c.n_heads * c.max_seq * c.head_dim * es;     // one sequence of one layer
-    TRJ_CHECK_CUDA(launch_embed(ctx->embed, c.dtype, tokens, ctx->h, M, d, st));
+    LAUNCH(PROF_ELEMENTWISE, launch_embed(ctx->embed, c.dtype, tokens, ctx->h, M, d, st));
     for (int l = 0; l < c.n_layers; ++l) {
         char* k_slab = (char*)k_cache + ((size_t)l * c.max_batch + b0) * seq_stride;
         char* v_slab = (char*)v_cache + ((size_t)l * c.max_batch + b0) * seq_stride;
-        TRJ_CHECK_CUDA(launch_add_rmsnorm(ctx->h, l == 0 ? nullptr : ctx->y, ctx->attn_norm[l], ctx->x, c.dtype, M, d, c.rms_eps, st));
-        TRJ_CHECK_CUDA(launch_gemm_simt(ctx->x, ctx->wqkv[l], ctx->y, M, 3 * HD, d, c.dtype, st));
-        TRJ_CHECK_CUDA(launch_rope_kv_write(ctx->y, ctx->inv_freq, depth, bt, ctx->q, k_slab, v_slab, c.dtype,
-                                            c.n_heads, c.head_dim, c.max_seq, st));
-        TRJ_CHECK_CUDA(launch_tree_attention_generic(ctx->q, k_slab, v_slab, anc, anc_words, bt, c.n_heads, c.head_dim,
-                                                     c.max_seq, c.dtype, ctx->x, st));
-        TRJ_CHECK_CUDA(launch_gemm_simt(ctx->x, ctx->wo[l], ctx->y, M, d, HD, c.dtype, st));
-        TRJ_CHECK_CUDA(launch_add_rmsnorm(ctx->h, ctx->y, ctx->mlp_norm[l], ctx->x, c.dtype, M, d, c.rms_eps, st));
-        TRJ_CHECK_CUDA(launch_gemm_simt(ctx->x, ctx->w_gate_up[l], ctx->y, M, 2 * c.d_ff, d, c.dtype, st));
-        TRJ_CHECK_CUDA(launch_swiglu(ctx->y, ctx->act, c.dtype, M, c.d_ff, st));
-        TRJ_CHECK_CUDA(launch_gemm_simt(ctx->act, ctx->w_down[l], ctx->y, M, d, c.d_ff, c.dtype, st));
+        LAUNCH(PROF_ELEMENTWISE, launch_add_rmsnorm(ctx->h, l == 0 ? nullptr : ctx->y, ctx->attn_norm[l], ctx->x, ctx->x_lo,
+                                                    c.dtype, M, d, c.rms_eps, st));
+        LAUNCH(PROF_GEMM, launch_gemm_simt(ctx->x, ctx->x_lo, ctx->wqkv[l], ctx->y, M, 3 * HD, d, c.dtype, st));
+        LAUNCH(PROF_ROPE, launch_rope_kv_write(ctx->y, ctx->inv_freq, depth, bt, ctx->q, k_slab, v_slab, c.dtype,
+                                               c.n_heads, c.head_dim, c.max_seq, st));
+        // the attention output is a bf16 tensor of its own right (no low half)
+        LAUNCH(PROF_ATTENTION, launch_tree_attention_generic(ctx->q, k_slab, v_slab, anc, anc_words, bt, c.n_heads,
+                                                             c.head_dim, c.max_seq, c.dtype, ctx->x, st));
+        LAUNCH(PROF_GEMM, launch_gemm_simt(ctx->x, nullptr, ctx->wo[l], ctx->y, M, d, HD, c.dtype, st));
+        LAUNCH(PROF_ELEMENTWISE, launch_add_rmsnorm(ctx->h, ctx->y, ctx->mlp_norm[l], ctx->x, ctx->x_lo, c.dtype, M, d,
+                                                    c.rms_eps, st));
+        LAUNCH(PROF_GEMM, launch_gemm_simt(ctx->x, ctx->x_lo, ctx->w_gate_up[l], ctx->y, M, 2 * c.d_ff, d, c.dtype, st));
+        LAUNCH(PROF_ELEMENTWISE, launch_swiglu(ctx->y, ctx->act, ctx->act_lo, c.dtype, M, c.d_ff, st));
+        LAUNCH(PROF_GEMM, launch_gemm_simt(ctx->act, ctx->act_lo, ctx->w_down[l], ctx->y, M, d, c.d_ff, c.dtype, st));
     }
-    TRJ_CHECK_CUDA(launch_add_rmsnorm(ctx->h, ctx->y, ctx->final_norm, ctx->x, c.dtype, M, d, c.rms_eps, st));
-    if (lm_rows > 0)
-        TRJ_CHECK_CUDA(launch_gemm_simt((char*)ctx->x + (size_t)lm_first * d * es, ctx->lm_head,
-                                        ctx->logits + (size_t)lm_first * c.vocab, lm_rows, c.vocab, d, c.dtype, st));
+    LAUNCH(PROF_ELEMENTWISE, launch_add_rmsnorm(ctx->h, ctx->y, ctx->final_norm, ctx->x, ctx->x_lo, c.dtype, M, d,
+                                                c.rms_eps, st));
+    if (lm_rows > 0) {
+        const size_t off = (size_t)lm_first * d * es;
+        LAUNCH(PROF_GEMM, launch_gemm_simt((char*)ctx->x + off, ctx->x_lo ? (char*)ctx->x_lo + off : nullptr, ctx->lm_head,
+                                           ctx->logits + (size_t)lm_first * c.vocab, lm_rows, c.vocab, d, c.dtype, st));
+    }
     return TRJ_OK;
 }
 
@@ -285,7 +317,36 @@ extern "C" trj_status trj_destroy(trj_ctx* ctx) {
     if (!ctx) return TRJ_OK;
     if (ctx->pin_in) cudaFreeHost(ctx->pin_in);
     if (ctx->pin_out) cudaFreeHost(ctx->pin_out);
+    for (cudaEvent_t e : ctx->prof_ev) cudaEventDestroy(e);
     delete ctx;
+    return TRJ_OK;
+}
+
+extern "C" uint64_t trj_launch_count(void) { return launches_so_far(); }
+
+extern "C" trj_status trj_profile_enable(trj_ctx* ctx, int32_t on) {
+    TRJ_REQUIRE(ctx, TRJ_EINVAL, "profile_enable: null context");
+    if (on && ctx->prof_ev.empty()) {
+        ctx->prof_ev.resize(2 * PROF_MAX_LAUNCHES);
+        ctx->prof_cat.resize(PROF_MAX_LAUNCHES);
+        for (cudaEvent_t& e : ctx->prof_ev) TRJ_CHECK_CUDA(cudaEventCreate(&e));
+    }
+    ctx->prof_on = on != 0;
+    ctx->prof_used = 0;
+    return TRJ_OK;
+}
+
+extern "C" trj_status trj_profile_read(trj_ctx* ctx, float* ms, int32_t* launches) {
+    TRJ_REQUIRE(ctx && ms && launches, TRJ_EINVAL, "profile_read: null pointer");
+    for (int c = 0; c < TRJ_PROF_CATEGORIES; ++c) { ms[c] = 0.f; launches[c] = 0; }
+    for (size_t i = 0; i < ctx->prof_used; ++i) {
+        TRJ_CHECK_CUDA(cudaEventSynchronize(ctx->prof_ev[2 * i + 1]));
+        float t = 0.f;
+        TRJ_CHECK_CUDA(cudaEventElapsedTime(&t, ctx->prof_ev[2 * i], ctx->prof_ev[2 * i + 1]));
+        ms[ctx->prof_cat[i]] += t;
+        launches[ctx->prof_cat[i]] += 1;
+    }
+    ctx->prof_used = 0;
     return TRJ_OK;
 }
 
@@ -302,9 +363,9 @@ extern "C" trj_status trj_verify_step(trj_ctx* ctx, void* k_cache, void* v_cache
     Batch bt{seq_len, row_off, B, rows_total, max_rows, max_len};
     s = forward(ctx, k_cache, v_cache, 0, bt, tokens, depth, anc, anc_words, 0, rows_total, st);
     if (s != TRJ_OK) return s;
-    TRJ_CHECK_CUDA(launch_argmax_accept(ctx->logits, TRJ_F32, ctx->cfg.vocab, tokens, parent, depth, row_off, B,
-                                        rows_total, node_argmax, margin, nullptr, nullptr, nullptr, true, false,
-                                        ctx->argmax_ws, st));
+    LAUNCH(PROF_ARGMAX, launch_argmax_accept(ctx->logits, TRJ_F32, ctx->cfg.vocab, tokens, parent, depth, row_off, B,
+                                             rows_total, node_argmax, margin, nullptr, nullptr, nullptr, true, false,
+                                             ctx->argmax_ws, st));
     if (logits)
         TRJ_CHECK_CUDA(cudaMemcpyAsync(logits, ctx->logits, sizeof(float) * (size_t)rows_total * ctx->cfg.vocab,
                                        cudaMemcpyDeviceToDevice, st));
@@ -317,9 +378,10 @@ extern "C" trj_status trj_accept(trj_ctx* ctx, const int32_t* tokens, const int3
     TRJ_REQUIRE(ctx, TRJ_EINVAL, "accept: null context");
     TRJ_REQUIRE(tokens && parent && depth && row_off && node_argmax && k_acc && path && bonus, TRJ_EINVAL, "accept: null pointer");
     TRJ_REQUIRE(B >= 1 && B <= ctx->cfg.max_batch && rows_total >= B, TRJ_ECAPACITY, "accept: bad batch");
-    TRJ_CHECK_CUDA(launch_argmax_accept(nullptr, TRJ_F32, 0, tokens, parent, depth, row_off, B, rows_total,
-                                        const_cast<int32_t*>(node_argmax), nullptr, k_acc, path, bonus, false, true,
-                                        ctx->argmax_ws, (cudaStream_t)stream));
+    cudaStream_t st = (cudaStream_t)stream;
+    LAUNCH(PROF_ARGMAX, launch_argmax_accept(nullptr, TRJ_F32, 0, tokens, parent, depth, row_off, B, rows_total,
+                                             const_cast<int32_t*>(node_argmax), nullptr, k_acc, path, bonus, false, true,
+                                             ctx->argmax_ws, st));
     return TRJ_OK;
 }
 
@@ -329,8 +391,9 @@ extern "C" trj_status trj_compact_kv(trj_ctx* ctx, void* k_cache, void* v_cache,
     TRJ_REQUIRE(k_cache && v_cache && seq_len && k_acc && path, TRJ_EINVAL, "compact_kv: null pointer");
     const trj_model_cfg& c = ctx->cfg;
     TRJ_REQUIRE(B >= 1 && B <= c.max_batch, TRJ_ECAPACITY, "compact_kv: batch %d outside 1..%d", B, c.max_batch);
-    TRJ_CHECK_CUDA(launch_compact(k_cache, v_cache, c.n_layers, c.max_batch, B, c.n_heads, c.max_seq, c.head_dim,
-                                  c.dtype, seq_len, k_acc, path, (cudaStream_t)stream));
+    cudaStream_t st = (cudaStream_t)stream;
+    LAUNCH(PROF_COMPACT, launch_compact(k_cache, v_cache, c.n_layers, c.max_batch, B, c.n_heads, c.max_seq, c.head_dim,
+                                        c.dtype, seq_len, k_acc, path, st));
     return TRJ_OK;
 }
 
@@ -386,10 +449,10 @@ extern "C" trj_status trj_step_host(trj_ctx* ctx, void* k_cache, void* v_cache, 
     Batch bt{seq_len, d_off, 1, M, M, max_len};
     s = forward(ctx, k_cache, v_cache, 0, bt, d_tokens, d_depth, d_anc, 2, 0, M, st);
     if (s != TRJ_OK) return s;
-    TRJ_CHECK_CUDA(launch_argmax_accept(ctx->logits, TRJ_F32, c.vocab, d_tokens, d_parent, d_depth, d_off, 1, M, d_pred,
-                                        nullptr, d_k, d_path, d_bonus, true, true, ctx->argmax_ws, st));
-    TRJ_CHECK_CUDA(launch_compact(k_cache, v_cache, c.n_layers, c.max_batch, 1, c.n_heads, c.max_seq, c.head_dim,
-                                  c.dtype, seq_len, d_k, d_path, st));
+    LAUNCH(PROF_ARGMAX, launch_argmax_accept(ctx->logits, TRJ_F32, c.vocab, d_tokens, d_parent, d_depth, d_off, 1, M, d_pred,
+                                             nullptr, d_k, d_path, d_bonus, true, true, ctx->argmax_ws, st));
+    LAUNCH(PROF_COMPACT, launch_compact(k_cache, v_cache, c.n_layers, c.max_batch, 1, c.n_heads, c.max_seq, c.head_dim,
+                                        c.dtype, seq_len, d_k, d_path, st));
     TRJ_CHECK_CUDA(cudaMemcpyAsync(ctx->pin_out, ctx->step_out, sizeof(int32_t) * STEP_OUT_INTS, cudaMemcpyDeviceToHost, st));
     TRJ_CHECK_CUDA(cudaStreamSynchronize(st));
     std::memcpy(tokens, h_tokens, sizeof(int32_t) * M);

@@ -1,6 +1,7 @@
 // Shape-generic kernels of the verification step (fp32 or bf16 storage, fp32 arithmetic).
 // They serve every shape the specialised sm_100a kernels do not cover (fp32 models, odd head
 // sizes) and all the small element-wise steps between the projections.
+#include <atomic>
 #include "trj_internal.h"
 
 namespace trj {
@@ -12,6 +13,15 @@ template <> __device__ __forceinline__ float to_f<__nv_bfloat16>(__nv_bfloat16 v
 template <typename T> __device__ __forceinline__ T from_f(float v);
 template <> __device__ __forceinline__ float from_f<float>(float v) { return v; }
 template <> __device__ __forceinline__ __nv_bfloat16 from_f<__nv_bfloat16>(float v) { return __float2bfloat16_rn(v); }
+
+// Activations that feed a projection keep (almost) fp32 precision in bf16 models: the value is
+// stored as a bf16 pair hi + lo (lo = the rounding error of hi), which the projection adds back.
+template <typename T>
+__device__ __forceinline__ void store_split(T* hi, T* lo, size_t i, float v) {
+    const T h = from_f<T>(v);
+    hi[i] = h;
+    if (lo) lo[i] = from_f<T>(v - to_f(h));
+}
 
 __device__ __forceinline__ float warp_sum(float v) {
 #pragma unroll
@@ -43,7 +53,8 @@ __global__ void embed_kernel(const T* __restrict__ embed, const int32_t* __restr
 // ---------------------------------------------------------------- residual add + RMSNorm
 template <typename T>
 __global__ void add_rmsnorm_kernel(float* __restrict__ h, const float* __restrict__ add,
-                                   const float* __restrict__ gain, T* __restrict__ x, int d, float eps) {
+                                   const float* __restrict__ gain, T* __restrict__ x, T* __restrict__ x_lo,
+                                   int d, float eps) {
     __shared__ float red[32];
     const int row = blockIdx.x;
     float* hr = h + (size_t)row * d;
@@ -63,14 +74,15 @@ __global__ void add_rmsnorm_kernel(float* __restrict__ h, const float* __restric
     }
     __syncthreads();
     const float inv = rsqrtf(red[0] / (float)d + eps);
-    for (int c = threadIdx.x; c < d; c += blockDim.x) x[(size_t)row * d + c] = from_f<T>(hr[c] * inv * gain[c]);
+    for (int c = threadIdx.x; c < d; c += blockDim.x) store_split(x, x_lo, (size_t)row * d + c, hr[c] * inv * gain[c]);
 }
 
 // ---------------------------------------------------------------- plain tiled GEMM
-// y[M][N] = x[M][K] . w[N][K]^T ; 64x64 tile, 16-deep slices, 4x4 outputs per thread.
+// y[M][N] = (x + x_lo)[M][K] . w[N][K]^T ; 64x64 tile, 16-deep slices, 4x4 outputs per thread.
 template <typename T>
-__global__ void __launch_bounds__(256) gemm_simt_kernel(const T* __restrict__ x, const T* __restrict__ w,
-                                                        float* __restrict__ y, int M, int N, int K) {
+__global__ void __launch_bounds__(256) gemm_simt_kernel(const T* __restrict__ x, const T* __restrict__ x_lo,
+                                                        const T* __restrict__ w, float* __restrict__ y,
+                                                        int M, int N, int K) {
     constexpr int BM = 64, BN = 64, BK = 16;
     __shared__ float xs[BK][BM + 4];
     __shared__ float ws[BK][BN + 4];
@@ -83,7 +95,12 @@ __global__ void __launch_bounds__(256) gemm_simt_kernel(const T* __restrict__ x,
         for (int i = 0; i < 4; ++i) {
             const int k = k0 + lk + i;
             const int xm = m0 + lr, wn = n0 + lr;
-            xs[lk + i][lr] = (xm < M && k < K) ? to_f(x[(size_t)xm * K + k]) : 0.f;
+            float xv = 0.f;
+            if (xm < M && k < K) {
+                xv = to_f(x[(size_t)xm * K + k]);
+                if (x_lo) xv += to_f(x_lo[(size_t)xm * K + k]);
+            }
+            xs[lk + i][lr] = xv;
             ws[lk + i][lr] = (wn < N && k < K) ? to_f(w[(size_t)wn * K + k]) : 0.f;
         }
         __syncthreads();
@@ -215,12 +232,13 @@ __global__ void __launch_bounds__(128) tree_attention_generic_kernel(
 
 // ---------------------------------------------------------------- SwiGLU
 template <typename T>
-__global__ void swiglu_kernel(const float* __restrict__ gu, T* __restrict__ act, int rows, int f) {
+__global__ void swiglu_kernel(const float* __restrict__ gu, T* __restrict__ act, T* __restrict__ act_lo,
+                              int rows, int f) {
     const size_t n = (size_t)rows * f;
     for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x) {
         const size_t r = i / f, c = i % f;
         const float g = gu[r * 2 * f + c], u = gu[r * 2 * f + f + c];
-        act[i] = from_f<T>(g / (1.f + expf(-g)) * u);
+        store_split(act, act_lo, i, g / (1.f + expf(-g)) * u);
     }
 }
 
@@ -374,32 +392,40 @@ __global__ void bump_len_kernel(int32_t* seq_len_b, int delta) { *seq_len_b += d
 }  // namespace
 
 // ============================================================================ launchers
+static std::atomic<uint64_t> g_launches{0};
+void count_launch() { g_launches.fetch_add(1, std::memory_order_relaxed); }
+uint64_t launches_so_far() { return g_launches.load(std::memory_order_relaxed); }
+
 #define DISPATCH_T(dtype, ...)                                         \
     if ((dtype) == TRJ_BF16) { using T = __nv_bfloat16; __VA_ARGS__; } \
     else { using T = float; __VA_ARGS__; }
 
 cudaError_t launch_embed(const void* embed, int32_t dtype, const int32_t* tokens, float* h,
                          int32_t rows, int32_t d, cudaStream_t st) {
+    count_launch();
     DISPATCH_T(dtype, embed_kernel<T><<<rows, 256, 0, st>>>((const T*)embed, tokens, h, d));
     return cudaGetLastError();
 }
 
-cudaError_t launch_add_rmsnorm(float* h, const float* add, const float* gain, void* x, int32_t dtype,
+cudaError_t launch_add_rmsnorm(float* h, const float* add, const float* gain, void* x, void* x_lo, int32_t dtype,
                                int32_t rows, int32_t d, float eps, cudaStream_t st) {
-    DISPATCH_T(dtype, add_rmsnorm_kernel<T><<<rows, 256, 0, st>>>(h, add, gain, (T*)x, d, eps));
+    count_launch();
+    DISPATCH_T(dtype, add_rmsnorm_kernel<T><<<rows, 256, 0, st>>>(h, add, gain, (T*)x, (T*)x_lo, d, eps));
     return cudaGetLastError();
 }
 
-cudaError_t launch_gemm_simt(const void* x, const void* w, float* y, int32_t M, int32_t N, int32_t K,
-                             int32_t dtype, cudaStream_t st) {
+cudaError_t launch_gemm_simt(const void* x, const void* x_lo, const void* w, float* y, int32_t M, int32_t N,
+                             int32_t K, int32_t dtype, cudaStream_t st) {
+    count_launch();
     dim3 grid((N + 63) / 64, (M + 63) / 64);
-    DISPATCH_T(dtype, gemm_simt_kernel<T><<<grid, 256, 0, st>>>((const T*)x, (const T*)w, y, M, N, K));
+    DISPATCH_T(dtype, gemm_simt_kernel<T><<<grid, 256, 0, st>>>((const T*)x, (const T*)x_lo, (const T*)w, y, M, N, K));
     return cudaGetLastError();
 }
 
 cudaError_t launch_rope_kv_write(const float* qkv, const double* inv_freq, const int32_t* depth,
                                  const Batch& bt, void* q_out, void* k_slab, void* v_slab, int32_t dtype,
                                  int32_t H, int32_t D, int32_t max_seq, cudaStream_t st) {
+    count_launch();
     dim3 grid(bt.rows_total, H);
     DISPATCH_T(dtype, rope_kv_write_kernel<T><<<grid, 64, 0, st>>>(qkv, inv_freq, depth, bt.seq_len, bt.row_off,
                                                                   bt.B, (T*)q_out, (T*)k_slab, (T*)v_slab, H, D, max_seq));
@@ -410,6 +436,7 @@ cudaError_t launch_tree_attention_generic(const void* q, const void* k_slab, con
                                           const uint64_t* anc, int32_t anc_words, const Batch& bt,
                                           int32_t H, int32_t D, int32_t max_seq, int32_t dtype,
                                           void* out, cudaStream_t st) {
+    count_launch();
     dim3 grid(bt.rows_total, H);
 #define ATT(DD)                                                                                          \
     DISPATCH_T(dtype, tree_attention_generic_kernel<T, DD><<<grid, 128, 0, st>>>(                        \
@@ -422,10 +449,12 @@ cudaError_t launch_tree_attention_generic(const void* q, const void* k_slab, con
     return cudaGetLastError();
 }
 
-cudaError_t launch_swiglu(const float* gu, void* act, int32_t dtype, int32_t rows, int32_t f, cudaStream_t st) {
+cudaError_t launch_swiglu(const float* gu, void* act, void* act_lo, int32_t dtype, int32_t rows, int32_t f,
+                          cudaStream_t st) {
+    count_launch();
     const size_t n = (size_t)rows * f;
     const int blocks = (int)((n + 255) / 256 < 1184 ? (n + 255) / 256 : 1184);
-    DISPATCH_T(dtype, swiglu_kernel<T><<<blocks, 256, 0, st>>>(gu, (T*)act, rows, f));
+    DISPATCH_T(dtype, swiglu_kernel<T><<<blocks, 256, 0, st>>>(gu, (T*)act, (T*)act_lo, rows, f));
     return cudaGetLastError();
 }
 
@@ -439,6 +468,7 @@ cudaError_t launch_argmax_accept(const void* logits, int32_t dtype, int32_t V,
                                  const int32_t* row_off, int32_t B, int32_t rows_total,
                                  int32_t* node_argmax, float* margin, int32_t* k_acc, int32_t* path,
                                  int32_t* bonus, bool do_argmax, bool do_accept, void* ws, cudaStream_t st) {
+    if (do_argmax || do_accept) count_launch();
     if (do_argmax) {
         unsigned int* tickets = (unsigned int*)ws;
         Top* partial = (Top*)((char*)ws + align_up(sizeof(unsigned int) * TRJ_MAX_BATCH, 256));
@@ -455,6 +485,7 @@ cudaError_t launch_argmax_accept(const void* logits, int32_t dtype, int32_t V,
 cudaError_t launch_compact(void* k_cache, void* v_cache, int32_t L, int32_t B_cache, int32_t B, int32_t H,
                            int32_t max_seq, int32_t D, int32_t dtype, int32_t* seq_len,
                            const int32_t* k_acc, const int32_t* path, cudaStream_t st) {
+    count_launch(); count_launch();
     const int row_vec = (int)(D * dtype_size(dtype) / 16);
     const size_t smem = sizeof(uint4) * COMPACT_BATCH * row_vec;
     compact_kernel<<<L * B * H * 2, 256, smem, st>>>((uint4*)k_cache, (uint4*)v_cache, B_cache, B, H, max_seq,
@@ -466,10 +497,12 @@ cudaError_t launch_compact(void* k_cache, void* v_cache, int32_t L, int32_t B_ca
 }
 
 cudaError_t launch_set_chunk(int32_t* row_off2, int32_t m, cudaStream_t st) {
+    count_launch();
     set_chunk_kernel<<<1, 1, 0, st>>>(row_off2, m);
     return cudaGetLastError();
 }
 cudaError_t launch_bump_len(int32_t* seq_len_b, int32_t delta, cudaStream_t st) {
+    count_launch();
     bump_len_kernel<<<1, 1, 0, st>>>(seq_len_b, delta);
     return cudaGetLastError();
 }

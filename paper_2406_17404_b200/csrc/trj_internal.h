@@ -28,6 +28,10 @@ inline size_t dtype_size(int32_t dt) { return dt == TRJ_BF16 ? 2 : 4; }
 trj_status tree_from_parents_impl(const int32_t* parent, int32_t M, int32_t anc_words,
                                   int32_t* depth, uint64_t* anc);
 
+// ---- launch accounting: every kernel launch of the library passes through count_launch() -------
+void count_launch();
+uint64_t launches_so_far();
+
 // ---- generic kernels (kernels_generic.cu); every launcher only enqueues ------
 // Geometry of a ragged batch of trees over a KV cache slab of one layer.
 struct Batch {
@@ -39,11 +43,12 @@ struct Batch {
 cudaError_t launch_embed(const void* embed, int32_t dtype, const int32_t* tokens, float* h,
                          int32_t rows, int32_t d, cudaStream_t st);
 // h += add (when add != nullptr, h is updated in place); x = rmsnorm(h) * gain, stored as dtype.
-cudaError_t launch_add_rmsnorm(float* h, const float* add, const float* gain, void* x, int32_t dtype,
+// In bf16 models x is written as a bf16 pair: x (hi) and x_lo (the rounding error of hi); x_lo may be null.
+cudaError_t launch_add_rmsnorm(float* h, const float* add, const float* gain, void* x, void* x_lo, int32_t dtype,
                                int32_t rows, int32_t d, float eps, cudaStream_t st);
-// y[M][N] fp32 = x[M][K] . w[N][K]^T, plain shared-memory tiled FMA kernel.
-cudaError_t launch_gemm_simt(const void* x, const void* w, float* y, int32_t M, int32_t N, int32_t K,
-                             int32_t dtype, cudaStream_t st);
+// y[M][N] fp32 = (x + x_lo)[M][K] . w[N][K]^T (x_lo may be null), plain shared-memory tiled FMA kernel.
+cudaError_t launch_gemm_simt(const void* x, const void* x_lo, const void* w, float* y, int32_t M, int32_t N,
+                             int32_t K, int32_t dtype, cudaStream_t st);
 // Rotary embedding of q and k at position seq_len[b] + depth[row]; q -> q_out [rows][H][D];
 // k, v -> cache rows seq_len[b] + local row of the layer slab [B][H][max_seq][D].
 cudaError_t launch_rope_kv_write(const float* qkv, const double* inv_freq, const int32_t* depth,
@@ -54,7 +59,8 @@ cudaError_t launch_tree_attention_generic(const void* q, const void* k_slab, con
                                           int32_t H, int32_t D, int32_t max_seq, int32_t dtype,
                                           void* out, cudaStream_t st);
 // act[M][f] (dtype) = silu(gu[:, :f]) * gu[:, f:]
-cudaError_t launch_swiglu(const float* gu, void* act, int32_t dtype, int32_t rows, int32_t f, cudaStream_t st);
+cudaError_t launch_swiglu(const float* gu, void* act, void* act_lo, int32_t dtype, int32_t rows, int32_t f,
+                          cudaStream_t st);
 
 // Arg-max over the vocabulary and/or acceptance.  do_argmax: compute node_argmax (+margin) from
 // logits; do_accept: walk the tree and write k_acc/path/bonus.  ws: tickets + partials.
