@@ -1,0 +1,419 @@
+#!/usr/bin/env python
+"""Benchmark of the TR-Jacobi verification step (one B200 per rank, replicas only).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+
+Workload (N = 1 and every rank of N > 1): a LLaMA-2-7B-shaped random-init bf16 decoder, a 512-token
+random prompt already prefilled, TR-Jacobi trees of 32 draft tokens + root (Jacobi window 5 plus nine
+retrieved branches of 3).  One step = the whole hot path: tree build, verification forward over the 33
+rows, per-node arg-max, longest-path acceptance, KV compaction.  Prints ONE JSON line.
+
+`value`   draft tokens verified per second with the tree already resident in HBM (CUDA events).
+`e2e`     the same metric through trj_step_host: host integers in, host result out, H2D/D2H inside.
+`roofline` the projection kernels (they stream the 13.2 GB of weights): algorithmic bytes / device time.
+`tree_attention` the op-level tree attention of the 64-row / prefix-1024 and 128-row / prefix-8192 cases.
+`cpu_baseline` the CPU oracle timed on a bounded sample (two of the 32 layers + LM head, scaled).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+WIDTH, N_BRANCHES, BRANCH_LEN = 5, 9, 3
+TREE_ROWS = 1 + WIDTH + N_BRANCHES * BRANCH_LEN          # 33
+DRAFTS = TREE_ROWS - 1                                   # 32 draft tokens per step
+PROMPT = 512
+METRIC = "draft_tokens_verified_per_s"
+UNIT = "tokens/s"
+# DRAM traffic (read + write bytes) of ALL projection launches of one step, from an ncu capture of the
+# current projection kernel; None until measured or after the kernel changed.
+GEMM_TRAFFIC_BYTES_PER_STEP = None
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return {"hbm_gbs": float(p["hbm_gbs"]), "bf16_tflops": float(p["bf16_tflops"]),
+                "bf16_tflops_sustained": float(p.get("bf16_tflops_sustained", p["bf16_tflops"])), "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
+
+
+class ClockSampler:
+    """nvidia-smi clock / throttle-reason samples taken while the timed region runs."""
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.proc, self.file = index, None, None
+
+    def start(self):
+        try:
+            self.file = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
+            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
+                                          "-lms", "100", "-i", str(self.index)], stdout=self.file, stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.proc is None:
+            return out
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        self.file.flush()
+        self.file.seek(0)
+        sm, mx, reasons = [], [], set()
+        names = ("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap")
+        for line in self.file.read().splitlines():
+            parts = [p.strip() for p in line.split(",")]
+            if len(parts) < 7:
+                continue
+            try:
+                sm.append(float(parts[0])); mx.append(float(parts[1]))
+            except ValueError:
+                continue
+            for n, v in zip(names, parts[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        self.file.close()
+        os.unlink(self.file.name)
+        if sm:
+            out.update(sm_mhz=statistics.median(sm), sm_max_mhz=max(mx), reasons=sorted(reasons), samples=len(sm))
+        return out
+
+
+# --------------------------------------------------------------------------------------- our arm
+def device_weights(cfg, seed, device):
+    """Random-init weights ~ N(0, 0.02) drawn on the device (seeded), stored as bf16; norm gains 1."""
+    import torch
+    g = torch.Generator(device=device)
+    g.manual_seed(seed)
+
+    def mat(rows, cols):
+        return (torch.randn(rows, cols, generator=g, device=device, dtype=torch.float32) * cfg.weight_std).to(torch.bfloat16)
+    d, f, hd = cfg.d_model, cfg.d_ff, cfg.n_heads * cfg.head_dim
+    ones = lambda: torch.ones(d, dtype=torch.float32, device=device)
+    layers = [{"attn_norm": ones(), "wqkv": mat(3 * hd, d), "wo": mat(d, hd), "mlp_norm": ones(),
+               "w_gate_up": mat(2 * f, d), "w_down": mat(d, f)} for _ in range(cfg.n_layers)]
+    glob = {"embed": mat(cfg.vocab, d), "lm_head": mat(cfg.vocab, d), "final_norm": ones()}
+    return layers, glob
+
+
+def gemm_bytes_per_step(cfg, rows):
+    """Algorithmic bytes of all projections of one verification step: every weight once (bf16), the
+    split-bf16 activations in (attention output: single bf16) and the fp32 results out."""
+    d, f, hd, v = cfg.d_model, cfg.d_ff, cfg.n_heads * cfg.head_dim, cfg.vocab
+    per_layer = [(3 * hd, d, 2), (d, hd, 1), (2 * f, d, 2), (d, f, 2)]      # (N, K, activation halves)
+    total = 0
+    for n, k, halves in per_layer:
+        total += cfg.n_layers * (n * k * 2 + rows * k * 2 * halves + rows * n * 4)
+    total += v * d * 2 + rows * d * 2 * 2 + rows * v * 4
+    return total
+
+
+def bench_tree_attention(trj, torch, peaks, steps, warmup):
+    """Op-level tree attention on the two op-level shapes, over distinct caches larger than L2."""
+    out = []
+    for name, prefix, rows, depth, n_caches in (("cfg2: 32x128 heads, prefix 1024, 64-row tree", 1024, 64, 6, 32),
+                                                ("cfg4: 32x128 heads, prefix 8192, 128-row tree", 8192, 128, 8, 4)):
+        import synth
+        h, d = 32, 128
+        total = prefix + rows
+        g = torch.Generator(device="cuda"); g.manual_seed(7)
+        k = torch.randn(n_caches, 1, h, total, d, generator=g, device="cuda", dtype=torch.float32).to(torch.bfloat16)
+        v = torch.randn(n_caches, 1, h, total, d, generator=g, device="cuda", dtype=torch.float32).to(torch.bfloat16)
+        q = torch.randn(n_caches, rows, h, d, generator=g, device="cuda", dtype=torch.float32).to(torch.bfloat16)
+        o = torch.empty_like(q)
+        parent = synth.random_tree(1, rows, depth, 3 if rows == 64 else 4)
+        _, anc = trj.tree_from_parents(parent)
+        anc_d = torch.from_numpy(anc.view(np.int64)).cuda()
+        seq_len = torch.tensor([prefix], dtype=torch.int32, device="cuda")
+        row_off = torch.tensor([0, rows], dtype=torch.int32, device="cuda")
+        ws = torch.empty(max(256, trj.tree_attention_workspace(rows, 1, h, d, total)), dtype=torch.uint8, device="cuda")
+
+        def one_pass():
+            for c in range(n_caches):
+                trj.tree_attention(q[c], k[c], v[c], seq_len, row_off, anc_d, max_rows=rows, max_len=total, out=o[c], workspace=ws)
+        for _ in range(warmup):
+            one_pass()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(steps):
+            one_pass()
+        e1.record()
+        torch.cuda.synchronize()
+        us = e0.elapsed_time(e1) * 1e3 / (steps * n_caches)
+        nbytes = 2 * h * total * d * 2 + 2 * rows * h * d * 2            # K, V (prefix + tree rows) + q + out
+        gbs = nbytes / us / 1e3
+        out.append({"workload": name, "us_per_launch": round(us, 2), "algorithmic_bytes": nbytes, "hbm_gbs": round(gbs, 1),
+                    "frac_of_" + peaks["source"] + "_peak": round(gbs / peaks["hbm_gbs"], 4),
+                    "distinct_caches": n_caches})
+        del k, v, q, o
+    return out
+
+
+def oracle_sample(cfg_full, seed=0):
+    """The CPU oracle on a bounded sample of the workload: one verification step of a 2-layer slice of the
+    7B shape (33 rows over a 512-row cache) plus the LM head; the layer part is scaled by n_layers / 2."""
+    import oracle
+    import synth
+    from oracle.model import rmsnorm
+    cfg = cfg_full.with_layers(2)
+    layers = [synth.layer_weights(cfg, seed, l) for l in range(2)]
+    glob = synth.global_weights(cfg, seed)
+    dec = oracle.Decoder(cfg, layers, glob)
+    cache = dec.new_cache(PROMPT + TREE_ROWS)
+    g = synth.stream(seed, "oracle_cache")
+    cache.k[:, :, :PROMPT] = g.standard_normal(cache.k[:, :, :PROMPT].shape)
+    cache.v[:, :, :PROMPT] = g.standard_normal(cache.v[:, :, :PROMPT].shape)
+    cache.seq_len = PROMPT
+    window = synth.prompt(seed + 1, WIDTH, cfg.vocab)
+    branches = synth.prompt(seed + 2, N_BRANCHES * BRANCH_LEN, cfg.vocab).reshape(N_BRANCHES, BRANCH_LEN)
+    tokens, parent = oracle.build_tree(17, window, branches)
+    # time the LM head on its own so that only the layer part is scaled
+    x = np.asarray(glob["embed"], np.float64)[tokens]
+    t0 = time.perf_counter()
+    _ = rmsnorm(x, np.asarray(glob["final_norm"], np.float64), cfg.rms_eps) @ np.asarray(glob["lm_head"], np.float64).T
+    t_head = time.perf_counter() - t0
+    t0 = time.perf_counter()
+    from oracle.model import verify_step
+    verify_step(dec, cache, tokens, parent)
+    t_step2 = time.perf_counter() - t0
+    t_layers = max(t_step2 - t_head, 0.0)
+    t_full = t_layers * cfg_full.n_layers / 2 + t_head
+    return t_full, {"two_layers_plus_head_s": round(t_step2, 3), "lm_head_s": round(t_head, 3)}
+
+
+def cpu_threads():
+    try:
+        from threadpoolctl import threadpool_info
+        n = max((p.get("num_threads", 1) for p in threadpool_info()), default=1)
+        return int(n)
+    except Exception:
+        return os.cpu_count() or 1
+
+
+def run_reference(args, rank, world):
+    if rank != 0:
+        return
+    import synth
+    cfg = synth.LLAMA7B
+    times = []
+    detail = {}
+    for i in range(args.warmup + args.steps):
+        t, detail = oracle_sample(cfg, seed=i)
+        if i >= args.warmup:
+            times.append(t)
+    ms = 1e3 * sum(times) / len(times)
+    val = DRAFTS / (ms / 1e3)
+    cores = cpu_threads()
+    line = {"impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "f64", "data": "synthetic",
+            "config": workload_config(cfg, "cpu oracle"),
+            "cpu_baseline": {"value": val, "unit": UNIT, "cores": cores, "kind": "oracle",
+                             "sample": "one verification step of layers 0-1 of 32 plus the LM head per timed step; "
+                                       "layer time scaled by 16", **detail},
+            "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(line), flush=True)
+
+
+def workload_config(cfg, l2_note):
+    return {"workload": "configs[2]: LLaMA-2-7B-shaped random-init decoder, bf16, prompt 512, TR-Jacobi trees of 32 "
+                        "draft tokens + root (window 5 + 9 retrieved branches of 3); one full verification step",
+            "n_layers": cfg.n_layers, "d_model": cfg.d_model, "n_heads": cfg.n_heads, "head_dim": cfg.head_dim,
+            "d_ff": cfg.d_ff, "vocab": cfg.vocab, "tree_rows": TREE_ROWS, "draft_tokens_per_step": DRAFTS,
+            "prefix": PROMPT, "batch": 1, "parallelism": "replicas", "l2": l2_note}
+
+
+def run_ours(args, rank, world, local_rank):
+    import torch
+    import torch.distributed as dist
+    import synth
+    import paper_2406_17404_b200 as trj
+    from paper_2406_17404_b200 import decode
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the verification step has no CPU path")
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    trj.lib()
+    peaks = measured_peaks()
+    cfg = synth.LLAMA7B if not args.layers else synth.LLAMA7B.with_layers(args.layers)
+    layers, glob = device_weights(cfg, 1234 + rank, dev)
+    model = trj.Model(cfg, layers, glob, max_batch=1, max_seq=PROMPT + 1024, max_rows=trj.MAX_ROWS)
+    prompt = synth.prompt(100 + rank, PROMPT, cfg.vocab)
+    draw = lambda s, n: synth.noise_draws(rank, s, n)
+
+    # ---- warm-up: real decode steps (also gives a realistic tree for the resident-input loop)
+    trace = []
+    decode.tr_jacobi_generate(model, prompt, max(args.warmup, 3) * 1 + 1, WIDTH, N_BRANCHES, BRANCH_LEN, draw, trace=trace)
+    last = trace[-1]
+    depth, anc = trj.tree_from_parents(last["parent"])
+    i32 = lambda a: torch.from_numpy(np.ascontiguousarray(a, dtype=np.int32)).to(dev)
+    d_tok, d_par, d_dep, d_off = i32(last["tokens"]), i32(last["parent"]), i32(depth), i32([0, TREE_ROWS])
+    d_anc = torch.from_numpy(anc.view(np.int64)).to(dev)
+    seq0 = model.seq_len.clone()
+    s_now = int(seq0[0])
+    pred = torch.empty(TREE_ROWS, dtype=torch.int32, device=dev)
+    acc = {"k_acc": torch.empty(1, dtype=torch.int32, device=dev), "bonus": torch.empty(1, dtype=torch.int32, device=dev),
+           "path": torch.empty(1, trj.PATH_STRIDE, dtype=torch.int32, device=dev)}
+
+    def resident_step():
+        model.seq_len.copy_(seq0)
+        model.verify_step(d_tok, d_par, d_dep, d_anc, d_off, max_rows=TREE_ROWS, max_len=s_now + TREE_ROWS, node_argmax=pred)
+        model.accept(d_tok, d_par, d_dep, d_off, pred, out=acc)
+        model.compact_kv(acc["k_acc"], acc["path"])
+
+    for _ in range(max(args.warmup, 3)):
+        resident_step()
+    torch.cuda.synchronize()
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    # ---- timed region 1: inputs resident in HBM
+    sampler = ClockSampler(local_rank)
+    barrier()
+    sampler.start()
+    launches0 = trj.launch_count()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(args.steps):
+        resident_step()
+    e1.record()
+    barrier()
+    launches = trj.launch_count() - launches0
+    ms_total = e0.elapsed_time(e1)
+
+    # ---- timed region 2: end to end through trj_step_host (host ints in, host result out)
+    committed = [int(t) for t in prompt] + [int(x) for x in []]
+    model.seq_len.zero_()
+    first = model.prefill(i32(prompt))
+    committed = [int(t) for t in prompt] + [int(first.item())]
+    window = np.array([committed[int(d) % len(committed)] for d in draw(0, WIDTH)], np.int32)
+    e2e_steps, mat = [], []
+    for step in range(1, max(args.warmup, 3) + args.steps + 1):
+        if step == max(args.warmup, 3) + 1:
+            barrier()
+            t0 = time.perf_counter()
+        draws = np.asarray(draw(step, WIDTH + N_BRANCHES * BRANCH_LEN), np.int64)
+        branches = trj.retrieve(committed, N_BRANCHES, BRANCH_LEN, draws[WIDTH:])
+        res = model.step_host(committed[-1], window, branches, max_len=len(committed) - 1 + TREE_ROWS)
+        committed += [int(res["tokens"][r]) for r in res["path"][1:]] + [int(res["bonus"])]
+        window = trj.refill_window(res["parent"], res["node_argmax"], int(res["path"][-1]), WIDTH, committed, draws[:WIDTH])
+        mat.append(res["k_acc"] + 1)
+    torch.cuda.synchronize()
+    e2e_s = time.perf_counter() - t0
+    barrier()
+    clocks = sampler.stop()
+
+    # ---- per-kernel device time of the same step (profiled pass, not part of `value`)
+    model.profile_enable(True)
+    for _ in range(args.steps):
+        resident_step()
+    torch.cuda.synchronize()
+    prof = model.profile_read()
+    model.profile_enable(False)
+
+    # ---- aggregate over ranks: max time, summed units
+    if world > 1:
+        t = torch.tensor([ms_total, e2e_s], dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms_total, e2e_s = float(t[0]), float(t[1])
+        n = torch.tensor([launches], dtype=torch.int64, device=dev)
+        dist.all_reduce(n, op=dist.ReduceOp.SUM)
+        launches = int(n[0])
+    if rank != 0:
+        return
+    ms_step = ms_total / args.steps
+    value = world * DRAFTS / (ms_step / 1e3)
+    e2e_value = world * DRAFTS * args.steps / e2e_s
+
+    gemm_ms, gemm_launches = prof["gemm"]
+    gemm_ms_step = gemm_ms / args.steps
+    gbytes = gemm_bytes_per_step(cfg, TREE_ROWS)
+    achieved = gbytes / (gemm_ms_step / 1e3) / 1e9 if gemm_ms_step > 0 else None
+    roofline = {"bound": "hbm", "kernel": "projection GEMMs (all %d launches of a step)" % (gemm_launches // args.steps),
+                "achieved": achieved, "peak": peaks["hbm_gbs"], "peak_source": peaks["source"], "unit": "GB/s",
+                "frac": achieved / peaks["hbm_gbs"] if achieved else None,
+                "traffic": GEMM_TRAFFIC_BYTES_PER_STEP, "algorithmic_bytes_per_step": gbytes,
+                "device_ms_per_step": gemm_ms_step}
+    step_ms_prof = sum(v[0] for v in prof.values()) / args.steps
+    breakdown = {k: {"ms_per_step": round(v[0] / args.steps, 4), "launches_per_step": v[1] // args.steps} for k, v in prof.items()}
+
+    line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+            "ms_per_step": ms_step, "verify_step_us": ms_step * 1e3, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "bf16", "data": "synthetic (seeded random weights, prompt and drafts)",
+            "config": workload_config(cfg, "13.2 GB of weights per step, far larger than the 126 MB L2"),
+            "clocks": clocks, "gpu_launches": launches,
+            "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": trj.STEP_H2D_BYTES,
+                    "d2h_bytes_per_step": trj.STEP_D2H_BYTES, "ms_per_step": 1e3 * e2e_s / args.steps,
+                    "tokens_committed_per_step": sum(mat[-args.steps:]) / args.steps},
+            "roofline": roofline, "kernel_breakdown": breakdown, "profiled_step_ms": step_ms_prof}
+    if world == 1:
+        if not args.no_attention:
+            line["tree_attention"] = bench_tree_attention(trj, torch, peaks, max(args.steps, 5), 3)
+        if not args.no_cpu:
+            t_full, detail = oracle_sample(synth.LLAMA7B)
+            line["cpu_baseline"] = {"value": DRAFTS / t_full, "unit": UNIT, "cores": cpu_threads(), "kind": "oracle",
+                                    "sample": "one verification step of layers 0-1 of 32 plus the LM head (33 rows, "
+                                              "512-row cache); layer time scaled by 16", "s_per_step_scaled": round(t_full, 2),
+                                    **detail}
+    print(json.dumps(line), flush=True)
+    model.close()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--layers", type=int, default=0, help="debug: fewer layers than the 7B shape (invalidates the number)")
+    ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-oracle baseline leg")
+    ap.add_argument("--no-attention", action="store_true", help="skip the op-level tree-attention leg")
+    args = ap.parse_args()
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if args.impl == "reference":
+        args.steps = min(args.steps, 3)
+        args.warmup = min(args.warmup, 1)
+        run_reference(args, rank, world)
+        return
+    if world > 1:
+        import torch
+        import torch.distributed as dist
+        torch.cuda.set_device(local_rank)
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    try:
+        run_ours(args, rank, world, local_rank)
+    finally:
+        if world > 1:
+            import torch.distributed as dist
+            dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

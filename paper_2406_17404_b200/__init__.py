@@ -19,6 +19,9 @@ LIB_PATH = os.path.join(_HERE, "libtrj.so")
 MAX_ROWS = 128
 MAX_BATCH = 64
 PATH_STRIDE = 128
+# bytes trj_step_host moves per call: tokens/parent/depth/row_off + ancestor words in, predictions/k/bonus/path out
+STEP_H2D_BYTES = (3 * MAX_ROWS + 4) * 4 + MAX_ROWS * 2 * 8
+STEP_D2H_BYTES = (MAX_ROWS + 2 + PATH_STRIDE) * 4
 F32, BF16 = 0, 1
 
 _lib = None
@@ -346,11 +349,13 @@ class Model:
         return first
 
     def verify_step(self, tokens, parent, depth, anc, row_off, *, max_rows: int, max_len: int,
-                    want_logits: bool = False, want_margin: bool = False, stream=None):
-        """trj_verify_step: dict(node_argmax, margin | None, logits | None)."""
+                    want_logits: bool = False, want_margin: bool = False, node_argmax=None, stream=None):
+        """trj_verify_step: dict(node_argmax, margin | None, logits | None).  ``node_argmax`` may be a
+        preallocated int32 tensor [rows]."""
         torch = _torch()
         rows, batch = tokens.numel(), row_off.numel() - 1
-        node_argmax = torch.empty(rows, dtype=torch.int32, device=self.device)
+        if node_argmax is None:
+            node_argmax = torch.empty(rows, dtype=torch.int32, device=self.device)
         margin = torch.empty(rows, dtype=torch.float32, device=self.device) if want_margin else None
         logits = torch.empty(rows, self.cfg.vocab, dtype=torch.float32, device=self.device) if want_logits else None
         _check(lib().trj_verify_step(
@@ -361,12 +366,15 @@ class Model:
             _dev(logits) if want_logits else None, _stream(stream)))
         return {"node_argmax": node_argmax, "margin": margin, "logits": logits}
 
-    def accept(self, tokens, parent, depth, row_off, node_argmax, stream=None):
-        """trj_accept: dict(k_acc [B], path [B, PATH_STRIDE], bonus [B])."""
+    def accept(self, tokens, parent, depth, row_off, node_argmax, out=None, stream=None):
+        """trj_accept: dict(k_acc [B], path [B, PATH_STRIDE], bonus [B]); ``out`` may hold preallocated ones."""
         torch = _torch()
         batch = row_off.numel() - 1
         i32 = dict(dtype=torch.int32, device=self.device)
-        k_acc, bonus, path = torch.empty(batch, **i32), torch.empty(batch, **i32), torch.empty(batch, PATH_STRIDE, **i32)
+        if out is not None:
+            k_acc, bonus, path = out["k_acc"], out["bonus"], out["path"]
+        else:
+            k_acc, bonus, path = torch.empty(batch, **i32), torch.empty(batch, **i32), torch.empty(batch, PATH_STRIDE, **i32)
         _check(lib().trj_accept(self._handle, _dev(tokens, torch.int32), _dev(parent, torch.int32),
                                 _dev(depth, torch.int32), _dev(row_off, torch.int32), batch, tokens.numel(),
                                 _dev(node_argmax, torch.int32), _dev(k_acc), _dev(path), _dev(bonus), _stream(stream)))
