@@ -266,14 +266,15 @@ def compact_rows(k_cache, v_cache, seq_len, k_acc, path, stream=None) -> None:
 
 
 def gemm(x, w, *, out=None, workspace=None, stream=None):
-    """trj_gemm: y [M, N] fp32 = x [M, K] . w [N, K]^T."""
+    """trj_gemm: y [M, N] fp32 = x [M, K] . w [N, K]^T.  The first int32 of ``workspace`` is a device
+    status word (0, or 4 after a bounded device-side wait expired); a fresh workspace is zeroed here."""
     torch = _torch()
     m, k = x.shape
     n = w.shape[0]
     if out is None:
         out = torch.empty(m, n, dtype=torch.float32, device=x.device)
     if workspace is None:
-        workspace = _scratch(lib().trj_gemm_workspace(m, n, k), x.device)
+        workspace = _scratch(lib().trj_gemm_workspace(m, n, k), x.device, zero=True)
     _check(lib().trj_gemm(_dev(x, name="x"), _dev(w, x.dtype, "w"), _dev(out, torch.float32, "out"), m, n, k,
                           _dtype_code(x), _dev(workspace, torch.uint8), workspace.numel(), _stream(stream)))
     return out

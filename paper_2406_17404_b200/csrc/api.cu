@@ -3,6 +3,7 @@
 #include <cmath>
 #include <cstring>
 #include <new>
+#include <utility>
 #include <vector>
 #include "trj_internal.h"
 
@@ -94,8 +95,7 @@ extern "C" trj_status trj_compact_rows(void* k_cache, void* v_cache, int32_t L, 
 }
 
 extern "C" size_t trj_gemm_workspace(int32_t M, int32_t N, int32_t K) {
-    (void)M; (void)N; (void)K;
-    return 256;
+    return gemm_tc_workspace(M, N, K);
 }
 
 extern "C" trj_status trj_gemm(const void* x, const void* w, float* y, int32_t M, int32_t N, int32_t K,
@@ -104,7 +104,7 @@ extern "C" trj_status trj_gemm(const void* x, const void* w, float* y, int32_t M
     TRJ_REQUIRE(dtype_ok(dtype), TRJ_EINVAL, "gemm: unknown dtype %d", dtype);
     TRJ_REQUIRE(M >= 1 && N >= 1 && K >= 1, TRJ_EINVAL, "gemm: bad sizes");
     TRJ_REQUIRE(workspace && workspace_bytes >= trj_gemm_workspace(M, N, K), TRJ_ECAPACITY, "gemm: workspace too small");
-    TRJ_CHECK_CUDA(launch_gemm_simt(x, nullptr, w, y, M, N, K, dtype, (cudaStream_t)stream));
+    TRJ_CHECK_CUDA(launch_gemm(x, nullptr, w, y, M, N, K, dtype, workspace, workspace_bytes, (cudaStream_t)stream));
     return TRJ_OK;
 }
 
@@ -152,7 +152,10 @@ size_t carve(const trj_model_cfg& c, void* ws, trj_ctx* ctx) {
     char* argmax_ws = cv.take<char>(argmax_workspace_bytes(rows, c.max_batch));
     const size_t attn_bytes = trj_tree_attention_workspace(rows, c.max_batch, c.n_heads, c.head_dim, c.max_seq);
     char* attn_ws = cv.take<char>(attn_bytes);
-    const size_t gemm_bytes = trj_gemm_workspace(rows, (int32_t)std::max(wide, (size_t)c.vocab), std::max(c.d_model, c.d_ff));
+    size_t gemm_bytes = 256;
+    for (auto nk : {std::pair<int, int>{3 * HD, c.d_model}, {c.d_model, HD}, {2 * c.d_ff, c.d_model},
+                    {c.d_model, c.d_ff}, {c.vocab, c.d_model}})
+        gemm_bytes = std::max(gemm_bytes, gemm_tc_workspace(rows, nk.first, nk.second));
     char* gemm_ws = cv.take<char>(gemm_bytes);
     int32_t* chain_depth = cv.take<int32_t>(TRJ_MAX_ROWS);
     uint64_t* chain_anc = cv.take<uint64_t>(TRJ_MAX_ROWS * 2);
@@ -221,25 +224,28 @@ trj_status forward(trj_ctx* ctx, void* k_cache, void* v_cache, int32_t b0, const
         char* v_slab = (char*)v_cache + ((size_t)l * c.max_batch + b0) * seq_stride;
         LAUNCH(PROF_ELEMENTWISE, launch_add_rmsnorm(ctx->h, l == 0 ? nullptr : ctx->y, ctx->attn_norm[l], ctx->x, ctx->x_lo,
                                                     c.dtype, M, d, c.rms_eps, st));
-        LAUNCH(PROF_GEMM, launch_gemm_simt(ctx->x, ctx->x_lo, ctx->wqkv[l], ctx->y, M, 3 * HD, d, c.dtype, st));
+        LAUNCH(PROF_GEMM, launch_gemm(ctx->x, ctx->x_lo, ctx->wqkv[l], ctx->y, M, 3 * HD, d, c.dtype, ctx->gemm_ws, ctx->gemm_ws_bytes, st));
         LAUNCH(PROF_ROPE, launch_rope_kv_write(ctx->y, ctx->inv_freq, depth, bt, ctx->q, k_slab, v_slab, c.dtype,
                                                c.n_heads, c.head_dim, c.max_seq, st));
         // the attention output is a bf16 tensor of its own right (no low half)
         LAUNCH(PROF_ATTENTION, launch_tree_attention_generic(ctx->q, k_slab, v_slab, anc, anc_words, bt, c.n_heads,
                                                              c.head_dim, c.max_seq, c.dtype, ctx->x, st));
-        LAUNCH(PROF_GEMM, launch_gemm_simt(ctx->x, nullptr, ctx->wo[l], ctx->y, M, d, HD, c.dtype, st));
+        LAUNCH(PROF_GEMM, launch_gemm(ctx->x, nullptr, ctx->wo[l], ctx->y, M, d, HD, c.dtype, ctx->gemm_ws, ctx->gemm_ws_bytes, st));
         LAUNCH(PROF_ELEMENTWISE, launch_add_rmsnorm(ctx->h, ctx->y, ctx->mlp_norm[l], ctx->x, ctx->x_lo, c.dtype, M, d,
                                                     c.rms_eps, st));
-        LAUNCH(PROF_GEMM, launch_gemm_simt(ctx->x, ctx->x_lo, ctx->w_gate_up[l], ctx->y, M, 2 * c.d_ff, d, c.dtype, st));
+        LAUNCH(PROF_GEMM, launch_gemm(ctx->x, ctx->x_lo, ctx->w_gate_up[l], ctx->y, M, 2 * c.d_ff, d, c.dtype, ctx->gemm_ws,
+                                      ctx->gemm_ws_bytes, st));
         LAUNCH(PROF_ELEMENTWISE, launch_swiglu(ctx->y, ctx->act, ctx->act_lo, c.dtype, M, c.d_ff, st));
-        LAUNCH(PROF_GEMM, launch_gemm_simt(ctx->act, ctx->act_lo, ctx->w_down[l], ctx->y, M, d, c.d_ff, c.dtype, st));
+        LAUNCH(PROF_GEMM, launch_gemm(ctx->act, ctx->act_lo, ctx->w_down[l], ctx->y, M, d, c.d_ff, c.dtype, ctx->gemm_ws,
+                                      ctx->gemm_ws_bytes, st));
     }
     LAUNCH(PROF_ELEMENTWISE, launch_add_rmsnorm(ctx->h, ctx->y, ctx->final_norm, ctx->x, ctx->x_lo, c.dtype, M, d,
                                                 c.rms_eps, st));
     if (lm_rows > 0) {
         const size_t off = (size_t)lm_first * d * es;
-        LAUNCH(PROF_GEMM, launch_gemm_simt((char*)ctx->x + off, ctx->x_lo ? (char*)ctx->x_lo + off : nullptr, ctx->lm_head,
-                                           ctx->logits + (size_t)lm_first * c.vocab, lm_rows, c.vocab, d, c.dtype, st));
+        LAUNCH(PROF_GEMM, launch_gemm((char*)ctx->x + off, ctx->x_lo ? (char*)ctx->x_lo + off : nullptr, ctx->lm_head,
+                                      ctx->logits + (size_t)lm_first * c.vocab, lm_rows, c.vocab, d, c.dtype,
+                                      ctx->gemm_ws, ctx->gemm_ws_bytes, st));
     }
     return TRJ_OK;
 }

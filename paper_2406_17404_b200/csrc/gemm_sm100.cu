@@ -1,0 +1,329 @@
+// Projection GEMM for sm_100a: y[M][N] = (x + x_lo)[M][K] . w[N][K]^T with M <= 128 tree rows.
+//
+// The verification step multiplies a handful of rows (tens) by every weight matrix, so the job is
+// to stream the weights from HBM once, at full bandwidth.  The roles are swapped with respect to a
+// usual GEMM: a CTA owns 128 weight rows (the M dimension of one tcgen05.mma, accumulator lanes in
+// TMEM) and ALL activation rows are the N dimension (columns of the accumulator).  Weight tiles
+// [128 x 64] and the activation tile [rows x 64] arrive by TMA into 128-byte-swizzled shared memory,
+// one elected thread issues the MMAs, and the 128 threads read the accumulator back with tcgen05.ld.
+// In bf16 models the activations come as a bf16 pair hi + lo (lo = rounding error of hi); the two
+// halves are simply further accumulator columns that the epilogue adds, so the product keeps fp32-like
+// input precision at no cost in weight traffic.  K is split across CTAs when a matrix has too few
+// 128-row tiles to keep every SM loading; partial sums go to a workspace and are added in a fixed
+// order, so results do not depend on scheduling.
+#include <cuda.h>
+#include <mutex>
+#include "trj_internal.h"
+
+namespace trj {
+namespace {
+
+constexpr int TC_BM = 128;            // weight rows per CTA = UMMA M
+constexpr int TC_BK = 64;             // bf16 elements per stage row = one 128-byte swizzle span
+constexpr int TC_THREADS = 128;
+constexpr int TC_MAX_STAGES = 8;
+constexpr uint32_t TC_A_BYTES = TC_BM * TC_BK * 2;
+constexpr uint32_t WAIT_LIMIT = 1u << 21;   // polls before a wait gives up (well over 100 ms)
+
+struct TcParams {
+    int M, N, K;
+    int m_pad;          // activation rows rounded up to 16
+    int halves;         // 1: x only, 2: x and x_lo
+    int n_mma;          // accumulator columns = m_pad * halves
+    int tmem_cols;      // power of two >= max(32, n_mma)
+    int kblocks;        // K / 64
+    int splits, stages;
+    float* out;         // [splits][M][N]
+    int* status;        // device word: 0, or TRJ_ETIMEOUT once a wait expired
+};
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+                 : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok != 0;
+}
+// Bounded wait: gives up after WAIT_LIMIT polls or as soon as another role of the CTA gave up.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* status) {
+    for (uint32_t i = 0; i < WAIT_LIMIT; ++i) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if (i > 32) {
+            if (*abort_flag) return false;
+            __nanosleep(64);
+        }
+    }
+    *abort_flag = 1;
+    atomicExch(status, (int)TRJ_ETIMEOUT);
+    return false;
+}
+
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int c_inner, int c_outer, uint32_t bar) {
+    asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+                 ::"r"(dst), "l"(map), "r"(c_inner), "r"(c_outer), "r"(bar) : "memory");
+}
+
+// Shared-memory matrix descriptor of a K-major tile with 128-byte swizzle: rows are 128 bytes apart,
+// groups of 8 rows 1024 bytes apart (stride byte offset), descriptor version 1 (sm_100).
+__device__ __forceinline__ uint64_t umma_desc_sw128(uint32_t smem_addr) {
+    uint64_t d = 0;
+    d |= (uint64_t)((smem_addr & 0x3FFFF) >> 4);          // start address, 16-byte units
+    d |= (uint64_t)1 << 16;                               // leading byte offset (unused with swizzle)
+    d |= (uint64_t)(1024 >> 4) << 32;                     // stride byte offset
+    d |= (uint64_t)1 << 46;                               // descriptor version
+    d |= (uint64_t)2 << 61;                               // 128-byte swizzle
+    return d;
+}
+
+// Instruction descriptor of kind::f16: bf16 x bf16 -> fp32, both operands K-major, shape 128 x n.
+__device__ __forceinline__ uint32_t umma_idesc_bf16(int n) {
+    return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(TC_BM >> 4) << 24);
+}
+
+__device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
+    asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+                 "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+                 ::"r"(tmem_d), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
+}
+__device__ __forceinline__ void umma_commit(uint32_t bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, float* v) {
+    uint32_t r[16];
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+                   "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+                 : "r"(taddr) : "memory");
+#pragma unroll
+    for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]);
+}
+
+__global__ void __launch_bounds__(TC_THREADS) gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w,
+                                                             const __grid_constant__ CUtensorMap map_x,
+                                                             const __grid_constant__ CUtensorMap map_xlo,
+                                                             const TcParams p) {
+    extern __shared__ uint8_t smem_raw[];
+    __shared__ __align__(8) uint64_t bars[2 * TC_MAX_STAGES + 1];
+    __shared__ uint32_t tmem_base_slot;
+    __shared__ int abort_flag;
+
+    const uint32_t tiles_base = (smem_u32(smem_raw) + 1023u) & ~1023u;     // swizzled tiles need 1024-byte alignment
+    const uint32_t b_bytes = (uint32_t)p.n_mma * TC_BK * 2;
+    const uint32_t stage_bytes = TC_A_BYTES + b_bytes;
+    const uint32_t full0 = smem_u32(&bars[0]), empty0 = smem_u32(&bars[TC_MAX_STAGES]);
+    const uint32_t accum_bar = smem_u32(&bars[2 * TC_MAX_STAGES]);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int n0 = blockIdx.x * TC_BM;
+    const int kb0 = (int)((long long)blockIdx.y * p.kblocks / p.splits);
+    const int kb1 = (int)((long long)(blockIdx.y + 1) * p.kblocks / p.splits);
+    const int nkb = kb1 - kb0;
+
+    if (threadIdx.x == 0) {
+        abort_flag = 0;
+        for (int s = 0; s < p.stages; ++s) { mbar_init(full0 + 8 * s, 1); mbar_init(empty0 + 8 * s, 1); }
+        mbar_init(accum_bar, 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 1) {      // one warp allocates the accumulator columns
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
+                     ::"r"(smem_u32(&tmem_base_slot)), "r"((uint32_t)p.tmem_cols) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    const uint32_t tmem_base = tmem_base_slot;
+
+    if (threadIdx.x == 0) {
+        // ---------------- producer: stream weight and activation tiles
+        for (int i = 0; i < nkb; ++i) {
+            const int s = i % p.stages;
+            const uint32_t phase = (uint32_t)(i / p.stages) & 1u;
+            if (!mbar_wait(empty0 + 8 * s, phase ^ 1u, &abort_flag, p.status)) break;
+            const uint32_t a_dst = tiles_base + s * stage_bytes, b_dst = a_dst + TC_A_BYTES;
+            const uint32_t bar = full0 + 8 * s;
+            mbar_expect_tx(bar, stage_bytes);
+            const int k = (kb0 + i) * TC_BK;
+            tma_load_2d(a_dst, &map_w, k, n0, bar);
+            tma_load_2d(b_dst, &map_x, k, 0, bar);
+            if (p.halves == 2) tma_load_2d(b_dst + (uint32_t)p.m_pad * TC_BK * 2, &map_xlo, k, 0, bar);
+        }
+    } else if (threadIdx.x == 32) {
+        // ---------------- MMA issuer
+        const uint32_t idesc = umma_idesc_bf16(p.n_mma);
+        bool ok = true;
+        for (int i = 0; i < nkb && ok; ++i) {
+            const int s = i % p.stages;
+            const uint32_t phase = (uint32_t)(i / p.stages) & 1u;
+            ok = mbar_wait(full0 + 8 * s, phase, &abort_flag, p.status);
+            if (!ok) break;
+            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+            const uint32_t a_addr = tiles_base + s * stage_bytes;
+            const uint64_t a_desc = umma_desc_sw128(a_addr), b_desc = umma_desc_sw128(a_addr + TC_A_BYTES);
+#pragma unroll
+            for (int kk = 0; kk < TC_BK / 16; ++kk)      // 16 bf16 = 32 bytes = 2 descriptor units per MMA
+                umma_bf16(tmem_base, a_desc + 2 * kk, b_desc + 2 * kk, idesc, (i > 0 || kk > 0) ? 1u : 0u);
+            umma_commit(empty0 + 8 * s);                 // frees the stage once these MMAs have read it
+        }
+        if (ok) umma_commit(accum_bar);                  // accumulator complete
+    }
+    __syncwarp();
+
+    // ---------------- epilogue: lane = weight row, columns = activation rows (hi half, then lo half)
+    const bool ready = mbar_wait(accum_bar, 0, &abort_flag, p.status);
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    if (ready) {
+        const int n = n0 + warp * 32 + lane;
+        const uint32_t taddr = tmem_base + ((uint32_t)(warp * 32) << 16);
+        float* out = p.out + (size_t)blockIdx.y * p.M * p.N;
+        for (int c0 = 0; c0 < p.m_pad; c0 += 16) {
+            float hi[16], lo[16];
+            tmem_ld16(taddr + c0, hi);
+            if (p.halves == 2) tmem_ld16(taddr + p.m_pad + c0, lo);
+            asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+            for (int j = 0; j < 16; ++j) {
+                const int m = c0 + j;
+                if (m < p.M && n < p.N) out[(size_t)m * p.N + n] = p.halves == 2 ? hi[j] + lo[j] : hi[j];
+            }
+        }
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    if (abort_flag) {                                    // let copies that are still in flight land before the CTA leaves
+        for (int i = 0; i < 64; ++i) __nanosleep(1000);
+        __syncthreads();
+    }
+    if (warp == 1)
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)p.tmem_cols) : "memory");
+}
+
+// y[i] = sum_s part[s][i], fixed order.
+__global__ void reduce_splits_kernel(const float4* __restrict__ part, float4* __restrict__ y, size_t n4, int splits) {
+    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n4; i += (size_t)gridDim.x * blockDim.x) {
+        float4 a = part[i];
+        for (int s = 1; s < splits; ++s) {
+            const float4 b = part[(size_t)s * n4 + i];
+            a.x += b.x; a.y += b.y; a.z += b.z; a.w += b.w;
+        }
+        y[i] = a;
+    }
+}
+
+// ---------------------------------------------------------------- host side
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                  const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn() {
+    static EncodeTiledFn fn = nullptr;
+    static std::once_flag once;
+    std::call_once(once, [] {
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+            q == cudaDriverEntryPointSuccess)
+            fn = (EncodeTiledFn)p;
+    });
+    return fn;
+}
+
+// bf16 matrix [rows][K] row-major -> tiles of [box_rows][64] with 128-byte swizzle, zero fill out of range.
+bool make_map(CUtensorMap* map, const void* base, int rows, int K, int box_rows) {
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) return false;
+    const cuuint64_t dims[2] = {(cuuint64_t)K, (cuuint64_t)rows};
+    const cuuint64_t strides[1] = {(cuuint64_t)K * 2};
+    const cuuint32_t box[2] = {(cuuint32_t)TC_BK, (cuuint32_t)box_rows};
+    const cuuint32_t estr[2] = {1, 1};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+int round_up(int x, int a) { return (x + a - 1) / a * a; }
+
+}  // namespace
+
+bool gemm_tc_supported(const void* x, const void* x_lo, const void* w, const float* y, int32_t M, int32_t N, int32_t K,
+                       int32_t dtype) {
+    if (dtype != TRJ_BF16 || M < 1 || M > TRJ_MAX_ROWS || K % TC_BK != 0 || N < 4 || N % 4 != 0) return false;
+    if (((uintptr_t)x | (uintptr_t)x_lo | (uintptr_t)w | (uintptr_t)y) % 16 != 0) return false;
+    return encode_fn() != nullptr;
+}
+
+int gemm_tc_splits(int32_t N, int32_t K) {
+    const int tiles = (N + TC_BM - 1) / TC_BM, kblocks = K / TC_BK;
+    const int resident = 296;                      // two CTAs of this kernel fit on each of the 148 SMs
+    int s = resident / tiles;
+    if (s > kblocks / 4) s = kblocks / 4;          // keep at least four k-blocks per CTA
+    if (s > 16) s = 16;
+    return s < 1 ? 1 : s;
+}
+
+// Workspace: a 256-byte header whose first word is the device status, then the split-K partial sums.
+size_t gemm_tc_workspace(int32_t M, int32_t N, int32_t K) {
+    if (K % TC_BK != 0 || K < TC_BK) return 256;
+    const int s = gemm_tc_splits(N, K);
+    return 256 + (s > 1 ? align_up((size_t)s * M * N * sizeof(float), 256) : 0);
+}
+
+cudaError_t launch_gemm_tc(const void* x, const void* x_lo, const void* w, float* y, int32_t M, int32_t N, int32_t K,
+                           void* workspace, cudaStream_t st) {
+    int* status = (int*)workspace;
+    workspace = (char*)workspace + 256;
+    static std::once_flag once;
+    static cudaError_t attr_err = cudaSuccess;
+    std::call_once(once, [] {
+        attr_err = cudaFuncSetAttribute(gemm_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024);
+    });
+    if (attr_err != cudaSuccess) return attr_err;
+    TcParams p;
+    p.M = M; p.N = N; p.K = K;
+    p.m_pad = round_up(M, 16);
+    p.halves = x_lo ? 2 : 1;
+    p.n_mma = p.m_pad * p.halves;
+    p.tmem_cols = 32;
+    while (p.tmem_cols < p.n_mma) p.tmem_cols *= 2;
+    p.kblocks = K / TC_BK;
+    p.splits = gemm_tc_splits(N, K);
+    const size_t stage = TC_A_BYTES + (size_t)p.n_mma * TC_BK * 2;
+    size_t budget = 108 * 1024;                    // two CTAs per SM when three stages fit, else one CTA per SM
+    if (3 * stage > budget) budget = 216 * 1024;
+    p.stages = (int)(budget / stage);
+    if (p.stages > TC_MAX_STAGES) p.stages = TC_MAX_STAGES;
+    if (p.stages < 2) return cudaErrorInvalidConfiguration;
+    p.out = p.splits > 1 ? (float*)workspace : y;
+    p.status = status;
+    CUtensorMap map_w, map_x, map_xlo;
+    if (!make_map(&map_w, w, N, K, TC_BM) || !make_map(&map_x, x, M, K, p.m_pad) ||
+        !make_map(&map_xlo, x_lo ? x_lo : x, M, K, p.m_pad))
+        return cudaErrorInvalidValue;
+    count_launch();
+    dim3 grid((N + TC_BM - 1) / TC_BM, p.splits);
+    gemm_tc_kernel<<<grid, TC_THREADS, p.stages * stage + 1024, st>>>(map_w, map_x, map_xlo, p);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess || p.splits == 1) return e;
+    count_launch();
+    const size_t n4 = (size_t)M * N / 4;           // N % 4 == 0 is part of gemm_tc_supported
+    reduce_splits_kernel<<<(unsigned)((n4 + 255) / 256 < 592 ? (n4 + 255) / 256 : 592), 256, 0, st>>>(
+        (const float4*)workspace, (float4*)y, n4, p.splits);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_gemm(const void* x, const void* x_lo, const void* w, float* y, int32_t M, int32_t N, int32_t K,
+                        int32_t dtype, void* workspace, size_t workspace_bytes, cudaStream_t st) {
+    if (workspace && workspace_bytes >= gemm_tc_workspace(M, N, K) && ((uintptr_t)workspace % 256) == 0 &&
+        gemm_tc_supported(x, x_lo, w, y, M, N, K, dtype))
+        return launch_gemm_tc(x, x_lo, w, y, M, N, K, workspace, st);
+    return launch_gemm_simt(x, x_lo, w, y, M, N, K, dtype, st);
+}
+
+}  // namespace trj

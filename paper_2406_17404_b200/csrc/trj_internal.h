@@ -49,6 +49,18 @@ cudaError_t launch_add_rmsnorm(float* h, const float* add, const float* gain, vo
 // y[M][N] fp32 = (x + x_lo)[M][K] . w[N][K]^T (x_lo may be null), plain shared-memory tiled FMA kernel.
 cudaError_t launch_gemm_simt(const void* x, const void* x_lo, const void* w, float* y, int32_t M, int32_t N,
                              int32_t K, int32_t dtype, cudaStream_t st);
+// tcgen05 / TMA projection kernel (gemm_sm100.cu): bf16, M <= 128 rows, K a multiple of 64.  The workspace
+// (gemm_tc_workspace bytes, 256-byte aligned) starts with a status word that a device-side wait sets to
+// TRJ_ETIMEOUT if it expires; the rest holds split-K partial sums.
+bool gemm_tc_supported(const void* x, const void* x_lo, const void* w, const float* y, int32_t M, int32_t N, int32_t K,
+                       int32_t dtype);
+size_t gemm_tc_workspace(int32_t M, int32_t N, int32_t K);
+cudaError_t launch_gemm_tc(const void* x, const void* x_lo, const void* w, float* y, int32_t M, int32_t N, int32_t K,
+                           void* workspace, cudaStream_t st);
+// Picks the tcgen05 kernel when the shape allows it, the plain kernel otherwise.
+cudaError_t launch_gemm(const void* x, const void* x_lo, const void* w, float* y, int32_t M, int32_t N, int32_t K,
+                        int32_t dtype, void* workspace, size_t workspace_bytes, cudaStream_t st);
+
 // Rotary embedding of q and k at position seq_len[b] + depth[row]; q -> q_out [rows][H][D];
 // k, v -> cache rows seq_len[b] + local row of the layer slab [B][H][max_seq][D].
 cudaError_t launch_rope_kv_write(const float* qkv, const double* inv_freq, const int32_t* depth,

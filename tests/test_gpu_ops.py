@@ -186,14 +186,20 @@ def test_compaction_long_chain_overlapping_ranges(trj):
 
 
 # ----------------------------------------------------------------------------- projection GEMM
-@pytest.mark.parametrize("dtype,m,n,k", [("bf16", 33, 512, 4096), ("bf16", 1, 130, 688), ("f32", 11, 1376, 256),
-                                         ("bf16", 128, 257, 1104), ("f32", 70, 64, 688)])
+@pytest.mark.parametrize("dtype,m,n,k", [
+    ("bf16", 33, 512, 4096), ("bf16", 1, 130, 688), ("f32", 11, 1376, 256), ("bf16", 128, 257, 1104), ("f32", 70, 64, 688),
+    # shapes the tcgen05 kernel takes: K % 64 == 0, N % 4 == 0, M <= 128; ragged N tiles, one k-block, deep split-K
+    ("bf16", 48, 384, 64), ("bf16", 17, 132, 128), ("bf16", 33, 12288, 4096), ("bf16", 128, 4096, 11008),
+    ("bf16", 1, 32000, 4096), ("bf16", 64, 22016, 4096), ("bf16", 16, 128, 8192), ("bf16", 100, 1000, 192),
+])
 def test_gemm(trj, dtype, m, n, k):
     g = synth.stream(m * n, "gemm")
     x = g.standard_normal((m, k), dtype=np.float32)
     w = g.standard_normal((n, k), dtype=np.float32) * 0.02
     if dtype == "bf16":
         x, w = synth.round_bf16(x), synth.round_bf16(w)
-    y = trj.gemm(to_dev(x, dtype), to_dev(w, dtype)).cpu().numpy()
+    ws = torch.zeros(trj.lib().trj_gemm_workspace(m, n, k), dtype=torch.uint8, device="cuda")
+    y = trj.gemm(to_dev(x, dtype), to_dev(w, dtype), workspace=ws).cpu().numpy()
+    assert int(ws[:4].view(torch.int32)[0]) == 0           # no device-side wait expired
     ref = x.astype(np.float64) @ w.astype(np.float64).T
     assert np.abs(y - ref).max() <= 1e-4 * max(1.0, np.abs(ref).max())
