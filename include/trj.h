@@ -151,7 +151,9 @@ trj_status trj_refill_window(const int32_t* parent, const int32_t* node_argmax, 
  *   max_rows   upper bound of rows per sequence (<= TRJ_MAX_ROWS)
  *   max_len    upper bound of seq_len[b] + rows of b, <= max_seq (sizes the KV split)
  *   workspace  dev, at least trj_tree_attention_workspace(...) bytes, 256-byte aligned;
- *              holds split-KV partial results, contents undefined afterwards.
+ *              holds split-KV partial results, contents undefined afterwards.  Its first
+ *              int32 is a status word: the kernels set it to TRJ_ETIMEOUT if a bounded
+ *              device-side wait expires and never clear it (zero it to be able to read it).
  * TRJ_EUNSUPPORTED for a head_dim the build has no kernel for (supported: 64, 128). */
 size_t trj_tree_attention_workspace(int32_t rows_total, int32_t B, int32_t H, int32_t D, int32_t max_len);
 trj_status trj_tree_attention(const void* q, const void* k_cache, const void* v_cache,
@@ -259,7 +261,8 @@ trj_status trj_step_host(trj_ctx* ctx, void* k_cache, void* v_cache, int32_t* se
  * The projections as a stand-alone op: y[M][N] (fp32) = x[M][K] . w[N][K]^T,
  * x and w of `dtype`, all dev.  Used by the model path for every projection
  * and exposed for measurement.  workspace: dev, >= trj_gemm_workspace(M, N, K)
- * bytes, 256-byte aligned (split-K partial sums). */
+ * bytes, 256-byte aligned (split-K partial sums); its first int32 is a status
+ * word with the same meaning as in trj_tree_attention. */
 size_t     trj_gemm_workspace(int32_t M, int32_t N, int32_t K);
 trj_status trj_gemm(const void* x, const void* w, float* y, int32_t M, int32_t N, int32_t K,
                     int32_t dtype, void* workspace, size_t workspace_bytes, void* stream);

@@ -29,8 +29,8 @@ struct Carver {
 
 // ---------------------------------------------------------------------------- op-level entry points
 extern "C" size_t trj_tree_attention_workspace(int32_t rows_total, int32_t B, int32_t H, int32_t D, int32_t max_len) {
-    (void)rows_total; (void)B; (void)H; (void)D; (void)max_len;
-    return 256;
+    (void)rows_total; (void)max_len;
+    return D == 128 ? tree_attention_tc_workspace(B, H) : 256;
 }
 
 extern "C" trj_status trj_tree_attention(const void* q, const void* k_cache, const void* v_cache,
@@ -52,8 +52,8 @@ extern "C" trj_status trj_tree_attention(const void* q, const void* k_cache, con
                 TRJ_ECAPACITY, "tree_attention: workspace too small");
     if (rows_total == 0) return TRJ_OK;
     Batch bt{seq_len, row_off, B, rows_total, max_rows, max_len};
-    TRJ_CHECK_CUDA(launch_tree_attention_generic(q, k_cache, v_cache, anc, anc_words, bt, H, D, max_seq, dtype, out,
-                                                 (cudaStream_t)stream));
+    TRJ_CHECK_CUDA(launch_tree_attention(q, k_cache, v_cache, anc, anc_words, bt, H, D, max_seq, dtype, out, workspace,
+                                         workspace_bytes, (cudaStream_t)stream));
     return TRJ_OK;
 }
 
@@ -228,8 +228,8 @@ trj_status forward(trj_ctx* ctx, void* k_cache, void* v_cache, int32_t b0, const
         LAUNCH(PROF_ROPE, launch_rope_kv_write(ctx->y, ctx->inv_freq, depth, bt, ctx->q, k_slab, v_slab, c.dtype,
                                                c.n_heads, c.head_dim, c.max_seq, st));
         // the attention output is a bf16 tensor of its own right (no low half)
-        LAUNCH(PROF_ATTENTION, launch_tree_attention_generic(ctx->q, k_slab, v_slab, anc, anc_words, bt, c.n_heads,
-                                                             c.head_dim, c.max_seq, c.dtype, ctx->x, st));
+        LAUNCH(PROF_ATTENTION, launch_tree_attention(ctx->q, k_slab, v_slab, anc, anc_words, bt, c.n_heads, c.head_dim,
+                                                     c.max_seq, c.dtype, ctx->x, ctx->attn_ws, ctx->attn_ws_bytes, st));
         LAUNCH(PROF_GEMM, launch_gemm(ctx->x, nullptr, ctx->wo[l], ctx->y, M, d, HD, c.dtype, ctx->gemm_ws, ctx->gemm_ws_bytes, st));
         LAUNCH(PROF_ELEMENTWISE, launch_add_rmsnorm(ctx->h, ctx->y, ctx->mlp_norm[l], ctx->x, ctx->x_lo, c.dtype, M, d,
                                                     c.rms_eps, st));

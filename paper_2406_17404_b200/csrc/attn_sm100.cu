@@ -1,0 +1,606 @@
+// Tree-masked attention for sm_100a (bf16, head_dim 128, up to 128 tree rows per sequence).
+//
+// Work is cut into units of one 128-key tile of one (sequence, head); the units, laid out sequence-
+// major, are dealt in equal contiguous ranges to a persistent grid of one CTA per SM, so a long prefix
+// is split over several CTAs (split-KV) and short sequences are packed several per CTA.  Inside a CTA:
+//   * one thread streams Q (per segment) and the K/V tiles with TMA into 128-byte-swizzled shared memory;
+//   * one thread issues tcgen05.mma: S = Q.K^T into TMEM (two S buffers), then O += P.V with the
+//     accumulator resident in TMEM for the whole segment;
+//   * four warps own one query row per thread (TMEM lane = row): they read S, apply the ancestor bitmask
+//     on tiles that reach the tree rows, keep an online softmax whose running maximum is only raised when
+//     a tile exceeds it by more than 2^8 (then O is rescaled in TMEM), and write P as bf16 into shared
+//     memory in the layout the second MMA reads.
+// A segment that covers all tiles of its (sequence, head) writes the normalised bf16 output itself;
+// otherwise it leaves (max, sum, O) in the workspace and a second kernel merges the pieces in a fixed
+// order.  Every wait on an mbarrier is bounded; on expiry the CTA records TRJ_ETIMEOUT and leaves.
+#include <cuda.h>
+#include <mutex>
+#include "trj_internal.h"
+
+namespace trj {
+namespace {
+
+constexpr int AT_ROWS = 128;                 // query rows per CTA = UMMA M = TMEM lanes
+constexpr int AT_KEYS = 128;                 // keys per tile
+constexpr int AT_D = 128;                    // head_dim
+constexpr int AT_THREADS = 192;              // 4 softmax warps + TMA warp + MMA warp
+constexpr uint32_t AT_SUB = 128 * 128;       // one [128 x 64 bf16] swizzled sub-tile: 16 KB
+constexpr uint32_t AT_TILE = 2 * AT_SUB;     // Q, P, a K tile or a V tile: 32 KB
+constexpr int AT_RING = 4;                   // K/V ring slots (tile g: K in slot 2g%4, V in 2g%4+1)
+constexpr uint32_t AT_SMEM = (2 + AT_RING) * AT_TILE + 1024;
+constexpr uint32_t AT_WAIT_LIMIT = 1u << 21;
+constexpr float AT_RESCALE_GAP = 8.f;        // raise the running max only when exceeded by 2^8
+constexpr size_t AT_SLOT_FLOATS = (size_t)AT_D * AT_ROWS + 2 * AT_ROWS;   // O^T [d][row], m[row], l[row]
+
+// barrier indices
+enum { B_KV_FULL = 0, B_KV_EMPTY = 4, B_Q_FULL = 8, B_Q_EMPTY = 9, B_S_FULL = 10, B_P_READY = 12, B_P_FREE = 13,
+       B_O_READY = 14, B_O_FREE = 15, B_COUNT = 16 };
+
+struct AtParams {
+    const int32_t* seq_len; const int32_t* row_off; const uint64_t* anc;
+    int anc_words, B, H, max_seq;
+    __nv_bfloat16* out;          // [rows_total][H][128]
+    float* slots;                // partial results, AT_SLOT_FLOATS each
+    int* status;
+    float scale_log2;            // log2(e) / sqrt(D)
+};
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+                 : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok != 0;
+}
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* status) {
+    for (uint32_t i = 0; i < AT_WAIT_LIMIT; ++i) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if (i > 32) {
+            if (*abort_flag) return false;
+            __nanosleep(64);
+        }
+    }
+    *abort_flag = 1;
+    atomicExch(status, (int)TRJ_ETIMEOUT);
+    return false;
+}
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int c_inner, int c_outer, uint32_t bar) {
+    asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+                 ::"r"(dst), "l"(map), "r"(c_inner), "r"(c_outer), "r"(bar) : "memory");
+}
+
+// K-major operand (rows 128 bytes apart, 8-row groups 1024 bytes apart), 128-byte swizzle.
+__device__ __forceinline__ uint64_t desc_kmajor(uint32_t addr) {
+    return (uint64_t)((addr & 0x3FFFF) >> 4) | ((uint64_t)1 << 16) | ((uint64_t)(1024 >> 4) << 32) |
+           ((uint64_t)1 << 46) | ((uint64_t)2 << 61);
+}
+// MN-major operand (V: keys are the contraction dim, head_dim is contiguous): 64-element spans of the
+// MN dim are 128-byte rows, one per key; 8-key groups 1024 bytes apart (stride offset); the second
+// 64-element block of the MN dim lies one sub-tile further (leading offset).
+__device__ __forceinline__ uint64_t desc_mnmajor(uint32_t addr) {
+    return (uint64_t)((addr & 0x3FFFF) >> 4) | ((uint64_t)(AT_SUB >> 4) << 16) | ((uint64_t)(1024 >> 4) << 32) |
+           ((uint64_t)1 << 46) | ((uint64_t)2 << 61);
+}
+__device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
+    asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+                 "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+                 ::"r"(tmem_d), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
+}
+__device__ __forceinline__ void umma_commit(uint32_t bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, float* v) {
+    uint32_t r[32];
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+                 "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+                 "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+                   "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+                   "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+                   "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+                 : "r"(taddr) : "memory");
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+    for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
+}
+__device__ __forceinline__ void tmem_st32(uint32_t taddr, const float* v) {
+    asm volatile("tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
+                 "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, "
+                 "%17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, %32};"
+                 ::"r"(taddr),
+                   "r"(__float_as_uint(v[0])), "r"(__float_as_uint(v[1])), "r"(__float_as_uint(v[2])), "r"(__float_as_uint(v[3])),
+                   "r"(__float_as_uint(v[4])), "r"(__float_as_uint(v[5])), "r"(__float_as_uint(v[6])), "r"(__float_as_uint(v[7])),
+                   "r"(__float_as_uint(v[8])), "r"(__float_as_uint(v[9])), "r"(__float_as_uint(v[10])), "r"(__float_as_uint(v[11])),
+                   "r"(__float_as_uint(v[12])), "r"(__float_as_uint(v[13])), "r"(__float_as_uint(v[14])), "r"(__float_as_uint(v[15])),
+                   "r"(__float_as_uint(v[16])), "r"(__float_as_uint(v[17])), "r"(__float_as_uint(v[18])), "r"(__float_as_uint(v[19])),
+                   "r"(__float_as_uint(v[20])), "r"(__float_as_uint(v[21])), "r"(__float_as_uint(v[22])), "r"(__float_as_uint(v[23])),
+                   "r"(__float_as_uint(v[24])), "r"(__float_as_uint(v[25])), "r"(__float_as_uint(v[26])), "r"(__float_as_uint(v[27])),
+                   "r"(__float_as_uint(v[28])), "r"(__float_as_uint(v[29])), "r"(__float_as_uint(v[30])), "r"(__float_as_uint(v[31]))
+                 : "memory");
+    asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ uint32_t pack_bf16(float a, float b) {
+    const __nv_bfloat162 h = __floats2bfloat162_rn(a, b);      // .x (low half) = a
+    return *reinterpret_cast<const uint32_t*>(&h);
+}
+__device__ __forceinline__ float bf16_round(float a) { return __bfloat162float(__float2bfloat16_rn(a)); }
+
+// 128-bit (lo, hi) shifts by 0..127 bits; the left shift fills the vacated low bits with ones.
+__device__ __forceinline__ void shr128(uint64_t& lo, uint64_t& hi, int n) {
+    if (n == 0) return;
+    if (n < 64) { lo = (lo >> n) | (hi << (64 - n)); hi >>= n; }
+    else { lo = hi >> (n - 64); hi = 0; }
+}
+__device__ __forceinline__ void shl128_fill(uint64_t& lo, uint64_t& hi, int n) {
+    if (n == 0) return;
+    if (n < 64) { hi = (hi << n) | (lo >> (64 - n)); lo = (lo << n) | ((1ull << n) - 1); }
+    else { hi = (n == 64 ? lo : (lo << (n - 64)) | ((1ull << (n - 64)) - 1)); lo = ~0ull; }
+}
+
+// Where a unit index falls: sequence, head, tile, and the geometry of that sequence.
+struct Where { int b, h, t, tiles, S, rows, bh; };
+
+struct Sched {
+    int B, H;
+    int tiles[TRJ_MAX_BATCH];           // key tiles of each sequence
+    long long first[TRJ_MAX_BATCH + 1]; // first unit of each sequence
+    __device__ void locate(long long u, const int32_t* seq_len, const int32_t* row_off, Where& w) const {
+        int b = 0;
+        while (b + 1 < B && u >= first[b + 1]) ++b;
+        const long long r = u - first[b];
+        w.b = b; w.tiles = tiles[b];
+        w.h = (int)(r / w.tiles); w.t = (int)(r % w.tiles);
+        w.S = seq_len[b]; w.rows = row_off[b + 1] - row_off[b];
+        w.bh = b * H + w.h;
+    }
+};
+
+__device__ __forceinline__ void build_sched(Sched& s, const AtParams& p) {
+    s.B = p.B; s.H = p.H;
+    long long u = 0;
+    for (int b = 0; b < p.B; ++b) {
+        const int total = p.seq_len[b] + (p.row_off[b + 1] - p.row_off[b]);
+        s.tiles[b] = (total + AT_KEYS - 1) / AT_KEYS;
+        s.first[b] = u;
+        u += (long long)s.tiles[b] * p.H;
+    }
+    s.first[p.B] = u;
+}
+
+__global__ void __launch_bounds__(AT_THREADS, 1) tree_attention_tc_kernel(const __grid_constant__ CUtensorMap map_q,
+                                                                          const __grid_constant__ CUtensorMap map_k,
+                                                                          const __grid_constant__ CUtensorMap map_v,
+                                                                          const AtParams p) {
+    extern __shared__ uint8_t smem_raw[];
+    __shared__ __align__(8) uint64_t bars[B_COUNT];
+    __shared__ uint32_t tmem_base_slot;
+    __shared__ int abort_flag;
+    __shared__ Sched sched;
+
+    const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    uint8_t* base_ptr = smem_raw + (base - smem_u32(smem_raw));
+    const uint32_t q_smem = base, p_smem = base + AT_TILE, ring_smem = base + 2 * AT_TILE;
+    const uint32_t bar0 = smem_u32(&bars[0]);
+    auto bar = [&](int i) { return bar0 + 8u * (uint32_t)i; };
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+    if (threadIdx.x == 0) {
+        abort_flag = 0;
+        build_sched(sched, p);
+        for (int i = 0; i < B_COUNT; ++i) mbar_init(bar(i), (i == B_P_READY || i == B_O_FREE) ? 128 : 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 5) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
+                     ::"r"(smem_u32(&tmem_base_slot)), "r"(512u) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    const uint32_t tmem = tmem_base_slot;
+    const uint32_t tmem_s[2] = {tmem, tmem + 128}, tmem_o = tmem + 256;
+
+    // this CTA's contiguous range of units
+    const long long U = sched.first[p.B];
+    const long long u_begin = U * blockIdx.x / gridDim.x, u_end = U * (blockIdx.x + 1) / gridDim.x;
+
+    if (warp == 4) {
+        if (lane == 0) {
+            // ------------------------------------------------ TMA producer
+            int g = 0, e = 0;
+            bool ok = true;
+            for (long long u = u_begin; u < u_end && ok;) {
+                Where w; sched.locate(u, p.seq_len, p.row_off, w);
+                const int t_end = (int)min((long long)w.tiles, w.t + (u_end - u));
+                // Q of this segment (after the previous segment's S = Q.K^T products have finished)
+                ok = mbar_wait(bar(B_Q_EMPTY), (uint32_t)(e & 1) ^ 1u, &abort_flag, p.status);
+                if (!ok) break;
+                mbar_expect_tx(bar(B_Q_FULL), AT_TILE);
+                tma_load_2d(q_smem, &map_q, w.h * AT_D, p.row_off[w.b], bar(B_Q_FULL));
+                tma_load_2d(q_smem + AT_SUB, &map_q, w.h * AT_D + 64, p.row_off[w.b], bar(B_Q_FULL));
+                const int cache_row0 = (w.b * p.H + w.h) * p.max_seq;
+                for (int t = w.t; t < t_end && ok; ++t, ++g) {
+                    for (int kv = 0; kv < 2 && ok; ++kv) {
+                        const int slot = (2 * g + kv) % AT_RING;
+                        const uint32_t phase = (uint32_t)((2 * g + kv) / AT_RING) & 1u;
+                        ok = mbar_wait(bar(B_KV_EMPTY + slot), phase ^ 1u, &abort_flag, p.status);
+                        if (!ok) break;
+                        const uint32_t dst = ring_smem + slot * AT_TILE;
+                        mbar_expect_tx(bar(B_KV_FULL + slot), AT_TILE);
+                        const CUtensorMap* map = kv ? &map_v : &map_k;
+                        tma_load_2d(dst, map, 0, cache_row0 + t * AT_KEYS, bar(B_KV_FULL + slot));
+                        tma_load_2d(dst + AT_SUB, map, 64, cache_row0 + t * AT_KEYS, bar(B_KV_FULL + slot));
+                    }
+                }
+                u += t_end - w.t;
+                ++e;
+            }
+        }
+    } else if (warp == 5) {
+        if (lane == 0) {
+            // ------------------------------------------------ MMA issuer
+            // S = Q.K^T: both K-major, 128 x 128.  O += P.V: P K-major, V MN-major, 128 x 128.
+            const uint32_t idesc_qk = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(AT_KEYS >> 3) << 17) | ((uint32_t)(AT_ROWS >> 4) << 24);
+            const uint32_t idesc_pv = idesc_qk | (1u << 16);
+            int g = 0, e = 0;
+            bool ok = true;
+            auto issue_qk = [&](int gg) -> bool {
+                const int slot = (2 * gg) % AT_RING;
+                if (!mbar_wait(bar(B_KV_FULL + slot), (uint32_t)((2 * gg) / AT_RING) & 1u, &abort_flag, p.status)) return false;
+                asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                const uint32_t k_smem = ring_smem + slot * AT_TILE;
+#pragma unroll
+                for (int kk = 0; kk < 8; ++kk) {            // 8 x 16 elements of head_dim: two sub-tiles of four steps
+                    const uint32_t off = (kk >> 2) * AT_SUB + (kk & 3) * 32;
+                    umma_bf16(tmem_s[gg & 1], desc_kmajor(q_smem + off), desc_kmajor(k_smem + off), idesc_qk, kk > 0);
+                }
+                umma_commit(bar(B_S_FULL + (gg & 1)));
+                umma_commit(bar(B_KV_EMPTY + slot));
+                return true;
+            };
+            for (long long u = u_begin; u < u_end && ok;) {
+                Where w; sched.locate(u, p.seq_len, p.row_off, w);
+                const int n_tiles = (int)min((long long)(w.tiles - w.t), u_end - u);
+                const int g0 = g, g1 = g + n_tiles;
+                ok = mbar_wait(bar(B_Q_FULL), (uint32_t)(e & 1), &abort_flag, p.status);
+                if (!ok) break;
+                asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                ok = issue_qk(g0);
+                for (g = g0; g < g1 && ok; ++g) {
+                    if (g + 1 < g1) ok = issue_qk(g + 1);
+                    else umma_commit(bar(B_Q_EMPTY));        // every S product of the segment has been issued
+                    if (!ok) break;
+                    ok = mbar_wait(bar(B_P_READY), (uint32_t)(g & 1), &abort_flag, p.status);
+                    if (ok && g == g0 && e > 0) ok = mbar_wait(bar(B_O_FREE), (uint32_t)((e - 1) & 1), &abort_flag, p.status);
+                    const int slot = (2 * g + 1) % AT_RING;
+                    if (ok) ok = mbar_wait(bar(B_KV_FULL + slot), (uint32_t)((2 * g + 1) / AT_RING) & 1u, &abort_flag, p.status);
+                    if (!ok) break;
+                    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                    const uint32_t v_smem = ring_smem + slot * AT_TILE;
+#pragma unroll
+                    for (int kk = 0; kk < 8; ++kk) {        // 8 x 16 keys
+                        const uint32_t p_off = (kk >> 2) * AT_SUB + (kk & 3) * 32;     // P: two 64-key sub-tiles
+                        const uint32_t v_off = kk * 16 * 128;                          // V: 16 keys = 16 rows of 128 bytes
+                        umma_bf16(tmem_o, desc_kmajor(p_smem + p_off), desc_mnmajor(v_smem + v_off), idesc_pv,
+                                  (g > g0 || kk > 0) ? 1u : 0u);
+                    }
+                    umma_commit(bar(B_P_FREE));
+                    umma_commit(bar(B_KV_EMPTY + slot));
+                }
+                if (ok) umma_commit(bar(B_O_READY));
+                u += n_tiles;
+                ++e;
+            }
+        }
+    } else {
+        // ------------------------------------------------ softmax + epilogue: thread = query row
+        const int row = threadIdx.x;                         // 0..127 == TMEM lane
+        const uint32_t lane_addr = (uint32_t)(warp * 32) << 16;
+        int g = 0, e = 0;
+        bool ok = true;
+        for (long long u = u_begin; u < u_end && ok;) {
+            Where w; sched.locate(u, p.seq_len, p.row_off, w);
+            const int n_tiles = (int)min((long long)(w.tiles - w.t), u_end - u);
+            const int g0 = g, g1 = g + n_tiles;
+            const bool live = row < w.rows;
+            const int grow = p.row_off[w.b] + row;           // global row (valid when live)
+            uint64_t m0 = 0, m1 = 0;
+            if (live) {
+                m0 = p.anc[(size_t)grow * p.anc_words];
+                if (p.anc_words > 1) m1 = p.anc[(size_t)grow * p.anc_words + 1];
+            }
+            const int total = w.S + w.rows;
+            float m_ref = -INFINITY, l_sum = 0.f;
+            for (g = g0; g < g1 && ok; ++g) {
+                const int key0 = (w.t + (g - g0)) * AT_KEYS;
+                const bool edge = key0 + AT_KEYS > w.S;      // the tile reaches tree rows or the end of the keys
+                ok = __all_sync(0xffffffffu, mbar_wait(bar(B_S_FULL + (g & 1)), (uint32_t)(g >> 1) & 1u, &abort_flag, p.status));
+                if (!ok) break;
+                asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                // visibility of the 128 columns of this row as two 64-bit words (bit c = key0 + c): column c is
+                // tree row tt = key0 + c - S; it is visible if tt < 0 (prefix) or if bit tt of the row's mask is set
+                uint64_t vis0 = ~0ull, vis1 = ~0ull;
+                if (edge) {
+                    const int d = key0 - w.S;                // -127 .. 127 on an edge tile
+                    if (d >= 0) { vis0 = m0; vis1 = m1; shr128(vis0, vis1, d); }
+                    else { vis0 = m0; vis1 = m1; shl128_fill(vis0, vis1, -d); }
+                }
+                // pass 1: maximum of the visible scores of the tile
+                float mt = -INFINITY;
+#pragma unroll 1
+                for (int c0 = 0; c0 < AT_KEYS; c0 += 32) {
+                    float s[32];
+                    tmem_ld32(tmem_s[g & 1] + lane_addr + c0, s);
+                    const uint32_t bits = (uint32_t)((c0 < 64 ? vis0 : vis1) >> (c0 & 63));
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) if ((bits >> i) & 1u) mt = fmaxf(mt, s[i]);
+                }
+                mt *= p.scale_log2;
+                // the P buffer and the O accumulator are free once the previous P.V product has finished
+                if (g > 0) ok = __all_sync(0xffffffffu, mbar_wait(bar(B_P_FREE), (uint32_t)((g - 1) & 1), &abort_flag, p.status));
+                if (!ok) break;
+                asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                float factor = 1.f;
+                if (live && mt > -INFINITY) {
+                    if (m_ref == -INFINITY) m_ref = mt;
+                    else if (mt > m_ref + AT_RESCALE_GAP) { factor = exp2f(m_ref - mt); m_ref = mt; }
+                }
+                if (g > g0 && __any_sync(0xffffffffu, factor != 1.f)) {
+                    l_sum *= factor;
+#pragma unroll 1
+                    for (int c0 = 0; c0 < AT_D; c0 += 32) {
+                        float o[32];
+                        tmem_ld32(tmem_o + lane_addr + c0, o);
+#pragma unroll
+                        for (int i = 0; i < 32; ++i) o[i] *= factor;
+                        tmem_st32(tmem_o + lane_addr + c0, o);
+                    }
+                }
+                // pass 2: P = 2^(s * c - m_ref) as bf16, into the K-major swizzled layout of the P operand
+                const float m_use = (m_ref == -INFINITY) ? 0.f : m_ref;
+#pragma unroll 1
+                for (int c0 = 0; c0 < AT_KEYS; c0 += 32) {
+                    float s[32];
+                    tmem_ld32(tmem_s[g & 1] + lane_addr + c0, s);
+                    const uint32_t bits = live ? (uint32_t)((c0 < 64 ? vis0 : vis1) >> (c0 & 63)) : 0u;
+                    uint32_t packed[16];
+#pragma unroll
+                    for (int i = 0; i < 32; i += 2) {
+                        float a = ((bits >> i) & 1u) ? bf16_round(exp2f(fmaf(s[i], p.scale_log2, -m_use))) : 0.f;
+                        float b = ((bits >> (i + 1)) & 1u) ? bf16_round(exp2f(fmaf(s[i + 1], p.scale_log2, -m_use))) : 0.f;
+                        l_sum += a + b;
+                        packed[i >> 1] = pack_bf16(a, b);
+                    }
+                    // 32 keys = four 16-byte chunks of this row inside sub-tile c0 / 64
+                    uint8_t* sub = base_ptr + AT_TILE + (c0 >> 6) * AT_SUB + row * 128;
+#pragma unroll
+                    for (int ch = 0; ch < 4; ++ch) {
+                        const int chunk = ((c0 & 63) >> 3) + ch;
+                        *reinterpret_cast<uint4*>(sub + ((chunk ^ (row & 7)) << 4)) =
+                            make_uint4(packed[4 * ch], packed[4 * ch + 1], packed[4 * ch + 2], packed[4 * ch + 3]);
+                    }
+                }
+                // keys past the end of the sequence hold whatever the cache holds: clear those V rows so
+                // that 0 * garbage cannot poison the product
+                if (key0 + AT_KEYS > total) {
+                    const int slot = (2 * g + 1) % AT_RING;
+                    ok = __all_sync(0xffffffffu, mbar_wait(bar(B_KV_FULL + slot), (uint32_t)((2 * g + 1) / AT_RING) & 1u, &abort_flag, p.status));
+                    if (!ok) break;
+                    uint8_t* v_ptr = base_ptr + 2 * AT_TILE + slot * AT_TILE;
+                    const int first_bad = max(total - key0, 0);
+                    for (int i = first_bad * 8 + row; i < AT_KEYS * 8; i += 128) {      // 16-byte chunks, both sub-tiles
+                        *reinterpret_cast<uint4*>(v_ptr + i * 16) = make_uint4(0, 0, 0, 0);
+                        *reinterpret_cast<uint4*>(v_ptr + AT_SUB + i * 16) = make_uint4(0, 0, 0, 0);
+                    }
+                }
+                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+                mbar_arrive(bar(B_P_READY));
+            }
+            if (!ok) break;
+            // ---- epilogue of the segment
+            ok = __all_sync(0xffffffffu, mbar_wait(bar(B_O_READY), (uint32_t)(e & 1), &abort_flag, p.status));
+            if (!ok) break;
+            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+            const bool whole = (w.t == 0 && n_tiles == w.tiles);
+            if (whole) {
+                const float inv = live ? 1.f / l_sum : 0.f;
+                __nv_bfloat16* dst = p.out + ((size_t)grow * p.H + w.h) * AT_D;
+#pragma unroll 1
+                for (int c0 = 0; c0 < AT_D; c0 += 32) {
+                    float o[32];
+                    tmem_ld32(tmem_o + lane_addr + c0, o);
+                    if (live) {
+#pragma unroll
+                        for (int ch = 0; ch < 4; ++ch)
+                            *reinterpret_cast<uint4*>(dst + c0 + 8 * ch) =
+                                make_uint4(pack_bf16(o[8 * ch] * inv, o[8 * ch + 1] * inv), pack_bf16(o[8 * ch + 2] * inv, o[8 * ch + 3] * inv),
+                                           pack_bf16(o[8 * ch + 4] * inv, o[8 * ch + 5] * inv), pack_bf16(o[8 * ch + 6] * inv, o[8 * ch + 7] * inv));
+                    }
+                }
+            } else {
+                float* slot = p.slots + (size_t)(w.bh + (int)blockIdx.x) * AT_SLOT_FLOATS;
+#pragma unroll 1
+                for (int c0 = 0; c0 < AT_D; c0 += 32) {
+                    float o[32];
+                    tmem_ld32(tmem_o + lane_addr + c0, o);
+                    if (live) {
+#pragma unroll
+                        for (int i = 0; i < 32; ++i) slot[(size_t)(c0 + i) * AT_ROWS + row] = o[i];
+                    }
+                }
+                if (live) { slot[AT_D * AT_ROWS + row] = m_ref; slot[AT_D * AT_ROWS + AT_ROWS + row] = l_sum; }
+            }
+            asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+            mbar_arrive(bar(B_O_FREE));
+            u += n_tiles;
+            ++e;
+        }
+    }
+    __syncwarp();
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    if (abort_flag) {                                        // let copies still in flight land before the CTA leaves
+        for (int i = 0; i < 64; ++i) __nanosleep(1000);
+        __syncthreads();
+    }
+    if (warp == 5)
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(512u) : "memory");
+}
+
+// Merges the pieces of every (sequence, head) that more than one CTA worked on.  One CTA per
+// (sequence, head), thread = row; pieces are taken in ascending CTA order.
+__global__ void __launch_bounds__(128) tree_attention_combine_kernel(const AtParams p, int grid_main) {
+    __shared__ Sched sched;
+    __shared__ float stage[AT_ROWS][33];
+    if (threadIdx.x == 0) build_sched(sched, p);
+    __syncthreads();
+    const int bh = blockIdx.x, b = bh / p.H, h = bh % p.H;
+    const long long U = sched.first[p.B];
+    const long long u0 = sched.first[b] + (long long)h * sched.tiles[b], u1 = u0 + sched.tiles[b];
+    // CTA c of the main kernel owns units [U*c/G, U*(c+1)/G): the owner of unit u is the largest c with U*c/G <= u
+    auto owner = [&](long long u) { return (int)(((u + 1) * grid_main + U - 1) / U - 1); };
+    const int c_first = owner(u0), c_last = owner(u1 - 1);
+    if (c_first == c_last) return;                           // written directly by its only CTA
+    const int row = threadIdx.x, rows = p.row_off[b + 1] - p.row_off[b];
+    const bool live = row < rows;
+    // a CTA in between may own no unit at all (grid larger than the unit count): it wrote nothing
+    auto has_piece = [&](int c) {
+        const long long rb = U * c / grid_main, re = U * (c + 1) / grid_main;
+        return (rb > u0 ? rb : u0) < (re < u1 ? re : u1);
+    };
+    float m_all = -INFINITY;
+    for (int c = c_first; c <= c_last; ++c)
+        if (live && has_piece(c)) m_all = fmaxf(m_all, p.slots[(size_t)(bh + c) * AT_SLOT_FLOATS + AT_D * AT_ROWS + row]);
+    float l_all = 0.f;
+    for (int c = c_first; c <= c_last; ++c) {
+        if (!live) break;
+        if (!has_piece(c)) continue;
+        const float* slot = p.slots + (size_t)(bh + c) * AT_SLOT_FLOATS;
+        const float m = slot[AT_D * AT_ROWS + row];
+        if (m > -INFINITY) l_all += slot[AT_D * AT_ROWS + AT_ROWS + row] * exp2f(m - m_all);
+    }
+    const float inv = live ? 1.f / l_all : 0.f;
+    for (int c0 = 0; c0 < AT_D; c0 += 32) {
+        float acc[32];
+#pragma unroll
+        for (int i = 0; i < 32; ++i) acc[i] = 0.f;
+        for (int c = c_first; c <= c_last && live; ++c) {
+            if (!has_piece(c)) continue;
+            const float* slot = p.slots + (size_t)(bh + c) * AT_SLOT_FLOATS;
+            const float m = slot[AT_D * AT_ROWS + row];
+            if (m == -INFINITY) continue;
+            const float wgt = exp2f(m - m_all);
+#pragma unroll
+            for (int i = 0; i < 32; ++i) acc[i] = fmaf(slot[(size_t)(c0 + i) * AT_ROWS + row], wgt, acc[i]);
+        }
+#pragma unroll
+        for (int i = 0; i < 32; ++i) stage[row][i] = acc[i] * inv;
+        __syncthreads();
+        // 128 rows x 32 values -> each thread stores 8 consecutive values (16 bytes) of one row
+        for (int i = threadIdx.x; i < rows * 4; i += 128) {
+            const int r = i >> 2, q4 = (i & 3) * 8;
+            __nv_bfloat16* dst = p.out + ((size_t)(p.row_off[b] + r) * p.H + h) * AT_D + c0 + q4;
+            *reinterpret_cast<uint4*>(dst) =
+                make_uint4(pack_bf16(stage[r][q4], stage[r][q4 + 1]), pack_bf16(stage[r][q4 + 2], stage[r][q4 + 3]),
+                           pack_bf16(stage[r][q4 + 4], stage[r][q4 + 5]), pack_bf16(stage[r][q4 + 6], stage[r][q4 + 7]));
+        }
+        __syncthreads();
+    }
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                  const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+EncodeTiledFn at_encode_fn() {
+    static EncodeTiledFn fn = nullptr;
+    static std::once_flag once;
+    std::call_once(once, [] {
+        void* ptr = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &q) == cudaSuccess &&
+            q == cudaDriverEntryPointSuccess)
+            fn = (EncodeTiledFn)ptr;
+    });
+    return fn;
+}
+// bf16 matrix [rows][cols] row-major, boxes of [128 rows][64 cols], 128-byte swizzle, zero fill.
+bool at_make_map(CUtensorMap* map, const void* base_ptr, size_t rows, size_t cols) {
+    EncodeTiledFn fn = at_encode_fn();
+    if (!fn) return false;
+    const cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
+    const cuuint64_t strides[1] = {(cuuint64_t)cols * 2};
+    const cuuint32_t box[2] = {64, 128};
+    const cuuint32_t estr[2] = {1, 1};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base_ptr), dims, strides, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+constexpr int AT_MAX_GRID = 148;
+
+}  // namespace
+
+bool tree_attention_tc_supported(int32_t D, int32_t dtype, int32_t max_rows) {
+    return D == AT_D && dtype == TRJ_BF16 && max_rows <= AT_ROWS && at_encode_fn() != nullptr;
+}
+
+// Workspace: 256-byte header (status word), then one slot per possible piece: a CTA range can start a
+// new (sequence, head) at most B*H times in total and each of the <= 148 CTAs opens at most one more.
+size_t tree_attention_tc_workspace(int32_t B, int32_t H) {
+    return 256 + ((size_t)B * H + AT_MAX_GRID) * AT_SLOT_FLOATS * sizeof(float);
+}
+
+cudaError_t launch_tree_attention_tc(const void* q, const void* k_slab, const void* v_slab, const uint64_t* anc,
+                                     int32_t anc_words, const Batch& bt, int32_t H, int32_t max_seq, void* out,
+                                     void* workspace, cudaStream_t st) {
+    static std::once_flag once;
+    static cudaError_t attr_err = cudaSuccess;
+    std::call_once(once, [] {
+        attr_err = cudaFuncSetAttribute(tree_attention_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)AT_SMEM);
+    });
+    if (attr_err != cudaSuccess) return attr_err;
+    CUtensorMap map_q, map_k, map_v;
+    if (!at_make_map(&map_q, q, (size_t)bt.rows_total, (size_t)H * AT_D) ||
+        !at_make_map(&map_k, k_slab, (size_t)bt.B * H * max_seq, AT_D) ||
+        !at_make_map(&map_v, v_slab, (size_t)bt.B * H * max_seq, AT_D))
+        return cudaErrorInvalidValue;
+    AtParams p;
+    p.seq_len = bt.seq_len; p.row_off = bt.row_off; p.anc = anc; p.anc_words = anc_words;
+    p.B = bt.B; p.H = H; p.max_seq = max_seq;
+    p.out = (__nv_bfloat16*)out;
+    p.status = (int*)workspace;
+    p.slots = (float*)((char*)workspace + 256);
+    p.scale_log2 = 1.4426950408889634f / sqrtf((float)AT_D);
+    // the host only knows an upper bound of the key count; CTAs whose range is empty leave at once
+    const long long units_bound = (long long)bt.B * H * ((bt.max_len + AT_KEYS - 1) / AT_KEYS);
+    const int grid = (int)(units_bound < AT_MAX_GRID ? units_bound : AT_MAX_GRID);
+    count_launch();
+    tree_attention_tc_kernel<<<grid, AT_THREADS, AT_SMEM, st>>>(map_q, map_k, map_v, p);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+    count_launch();
+    tree_attention_combine_kernel<<<bt.B * H, 128, 0, st>>>(p, grid);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_tree_attention(const void* q, const void* k_slab, const void* v_slab, const uint64_t* anc,
+                                  int32_t anc_words, const Batch& bt, int32_t H, int32_t D, int32_t max_seq,
+                                  int32_t dtype, void* out, void* workspace, size_t workspace_bytes, cudaStream_t st) {
+    if (workspace && ((uintptr_t)workspace % 256) == 0 && workspace_bytes >= tree_attention_tc_workspace(bt.B, H) &&
+        tree_attention_tc_supported(D, dtype, bt.max_rows))
+        return launch_tree_attention_tc(q, k_slab, v_slab, anc, anc_words, bt, H, max_seq, out, workspace, st);
+    return launch_tree_attention_generic(q, k_slab, v_slab, anc, anc_words, bt, H, D, max_seq, dtype, out, st);
+}
+
+}  // namespace trj

@@ -17,8 +17,11 @@ TOL = {"bf16": 2e-2, "f32": 2e-5}
 
 
 def check_attention(trj, case, heads=None, seqs=None):
-    out = case.run(trj).float().cpu().numpy()
+    need = trj.tree_attention_workspace(int(case.row_off_host[-1]), len(case.rows), case.h, case.d, case.max_len)
+    ws = torch.zeros(max(256, need), dtype=torch.uint8, device="cuda")
+    out = case.run(trj, workspace=ws).float().cpu().numpy()
     torch.cuda.synchronize()
+    assert int(ws[:4].view(torch.int32)[0]) == 0           # no device-side wait expired
     worst = 0.0
     for b in (range(len(case.rows)) if seqs is None else seqs):
         r0, r1 = case.row_off_host[b], case.row_off_host[b + 1]
