@@ -118,9 +118,9 @@ def device_weights(cfg, seed, device):
 
 def gemm_bytes_per_step(cfg, rows):
     """Algorithmic bytes of all projections of one verification step: every weight once (bf16), the
-    split-bf16 activations in (attention output: single bf16) and the fp32 results out."""
+    split-bf16 activations in and the fp32 results out."""
     d, f, hd, v = cfg.d_model, cfg.d_ff, cfg.n_heads * cfg.head_dim, cfg.vocab
-    per_layer = [(3 * hd, d, 2), (d, hd, 1), (2 * f, d, 2), (d, f, 2)]      # (N, K, activation halves)
+    per_layer = [(3 * hd, d, 2), (d, hd, 2), (2 * f, d, 2), (d, f, 2)]      # (N, K, activation halves)
     total = 0
     for n, k, halves in per_layer:
         total += cfg.n_layers * (n * k * 2 + rows * k * 2 * halves + rows * n * 4)

@@ -15,10 +15,10 @@ tiling, no online softmax and no fusion.
 
 Precision: every floating-point step is fp64.  Inputs arrive as float32 arrays
 whose values are already representable in the storage type of the config
-(bf16 or fp32) and are widened exactly.  In a bf16 model the tensors that are
-the operands and the result of the attention op (q, the K/V cache rows, the
-attention output) are bf16 tensors by the config's definition, so the decoder
-rounds them to bf16 where they are stored; nothing else is rounded.
+(bf16 or fp32) and are widened exactly.  In a bf16 model the operands of the
+attention op (q and the K/V cache rows) are bf16 tensors by the config's
+definition, so the decoder rounds them to bf16 where they are stored; nothing
+else is rounded (the attention result feeds the output projection unrounded).
 
 Readings taken where the paper is silent (each one is a free choice that
 cannot change which tokens a greedy decoder commits, unless noted):

@@ -83,9 +83,9 @@ class Decoder:
         m, s = len(tokens), cache.seq_len
         n_heads, hd = c.n_heads, c.head_dim
         pos = s + depths(parent)
-        # bf16 configs: q, the K/V cache rows and the attention output are bf16 tensors (they are the
-        # operands and the result of the attention op at the library boundary); what such a tensor
-        # holds is the rounded value.  Everything else, and all arithmetic, stays fp64.
+        # bf16 configs: q and the K/V cache rows are bf16 tensors (the cache is stored in bf16 by the
+        # config's definition and q is the other operand of the attention op); what such a tensor holds
+        # is the rounded value.  Everything else, and all arithmetic, stays fp64.
         store = store_bf16 if c.dtype == "bf16" else (lambda t: t)
         h = np.asarray(self.glob["embed"], np.float64)[np.asarray(tokens, np.int64)]
         for l in range(c.n_layers):
@@ -97,8 +97,8 @@ class Decoder:
             q, k, v = store(rope(q, pos, c.rope_theta)), store(rope(k, pos, c.rope_theta)), store(v)
             cache.k[l][:, s:s + m, :] = k.transpose(1, 0, 2)
             cache.v[l][:, s:s + m, :] = v.transpose(1, 0, 2)
-            att = store(tree_attention(q, cache.k[l][:, :s], cache.v[l][:, :s],
-                                       cache.k[l][:, s:s + m], cache.v[l][:, s:s + m], parent))
+            att = tree_attention(q, cache.k[l][:, :s], cache.v[l][:, :s],
+                                 cache.k[l][:, s:s + m], cache.v[l][:, s:s + m], parent)
             h = h + att.reshape(m, n_heads * hd) @ np.asarray(w["wo"], np.float64).T
             x = rmsnorm(h, np.asarray(w["mlp_norm"], np.float64), c.rms_eps)
             gu = x @ np.asarray(w["w_gate_up"], np.float64).T

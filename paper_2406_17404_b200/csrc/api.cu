@@ -52,8 +52,8 @@ extern "C" trj_status trj_tree_attention(const void* q, const void* k_cache, con
                 TRJ_ECAPACITY, "tree_attention: workspace too small");
     if (rows_total == 0) return TRJ_OK;
     Batch bt{seq_len, row_off, B, rows_total, max_rows, max_len};
-    TRJ_CHECK_CUDA(launch_tree_attention(q, k_cache, v_cache, anc, anc_words, bt, H, D, max_seq, dtype, out, workspace,
-                                         workspace_bytes, (cudaStream_t)stream));
+    TRJ_CHECK_CUDA(launch_tree_attention(q, k_cache, v_cache, anc, anc_words, bt, H, D, max_seq, dtype, out, nullptr,
+                                         workspace, workspace_bytes, (cudaStream_t)stream));
     return TRJ_OK;
 }
 
@@ -227,10 +227,12 @@ trj_status forward(trj_ctx* ctx, void* k_cache, void* v_cache, int32_t b0, const
         LAUNCH(PROF_GEMM, launch_gemm(ctx->x, ctx->x_lo, ctx->wqkv[l], ctx->y, M, 3 * HD, d, c.dtype, ctx->gemm_ws, ctx->gemm_ws_bytes, st));
         LAUNCH(PROF_ROPE, launch_rope_kv_write(ctx->y, ctx->inv_freq, depth, bt, ctx->q, k_slab, v_slab, c.dtype,
                                                c.n_heads, c.head_dim, c.max_seq, st));
-        // the attention output is a bf16 tensor of its own right (no low half)
+        // inside the decoder the attention result reaches the output projection as a bf16 pair, like every
+        // other projection input
         LAUNCH(PROF_ATTENTION, launch_tree_attention(ctx->q, k_slab, v_slab, anc, anc_words, bt, c.n_heads, c.head_dim,
-                                                     c.max_seq, c.dtype, ctx->x, ctx->attn_ws, ctx->attn_ws_bytes, st));
-        LAUNCH(PROF_GEMM, launch_gemm(ctx->x, nullptr, ctx->wo[l], ctx->y, M, d, HD, c.dtype, ctx->gemm_ws, ctx->gemm_ws_bytes, st));
+                                                     c.max_seq, c.dtype, ctx->x, ctx->x_lo, ctx->attn_ws,
+                                                     ctx->attn_ws_bytes, st));
+        LAUNCH(PROF_GEMM, launch_gemm(ctx->x, ctx->x_lo, ctx->wo[l], ctx->y, M, d, HD, c.dtype, ctx->gemm_ws, ctx->gemm_ws_bytes, st));
         LAUNCH(PROF_ELEMENTWISE, launch_add_rmsnorm(ctx->h, ctx->y, ctx->mlp_norm[l], ctx->x, ctx->x_lo, c.dtype, M, d,
                                                     c.rms_eps, st));
         LAUNCH(PROF_GEMM, launch_gemm(ctx->x, ctx->x_lo, ctx->w_gate_up[l], ctx->y, M, 2 * c.d_ff, d, c.dtype, ctx->gemm_ws,

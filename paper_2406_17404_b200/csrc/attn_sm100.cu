@@ -40,6 +40,7 @@ struct AtParams {
     const int32_t* seq_len; const int32_t* row_off; const uint64_t* anc;
     int anc_words, B, H, max_seq;
     __nv_bfloat16* out;          // [rows_total][H][128]
+    __nv_bfloat16* out_lo;       // optional: rounding error of `out` as a second bf16 tensor (same shape)
     float* slots;                // partial results, AT_SLOT_FLOATS each
     int* status;
     float scale_log2;            // log2(e) / sqrt(D)
@@ -133,6 +134,16 @@ __device__ __forceinline__ uint32_t pack_bf16(float a, float b) {
     return *reinterpret_cast<const uint32_t*>(&h);
 }
 __device__ __forceinline__ float bf16_round(float a) { return __bfloat162float(__float2bfloat16_rn(a)); }
+// Stores 8 consecutive outputs as bf16 (16 bytes) and, when asked, the rounding errors as a second bf16 vector.
+__device__ __forceinline__ void store8_split(__nv_bfloat16* hi, __nv_bfloat16* lo, const float* v) {
+    *reinterpret_cast<uint4*>(hi) = make_uint4(pack_bf16(v[0], v[1]), pack_bf16(v[2], v[3]), pack_bf16(v[4], v[5]), pack_bf16(v[6], v[7]));
+    if (lo) {
+        float r[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) r[i] = v[i] - bf16_round(v[i]);
+        *reinterpret_cast<uint4*>(lo) = make_uint4(pack_bf16(r[0], r[1]), pack_bf16(r[2], r[3]), pack_bf16(r[4], r[5]), pack_bf16(r[6], r[7]));
+    }
+}
 
 // 128-bit (lo, hi) shifts by 0..127 bits; the left shift fills the vacated low bits with ones.
 __device__ __forceinline__ void shr128(uint64_t& lo, uint64_t& hi, int n) {
@@ -415,17 +426,17 @@ __global__ void __launch_bounds__(AT_THREADS, 1) tree_attention_tc_kernel(const 
             const bool whole = (w.t == 0 && n_tiles == w.tiles);
             if (whole) {
                 const float inv = live ? 1.f / l_sum : 0.f;
-                __nv_bfloat16* dst = p.out + ((size_t)grow * p.H + w.h) * AT_D;
+                const size_t off = ((size_t)grow * p.H + w.h) * AT_D;
 #pragma unroll 1
                 for (int c0 = 0; c0 < AT_D; c0 += 32) {
                     float o[32];
                     tmem_ld32(tmem_o + lane_addr + c0, o);
                     if (live) {
 #pragma unroll
+                        for (int i = 0; i < 32; ++i) o[i] *= inv;
+#pragma unroll
                         for (int ch = 0; ch < 4; ++ch)
-                            *reinterpret_cast<uint4*>(dst + c0 + 8 * ch) =
-                                make_uint4(pack_bf16(o[8 * ch] * inv, o[8 * ch + 1] * inv), pack_bf16(o[8 * ch + 2] * inv, o[8 * ch + 3] * inv),
-                                           pack_bf16(o[8 * ch + 4] * inv, o[8 * ch + 5] * inv), pack_bf16(o[8 * ch + 6] * inv, o[8 * ch + 7] * inv));
+                            store8_split(p.out + off + c0 + 8 * ch, p.out_lo ? p.out_lo + off + c0 + 8 * ch : nullptr, o + 8 * ch);
                     }
                 }
             } else {
@@ -510,10 +521,8 @@ __global__ void __launch_bounds__(128) tree_attention_combine_kernel(const AtPar
         // 128 rows x 32 values -> each thread stores 8 consecutive values (16 bytes) of one row
         for (int i = threadIdx.x; i < rows * 4; i += 128) {
             const int r = i >> 2, q4 = (i & 3) * 8;
-            __nv_bfloat16* dst = p.out + ((size_t)(p.row_off[b] + r) * p.H + h) * AT_D + c0 + q4;
-            *reinterpret_cast<uint4*>(dst) =
-                make_uint4(pack_bf16(stage[r][q4], stage[r][q4 + 1]), pack_bf16(stage[r][q4 + 2], stage[r][q4 + 3]),
-                           pack_bf16(stage[r][q4 + 4], stage[r][q4 + 5]), pack_bf16(stage[r][q4 + 6], stage[r][q4 + 7]));
+            const size_t off = ((size_t)(p.row_off[b] + r) * p.H + h) * AT_D + c0 + q4;
+            store8_split(p.out + off, p.out_lo ? p.out_lo + off : nullptr, &stage[r][q4]);
         }
         __syncthreads();
     }
@@ -563,7 +572,7 @@ size_t tree_attention_tc_workspace(int32_t B, int32_t H) {
 
 cudaError_t launch_tree_attention_tc(const void* q, const void* k_slab, const void* v_slab, const uint64_t* anc,
                                      int32_t anc_words, const Batch& bt, int32_t H, int32_t max_seq, void* out,
-                                     void* workspace, cudaStream_t st) {
+                                     void* out_lo, void* workspace, cudaStream_t st) {
     static std::once_flag once;
     static cudaError_t attr_err = cudaSuccess;
     std::call_once(once, [] {
@@ -579,6 +588,7 @@ cudaError_t launch_tree_attention_tc(const void* q, const void* k_slab, const vo
     p.seq_len = bt.seq_len; p.row_off = bt.row_off; p.anc = anc; p.anc_words = anc_words;
     p.B = bt.B; p.H = H; p.max_seq = max_seq;
     p.out = (__nv_bfloat16*)out;
+    p.out_lo = (__nv_bfloat16*)out_lo;
     p.status = (int*)workspace;
     p.slots = (float*)((char*)workspace + 256);
     p.scale_log2 = 1.4426950408889634f / sqrtf((float)AT_D);
@@ -596,11 +606,12 @@ cudaError_t launch_tree_attention_tc(const void* q, const void* k_slab, const vo
 
 cudaError_t launch_tree_attention(const void* q, const void* k_slab, const void* v_slab, const uint64_t* anc,
                                   int32_t anc_words, const Batch& bt, int32_t H, int32_t D, int32_t max_seq,
-                                  int32_t dtype, void* out, void* workspace, size_t workspace_bytes, cudaStream_t st) {
+                                  int32_t dtype, void* out, void* out_lo, void* workspace, size_t workspace_bytes,
+                                  cudaStream_t st) {
     if (workspace && ((uintptr_t)workspace % 256) == 0 && workspace_bytes >= tree_attention_tc_workspace(bt.B, H) &&
         tree_attention_tc_supported(D, dtype, bt.max_rows))
-        return launch_tree_attention_tc(q, k_slab, v_slab, anc, anc_words, bt, H, max_seq, out, workspace, st);
-    return launch_tree_attention_generic(q, k_slab, v_slab, anc, anc_words, bt, H, D, max_seq, dtype, out, st);
+        return launch_tree_attention_tc(q, k_slab, v_slab, anc, anc_words, bt, H, max_seq, out, out_lo, workspace, st);
+    return launch_tree_attention_generic(q, k_slab, v_slab, anc, anc_words, bt, H, D, max_seq, dtype, out, out_lo, st);
 }
 
 }  // namespace trj

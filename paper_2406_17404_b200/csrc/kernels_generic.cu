@@ -163,7 +163,7 @@ template <typename T, int D>
 __global__ void __launch_bounds__(128) tree_attention_generic_kernel(
         const T* __restrict__ q, const T* __restrict__ k_slab, const T* __restrict__ v_slab,
         const uint64_t* __restrict__ anc, int anc_words, const int32_t* __restrict__ seq_len,
-        const int32_t* __restrict__ row_off, int B, int H, int max_seq, T* __restrict__ out) {
+        const int32_t* __restrict__ row_off, int B, int H, int max_seq, T* __restrict__ out, T* __restrict__ out_lo) {
     constexpr int PER = D / 32;                  // output dims per lane
     __shared__ float qs[D];
     __shared__ float part_m[4], part_l[4];
@@ -226,7 +226,7 @@ __global__ void __launch_bounds__(128) tree_attention_generic_kernel(
             l += part_l[w] * f;
             o += part_acc[w][c] * f;
         }
-        out[((size_t)row * H + hh) * D + c] = from_f<T>(o / l);
+        store_split(out, out_lo, ((size_t)row * H + hh) * D + c, o / l);
     }
 }
 
@@ -435,13 +435,13 @@ cudaError_t launch_rope_kv_write(const float* qkv, const double* inv_freq, const
 cudaError_t launch_tree_attention_generic(const void* q, const void* k_slab, const void* v_slab,
                                           const uint64_t* anc, int32_t anc_words, const Batch& bt,
                                           int32_t H, int32_t D, int32_t max_seq, int32_t dtype,
-                                          void* out, cudaStream_t st) {
+                                          void* out, void* out_lo, cudaStream_t st) {
     count_launch();
     dim3 grid(bt.rows_total, H);
 #define ATT(DD)                                                                                          \
     DISPATCH_T(dtype, tree_attention_generic_kernel<T, DD><<<grid, 128, 0, st>>>(                        \
                           (const T*)q, (const T*)k_slab, (const T*)v_slab, anc, anc_words, bt.seq_len,   \
-                          bt.row_off, bt.B, H, max_seq, (T*)out))
+                          bt.row_off, bt.B, H, max_seq, (T*)out, (T*)out_lo))
     if (D == 64) { ATT(64); }
     else if (D == 128) { ATT(128); }
     else return cudaErrorInvalidValue;

@@ -69,18 +69,20 @@ cudaError_t launch_rope_kv_write(const float* qkv, const double* inv_freq, const
 cudaError_t launch_tree_attention_generic(const void* q, const void* k_slab, const void* v_slab,
                                           const uint64_t* anc, int32_t anc_words, const Batch& bt,
                                           int32_t H, int32_t D, int32_t max_seq, int32_t dtype,
-                                          void* out, cudaStream_t st);
+                                          void* out, void* out_lo, cudaStream_t st);
 // tcgen05 / TMA tree attention (attn_sm100.cu): bf16, head_dim 128.  Workspace: status word in the first
 // 256 bytes, then split-KV partial results.
 bool tree_attention_tc_supported(int32_t D, int32_t dtype, int32_t max_rows);
 size_t tree_attention_tc_workspace(int32_t B, int32_t H);
 cudaError_t launch_tree_attention_tc(const void* q, const void* k_slab, const void* v_slab, const uint64_t* anc,
                                      int32_t anc_words, const Batch& bt, int32_t H, int32_t max_seq, void* out,
-                                     void* workspace, cudaStream_t st);
-// Picks the tcgen05 kernel when shape and workspace allow it, the generic kernel otherwise.
+                                     void* out_lo, void* workspace, cudaStream_t st);
+// Picks the tcgen05 kernel when shape and workspace allow it, the generic kernel otherwise.  out_lo (may be
+// null) receives the rounding error of `out` as a second tensor of the same type, for the projection that follows.
 cudaError_t launch_tree_attention(const void* q, const void* k_slab, const void* v_slab, const uint64_t* anc,
                                   int32_t anc_words, const Batch& bt, int32_t H, int32_t D, int32_t max_seq,
-                                  int32_t dtype, void* out, void* workspace, size_t workspace_bytes, cudaStream_t st);
+                                  int32_t dtype, void* out, void* out_lo, void* workspace, size_t workspace_bytes,
+                                  cudaStream_t st);
 
 // act[M][f] (dtype) = silu(gu[:, :f]) * gu[:, f:]
 cudaError_t launch_swiglu(const float* gu, void* act, void* act_lo, int32_t dtype, int32_t rows, int32_t f,
