@@ -151,13 +151,20 @@ def bench_tree_attention(trj, torch, peaks, steps, warmup):
         def one_pass():
             for c in range(n_caches):
                 trj.tree_attention(q[c], k[c], v[c], seq_len, row_off, anc_d, max_rows=rows, max_len=total, out=o[c], workspace=ws)
-        for _ in range(warmup):
+        side = torch.cuda.Stream()
+        with torch.cuda.stream(side):
             one_pass()
+        torch.cuda.synchronize()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=side):
+            one_pass()
+        for _ in range(warmup):
+            graph.replay()
         torch.cuda.synchronize()
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         e0.record()
         for _ in range(steps):
-            one_pass()
+            graph.replay()
         e1.record()
         torch.cuda.synchronize()
         us = e0.elapsed_time(e1) * 1e3 / (steps * n_caches)
@@ -283,8 +290,19 @@ def run_ours(args, rank, world, local_rank):
         model.accept(d_tok, d_par, d_dep, d_off, pred, out=acc)
         model.compact_kv(acc["k_acc"], acc["path"])
 
-    for _ in range(max(args.warmup, 3)):
+    # the launch sequence of a step is fixed, so it is replayed from a CUDA graph (no host work per launch)
+    side = torch.cuda.Stream(device=dev)
+    with torch.cuda.stream(side):
+        for _ in range(3):
+            resident_step()
+    torch.cuda.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    l0 = trj.launch_count()
+    with torch.cuda.graph(graph, stream=side):
         resident_step()
+    launches_per_step = trj.launch_count() - l0
+    for _ in range(max(args.warmup, 3)):
+        graph.replay()
     torch.cuda.synchronize()
 
     def barrier():
@@ -296,14 +314,13 @@ def run_ours(args, rank, world, local_rank):
     sampler = ClockSampler(local_rank)
     barrier()
     sampler.start()
-    launches0 = trj.launch_count()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     e0.record()
     for _ in range(args.steps):
-        resident_step()
+        graph.replay()
     e1.record()
     barrier()
-    launches = trj.launch_count() - launches0
+    launches = launches_per_step * args.steps
     ms_total = e0.elapsed_time(e1)
 
     # ---- timed region 2: end to end through trj_step_host (host ints in, host result out)
@@ -328,12 +345,21 @@ def run_ours(args, rank, world, local_rank):
     barrier()
     clocks = sampler.stop()
 
-    # ---- per-kernel device time of the same step (profiled pass, not part of `value`)
+    # ---- per-kernel device time of the same step: a second graph whose launches are bracketed by event
+    #      nodes (not part of `value`; the brackets cost a little)
     model.profile_enable(True)
-    for _ in range(args.steps):
+    pgraph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(pgraph, stream=side):
         resident_step()
-    torch.cuda.synchronize()
-    prof = model.profile_read()
+    prof = {k: [0.0, 0] for k in trj.PROF_CATEGORIES}
+    for i in range(args.steps + 1):
+        pgraph.replay()
+        torch.cuda.synchronize()
+        if i == 0:
+            continue                                         # first replay warms the instantiated graph
+        for k, (ms, n) in model.profile_read(keep=True).items():
+            prof[k][0] += ms
+            prof[k][1] += n
     model.profile_enable(False)
 
     # ---- aggregate over ranks: max time, summed units

@@ -250,7 +250,11 @@ trj_status trj_prefill(trj_ctx* ctx, void* k_cache, void* v_cache, int32_t* seq_
  *   host out: tokens/parent [M] (the tree that was scored), node_argmax [M],
  *             *k_acc, path [TRJ_PATH_STRIDE], *bonus, *n_rows
  *   dev     : k_cache, v_cache, seq_len [1] (advanced by k_acc + 1)
- *   max_len : host-known bound of seq_len[0] + M */
+ *   max_len : host-known bound of seq_len[0] + M
+ * From the second call on a context the launch sequence is captured once per
+ * (tree rows, launch geometry, buffer addresses) into a CUDA graph on a stream of
+ * the context and replayed; it still runs after everything already enqueued on
+ * `stream` and has completed when the call returns. */
 trj_status trj_step_host(trj_ctx* ctx, void* k_cache, void* v_cache, int32_t* seq_len, int32_t max_len,
                          int32_t root, const int32_t* window, int32_t W,
                          const int32_t* branches, int32_t R, int32_t branch_len,
@@ -278,11 +282,13 @@ trj_status trj_gemm(const void* x, const void* w, float* y, int32_t M, int32_t N
  * the launches per category (0 element-wise/norm, 1 projections, 2 rotary +
  * K/V append, 3 tree attention, 4 arg-max/accept, 5 compaction) into
  * ms[TRJ_PROF_CATEGORIES] / launches[TRJ_PROF_CATEGORIES] (host) and clears
- * the record. */
+ * the record unless keep != 0.  Launches made while the stream is being captured
+ * record their events as nodes of the graph, so every replay of that graph times
+ * itself again (read with keep = 1 after each replay). */
 #define TRJ_PROF_CATEGORIES 6
 uint64_t   trj_launch_count(void);
 trj_status trj_profile_enable(trj_ctx* ctx, int32_t on);
-trj_status trj_profile_read(trj_ctx* ctx, float* ms, int32_t* launches);
+trj_status trj_profile_read(trj_ctx* ctx, float* ms, int32_t* launches, int32_t keep);
 
 #ifdef __cplusplus
 }

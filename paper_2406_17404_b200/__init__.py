@@ -77,7 +77,7 @@ _SIGNATURES = {
     "trj_gemm": (_I, [_VP, _VP, _VP, _I, _I, _I, _I, _VP, _SZ, _VP]),
     "trj_launch_count": (C.c_uint64, []),
     "trj_profile_enable": (_I, [_VP, _I]),
-    "trj_profile_read": (_I, [_VP, C.POINTER(C.c_float), _I32P]),
+    "trj_profile_read": (_I, [_VP, C.POINTER(C.c_float), _I32P, _I]),
 }
 PROF_CATEGORIES = ("elementwise", "gemm", "rope_kv", "attention", "argmax_accept", "compact")
 EXPORTS = tuple(_SIGNATURES)
@@ -334,11 +334,11 @@ class Model:
     def profile_enable(self, on: bool = True) -> None:
         _check(lib().trj_profile_enable(self._handle, 1 if on else 0))
 
-    def profile_read(self) -> Dict[str, Tuple[float, int]]:
-        """trj_profile_read: {category: (device ms, launches)} since the last read."""
+    def profile_read(self, keep: bool = False) -> Dict[str, Tuple[float, int]]:
+        """trj_profile_read: {category: (device ms, launches)} since the last read (kept if ``keep``)."""
         ms = (C.c_float * len(PROF_CATEGORIES))()
         n = (C.c_int32 * len(PROF_CATEGORIES))()
-        _check(lib().trj_profile_read(self._handle, ms, n))
+        _check(lib().trj_profile_read(self._handle, ms, n, 1 if keep else 0))
         return {c: (float(ms[i]), int(n[i])) for i, c in enumerate(PROF_CATEGORIES)}
 
     def prefill(self, tokens, b: int = 0, stream=None):

@@ -126,6 +126,10 @@ struct trj_ctx {
     int32_t* pin_in; int32_t* pin_out;   // pinned host mirrors
     // optional per-launch device timing (trj_profile_enable)
     bool prof_on = false; std::vector<cudaEvent_t> prof_ev; std::vector<int> prof_cat; size_t prof_used = 0;
+    // CUDA graphs of trj_step_host, one per (tree rows, attention grid, buffers)
+    struct GraphEntry { int32_t M; int grid; void* k; void* v; void* len; cudaGraphExec_t exec; };
+    std::vector<GraphEntry> graphs;
+    cudaStream_t cap_stream = nullptr; cudaEvent_t order_ev = nullptr; uint64_t steps_done = 0;
 };
 
 namespace {
@@ -191,14 +195,21 @@ trj_status check_cfg(const trj_model_cfg* c) {
 enum { PROF_ELEMENTWISE = 0, PROF_GEMM = 1, PROF_ROPE = 2, PROF_ATTENTION = 3, PROF_ARGMAX = 4, PROF_COMPACT = 5 };
 constexpr size_t PROF_MAX_LAUNCHES = 8192;
 
+// Inside a stream capture the records become event nodes of the graph (external events), so a replayed
+// graph times its own kernels without any host gap in between.
+unsigned prof_flags(cudaStream_t st) {
+    cudaStreamCaptureStatus cs = cudaStreamCaptureStatusNone;
+    if (cudaStreamIsCapturing(st, &cs) != cudaSuccess) return cudaEventRecordDefault;
+    return cs == cudaStreamCaptureStatusActive ? cudaEventRecordExternal : cudaEventRecordDefault;
+}
 void prof_begin(trj_ctx* ctx, int cat, cudaStream_t st) {
     if (!ctx->prof_on || ctx->prof_used >= PROF_MAX_LAUNCHES) return;
     ctx->prof_cat[ctx->prof_used] = cat;
-    cudaEventRecord(ctx->prof_ev[2 * ctx->prof_used], st);
+    cudaEventRecordWithFlags(ctx->prof_ev[2 * ctx->prof_used], st, prof_flags(st));
 }
 void prof_end(trj_ctx* ctx, cudaStream_t st) {
     if (!ctx->prof_on || ctx->prof_used >= PROF_MAX_LAUNCHES) return;
-    cudaEventRecord(ctx->prof_ev[2 * ctx->prof_used + 1], st);
+    cudaEventRecordWithFlags(ctx->prof_ev[2 * ctx->prof_used + 1], st, prof_flags(st));
     ++ctx->prof_used;
 }
 #define LAUNCH(cat, expr)                  \
@@ -311,9 +322,13 @@ extern "C" trj_status trj_create(const trj_model_cfg* cfg, const trj_weights* w,
     if (e == cudaSuccess) e = cudaMemcpy(ctx->unit_row_off, unit, sizeof(unit), cudaMemcpyHostToDevice);
     if (e == cudaSuccess) e = cudaMallocHost((void**)&ctx->pin_in, STEP_IN_BYTES);
     if (e == cudaSuccess) e = cudaMallocHost((void**)&ctx->pin_out, sizeof(int32_t) * STEP_OUT_INTS);
+    if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&ctx->cap_stream, cudaStreamNonBlocking);
+    if (e == cudaSuccess) e = cudaEventCreateWithFlags(&ctx->order_ev, cudaEventDisableTiming);
     if (e != cudaSuccess) {
         if (ctx->pin_in) cudaFreeHost(ctx->pin_in);
         if (ctx->pin_out) cudaFreeHost(ctx->pin_out);
+        if (ctx->cap_stream) cudaStreamDestroy(ctx->cap_stream);
+        if (ctx->order_ev) cudaEventDestroy(ctx->order_ev);
         delete ctx;
         return fail(TRJ_ECUDA, "create: %s", cudaGetErrorString(e));
     }
@@ -326,6 +341,9 @@ extern "C" trj_status trj_destroy(trj_ctx* ctx) {
     if (ctx->pin_in) cudaFreeHost(ctx->pin_in);
     if (ctx->pin_out) cudaFreeHost(ctx->pin_out);
     for (cudaEvent_t e : ctx->prof_ev) cudaEventDestroy(e);
+    for (const trj_ctx::GraphEntry& g : ctx->graphs) cudaGraphExecDestroy(g.exec);
+    if (ctx->cap_stream) cudaStreamDestroy(ctx->cap_stream);
+    if (ctx->order_ev) cudaEventDestroy(ctx->order_ev);
     delete ctx;
     return TRJ_OK;
 }
@@ -344,7 +362,7 @@ extern "C" trj_status trj_profile_enable(trj_ctx* ctx, int32_t on) {
     return TRJ_OK;
 }
 
-extern "C" trj_status trj_profile_read(trj_ctx* ctx, float* ms, int32_t* launches) {
+extern "C" trj_status trj_profile_read(trj_ctx* ctx, float* ms, int32_t* launches, int32_t keep) {
     TRJ_REQUIRE(ctx && ms && launches, TRJ_EINVAL, "profile_read: null pointer");
     for (int c = 0; c < TRJ_PROF_CATEGORIES; ++c) { ms[c] = 0.f; launches[c] = 0; }
     for (size_t i = 0; i < ctx->prof_used; ++i) {
@@ -354,7 +372,7 @@ extern "C" trj_status trj_profile_read(trj_ctx* ctx, float* ms, int32_t* launche
         ms[ctx->prof_cat[i]] += t;
         launches[ctx->prof_cat[i]] += 1;
     }
-    ctx->prof_used = 0;
+    if (!keep) ctx->prof_used = 0;
     return TRJ_OK;
 }
 
@@ -430,6 +448,65 @@ extern "C" trj_status trj_prefill(trj_ctx* ctx, void* k_cache, void* v_cache, in
     return TRJ_OK;
 }
 
+namespace {
+
+// Everything trj_step_host puts on a stream between the host-side tree build and the final synchronise.
+trj_status enqueue_step(trj_ctx* ctx, void* k_cache, void* v_cache, int32_t* seq_len, int32_t M, int32_t max_len,
+                        cudaStream_t st) {
+    const trj_model_cfg& c = ctx->cfg;
+    TRJ_CHECK_CUDA(cudaMemcpyAsync(ctx->step_in, ctx->pin_in, STEP_IN_BYTES, cudaMemcpyHostToDevice, st));
+    int32_t* d_tokens = ctx->step_in, *d_parent = d_tokens + TRJ_MAX_ROWS, *d_depth = d_tokens + 2 * TRJ_MAX_ROWS;
+    int32_t* d_off = d_tokens + 3 * TRJ_MAX_ROWS;
+    uint64_t* d_anc = (uint64_t*)(d_tokens + STEP_IN_INTS);
+    int32_t* d_pred = ctx->step_out, *d_k = d_pred + TRJ_MAX_ROWS, *d_bonus = d_k + 1, *d_path = d_k + 2;
+    Batch bt{seq_len, d_off, 1, M, M, max_len};
+    trj_status s = forward(ctx, k_cache, v_cache, 0, bt, d_tokens, d_depth, d_anc, 2, 0, M, st);
+    if (s != TRJ_OK) return s;
+    LAUNCH(PROF_ARGMAX, launch_argmax_accept(ctx->logits, TRJ_F32, c.vocab, d_tokens, d_parent, d_depth, d_off, 1, M, d_pred,
+                                             nullptr, d_k, d_path, d_bonus, true, true, ctx->argmax_ws, st));
+    LAUNCH(PROF_COMPACT, launch_compact(k_cache, v_cache, c.n_layers, c.max_batch, 1, c.n_heads, c.max_seq, c.head_dim,
+                                        c.dtype, seq_len, d_k, d_path, st));
+    TRJ_CHECK_CUDA(cudaMemcpyAsync(ctx->pin_out, ctx->step_out, sizeof(int32_t) * STEP_OUT_INTS, cudaMemcpyDeviceToHost, st));
+    return TRJ_OK;
+}
+
+// The launch sequence of a step depends only on the tree size, the attention grid and the buffer addresses,
+// so after the first (plain) step it is captured once per such key and replayed as a CUDA graph.
+trj_status run_step(trj_ctx* ctx, void* k_cache, void* v_cache, int32_t* seq_len, int32_t M, int32_t max_len,
+                    cudaStream_t st) {
+    const int grid = tree_attention_grid(1, ctx->cfg.n_heads, max_len);
+    if (ctx->prof_on || ctx->steps_done == 0 || !ctx->cap_stream) {
+        trj_status s = enqueue_step(ctx, k_cache, v_cache, seq_len, M, max_len, st);
+        if (s != TRJ_OK) return s;
+        TRJ_CHECK_CUDA(cudaStreamSynchronize(st));
+        return TRJ_OK;
+    }
+    cudaGraphExec_t exec = nullptr;
+    for (const trj_ctx::GraphEntry& g : ctx->graphs)
+        if (g.M == M && g.grid == grid && g.k == k_cache && g.v == v_cache && g.len == seq_len) exec = g.exec;
+    if (!exec) {
+        cudaGraph_t graph = nullptr;
+        TRJ_CHECK_CUDA(cudaStreamBeginCapture(ctx->cap_stream, cudaStreamCaptureModeThreadLocal));
+        trj_status s = enqueue_step(ctx, k_cache, v_cache, seq_len, M, max_len, ctx->cap_stream);
+        cudaError_t e = cudaStreamEndCapture(ctx->cap_stream, &graph);
+        if (s != TRJ_OK) { if (graph) cudaGraphDestroy(graph); return s; }
+        if (e != cudaSuccess) return fail(TRJ_ECUDA, "step_host: graph capture: %s", cudaGetErrorString(e));
+        e = cudaGraphInstantiate(&exec, graph, 0);
+        cudaGraphDestroy(graph);
+        if (e != cudaSuccess) return fail(TRJ_ECUDA, "step_host: graph instantiate: %s", cudaGetErrorString(e));
+        if (ctx->graphs.size() >= 32) { cudaGraphExecDestroy(ctx->graphs.front().exec); ctx->graphs.erase(ctx->graphs.begin()); }
+        ctx->graphs.push_back({M, grid, k_cache, v_cache, seq_len, exec});
+    }
+    // keep the order of the caller's stream: the graph runs after everything already enqueued on it
+    TRJ_CHECK_CUDA(cudaEventRecord(ctx->order_ev, st));
+    TRJ_CHECK_CUDA(cudaStreamWaitEvent(ctx->cap_stream, ctx->order_ev, 0));
+    TRJ_CHECK_CUDA(cudaGraphLaunch(exec, ctx->cap_stream));
+    TRJ_CHECK_CUDA(cudaStreamSynchronize(ctx->cap_stream));
+    return TRJ_OK;
+}
+
+}  // namespace
+
 extern "C" trj_status trj_step_host(trj_ctx* ctx, void* k_cache, void* v_cache, int32_t* seq_len, int32_t max_len,
                                     int32_t root, const int32_t* window, int32_t W,
                                     const int32_t* branches, int32_t R, int32_t branch_len,
@@ -449,20 +526,9 @@ extern "C" trj_status trj_step_host(trj_ctx* ctx, void* k_cache, void* v_cache, 
     s = check_step_args(ctx, 1, M, M, max_len, 2);
     if (s != TRJ_OK) return s;
     h_off[0] = 0; h_off[1] = M;
-    TRJ_CHECK_CUDA(cudaMemcpyAsync(ctx->step_in, in, STEP_IN_BYTES, cudaMemcpyHostToDevice, st));
-    int32_t* d_tokens = ctx->step_in, *d_parent = d_tokens + TRJ_MAX_ROWS, *d_depth = d_tokens + 2 * TRJ_MAX_ROWS;
-    int32_t* d_off = d_tokens + 3 * TRJ_MAX_ROWS;
-    uint64_t* d_anc = (uint64_t*)(d_tokens + STEP_IN_INTS);
-    int32_t* d_pred = ctx->step_out, *d_k = d_pred + TRJ_MAX_ROWS, *d_bonus = d_k + 1, *d_path = d_k + 2;
-    Batch bt{seq_len, d_off, 1, M, M, max_len};
-    s = forward(ctx, k_cache, v_cache, 0, bt, d_tokens, d_depth, d_anc, 2, 0, M, st);
+    s = run_step(ctx, k_cache, v_cache, seq_len, M, max_len, st);
     if (s != TRJ_OK) return s;
-    LAUNCH(PROF_ARGMAX, launch_argmax_accept(ctx->logits, TRJ_F32, c.vocab, d_tokens, d_parent, d_depth, d_off, 1, M, d_pred,
-                                             nullptr, d_k, d_path, d_bonus, true, true, ctx->argmax_ws, st));
-    LAUNCH(PROF_COMPACT, launch_compact(k_cache, v_cache, c.n_layers, c.max_batch, 1, c.n_heads, c.max_seq, c.head_dim,
-                                        c.dtype, seq_len, d_k, d_path, st));
-    TRJ_CHECK_CUDA(cudaMemcpyAsync(ctx->pin_out, ctx->step_out, sizeof(int32_t) * STEP_OUT_INTS, cudaMemcpyDeviceToHost, st));
-    TRJ_CHECK_CUDA(cudaStreamSynchronize(st));
+    ++ctx->steps_done;
     std::memcpy(tokens, h_tokens, sizeof(int32_t) * M);
     std::memcpy(parent, h_parent, sizeof(int32_t) * M);
     *n_rows = M;

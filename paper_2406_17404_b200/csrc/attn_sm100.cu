@@ -560,6 +560,12 @@ constexpr int AT_MAX_GRID = 148;
 
 }  // namespace
 
+// The host only knows an upper bound of the key count; CTAs whose range turns out empty leave at once.
+int tree_attention_grid(int32_t B, int32_t H, int32_t max_len) {
+    const long long units_bound = (long long)B * H * ((max_len + AT_KEYS - 1) / AT_KEYS);
+    return (int)(units_bound < AT_MAX_GRID ? units_bound : AT_MAX_GRID);
+}
+
 bool tree_attention_tc_supported(int32_t D, int32_t dtype, int32_t max_rows) {
     return D == AT_D && dtype == TRJ_BF16 && max_rows <= AT_ROWS && at_encode_fn() != nullptr;
 }
@@ -592,9 +598,7 @@ cudaError_t launch_tree_attention_tc(const void* q, const void* k_slab, const vo
     p.status = (int*)workspace;
     p.slots = (float*)((char*)workspace + 256);
     p.scale_log2 = 1.4426950408889634f / sqrtf((float)AT_D);
-    // the host only knows an upper bound of the key count; CTAs whose range is empty leave at once
-    const long long units_bound = (long long)bt.B * H * ((bt.max_len + AT_KEYS - 1) / AT_KEYS);
-    const int grid = (int)(units_bound < AT_MAX_GRID ? units_bound : AT_MAX_GRID);
+    const int grid = tree_attention_grid(bt.B, H, bt.max_len);
     count_launch();
     tree_attention_tc_kernel<<<grid, AT_THREADS, AT_SMEM, st>>>(map_q, map_k, map_v, p);
     cudaError_t e = cudaGetLastError();

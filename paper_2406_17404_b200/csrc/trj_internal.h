@@ -74,6 +74,7 @@ cudaError_t launch_tree_attention_generic(const void* q, const void* k_slab, con
 // 256 bytes, then split-KV partial results.
 bool tree_attention_tc_supported(int32_t D, int32_t dtype, int32_t max_rows);
 size_t tree_attention_tc_workspace(int32_t B, int32_t H);
+int tree_attention_grid(int32_t B, int32_t H, int32_t max_len);     // CTAs the tcgen05 kernel is launched with
 cudaError_t launch_tree_attention_tc(const void* q, const void* k_slab, const void* v_slab, const uint64_t* anc,
                                      int32_t anc_words, const Batch& bt, int32_t H, int32_t max_seq, void* out,
                                      void* out_lo, void* workspace, cudaStream_t st);
