@@ -230,29 +230,32 @@ trj_status forward(trj_ctx* ctx, void* k_cache, void* v_cache, int32_t b0, const
     const size_t es = dtype_size(c.dtype);
     const size_t seq_stride = (size_t)c.n_heads * c.max_seq * c.head_dim * es;     // one sequence of one layer
     LAUNCH(PROF_ELEMENTWISE, launch_embed(ctx->embed, c.dtype, tokens, ctx->h, M, d, st));
+    Parts pr{nullptr, 1, 0};                 // result of the latest projection, possibly in split-K pieces
     for (int l = 0; l < c.n_layers; ++l) {
         char* k_slab = (char*)k_cache + ((size_t)l * c.max_batch + b0) * seq_stride;
         char* v_slab = (char*)v_cache + ((size_t)l * c.max_batch + b0) * seq_stride;
-        LAUNCH(PROF_ELEMENTWISE, launch_add_rmsnorm(ctx->h, l == 0 ? nullptr : ctx->y, ctx->attn_norm[l], ctx->x, ctx->x_lo,
-                                                    c.dtype, M, d, c.rms_eps, st));
-        LAUNCH(PROF_GEMM, launch_gemm(ctx->x, ctx->x_lo, ctx->wqkv[l], ctx->y, M, 3 * HD, d, c.dtype, ctx->gemm_ws, ctx->gemm_ws_bytes, st));
-        LAUNCH(PROF_ROPE, launch_rope_kv_write(ctx->y, ctx->inv_freq, depth, bt, ctx->q, k_slab, v_slab, c.dtype,
+        LAUNCH(PROF_ELEMENTWISE, launch_add_rmsnorm(ctx->h, pr, ctx->attn_norm[l], ctx->x, ctx->x_lo, c.dtype, M, d,
+                                                    c.rms_eps, st));
+        LAUNCH(PROF_GEMM, launch_gemm(ctx->x, ctx->x_lo, ctx->wqkv[l], ctx->y, M, 3 * HD, d, c.dtype, ctx->gemm_ws,
+                                      ctx->gemm_ws_bytes, st, &pr));
+        LAUNCH(PROF_ROPE, launch_rope_kv_write(pr, ctx->inv_freq, depth, bt, ctx->q, k_slab, v_slab, c.dtype,
                                                c.n_heads, c.head_dim, c.max_seq, st));
         // inside the decoder the attention result reaches the output projection as a bf16 pair, like every
         // other projection input
         LAUNCH(PROF_ATTENTION, launch_tree_attention(ctx->q, k_slab, v_slab, anc, anc_words, bt, c.n_heads, c.head_dim,
                                                      c.max_seq, c.dtype, ctx->x, ctx->x_lo, ctx->attn_ws,
                                                      ctx->attn_ws_bytes, st));
-        LAUNCH(PROF_GEMM, launch_gemm(ctx->x, ctx->x_lo, ctx->wo[l], ctx->y, M, d, HD, c.dtype, ctx->gemm_ws, ctx->gemm_ws_bytes, st));
-        LAUNCH(PROF_ELEMENTWISE, launch_add_rmsnorm(ctx->h, ctx->y, ctx->mlp_norm[l], ctx->x, ctx->x_lo, c.dtype, M, d,
+        LAUNCH(PROF_GEMM, launch_gemm(ctx->x, ctx->x_lo, ctx->wo[l], ctx->y, M, d, HD, c.dtype, ctx->gemm_ws,
+                                      ctx->gemm_ws_bytes, st, &pr));
+        LAUNCH(PROF_ELEMENTWISE, launch_add_rmsnorm(ctx->h, pr, ctx->mlp_norm[l], ctx->x, ctx->x_lo, c.dtype, M, d,
                                                     c.rms_eps, st));
         LAUNCH(PROF_GEMM, launch_gemm(ctx->x, ctx->x_lo, ctx->w_gate_up[l], ctx->y, M, 2 * c.d_ff, d, c.dtype, ctx->gemm_ws,
-                                      ctx->gemm_ws_bytes, st));
-        LAUNCH(PROF_ELEMENTWISE, launch_swiglu(ctx->y, ctx->act, ctx->act_lo, c.dtype, M, c.d_ff, st));
+                                      ctx->gemm_ws_bytes, st, &pr));
+        LAUNCH(PROF_ELEMENTWISE, launch_swiglu(pr, ctx->act, ctx->act_lo, c.dtype, M, c.d_ff, st));
         LAUNCH(PROF_GEMM, launch_gemm(ctx->act, ctx->act_lo, ctx->w_down[l], ctx->y, M, d, c.d_ff, c.dtype, ctx->gemm_ws,
-                                      ctx->gemm_ws_bytes, st));
+                                      ctx->gemm_ws_bytes, st, &pr));
     }
-    LAUNCH(PROF_ELEMENTWISE, launch_add_rmsnorm(ctx->h, ctx->y, ctx->final_norm, ctx->x, ctx->x_lo, c.dtype, M, d,
+    LAUNCH(PROF_ELEMENTWISE, launch_add_rmsnorm(ctx->h, pr, ctx->final_norm, ctx->x, ctx->x_lo, c.dtype, M, d,
                                                 c.rms_eps, st));
     if (lm_rows > 0) {
         const size_t off = (size_t)lm_first * d * es;

@@ -470,13 +470,14 @@ __global__ void __launch_bounds__(AT_THREADS, 1) tree_attention_tc_kernel(const 
 }
 
 // Merges the pieces of every (sequence, head) that more than one CTA worked on.  One CTA per
-// (sequence, head), thread = row; pieces are taken in ascending CTA order.
+// (sequence, head, 16-wide slice of head_dim), thread = row; pieces are taken in ascending CTA order.
+constexpr int CB_COLS = 16;
 __global__ void __launch_bounds__(128) tree_attention_combine_kernel(const AtParams p, int grid_main) {
     __shared__ Sched sched;
-    __shared__ float stage[AT_ROWS][33];
+    __shared__ float stage[AT_ROWS][CB_COLS + 1];
     if (threadIdx.x == 0) build_sched(sched, p);
     __syncthreads();
-    const int bh = blockIdx.x, b = bh / p.H, h = bh % p.H;
+    const int bh = blockIdx.x, b = bh / p.H, h = bh % p.H, c0 = blockIdx.y * CB_COLS;
     const long long U = sched.first[p.B];
     const long long u0 = sched.first[b] + (long long)h * sched.tiles[b], u1 = u0 + sched.tiles[b];
     // CTA c of the main kernel owns units [U*c/G, U*(c+1)/G): the owner of unit u is the largest c with U*c/G <= u
@@ -490,41 +491,33 @@ __global__ void __launch_bounds__(128) tree_attention_combine_kernel(const AtPar
         const long long rb = U * c / grid_main, re = U * (c + 1) / grid_main;
         return (rb > u0 ? rb : u0) < (re < u1 ? re : u1);
     };
-    float m_all = -INFINITY;
-    for (int c = c_first; c <= c_last; ++c)
-        if (live && has_piece(c)) m_all = fmaxf(m_all, p.slots[(size_t)(bh + c) * AT_SLOT_FLOATS + AT_D * AT_ROWS + row]);
-    float l_all = 0.f;
-    for (int c = c_first; c <= c_last; ++c) {
-        if (!live) break;
-        if (!has_piece(c)) continue;
-        const float* slot = p.slots + (size_t)(bh + c) * AT_SLOT_FLOATS;
-        const float m = slot[AT_D * AT_ROWS + row];
-        if (m > -INFINITY) l_all += slot[AT_D * AT_ROWS + AT_ROWS + row] * exp2f(m - m_all);
-    }
-    const float inv = live ? 1.f / l_all : 0.f;
-    for (int c0 = 0; c0 < AT_D; c0 += 32) {
-        float acc[32];
+    if (live) {
+        float m_all = -INFINITY;
+        for (int c = c_first; c <= c_last; ++c)
+            if (has_piece(c)) m_all = fmaxf(m_all, p.slots[(size_t)(bh + c) * AT_SLOT_FLOATS + AT_D * AT_ROWS + row]);
+        float l_all = 0.f, acc[CB_COLS];
 #pragma unroll
-        for (int i = 0; i < 32; ++i) acc[i] = 0.f;
-        for (int c = c_first; c <= c_last && live; ++c) {
+        for (int i = 0; i < CB_COLS; ++i) acc[i] = 0.f;
+        for (int c = c_first; c <= c_last; ++c) {
             if (!has_piece(c)) continue;
             const float* slot = p.slots + (size_t)(bh + c) * AT_SLOT_FLOATS;
             const float m = slot[AT_D * AT_ROWS + row];
             if (m == -INFINITY) continue;
             const float wgt = exp2f(m - m_all);
+            l_all = fmaf(slot[AT_D * AT_ROWS + AT_ROWS + row], wgt, l_all);
 #pragma unroll
-            for (int i = 0; i < 32; ++i) acc[i] = fmaf(slot[(size_t)(c0 + i) * AT_ROWS + row], wgt, acc[i]);
+            for (int i = 0; i < CB_COLS; ++i) acc[i] = fmaf(slot[(size_t)(c0 + i) * AT_ROWS + row], wgt, acc[i]);
         }
+        const float inv = 1.f / l_all;
 #pragma unroll
-        for (int i = 0; i < 32; ++i) stage[row][i] = acc[i] * inv;
-        __syncthreads();
-        // 128 rows x 32 values -> each thread stores 8 consecutive values (16 bytes) of one row
-        for (int i = threadIdx.x; i < rows * 4; i += 128) {
-            const int r = i >> 2, q4 = (i & 3) * 8;
-            const size_t off = ((size_t)(p.row_off[b] + r) * p.H + h) * AT_D + c0 + q4;
-            store8_split(p.out + off, p.out_lo ? p.out_lo + off : nullptr, &stage[r][q4]);
-        }
-        __syncthreads();
+        for (int i = 0; i < CB_COLS; ++i) stage[row][i] = acc[i] * inv;
+    }
+    __syncthreads();
+    // rows x 16 values -> each thread stores 8 consecutive values (16 bytes) of one row
+    for (int i = threadIdx.x; i < rows * 2; i += 128) {
+        const int r = i >> 1, q8 = (i & 1) * 8;
+        const size_t off = ((size_t)(p.row_off[b] + r) * p.H + h) * AT_D + c0 + q8;
+        store8_split(p.out + off, p.out_lo ? p.out_lo + off : nullptr, &stage[r][q8]);
     }
 }
 
@@ -604,7 +597,7 @@ cudaError_t launch_tree_attention_tc(const void* q, const void* k_slab, const vo
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
     count_launch();
-    tree_attention_combine_kernel<<<bt.B * H, 128, 0, st>>>(p, grid);
+    tree_attention_combine_kernel<<<dim3(bt.B * H, AT_D / CB_COLS), 128, 0, st>>>(p, grid);
     return cudaGetLastError();
 }
 

@@ -276,7 +276,7 @@ size_t gemm_tc_workspace(int32_t M, int32_t N, int32_t K) {
 }
 
 cudaError_t launch_gemm_tc(const void* x, const void* x_lo, const void* w, float* y, int32_t M, int32_t N, int32_t K,
-                           void* workspace, cudaStream_t st) {
+                           void* workspace, cudaStream_t st, Parts* parts) {
     int* status = (int*)workspace;
     workspace = (char*)workspace + 256;
     static std::once_flag once;
@@ -310,7 +310,8 @@ cudaError_t launch_gemm_tc(const void* x, const void* x_lo, const void* w, float
     dim3 grid((N + TC_BM - 1) / TC_BM, p.splits);
     gemm_tc_kernel<<<grid, TC_THREADS, p.stages * stage + 1024, st>>>(map_w, map_x, map_xlo, p);
     cudaError_t e = cudaGetLastError();
-    if (e != cudaSuccess || p.splits == 1) return e;
+    if (parts) *parts = Parts{p.out, p.splits, (size_t)M * N};
+    if (e != cudaSuccess || p.splits == 1 || parts) return e;
     count_launch();
     const size_t n4 = (size_t)M * N / 4;           // N % 4 == 0 is part of gemm_tc_supported
     reduce_splits_kernel<<<(unsigned)((n4 + 255) / 256 < 592 ? (n4 + 255) / 256 : 592), 256, 0, st>>>(
@@ -319,10 +320,11 @@ cudaError_t launch_gemm_tc(const void* x, const void* x_lo, const void* w, float
 }
 
 cudaError_t launch_gemm(const void* x, const void* x_lo, const void* w, float* y, int32_t M, int32_t N, int32_t K,
-                        int32_t dtype, void* workspace, size_t workspace_bytes, cudaStream_t st) {
+                        int32_t dtype, void* workspace, size_t workspace_bytes, cudaStream_t st, Parts* parts) {
     if (workspace && workspace_bytes >= gemm_tc_workspace(M, N, K) && ((uintptr_t)workspace % 256) == 0 &&
         gemm_tc_supported(x, x_lo, w, y, M, N, K, dtype))
-        return launch_gemm_tc(x, x_lo, w, y, M, N, K, workspace, st);
+        return launch_gemm_tc(x, x_lo, w, y, M, N, K, workspace, st, parts);
+    if (parts) *parts = whole(y);
     return launch_gemm_simt(x, x_lo, w, y, M, N, K, dtype, st);
 }
 

@@ -34,6 +34,21 @@ __device__ __forceinline__ float warp_max(float v) {
     return v;
 }
 
+// Sum of the split-K pieces of a projection result at flat index i (fixed order).
+__device__ __forceinline__ float parts_at(const Parts& p, size_t i) {
+    float v = p.ptr[i];
+    for (int s = 1; s < p.splits; ++s) v += p.ptr[(size_t)s * p.stride + i];
+    return v;
+}
+__device__ __forceinline__ float4 parts_at4(const Parts& p, size_t i4) {
+    float4 v = reinterpret_cast<const float4*>(p.ptr)[i4];
+    for (int s = 1; s < p.splits; ++s) {
+        const float4 b = reinterpret_cast<const float4*>(p.ptr + (size_t)s * p.stride)[i4];
+        v.x += b.x; v.y += b.y; v.z += b.z; v.w += b.w;
+    }
+    return v;
+}
+
 // Sequence that owns a global row (B is small: linear scan of the offsets).
 __device__ __forceinline__ int seq_of_row(const int32_t* row_off, int B, int row) {
     int b = 0;
@@ -51,8 +66,79 @@ __global__ void embed_kernel(const T* __restrict__ embed, const int32_t* __restr
 }
 
 // ---------------------------------------------------------------- residual add + RMSNorm
+// One CTA per row.  h += add (summing the split-K pieces of `add` on the way), x = rmsnorm(h) * gain.
+// Fast path: d % 4 == 0 and d <= 4 * 256 * RMS_CHUNKS; the row lives in registers between the two phases.
+constexpr int RMS_THREADS = 256;
+constexpr int RMS_CHUNKS = 8;
+
+__device__ __forceinline__ float block_sum(float v, float* red) {
+    v = warp_sum(v);
+    if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = v;
+    __syncthreads();
+    if (threadIdx.x < 32) {
+        float t = threadIdx.x < (blockDim.x >> 5) ? red[threadIdx.x] : 0.f;
+        t = warp_sum(t);
+        if (threadIdx.x == 0) red[0] = t;
+    }
+    __syncthreads();
+    return red[0];
+}
+
 template <typename T>
-__global__ void add_rmsnorm_kernel(float* __restrict__ h, const float* __restrict__ add,
+__device__ __forceinline__ void store_split4(T* hi, T* lo, size_t i, float4 v);
+template <>
+__device__ __forceinline__ void store_split4<float>(float* hi, float*, size_t i, float4 v) {
+    *reinterpret_cast<float4*>(hi + i) = v;
+}
+template <>
+__device__ __forceinline__ void store_split4<__nv_bfloat16>(__nv_bfloat16* hi, __nv_bfloat16* lo, size_t i, float4 v) {
+    const __nv_bfloat162 a = __floats2bfloat162_rn(v.x, v.y), b = __floats2bfloat162_rn(v.z, v.w);
+    uint2 pk;
+    pk.x = *reinterpret_cast<const uint32_t*>(&a); pk.y = *reinterpret_cast<const uint32_t*>(&b);
+    *reinterpret_cast<uint2*>(hi + i) = pk;
+    if (lo) {
+        const __nv_bfloat162 c = __floats2bfloat162_rn(v.x - __low2float(a), v.y - __high2float(a));
+        const __nv_bfloat162 e = __floats2bfloat162_rn(v.z - __low2float(b), v.w - __high2float(b));
+        pk.x = *reinterpret_cast<const uint32_t*>(&c); pk.y = *reinterpret_cast<const uint32_t*>(&e);
+        *reinterpret_cast<uint2*>(lo + i) = pk;
+    }
+}
+
+template <typename T>
+__global__ void __launch_bounds__(RMS_THREADS) add_rmsnorm_vec_kernel(float* __restrict__ h, const Parts add,
+                                                                     const float* __restrict__ gain, T* __restrict__ x,
+                                                                     T* __restrict__ x_lo, int d, float eps) {
+    __shared__ float red[32];
+    const int row = blockIdx.x, n4 = d >> 2;
+    float4 v[RMS_CHUNKS];
+    float ss = 0.f;
+#pragma unroll
+    for (int k = 0; k < RMS_CHUNKS; ++k) {
+        const int j = threadIdx.x + k * RMS_THREADS;
+        if (j < n4) {
+            v[k] = reinterpret_cast<const float4*>(h + (size_t)row * d)[j];
+            if (add.ptr) {
+                const float4 a = parts_at4(add, (size_t)row * n4 + j);
+                v[k].x += a.x; v[k].y += a.y; v[k].z += a.z; v[k].w += a.w;
+                reinterpret_cast<float4*>(h + (size_t)row * d)[j] = v[k];
+            }
+            ss += v[k].x * v[k].x + v[k].y * v[k].y + v[k].z * v[k].z + v[k].w * v[k].w;
+        }
+    }
+    const float inv = rsqrtf(block_sum(ss, red) / (float)d + eps);
+#pragma unroll
+    for (int k = 0; k < RMS_CHUNKS; ++k) {
+        const int j = threadIdx.x + k * RMS_THREADS;
+        if (j < n4) {
+            const float4 g = reinterpret_cast<const float4*>(gain)[j];
+            store_split4<T>(x, x_lo, (size_t)row * d + 4 * j,
+                            make_float4(v[k].x * inv * g.x, v[k].y * inv * g.y, v[k].z * inv * g.z, v[k].w * inv * g.w));
+        }
+    }
+}
+
+template <typename T>
+__global__ void add_rmsnorm_kernel(float* __restrict__ h, const Parts add,
                                    const float* __restrict__ gain, T* __restrict__ x, T* __restrict__ x_lo,
                                    int d, float eps) {
     __shared__ float red[32];
@@ -61,19 +147,10 @@ __global__ void add_rmsnorm_kernel(float* __restrict__ h, const float* __restric
     float ss = 0.f;
     for (int c = threadIdx.x; c < d; c += blockDim.x) {
         float v = hr[c];
-        if (add) { v += add[(size_t)row * d + c]; hr[c] = v; }
+        if (add.ptr) { v += parts_at(add, (size_t)row * d + c); hr[c] = v; }
         ss += v * v;
     }
-    ss = warp_sum(ss);
-    if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = ss;
-    __syncthreads();
-    if (threadIdx.x < 32) {
-        float t = threadIdx.x < (blockDim.x >> 5) ? red[threadIdx.x] : 0.f;
-        t = warp_sum(t);
-        if (threadIdx.x == 0) red[0] = t;
-    }
-    __syncthreads();
-    const float inv = rsqrtf(red[0] / (float)d + eps);
+    const float inv = rsqrtf(block_sum(ss, red) / (float)d + eps);
     for (int c = threadIdx.x; c < d; c += blockDim.x) store_split(x, x_lo, (size_t)row * d + c, hr[c] * inv * gain[c]);
 }
 
@@ -130,7 +207,7 @@ __global__ void __launch_bounds__(256) gemm_simt_kernel(const T* __restrict__ x,
 
 // ---------------------------------------------------------------- rotary embedding + K/V append
 template <typename T>
-__global__ void rope_kv_write_kernel(const float* __restrict__ qkv, const double* __restrict__ inv_freq,
+__global__ void rope_kv_write_kernel(const Parts qkv, const double* __restrict__ inv_freq,
                                      const int32_t* __restrict__ depth, const int32_t* __restrict__ seq_len,
                                      const int32_t* __restrict__ row_off, int B, T* __restrict__ q_out,
                                      T* __restrict__ k_slab, T* __restrict__ v_slab, int H, int D, int max_seq) {
@@ -139,20 +216,20 @@ __global__ void rope_kv_write_kernel(const float* __restrict__ qkv, const double
     const int local = row - row_off[b];
     const int pos = seq_len[b] + depth[row];
     const int half = D >> 1, HD = H * D;
-    const float* src = qkv + (size_t)row * 3 * HD + hh * D;
+    const size_t src = (size_t)row * 3 * HD + hh * D;        // flat index into the projection result
     const size_t cache_row = (((size_t)b * H + hh) * max_seq + seq_len[b] + local) * D;
     for (int i = threadIdx.x; i < half; i += blockDim.x) {
         double s, c;
         sincos((double)pos * inv_freq[i], &s, &c);
         const float cs = (float)c, sn = (float)s;
-        const float qa = src[i], qb = src[i + half];
+        const float qa = parts_at(qkv, src + i), qb = parts_at(qkv, src + i + half);
         q_out[(size_t)row * HD + hh * D + i] = from_f<T>(qa * cs - qb * sn);
         q_out[(size_t)row * HD + hh * D + i + half] = from_f<T>(qb * cs + qa * sn);
-        const float ka = src[HD + i], kb = src[HD + i + half];
+        const float ka = parts_at(qkv, src + HD + i), kb = parts_at(qkv, src + HD + i + half);
         k_slab[cache_row + i] = from_f<T>(ka * cs - kb * sn);
         k_slab[cache_row + i + half] = from_f<T>(kb * cs + ka * sn);
-        v_slab[cache_row + i] = from_f<T>(src[2 * HD + i]);
-        v_slab[cache_row + i + half] = from_f<T>(src[2 * HD + i + half]);
+        v_slab[cache_row + i] = from_f<T>(parts_at(qkv, src + 2 * HD + i));
+        v_slab[cache_row + i + half] = from_f<T>(parts_at(qkv, src + 2 * HD + i + half));
     }
 }
 
@@ -232,12 +309,12 @@ __global__ void __launch_bounds__(128) tree_attention_generic_kernel(
 
 // ---------------------------------------------------------------- SwiGLU
 template <typename T>
-__global__ void swiglu_kernel(const float* __restrict__ gu, T* __restrict__ act, T* __restrict__ act_lo,
+__global__ void swiglu_kernel(const Parts gu, T* __restrict__ act, T* __restrict__ act_lo,
                               int rows, int f) {
     const size_t n = (size_t)rows * f;
     for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x) {
         const size_t r = i / f, c = i % f;
-        const float g = gu[r * 2 * f + c], u = gu[r * 2 * f + f + c];
+        const float g = parts_at(gu, r * 2 * f + c), u = parts_at(gu, r * 2 * f + f + c);
         store_split(act, act_lo, i, g / (1.f + expf(-g)) * u);
     }
 }
@@ -407,10 +484,16 @@ cudaError_t launch_embed(const void* embed, int32_t dtype, const int32_t* tokens
     return cudaGetLastError();
 }
 
-cudaError_t launch_add_rmsnorm(float* h, const float* add, const float* gain, void* x, void* x_lo, int32_t dtype,
+cudaError_t launch_add_rmsnorm(float* h, const Parts& add, const float* gain, void* x, void* x_lo, int32_t dtype,
                                int32_t rows, int32_t d, float eps, cudaStream_t st) {
     count_launch();
-    DISPATCH_T(dtype, add_rmsnorm_kernel<T><<<rows, 256, 0, st>>>(h, add, gain, (T*)x, (T*)x_lo, d, eps));
+    const bool vec = d % 4 == 0 && d <= 4 * RMS_THREADS * RMS_CHUNKS && add.stride % 4 == 0 &&
+                     ((uintptr_t)h | (uintptr_t)add.ptr | (uintptr_t)gain | (uintptr_t)x | (uintptr_t)x_lo) % 16 == 0;
+    if (vec) {
+        DISPATCH_T(dtype, add_rmsnorm_vec_kernel<T><<<rows, RMS_THREADS, 0, st>>>(h, add, gain, (T*)x, (T*)x_lo, d, eps));
+    } else {
+        DISPATCH_T(dtype, add_rmsnorm_kernel<T><<<rows, 256, 0, st>>>(h, add, gain, (T*)x, (T*)x_lo, d, eps));
+    }
     return cudaGetLastError();
 }
 
@@ -422,7 +505,7 @@ cudaError_t launch_gemm_simt(const void* x, const void* x_lo, const void* w, flo
     return cudaGetLastError();
 }
 
-cudaError_t launch_rope_kv_write(const float* qkv, const double* inv_freq, const int32_t* depth,
+cudaError_t launch_rope_kv_write(const Parts& qkv, const double* inv_freq, const int32_t* depth,
                                  const Batch& bt, void* q_out, void* k_slab, void* v_slab, int32_t dtype,
                                  int32_t H, int32_t D, int32_t max_seq, cudaStream_t st) {
     count_launch();
@@ -449,7 +532,7 @@ cudaError_t launch_tree_attention_generic(const void* q, const void* k_slab, con
     return cudaGetLastError();
 }
 
-cudaError_t launch_swiglu(const float* gu, void* act, void* act_lo, int32_t dtype, int32_t rows, int32_t f,
+cudaError_t launch_swiglu(const Parts& gu, void* act, void* act_lo, int32_t dtype, int32_t rows, int32_t f,
                           cudaStream_t st) {
     count_launch();
     const size_t n = (size_t)rows * f;

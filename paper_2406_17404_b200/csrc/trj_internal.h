@@ -40,11 +40,15 @@ struct Batch {
     int32_t B, rows_total, max_rows, max_len;
 };
 
+// A projection result that may still be in split-K pieces: value(i) = sum over s < splits of ptr[s * stride + i].
+struct Parts { const float* ptr; int32_t splits; size_t stride; };
+inline Parts whole(const float* p) { return Parts{p, 1, 0}; }
+
 cudaError_t launch_embed(const void* embed, int32_t dtype, const int32_t* tokens, float* h,
                          int32_t rows, int32_t d, cudaStream_t st);
 // h += add (when add != nullptr, h is updated in place); x = rmsnorm(h) * gain, stored as dtype.
 // In bf16 models x is written as a bf16 pair: x (hi) and x_lo (the rounding error of hi); x_lo may be null.
-cudaError_t launch_add_rmsnorm(float* h, const float* add, const float* gain, void* x, void* x_lo, int32_t dtype,
+cudaError_t launch_add_rmsnorm(float* h, const Parts& add, const float* gain, void* x, void* x_lo, int32_t dtype,
                                int32_t rows, int32_t d, float eps, cudaStream_t st);
 // y[M][N] fp32 = (x + x_lo)[M][K] . w[N][K]^T (x_lo may be null), plain shared-memory tiled FMA kernel.
 cudaError_t launch_gemm_simt(const void* x, const void* x_lo, const void* w, float* y, int32_t M, int32_t N,
@@ -56,14 +60,16 @@ bool gemm_tc_supported(const void* x, const void* x_lo, const void* w, const flo
                        int32_t dtype);
 size_t gemm_tc_workspace(int32_t M, int32_t N, int32_t K);
 cudaError_t launch_gemm_tc(const void* x, const void* x_lo, const void* w, float* y, int32_t M, int32_t N, int32_t K,
-                           void* workspace, cudaStream_t st);
-// Picks the tcgen05 kernel when the shape allows it, the plain kernel otherwise.
+                           void* workspace, cudaStream_t st, Parts* parts);
+// Picks the tcgen05 kernel when the shape allows it, the plain kernel otherwise.  With `parts` non-null the
+// split-K pieces are left unreduced in the workspace for the consumer to add (*parts says where); otherwise
+// y holds the finished result.
 cudaError_t launch_gemm(const void* x, const void* x_lo, const void* w, float* y, int32_t M, int32_t N, int32_t K,
-                        int32_t dtype, void* workspace, size_t workspace_bytes, cudaStream_t st);
+                        int32_t dtype, void* workspace, size_t workspace_bytes, cudaStream_t st, Parts* parts = nullptr);
 
 // Rotary embedding of q and k at position seq_len[b] + depth[row]; q -> q_out [rows][H][D];
 // k, v -> cache rows seq_len[b] + local row of the layer slab [B][H][max_seq][D].
-cudaError_t launch_rope_kv_write(const float* qkv, const double* inv_freq, const int32_t* depth,
+cudaError_t launch_rope_kv_write(const Parts& qkv, const double* inv_freq, const int32_t* depth,
                                  const Batch& bt, void* q_out, void* k_slab, void* v_slab, int32_t dtype,
                                  int32_t H, int32_t D, int32_t max_seq, cudaStream_t st);
 cudaError_t launch_tree_attention_generic(const void* q, const void* k_slab, const void* v_slab,
@@ -86,7 +92,7 @@ cudaError_t launch_tree_attention(const void* q, const void* k_slab, const void*
                                   cudaStream_t st);
 
 // act[M][f] (dtype) = silu(gu[:, :f]) * gu[:, f:]
-cudaError_t launch_swiglu(const float* gu, void* act, void* act_lo, int32_t dtype, int32_t rows, int32_t f,
+cudaError_t launch_swiglu(const Parts& gu, void* act, void* act_lo, int32_t dtype, int32_t rows, int32_t f,
                           cudaStream_t st);
 
 // Arg-max over the vocabulary and/or acceptance.  do_argmax: compute node_argmax (+margin) from
