@@ -6,10 +6,11 @@
 //   * one thread streams Q (per segment) and the K/V tiles with TMA into 128-byte-swizzled shared memory;
 //   * one thread issues tcgen05.mma: S = Q.K^T into TMEM (two S buffers), then O += P.V with the
 //     accumulator resident in TMEM for the whole segment;
-//   * four warps own one query row per thread (TMEM lane = row): they read S, apply the ancestor bitmask
-//     on tiles that reach the tree rows, keep an online softmax whose running maximum is only raised when
-//     a tile exceeds it by more than 2^8 (then O is rescaled in TMEM), and write P as bf16 into shared
-//     memory in the layout the second MMA reads.
+//   * eight warps do the softmax: a thread owns half of one query row (TMEM lane = row, 64 of the 128
+//     columns); they read S once into registers, apply the ancestor bitmask on tiles that reach the tree
+//     rows, keep an online softmax whose running maximum is only raised when a tile exceeds it by more
+//     than 2^8 (then O is rescaled in TMEM), and write P as bf16 into shared memory in the layout the
+//     second MMA reads.
 // A segment that covers all tiles of its (sequence, head) writes the normalised bf16 output itself;
 // otherwise it leaves (max, sum, O) in the workspace and a second kernel merges the pieces in a fixed
 // order.  Every wait on an mbarrier is bounded; on expiry the CTA records TRJ_ETIMEOUT and leaves.
@@ -23,7 +24,7 @@ namespace {
 constexpr int AT_ROWS = 128;                 // query rows per CTA = UMMA M = TMEM lanes
 constexpr int AT_KEYS = 128;                 // keys per tile
 constexpr int AT_D = 128;                    // head_dim
-constexpr int AT_THREADS = 192;              // 4 softmax warps + TMA warp + MMA warp
+constexpr int AT_THREADS = 320;              // 8 softmax warps + TMA warp + MMA warp
 constexpr uint32_t AT_SUB = 128 * 128;       // one [128 x 64 bf16] swizzled sub-tile: 16 KB
 constexpr uint32_t AT_TILE = 2 * AT_SUB;     // Q, P, a K tile or a V tile: 32 KB
 constexpr int AT_RING = 4;                   // K/V ring slots (tile g: K in slot 2g%4, V in 2g%4+1)
@@ -133,6 +134,11 @@ __device__ __forceinline__ uint32_t pack_bf16(float a, float b) {
     const __nv_bfloat162 h = __floats2bfloat162_rn(a, b);      // .x (low half) = a
     return *reinterpret_cast<const uint32_t*>(&h);
 }
+__device__ __forceinline__ float fast_exp2(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
 __device__ __forceinline__ float bf16_round(float a) { return __bfloat162float(__float2bfloat16_rn(a)); }
 // Stores 8 consecutive outputs as bf16 (16 bytes) and, when asked, the rounding errors as a second bf16 vector.
 __device__ __forceinline__ void store8_split(__nv_bfloat16* hi, __nv_bfloat16* lo, const float* v) {
@@ -196,6 +202,7 @@ __global__ void __launch_bounds__(AT_THREADS, 1) tree_attention_tc_kernel(const 
     __shared__ uint32_t tmem_base_slot;
     __shared__ int abort_flag;
     __shared__ Sched sched;
+    __shared__ float pair_max[2][2][AT_ROWS], pair_sum[2][2][AT_ROWS];      // [parity][half][row]
 
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t* base_ptr = smem_raw + (base - smem_u32(smem_raw));
@@ -207,10 +214,10 @@ __global__ void __launch_bounds__(AT_THREADS, 1) tree_attention_tc_kernel(const 
     if (threadIdx.x == 0) {
         abort_flag = 0;
         build_sched(sched, p);
-        for (int i = 0; i < B_COUNT; ++i) mbar_init(bar(i), (i == B_P_READY || i == B_O_FREE) ? 128 : 1);
+        for (int i = 0; i < B_COUNT; ++i) mbar_init(bar(i), (i == B_P_READY || i == B_O_FREE) ? 256 : 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
-    if (warp == 5) {
+    if (warp == 9) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
                      ::"r"(smem_u32(&tmem_base_slot)), "r"(512u) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
@@ -225,7 +232,7 @@ __global__ void __launch_bounds__(AT_THREADS, 1) tree_attention_tc_kernel(const 
     const long long U = sched.first[p.B];
     const long long u_begin = U * blockIdx.x / gridDim.x, u_end = U * (blockIdx.x + 1) / gridDim.x;
 
-    if (warp == 4) {
+    if (warp == 8) {
         if (lane == 0) {
             // ------------------------------------------------ TMA producer
             int g = 0, e = 0;
@@ -257,7 +264,7 @@ __global__ void __launch_bounds__(AT_THREADS, 1) tree_attention_tc_kernel(const 
                 ++e;
             }
         }
-    } else if (warp == 5) {
+    } else if (warp == 9) {
         if (lane == 0) {
             // ------------------------------------------------ MMA issuer
             // S = Q.K^T: both K-major, 128 x 128.  O += P.V: P K-major, V MN-major, 128 x 128.
@@ -314,9 +321,14 @@ __global__ void __launch_bounds__(AT_THREADS, 1) tree_attention_tc_kernel(const 
             }
         }
     } else {
-        // ------------------------------------------------ softmax + epilogue: thread = query row
-        const int row = threadIdx.x;                         // 0..127 == TMEM lane
-        const uint32_t lane_addr = (uint32_t)(warp * 32) << 16;
+        // ------------------------------------------------ softmax + epilogue
+        // Eight warps: warp w owns rows 32*(w%4) .. +31 (its TMEM lanes) and key / head_dim columns
+        // 64*(w/4) .. +63, so two threads share a row and exchange their maxima and sums through shared memory.
+        const int rg = warp & 3, half = warp >> 2;
+        const int row = rg * 32 + lane;
+        const uint32_t lane_addr = (uint32_t)(rg * 32) << 16;
+        const uint32_t col0 = (uint32_t)half * 64;
+        const uint32_t pair_bar = 1 + rg;                    // named barrier of the two warps of a row group
         int g = 0, e = 0;
         bool ok = true;
         for (long long u = u_begin; u < u_end && ok;) {
@@ -324,6 +336,7 @@ __global__ void __launch_bounds__(AT_THREADS, 1) tree_attention_tc_kernel(const 
             const int n_tiles = (int)min((long long)(w.tiles - w.t), u_end - u);
             const int g0 = g, g1 = g + n_tiles;
             const bool live = row < w.rows;
+            const bool group_live = rg * 32 < w.rows;        // same for both warps of the pair
             const int grow = p.row_off[w.b] + row;           // global row (valid when live)
             uint64_t m0 = 0, m1 = 0;
             if (live) {
@@ -335,70 +348,68 @@ __global__ void __launch_bounds__(AT_THREADS, 1) tree_attention_tc_kernel(const 
             for (g = g0; g < g1 && ok; ++g) {
                 const int key0 = (w.t + (g - g0)) * AT_KEYS;
                 const bool edge = key0 + AT_KEYS > w.S;      // the tile reaches tree rows or the end of the keys
-                ok = __all_sync(0xffffffffu, mbar_wait(bar(B_S_FULL + (g & 1)), (uint32_t)(g >> 1) & 1u, &abort_flag, p.status));
-                if (!ok) break;
-                asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-                // visibility of the 128 columns of this row as two 64-bit words (bit c = key0 + c): column c is
-                // tree row tt = key0 + c - S; it is visible if tt < 0 (prefix) or if bit tt of the row's mask is set
-                uint64_t vis0 = ~0ull, vis1 = ~0ull;
-                if (edge) {
-                    const int d = key0 - w.S;                // -127 .. 127 on an edge tile
-                    if (d >= 0) { vis0 = m0; vis1 = m1; shr128(vis0, vis1, d); }
-                    else { vis0 = m0; vis1 = m1; shl128_fill(vis0, vis1, -d); }
-                }
-                // pass 1: maximum of the visible scores of the tile
+                float s[64];
                 float mt = -INFINITY;
-#pragma unroll 1
-                for (int c0 = 0; c0 < AT_KEYS; c0 += 32) {
-                    float s[32];
-                    tmem_ld32(tmem_s[g & 1] + lane_addr + c0, s);
-                    const uint32_t bits = (uint32_t)((c0 < 64 ? vis0 : vis1) >> (c0 & 63));
+                if (group_live) {
+                    ok = __all_sync(0xffffffffu, mbar_wait(bar(B_S_FULL + (g & 1)), (uint32_t)(g >> 1) & 1u, &abort_flag, p.status));
+                    if (!ok) break;
+                    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                    tmem_ld32(tmem_s[g & 1] + lane_addr + col0, s);
+                    tmem_ld32(tmem_s[g & 1] + lane_addr + col0 + 32, s + 32);
+                    if (edge) {
+                        // bit c of (vis0, vis1) = visibility of key key0 + c for this row: tree row tt = key0 + c - S
+                        // is visible if tt < 0 (prefix) or if bit tt of the row's ancestor mask is set
+                        uint64_t vis0 = m0, vis1 = m1;
+                        const int d = key0 - w.S;            // -127 .. 127 on an edge tile
+                        if (d >= 0) shr128(vis0, vis1, d); else shl128_fill(vis0, vis1, -d);
+                        const uint64_t vis = half ? vis1 : vis0;
 #pragma unroll
-                    for (int i = 0; i < 32; ++i) if ((bits >> i) & 1u) mt = fmaxf(mt, s[i]);
+                        for (int i = 0; i < 64; ++i) if (!((vis >> i) & 1ull)) s[i] = -INFINITY;
+                    }
+#pragma unroll
+                    for (int i = 0; i < 64; ++i) mt = fmaxf(mt, s[i]);
+                    pair_max[g & 1][half][row] = mt;
+                    asm volatile("bar.sync %0, 64;" ::"r"(pair_bar) : "memory");
+                    mt = fmaxf(mt, pair_max[g & 1][half ^ 1][row]) * p.scale_log2;
                 }
-                mt *= p.scale_log2;
                 // the P buffer and the O accumulator are free once the previous P.V product has finished
                 if (g > 0) ok = __all_sync(0xffffffffu, mbar_wait(bar(B_P_FREE), (uint32_t)((g - 1) & 1), &abort_flag, p.status));
                 if (!ok) break;
-                asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-                float factor = 1.f;
-                if (live && mt > -INFINITY) {
-                    if (m_ref == -INFINITY) m_ref = mt;
-                    else if (mt > m_ref + AT_RESCALE_GAP) { factor = exp2f(m_ref - mt); m_ref = mt; }
-                }
-                if (g > g0 && __any_sync(0xffffffffu, factor != 1.f)) {
-                    l_sum *= factor;
-#pragma unroll 1
-                    for (int c0 = 0; c0 < AT_D; c0 += 32) {
-                        float o[32];
-                        tmem_ld32(tmem_o + lane_addr + c0, o);
-#pragma unroll
-                        for (int i = 0; i < 32; ++i) o[i] *= factor;
-                        tmem_st32(tmem_o + lane_addr + c0, o);
+                if (group_live) {
+                    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                    float factor = 1.f;
+                    if (live && mt > -INFINITY) {
+                        if (m_ref == -INFINITY) m_ref = mt;
+                        else if (mt > m_ref + AT_RESCALE_GAP) { factor = fast_exp2(m_ref - mt); m_ref = mt; }
                     }
-                }
-                // pass 2: P = 2^(s * c - m_ref) as bf16, into the K-major swizzled layout of the P operand
-                const float m_use = (m_ref == -INFINITY) ? 0.f : m_ref;
+                    if (g > g0 && __any_sync(0xffffffffu, factor != 1.f)) {
+                        l_sum *= factor;
 #pragma unroll 1
-                for (int c0 = 0; c0 < AT_KEYS; c0 += 32) {
-                    float s[32];
-                    tmem_ld32(tmem_s[g & 1] + lane_addr + c0, s);
-                    const uint32_t bits = live ? (uint32_t)((c0 < 64 ? vis0 : vis1) >> (c0 & 63)) : 0u;
-                    uint32_t packed[16];
+                        for (int c0 = 0; c0 < 64; c0 += 32) {
+                            float o[32];
+                            tmem_ld32(tmem_o + lane_addr + col0 + c0, o);
 #pragma unroll
-                    for (int i = 0; i < 32; i += 2) {
-                        float a = ((bits >> i) & 1u) ? bf16_round(exp2f(fmaf(s[i], p.scale_log2, -m_use))) : 0.f;
-                        float b = ((bits >> (i + 1)) & 1u) ? bf16_round(exp2f(fmaf(s[i + 1], p.scale_log2, -m_use))) : 0.f;
-                        l_sum += a + b;
-                        packed[i >> 1] = pack_bf16(a, b);
+                            for (int i = 0; i < 32; ++i) o[i] *= factor;
+                            tmem_st32(tmem_o + lane_addr + col0 + c0, o);
+                        }
                     }
-                    // 32 keys = four 16-byte chunks of this row inside sub-tile c0 / 64
-                    uint8_t* sub = base_ptr + AT_TILE + (c0 >> 6) * AT_SUB + row * 128;
+                    // P = 2^(s * c - m_ref) as bf16 into the K-major swizzled layout of the P operand; masked
+                    // scores are -inf and give exactly 0.  Rows past the tree keep whatever P held: their
+                    // outputs are never stored.
+                    if (live) {
+                        const float m_use = (m_ref == -INFINITY) ? 0.f : m_ref;
+                        uint8_t* prow = base_ptr + AT_TILE + half * AT_SUB + row * 128;
 #pragma unroll
-                    for (int ch = 0; ch < 4; ++ch) {
-                        const int chunk = ((c0 & 63) >> 3) + ch;
-                        *reinterpret_cast<uint4*>(sub + ((chunk ^ (row & 7)) << 4)) =
-                            make_uint4(packed[4 * ch], packed[4 * ch + 1], packed[4 * ch + 2], packed[4 * ch + 3]);
+                        for (int ch = 0; ch < 8; ++ch) {
+                            float pv[8];
+#pragma unroll
+                            for (int i = 0; i < 8; ++i) {
+                                pv[i] = fast_exp2(fmaf(s[8 * ch + i], p.scale_log2, -m_use));
+                                l_sum += pv[i];
+                            }
+                            *reinterpret_cast<uint4*>(prow + ((ch ^ (row & 7)) << 4)) =
+                                make_uint4(pack_bf16(pv[0], pv[1]), pack_bf16(pv[2], pv[3]), pack_bf16(pv[4], pv[5]), pack_bf16(pv[6], pv[7]));
+                        }
                     }
                 }
                 // keys past the end of the sequence hold whatever the cache holds: clear those V rows so
@@ -409,7 +420,7 @@ __global__ void __launch_bounds__(AT_THREADS, 1) tree_attention_tc_kernel(const 
                     if (!ok) break;
                     uint8_t* v_ptr = base_ptr + 2 * AT_TILE + slot * AT_TILE;
                     const int first_bad = max(total - key0, 0);
-                    for (int i = first_bad * 8 + row; i < AT_KEYS * 8; i += 128) {      // 16-byte chunks, both sub-tiles
+                    for (int i = first_bad * 8 + (int)threadIdx.x; i < AT_KEYS * 8; i += 256) {      // 16-byte chunks, both sub-tiles
                         *reinterpret_cast<uint4*>(v_ptr + i * 16) = make_uint4(0, 0, 0, 0);
                         *reinterpret_cast<uint4*>(v_ptr + AT_SUB + i * 16) = make_uint4(0, 0, 0, 0);
                     }
@@ -423,34 +434,39 @@ __global__ void __launch_bounds__(AT_THREADS, 1) tree_attention_tc_kernel(const 
             ok = __all_sync(0xffffffffu, mbar_wait(bar(B_O_READY), (uint32_t)(e & 1), &abort_flag, p.status));
             if (!ok) break;
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-            const bool whole = (w.t == 0 && n_tiles == w.tiles);
-            if (whole) {
-                const float inv = live ? 1.f / l_sum : 0.f;
-                const size_t off = ((size_t)grow * p.H + w.h) * AT_D;
+            if (group_live) {
+                pair_sum[e & 1][half][row] = l_sum;
+                asm volatile("bar.sync %0, 64;" ::"r"(pair_bar) : "memory");
+                const float l_row = l_sum + pair_sum[e & 1][half ^ 1][row];
+                const bool whole_seg = (w.t == 0 && n_tiles == w.tiles);
+                if (whole_seg) {
+                    const float inv = live ? 1.f / l_row : 0.f;
+                    const size_t off = ((size_t)grow * p.H + w.h) * AT_D + col0;
 #pragma unroll 1
-                for (int c0 = 0; c0 < AT_D; c0 += 32) {
-                    float o[32];
-                    tmem_ld32(tmem_o + lane_addr + c0, o);
-                    if (live) {
+                    for (int c0 = 0; c0 < 64; c0 += 32) {
+                        float o[32];
+                        tmem_ld32(tmem_o + lane_addr + col0 + c0, o);
+                        if (live) {
 #pragma unroll
-                        for (int i = 0; i < 32; ++i) o[i] *= inv;
+                            for (int i = 0; i < 32; ++i) o[i] *= inv;
 #pragma unroll
-                        for (int ch = 0; ch < 4; ++ch)
-                            store8_split(p.out + off + c0 + 8 * ch, p.out_lo ? p.out_lo + off + c0 + 8 * ch : nullptr, o + 8 * ch);
+                            for (int ch = 0; ch < 4; ++ch)
+                                store8_split(p.out + off + c0 + 8 * ch, p.out_lo ? p.out_lo + off + c0 + 8 * ch : nullptr, o + 8 * ch);
+                        }
                     }
-                }
-            } else {
-                float* slot = p.slots + (size_t)(w.bh + (int)blockIdx.x) * AT_SLOT_FLOATS;
+                } else {
+                    float* slot = p.slots + (size_t)(w.bh + (int)blockIdx.x) * AT_SLOT_FLOATS;
 #pragma unroll 1
-                for (int c0 = 0; c0 < AT_D; c0 += 32) {
-                    float o[32];
-                    tmem_ld32(tmem_o + lane_addr + c0, o);
-                    if (live) {
+                    for (int c0 = 0; c0 < 64; c0 += 32) {
+                        float o[32];
+                        tmem_ld32(tmem_o + lane_addr + col0 + c0, o);
+                        if (live) {
 #pragma unroll
-                        for (int i = 0; i < 32; ++i) slot[(size_t)(c0 + i) * AT_ROWS + row] = o[i];
+                            for (int i = 0; i < 32; ++i) slot[(size_t)(col0 + c0 + i) * AT_ROWS + row] = o[i];
+                        }
                     }
+                    if (live && half == 0) { slot[AT_D * AT_ROWS + row] = m_ref; slot[AT_D * AT_ROWS + AT_ROWS + row] = l_row; }
                 }
-                if (live) { slot[AT_D * AT_ROWS + row] = m_ref; slot[AT_D * AT_ROWS + AT_ROWS + row] = l_sum; }
             }
             asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
             mbar_arrive(bar(B_O_FREE));
@@ -465,7 +481,7 @@ __global__ void __launch_bounds__(AT_THREADS, 1) tree_attention_tc_kernel(const 
         for (int i = 0; i < 64; ++i) __nanosleep(1000);
         __syncthreads();
     }
-    if (warp == 5)
+    if (warp == 9)
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(512u) : "memory");
 }
 
