@@ -188,6 +188,35 @@ trj_status trj_argmax_accept(const void* logits, int32_t dtype, int32_t V,
                              void* workspace, size_t workspace_bytes, void* stream);
 
 /* ------------------------------------------------------------------------
+ * trj_argmax_accept for callers that cannot hand over a workspace (the paper has
+ * no counterpart; this is a deployment convenience).  Some hosts of this library
+ * are not allowed to allocate device memory at all: a plug-in of an inference
+ * server that is given nothing but its input and output buffers, or a process
+ * whose memory pool was reserved in full at start-up by another framework, so
+ * that a cudaMalloc from inside a call would fail or break that framework's
+ * accounting.  For them the scratch (tickets and per-slice arg-max candidates)
+ * lives in a fixed array inside the library's device image, TRJ_STATIC_MAX_ROWS
+ * rows' worth (about 48 KB), which every GPU that loads the library keeps for the
+ * lifetime of the process.  Same inputs, outputs and results as
+ * trj_argmax_accept.  The call allocates nothing, neither device nor pinned
+ * memory.
+ *   - rows_total > TRJ_STATIC_MAX_ROWS is refused with TRJ_ECAPACITY (use the
+ *     workspace variant for larger batches).
+ *   - The first call on a device looks up the array's device address (a one-time
+ *     set-up done with that device current); make that first call outside any
+ *     stream capture.
+ *   - All calls on a device share the one array.  The tickets are cleared at the
+ *     start of every call, so the previous call's contents do not matter, but two
+ *     calls whose kernels overlap on the GPU (for instance on different
+ *     streams) corrupt each other: serialise them. */
+#define TRJ_STATIC_MAX_ROWS 1024
+trj_status trj_argmax_accept_static(const void* logits, int32_t dtype, int32_t V,
+                                    const int32_t* tokens, const int32_t* parent, const int32_t* depth,
+                                    const int32_t* row_off, int32_t B, int32_t rows_total,
+                                    int32_t* node_argmax, float* margin,
+                                    int32_t* k_acc, int32_t* path, int32_t* bonus, void* stream);
+
+/* ------------------------------------------------------------------------
  * KV compaction of the accepted path (implied by Section 3.3: decoding
  * continues from the accepted tokens).  For every layer, head and both K and
  * V, row seq_len[b] + path[b][j] moves to row seq_len[b] + j, j = 1..k_acc[b]

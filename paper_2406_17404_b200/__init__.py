@@ -63,6 +63,7 @@ _SIGNATURES = {
     "trj_tree_attention": (_I, [_VP, _VP, _VP, _VP, _VP, _VP, _I, _I, _I, _I, _I, _I, _I, _I, _I, _VP, _VP, _SZ, _VP]),
     "trj_argmax_accept_workspace": (_SZ, [_I, _I]),
     "trj_argmax_accept": (_I, [_VP, _I, _I, _VP, _VP, _VP, _VP, _I, _I, _VP, _VP, _VP, _VP, _VP, _VP, _SZ, _VP]),
+    "trj_argmax_accept_static": (_I, [_VP, _I, _I, _VP, _VP, _VP, _VP, _I, _I, _VP, _VP, _VP, _VP, _VP, _VP]),
     "trj_compact_rows": (_I, [_VP, _VP, _I, _I, _I, _I, _I, _I, _VP, _VP, _VP, _VP]),
     "trj_workspace_bytes": (_SZ, [C.POINTER(ModelCfg)]),
     "trj_create": (_I, [C.POINTER(ModelCfg), C.POINTER(Weights), _VP, _SZ, C.POINTER(_VP)]),
@@ -253,6 +254,28 @@ def argmax_accept(logits, tokens, parent, depth, row_off, *, want_margin: bool =
         batch, rows, _dev(node_argmax), _dev(margin) if want_margin else None, _dev(k_acc), _dev(path), _dev(bonus),
         _dev(workspace, torch.uint8, "workspace"), workspace.numel(), _stream(stream)))
     return {"node_argmax": node_argmax, "margin": margin, "k_acc": k_acc, "path": path, "bonus": bonus}
+
+
+STATIC_MAX_ROWS = 1024
+
+
+def argmax_accept_static(logits, tokens, parent, depth, row_off, out, *, stream=None) -> None:
+    """trj_argmax_accept_static: the workspace-free variant of :func:`argmax_accept`.
+
+    For hosts that may not allocate device memory (see ``include/trj.h``): the scratch is a fixed array inside
+    the library, good for ``STATIC_MAX_ROWS`` rows in total.  Nothing is allocated here either: ``out`` must hold
+    preallocated CUDA tensors ``node_argmax`` [rows] int32, ``margin`` [rows] float32 (or None), ``k_acc`` [B],
+    ``path`` [B, PATH_STRIDE] and ``bonus`` [B] int32.  Calls share the one array, so do not let two of them run
+    on the GPU at the same time; make the first call on a device outside any stream capture."""
+    torch = _torch()
+    rows, vocab = logits.shape
+    batch = row_off.numel() - 1
+    margin = out.get("margin")
+    _check(lib().trj_argmax_accept_static(
+        _dev(logits, name="logits"), _dtype_code(logits), vocab, _dev(tokens, torch.int32, "tokens"),
+        _dev(parent, torch.int32, "parent"), _dev(depth, torch.int32, "depth"), _dev(row_off, torch.int32, "row_off"),
+        batch, rows, _dev(out["node_argmax"], torch.int32), _dev(margin, torch.float32) if margin is not None else None,
+        _dev(out["k_acc"], torch.int32), _dev(out["path"], torch.int32), _dev(out["bonus"], torch.int32), _stream(stream)))
 
 
 def compact_rows(k_cache, v_cache, seq_len, k_acc, path, stream=None) -> None:

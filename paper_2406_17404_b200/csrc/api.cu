@@ -80,6 +80,24 @@ extern "C" trj_status trj_argmax_accept(const void* logits, int32_t dtype, int32
     return TRJ_OK;
 }
 
+extern "C" trj_status trj_argmax_accept_static(const void* logits, int32_t dtype, int32_t V,
+                                               const int32_t* tokens, const int32_t* parent, const int32_t* depth,
+                                               const int32_t* row_off, int32_t B, int32_t rows_total,
+                                               int32_t* node_argmax, float* margin,
+                                               int32_t* k_acc, int32_t* path, int32_t* bonus, void* stream) {
+    TRJ_REQUIRE(logits && tokens && parent && depth && row_off && node_argmax && k_acc && path && bonus,
+                TRJ_EINVAL, "argmax_accept_static: null pointer");
+    TRJ_REQUIRE(dtype_ok(dtype), TRJ_EINVAL, "argmax_accept_static: unknown dtype %d", dtype);
+    TRJ_REQUIRE(V >= 1 && B >= 1 && rows_total >= B, TRJ_EINVAL, "argmax_accept_static: bad sizes (every tree has a root)");
+    TRJ_REQUIRE(B <= TRJ_MAX_BATCH, TRJ_ECAPACITY, "argmax_accept_static: batch %d exceeds %d", B, TRJ_MAX_BATCH);
+    TRJ_REQUIRE(rows_total <= TRJ_STATIC_MAX_ROWS, TRJ_ECAPACITY,
+                "argmax_accept_static: %d rows exceed the built-in scratch of %d rows; use trj_argmax_accept with a workspace",
+                rows_total, TRJ_STATIC_MAX_ROWS);
+    TRJ_CHECK_CUDA(launch_argmax_accept_static(logits, dtype, V, tokens, parent, depth, row_off, B, rows_total,
+                                               node_argmax, margin, k_acc, path, bonus, (cudaStream_t)stream));
+    return TRJ_OK;
+}
+
 extern "C" trj_status trj_compact_rows(void* k_cache, void* v_cache, int32_t L, int32_t B, int32_t H,
                                        int32_t max_seq, int32_t D, int32_t dtype, int32_t* seq_len,
                                        const int32_t* k_acc, const int32_t* path, void* stream) {

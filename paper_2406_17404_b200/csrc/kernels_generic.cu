@@ -2,6 +2,7 @@
 // They serve every shape the specialised sm_100a kernels do not cover (fp32 models, odd head
 // sizes) and all the small element-wise steps between the projections.
 #include <atomic>
+#include <mutex>
 #include "trj_internal.h"
 
 namespace trj {
@@ -562,6 +563,56 @@ cudaError_t launch_argmax_accept(const void* logits, int32_t dtype, int32_t V,
     } else if (do_accept) {
         accept_only_kernel<<<B, 32, 0, st>>>(tokens, parent, depth, row_off, node_argmax, k_acc, path, bonus);
     }
+    return cudaGetLastError();
+}
+
+// ---------------------------------------------------------------- arg-max + accept without a caller workspace
+// Scratch of the allocation-free entry point: the tickets and the per-slice candidates live in this
+// file-scope device array, which every GPU that loads the library holds until the process exits.
+constexpr int STATIC_MAX_ROWS = TRJ_STATIC_MAX_ROWS;
+constexpr size_t STATIC_TICKET_BYTES = 256;
+constexpr size_t STATIC_SCRATCH_BYTES = STATIC_TICKET_BYTES + sizeof(Top) * ARGMAX_CHUNKS * (size_t)STATIC_MAX_ROWS;
+static __device__ __align__(256) unsigned char g_static_scratch[STATIC_SCRATCH_BYTES];
+
+// In host code `g_static_scratch` is only a handle for the runtime, not an address a kernel can use: the
+// device address is looked up once per device (with that device current) and remembered.
+static cudaError_t static_scratch_address(void** out) {
+    constexpr int MAX_DEVICES = 64;
+    static std::mutex mu;
+    static void* addr[MAX_DEVICES] = {};
+    int dev = -1;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    if (dev < 0 || dev >= MAX_DEVICES) return cudaErrorInvalidDevice;
+    std::lock_guard<std::mutex> lock(mu);
+    if (!addr[dev]) {
+        void* p = nullptr;
+        e = cudaGetSymbolAddress(&p, g_static_scratch);
+        if (e != cudaSuccess) return e;
+        addr[dev] = p;
+    }
+    *out = addr[dev];
+    return cudaSuccess;
+}
+
+cudaError_t launch_argmax_accept_static(const void* logits, int32_t dtype, int32_t V,
+                                        const int32_t* tokens, const int32_t* parent, const int32_t* depth,
+                                        const int32_t* row_off, int32_t B, int32_t rows_total,
+                                        int32_t* node_argmax, float* margin, int32_t* k_acc, int32_t* path,
+                                        int32_t* bonus, cudaStream_t st) {
+    void* scratch = nullptr;
+    cudaError_t e = static_scratch_address(&scratch);
+    if (e != cudaSuccess) return e;
+    // the array keeps whatever the previous call left: the tickets must start at zero
+    e = cudaMemsetAsync(scratch, 0, STATIC_TICKET_BYTES, st);
+    if (e != cudaSuccess) return e;
+    count_launch();
+    unsigned int* tickets = (unsigned int*)scratch;
+    Top* partial = (Top*)((char*)scratch + STATIC_TICKET_BYTES);
+    dim3 grid(rows_total, ARGMAX_CHUNKS);
+    DISPATCH_T(dtype, argmax_accept_kernel<T><<<grid, ARGMAX_THREADS, 0, st>>>(
+                          (const T*)logits, V, tokens, parent, depth, row_off, B, node_argmax, margin, k_acc,
+                          path, bonus, 1, tickets, partial));
     return cudaGetLastError();
 }
 

@@ -104,6 +104,13 @@ cudaError_t launch_argmax_accept(const void* logits, int32_t dtype, int32_t V,
                                  int32_t* node_argmax, float* margin, int32_t* k_acc, int32_t* path,
                                  int32_t* bonus, bool do_argmax, bool do_accept, void* ws, cudaStream_t st);
 
+// Same kernel with its scratch in a file-scope device array of the library (no workspace argument).
+cudaError_t launch_argmax_accept_static(const void* logits, int32_t dtype, int32_t V,
+                                        const int32_t* tokens, const int32_t* parent, const int32_t* depth,
+                                        const int32_t* row_off, int32_t B, int32_t rows_total,
+                                        int32_t* node_argmax, float* margin, int32_t* k_acc, int32_t* path,
+                                        int32_t* bonus, cudaStream_t st);
+
 cudaError_t launch_compact(void* k_cache, void* v_cache, int32_t L, int32_t B_cache, int32_t B, int32_t H,
                            int32_t max_seq, int32_t D, int32_t dtype, int32_t* seq_len,
                            const int32_t* k_acc, const int32_t* path, cudaStream_t st);
