@@ -20,19 +20,20 @@ namespace {
 
 constexpr int TC_BM = 128;            // weight rows per CTA = UMMA M
 constexpr int TC_BK = 64;             // bf16 elements per stage row = one 128-byte swizzle span
-constexpr int TC_THREADS = 128;
+constexpr int TC_THREADS = 192;           // TMA warp, MMA warp, four epilogue warps
 constexpr int TC_MAX_STAGES = 8;
 constexpr uint32_t TC_A_BYTES = TC_BM * TC_BK * 2;
+constexpr int TC_GRID = 148;              // one persistent CTA per SM
 constexpr uint32_t WAIT_LIMIT = 1u << 21;   // polls before a wait gives up (well over 100 ms)
 
 struct TcParams {
     int M, N, K;
-    int m_pad;          // activation rows rounded up to 16
+    int m_pad;          // activation rows rounded up (8 with a lo half, else 16)
     int halves;         // 1: x only, 2: x and x_lo
-    int n_mma;          // accumulator columns = m_pad * halves
-    int tmem_cols;      // power of two >= max(32, n_mma)
+    int n_mma;          // accumulator columns = m_pad * halves, a multiple of 16
+    int acc_cols;       // TMEM columns of one accumulator buffer: power of two >= max(16, n_mma); two are allocated
     int kblocks;        // K / 64
-    int splits, stages;
+    int tiles, splits, stages;
     float* out;         // [splits][M][N]
     int* status;        // device word: 0, or TRJ_ETIMEOUT once a wait expired
 };
@@ -41,6 +42,9 @@ __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)_
 
 __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
     asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
 }
 __device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
     asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
@@ -105,12 +109,16 @@ __device__ __forceinline__ void tmem_ld16(uint32_t taddr, float* v) {
     for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]);
 }
 
-__global__ void __launch_bounds__(TC_THREADS) gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w,
-                                                             const __grid_constant__ CUtensorMap map_x,
-                                                             const __grid_constant__ CUtensorMap map_xlo,
-                                                             const TcParams p) {
+// Persistent kernel: CTA c works on items c, c + grid, c + 2*grid, ... where an item is one 128-row weight tile
+// restricted to one K range (tile = item / splits, split = item % splits).  The TMA ring runs through item
+// boundaries, and the accumulator is double-buffered in TMEM so that the epilogue of one item overlaps the
+// loads and MMAs of the next.  Warp 0: TMA producer, warp 1: MMA issuer, warps 2-5: epilogue.
+__global__ void __launch_bounds__(TC_THREADS, 1) gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w,
+                                                                const __grid_constant__ CUtensorMap map_x,
+                                                                const __grid_constant__ CUtensorMap map_xlo,
+                                                                const TcParams p) {
     extern __shared__ uint8_t smem_raw[];
-    __shared__ __align__(8) uint64_t bars[2 * TC_MAX_STAGES + 1];
+    __shared__ __align__(8) uint64_t bars[2 * TC_MAX_STAGES + 4];
     __shared__ uint32_t tmem_base_slot;
     __shared__ int abort_flag;
 
@@ -118,22 +126,19 @@ __global__ void __launch_bounds__(TC_THREADS) gemm_tc_kernel(const __grid_consta
     const uint32_t b_bytes = (uint32_t)p.n_mma * TC_BK * 2;
     const uint32_t stage_bytes = TC_A_BYTES + b_bytes;
     const uint32_t full0 = smem_u32(&bars[0]), empty0 = smem_u32(&bars[TC_MAX_STAGES]);
-    const uint32_t accum_bar = smem_u32(&bars[2 * TC_MAX_STAGES]);
+    const uint32_t acc_full0 = smem_u32(&bars[2 * TC_MAX_STAGES]), acc_empty0 = smem_u32(&bars[2 * TC_MAX_STAGES + 2]);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int n0 = blockIdx.x * TC_BM;
-    const int kb0 = (int)((long long)blockIdx.y * p.kblocks / p.splits);
-    const int kb1 = (int)((long long)(blockIdx.y + 1) * p.kblocks / p.splits);
-    const int nkb = kb1 - kb0;
+    const int items = p.tiles * p.splits;
 
     if (threadIdx.x == 0) {
         abort_flag = 0;
         for (int s = 0; s < p.stages; ++s) { mbar_init(full0 + 8 * s, 1); mbar_init(empty0 + 8 * s, 1); }
-        mbar_init(accum_bar, 1);
+        for (int b = 0; b < 2; ++b) { mbar_init(acc_full0 + 8 * b, 1); mbar_init(acc_empty0 + 8 * b, 128); }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
-    if (warp == 1) {      // one warp allocates the accumulator columns
+    if (warp == 1) {      // one warp allocates the two accumulator buffers
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
-                     ::"r"(smem_u32(&tmem_base_slot)), "r"((uint32_t)p.tmem_cols) : "memory");
+                     ::"r"(smem_u32(&tmem_base_slot)), "r"((uint32_t)(2 * p.acc_cols)) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
@@ -141,68 +146,98 @@ __global__ void __launch_bounds__(TC_THREADS) gemm_tc_kernel(const __grid_consta
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     const uint32_t tmem_base = tmem_base_slot;
 
-    if (threadIdx.x == 0) {
-        // ---------------- producer: stream weight and activation tiles
-        for (int i = 0; i < nkb; ++i) {
-            const int s = i % p.stages;
-            const uint32_t phase = (uint32_t)(i / p.stages) & 1u;
-            if (!mbar_wait(empty0 + 8 * s, phase ^ 1u, &abort_flag, p.status)) break;
-            const uint32_t a_dst = tiles_base + s * stage_bytes, b_dst = a_dst + TC_A_BYTES;
-            const uint32_t bar = full0 + 8 * s;
-            mbar_expect_tx(bar, stage_bytes);
-            const int k = (kb0 + i) * TC_BK;
-            tma_load_2d(a_dst, &map_w, k, n0, bar);
-            tma_load_2d(b_dst, &map_x, k, 0, bar);
-            if (p.halves == 2) tma_load_2d(b_dst + (uint32_t)p.m_pad * TC_BK * 2, &map_xlo, k, 0, bar);
-        }
-    } else if (threadIdx.x == 32) {
-        // ---------------- MMA issuer
-        const uint32_t idesc = umma_idesc_bf16(p.n_mma);
-        bool ok = true;
-        for (int i = 0; i < nkb && ok; ++i) {
-            const int s = i % p.stages;
-            const uint32_t phase = (uint32_t)(i / p.stages) & 1u;
-            ok = mbar_wait(full0 + 8 * s, phase, &abort_flag, p.status);
-            if (!ok) break;
-            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-            const uint32_t a_addr = tiles_base + s * stage_bytes;
-            const uint64_t a_desc = umma_desc_sw128(a_addr), b_desc = umma_desc_sw128(a_addr + TC_A_BYTES);
-#pragma unroll
-            for (int kk = 0; kk < TC_BK / 16; ++kk)      // 16 bf16 = 32 bytes = 2 descriptor units per MMA
-                umma_bf16(tmem_base, a_desc + 2 * kk, b_desc + 2 * kk, idesc, (i > 0 || kk > 0) ? 1u : 0u);
-            umma_commit(empty0 + 8 * s);                 // frees the stage once these MMAs have read it
-        }
-        if (ok) umma_commit(accum_bar);                  // accumulator complete
-    }
-    __syncwarp();
-
-    // ---------------- epilogue: lane = weight row, columns = activation rows (hi half, then lo half)
-    const bool ready = mbar_wait(accum_bar, 0, &abort_flag, p.status);
-    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-    if (ready) {
-        const int n = n0 + warp * 32 + lane;
-        const uint32_t taddr = tmem_base + ((uint32_t)(warp * 32) << 16);
-        float* out = p.out + (size_t)blockIdx.y * p.M * p.N;
-        for (int c0 = 0; c0 < p.m_pad; c0 += 16) {
-            float hi[16], lo[16];
-            tmem_ld16(taddr + c0, hi);
-            if (p.halves == 2) tmem_ld16(taddr + p.m_pad + c0, lo);
-            asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-#pragma unroll
-            for (int j = 0; j < 16; ++j) {
-                const int m = c0 + j;
-                if (m < p.M && n < p.N) out[(size_t)m * p.N + n] = p.halves == 2 ? hi[j] + lo[j] : hi[j];
+    if (warp == 0) {
+        if (lane == 0) {
+            // ---------------- producer: stream weight and activation tiles, item after item
+            int fill = 0;                                    // running stage counter
+            bool ok = true;
+            for (int item = blockIdx.x; item < items && ok; item += gridDim.x) {
+                const int tile = item / p.splits, split = item % p.splits;
+                const int kb0 = (int)((long long)split * p.kblocks / p.splits);
+                const int kb1 = (int)((long long)(split + 1) * p.kblocks / p.splits);
+                for (int kb = kb0; kb < kb1; ++kb, ++fill) {
+                    const int s = fill % p.stages;
+                    const uint32_t phase = (uint32_t)(fill / p.stages) & 1u;
+                    ok = mbar_wait(empty0 + 8 * s, phase ^ 1u, &abort_flag, p.status);
+                    if (!ok) break;
+                    const uint32_t a_dst = tiles_base + s * stage_bytes, b_dst = a_dst + TC_A_BYTES;
+                    const uint32_t bar = full0 + 8 * s;
+                    mbar_expect_tx(bar, stage_bytes);
+                    tma_load_2d(a_dst, &map_w, kb * TC_BK, tile * TC_BM, bar);
+                    tma_load_2d(b_dst, &map_x, kb * TC_BK, 0, bar);
+                    if (p.halves == 2) tma_load_2d(b_dst + (uint32_t)p.m_pad * TC_BK * 2, &map_xlo, kb * TC_BK, 0, bar);
+                }
             }
         }
+    } else if (warp == 1) {
+        if (lane == 0) {
+            // ---------------- MMA issuer
+            const uint32_t idesc = umma_idesc_bf16(p.n_mma);
+            int fill = 0, j = 0;
+            bool ok = true;
+            for (int item = blockIdx.x; item < items && ok; item += gridDim.x, ++j) {
+                const int split = item % p.splits;
+                const int nkb = (int)((long long)(split + 1) * p.kblocks / p.splits) - (int)((long long)split * p.kblocks / p.splits);
+                const int buf = j & 1;
+                // the epilogue must have drained this accumulator buffer (two items ago)
+                ok = mbar_wait(acc_empty0 + 8 * buf, ((uint32_t)(j >> 1) & 1u) ^ 1u, &abort_flag, p.status);
+                if (!ok) break;
+                asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                const uint32_t d_tmem = tmem_base + (uint32_t)(buf * p.acc_cols);
+                for (int i = 0; i < nkb && ok; ++i, ++fill) {
+                    const int s = fill % p.stages;
+                    const uint32_t phase = (uint32_t)(fill / p.stages) & 1u;
+                    ok = mbar_wait(full0 + 8 * s, phase, &abort_flag, p.status);
+                    if (!ok) break;
+                    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                    const uint32_t a_addr = tiles_base + s * stage_bytes;
+                    const uint64_t a_desc = umma_desc_sw128(a_addr), b_desc = umma_desc_sw128(a_addr + TC_A_BYTES);
+#pragma unroll
+                    for (int kk = 0; kk < TC_BK / 16; ++kk)  // 16 bf16 = 32 bytes = 2 descriptor units per MMA
+                        umma_bf16(d_tmem, a_desc + 2 * kk, b_desc + 2 * kk, idesc, (i > 0 || kk > 0) ? 1u : 0u);
+                    umma_commit(empty0 + 8 * s);             // frees the stage once these MMAs have read it
+                }
+                if (ok) umma_commit(acc_full0 + 8 * buf);    // accumulator of this item complete
+            }
+        }
+    } else {
+        // ---------------- epilogue: lane = weight row, columns = activation rows (hi half, then lo half)
+        const int q = warp & 3;                              // TMEM lane group this warp may access
+        int j = 0;
+        bool ok = true;
+        for (int item = blockIdx.x; item < items && ok; item += gridDim.x, ++j) {
+            const int tile = item / p.splits, split = item % p.splits;
+            const int buf = j & 1;
+            ok = __all_sync(0xffffffffu, mbar_wait(acc_full0 + 8 * buf, (uint32_t)(j >> 1) & 1u, &abort_flag, p.status));
+            if (!ok) break;
+            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+            const int n = tile * TC_BM + q * 32 + lane;
+            const uint32_t taddr = tmem_base + (uint32_t)(buf * p.acc_cols) + ((uint32_t)(q * 32) << 16);
+            float* out = p.out + (size_t)split * p.M * p.N;
+            for (int c0 = 0; c0 < p.m_pad; c0 += 16) {
+                float hi[16], lo[16];
+                tmem_ld16(taddr + c0, hi);
+                if (p.halves == 2) tmem_ld16(taddr + p.m_pad + c0, lo);
+                asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+                for (int jj = 0; jj < 16; ++jj) {
+                    const int m = c0 + jj;
+                    if (m < p.M && n < p.N) out[(size_t)m * p.N + n] = p.halves == 2 ? hi[jj] + lo[jj] : hi[jj];
+                }
+            }
+            asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+            mbar_arrive(acc_empty0 + 8 * buf);
+        }
     }
+    __syncwarp();
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     __syncthreads();
-    if (abort_flag) {                                    // let copies that are still in flight land before the CTA leaves
+    if (abort_flag) {                                        // let copies that are still in flight land before the CTA leaves
         for (int i = 0; i < 64; ++i) __nanosleep(1000);
         __syncthreads();
     }
     if (warp == 1)
-        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)p.tmem_cols) : "memory");
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)(2 * p.acc_cols)) : "memory");
 }
 
 // y[i] = sum_s part[s][i], fixed order.
@@ -259,19 +294,26 @@ bool gemm_tc_supported(const void* x, const void* x_lo, const void* w, const flo
     return encode_fn() != nullptr;
 }
 
-int gemm_tc_splits(int32_t N, int32_t K) {
+// Number of K ranges per weight tile.  Items (tiles x splits) are dealt round-robin to a grid of at most 148
+// CTAs, so the choice trades balance (items close to a multiple of 148) against the extra traffic of the
+// partial sums, about 2*splits*M/K of the weight bytes.
+int gemm_tc_splits(int32_t M, int32_t N, int32_t K) {
     const int tiles = (N + TC_BM - 1) / TC_BM, kblocks = K / TC_BK;
-    const int resident = 296;                      // two CTAs of this kernel fit on each of the 148 SMs
-    int s = resident / tiles;
-    if (s > kblocks / 4) s = kblocks / 4;          // keep at least four k-blocks per CTA
-    if (s > 16) s = 16;
-    return s < 1 ? 1 : s;
+    int best = 1;
+    double best_score = 0.0;
+    for (int s = 1; s <= 16 && s <= (kblocks >= 4 ? kblocks / 4 : 1); ++s) {
+        const int items = tiles * s, rounds = (items + TC_GRID - 1) / TC_GRID;
+        const double balance = (double)items / ((double)rounds * TC_GRID);
+        const double score = balance / (1.0 + 2.0 * s * M / K);
+        if (score > best_score * 1.02) { best_score = score; best = s; }      // prefer fewer splits on near ties
+    }
+    return best;
 }
 
 // Workspace: a 256-byte header whose first word is the device status, then the split-K partial sums.
 size_t gemm_tc_workspace(int32_t M, int32_t N, int32_t K) {
     if (K % TC_BK != 0 || K < TC_BK) return 256;
-    const int s = gemm_tc_splits(N, K);
+    const int s = gemm_tc_splits(M, N, K);
     return 256 + (s > 1 ? align_up((size_t)s * M * N * sizeof(float), 256) : 0);
 }
 
@@ -287,17 +329,18 @@ cudaError_t launch_gemm_tc(const void* x, const void* x_lo, const void* w, float
     if (attr_err != cudaSuccess) return attr_err;
     TcParams p;
     p.M = M; p.N = N; p.K = K;
-    p.m_pad = round_up(M, 16);
     p.halves = x_lo ? 2 : 1;
+    p.m_pad = round_up(M, p.halves == 2 ? 8 : 16);       // the lo box must start on a 1024-byte boundary: 8 rows
     p.n_mma = p.m_pad * p.halves;
-    p.tmem_cols = 32;
-    while (p.tmem_cols < p.n_mma) p.tmem_cols *= 2;
+    // the epilogue reads 16 columns at a time from each half, so a buffer must cover the last such read
+    const int reach = (p.halves == 2 ? p.m_pad : 0) + round_up(p.m_pad, 16);
+    p.acc_cols = 16;
+    while (p.acc_cols < reach) p.acc_cols *= 2;
     p.kblocks = K / TC_BK;
-    p.splits = gemm_tc_splits(N, K);
+    p.tiles = (N + TC_BM - 1) / TC_BM;
+    p.splits = gemm_tc_splits(M, N, K);
     const size_t stage = TC_A_BYTES + (size_t)p.n_mma * TC_BK * 2;
-    size_t budget = 108 * 1024;                    // two CTAs per SM when three stages fit, else one CTA per SM
-    if (3 * stage > budget) budget = 216 * 1024;
-    p.stages = (int)(budget / stage);
+    p.stages = (int)((216 * 1024) / stage);
     if (p.stages > TC_MAX_STAGES) p.stages = TC_MAX_STAGES;
     if (p.stages < 2) return cudaErrorInvalidConfiguration;
     p.out = p.splits > 1 ? (float*)workspace : y;
@@ -307,8 +350,8 @@ cudaError_t launch_gemm_tc(const void* x, const void* x_lo, const void* w, float
         !make_map(&map_xlo, x_lo ? x_lo : x, M, K, p.m_pad))
         return cudaErrorInvalidValue;
     count_launch();
-    dim3 grid((N + TC_BM - 1) / TC_BM, p.splits);
-    gemm_tc_kernel<<<grid, TC_THREADS, p.stages * stage + 1024, st>>>(map_w, map_x, map_xlo, p);
+    const int items = p.tiles * p.splits;
+    gemm_tc_kernel<<<items < TC_GRID ? items : TC_GRID, TC_THREADS, p.stages * stage + 1024, st>>>(map_w, map_x, map_xlo, p);
     cudaError_t e = cudaGetLastError();
     if (parts) *parts = Parts{p.out, p.splits, (size_t)M * N};
     if (e != cudaSuccess || p.splits == 1 || parts) return e;
