@@ -263,6 +263,8 @@ def run_ours(args, rank, world, local_rank):
     torch.cuda.set_device(local_rank)
     dev = torch.device("cuda", local_rank)
     trj.lib()
+    if args.no_pdl:
+        trj.set_pdl(False)
     peaks = measured_peaks()
     cfg = synth.LLAMA7B if not args.layers else synth.LLAMA7B.with_layers(args.layers)
     layers, glob = device_weights(cfg, 1234 + rank, dev)
@@ -417,6 +419,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--layers", type=int, default=0, help="debug: fewer layers than the 7B shape (invalidates the number)")
+    ap.add_argument("--no-pdl", action="store_true", help="launch the kernels fully serialised (comparison only)")
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-oracle baseline leg")
     ap.add_argument("--no-attention", action="store_true", help="skip the op-level tree-attention leg")
     args = ap.parse_args()

@@ -316,6 +316,11 @@ trj_status trj_gemm(const void* x, const void* w, float* y, int32_t M, int32_t N
  * itself again (read with keep = 1 after each replay). */
 #define TRJ_PROF_CATEGORIES 6
 uint64_t   trj_launch_count(void);
+/* Programmatic dependent launch (on by default): the kernels of a step are launched so that each may
+ * be scheduled, and may prefetch weights, while its predecessor in the stream is still running.
+ * trj_set_pdl(0) launches them fully serialised instead (for comparison).  Process-wide; set it
+ * before the first step of a context, because a cached CUDA graph keeps the mode it was captured in. */
+void       trj_set_pdl(int32_t on);
 trj_status trj_profile_enable(trj_ctx* ctx, int32_t on);
 trj_status trj_profile_read(trj_ctx* ctx, float* ms, int32_t* launches, int32_t keep);
 

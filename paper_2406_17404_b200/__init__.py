@@ -77,6 +77,7 @@ _SIGNATURES = {
     "trj_gemm_workspace": (_SZ, [_I, _I, _I]),
     "trj_gemm": (_I, [_VP, _VP, _VP, _I, _I, _I, _I, _VP, _SZ, _VP]),
     "trj_launch_count": (C.c_uint64, []),
+    "trj_set_pdl": (None, [_I]),
     "trj_profile_enable": (_I, [_VP, _I]),
     "trj_profile_read": (_I, [_VP, C.POINTER(C.c_float), _I32P, _I]),
 }
@@ -106,6 +107,11 @@ def _check(status: int) -> None:
 
 def version() -> str:
     return lib().trj_version().decode()
+
+
+def set_pdl(on: bool) -> None:
+    """trj_set_pdl: programmatic dependent launch of the step's kernels on (default) or off."""
+    lib().trj_set_pdl(1 if on else 0)
 
 
 def launch_count() -> int:

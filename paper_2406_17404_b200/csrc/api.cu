@@ -370,6 +370,7 @@ extern "C" trj_status trj_destroy(trj_ctx* ctx) {
 }
 
 extern "C" uint64_t trj_launch_count(void) { return launches_so_far(); }
+extern "C" void trj_set_pdl(int32_t on) { set_pdl(on != 0); }
 
 extern "C" trj_status trj_profile_enable(trj_ctx* ctx, int32_t on) {
     TRJ_REQUIRE(ctx, TRJ_EINVAL, "profile_enable: null context");

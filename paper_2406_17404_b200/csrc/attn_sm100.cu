@@ -211,9 +211,9 @@ __global__ void __launch_bounds__(AT_THREADS, 1) tree_attention_tc_kernel(const 
     auto bar = [&](int i) { return bar0 + 8u * (uint32_t)i; };
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
+    pdl_launch_dependents();
     if (threadIdx.x == 0) {
         abort_flag = 0;
-        build_sched(sched, p);
         for (int i = 0; i < B_COUNT; ++i) mbar_init(bar(i), (i == B_P_READY || i == B_O_FREE) ? 256 : 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -222,6 +222,9 @@ __global__ void __launch_bounds__(AT_THREADS, 1) tree_attention_tc_kernel(const 
                      ::"r"(smem_u32(&tmem_base_slot)), "r"(512u) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
+    // barriers and TMEM are set up while the previous kernel may still run; its results are needed from here on
+    pdl_wait();
+    if (threadIdx.x == 0) build_sched(sched, p);
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     __syncthreads();
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
@@ -491,6 +494,7 @@ constexpr int CB_COLS = 16;
 __global__ void __launch_bounds__(128) tree_attention_combine_kernel(const AtParams p, int grid_main) {
     __shared__ Sched sched;
     __shared__ float stage[AT_ROWS][CB_COLS + 1];
+    pdl_prologue();
     if (threadIdx.x == 0) build_sched(sched, p);
     __syncthreads();
     const int bh = blockIdx.x, b = bh / p.H, h = bh % p.H, c0 = blockIdx.y * CB_COLS;
@@ -609,12 +613,12 @@ cudaError_t launch_tree_attention_tc(const void* q, const void* k_slab, const vo
     p.scale_log2 = 1.4426950408889634f / sqrtf((float)AT_D);
     const int grid = tree_attention_grid(bt.B, H, bt.max_len);
     count_launch();
-    tree_attention_tc_kernel<<<grid, AT_THREADS, AT_SMEM, st>>>(map_q, map_k, map_v, p);
-    cudaError_t e = cudaGetLastError();
+    cudaError_t e = launch_chain(tree_attention_tc_kernel, dim3(grid), dim3(AT_THREADS), AT_SMEM, st, map_q, map_k, map_v, p);
+    if (e == cudaSuccess) e = cudaGetLastError();
     if (e != cudaSuccess) return e;
     count_launch();
-    tree_attention_combine_kernel<<<dim3(bt.B * H, AT_D / CB_COLS), 128, 0, st>>>(p, grid);
-    return cudaGetLastError();
+    e = launch_chain(tree_attention_combine_kernel, dim3(bt.B * H, AT_D / CB_COLS), dim3(128), 0, st, p, grid);
+    return e != cudaSuccess ? e : cudaGetLastError();
 }
 
 cudaError_t launch_tree_attention(const void* q, const void* k_slab, const void* v_slab, const uint64_t* anc,

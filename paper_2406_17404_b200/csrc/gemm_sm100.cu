@@ -130,6 +130,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) gemm_tc_kernel(const __grid_con
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int items = p.tiles * p.splits;
 
+    pdl_launch_dependents();
     if (threadIdx.x == 0) {
         abort_flag = 0;
         for (int s = 0; s < p.stages; ++s) { mbar_init(full0 + 8 * s, 1); mbar_init(empty0 + 8 * s, 1); }
@@ -148,25 +149,41 @@ __global__ void __launch_bounds__(TC_THREADS, 1) gemm_tc_kernel(const __grid_con
 
     if (warp == 0) {
         if (lane == 0) {
-            // ---------------- producer: stream weight and activation tiles, item after item
-            int fill = 0;                                    // running stage counter
+            // ---------------- producer: stream weight and activation tiles, item after item.
+            // Weights are constants, so the first ring-full of weight tiles is requested BEFORE waiting for the
+            // previous kernel of the stream; the activation tiles of those stages follow after the wait.
             bool ok = true;
-            for (int item = blockIdx.x; item < items && ok; item += gridDim.x) {
-                const int tile = item / p.splits, split = item % p.splits;
-                const int kb0 = (int)((long long)split * p.kblocks / p.splits);
-                const int kb1 = (int)((long long)(split + 1) * p.kblocks / p.splits);
-                for (int kb = kb0; kb < kb1; ++kb, ++fill) {
-                    const int s = fill % p.stages;
-                    const uint32_t phase = (uint32_t)(fill / p.stages) & 1u;
-                    ok = mbar_wait(empty0 + 8 * s, phase ^ 1u, &abort_flag, p.status);
-                    if (!ok) break;
-                    const uint32_t a_dst = tiles_base + s * stage_bytes, b_dst = a_dst + TC_A_BYTES;
-                    const uint32_t bar = full0 + 8 * s;
-                    mbar_expect_tx(bar, stage_bytes);
-                    tma_load_2d(a_dst, &map_w, kb * TC_BK, tile * TC_BM, bar);
-                    tma_load_2d(b_dst, &map_x, kb * TC_BK, 0, bar);
-                    if (p.halves == 2) tma_load_2d(b_dst + (uint32_t)p.m_pad * TC_BK * 2, &map_xlo, kb * TC_BK, 0, bar);
+            int prefetched = 0;
+            for (int pass = 0; pass < 2 && ok; ++pass) {
+                int fill = 0;                                // running stage counter
+                for (int item = blockIdx.x; item < items && ok; item += gridDim.x) {
+                    const int tile = item / p.splits, split = item % p.splits;
+                    const int kb0 = (int)((long long)split * p.kblocks / p.splits);
+                    const int kb1 = (int)((long long)(split + 1) * p.kblocks / p.splits);
+                    for (int kb = kb0; kb < kb1; ++kb, ++fill) {
+                        const int s = fill % p.stages;
+                        const uint32_t a_dst = tiles_base + s * stage_bytes, b_dst = a_dst + TC_A_BYTES;
+                        const uint32_t bar = full0 + 8 * s;
+                        if (pass == 0) {                     // weights only, at most one ring-full
+                            if (fill >= p.stages) break;
+                            mbar_expect_tx(bar, stage_bytes);
+                            tma_load_2d(a_dst, &map_w, kb * TC_BK, tile * TC_BM, bar);
+                            prefetched = fill + 1;
+                            continue;
+                        }
+                        if (fill >= prefetched) {
+                            const uint32_t phase = (uint32_t)(fill / p.stages) & 1u;
+                            ok = mbar_wait(empty0 + 8 * s, phase ^ 1u, &abort_flag, p.status);
+                            if (!ok) break;
+                            mbar_expect_tx(bar, stage_bytes);
+                            tma_load_2d(a_dst, &map_w, kb * TC_BK, tile * TC_BM, bar);
+                        }
+                        tma_load_2d(b_dst, &map_x, kb * TC_BK, 0, bar);
+                        if (p.halves == 2) tma_load_2d(b_dst + (uint32_t)p.m_pad * TC_BK * 2, &map_xlo, kb * TC_BK, 0, bar);
+                    }
+                    if (pass == 0 && fill >= p.stages) break;
                 }
+                if (pass == 0) pdl_wait();                   // activations come from the previous kernel
             }
         }
     } else if (warp == 1) {
@@ -205,6 +222,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) gemm_tc_kernel(const __grid_con
         const int q = warp & 3;                              // TMEM lane group this warp may access
         int j = 0;
         bool ok = true;
+        pdl_wait();                                          // the output buffer may still be read by the previous kernel
         for (int item = blockIdx.x; item < items && ok; item += gridDim.x, ++j) {
             const int tile = item / p.splits, split = item % p.splits;
             const int buf = j & 1;
@@ -351,8 +369,9 @@ cudaError_t launch_gemm_tc(const void* x, const void* x_lo, const void* w, float
         return cudaErrorInvalidValue;
     count_launch();
     const int items = p.tiles * p.splits;
-    gemm_tc_kernel<<<items < TC_GRID ? items : TC_GRID, TC_THREADS, p.stages * stage + 1024, st>>>(map_w, map_x, map_xlo, p);
-    cudaError_t e = cudaGetLastError();
+    cudaError_t e = launch_chain(gemm_tc_kernel, dim3(items < TC_GRID ? items : TC_GRID), dim3(TC_THREADS),
+                                 p.stages * stage + 1024, st, map_w, map_x, map_xlo, p);
+    if (e == cudaSuccess) e = cudaGetLastError();
     if (parts) *parts = Parts{p.out, p.splits, (size_t)M * N};
     if (e != cudaSuccess || p.splits == 1 || parts) return e;
     count_launch();

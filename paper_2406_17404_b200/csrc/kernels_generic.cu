@@ -61,6 +61,7 @@ __device__ __forceinline__ int seq_of_row(const int32_t* row_off, int B, int row
 template <typename T>
 __global__ void embed_kernel(const T* __restrict__ embed, const int32_t* __restrict__ tokens,
                              float* __restrict__ h, int d) {
+    pdl_prologue();
     const int row = blockIdx.x;
     const T* src = embed + (size_t)tokens[row] * d;
     for (int c = threadIdx.x; c < d; c += blockDim.x) h[(size_t)row * d + c] = to_f(src[c]);
@@ -109,6 +110,7 @@ template <typename T>
 __global__ void __launch_bounds__(RMS_THREADS) add_rmsnorm_vec_kernel(float* __restrict__ h, const Parts add,
                                                                      const float* __restrict__ gain, T* __restrict__ x,
                                                                      T* __restrict__ x_lo, int d, float eps) {
+    pdl_prologue();
     __shared__ float red[32];
     const int row = blockIdx.x, n4 = d >> 2;
     float4 v[RMS_CHUNKS];
@@ -142,6 +144,7 @@ template <typename T>
 __global__ void add_rmsnorm_kernel(float* __restrict__ h, const Parts add,
                                    const float* __restrict__ gain, T* __restrict__ x, T* __restrict__ x_lo,
                                    int d, float eps) {
+    pdl_prologue();
     __shared__ float red[32];
     const int row = blockIdx.x;
     float* hr = h + (size_t)row * d;
@@ -212,6 +215,7 @@ __global__ void rope_kv_write_kernel(const Parts qkv, const double* __restrict__
                                      const int32_t* __restrict__ depth, const int32_t* __restrict__ seq_len,
                                      const int32_t* __restrict__ row_off, int B, T* __restrict__ q_out,
                                      T* __restrict__ k_slab, T* __restrict__ v_slab, int H, int D, int max_seq) {
+    pdl_prologue();
     const int row = blockIdx.x, hh = blockIdx.y;
     const int b = seq_of_row(row_off, B, row);
     const int local = row - row_off[b];
@@ -312,6 +316,7 @@ __global__ void __launch_bounds__(128) tree_attention_generic_kernel(
 template <typename T>
 __global__ void swiglu_kernel(const Parts gu, T* __restrict__ act, T* __restrict__ act_lo,
                               int rows, int f) {
+    pdl_prologue();
     const size_t n = (size_t)rows * f;
     for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x) {
         const size_t r = i / f, c = i % f;
@@ -374,6 +379,7 @@ __global__ void __launch_bounds__(ARGMAX_THREADS) argmax_accept_kernel(
         const int32_t* __restrict__ row_off, int B, int32_t* node_argmax,
         float* __restrict__ margin, int32_t* __restrict__ k_acc, int32_t* __restrict__ path,
         int32_t* __restrict__ bonus, int do_accept, unsigned int* tickets, Top* partial) {
+    pdl_prologue();
     __shared__ Top red[ARGMAX_THREADS / 32];
     __shared__ int last_flag;
     const int row = blockIdx.x, chunk = blockIdx.y;
@@ -420,6 +426,7 @@ __global__ void accept_only_kernel(const int32_t* __restrict__ tokens, const int
                                    const int32_t* __restrict__ depth, const int32_t* __restrict__ row_off,
                                    const int32_t* __restrict__ node_argmax, int32_t* __restrict__ k_acc,
                                    int32_t* __restrict__ path, int32_t* __restrict__ bonus) {
+    pdl_prologue();
     const int b = blockIdx.x, r0 = row_off[b], rows = row_off[b + 1] - r0;
     accept_sequence(tokens + r0, parent + r0, depth + r0, node_argmax + r0, rows,
                     k_acc + b, path + (size_t)b * TRJ_PATH_STRIDE, bonus + b);
@@ -435,6 +442,7 @@ __global__ void __launch_bounds__(256) compact_kernel(uint4* __restrict__ k_cach
                                                       const int32_t* __restrict__ seq_len,
                                                       const int32_t* __restrict__ k_acc,
                                                       const int32_t* __restrict__ path) {
+    pdl_prologue();
     extern __shared__ uint4 stage[];             // [COMPACT_BATCH][row_vec]
     int idx = blockIdx.x;
     const int kv = idx & 1; idx >>= 1;
@@ -461,6 +469,7 @@ __global__ void __launch_bounds__(256) compact_kernel(uint4* __restrict__ k_cach
 }
 
 __global__ void advance_len_kernel(int32_t* seq_len, const int32_t* k_acc, int B) {
+    pdl_prologue();
     const int b = blockIdx.x * blockDim.x + threadIdx.x;
     if (b < B) seq_len[b] += k_acc[b] + 1;
 }
@@ -470,6 +479,9 @@ __global__ void bump_len_kernel(int32_t* seq_len_b, int delta) { *seq_len_b += d
 }  // namespace
 
 // ============================================================================ launchers
+static std::atomic<bool> g_pdl{true};
+bool pdl_enabled() { return g_pdl.load(std::memory_order_relaxed); }
+void set_pdl(bool on) { g_pdl.store(on, std::memory_order_relaxed); }
 static std::atomic<uint64_t> g_launches{0};
 void count_launch() { g_launches.fetch_add(1, std::memory_order_relaxed); }
 uint64_t launches_so_far() { return g_launches.load(std::memory_order_relaxed); }
@@ -481,21 +493,23 @@ uint64_t launches_so_far() { return g_launches.load(std::memory_order_relaxed); 
 cudaError_t launch_embed(const void* embed, int32_t dtype, const int32_t* tokens, float* h,
                          int32_t rows, int32_t d, cudaStream_t st) {
     count_launch();
-    DISPATCH_T(dtype, embed_kernel<T><<<rows, 256, 0, st>>>((const T*)embed, tokens, h, d));
-    return cudaGetLastError();
+    cudaError_t launch_err = cudaSuccess;
+    DISPATCH_T(dtype, launch_err = launch_chain(embed_kernel<T>, dim3(rows), dim3(256), 0, st, (const T*)embed, tokens, h, d));
+    return launch_err != cudaSuccess ? launch_err : cudaGetLastError();
 }
 
 cudaError_t launch_add_rmsnorm(float* h, const Parts& add, const float* gain, void* x, void* x_lo, int32_t dtype,
                                int32_t rows, int32_t d, float eps, cudaStream_t st) {
     count_launch();
+    cudaError_t launch_err = cudaSuccess;
     const bool vec = d % 4 == 0 && d <= 4 * RMS_THREADS * RMS_CHUNKS && add.stride % 4 == 0 &&
                      ((uintptr_t)h | (uintptr_t)add.ptr | (uintptr_t)gain | (uintptr_t)x | (uintptr_t)x_lo) % 16 == 0;
     if (vec) {
-        DISPATCH_T(dtype, add_rmsnorm_vec_kernel<T><<<rows, RMS_THREADS, 0, st>>>(h, add, gain, (T*)x, (T*)x_lo, d, eps));
+        DISPATCH_T(dtype, launch_err = launch_chain(add_rmsnorm_vec_kernel<T>, dim3(rows), dim3(RMS_THREADS), 0, st, h, add, gain, (T*)x, (T*)x_lo, d, eps));
     } else {
-        DISPATCH_T(dtype, add_rmsnorm_kernel<T><<<rows, 256, 0, st>>>(h, add, gain, (T*)x, (T*)x_lo, d, eps));
+        DISPATCH_T(dtype, launch_err = launch_chain(add_rmsnorm_kernel<T>, dim3(rows), dim3(256), 0, st, h, add, gain, (T*)x, (T*)x_lo, d, eps));
     }
-    return cudaGetLastError();
+    return launch_err != cudaSuccess ? launch_err : cudaGetLastError();
 }
 
 cudaError_t launch_gemm_simt(const void* x, const void* x_lo, const void* w, float* y, int32_t M, int32_t N,
@@ -510,10 +524,11 @@ cudaError_t launch_rope_kv_write(const Parts& qkv, const double* inv_freq, const
                                  const Batch& bt, void* q_out, void* k_slab, void* v_slab, int32_t dtype,
                                  int32_t H, int32_t D, int32_t max_seq, cudaStream_t st) {
     count_launch();
+    cudaError_t launch_err = cudaSuccess;
     dim3 grid(bt.rows_total, H);
-    DISPATCH_T(dtype, rope_kv_write_kernel<T><<<grid, 64, 0, st>>>(qkv, inv_freq, depth, bt.seq_len, bt.row_off,
+    DISPATCH_T(dtype, launch_err = launch_chain(rope_kv_write_kernel<T>, grid, dim3(64), 0, st, qkv, inv_freq, depth, bt.seq_len, bt.row_off,
                                                                   bt.B, (T*)q_out, (T*)k_slab, (T*)v_slab, H, D, max_seq));
-    return cudaGetLastError();
+    return launch_err != cudaSuccess ? launch_err : cudaGetLastError();
 }
 
 cudaError_t launch_tree_attention_generic(const void* q, const void* k_slab, const void* v_slab,
@@ -536,10 +551,11 @@ cudaError_t launch_tree_attention_generic(const void* q, const void* k_slab, con
 cudaError_t launch_swiglu(const Parts& gu, void* act, void* act_lo, int32_t dtype, int32_t rows, int32_t f,
                           cudaStream_t st) {
     count_launch();
+    cudaError_t launch_err = cudaSuccess;
     const size_t n = (size_t)rows * f;
     const int blocks = (int)((n + 255) / 256 < 1184 ? (n + 255) / 256 : 1184);
-    DISPATCH_T(dtype, swiglu_kernel<T><<<blocks, 256, 0, st>>>(gu, (T*)act, (T*)act_lo, rows, f));
-    return cudaGetLastError();
+    DISPATCH_T(dtype, launch_err = launch_chain(swiglu_kernel<T>, dim3(blocks), dim3(256), 0, st, gu, (T*)act, (T*)act_lo, rows, f));
+    return launch_err != cudaSuccess ? launch_err : cudaGetLastError();
 }
 
 size_t argmax_workspace_bytes(int32_t rows_total, int32_t B) {
@@ -553,17 +569,19 @@ cudaError_t launch_argmax_accept(const void* logits, int32_t dtype, int32_t V,
                                  int32_t* node_argmax, float* margin, int32_t* k_acc, int32_t* path,
                                  int32_t* bonus, bool do_argmax, bool do_accept, void* ws, cudaStream_t st) {
     if (do_argmax || do_accept) count_launch();
+    cudaError_t launch_err = cudaSuccess;
     if (do_argmax) {
         unsigned int* tickets = (unsigned int*)ws;
         Top* partial = (Top*)((char*)ws + align_up(sizeof(unsigned int) * TRJ_MAX_BATCH, 256));
         dim3 grid(rows_total, ARGMAX_CHUNKS);
-        DISPATCH_T(dtype, argmax_accept_kernel<T><<<grid, ARGMAX_THREADS, 0, st>>>(
-                              (const T*)logits, V, tokens, parent, depth, row_off, B, node_argmax, margin, k_acc,
-                              path, bonus, do_accept ? 1 : 0, tickets, partial));
+        DISPATCH_T(dtype, launch_err = launch_chain(argmax_accept_kernel<T>, grid, dim3(ARGMAX_THREADS), 0, st,
+                                                    (const T*)logits, V, tokens, parent, depth, row_off, B, node_argmax,
+                                                    margin, k_acc, path, bonus, do_accept ? 1 : 0, tickets, partial));
     } else if (do_accept) {
-        accept_only_kernel<<<B, 32, 0, st>>>(tokens, parent, depth, row_off, node_argmax, k_acc, path, bonus);
+        launch_err = launch_chain(accept_only_kernel, dim3(B), dim3(32), 0, st, tokens, parent, depth, row_off,
+                                  (const int32_t*)node_argmax, k_acc, path, bonus);
     }
-    return cudaGetLastError();
+    return launch_err != cudaSuccess ? launch_err : cudaGetLastError();
 }
 
 // ---------------------------------------------------------------- arg-max + accept without a caller workspace
@@ -622,12 +640,12 @@ cudaError_t launch_compact(void* k_cache, void* v_cache, int32_t L, int32_t B_ca
     count_launch(); count_launch();
     const int row_vec = (int)(D * dtype_size(dtype) / 16);
     const size_t smem = sizeof(uint4) * COMPACT_BATCH * row_vec;
-    compact_kernel<<<L * B * H * 2, 256, smem, st>>>((uint4*)k_cache, (uint4*)v_cache, B_cache, B, H, max_seq,
-                                                     row_vec, seq_len, k_acc, path);
-    cudaError_t e = cudaGetLastError();
+    cudaError_t e = launch_chain(compact_kernel, dim3(L * B * H * 2), dim3(256), smem, st, (uint4*)k_cache, (uint4*)v_cache,
+                                 B_cache, B, H, max_seq, row_vec, (const int32_t*)seq_len, k_acc, path);
+    if (e == cudaSuccess) e = cudaGetLastError();
     if (e != cudaSuccess) return e;
-    advance_len_kernel<<<(B + 63) / 64, 64, 0, st>>>(seq_len, k_acc, B);
-    return cudaGetLastError();
+    e = launch_chain(advance_len_kernel, dim3((B + 63) / 64), dim3(64), 0, st, seq_len, k_acc, B);
+    return e != cudaSuccess ? e : cudaGetLastError();
 }
 
 cudaError_t launch_set_chunk(int32_t* row_off2, int32_t m, cudaStream_t st) {

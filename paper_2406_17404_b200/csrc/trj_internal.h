@@ -28,6 +28,31 @@ inline size_t dtype_size(int32_t dt) { return dt == TRJ_BF16 ? 2 : 4; }
 trj_status tree_from_parents_impl(const int32_t* parent, int32_t M, int32_t anc_words,
                                   int32_t* depth, uint64_t* anc);
 
+// ---- programmatic dependent launch -----------------------------------------------------------------
+// Kernels of the step are launched so that a kernel may be scheduled while its predecessor in the stream
+// is still running: every such kernel first lets ITS successor start (launch_dependents) and then waits
+// for its predecessor to finish and flush (wait) before it touches any data the predecessor may write.
+// Launched without the attribute, both instructions do nothing.
+bool pdl_enabled();
+void set_pdl(bool on);
+#ifdef __CUDACC__
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_prologue() { pdl_launch_dependents(); pdl_wait(); }
+
+template <typename... KArgs, typename... Args>
+cudaError_t launch_chain(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args&&... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = pdl_enabled() ? 1 : 0;
+    return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+#endif
+
 // ---- launch accounting: every kernel launch of the library passes through count_launch() -------
 void count_launch();
 uint64_t launches_so_far();
