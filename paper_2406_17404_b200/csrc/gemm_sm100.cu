@@ -23,7 +23,7 @@ constexpr int TC_BK = 64;             // bf16 elements per stage row = one 128-b
 constexpr int TC_THREADS = 192;           // TMA warp, MMA warp, four epilogue warps
 constexpr int TC_MAX_STAGES = 8;
 constexpr uint32_t TC_A_BYTES = TC_BM * TC_BK * 2;
-constexpr int TC_GRID = 148;              // one persistent CTA per SM
+constexpr int TC_GRID = 296;              // two persistent CTAs per SM: one's ramp and tail overlap the other's stream
 constexpr uint32_t WAIT_LIMIT = 1u << 21;   // polls before a wait gives up (well over 100 ms)
 
 struct TcParams {
@@ -113,7 +113,7 @@ __device__ __forceinline__ void tmem_ld16(uint32_t taddr, float* v) {
 // restricted to one K range (tile = item / splits, split = item % splits).  The TMA ring runs through item
 // boundaries, and the accumulator is double-buffered in TMEM so that the epilogue of one item overlaps the
 // loads and MMAs of the next.  Warp 0: TMA producer, warp 1: MMA issuer, warps 2-5: epilogue.
-__global__ void __launch_bounds__(TC_THREADS, 1) gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w,
+__global__ void __launch_bounds__(TC_THREADS, 2) gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w,
                                                                 const __grid_constant__ CUtensorMap map_x,
                                                                 const __grid_constant__ CUtensorMap map_xlo,
                                                                 const TcParams p) {
@@ -312,7 +312,7 @@ bool gemm_tc_supported(const void* x, const void* x_lo, const void* w, const flo
     return encode_fn() != nullptr;
 }
 
-// Number of K ranges per weight tile.  Items (tiles x splits) are dealt round-robin to a grid of at most 148
+// Number of K ranges per weight tile.  Items (tiles x splits) are dealt round-robin to a grid of at most 296
 // CTAs, so the choice trades balance (items close to a multiple of 148) against the extra traffic of the
 // partial sums, about 2*splits*M/K of the weight bytes.
 int gemm_tc_splits(int32_t M, int32_t N, int32_t K) {
@@ -358,8 +358,10 @@ cudaError_t launch_gemm_tc(const void* x, const void* x_lo, const void* w, float
     p.tiles = (N + TC_BM - 1) / TC_BM;
     p.splits = gemm_tc_splits(M, N, K);
     const size_t stage = TC_A_BYTES + (size_t)p.n_mma * TC_BK * 2;
-    p.stages = (int)((216 * 1024) / stage);
-    if (p.stages > TC_MAX_STAGES) p.stages = TC_MAX_STAGES;
+    // four stages in at most ~108 KB let two CTAs share an SM; wider activation tiles get one CTA per SM
+    p.stages = (int)((108 * 1024) / stage);
+    if (p.stages < 3) p.stages = (int)((216 * 1024) / stage);
+    if (p.stages > 4) p.stages = 4;
     if (p.stages < 2) return cudaErrorInvalidConfiguration;
     p.out = p.splits > 1 ? (float*)workspace : y;
     p.status = status;
