@@ -251,6 +251,24 @@ def workload_config(cfg, l2_note):
             "prefix": PROMPT, "batch": 1, "parallelism": "replicas", "l2": l2_note}
 
 
+def aggregate_over_ranks(ms_total, e2e_s, launches, world, device):
+    """Replicas only: the job takes as long as its slowest rank (MAX of the times) and launches add up."""
+    if world <= 1:
+        return ms_total, e2e_s, launches
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([ms_total, e2e_s], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    n = torch.tensor([launches], dtype=torch.int64, device=device)
+    dist.all_reduce(n, op=dist.ReduceOp.SUM)
+    return float(t[0]), float(t[1]), int(n[0])
+
+
+def whole_job_rate(world, units_per_rank, seconds):
+    """Units all ranks processed divided by the (max-over-ranks) time: every replica does the same work."""
+    return world * units_per_rank / seconds
+
+
 def run_ours(args, rank, world, local_rank):
     import torch
     import torch.distributed as dist
@@ -365,18 +383,12 @@ def run_ours(args, rank, world, local_rank):
     model.profile_enable(False)
 
     # ---- aggregate over ranks: max time, summed units
-    if world > 1:
-        t = torch.tensor([ms_total, e2e_s], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms_total, e2e_s = float(t[0]), float(t[1])
-        n = torch.tensor([launches], dtype=torch.int64, device=dev)
-        dist.all_reduce(n, op=dist.ReduceOp.SUM)
-        launches = int(n[0])
+    ms_total, e2e_s, launches = aggregate_over_ranks(ms_total, e2e_s, launches, world, dev)
     if rank != 0:
         return
     ms_step = ms_total / args.steps
-    value = world * DRAFTS / (ms_step / 1e3)
-    e2e_value = world * DRAFTS * args.steps / e2e_s
+    value = whole_job_rate(world, DRAFTS * args.steps, ms_total / 1e3)
+    e2e_value = whole_job_rate(world, DRAFTS * args.steps, e2e_s)
 
     gemm_ms, gemm_launches = prof["gemm"]
     gemm_ms_step = gemm_ms / args.steps
