@@ -4,13 +4,13 @@
 // major, are dealt in equal contiguous ranges to a persistent grid of one CTA per SM, so a long prefix
 // is split over several CTAs (split-KV) and short sequences are packed several per CTA.  Inside a CTA:
 //   * one thread streams Q (per segment) and the K/V tiles with TMA into 128-byte-swizzled shared memory;
-//   * one thread issues tcgen05.mma: S = Q.K^T into TMEM (two S buffers), then O += P.V with the
-//     accumulator resident in TMEM for the whole segment;
+//   * one thread issues tcgen05.mma: S = Q.K^T into TMEM (two S buffers), then O += P.V with P read from
+//     TMEM as well (two P buffers) and the accumulator resident in TMEM for the whole segment;
 //   * eight warps do the softmax: a thread owns half of one query row (TMEM lane = row, 64 of the 128
 //     columns); they read S once into registers, apply the ancestor bitmask on tiles that reach the tree
 //     rows, keep an online softmax whose running maximum is only raised when a tile exceeds it by more
-//     than 2^8 (then O is rescaled in TMEM), and write P as bf16 into shared memory in the layout the
-//     second MMA reads.
+//     than 2^8 (then O is rescaled in TMEM), and store P as bf16 pairs back into TMEM, where the second
+//     MMA reads it as its A operand: the softmax of a tile never waits for the previous tile's P.V.
 // A segment that covers all tiles of its (sequence, head) writes the normalised bf16 output itself;
 // otherwise it leaves (max, sum, O) in the workspace and a second kernel merges the pieces in a fixed
 // order.  Every wait on an mbarrier is bounded; on expiry the CTA records TRJ_ETIMEOUT and leaves.
@@ -27,15 +27,15 @@ constexpr int AT_D = 128;                    // head_dim
 constexpr int AT_THREADS = 320;              // 8 softmax warps + TMA warp + MMA warp
 constexpr uint32_t AT_SUB = 128 * 128;       // one [128 x 64 bf16] swizzled sub-tile: 16 KB
 constexpr uint32_t AT_TILE = 2 * AT_SUB;     // Q, P, a K tile or a V tile: 32 KB
-constexpr int AT_RING = 4;                   // K/V ring slots (tile g: K in slot 2g%4, V in 2g%4+1)
-constexpr uint32_t AT_SMEM = (2 + AT_RING) * AT_TILE + 1024;
+constexpr int AT_RING = 5;                   // K/V ring slots; load n = 2g + (0: K, 1: V) of tile g goes to slot n % 5
+constexpr uint32_t AT_SMEM = (1 + AT_RING) * AT_TILE + 1024;
 constexpr uint32_t AT_WAIT_LIMIT = 1u << 21;
 constexpr float AT_RESCALE_GAP = 8.f;        // raise the running max only when exceeded by 2^8
 constexpr size_t AT_SLOT_FLOATS = (size_t)AT_D * AT_ROWS + 2 * AT_ROWS;   // O^T [d][row], m[row], l[row]
 
 // barrier indices
-enum { B_KV_FULL = 0, B_KV_EMPTY = 4, B_Q_FULL = 8, B_Q_EMPTY = 9, B_S_FULL = 10, B_P_READY = 12, B_P_FREE = 13,
-       B_O_READY = 14, B_O_FREE = 15, B_COUNT = 16 };
+enum { B_KV_FULL = 0, B_KV_EMPTY = 5, B_Q_FULL = 10, B_Q_EMPTY = 11, B_S_FULL = 12, B_P_READY = 14, B_P_FREE = 16,
+       B_O_READY = 18, B_O_FREE = 19, B_COUNT = 20 };
 
 struct AtParams {
     const int32_t* seq_len; const int32_t* row_off; const uint64_t* anc;
@@ -97,6 +97,12 @@ __device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t a_desc, uint
                  "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
                  ::"r"(tmem_d), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
 }
+// Same with the A operand (P) read from tensor memory: lane = row, 16 contraction elements = 8 columns.
+__device__ __forceinline__ void umma_bf16_ts(uint32_t tmem_d, uint32_t tmem_a, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
+    asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+                 "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
+                 ::"r"(tmem_d), "r"(tmem_a), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
+}
 __device__ __forceinline__ void umma_commit(uint32_t bar) {
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
 }
@@ -127,6 +133,18 @@ __device__ __forceinline__ void tmem_st32(uint32_t taddr, const float* v) {
                    "r"(__float_as_uint(v[20])), "r"(__float_as_uint(v[21])), "r"(__float_as_uint(v[22])), "r"(__float_as_uint(v[23])),
                    "r"(__float_as_uint(v[24])), "r"(__float_as_uint(v[25])), "r"(__float_as_uint(v[26])), "r"(__float_as_uint(v[27])),
                    "r"(__float_as_uint(v[28])), "r"(__float_as_uint(v[29])), "r"(__float_as_uint(v[30])), "r"(__float_as_uint(v[31]))
+                 : "memory");
+    asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_st32u(uint32_t taddr, const uint32_t* v) {
+    asm volatile("tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
+                 "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, "
+                 "%17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, %32};"
+                 ::"r"(taddr),
+                   "r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3]), "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7]),
+                   "r"(v[8]), "r"(v[9]), "r"(v[10]), "r"(v[11]), "r"(v[12]), "r"(v[13]), "r"(v[14]), "r"(v[15]),
+                   "r"(v[16]), "r"(v[17]), "r"(v[18]), "r"(v[19]), "r"(v[20]), "r"(v[21]), "r"(v[22]), "r"(v[23]),
+                   "r"(v[24]), "r"(v[25]), "r"(v[26]), "r"(v[27]), "r"(v[28]), "r"(v[29]), "r"(v[30]), "r"(v[31])
                  : "memory");
     asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
 }
@@ -206,7 +224,7 @@ __global__ void __launch_bounds__(AT_THREADS, 1) tree_attention_tc_kernel(const 
 
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t* base_ptr = smem_raw + (base - smem_u32(smem_raw));
-    const uint32_t q_smem = base, p_smem = base + AT_TILE, ring_smem = base + 2 * AT_TILE;
+    const uint32_t q_smem = base, ring_smem = base + AT_TILE;
     const uint32_t bar0 = smem_u32(&bars[0]);
     auto bar = [&](int i) { return bar0 + 8u * (uint32_t)i; };
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -214,7 +232,7 @@ __global__ void __launch_bounds__(AT_THREADS, 1) tree_attention_tc_kernel(const 
     pdl_launch_dependents();
     if (threadIdx.x == 0) {
         abort_flag = 0;
-        for (int i = 0; i < B_COUNT; ++i) mbar_init(bar(i), (i == B_P_READY || i == B_O_FREE) ? 256 : 1);
+        for (int i = 0; i < B_COUNT; ++i) mbar_init(bar(i), (i == B_P_READY || i == B_P_READY + 1 || i == B_O_FREE) ? 256 : 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (warp == 9) {
@@ -229,7 +247,8 @@ __global__ void __launch_bounds__(AT_THREADS, 1) tree_attention_tc_kernel(const 
     __syncthreads();
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     const uint32_t tmem = tmem_base_slot;
-    const uint32_t tmem_s[2] = {tmem, tmem + 128}, tmem_o = tmem + 256;
+    // TMEM columns: S buffers 0-127 and 128-255, O 256-383, P buffers (bf16 pairs, 64 columns each) 384-447 and 448-511
+    const uint32_t tmem_s[2] = {tmem, tmem + 128}, tmem_o = tmem + 256, tmem_p[2] = {tmem + 384, tmem + 448};
 
     // this CTA's contiguous range of units
     const long long U = sched.first[p.B];
@@ -270,7 +289,7 @@ __global__ void __launch_bounds__(AT_THREADS, 1) tree_attention_tc_kernel(const 
     } else if (warp == 9) {
         if (lane == 0) {
             // ------------------------------------------------ MMA issuer
-            // S = Q.K^T: both K-major, 128 x 128.  O += P.V: P K-major, V MN-major, 128 x 128.
+            // S = Q.K^T: both K-major from shared memory, 128 x 128.  O += P.V: P from TMEM, V MN-major, 128 x 128.
             const uint32_t idesc_qk = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(AT_KEYS >> 3) << 17) | ((uint32_t)(AT_ROWS >> 4) << 24);
             const uint32_t idesc_pv = idesc_qk | (1u << 16);
             int g = 0, e = 0;
@@ -301,7 +320,7 @@ __global__ void __launch_bounds__(AT_THREADS, 1) tree_attention_tc_kernel(const 
                     if (g + 1 < g1) ok = issue_qk(g + 1);
                     else umma_commit(bar(B_Q_EMPTY));        // every S product of the segment has been issued
                     if (!ok) break;
-                    ok = mbar_wait(bar(B_P_READY), (uint32_t)(g & 1), &abort_flag, p.status);
+                    ok = mbar_wait(bar(B_P_READY + (g & 1)), (uint32_t)(g >> 1) & 1u, &abort_flag, p.status);
                     if (ok && g == g0 && e > 0) ok = mbar_wait(bar(B_O_FREE), (uint32_t)((e - 1) & 1), &abort_flag, p.status);
                     const int slot = (2 * g + 1) % AT_RING;
                     if (ok) ok = mbar_wait(bar(B_KV_FULL + slot), (uint32_t)((2 * g + 1) / AT_RING) & 1u, &abort_flag, p.status);
@@ -310,12 +329,12 @@ __global__ void __launch_bounds__(AT_THREADS, 1) tree_attention_tc_kernel(const 
                     const uint32_t v_smem = ring_smem + slot * AT_TILE;
 #pragma unroll
                     for (int kk = 0; kk < 8; ++kk) {        // 8 x 16 keys
-                        const uint32_t p_off = (kk >> 2) * AT_SUB + (kk & 3) * 32;     // P: two 64-key sub-tiles
                         const uint32_t v_off = kk * 16 * 128;                          // V: 16 keys = 16 rows of 128 bytes
-                        umma_bf16(tmem_o, desc_kmajor(p_smem + p_off), desc_mnmajor(v_smem + v_off), idesc_pv,
-                                  (g > g0 || kk > 0) ? 1u : 0u);
+                        // P comes straight from TMEM: 16 keys = 8 columns of bf16 pairs
+                        umma_bf16_ts(tmem_o, tmem_p[g & 1] + 8 * kk, desc_mnmajor(v_smem + v_off), idesc_pv,
+                                     (g > g0 || kk > 0) ? 1u : 0u);
                     }
-                    umma_commit(bar(B_P_FREE));
+                    umma_commit(bar(B_P_FREE + (g & 1)));
                     umma_commit(bar(B_KV_EMPTY + slot));
                 }
                 if (ok) umma_commit(bar(B_O_READY));
@@ -375,17 +394,21 @@ __global__ void __launch_bounds__(AT_THREADS, 1) tree_attention_tc_kernel(const 
                     asm volatile("bar.sync %0, 64;" ::"r"(pair_bar) : "memory");
                     mt = fmaxf(mt, pair_max[g & 1][half ^ 1][row]) * p.scale_log2;
                 }
-                // the P buffer and the O accumulator are free once the previous P.V product has finished
-                if (g > 0) ok = __all_sync(0xffffffffu, mbar_wait(bar(B_P_FREE), (uint32_t)((g - 1) & 1), &abort_flag, p.status));
+                // this tile's P buffer was last read by the P.V product of two tiles ago
+                if (g > 1) ok = __all_sync(0xffffffffu, mbar_wait(bar(B_P_FREE + (g & 1)), ((uint32_t)(g >> 1) & 1u) ^ 1u, &abort_flag, p.status));
                 if (!ok) break;
+                asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                 if (group_live) {
-                    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                     float factor = 1.f;
                     if (live && mt > -INFINITY) {
                         if (m_ref == -INFINITY) m_ref = mt;
                         else if (mt > m_ref + AT_RESCALE_GAP) { factor = fast_exp2(m_ref - mt); m_ref = mt; }
                     }
                     if (g > g0 && __any_sync(0xffffffffu, factor != 1.f)) {
+                        // O may only be touched once the previous P.V product has finished
+                        ok = __all_sync(0xffffffffu, mbar_wait(bar(B_P_FREE + ((g - 1) & 1)), (uint32_t)((g - 1) >> 1) & 1u, &abort_flag, p.status));
+                        if (!ok) break;
+                        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                         l_sum *= factor;
 #pragma unroll 1
                         for (int c0 = 0; c0 < 64; c0 += 32) {
@@ -396,24 +419,21 @@ __global__ void __launch_bounds__(AT_THREADS, 1) tree_attention_tc_kernel(const 
                             tmem_st32(tmem_o + lane_addr + col0 + c0, o);
                         }
                     }
-                    // P = 2^(s * c - m_ref) as bf16 into the K-major swizzled layout of the P operand; masked
-                    // scores are -inf and give exactly 0.  Rows past the tree keep whatever P held: their
-                    // outputs are never stored.
-                    if (live) {
-                        const float m_use = (m_ref == -INFINITY) ? 0.f : m_ref;
-                        uint8_t* prow = base_ptr + AT_TILE + half * AT_SUB + row * 128;
+                    // P = 2^(s * c - m_ref) as bf16 pairs into this tile's P buffer in TMEM (lane = row, one column
+                    // per two keys); masked scores are -inf and give exactly 0.  Rows past the tree store zeros.
+                    const float m_use = (m_ref == -INFINITY) ? 0.f : m_ref;
+                    uint32_t packed[32];
 #pragma unroll
-                        for (int ch = 0; ch < 8; ++ch) {
-                            float pv[8];
-#pragma unroll
-                            for (int i = 0; i < 8; ++i) {
-                                pv[i] = fast_exp2(fmaf(s[8 * ch + i], p.scale_log2, -m_use));
-                                l_sum += pv[i];
-                            }
-                            *reinterpret_cast<uint4*>(prow + ((ch ^ (row & 7)) << 4)) =
-                                make_uint4(pack_bf16(pv[0], pv[1]), pack_bf16(pv[2], pv[3]), pack_bf16(pv[4], pv[5]), pack_bf16(pv[6], pv[7]));
+                    for (int i = 0; i < 64; i += 2) {
+                        float a = 0.f, b = 0.f;
+                        if (live) {
+                            a = fast_exp2(fmaf(s[i], p.scale_log2, -m_use));
+                            b = fast_exp2(fmaf(s[i + 1], p.scale_log2, -m_use));
+                            l_sum += a + b;
                         }
+                        packed[i >> 1] = pack_bf16(a, b);
                     }
+                    tmem_st32u(tmem_p[g & 1] + lane_addr + 32 * half, packed);
                 }
                 // keys past the end of the sequence hold whatever the cache holds: clear those V rows so
                 // that 0 * garbage cannot poison the product
@@ -421,7 +441,7 @@ __global__ void __launch_bounds__(AT_THREADS, 1) tree_attention_tc_kernel(const 
                     const int slot = (2 * g + 1) % AT_RING;
                     ok = __all_sync(0xffffffffu, mbar_wait(bar(B_KV_FULL + slot), (uint32_t)((2 * g + 1) / AT_RING) & 1u, &abort_flag, p.status));
                     if (!ok) break;
-                    uint8_t* v_ptr = base_ptr + 2 * AT_TILE + slot * AT_TILE;
+                    uint8_t* v_ptr = base_ptr + AT_TILE + slot * AT_TILE;
                     const int first_bad = max(total - key0, 0);
                     for (int i = first_bad * 8 + (int)threadIdx.x; i < AT_KEYS * 8; i += 256) {      // 16-byte chunks, both sub-tiles
                         *reinterpret_cast<uint4*>(v_ptr + i * 16) = make_uint4(0, 0, 0, 0);
@@ -430,7 +450,7 @@ __global__ void __launch_bounds__(AT_THREADS, 1) tree_attention_tc_kernel(const 
                 }
                 asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
                 asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-                mbar_arrive(bar(B_P_READY));
+                mbar_arrive(bar(B_P_READY + (g & 1)));
             }
             if (!ok) break;
             // ---- epilogue of the segment
