@@ -120,6 +120,27 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, float* v) {
 #pragma unroll
     for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
 }
+// Two back-to-back 32-column loads with one wait (64 consecutive columns).
+__device__ __forceinline__ void tmem_ld64(uint32_t taddr, float* v) {
+    uint32_t r[64];
+#define TRJ_LD32(base, off)                                                                                          \
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x32.b32 "                                                           \
+                 "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "                            \
+                 "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"            \
+                 : "=r"(r[off + 0]), "=r"(r[off + 1]), "=r"(r[off + 2]), "=r"(r[off + 3]), "=r"(r[off + 4]), "=r"(r[off + 5]),   \
+                   "=r"(r[off + 6]), "=r"(r[off + 7]), "=r"(r[off + 8]), "=r"(r[off + 9]), "=r"(r[off + 10]), "=r"(r[off + 11]), \
+                   "=r"(r[off + 12]), "=r"(r[off + 13]), "=r"(r[off + 14]), "=r"(r[off + 15]), "=r"(r[off + 16]),               \
+                   "=r"(r[off + 17]), "=r"(r[off + 18]), "=r"(r[off + 19]), "=r"(r[off + 20]), "=r"(r[off + 21]),               \
+                   "=r"(r[off + 22]), "=r"(r[off + 23]), "=r"(r[off + 24]), "=r"(r[off + 25]), "=r"(r[off + 26]),               \
+                   "=r"(r[off + 27]), "=r"(r[off + 28]), "=r"(r[off + 29]), "=r"(r[off + 30]), "=r"(r[off + 31])                \
+                 : "r"(base) : "memory")
+    TRJ_LD32(taddr, 0);
+    TRJ_LD32(taddr + 32, 32);
+#undef TRJ_LD32
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+    for (int i = 0; i < 64; ++i) v[i] = __uint_as_float(r[i]);
+}
 __device__ __forceinline__ void tmem_st32(uint32_t taddr, const float* v) {
     asm volatile("tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
                  "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, "
@@ -376,8 +397,7 @@ __global__ void __launch_bounds__(AT_THREADS, 1) tree_attention_tc_kernel(const 
                     ok = __all_sync(0xffffffffu, mbar_wait(bar(B_S_FULL + (g & 1)), (uint32_t)(g >> 1) & 1u, &abort_flag, p.status));
                     if (!ok) break;
                     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-                    tmem_ld32(tmem_s[g & 1] + lane_addr + col0, s);
-                    tmem_ld32(tmem_s[g & 1] + lane_addr + col0 + 32, s + 32);
+                    tmem_ld64(tmem_s[g & 1] + lane_addr + col0, s);
                     if (edge) {
                         // bit c of (vis0, vis1) = visibility of key key0 + c for this row: tree row tt = key0 + c - S
                         // is visible if tt < 0 (prefix) or if bit tt of the row's ancestor mask is set
@@ -388,8 +408,15 @@ __global__ void __launch_bounds__(AT_THREADS, 1) tree_attention_tc_kernel(const 
 #pragma unroll
                         for (int i = 0; i < 64; ++i) if (!((vis >> i) & 1ull)) s[i] = -INFINITY;
                     }
+                    {   // four independent chains instead of one 64-long dependency chain
+                        float mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
 #pragma unroll
-                    for (int i = 0; i < 64; ++i) mt = fmaxf(mt, s[i]);
+                        for (int i = 0; i < 64; i += 4) {
+                            mx[0] = fmaxf(mx[0], s[i]); mx[1] = fmaxf(mx[1], s[i + 1]);
+                            mx[2] = fmaxf(mx[2], s[i + 2]); mx[3] = fmaxf(mx[3], s[i + 3]);
+                        }
+                        mt = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3]));
+                    }
                     pair_max[g & 1][half][row] = mt;
                     asm volatile("bar.sync %0, 64;" ::"r"(pair_bar) : "memory");
                     mt = fmaxf(mt, pair_max[g & 1][half ^ 1][row]) * p.scale_log2;
@@ -423,15 +450,22 @@ __global__ void __launch_bounds__(AT_THREADS, 1) tree_attention_tc_kernel(const 
                     // per two keys); masked scores are -inf and give exactly 0.  Rows past the tree store zeros.
                     const float m_use = (m_ref == -INFINITY) ? 0.f : m_ref;
                     uint32_t packed[32];
+                    if (live) {
+                        float ls[4] = {0.f, 0.f, 0.f, 0.f};  // independent partial sums
 #pragma unroll
-                    for (int i = 0; i < 64; i += 2) {
-                        float a = 0.f, b = 0.f;
-                        if (live) {
-                            a = fast_exp2(fmaf(s[i], p.scale_log2, -m_use));
-                            b = fast_exp2(fmaf(s[i + 1], p.scale_log2, -m_use));
-                            l_sum += a + b;
+                        for (int i = 0; i < 64; i += 4) {
+                            const float a = fast_exp2(fmaf(s[i], p.scale_log2, -m_use));
+                            const float b = fast_exp2(fmaf(s[i + 1], p.scale_log2, -m_use));
+                            const float c = fast_exp2(fmaf(s[i + 2], p.scale_log2, -m_use));
+                            const float d = fast_exp2(fmaf(s[i + 3], p.scale_log2, -m_use));
+                            ls[0] += a; ls[1] += b; ls[2] += c; ls[3] += d;
+                            packed[i >> 1] = pack_bf16(a, b);
+                            packed[(i >> 1) + 1] = pack_bf16(c, d);
                         }
-                        packed[i >> 1] = pack_bf16(a, b);
+                        l_sum += (ls[0] + ls[1]) + (ls[2] + ls[3]);
+                    } else {
+#pragma unroll
+                        for (int i = 0; i < 32; ++i) packed[i] = 0u;
                     }
                     tmem_st32u(tmem_p[g & 1] + lane_addr + 32 * half, packed);
                 }
@@ -447,8 +481,8 @@ __global__ void __launch_bounds__(AT_THREADS, 1) tree_attention_tc_kernel(const 
                         *reinterpret_cast<uint4*>(v_ptr + i * 16) = make_uint4(0, 0, 0, 0);
                         *reinterpret_cast<uint4*>(v_ptr + AT_SUB + i * 16) = make_uint4(0, 0, 0, 0);
                     }
+                    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");      // the MMA reads V through the async proxy
                 }
-                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
                 asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
                 mbar_arrive(bar(B_P_READY + (g & 1)));
             }
