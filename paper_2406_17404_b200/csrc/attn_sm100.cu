@@ -548,7 +548,9 @@ constexpr int CB_COLS = 16;
 __global__ void __launch_bounds__(128) tree_attention_combine_kernel(const AtParams p, int grid_main) {
     __shared__ Sched sched;
     __shared__ float stage[AT_ROWS][CB_COLS + 1];
-    pdl_prologue();
+    // the geometry (sequence lengths, row offsets) is not produced by the main kernel: work it out while that
+    // kernel may still be running, and wait for its pieces only afterwards
+    pdl_launch_dependents();
     if (threadIdx.x == 0) build_sched(sched, p);
     __syncthreads();
     const int bh = blockIdx.x, b = bh / p.H, h = bh % p.H, c0 = blockIdx.y * CB_COLS;
@@ -557,7 +559,6 @@ __global__ void __launch_bounds__(128) tree_attention_combine_kernel(const AtPar
     // CTA c of the main kernel owns units [U*c/G, U*(c+1)/G): the owner of unit u is the largest c with U*c/G <= u
     auto owner = [&](long long u) { return (int)(((u + 1) * grid_main + U - 1) / U - 1); };
     const int c_first = owner(u0), c_last = owner(u1 - 1);
-    if (c_first == c_last) return;                           // written directly by its only CTA
     const int row = threadIdx.x, rows = p.row_off[b + 1] - p.row_off[b];
     const bool live = row < rows;
     // a CTA in between may own no unit at all (grid larger than the unit count): it wrote nothing
@@ -565,6 +566,8 @@ __global__ void __launch_bounds__(128) tree_attention_combine_kernel(const AtPar
         const long long rb = U * c / grid_main, re = U * (c + 1) / grid_main;
         return (rb > u0 ? rb : u0) < (re < u1 ? re : u1);
     };
+    pdl_wait();
+    if (c_first == c_last) return;                           // written directly by its only CTA
     if (live) {
         float m_all = -INFINITY;
         for (int c = c_first; c <= c_last; ++c)
