@@ -627,12 +627,17 @@ bool at_make_map(CUtensorMap* map, const void* base_ptr, size_t rows, size_t col
 }
 
 constexpr int AT_MAX_GRID = 148;
+constexpr int AT_WHOLE_HEAD_TILES = 8;      // up to 1024 keys per head are handled by a single CTA when B == 1
 
 }  // namespace
 
 // The host only knows an upper bound of the key count; CTAs whose range turns out empty leave at once.
 int tree_attention_grid(int32_t B, int32_t H, int32_t max_len) {
-    const long long units_bound = (long long)B * H * ((max_len + AT_KEYS - 1) / AT_KEYS);
+    const int tiles_bound = (max_len + AT_KEYS - 1) / AT_KEYS;
+    const long long units_bound = (long long)B * H * tiles_bound;
+    // One short sequence (a decoding step with a few hundred cached tokens): give every head to one CTA.  Equal
+    // ranges then coincide with the heads, nothing is split, no pieces are written and no merge is needed.
+    if (B == 1 && tiles_bound <= AT_WHOLE_HEAD_TILES && H <= AT_MAX_GRID) return H;
     return (int)(units_bound < AT_MAX_GRID ? units_bound : AT_MAX_GRID);
 }
 
@@ -673,6 +678,7 @@ cudaError_t launch_tree_attention_tc(const void* q, const void* k_slab, const vo
     cudaError_t e = launch_chain(tree_attention_tc_kernel, dim3(grid), dim3(AT_THREADS), AT_SMEM, st, map_q, map_k, map_v, p);
     if (e == cudaSuccess) e = cudaGetLastError();
     if (e != cudaSuccess) return e;
+    if (bt.B == 1 && grid == H) return e;                    // ranges coincide with heads: nothing to merge
     count_launch();
     e = launch_chain(tree_attention_combine_kernel, dim3(bt.B * H, AT_D / CB_COLS), dim3(128), 0, st, p, grid);
     return e != cudaSuccess ? e : cudaGetLastError();
