@@ -36,9 +36,10 @@ DRAFTS = TREE_ROWS - 1                                   # 32 draft tokens per s
 PROMPT = 512
 METRIC = "draft_tokens_verified_per_s"
 UNIT = "tokens/s"
-# DRAM traffic (read + write bytes) of ALL projection launches of one step, from an ncu capture of the
-# current projection kernel; None until measured or after the kernel changed.
-GEMM_TRAFFIC_BYTES_PER_STEP = None
+# DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) of ALL 129 projection launches of one step, from
+# an ncu capture of the current projection kernel (profiles/gemm_tc_traffic_llama7b_33rows.md); set to None
+# whenever that kernel changes.
+GEMM_TRAFFIC_BYTES_PER_STEP = 13371811072 + 186714624
 
 
 def measured_peaks():
