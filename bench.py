@@ -129,52 +129,107 @@ def gemm_bytes_per_step(cfg, rows):
     return total
 
 
+def graph_us(torch, fn, steps, warmup):
+    """Average device time of one call of ``fn`` (a fixed launch sequence), replayed from a CUDA graph."""
+    side = torch.cuda.Stream()
+    with torch.cuda.stream(side):
+        fn()
+    torch.cuda.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph, stream=side):
+        fn()
+    for _ in range(warmup):
+        graph.replay()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(steps):
+        graph.replay()
+    e1.record()
+    torch.cuda.synchronize()
+    return e0.elapsed_time(e1) * 1e3 / steps
+
+
 def bench_tree_attention(trj, torch, peaks, steps, warmup):
-    """Op-level tree attention on the two op-level shapes, over distinct caches larger than L2."""
+    """Op-level tree attention on the op-level shapes (configs 2, 4, 5), over distinct caches larger than L2."""
+    import synth
     out = []
-    for name, prefix, rows, depth, n_caches in (("cfg2: 32x128 heads, prefix 1024, 64-row tree", 1024, 64, 6, 32),
-                                                ("cfg4: 32x128 heads, prefix 8192, 128-row tree", 8192, 128, 8, 4)):
-        import synth
-        h, d = 32, 128
-        total = prefix + rows
+    h, d = 32, 128
+    s5, m5 = synth.ragged_batch(4, 8, (256, 4096), (16, 64))
+    cases = (("cfg2: 32x128 heads, prefix 1024, 64-row tree", [1024], [64], 6, 3, 32),
+             ("cfg4: 32x128 heads, prefix 8192, 128-row tree", [8192], [128], 8, 4, 4),
+             ("cfg5: 8 sequences, prefix 256-4096, 16-64-row trees", s5.tolist(), m5.tolist(), 6, 3, 2))
+    for name, prefixes, rows_list, depth, kids, n_caches in cases:
+        nb, rows_total = len(prefixes), sum(rows_list)
+        max_seq = max(s + m for s, m in zip(prefixes, rows_list))
         g = torch.Generator(device="cuda"); g.manual_seed(7)
-        k = torch.randn(n_caches, 1, h, total, d, generator=g, device="cuda", dtype=torch.float32).to(torch.bfloat16)
-        v = torch.randn(n_caches, 1, h, total, d, generator=g, device="cuda", dtype=torch.float32).to(torch.bfloat16)
-        q = torch.randn(n_caches, rows, h, d, generator=g, device="cuda", dtype=torch.float32).to(torch.bfloat16)
+        rnd = lambda *shape: torch.randn(*shape, generator=g, device="cuda", dtype=torch.float32).to(torch.bfloat16)
+        k, v, q = rnd(n_caches, nb, h, max_seq, d), rnd(n_caches, nb, h, max_seq, d), rnd(n_caches, rows_total, h, d)
         o = torch.empty_like(q)
-        parent = synth.random_tree(1, rows, depth, 3 if rows == 64 else 4)
-        _, anc = trj.tree_from_parents(parent)
+        anc = np.concatenate([trj.tree_from_parents(synth.random_tree(1 + i, m, min(depth, m - 1), kids))[1]
+                              for i, m in enumerate(rows_list)], 0)
         anc_d = torch.from_numpy(anc.view(np.int64)).cuda()
-        seq_len = torch.tensor([prefix], dtype=torch.int32, device="cuda")
-        row_off = torch.tensor([0, rows], dtype=torch.int32, device="cuda")
-        ws = torch.empty(max(256, trj.tree_attention_workspace(rows, 1, h, d, total)), dtype=torch.uint8, device="cuda")
+        seq_len = torch.tensor(prefixes, dtype=torch.int32, device="cuda")
+        row_off = torch.tensor(np.concatenate([[0], np.cumsum(rows_list)]), dtype=torch.int32, device="cuda")
+        ws = torch.zeros(max(256, trj.tree_attention_workspace(rows_total, nb, h, d, max_seq)), dtype=torch.uint8, device="cuda")
 
         def one_pass():
             for c in range(n_caches):
-                trj.tree_attention(q[c], k[c], v[c], seq_len, row_off, anc_d, max_rows=rows, max_len=total, out=o[c], workspace=ws)
-        side = torch.cuda.Stream()
-        with torch.cuda.stream(side):
-            one_pass()
-        torch.cuda.synchronize()
-        graph = torch.cuda.CUDAGraph()
-        with torch.cuda.graph(graph, stream=side):
-            one_pass()
-        for _ in range(warmup):
-            graph.replay()
-        torch.cuda.synchronize()
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        e0.record()
-        for _ in range(steps):
-            graph.replay()
-        e1.record()
-        torch.cuda.synchronize()
-        us = e0.elapsed_time(e1) * 1e3 / (steps * n_caches)
-        nbytes = 2 * h * total * d * 2 + 2 * rows * h * d * 2            # K, V (prefix + tree rows) + q + out
+                trj.tree_attention(q[c], k[c], v[c], seq_len, row_off, anc_d, max_rows=max(rows_list), max_len=max_seq,
+                                   out=o[c], workspace=ws)
+        us = graph_us(torch, one_pass, steps, warmup) / n_caches
+        nbytes = sum(2 * h * (s + m) * d * 2 for s, m in zip(prefixes, rows_list)) + 2 * rows_total * h * d * 2
         gbs = nbytes / us / 1e3
         out.append({"workload": name, "us_per_launch": round(us, 2), "algorithmic_bytes": nbytes, "hbm_gbs": round(gbs, 1),
                     "frac_of_" + peaks["source"] + "_peak": round(gbs / peaks["hbm_gbs"], 4),
                     "distinct_caches": n_caches})
         del k, v, q, o
+    return out
+
+
+def bench_small_ops(trj, torch, peaks, steps, warmup):
+    """Arg-max + acceptance on the 64 x 32000 logits of config 2 and KV compaction of a 7B-shaped cache."""
+    import synth
+    out = []
+    # arg-max + accept: 32 distinct bf16 logit arrays (131 MB in total, larger than L2)
+    rows, vocab, n_arr = 64, 32000, 32
+    g = torch.Generator(device="cuda"); g.manual_seed(11)
+    logits = torch.randn(n_arr, rows, vocab, generator=g, device="cuda", dtype=torch.float32).to(torch.bfloat16)
+    parent = synth.random_tree(1, rows, 6, 3)
+    depth, _ = trj.tree_from_parents(parent)
+    i32 = lambda a: torch.from_numpy(np.ascontiguousarray(a, dtype=np.int32)).cuda()
+    tokens, d_parent, d_depth, off = i32(synth.prompt(3, rows, vocab)), i32(parent), i32(depth), i32([0, rows])
+    outs = {"node_argmax": torch.empty(rows, dtype=torch.int32, device="cuda"), "margin": None,
+            "k_acc": torch.empty(1, dtype=torch.int32, device="cuda"), "bonus": torch.empty(1, dtype=torch.int32, device="cuda"),
+            "path": torch.empty(1, trj.PATH_STRIDE, dtype=torch.int32, device="cuda")}
+    trj.argmax_accept_static(logits[0], tokens, d_parent, d_depth, off, outs)      # one-time set-up outside the capture
+    torch.cuda.synchronize()
+
+    def argmax_pass():
+        for a in range(n_arr):
+            trj.argmax_accept_static(logits[a], tokens, d_parent, d_depth, off, outs)
+    us = graph_us(torch, argmax_pass, steps, warmup) / n_arr
+    nbytes = rows * vocab * 2
+    out.append({"op": "argmax_accept, 64 x 32000 bf16 logits (cfg2)", "us_per_launch": round(us, 2),
+                "algorithmic_bytes": nbytes, "hbm_gbs": round(nbytes / us / 1e3, 1)})
+    del logits
+    # compaction: 32 layers x 32 heads x 128, k = 4 accepted rows of a 33-row tree behind a 512-row prefix
+    n_layers, h, d, max_seq, k_acc = 32, 32, 128, 640, 4
+    kc = torch.zeros(n_layers, 1, h, max_seq, d, dtype=torch.bfloat16, device="cuda")
+    vc = torch.zeros_like(kc)
+    seq0 = torch.tensor([512], dtype=torch.int32, device="cuda")
+    seq = seq0.clone()
+    path = torch.full((1, trj.PATH_STRIDE), -1, dtype=torch.int32, device="cuda")
+    path[0, :5] = torch.tensor([0, 6, 7, 8, 9], dtype=torch.int32)
+    kk = torch.tensor([k_acc], dtype=torch.int32, device="cuda")
+
+    def compact_pass():
+        seq.copy_(seq0)
+        trj.compact_rows(kc, vc, seq, kk, path)
+    us = graph_us(torch, compact_pass, steps, warmup)
+    nbytes = 2 * 2 * k_acc * n_layers * h * d * 2                       # K and V, read + write
+    out.append({"op": "compact_rows, 7B cache, k = 4", "us_per_launch": round(us, 2), "algorithmic_bytes": nbytes,
+                "hbm_gbs": round(nbytes / us / 1e3, 1)})
     return out
 
 
@@ -415,6 +470,7 @@ def run_ours(args, rank, world, local_rank):
     if world == 1:
         if not args.no_attention:
             line["tree_attention"] = bench_tree_attention(trj, torch, peaks, max(args.steps, 5), 3)
+            line["small_ops"] = bench_small_ops(trj, torch, peaks, max(args.steps, 5), 3)
         if not args.no_cpu:
             t_full, detail = oracle_sample(synth.LLAMA7B)
             line["cpu_baseline"] = {"value": DRAFTS / t_full, "unit": UNIT, "cores": cpu_threads(), "kind": "oracle",

@@ -196,7 +196,7 @@ trj_status trj_argmax_accept(const void* logits, int32_t dtype, int32_t V,
  * that a cudaMalloc from inside a call would fail or break that framework's
  * accounting.  For them the scratch (tickets and per-slice arg-max candidates)
  * lives in a fixed array inside the library's device image, TRJ_STATIC_MAX_ROWS
- * rows' worth (about 48 KB), which every GPU that loads the library keeps for the
+ * rows' worth (about 96 KB), which every GPU that loads the library keeps for the
  * lifetime of the process.  Same inputs, outputs and results as
  * trj_argmax_accept.  The call allocates nothing, neither device nor pinned
  * memory.

@@ -349,27 +349,36 @@ __device__ __forceinline__ Top top_shfl_xor(const Top& t, int o) {
 }
 
 constexpr int ARGMAX_THREADS = 256;
-constexpr int ARGMAX_CHUNKS = 4;              // vocabulary slices per row (one CTA each)
+constexpr int ARGMAX_CHUNKS = 8;              // vocabulary slices per row (one CTA each)
 
 // The acceptance walk of one sequence, run by one CTA after every prediction of it is known.
 __device__ void accept_sequence(const int32_t* tokens, const int32_t* parent, const int32_t* depth,
                                 const int32_t* pred, int rows, int32_t* k_acc, int32_t* path, int32_t* bonus) {
     __shared__ unsigned char ok[TRJ_MAX_ROWS];
+    __shared__ int32_t s_tok[TRJ_MAX_ROWS], s_par[TRJ_MAX_ROWS], s_dep[TRJ_MAX_ROWS], s_pred[TRJ_MAX_ROWS];
+    __shared__ int s_best;
+    // all threads fetch the tree, then one thread walks it out of shared memory
+    for (int i = threadIdx.x; i < rows; i += blockDim.x) {
+        s_tok[i] = tokens[i]; s_par[i] = parent[i]; s_dep[i] = depth[i]; s_pred[i] = pred[i];
+    }
+    __syncthreads();
     if (threadIdx.x == 0) {
         ok[0] = 1;
         int best = 0, best_depth = 0;
         for (int i = 1; i < rows; ++i) {
-            const int p = parent[i];
-            const unsigned char o = ok[p] && tokens[i] == pred[p];
+            const int p = s_par[i];
+            const unsigned char o = ok[p] && s_tok[i] == s_pred[p];
             ok[i] = o;
-            if (o && depth[i] > best_depth) { best = i; best_depth = depth[i]; }
+            if (o && s_dep[i] > best_depth) { best = i; best_depth = s_dep[i]; }
         }
         *k_acc = best_depth;
-        *bonus = pred[best];
+        *bonus = s_pred[best];
         int node = best;
-        for (int j = best_depth; j >= 0; --j) { path[j] = node; node = parent[node]; }
-        for (int j = best_depth + 1; j < TRJ_PATH_STRIDE; ++j) path[j] = -1;
+        for (int j = best_depth; j >= 0; --j) { path[j] = node; node = s_par[node]; }
+        s_best = best_depth;
     }
+    __syncthreads();
+    for (int j = s_best + 1 + (int)threadIdx.x; j < TRJ_PATH_STRIDE; j += blockDim.x) path[j] = -1;
 }
 
 template <typename T>
@@ -387,7 +396,17 @@ __global__ void __launch_bounds__(ARGMAX_THREADS) argmax_accept_kernel(
     const int v0 = chunk * per, v1 = min(V, v0 + per);
     const T* lr = logits + (size_t)row * V;
     Top t{-INFINITY, 0x7fffffff, -INFINITY};
-    for (int v = v0 + threadIdx.x; v < v1; v += ARGMAX_THREADS) top_push(t, to_f(lr[v]), v);
+    constexpr int VEC = 16 / (int)sizeof(T);                 // elements per 16-byte load
+    if (V % VEC == 0 && per % VEC == 0 && ((uintptr_t)logits % 16) == 0) {
+        for (int v = v0 + threadIdx.x * VEC; v < v1; v += ARGMAX_THREADS * VEC) {
+            const uint4 raw = *reinterpret_cast<const uint4*>(lr + v);
+            const T* e = reinterpret_cast<const T*>(&raw);
+#pragma unroll
+            for (int i = 0; i < VEC; ++i) top_push(t, to_f(e[i]), v + i);
+        }
+    } else {
+        for (int v = v0 + threadIdx.x; v < v1; v += ARGMAX_THREADS) top_push(t, to_f(lr[v]), v);
+    }
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) t = top_merge(t, top_shfl_xor(t, o));
     if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = t;
