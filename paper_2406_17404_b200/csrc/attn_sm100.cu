@@ -251,6 +251,11 @@ __global__ void __launch_bounds__(AT_THREADS, 1) tree_attention_tc_kernel(const 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
     pdl_launch_dependents();
+    if (threadIdx.x == 32) {                                 // have the tensor maps on their way before the first copy needs them
+        asm volatile("prefetch.tensormap [%0];" ::"l"(&map_q) : "memory");
+        asm volatile("prefetch.tensormap [%0];" ::"l"(&map_k) : "memory");
+        asm volatile("prefetch.tensormap [%0];" ::"l"(&map_v) : "memory");
+    }
     if (threadIdx.x == 0) {
         abort_flag = 0;
         for (int i = 0; i < B_COUNT; ++i) mbar_init(bar(i), (i == B_P_READY || i == B_P_READY + 1 || i == B_O_FREE) ? 256 : 1);

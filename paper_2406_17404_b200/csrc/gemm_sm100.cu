@@ -131,6 +131,11 @@ __global__ void __launch_bounds__(TC_THREADS, 2) gemm_tc_kernel(const __grid_con
     const int items = p.tiles * p.splits;
 
     pdl_launch_dependents();
+    if (threadIdx.x == 32) {                                 // have the tensor maps on their way before the first copy needs them
+        asm volatile("prefetch.tensormap [%0];" ::"l"(&map_w) : "memory");
+        asm volatile("prefetch.tensormap [%0];" ::"l"(&map_x) : "memory");
+        asm volatile("prefetch.tensormap [%0];" ::"l"(&map_xlo) : "memory");
+    }
     if (threadIdx.x == 0) {
         abort_flag = 0;
         for (int s = 0; s < p.stages; ++s) { mbar_init(full0 + 8 * s, 1); mbar_init(empty0 + 8 * s, 1); }
