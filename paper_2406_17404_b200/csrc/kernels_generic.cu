@@ -69,9 +69,9 @@ __global__ void embed_kernel(const T* __restrict__ embed, const int32_t* __restr
 
 // ---------------------------------------------------------------- residual add + RMSNorm
 // One CTA per row.  h += add (summing the split-K pieces of `add` on the way), x = rmsnorm(h) * gain.
-// Fast path: d % 4 == 0 and d <= 4 * 256 * RMS_CHUNKS; the row lives in registers between the two phases.
-constexpr int RMS_THREADS = 256;
-constexpr int RMS_CHUNKS = 8;
+// Fast path: d % 4 == 0 and d <= 4 * RMS_THREADS * RMS_CHUNKS; the row lives in registers between the two phases.
+constexpr int RMS_THREADS = 1024;             // many loads in flight: the row and its split-K pieces come from L2
+constexpr int RMS_CHUNKS = 2;
 
 __device__ __forceinline__ float block_sum(float v, float* red) {
     v = warp_sum(v);
@@ -224,9 +224,12 @@ __global__ void rope_kv_write_kernel(const Parts qkv, const double* __restrict__
     const size_t src = (size_t)row * 3 * HD + hh * D;        // flat index into the projection result
     const size_t cache_row = (((size_t)b * H + hh) * max_seq + seq_len[b] + local) * D;
     for (int i = threadIdx.x; i < half; i += blockDim.x) {
-        double s, c;
-        sincos((double)pos * inv_freq[i], &s, &c);
-        const float cs = (float)c, sn = (float)s;
+        // angle in fp64 (positions reach thousands of radians), reduced to [-pi, pi] there; sin/cos of the reduced
+        // angle in fp32 are then accurate to ~1e-7
+        const double ang = (double)pos * inv_freq[i];
+        const double red = ang - 6.283185307179586476925 * rint(ang * 0.15915494309189533577);
+        float sn, cs;
+        sincosf((float)red, &sn, &cs);
         const float qa = parts_at(qkv, src + i), qb = parts_at(qkv, src + i + half);
         q_out[(size_t)row * HD + hh * D + i] = from_f<T>(qa * cs - qb * sn);
         q_out[(size_t)row * HD + hh * D + i + half] = from_f<T>(qb * cs + qa * sn);
