@@ -243,6 +243,7 @@ void prof_end(trj_ctx* ctx, cudaStream_t st) {
 trj_status forward(trj_ctx* ctx, void* k_cache, void* v_cache, int32_t b0, const Batch& bt,
                    const int32_t* tokens, const int32_t* depth, const uint64_t* anc, int32_t anc_words,
                    int32_t lm_first, int32_t lm_rows, cudaStream_t st) {
+    ChainScope chain;                        // the embedding below is the chain's fence
     const trj_model_cfg& c = ctx->cfg;
     const int M = bt.rows_total, d = c.d_model, HD = c.n_heads * c.head_dim;
     const size_t es = dtype_size(c.dtype);
@@ -408,6 +409,7 @@ extern "C" trj_status trj_verify_step(trj_ctx* ctx, void* k_cache, void* v_cache
     TRJ_REQUIRE(k_cache && v_cache && seq_len && tokens && parent && depth && anc && row_off && node_argmax,
                 TRJ_EINVAL, "verify_step: null pointer");
     cudaStream_t st = (cudaStream_t)stream;
+    ChainScope chain;
     Batch bt{seq_len, row_off, B, rows_total, max_rows, max_len};
     s = forward(ctx, k_cache, v_cache, 0, bt, tokens, depth, anc, anc_words, 0, rows_total, st);
     if (s != TRJ_OK) return s;
@@ -427,6 +429,7 @@ extern "C" trj_status trj_accept(trj_ctx* ctx, const int32_t* tokens, const int3
     TRJ_REQUIRE(tokens && parent && depth && row_off && node_argmax && k_acc && path && bonus, TRJ_EINVAL, "accept: null pointer");
     TRJ_REQUIRE(B >= 1 && B <= ctx->cfg.max_batch && rows_total >= B, TRJ_ECAPACITY, "accept: bad batch");
     cudaStream_t st = (cudaStream_t)stream;
+    ChainScope chain;                        // these kernels wait for their predecessor before reading anything
     LAUNCH(PROF_ARGMAX, launch_argmax_accept(nullptr, TRJ_F32, 0, tokens, parent, depth, row_off, B, rows_total,
                                              const_cast<int32_t*>(node_argmax), nullptr, k_acc, path, bonus, false, true,
                                              ctx->argmax_ws, st));
@@ -440,6 +443,7 @@ extern "C" trj_status trj_compact_kv(trj_ctx* ctx, void* k_cache, void* v_cache,
     const trj_model_cfg& c = ctx->cfg;
     TRJ_REQUIRE(B >= 1 && B <= c.max_batch, TRJ_ECAPACITY, "compact_kv: batch %d outside 1..%d", B, c.max_batch);
     cudaStream_t st = (cudaStream_t)stream;
+    ChainScope chain;
     LAUNCH(PROF_COMPACT, launch_compact(k_cache, v_cache, c.n_layers, c.max_batch, B, c.n_heads, c.max_seq, c.head_dim,
                                         c.dtype, seq_len, k_acc, path, st));
     return TRJ_OK;
@@ -476,6 +480,7 @@ namespace {
 trj_status enqueue_step(trj_ctx* ctx, void* k_cache, void* v_cache, int32_t* seq_len, int32_t M, int32_t max_len,
                         cudaStream_t st) {
     const trj_model_cfg& c = ctx->cfg;
+    ChainScope chain;
     TRJ_CHECK_CUDA(cudaMemcpyAsync(ctx->step_in, ctx->pin_in, STEP_IN_BYTES, cudaMemcpyHostToDevice, st));
     int32_t* d_tokens = ctx->step_in, *d_parent = d_tokens + TRJ_MAX_ROWS, *d_depth = d_tokens + 2 * TRJ_MAX_ROWS;
     int32_t* d_off = d_tokens + 3 * TRJ_MAX_ROWS;

@@ -266,12 +266,15 @@ __global__ void __launch_bounds__(AT_THREADS, 1) tree_attention_tc_kernel(const 
                      ::"r"(smem_u32(&tmem_base_slot)), "r"(512u) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
-    // barriers and TMEM are set up while the previous kernel may still run; its results are needed from here on
-    pdl_wait();
+    // Barriers, TMEM and the schedule are set up while the previous kernel may still run: the batch geometry is
+    // older than the chain this kernel is launched in.  So are the cache rows below seq_len, which the copy thread
+    // starts to fetch before it waits; everything else (q, the tree's own K/V rows) is touched after the wait.
     if (threadIdx.x == 0) build_sched(sched, p);
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     __syncthreads();
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    const bool copy_thread = warp == 8 && lane == 0;
+    if (!copy_thread) pdl_wait();
     const uint32_t tmem = tmem_base_slot;
     // TMEM columns: S buffers 0-127 and 128-255, O 256-383, P buffers (bf16 pairs, 64 columns each) 384-447 and 448-511
     const uint32_t tmem_s[2] = {tmem, tmem + 128}, tmem_o = tmem + 256, tmem_p[2] = {tmem + 384, tmem + 448};
@@ -285,18 +288,30 @@ __global__ void __launch_bounds__(AT_THREADS, 1) tree_attention_tc_kernel(const 
             // ------------------------------------------------ TMA producer
             int g = 0, e = 0;
             bool ok = true;
+            bool waited = false;                             // for the previous kernel (see above)
             for (long long u = u_begin; u < u_end && ok;) {
                 Where w; sched.locate(u, p.seq_len, p.row_off, w);
                 const int t_end = (int)min((long long)w.tiles, w.t + (u_end - u));
                 // Q of this segment (after the previous segment's S = Q.K^T products have finished)
-                ok = mbar_wait(bar(B_Q_EMPTY), (uint32_t)(e & 1) ^ 1u, &abort_flag, p.status);
-                if (!ok) break;
-                mbar_expect_tx(bar(B_Q_FULL), AT_TILE);
-                tma_load_2d(q_smem, &map_q, w.h * AT_D, p.row_off[w.b], bar(B_Q_FULL));
-                tma_load_2d(q_smem + AT_SUB, &map_q, w.h * AT_D + 64, p.row_off[w.b], bar(B_Q_FULL));
+                auto load_q = [&]() -> bool {
+                    if (!mbar_wait(bar(B_Q_EMPTY), (uint32_t)(e & 1) ^ 1u, &abort_flag, p.status)) return false;
+                    mbar_expect_tx(bar(B_Q_FULL), AT_TILE);
+                    tma_load_2d(q_smem, &map_q, w.h * AT_D, p.row_off[w.b], bar(B_Q_FULL));
+                    tma_load_2d(q_smem + AT_SUB, &map_q, w.h * AT_D + 64, p.row_off[w.b], bar(B_Q_FULL));
+                    return true;
+                };
+                bool q_loaded = false;
+                if (waited) { ok = load_q(); q_loaded = true; if (!ok) break; }
                 const int cache_row0 = (w.b * p.H + w.h) * p.max_seq;
+                const int old_tiles = p.seq_len[w.b] / AT_KEYS;          // tiles that hold cached rows only
                 for (int t = w.t; t < t_end && ok; ++t, ++g) {
                     for (int kv = 0; kv < 2 && ok; ++kv) {
+                        if (!q_loaded && (t >= old_tiles || 2 * g + kv >= AT_RING)) {
+                            // the first tile with rows of this step, or a ring slot that must be drained first
+                            if (!waited) { pdl_wait(); waited = true; }
+                            ok = load_q(); q_loaded = true;
+                            if (!ok) break;
+                        }
                         const int slot = (2 * g + kv) % AT_RING;
                         const uint32_t phase = (uint32_t)((2 * g + kv) / AT_RING) & 1u;
                         ok = mbar_wait(bar(B_KV_EMPTY + slot), phase ^ 1u, &abort_flag, p.status);
@@ -308,9 +323,14 @@ __global__ void __launch_bounds__(AT_THREADS, 1) tree_attention_tc_kernel(const 
                         tma_load_2d(dst + AT_SUB, map, 64, cache_row0 + t * AT_KEYS, bar(B_KV_FULL + slot));
                     }
                 }
+                if (ok && !q_loaded) {                       // a segment of cached tiles that fit the ring
+                    if (!waited) { pdl_wait(); waited = true; }
+                    ok = load_q();
+                }
                 u += t_end - w.t;
                 ++e;
             }
+            if (!waited) pdl_wait();
         }
     } else if (warp == 9) {
         if (lane == 0) {

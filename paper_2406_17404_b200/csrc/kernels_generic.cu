@@ -61,7 +61,8 @@ __device__ __forceinline__ int seq_of_row(const int32_t* row_off, int B, int row
 template <typename T>
 __global__ void embed_kernel(const T* __restrict__ embed, const int32_t* __restrict__ tokens,
                              float* __restrict__ h, int d) {
-    pdl_prologue();
+    pdl_wait();                                  // the chain's fence: everything enqueued earlier is complete
+    pdl_launch_dependents();                     // before any later kernel of the chain may start
     const int row = blockIdx.x;
     const T* src = embed + (size_t)tokens[row] * d;
     for (int c = threadIdx.x; c < d; c += blockDim.x) h[(size_t)row * d + c] = to_f(src[c]);
@@ -215,7 +216,9 @@ __global__ void rope_kv_write_kernel(const Parts qkv, const double* __restrict__
                                      const int32_t* __restrict__ depth, const int32_t* __restrict__ seq_len,
                                      const int32_t* __restrict__ row_off, int B, T* __restrict__ q_out,
                                      T* __restrict__ k_slab, T* __restrict__ v_slab, int H, int D, int max_seq) {
-    pdl_prologue();
+    pdl_launch_dependents();
+    // geometry and the rotation of this thread's first element do not depend on the projection: have them
+    // ready before waiting for it
     const int row = blockIdx.x, hh = blockIdx.y;
     const int b = seq_of_row(row_off, B, row);
     const int local = row - row_off[b];
@@ -223,21 +226,32 @@ __global__ void rope_kv_write_kernel(const Parts qkv, const double* __restrict__
     const int half = D >> 1, HD = H * D;
     const size_t src = (size_t)row * 3 * HD + hh * D;        // flat index into the projection result
     const size_t cache_row = (((size_t)b * H + hh) * max_seq + seq_len[b] + local) * D;
-    for (int i = threadIdx.x; i < half; i += blockDim.x) {
+    auto rotation = [&](int i, float& sn, float& cs) {
         // angle in fp64 (positions reach thousands of radians), reduced to [-pi, pi] there; sin/cos of the reduced
         // angle in fp32 are then accurate to ~1e-7
         const double ang = (double)pos * inv_freq[i];
         const double red = ang - 6.283185307179586476925 * rint(ang * 0.15915494309189533577);
-        float sn, cs;
         sincosf((float)red, &sn, &cs);
-        const float qa = parts_at(qkv, src + i), qb = parts_at(qkv, src + i + half);
+    };
+    float sn = 0.f, cs = 1.f;
+    if ((int)threadIdx.x < half) rotation(threadIdx.x, sn, cs);
+    pdl_wait();
+    for (int i = threadIdx.x; i < half; i += blockDim.x) {
+        if (i != (int)threadIdx.x) rotation(i, sn, cs);
+        // all loads first: the stores below could alias them as far as the compiler knows
+        float qa = 0.f, qb = 0.f, ka = 0.f, kb = 0.f, va = 0.f, vb = 0.f;
+        for (int s = 0; s < qkv.splits; ++s) {               // six independent loads per split-K piece
+            const float* piece = qkv.ptr + (size_t)s * qkv.stride + src + i;
+            qa += piece[0];      qb += piece[half];
+            ka += piece[HD];     kb += piece[HD + half];
+            va += piece[2 * HD]; vb += piece[2 * HD + half];
+        }
         q_out[(size_t)row * HD + hh * D + i] = from_f<T>(qa * cs - qb * sn);
         q_out[(size_t)row * HD + hh * D + i + half] = from_f<T>(qb * cs + qa * sn);
-        const float ka = parts_at(qkv, src + HD + i), kb = parts_at(qkv, src + HD + i + half);
         k_slab[cache_row + i] = from_f<T>(ka * cs - kb * sn);
         k_slab[cache_row + i + half] = from_f<T>(kb * cs + ka * sn);
-        v_slab[cache_row + i] = from_f<T>(parts_at(qkv, src + 2 * HD + i));
-        v_slab[cache_row + i + half] = from_f<T>(parts_at(qkv, src + 2 * HD + i + half));
+        v_slab[cache_row + i] = from_f<T>(va);
+        v_slab[cache_row + i + half] = from_f<T>(vb);
     }
 }
 
@@ -504,6 +518,10 @@ __global__ void bump_len_kernel(int32_t* seq_len_b, int delta) { *seq_len_b += d
 static std::atomic<bool> g_pdl{true};
 bool pdl_enabled() { return g_pdl.load(std::memory_order_relaxed); }
 void set_pdl(bool on) { g_pdl.store(on, std::memory_order_relaxed); }
+static thread_local int t_chain_depth = 0;
+bool chain_active() { return t_chain_depth > 0 && pdl_enabled(); }
+ChainScope::ChainScope() { ++t_chain_depth; }
+ChainScope::~ChainScope() { --t_chain_depth; }
 static std::atomic<uint64_t> g_launches{0};
 void count_launch() { g_launches.fetch_add(1, std::memory_order_relaxed); }
 uint64_t launches_so_far() { return g_launches.load(std::memory_order_relaxed); }

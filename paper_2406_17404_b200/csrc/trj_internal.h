@@ -29,12 +29,20 @@ trj_status tree_from_parents_impl(const int32_t* parent, int32_t M, int32_t anc_
                                   int32_t* depth, uint64_t* anc);
 
 // ---- programmatic dependent launch -----------------------------------------------------------------
-// Kernels of the step are launched so that a kernel may be scheduled while its predecessor in the stream
-// is still running: every such kernel first lets ITS successor start (launch_dependents) and then waits
-// for its predecessor to finish and flush (wait) before it touches any data the predecessor may write.
-// Launched without the attribute, both instructions do nothing.
+// Inside a chain (a ChainScope on the calling thread: the model forward and the steps that follow it),
+// kernels are launched so that a kernel may be scheduled while its predecessor in the stream is still
+// running: every such kernel first lets ITS successor start (launch_dependents) and then waits for its
+// predecessor to finish and flush (wait) before it touches any data the predecessor may write.
+// The first kernel of a forward (the embedding) is the chain's fence: it waits BEFORE it lets its
+// successor start.  A chain kernel that has started therefore knows that everything enqueued before that
+// embedding is complete, so ahead of its own wait it may read what only earlier work wrote: the batch
+// geometry (seq_len, row_off, depth), weights, and cache rows below seq_len.  Anything written inside the
+// chain is read after the wait.  Outside a chain (the op-level entry points, whose predecessor is
+// unknown) kernels are launched without the attribute, and both instructions do nothing.
 bool pdl_enabled();
 void set_pdl(bool on);
+bool chain_active();                      // this thread is inside a ChainScope and PDL is enabled
+struct ChainScope { ChainScope(); ~ChainScope(); ChainScope(const ChainScope&) = delete; };
 #ifdef __CUDACC__
 __device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
@@ -48,7 +56,7 @@ cudaError_t launch_chain(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
-    cfg.numAttrs = pdl_enabled() ? 1 : 0;
+    cfg.numAttrs = chain_active() ? 1 : 0;
     return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
 }
 #endif
