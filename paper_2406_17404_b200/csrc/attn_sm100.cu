@@ -31,6 +31,7 @@ constexpr int AT_RING = 5;                   // K/V ring slots; load n = 2g + (0
 constexpr uint32_t AT_SMEM = (1 + AT_RING) * AT_TILE + 1024;
 constexpr uint32_t AT_WAIT_LIMIT = 1u << 21;
 constexpr float AT_RESCALE_GAP = 8.f;        // raise the running max only when exceeded by 2^8
+constexpr int AT_PIECE_STRIDE = AT_D + 4;      // floats per row of a piece in shared memory (16-byte stores without bank conflicts)
 constexpr size_t AT_SLOT_FLOATS = (size_t)AT_D * AT_ROWS + 2 * AT_ROWS;   // O^T [d][row], m[row], l[row]
 
 // barrier indices
@@ -45,6 +46,7 @@ struct AtParams {
     float* slots;                // partial results, AT_SLOT_FLOATS each
     int* status;
     float scale_log2;            // log2(e) / sqrt(D)
+    int cluster;                 // CTAs per thread-block cluster that share one head (1: no clusters)
 };
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -190,6 +192,34 @@ __device__ __forceinline__ void store8_split(__nv_bfloat16* hi, __nv_bfloat16* l
     }
 }
 
+// Same for 4 outputs (8 bytes each).
+__device__ __forceinline__ void store4_split(__nv_bfloat16* hi, __nv_bfloat16* lo, float a, float b, float c, float d) {
+    *reinterpret_cast<uint2*>(hi) = make_uint2(pack_bf16(a, b), pack_bf16(c, d));
+    if (lo)
+        *reinterpret_cast<uint2*>(lo) = make_uint2(pack_bf16(a - bf16_round(a), b - bf16_round(b)),
+                                                   pack_bf16(c - bf16_round(c), d - bf16_round(d)));
+}
+// Distributed shared memory: the address of `local` (a shared::cta address) in CTA `rank` of the cluster, and loads from it.
+__device__ __forceinline__ uint32_t cluster_addr(uint32_t local, int rank) {
+    uint32_t r;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(local), "r"(rank));
+    return r;
+}
+__device__ __forceinline__ float ld_cluster(uint32_t addr) {
+    float v;
+    asm volatile("ld.shared::cluster.f32 %0, [%1];" : "=f"(v) : "r"(addr) : "memory");
+    return v;
+}
+__device__ __forceinline__ float4 ld_cluster4(uint32_t addr) {
+    float4 v;
+    asm volatile("ld.shared::cluster.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(addr) : "memory");
+    return v;
+}
+__device__ __forceinline__ void cluster_sync_all() {
+    asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+    asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+
 // 128-bit (lo, hi) shifts by 0..127 bits; the left shift fills the vacated low bits with ones.
 __device__ __forceinline__ void shr128(uint64_t& lo, uint64_t& hi, int n) {
     if (n == 0) return;
@@ -242,6 +272,7 @@ __global__ void __launch_bounds__(AT_THREADS, 1) tree_attention_tc_kernel(const 
     __shared__ int abort_flag;
     __shared__ Sched sched;
     __shared__ float pair_max[2][2][AT_ROWS], pair_sum[2][2][AT_ROWS];      // [parity][half][row]
+    __shared__ float piece_m[AT_ROWS], piece_l[AT_ROWS];                     // this CTA's piece of a head shared by a cluster
 
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t* base_ptr = smem_raw + (base - smem_u32(smem_raw));
@@ -270,6 +301,7 @@ __global__ void __launch_bounds__(AT_THREADS, 1) tree_attention_tc_kernel(const 
     // older than the chain this kernel is launched in.  So are the cache rows below seq_len, which the copy thread
     // starts to fetch before it waits; everything else (q, the tree's own K/V rows) is touched after the wait.
     if (threadIdx.x == 0) build_sched(sched, p);
+    if (threadIdx.x < AT_ROWS) piece_m[threadIdx.x] = -INFINITY;             // no piece yet
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     __syncthreads();
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
@@ -281,7 +313,15 @@ __global__ void __launch_bounds__(AT_THREADS, 1) tree_attention_tc_kernel(const 
 
     // this CTA's contiguous range of units
     const long long U = sched.first[p.B];
-    const long long u_begin = U * blockIdx.x / gridDim.x, u_end = U * (blockIdx.x + 1) / gridDim.x;
+    long long u_begin = U * blockIdx.x / gridDim.x, u_end = U * (blockIdx.x + 1) / gridDim.x;
+    float* piece_o = reinterpret_cast<float*>(base_ptr + AT_TILE);          // [row][AT_PIECE_STRIDE], over the K/V ring once it is idle
+    if (p.cluster > 1) {
+        // one sequence, one head per cluster: the head's tiles are shared out among the CTAs of the cluster, every
+        // CTA leaves its piece in its own shared memory, and after a cluster barrier each CTA merges a slice of head_dim
+        const int head = blockIdx.x / p.cluster, rank = blockIdx.x % p.cluster, T = sched.tiles[0];
+        u_begin = (long long)head * T + T * rank / p.cluster;
+        u_end = (long long)head * T + T * (rank + 1) / p.cluster;
+    }
 
     if (warp == 8) {
         if (lane == 0) {
@@ -521,7 +561,20 @@ __global__ void __launch_bounds__(AT_THREADS, 1) tree_attention_tc_kernel(const 
                 asm volatile("bar.sync %0, 64;" ::"r"(pair_bar) : "memory");
                 const float l_row = l_sum + pair_sum[e & 1][half ^ 1][row];
                 const bool whole_seg = (w.t == 0 && n_tiles == w.tiles);
-                if (whole_seg) {
+                if (p.cluster > 1) {
+                    // all products that read the ring have finished (B_O_READY), and this CTA loads nothing more
+#pragma unroll 1
+                    for (int c0 = 0; c0 < 64; c0 += 32) {
+                        float o[32];
+                        tmem_ld32(tmem_o + lane_addr + col0 + c0, o);
+                        if (live) {
+                            float4* dst = reinterpret_cast<float4*>(piece_o + (size_t)row * AT_PIECE_STRIDE + col0 + c0);
+#pragma unroll
+                            for (int i = 0; i < 8; ++i) dst[i] = make_float4(o[4 * i], o[4 * i + 1], o[4 * i + 2], o[4 * i + 3]);
+                        }
+                    }
+                    if (live && half == 0) { piece_m[row] = m_ref; piece_l[row] = l_row; }
+                } else if (whole_seg) {
                     const float inv = live ? 1.f / l_row : 0.f;
                     const size_t off = ((size_t)grow * p.H + w.h) * AT_D + col0;
 #pragma unroll 1
@@ -562,6 +615,37 @@ __global__ void __launch_bounds__(AT_THREADS, 1) tree_attention_tc_kernel(const 
     if (abort_flag) {                                        // let copies still in flight land before the CTA leaves
         for (int i = 0; i < 64; ++i) __nanosleep(1000);
         __syncthreads();
+    }
+    if (p.cluster > 1) {
+        // Every CTA of the cluster gets here, with or without a piece, and also after a wait that gave up.
+        cluster_sync_all();                                  // all pieces are in place and visible
+        const int C = p.cluster, rank = blockIdx.x % C, head = blockIdx.x / C;
+        const int rows = p.row_off[1] - p.row_off[0], width = AT_D / C, groups = width / 4;
+        const uint32_t m_local = smem_u32(piece_m), l_local = smem_u32(piece_l), o_local = smem_u32(piece_o);
+        if (threadIdx.x < 256 && !abort_flag) {
+            for (int i = threadIdx.x; i < rows * groups; i += 256) {
+                const int row = i / groups, col = rank * width + 4 * (i % groups);
+                float m_c[8], m_all = -INFINITY;
+#pragma unroll
+                for (int c = 0; c < 8; ++c)
+                    if (c < C) { m_c[c] = ld_cluster(cluster_addr(m_local + 4u * row, c)); m_all = fmaxf(m_all, m_c[c]); }
+                float l_all = 0.f;
+                float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+                for (int c = 0; c < 8; ++c) {                // pieces in ascending tile order
+                    if (c >= C || m_c[c] == -INFINITY) continue;
+                    const float wgt = exp2f(m_c[c] - m_all);
+                    l_all = fmaf(ld_cluster(cluster_addr(l_local + 4u * row, c)), wgt, l_all);
+                    const float4 o = ld_cluster4(cluster_addr(o_local + 4u * (uint32_t)(row * AT_PIECE_STRIDE + col), c));
+                    acc.x = fmaf(o.x, wgt, acc.x); acc.y = fmaf(o.y, wgt, acc.y);
+                    acc.z = fmaf(o.z, wgt, acc.z); acc.w = fmaf(o.w, wgt, acc.w);
+                }
+                const float inv = 1.f / l_all;
+                const size_t off = ((size_t)(p.row_off[0] + row) * p.H + head) * AT_D + col;
+                store4_split(p.out + off, p.out_lo ? p.out_lo + off : nullptr, acc.x * inv, acc.y * inv, acc.z * inv, acc.w * inv);
+            }
+        }
+        cluster_sync_all();                                  // nobody leaves while its piece may still be read
     }
     if (warp == 9)
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(512u) : "memory");
@@ -652,19 +736,53 @@ bool at_make_map(CUtensorMap* map, const void* base_ptr, size_t rows, size_t col
 }
 
 constexpr int AT_MAX_GRID = 148;
-constexpr int AT_WHOLE_HEAD_TILES = 8;      // up to 1024 keys per head are handled by a single CTA when B == 1
+constexpr int AT_WHOLE_HEAD_TILES = 8;      // up to 1024 keys: heads are handled one by one when B == 1
+
+// How many CTAs may share a head (as one thread-block cluster) when every head is handled on its own: the largest
+// of 4 and 2 for which all H clusters are resident at once, else 1.  Asked of the driver once per head count.
+int at_cluster_size(int H) {
+    static std::mutex mu;
+    static int cached_h = -1, cached_c = 1;
+    std::lock_guard<std::mutex> lock(mu);
+    if (cached_h == H) return cached_c;
+    int pick = 1;
+    if (cudaFuncSetAttribute(tree_attention_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)AT_SMEM) == cudaSuccess) {
+        for (int c = 4; c >= 2 && pick == 1; c /= 2) {
+            if (H * c > AT_MAX_GRID) continue;
+            cudaLaunchConfig_t cfg = {};
+            cfg.gridDim = dim3(H * c); cfg.blockDim = dim3(AT_THREADS); cfg.dynamicSmemBytes = AT_SMEM;
+            cudaLaunchAttribute attr[1];
+            attr[0].id = cudaLaunchAttributeClusterDimension;
+            attr[0].val.clusterDim.x = c; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+            cfg.attrs = attr; cfg.numAttrs = 1;
+            int n = 0;
+            if (cudaOccupancyMaxActiveClusters(&n, tree_attention_tc_kernel, &cfg) == cudaSuccess && n >= H) pick = c;
+        }
+    }
+    (void)cudaGetLastError();                                // a refused query is not an error of the caller
+    cached_h = H; cached_c = pick;
+    return pick;
+}
+
+// Launch shape.  The host only knows an upper bound of the key count; CTAs whose range turns out empty do no work.
+struct AtPlan { int grid, cluster; bool merge_kernel; };
+AtPlan at_plan(int32_t B, int32_t H, int32_t max_len) {
+    const int tiles_bound = (max_len + AT_KEYS - 1) / AT_KEYS;
+    const long long units_bound = (long long)B * H * tiles_bound;
+    // One short sequence (a decoding step with a few hundred cached tokens): every head on its own.  A head's
+    // tiles are shared by the CTAs of a cluster, which merge their pieces through distributed shared memory;
+    // where clusters do not fit (or there is a single tile) one CTA takes the whole head.  No pieces go through
+    // global memory and no merge kernel is needed.
+    if (B == 1 && tiles_bound <= AT_WHOLE_HEAD_TILES && H <= AT_MAX_GRID) {
+        const int c = tiles_bound >= 2 ? at_cluster_size(H) : 1;
+        return AtPlan{H * c, c, false};
+    }
+    return AtPlan{(int)(units_bound < AT_MAX_GRID ? units_bound : AT_MAX_GRID), 1, true};
+}
 
 }  // namespace
 
-// The host only knows an upper bound of the key count; CTAs whose range turns out empty leave at once.
-int tree_attention_grid(int32_t B, int32_t H, int32_t max_len) {
-    const int tiles_bound = (max_len + AT_KEYS - 1) / AT_KEYS;
-    const long long units_bound = (long long)B * H * tiles_bound;
-    // One short sequence (a decoding step with a few hundred cached tokens): give every head to one CTA.  Equal
-    // ranges then coincide with the heads, nothing is split, no pieces are written and no merge is needed.
-    if (B == 1 && tiles_bound <= AT_WHOLE_HEAD_TILES && H <= AT_MAX_GRID) return H;
-    return (int)(units_bound < AT_MAX_GRID ? units_bound : AT_MAX_GRID);
-}
+int tree_attention_grid(int32_t B, int32_t H, int32_t max_len) { return at_plan(B, H, max_len).grid; }
 
 bool tree_attention_tc_supported(int32_t D, int32_t dtype, int32_t max_rows) {
     return D == AT_D && dtype == TRJ_BF16 && max_rows <= AT_ROWS && at_encode_fn() != nullptr;
@@ -698,14 +816,29 @@ cudaError_t launch_tree_attention_tc(const void* q, const void* k_slab, const vo
     p.status = (int*)workspace;
     p.slots = (float*)((char*)workspace + 256);
     p.scale_log2 = 1.4426950408889634f / sqrtf((float)AT_D);
-    const int grid = tree_attention_grid(bt.B, H, bt.max_len);
+    const AtPlan plan = at_plan(bt.B, H, bt.max_len);
+    p.cluster = plan.cluster;
     count_launch();
-    cudaError_t e = launch_chain(tree_attention_tc_kernel, dim3(grid), dim3(AT_THREADS), AT_SMEM, st, map_q, map_k, map_v, p);
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(plan.grid); cfg.blockDim = dim3(AT_THREADS); cfg.dynamicSmemBytes = AT_SMEM; cfg.stream = st;
+    cudaLaunchAttribute attr[2];
+    int n_attr = 0;
+    if (chain_active()) {
+        attr[n_attr].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[n_attr].val.programmaticStreamSerializationAllowed = 1;
+        ++n_attr;
+    }
+    if (plan.cluster > 1) {
+        attr[n_attr].id = cudaLaunchAttributeClusterDimension;
+        attr[n_attr].val.clusterDim.x = plan.cluster; attr[n_attr].val.clusterDim.y = 1; attr[n_attr].val.clusterDim.z = 1;
+        ++n_attr;
+    }
+    cfg.attrs = attr; cfg.numAttrs = n_attr;
+    cudaError_t e = cudaLaunchKernelEx(&cfg, tree_attention_tc_kernel, map_q, map_k, map_v, p);
     if (e == cudaSuccess) e = cudaGetLastError();
-    if (e != cudaSuccess) return e;
-    if (bt.B == 1 && grid == H) return e;                    // ranges coincide with heads: nothing to merge
+    if (e != cudaSuccess || !plan.merge_kernel) return e;
     count_launch();
-    e = launch_chain(tree_attention_combine_kernel, dim3(bt.B * H, AT_D / CB_COLS), dim3(128), 0, st, p, grid);
+    e = launch_chain(tree_attention_combine_kernel, dim3(bt.B * H, AT_D / CB_COLS), dim3(128), 0, st, p, plan.grid);
     return e != cudaSuccess ? e : cudaGetLastError();
 }
 

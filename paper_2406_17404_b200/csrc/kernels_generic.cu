@@ -50,6 +50,23 @@ __device__ __forceinline__ float4 parts_at4(const Parts& p, size_t i4) {
     return v;
 }
 
+// Same for four consecutive values.  The pieces are requested eight at a time before any is added, so the
+// loads overlap; the additions keep the order of the pieces.
+__device__ __forceinline__ float4 parts_at4_batched(const Parts& p, size_t i4) {
+    constexpr int BATCH = 8;
+    float4 v = reinterpret_cast<const float4*>(p.ptr)[i4];
+    for (int s0 = 1; s0 < p.splits; s0 += BATCH) {
+        float4 b[BATCH];
+#pragma unroll
+        for (int j = 0; j < BATCH; ++j)
+            if (s0 + j < p.splits) b[j] = reinterpret_cast<const float4*>(p.ptr + (size_t)(s0 + j) * p.stride)[i4];
+#pragma unroll
+        for (int j = 0; j < BATCH; ++j)
+            if (s0 + j < p.splits) { v.x += b[j].x; v.y += b[j].y; v.z += b[j].z; v.w += b[j].w; }
+    }
+    return v;
+}
+
 // Sequence that owns a global row (B is small: linear scan of the offsets).
 __device__ __forceinline__ int seq_of_row(const int32_t* row_off, int B, int row) {
     int b = 0;
@@ -255,6 +272,61 @@ __global__ void rope_kv_write_kernel(const Parts qkv, const double* __restrict__
     }
 }
 
+// Four consecutive dimensions per thread (head_dim / 2 a multiple of 4): 16-byte loads of the projection pieces,
+// 8-byte (bf16) or 16-byte (fp32) stores.  One CTA covers ROPE_HEADS heads of a row.
+constexpr int ROPE_HEADS = 8;
+template <typename T>
+__global__ void rope_kv_write_vec_kernel(const Parts qkv, const double* __restrict__ inv_freq,
+                                         const int32_t* __restrict__ depth, const int32_t* __restrict__ seq_len,
+                                         const int32_t* __restrict__ row_off, int B, T* __restrict__ q_out,
+                                         T* __restrict__ k_slab, T* __restrict__ v_slab, int H, int D, int max_seq) {
+    pdl_launch_dependents();
+    // geometry and rotations do not depend on the projection: have them ready before waiting for it
+    const int half = D >> 1, HD = H * D, per_head = half >> 2;
+    const int row = blockIdx.x, hh = blockIdx.y * ROPE_HEADS + (int)threadIdx.x / per_head;
+    const int i = ((int)threadIdx.x % per_head) * 4;
+    if (hh >= H) return;
+    const int b = seq_of_row(row_off, B, row);
+    const int local = row - row_off[b];
+    const int pos = seq_len[b] + depth[row];
+    const size_t src = (size_t)row * 3 * HD + hh * D + i;    // flat index into the projection result
+    const size_t cache_at = (((size_t)b * H + hh) * max_seq + seq_len[b] + local) * D + i;
+    const size_t q_at = (size_t)row * HD + hh * D + i;
+    float sn[4], cs[4];
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+        // angle in fp64 (positions reach thousands of radians), reduced to [-pi, pi] there; sin/cos of the reduced
+        // angle in fp32 are then accurate to ~1e-7
+        const double ang = (double)pos * inv_freq[i + e];
+        const double red = ang - 6.283185307179586476925 * rint(ang * 0.15915494309189533577);
+        sincosf((float)red, &sn[e], &cs[e]);
+    }
+    pdl_wait();
+    float4 acc[6];                                           // q, k, v: first and second half of the head
+#pragma unroll
+    for (int e = 0; e < 6; ++e) acc[e] = make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int s = 0; s < qkv.splits; ++s) {                   // six independent loads per split-K piece
+        const float* piece = qkv.ptr + (size_t)s * qkv.stride + src;
+        float4 t[6];
+#pragma unroll
+        for (int e = 0; e < 6; ++e) t[e] = *reinterpret_cast<const float4*>(piece + (e >> 1) * HD + (e & 1) * half);
+#pragma unroll
+        for (int e = 0; e < 6; ++e) { acc[e].x += t[e].x; acc[e].y += t[e].y; acc[e].z += t[e].z; acc[e].w += t[e].w; }
+    }
+    auto rot_lo = [&](const float4& a, const float4& bb) {
+        return make_float4(a.x * cs[0] - bb.x * sn[0], a.y * cs[1] - bb.y * sn[1], a.z * cs[2] - bb.z * sn[2], a.w * cs[3] - bb.w * sn[3]);
+    };
+    auto rot_hi = [&](const float4& a, const float4& bb) {
+        return make_float4(bb.x * cs[0] + a.x * sn[0], bb.y * cs[1] + a.y * sn[1], bb.z * cs[2] + a.z * sn[2], bb.w * cs[3] + a.w * sn[3]);
+    };
+    store_split4<T>(q_out, nullptr, q_at, rot_lo(acc[0], acc[1]));
+    store_split4<T>(q_out, nullptr, q_at + half, rot_hi(acc[0], acc[1]));
+    store_split4<T>(k_slab, nullptr, cache_at, rot_lo(acc[2], acc[3]));
+    store_split4<T>(k_slab, nullptr, cache_at + half, rot_hi(acc[2], acc[3]));
+    store_split4<T>(v_slab, nullptr, cache_at, acc[4]);
+    store_split4<T>(v_slab, nullptr, cache_at + half, acc[5]);
+}
+
 // ---------------------------------------------------------------- tree attention, one CTA per (row, head)
 // 4 warps split the keys; inside a warp every lane scores one key of a 32-key chunk, the chunk's
 // statistics are merged with an online softmax, and P.V is accumulated with lanes spread over D.
@@ -339,6 +411,21 @@ __global__ void swiglu_kernel(const Parts gu, T* __restrict__ act, T* __restrict
         const size_t r = i / f, c = i % f;
         const float g = parts_at(gu, r * 2 * f + c), u = parts_at(gu, r * 2 * f + f + c);
         store_split(act, act_lo, i, g / (1.f + expf(-g)) * u);
+    }
+}
+
+// Four columns per thread (f a multiple of 4).
+template <typename T>
+__global__ void swiglu_vec_kernel(const Parts gu, T* __restrict__ act, T* __restrict__ act_lo, int rows, int f) {
+    pdl_prologue();
+    const int f4 = f >> 2;
+    const size_t n4 = (size_t)rows * f4;
+    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n4; i += (size_t)gridDim.x * blockDim.x) {
+        const size_t r = i / f4, c4 = i % f4;
+        const float4 g = parts_at4_batched(gu, r * 2 * f4 + c4), u = parts_at4_batched(gu, r * 2 * f4 + f4 + c4);
+        store_split4<T>(act, act_lo, 4 * i,
+                        make_float4(g.x / (1.f + expf(-g.x)) * u.x, g.y / (1.f + expf(-g.y)) * u.y,
+                                    g.z / (1.f + expf(-g.z)) * u.z, g.w / (1.f + expf(-g.w)) * u.w));
     }
 }
 
@@ -565,9 +652,17 @@ cudaError_t launch_rope_kv_write(const Parts& qkv, const double* inv_freq, const
                                  int32_t H, int32_t D, int32_t max_seq, cudaStream_t st) {
     count_launch();
     cudaError_t launch_err = cudaSuccess;
-    dim3 grid(bt.rows_total, H);
-    DISPATCH_T(dtype, launch_err = launch_chain(rope_kv_write_kernel<T>, grid, dim3(64), 0, st, qkv, inv_freq, depth, bt.seq_len, bt.row_off,
-                                                                  bt.B, (T*)q_out, (T*)k_slab, (T*)v_slab, H, D, max_seq));
+    const int per_head = D / 8;                              // threads per head in the vector kernel
+    const bool vec = D % 8 == 0 && per_head * ROPE_HEADS <= 1024 && qkv.stride % 4 == 0 && ((uintptr_t)qkv.ptr % 16) == 0;
+    if (vec) {
+        dim3 grid(bt.rows_total, (H + ROPE_HEADS - 1) / ROPE_HEADS);
+        DISPATCH_T(dtype, launch_err = launch_chain(rope_kv_write_vec_kernel<T>, grid, dim3(per_head * ROPE_HEADS), 0, st, qkv, inv_freq, depth,
+                                                    bt.seq_len, bt.row_off, bt.B, (T*)q_out, (T*)k_slab, (T*)v_slab, H, D, max_seq));
+    } else {
+        dim3 grid(bt.rows_total, H);
+        DISPATCH_T(dtype, launch_err = launch_chain(rope_kv_write_kernel<T>, grid, dim3(64), 0, st, qkv, inv_freq, depth, bt.seq_len, bt.row_off,
+                                                    bt.B, (T*)q_out, (T*)k_slab, (T*)v_slab, H, D, max_seq));
+    }
     return launch_err != cudaSuccess ? launch_err : cudaGetLastError();
 }
 
@@ -592,9 +687,14 @@ cudaError_t launch_swiglu(const Parts& gu, void* act, void* act_lo, int32_t dtyp
                           cudaStream_t st) {
     count_launch();
     cudaError_t launch_err = cudaSuccess;
-    const size_t n = (size_t)rows * f;
-    const int blocks = (int)((n + 255) / 256 < 1184 ? (n + 255) / 256 : 1184);
-    DISPATCH_T(dtype, launch_err = launch_chain(swiglu_kernel<T>, dim3(blocks), dim3(256), 0, st, gu, (T*)act, (T*)act_lo, rows, f));
+    const bool vec = f % 4 == 0 && gu.stride % 4 == 0 && ((uintptr_t)gu.ptr % 16) == 0;
+    const size_t n = (size_t)rows * (vec ? f / 4 : f);
+    const int blocks = (int)((n + 127) / 128 < 2368 ? (n + 127) / 128 : 2368);
+    if (vec) {
+        DISPATCH_T(dtype, launch_err = launch_chain(swiglu_vec_kernel<T>, dim3(blocks), dim3(128), 0, st, gu, (T*)act, (T*)act_lo, rows, f));
+    } else {
+        DISPATCH_T(dtype, launch_err = launch_chain(swiglu_kernel<T>, dim3(blocks), dim3(128), 0, st, gu, (T*)act, (T*)act_lo, rows, f));
+    }
     return launch_err != cudaSuccess ? launch_err : cudaGetLastError();
 }
 
