@@ -39,7 +39,7 @@ UNIT = "tokens/s"
 # DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) of ALL 129 projection launches of one step, from
 # an ncu capture of the current projection kernel (profiles/gemm_tc_traffic_llama7b_33rows.md); set to None
 # whenever that kernel changes.
-GEMM_TRAFFIC_BYTES_PER_STEP = 13371811072 + 186714624
+GEMM_TRAFFIC_BYTES_PER_STEP = 13373281536 + 181045248
 
 
 def measured_peaks():
@@ -156,7 +156,8 @@ def bench_tree_attention(trj, torch, peaks, steps, warmup):
     out = []
     h, d = 32, 128
     s5, m5 = synth.ragged_batch(4, 8, (256, 4096), (16, 64))
-    cases = (("cfg2: 32x128 heads, prefix 1024, 64-row tree", [1024], [64], 6, 3, 32),
+    cases = (("cfg3 (the step's shape): 32x128 heads, prefix 512, 33-row tree", [512], [33], 6, 3, 16),
+             ("cfg2: 32x128 heads, prefix 1024, 64-row tree", [1024], [64], 6, 3, 32),
              ("cfg4: 32x128 heads, prefix 8192, 128-row tree", [8192], [128], 8, 4, 4),
              ("cfg5: 8 sequences, prefix 256-4096, 16-64-row trees", s5.tolist(), m5.tolist(), 6, 3, 2))
     for name, prefixes, rows_list, depth, kids, n_caches in cases:
