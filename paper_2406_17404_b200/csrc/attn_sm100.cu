@@ -238,14 +238,16 @@ struct Where { int b, h, t, tiles, S, rows, bh; };
 struct Sched {
     int B, H;
     int tiles[TRJ_MAX_BATCH];           // key tiles of each sequence
+    int S[TRJ_MAX_BATCH];               // cached rows of each sequence (a copy of seq_len: no global load on the critical path)
+    int row0[TRJ_MAX_BATCH + 1];        // a copy of row_off
     long long first[TRJ_MAX_BATCH + 1]; // first unit of each sequence
-    __device__ void locate(long long u, const int32_t* seq_len, const int32_t* row_off, Where& w) const {
+    __device__ void locate(long long u, Where& w) const {
         int b = 0;
         while (b + 1 < B && u >= first[b + 1]) ++b;
         const long long r = u - first[b];
         w.b = b; w.tiles = tiles[b];
         w.h = (int)(r / w.tiles); w.t = (int)(r % w.tiles);
-        w.S = seq_len[b]; w.rows = row_off[b + 1] - row_off[b];
+        w.S = S[b]; w.rows = row0[b + 1] - row0[b];
         w.bh = b * H + w.h;
     }
 };
@@ -253,8 +255,11 @@ struct Sched {
 __device__ __forceinline__ void build_sched(Sched& s, const AtParams& p) {
     s.B = p.B; s.H = p.H;
     long long u = 0;
+    s.row0[0] = p.row_off[0];
     for (int b = 0; b < p.B; ++b) {
-        const int total = p.seq_len[b] + (p.row_off[b + 1] - p.row_off[b]);
+        s.S[b] = p.seq_len[b];
+        s.row0[b + 1] = p.row_off[b + 1];
+        const int total = s.S[b] + (s.row0[b + 1] - s.row0[b]);
         s.tiles[b] = (total + AT_KEYS - 1) / AT_KEYS;
         s.first[b] = u;
         u += (long long)s.tiles[b] * p.H;
@@ -330,28 +335,26 @@ __global__ void __launch_bounds__(AT_THREADS, 1) tree_attention_tc_kernel(const 
             bool ok = true;
             bool waited = false;                             // for the previous kernel (see above)
             for (long long u = u_begin; u < u_end && ok;) {
-                Where w; sched.locate(u, p.seq_len, p.row_off, w);
+                Where w; sched.locate(u, w);
                 const int t_end = (int)min((long long)w.tiles, w.t + (u_end - u));
                 // Q of this segment (after the previous segment's S = Q.K^T products have finished)
                 auto load_q = [&]() -> bool {
                     if (!mbar_wait(bar(B_Q_EMPTY), (uint32_t)(e & 1) ^ 1u, &abort_flag, p.status)) return false;
                     mbar_expect_tx(bar(B_Q_FULL), AT_TILE);
-                    tma_load_2d(q_smem, &map_q, w.h * AT_D, p.row_off[w.b], bar(B_Q_FULL));
-                    tma_load_2d(q_smem + AT_SUB, &map_q, w.h * AT_D + 64, p.row_off[w.b], bar(B_Q_FULL));
+                    tma_load_2d(q_smem, &map_q, w.h * AT_D, sched.row0[w.b], bar(B_Q_FULL));
+                    tma_load_2d(q_smem + AT_SUB, &map_q, w.h * AT_D + 64, sched.row0[w.b], bar(B_Q_FULL));
                     return true;
                 };
-                bool q_loaded = false;
-                if (waited) { ok = load_q(); q_loaded = true; if (!ok) break; }
+                // the first segment's Q is requested by the MMA thread as soon as the previous kernel is done, so
+                // that it does not queue behind the cache tiles this thread asks for ahead of the wait
+                if (e > 0) { ok = load_q(); if (!ok) break; }
                 const int cache_row0 = (w.b * p.H + w.h) * p.max_seq;
-                const int old_tiles = p.seq_len[w.b] / AT_KEYS;          // tiles that hold cached rows only
+                const int old_tiles = w.S / AT_KEYS;          // tiles that hold cached rows only
                 for (int t = w.t; t < t_end && ok; ++t, ++g) {
                     for (int kv = 0; kv < 2 && ok; ++kv) {
-                        if (!q_loaded && (t >= old_tiles || 2 * g + kv >= AT_RING)) {
-                            // the first tile with rows of this step, or a ring slot that must be drained first
-                            if (!waited) { pdl_wait(); waited = true; }
-                            ok = load_q(); q_loaded = true;
-                            if (!ok) break;
-                        }
+                        // rows of this step, or a ring slot that is only freed once Q has arrived: bounded waits
+                        // must not start while the previous kernel may still run
+                        if (!waited && (t >= old_tiles || 2 * g + kv >= AT_RING)) { pdl_wait(); waited = true; }
                         const int slot = (2 * g + kv) % AT_RING;
                         const uint32_t phase = (uint32_t)((2 * g + kv) / AT_RING) & 1u;
                         ok = mbar_wait(bar(B_KV_EMPTY + slot), phase ^ 1u, &abort_flag, p.status);
@@ -363,10 +366,7 @@ __global__ void __launch_bounds__(AT_THREADS, 1) tree_attention_tc_kernel(const 
                         tma_load_2d(dst + AT_SUB, map, 64, cache_row0 + t * AT_KEYS, bar(B_KV_FULL + slot));
                     }
                 }
-                if (ok && !q_loaded) {                       // a segment of cached tiles that fit the ring
-                    if (!waited) { pdl_wait(); waited = true; }
-                    ok = load_q();
-                }
+                if (!waited) { pdl_wait(); waited = true; }  // the next segment's Q comes from the previous kernel
                 u += t_end - w.t;
                 ++e;
             }
@@ -385,8 +385,8 @@ __global__ void __launch_bounds__(AT_THREADS, 1) tree_attention_tc_kernel(const 
                 if (!mbar_wait(bar(B_KV_FULL + slot), (uint32_t)((2 * gg) / AT_RING) & 1u, &abort_flag, p.status)) return false;
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                 const uint32_t k_smem = ring_smem + slot * AT_TILE;
-#pragma unroll
-                for (int kk = 0; kk < 8; ++kk) {            // 8 x 16 elements of head_dim: two sub-tiles of four steps
+#pragma unroll 1
+                for (int kk = 0; kk < 8; ++kk) {            // 8 x 16 elements of head_dim (rolled: one thread, cold code): two sub-tiles of four steps
                     const uint32_t off = (kk >> 2) * AT_SUB + (kk & 3) * 32;
                     umma_bf16(tmem_s[gg & 1], desc_kmajor(q_smem + off), desc_kmajor(k_smem + off), idesc_qk, kk > 0);
                 }
@@ -395,9 +395,14 @@ __global__ void __launch_bounds__(AT_THREADS, 1) tree_attention_tc_kernel(const 
                 return true;
             };
             for (long long u = u_begin; u < u_end && ok;) {
-                Where w; sched.locate(u, p.seq_len, p.row_off, w);
+                Where w; sched.locate(u, w);
                 const int n_tiles = (int)min((long long)(w.tiles - w.t), u_end - u);
                 const int g0 = g, g1 = g + n_tiles;
+                if (e == 0) {                                // first segment: this thread has waited for the previous kernel
+                    mbar_expect_tx(bar(B_Q_FULL), AT_TILE);
+                    tma_load_2d(q_smem, &map_q, w.h * AT_D, sched.row0[w.b], bar(B_Q_FULL));
+                    tma_load_2d(q_smem + AT_SUB, &map_q, w.h * AT_D + 64, sched.row0[w.b], bar(B_Q_FULL));
+                }
                 ok = mbar_wait(bar(B_Q_FULL), (uint32_t)(e & 1), &abort_flag, p.status);
                 if (!ok) break;
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
@@ -413,7 +418,7 @@ __global__ void __launch_bounds__(AT_THREADS, 1) tree_attention_tc_kernel(const 
                     if (!ok) break;
                     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                     const uint32_t v_smem = ring_smem + slot * AT_TILE;
-#pragma unroll
+#pragma unroll 1
                     for (int kk = 0; kk < 8; ++kk) {        // 8 x 16 keys
                         const uint32_t v_off = kk * 16 * 128;                          // V: 16 keys = 16 rows of 128 bytes
                         // P comes straight from TMEM: 16 keys = 8 columns of bf16 pairs
@@ -440,12 +445,12 @@ __global__ void __launch_bounds__(AT_THREADS, 1) tree_attention_tc_kernel(const 
         int g = 0, e = 0;
         bool ok = true;
         for (long long u = u_begin; u < u_end && ok;) {
-            Where w; sched.locate(u, p.seq_len, p.row_off, w);
+            Where w; sched.locate(u, w);
             const int n_tiles = (int)min((long long)(w.tiles - w.t), u_end - u);
             const int g0 = g, g1 = g + n_tiles;
             const bool live = row < w.rows;
             const bool group_live = rg * 32 < w.rows;        // same for both warps of the pair
-            const int grow = p.row_off[w.b] + row;           // global row (valid when live)
+            const int grow = sched.row0[w.b] + row;           // global row (valid when live)
             uint64_t m0 = 0, m1 = 0;
             if (live) {
                 m0 = p.anc[(size_t)grow * p.anc_words];
@@ -620,28 +625,36 @@ __global__ void __launch_bounds__(AT_THREADS, 1) tree_attention_tc_kernel(const 
         // Every CTA of the cluster gets here, with or without a piece, and also after a wait that gave up.
         cluster_sync_all();                                  // all pieces are in place and visible
         const int C = p.cluster, rank = blockIdx.x % C, head = blockIdx.x / C;
-        const int rows = p.row_off[1] - p.row_off[0], width = AT_D / C, groups = width / 4;
+        const int rows = sched.row0[1] - sched.row0[0], width = AT_D / C, groups = width / 4;
         const uint32_t m_local = smem_u32(piece_m), l_local = smem_u32(piece_l), o_local = smem_u32(piece_o);
         if (threadIdx.x < 256 && !abort_flag) {
             for (int i = threadIdx.x; i < rows * groups; i += 256) {
                 const int row = i / groups, col = rank * width + 4 * (i % groups);
-                float m_c[8], m_all = -INFINITY;
+                // every piece's statistics and values are requested before any is used
+                float m_c[8], l_c[8], m_all = -INFINITY;
+                float4 o_c[8];
 #pragma unroll
-                for (int c = 0; c < 8; ++c)
-                    if (c < C) { m_c[c] = ld_cluster(cluster_addr(m_local + 4u * row, c)); m_all = fmaxf(m_all, m_c[c]); }
+                for (int c = 0; c < 8; ++c) {
+                    if (c < C) {
+                        m_c[c] = ld_cluster(cluster_addr(m_local + 4u * row, c));
+                        l_c[c] = ld_cluster(cluster_addr(l_local + 4u * row, c));
+                        o_c[c] = ld_cluster4(cluster_addr(o_local + 4u * (uint32_t)(row * AT_PIECE_STRIDE + col), c));
+                    }
+                }
+#pragma unroll
+                for (int c = 0; c < 8; ++c) if (c < C) m_all = fmaxf(m_all, m_c[c]);
                 float l_all = 0.f;
                 float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
-                for (int c = 0; c < 8; ++c) {                // pieces in ascending tile order
+                for (int c = 0; c < 8; ++c) {                // pieces in ascending tile order; one without keys holds no data
                     if (c >= C || m_c[c] == -INFINITY) continue;
                     const float wgt = exp2f(m_c[c] - m_all);
-                    l_all = fmaf(ld_cluster(cluster_addr(l_local + 4u * row, c)), wgt, l_all);
-                    const float4 o = ld_cluster4(cluster_addr(o_local + 4u * (uint32_t)(row * AT_PIECE_STRIDE + col), c));
-                    acc.x = fmaf(o.x, wgt, acc.x); acc.y = fmaf(o.y, wgt, acc.y);
-                    acc.z = fmaf(o.z, wgt, acc.z); acc.w = fmaf(o.w, wgt, acc.w);
+                    l_all = fmaf(l_c[c], wgt, l_all);
+                    acc.x = fmaf(o_c[c].x, wgt, acc.x); acc.y = fmaf(o_c[c].y, wgt, acc.y);
+                    acc.z = fmaf(o_c[c].z, wgt, acc.z); acc.w = fmaf(o_c[c].w, wgt, acc.w);
                 }
                 const float inv = 1.f / l_all;
-                const size_t off = ((size_t)(p.row_off[0] + row) * p.H + head) * AT_D + col;
+                const size_t off = ((size_t)(sched.row0[0] + row) * p.H + head) * AT_D + col;
                 store4_split(p.out + off, p.out_lo ? p.out_lo + off : nullptr, acc.x * inv, acc.y * inv, acc.z * inv, acc.w * inv);
             }
         }
