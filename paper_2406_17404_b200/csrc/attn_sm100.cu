@@ -240,13 +240,14 @@ struct Sched {
     int tiles[TRJ_MAX_BATCH];           // key tiles of each sequence
     int S[TRJ_MAX_BATCH];               // cached rows of each sequence (a copy of seq_len: no global load on the critical path)
     int row0[TRJ_MAX_BATCH + 1];        // a copy of row_off
-    long long first[TRJ_MAX_BATCH + 1]; // first unit of each sequence
-    __device__ void locate(long long u, Where& w) const {
+    int first[TRJ_MAX_BATCH + 1];       // first unit of each sequence (the launcher checks that the count fits an int)
+    int u_begin, u_end;                 // this CTA's units
+    __device__ void locate(int u, Where& w) const {
         int b = 0;
         while (b + 1 < B && u >= first[b + 1]) ++b;
-        const long long r = u - first[b];
+        const int r = u - first[b];
         w.b = b; w.tiles = tiles[b];
-        w.h = (int)(r / w.tiles); w.t = (int)(r % w.tiles);
+        w.h = r / w.tiles; w.t = r % w.tiles;
         w.S = S[b]; w.rows = row0[b + 1] - row0[b];
         w.bh = b * H + w.h;
     }
@@ -254,7 +255,7 @@ struct Sched {
 
 __device__ __forceinline__ void build_sched(Sched& s, const AtParams& p) {
     s.B = p.B; s.H = p.H;
-    long long u = 0;
+    int u = 0;
     s.row0[0] = p.row_off[0];
     for (int b = 0; b < p.B; ++b) {
         s.S[b] = p.seq_len[b];
@@ -262,9 +263,22 @@ __device__ __forceinline__ void build_sched(Sched& s, const AtParams& p) {
         const int total = s.S[b] + (s.row0[b + 1] - s.row0[b]);
         s.tiles[b] = (total + AT_KEYS - 1) / AT_KEYS;
         s.first[b] = u;
-        u += (long long)s.tiles[b] * p.H;
+        u += s.tiles[b] * p.H;
     }
     s.first[p.B] = u;
+}
+// The calling CTA's units.  Without clusters: equal contiguous ranges of all units.  With clusters (one sequence,
+// one head per cluster): the head's tiles are shared out among the CTAs of the cluster.
+__device__ __forceinline__ void build_range(Sched& s, const AtParams& p) {
+    if (p.cluster > 1) {
+        const int head = blockIdx.x / p.cluster, rank = blockIdx.x % p.cluster, T = s.tiles[0];
+        s.u_begin = head * T + T * rank / p.cluster;
+        s.u_end = head * T + T * (rank + 1) / p.cluster;
+    } else {
+        const long long U = s.first[p.B];
+        s.u_begin = (int)(U * blockIdx.x / gridDim.x);
+        s.u_end = (int)(U * (blockIdx.x + 1) / gridDim.x);
+    }
 }
 
 __global__ void __launch_bounds__(AT_THREADS, 1) tree_attention_tc_kernel(const __grid_constant__ CUtensorMap map_q,
@@ -305,28 +319,20 @@ __global__ void __launch_bounds__(AT_THREADS, 1) tree_attention_tc_kernel(const 
     // Barriers, TMEM and the schedule are set up while the previous kernel may still run: the batch geometry is
     // older than the chain this kernel is launched in.  So are the cache rows below seq_len, which the copy thread
     // starts to fetch before it waits; everything else (q, the tree's own K/V rows) is touched after the wait.
-    if (threadIdx.x == 0) build_sched(sched, p);
+    if (threadIdx.x == 0) { build_sched(sched, p); build_range(sched, p); }
     if (threadIdx.x < AT_ROWS) piece_m[threadIdx.x] = -INFINITY;             // no piece yet
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     __syncthreads();
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-    const bool copy_thread = warp == 8 && lane == 0;
-    if (!copy_thread) pdl_wait();
+    // Every role works out its first segment before it waits for the previous kernel (one thread's integer
+    // divisions and address arithmetic take a microsecond that would otherwise sit on the critical path).
     const uint32_t tmem = tmem_base_slot;
     // TMEM columns: S buffers 0-127 and 128-255, O 256-383, P buffers (bf16 pairs, 64 columns each) 384-447 and 448-511
     const uint32_t tmem_s[2] = {tmem, tmem + 128}, tmem_o = tmem + 256, tmem_p[2] = {tmem + 384, tmem + 448};
-
-    // this CTA's contiguous range of units
-    const long long U = sched.first[p.B];
-    long long u_begin = U * blockIdx.x / gridDim.x, u_end = U * (blockIdx.x + 1) / gridDim.x;
+    const int u_begin = sched.u_begin, u_end = sched.u_end;
+    // With clusters every CTA leaves its piece in its own shared memory, and after a cluster barrier each CTA
+    // merges a slice of head_dim from all pieces.
     float* piece_o = reinterpret_cast<float*>(base_ptr + AT_TILE);          // [row][AT_PIECE_STRIDE], over the K/V ring once it is idle
-    if (p.cluster > 1) {
-        // one sequence, one head per cluster: the head's tiles are shared out among the CTAs of the cluster, every
-        // CTA leaves its piece in its own shared memory, and after a cluster barrier each CTA merges a slice of head_dim
-        const int head = blockIdx.x / p.cluster, rank = blockIdx.x % p.cluster, T = sched.tiles[0];
-        u_begin = (long long)head * T + T * rank / p.cluster;
-        u_end = (long long)head * T + T * (rank + 1) / p.cluster;
-    }
 
     if (warp == 8) {
         if (lane == 0) {
@@ -334,9 +340,9 @@ __global__ void __launch_bounds__(AT_THREADS, 1) tree_attention_tc_kernel(const 
             int g = 0, e = 0;
             bool ok = true;
             bool waited = false;                             // for the previous kernel (see above)
-            for (long long u = u_begin; u < u_end && ok;) {
+            for (int u = u_begin; u < u_end && ok;) {
                 Where w; sched.locate(u, w);
-                const int t_end = (int)min((long long)w.tiles, w.t + (u_end - u));
+                const int t_end = min(w.tiles, w.t + (u_end - u));
                 // Q of this segment (after the previous segment's S = Q.K^T products have finished)
                 auto load_q = [&]() -> bool {
                     if (!mbar_wait(bar(B_Q_EMPTY), (uint32_t)(e & 1) ^ 1u, &abort_flag, p.status)) return false;
@@ -394,11 +400,12 @@ __global__ void __launch_bounds__(AT_THREADS, 1) tree_attention_tc_kernel(const 
                 umma_commit(bar(B_KV_EMPTY + slot));
                 return true;
             };
-            for (long long u = u_begin; u < u_end && ok;) {
+            for (int u = u_begin; u < u_end && ok;) {
                 Where w; sched.locate(u, w);
-                const int n_tiles = (int)min((long long)(w.tiles - w.t), u_end - u);
+                const int n_tiles = min(w.tiles - w.t, u_end - u);
                 const int g0 = g, g1 = g + n_tiles;
-                if (e == 0) {                                // first segment: this thread has waited for the previous kernel
+                if (e == 0) {                                // first segment: Q as soon as the previous kernel is done
+                    pdl_wait();
                     mbar_expect_tx(bar(B_Q_FULL), AT_TILE);
                     tma_load_2d(q_smem, &map_q, w.h * AT_D, sched.row0[w.b], bar(B_Q_FULL));
                     tma_load_2d(q_smem + AT_SUB, &map_q, w.h * AT_D + 64, sched.row0[w.b], bar(B_Q_FULL));
@@ -444,9 +451,9 @@ __global__ void __launch_bounds__(AT_THREADS, 1) tree_attention_tc_kernel(const 
         const uint32_t pair_bar = 1 + rg;                    // named barrier of the two warps of a row group
         int g = 0, e = 0;
         bool ok = true;
-        for (long long u = u_begin; u < u_end && ok;) {
+        for (int u = u_begin; u < u_end && ok;) {
             Where w; sched.locate(u, w);
-            const int n_tiles = (int)min((long long)(w.tiles - w.t), u_end - u);
+            const int n_tiles = min(w.tiles - w.t, u_end - u);
             const int g0 = g, g1 = g + n_tiles;
             const bool live = row < w.rows;
             const bool group_live = rg * 32 < w.rows;        // same for both warps of the pair
@@ -458,6 +465,7 @@ __global__ void __launch_bounds__(AT_THREADS, 1) tree_attention_tc_kernel(const 
             }
             const int total = w.S + w.rows;
             float m_ref = -INFINITY, l_sum = 0.f;
+            if (e == 0) pdl_wait();                          // the ancestor masks above are older than the chain
             for (g = g0; g < g1 && ok; ++g) {
                 const int key0 = (w.t + (g - g0)) * AT_KEYS;
                 const bool edge = key0 + AT_KEYS > w.S;      // the tile reaches tree rows or the end of the keys
@@ -623,12 +631,13 @@ __global__ void __launch_bounds__(AT_THREADS, 1) tree_attention_tc_kernel(const 
     }
     if (p.cluster > 1) {
         // Every CTA of the cluster gets here, with or without a piece, and also after a wait that gave up.
+        pdl_wait();                                          // threads that had no role have not waited yet
         cluster_sync_all();                                  // all pieces are in place and visible
         const int C = p.cluster, rank = blockIdx.x % C, head = blockIdx.x / C;
         const int rows = sched.row0[1] - sched.row0[0], width = AT_D / C, groups = width / 4;
         const uint32_t m_local = smem_u32(piece_m), l_local = smem_u32(piece_l), o_local = smem_u32(piece_o);
-        if (threadIdx.x < 256 && !abort_flag) {
-            for (int i = threadIdx.x; i < rows * groups; i += 256) {
+        if (!abort_flag) {
+            for (int i = threadIdx.x; i < rows * groups; i += AT_THREADS) {
                 const int row = i / groups, col = rank * width + 4 * (i % groups);
                 // every piece's statistics and values are requested before any is used
                 float m_c[8], l_c[8], m_all = -INFINITY;
@@ -829,6 +838,7 @@ cudaError_t launch_tree_attention_tc(const void* q, const void* k_slab, const vo
     p.status = (int*)workspace;
     p.slots = (float*)((char*)workspace + 256);
     p.scale_log2 = 1.4426950408889634f / sqrtf((float)AT_D);
+    if ((long long)bt.B * H * ((bt.max_len + AT_KEYS - 1) / AT_KEYS) > 0x7fffffffLL) return cudaErrorInvalidValue;   // unit indices are ints
     const AtPlan plan = at_plan(bt.B, H, bt.max_len);
     p.cluster = plan.cluster;
     count_launch();
