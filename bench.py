@@ -234,6 +234,20 @@ def bench_small_ops(trj, torch, peaks, steps, warmup):
     return out
 
 
+def run_ops_only(args):
+    """The op-level legs alone (no model): one JSON line, not the bench contract's."""
+    import torch
+    import paper_2406_17404_b200 as trj
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the verification step has no CPU path")
+    torch.cuda.set_device(0)
+    trj.lib()
+    peaks = measured_peaks()
+    steps = max(args.steps, 5)
+    print(json.dumps({"ops_only": True, "tree_attention": bench_tree_attention(trj, torch, peaks, steps, 3),
+                      "small_ops": bench_small_ops(trj, torch, peaks, steps, 3)}), flush=True)
+
+
 def oracle_sample(cfg_full, seed=0):
     """The CPU oracle on a bounded sample of the workload: one verification step of a 2-layer slice of the
     7B shape (33 rows over a 512-row cache) plus the LM head; the layer part is scaled by n_layers / 2."""
@@ -492,10 +506,16 @@ def main():
     ap.add_argument("--no-pdl", action="store_true", help="launch the kernels fully serialised (comparison only)")
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-oracle baseline leg")
     ap.add_argument("--no-attention", action="store_true", help="skip the op-level tree-attention leg")
+    ap.add_argument("--ops-only", action="store_true",
+                    help="only the op-level legs (tree attention, arg-max + accept, compaction): a small run for profiling")
     args = ap.parse_args()
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if args.ops_only:
+        if rank == 0:
+            run_ops_only(args)
+        return
     if args.impl == "reference":
         args.steps = min(args.steps, 3)
         args.warmup = min(args.warmup, 1)

@@ -861,7 +861,9 @@ cudaError_t launch_tree_attention_tc(const void* q, const void* k_slab, const vo
     if (e == cudaSuccess) e = cudaGetLastError();
     if (e != cudaSuccess || !plan.merge_kernel) return e;
     count_launch();
-    e = launch_chain(tree_attention_combine_kernel, dim3(bt.B * H, AT_D / CB_COLS), dim3(128), 0, st, p, plan.grid);
+    // The merge kernel's predecessor is always the kernel above, and ahead of its wait it reads only the batch
+    // geometry, which was complete before that kernel could start: programmatic launch is safe outside a chain too.
+    e = launch_dependent(pdl_enabled(), tree_attention_combine_kernel, dim3(bt.B * H, AT_D / CB_COLS), dim3(128), 0, st, p, plan.grid);
     return e != cudaSuccess ? e : cudaGetLastError();
 }
 
