@@ -791,13 +791,12 @@ struct AtPlan { int grid, cluster; bool merge_kernel; };
 AtPlan at_plan(int32_t B, int32_t H, int32_t max_len) {
     const int tiles_bound = (max_len + AT_KEYS - 1) / AT_KEYS;
     const long long units_bound = (long long)B * H * tiles_bound;
-    // One short sequence (a decoding step with a few hundred cached tokens): every head on its own.  A head's
-    // tiles are shared by the CTAs of a cluster, which merge their pieces through distributed shared memory;
-    // where clusters do not fit (or there is a single tile) one CTA takes the whole head.  No pieces go through
-    // global memory and no merge kernel is needed.
-    if (B == 1 && tiles_bound <= AT_WHOLE_HEAD_TILES && H <= AT_MAX_GRID) {
+    // One sequence: every head on its own.  A head's tiles are shared by the CTAs of a cluster, which merge their
+    // pieces through distributed shared memory: no pieces go through global memory and no merge kernel is needed.
+    // Where clusters do not fit, one CTA takes a whole head of up to AT_WHOLE_HEAD_TILES tiles.
+    if (B == 1 && H <= AT_MAX_GRID) {
         const int c = tiles_bound >= 2 ? at_cluster_size(H) : 1;
-        return AtPlan{H * c, c, false};
+        if (c > 1 || tiles_bound <= AT_WHOLE_HEAD_TILES) return AtPlan{H * c, c, false};
     }
     return AtPlan{(int)(units_bound < AT_MAX_GRID ? units_bound : AT_MAX_GRID), 1, true};
 }
