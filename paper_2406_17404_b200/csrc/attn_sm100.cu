@@ -94,17 +94,38 @@ __device__ __forceinline__ uint64_t desc_mnmajor(uint32_t addr) {
     return (uint64_t)((addr & 0x3FFFF) >> 4) | ((uint64_t)(AT_SUB >> 4) << 16) | ((uint64_t)(1024 >> 4) << 32) |
            ((uint64_t)1 << 46) | ((uint64_t)2 << 61);
 }
-__device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
-    asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
-                 "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-                 ::"r"(tmem_d), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
+// Eight MMAs in one go.  A single thread issues them, and its integer work per MMA is what limits the tile loop,
+// so the descriptors are not rebuilt: the high words are constants and a step along the contraction dimension
+// only adds to the start-address field of the low word (the operands stay inside one 256 KB window).
+// S = Q.K^T for one tile: both operands K-major; step kk adds (kk / 4) sub-tiles + (kk % 4) * 32 bytes.
+#define TRJ_MMA_SS(step, pred)                                                            \
+    "add.u32 al, %1, " #step ";\n\tadd.u32 bl, %2, " #step ";\n\t"                        \
+    "mov.b64 da, {al, %3};\n\tmov.b64 db, {bl, %3};\n\t"                                  \
+    "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %4, " #pred ";\n\t"
+__device__ __forceinline__ void umma8_qk(uint32_t tmem_d, uint32_t a_lo, uint32_t b_lo, uint32_t desc_hi, uint32_t idesc) {
+    asm volatile("{\n\t.reg .pred pt, pf;\n\t.reg .b32 al, bl;\n\t.reg .b64 da, db;\n\t"
+                 "setp.eq.b32 pt, 0, 0;\n\tsetp.ne.b32 pf, 0, 0;\n\t"
+                 TRJ_MMA_SS(0, pf) TRJ_MMA_SS(2, pt) TRJ_MMA_SS(4, pt) TRJ_MMA_SS(6, pt)
+                 TRJ_MMA_SS(1024, pt) TRJ_MMA_SS(1026, pt) TRJ_MMA_SS(1028, pt) TRJ_MMA_SS(1030, pt)
+                 "}"
+                 ::"r"(tmem_d), "r"(a_lo), "r"(b_lo), "r"(desc_hi), "r"(idesc) : "memory");
 }
-// Same with the A operand (P) read from tensor memory: lane = row, 16 contraction elements = 8 columns.
-__device__ __forceinline__ void umma_bf16_ts(uint32_t tmem_d, uint32_t tmem_a, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
-    asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
-                 "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
-                 ::"r"(tmem_d), "r"(tmem_a), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
+#undef TRJ_MMA_SS
+// O (+)= P.V for one tile: P from tensor memory (16 keys = 8 columns per step), V MN-major (16 keys = 2048 bytes per step).
+#define TRJ_MMA_TS(kk, pred)                                                              \
+    "add.u32 ta, %1, " #kk "*8;\n\tadd.u32 bl, %2, " #kk "*128;\n\t"                      \
+    "mov.b64 db, {bl, %3};\n\t"                                                            \
+    "tcgen05.mma.cta_group::1.kind::f16 [%0], [ta], db, %4, " #pred ";\n\t"
+__device__ __forceinline__ void umma8_pv(uint32_t tmem_d, uint32_t tmem_a, uint32_t b_lo, uint32_t desc_hi, uint32_t idesc,
+                                         uint32_t accumulate_first) {
+    asm volatile("{\n\t.reg .pred pt, pf;\n\t.reg .b32 ta, bl;\n\t.reg .b64 db;\n\t"
+                 "setp.eq.b32 pt, 0, 0;\n\tsetp.ne.b32 pf, %5, 0;\n\t"
+                 TRJ_MMA_TS(0, pf) TRJ_MMA_TS(1, pt) TRJ_MMA_TS(2, pt) TRJ_MMA_TS(3, pt)
+                 TRJ_MMA_TS(4, pt) TRJ_MMA_TS(5, pt) TRJ_MMA_TS(6, pt) TRJ_MMA_TS(7, pt)
+                 "}"
+                 ::"r"(tmem_d), "r"(tmem_a), "r"(b_lo), "r"(desc_hi), "r"(idesc), "r"(accumulate_first) : "memory");
 }
+#undef TRJ_MMA_TS
 __device__ __forceinline__ void umma_commit(uint32_t bar) {
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
 }
@@ -391,11 +412,9 @@ __global__ void __launch_bounds__(AT_THREADS, 1) tree_attention_tc_kernel(const 
                 if (!mbar_wait(bar(B_KV_FULL + slot), (uint32_t)((2 * gg) / AT_RING) & 1u, &abort_flag, p.status)) return false;
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                 const uint32_t k_smem = ring_smem + slot * AT_TILE;
-#pragma unroll 1
-                for (int kk = 0; kk < 8; ++kk) {            // 8 x 16 elements of head_dim (rolled: one thread, cold code): two sub-tiles of four steps
-                    const uint32_t off = (kk >> 2) * AT_SUB + (kk & 3) * 32;
-                    umma_bf16(tmem_s[gg & 1], desc_kmajor(q_smem + off), desc_kmajor(k_smem + off), idesc_qk, kk > 0);
-                }
+                // 8 x 16 elements of head_dim: two sub-tiles of four steps
+                const uint64_t q_desc = desc_kmajor(q_smem), k_desc = desc_kmajor(k_smem);
+                umma8_qk(tmem_s[gg & 1], (uint32_t)q_desc, (uint32_t)k_desc, (uint32_t)(q_desc >> 32), idesc_qk);
                 umma_commit(bar(B_S_FULL + (gg & 1)));
                 umma_commit(bar(B_KV_EMPTY + slot));
                 return true;
@@ -425,13 +444,9 @@ __global__ void __launch_bounds__(AT_THREADS, 1) tree_attention_tc_kernel(const 
                     if (!ok) break;
                     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                     const uint32_t v_smem = ring_smem + slot * AT_TILE;
-#pragma unroll 1
-                    for (int kk = 0; kk < 8; ++kk) {        // 8 x 16 keys
-                        const uint32_t v_off = kk * 16 * 128;                          // V: 16 keys = 16 rows of 128 bytes
-                        // P comes straight from TMEM: 16 keys = 8 columns of bf16 pairs
-                        umma_bf16_ts(tmem_o, tmem_p[g & 1] + 8 * kk, desc_mnmajor(v_smem + v_off), idesc_pv,
-                                     (g > g0 || kk > 0) ? 1u : 0u);
-                    }
+                    // 8 x 16 keys; P comes straight from TMEM
+                    const uint64_t v_desc = desc_mnmajor(v_smem);
+                    umma8_pv(tmem_o, tmem_p[g & 1], (uint32_t)v_desc, (uint32_t)(v_desc >> 32), idesc_pv, g > g0 ? 1u : 0u);
                     umma_commit(bar(B_P_FREE + (g & 1)));
                     umma_commit(bar(B_KV_EMPTY + slot));
                 }

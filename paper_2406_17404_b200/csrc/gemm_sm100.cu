@@ -69,6 +69,18 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
     return false;
 }
 
+// Weights are read once per step and are far larger than L2: they are loaded with an evict-first policy so that
+// they do not push out what is reused between kernels (activations, split-K pieces, and the kernels' own code).
+__device__ __forceinline__ uint64_t l2_evict_first_policy() {
+    uint64_t policy;
+    asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(policy));
+    return policy;
+}
+__device__ __forceinline__ void tma_load_2d_hint(uint32_t dst, const CUtensorMap* map, int c_inner, int c_outer, uint32_t bar,
+                                                 uint64_t policy) {
+    asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1, {%2, %3}], [%4], %5;"
+                 ::"r"(dst), "l"(map), "r"(c_inner), "r"(c_outer), "r"(bar), "l"(policy) : "memory");
+}
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int c_inner, int c_outer, uint32_t bar) {
     asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
                  ::"r"(dst), "l"(map), "r"(c_inner), "r"(c_outer), "r"(bar) : "memory");
@@ -159,6 +171,7 @@ __global__ void __launch_bounds__(TC_THREADS, 2) gemm_tc_kernel(const __grid_con
             // previous kernel of the stream; the activation tiles of those stages follow after the wait.
             bool ok = true;
             int prefetched = 0;
+            const uint64_t w_policy = l2_evict_first_policy();
             for (int pass = 0; pass < 2 && ok; ++pass) {
                 int fill = 0;                                // running stage counter
                 for (int item = blockIdx.x; item < items && ok; item += gridDim.x) {
@@ -172,7 +185,7 @@ __global__ void __launch_bounds__(TC_THREADS, 2) gemm_tc_kernel(const __grid_con
                         if (pass == 0) {                     // weights only, at most one ring-full
                             if (fill >= p.stages) break;
                             mbar_expect_tx(bar, stage_bytes);
-                            tma_load_2d(a_dst, &map_w, kb * TC_BK, tile * TC_BM, bar);
+                            tma_load_2d_hint(a_dst, &map_w, kb * TC_BK, tile * TC_BM, bar, w_policy);
                             prefetched = fill + 1;
                             continue;
                         }
@@ -181,7 +194,7 @@ __global__ void __launch_bounds__(TC_THREADS, 2) gemm_tc_kernel(const __grid_con
                             ok = mbar_wait(empty0 + 8 * s, phase ^ 1u, &abort_flag, p.status);
                             if (!ok) break;
                             mbar_expect_tx(bar, stage_bytes);
-                            tma_load_2d(a_dst, &map_w, kb * TC_BK, tile * TC_BM, bar);
+                            tma_load_2d_hint(a_dst, &map_w, kb * TC_BK, tile * TC_BM, bar, w_policy);
                         }
                         tma_load_2d(b_dst, &map_x, kb * TC_BK, 0, bar);
                         if (p.halves == 2) tma_load_2d(b_dst + (uint32_t)p.m_pad * TC_BK * 2, &map_xlo, kb * TC_BK, 0, bar);
