@@ -77,6 +77,18 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
     atomicExch(status, (int)TRJ_ETIMEOUT);
     return false;
 }
+// Cache tiles are read once per launch and, over a step, are larger than L2: evict-first keeps them from pushing
+// out what is reused between kernels.
+__device__ __forceinline__ uint64_t l2_evict_first_policy() {
+    uint64_t policy;
+    asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(policy));
+    return policy;
+}
+__device__ __forceinline__ void tma_load_2d_hint(uint32_t dst, const CUtensorMap* map, int c_inner, int c_outer, uint32_t bar,
+                                                 uint64_t policy) {
+    asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1, {%2, %3}], [%4], %5;"
+                 ::"r"(dst), "l"(map), "r"(c_inner), "r"(c_outer), "r"(bar), "l"(policy) : "memory");
+}
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int c_inner, int c_outer, uint32_t bar) {
     asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
                  ::"r"(dst), "l"(map), "r"(c_inner), "r"(c_outer), "r"(bar) : "memory");
@@ -361,6 +373,7 @@ __global__ void __launch_bounds__(AT_THREADS, 1) tree_attention_tc_kernel(const 
             int g = 0, e = 0;
             bool ok = true;
             bool waited = false;                             // for the previous kernel (see above)
+            const uint64_t kv_policy = l2_evict_first_policy();
             for (int u = u_begin; u < u_end && ok;) {
                 Where w; sched.locate(u, w);
                 const int t_end = min(w.tiles, w.t + (u_end - u));
@@ -389,8 +402,8 @@ __global__ void __launch_bounds__(AT_THREADS, 1) tree_attention_tc_kernel(const 
                         const uint32_t dst = ring_smem + slot * AT_TILE;
                         mbar_expect_tx(bar(B_KV_FULL + slot), AT_TILE);
                         const CUtensorMap* map = kv ? &map_v : &map_k;
-                        tma_load_2d(dst, map, 0, cache_row0 + t * AT_KEYS, bar(B_KV_FULL + slot));
-                        tma_load_2d(dst + AT_SUB, map, 64, cache_row0 + t * AT_KEYS, bar(B_KV_FULL + slot));
+                        tma_load_2d_hint(dst, map, 0, cache_row0 + t * AT_KEYS, bar(B_KV_FULL + slot), kv_policy);
+                        tma_load_2d_hint(dst + AT_SUB, map, 64, cache_row0 + t * AT_KEYS, bar(B_KV_FULL + slot), kv_policy);
                     }
                 }
                 if (!waited) { pdl_wait(); waited = true; }  // the next segment's Q comes from the previous kernel
