@@ -464,12 +464,20 @@ def run_ours(args, rank, world, local_rank):
     gemm_ms, gemm_launches = prof["gemm"]
     gemm_ms_step = gemm_ms / args.steps
     gbytes = gemm_bytes_per_step(cfg, TREE_ROWS)
-    achieved = gbytes / (gemm_ms_step / 1e3) / 1e9 if gemm_ms_step > 0 else None
+    # Inside the replayed step the projections overlap their neighbours (programmatic dependent launch), so their
+    # own duration cannot be bracketed without changing it: event nodes around every launch serialise the chain and
+    # make the 129 projections alone look longer than the whole real step.  The roofline therefore charges the
+    # WHOLE step's device time (timed region 1, CUDA events) to the projections, an upper bound of their duration;
+    # the bracketed figure is kept beside it.
+    gemm_ms_upper = min(gemm_ms_step, ms_step) if gemm_ms_step > 0 else ms_step
+    achieved = gbytes / (gemm_ms_upper / 1e3) / 1e9
     roofline = {"bound": "hbm", "kernel": "projection GEMMs (all %d launches of a step)" % (gemm_launches // args.steps),
                 "achieved": achieved, "peak": peaks["hbm_gbs"], "peak_source": peaks["source"], "unit": "GB/s",
-                "frac": achieved / peaks["hbm_gbs"] if achieved else None,
+                "frac": achieved / peaks["hbm_gbs"],
                 "traffic": GEMM_TRAFFIC_BYTES_PER_STEP, "algorithmic_bytes_per_step": gbytes,
-                "device_ms_per_step": gemm_ms_step}
+                "device_ms_per_step": gemm_ms_upper,
+                "duration_basis": "whole replayed step (upper bound)" if gemm_ms_upper == ms_step else "event brackets",
+                "bracketed_ms_per_step": gemm_ms_step}
     step_ms_prof = sum(v[0] for v in prof.values()) / args.steps
     breakdown = {k: {"ms_per_step": round(v[0] / args.steps, 4), "launches_per_step": v[1] // args.steps} for k, v in prof.items()}
 

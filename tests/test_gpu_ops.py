@@ -45,6 +45,18 @@ def test_tree_attention_small(trj, dtype, h, d, s, m):
     check_attention(trj, case)
 
 
+@pytest.mark.parametrize("h,s,m", [
+    (2, 3000, 128),      # clusters of 4 with six or seven key tiles per CTA (the K/V ring wraps)
+    (40, 700, 20),       # 4 x 40 CTAs would not fit: clusters of 2
+    (80, 1500, 16),      # no clusters and more tiles than one CTA takes per head: contiguous ranges + merge kernel
+    (80, 600, 16),       # no clusters, few tiles: one CTA per head
+])
+def test_tree_attention_launch_shapes_single_sequence(trj, h, s, m):
+    """One sequence, head counts and lengths that exercise every launch shape the host chooses from."""
+    case = AttnCase(trj, h, h, 128, [s], [m], [synth.random_tree(h + s, m, min(8, m - 1), 3)], "bf16")
+    check_attention(trj, case, heads=[0, h // 2, h - 1])
+
+
 def test_tree_attention_chain_is_causal(trj):
     """A chain tree on the GPU reproduces causal attention (oracle pinned to a library routine)."""
     m = 96
