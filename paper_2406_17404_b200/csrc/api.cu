@@ -136,6 +136,7 @@ struct trj_ctx {
     float* h; float* y; float* logits;
     void* x; void* x_lo; void* q; void* act; void* act_lo;   // *_lo: low halves of split bf16 activations
     double* inv_freq;
+    int sm_count;          // SMs of the device the context lives on
     void* argmax_ws; void* attn_ws; size_t attn_ws_bytes; void* gemm_ws; size_t gemm_ws_bytes;
     // chain-tree tables for prefill and the staging area of trj_step_host (device)
     int32_t* chain_depth; uint64_t* chain_anc; int32_t* chunk_row_off; int32_t* unit_row_off;
@@ -248,6 +249,12 @@ trj_status forward(trj_ctx* ctx, void* k_cache, void* v_cache, int32_t b0, const
     const int M = bt.rows_total, d = c.d_model, HD = c.n_heads * c.head_dim;
     const size_t es = dtype_size(c.dtype);
     const size_t seq_stride = (size_t)c.n_heads * c.max_seq * c.head_dim * es;     // one sequence of one layer
+    // CTAs of the attention launch: what it leaves of the device is free while it runs (the plain kernel fills it)
+    const bool attn_tc = ctx->attn_ws && ((uintptr_t)ctx->attn_ws % 256) == 0 &&
+                         ctx->attn_ws_bytes >= tree_attention_tc_workspace(bt.B, c.n_heads) &&
+                         tree_attention_tc_supported(c.head_dim, c.dtype, bt.max_rows);
+    const int attn_grid = attn_tc ? tree_attention_grid(bt.B, c.n_heads, bt.max_len) : ctx->sm_count;
+    constexpr size_t AHEAD_BYTES = (size_t)32 << 20;         // measured optimum on the 7B shape (16-40 MB are close)
     LAUNCH(PROF_ELEMENTWISE, launch_embed(ctx->embed, c.dtype, tokens, ctx->h, M, d, st));
     Parts pr{nullptr, 1, 0};                 // result of the latest projection, possibly in split-K pieces
     for (int l = 0; l < c.n_layers; ++l) {
@@ -264,8 +271,11 @@ trj_status forward(trj_ctx* ctx, void* k_cache, void* v_cache, int32_t b0, const
         LAUNCH(PROF_ATTENTION, launch_tree_attention(ctx->q, k_slab, v_slab, anc, anc_words, bt, c.n_heads, c.head_dim,
                                                      c.max_seq, c.dtype, ctx->x, ctx->x_lo, ctx->attn_ws,
                                                      ctx->attn_ws_bytes, st));
+        // While the attention kernel runs, HBM is nearly idle and the SMs it leaves free go to the first CTAs of
+        // the output projection, which only wait: they ask for the start of the gate/up weights into L2.
+        const WeightPrefetch ahead{ctx->w_gate_up[l], 2 * c.d_ff, d, AHEAD_BYTES, 2 * std::max(0, ctx->sm_count - attn_grid)};
         LAUNCH(PROF_GEMM, launch_gemm(ctx->x, ctx->x_lo, ctx->wo[l], ctx->y, M, d, HD, c.dtype, ctx->gemm_ws,
-                                      ctx->gemm_ws_bytes, st, &pr));
+                                      ctx->gemm_ws_bytes, st, &pr, &ahead));
         LAUNCH(PROF_ELEMENTWISE, launch_add_rmsnorm(ctx->h, pr, ctx->mlp_norm[l], ctx->x, ctx->x_lo, c.dtype, M, d,
                                                     c.rms_eps, st));
         LAUNCH(PROF_GEMM, launch_gemm(ctx->x, ctx->x_lo, ctx->w_gate_up[l], ctx->y, M, 2 * c.d_ff, d, c.dtype, ctx->gemm_ws,
@@ -321,6 +331,12 @@ extern "C" trj_status trj_create(const trj_model_cfg* cfg, const trj_weights* w,
     trj_ctx* ctx = new (std::nothrow) trj_ctx();
     TRJ_REQUIRE(ctx, TRJ_ECUDA, "create: out of host memory");
     ctx->cfg = *cfg;
+    {
+        int dev = 0, sms = 0;
+        if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
+            sms = 0;
+        ctx->sm_count = sms;
+    }
     ctx->embed = w->embed; ctx->lm_head = w->lm_head; ctx->final_norm = w->final_norm;
     for (int l = 0; l < cfg->n_layers; ++l) {
         ctx->attn_norm.push_back(w->attn_norm[l]); ctx->mlp_norm.push_back(w->mlp_norm[l]);

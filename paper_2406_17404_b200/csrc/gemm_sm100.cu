@@ -36,6 +36,7 @@ struct TcParams {
     int tiles, splits, stages;
     float* out;         // [splits][M][N]
     int* status;        // device word: 0, or TRJ_ETIMEOUT once a wait expired
+    int ahead_boxes, ahead_kblocks, ahead_ctas;   // [128 x 64] tiles of a later projection's weights to request into L2
 };
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -80,6 +81,11 @@ __device__ __forceinline__ void tma_load_2d_hint(uint32_t dst, const CUtensorMap
                                                  uint64_t policy) {
     asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1, {%2, %3}], [%4], %5;"
                  ::"r"(dst), "l"(map), "r"(c_inner), "r"(c_outer), "r"(bar), "l"(policy) : "memory");
+}
+// Asks for one box of the tensor to be brought into L2; nothing is written to shared memory and nothing signals.
+__device__ __forceinline__ void tma_prefetch_l2_2d(const CUtensorMap* map, int c_inner, int c_outer) {
+    asm volatile("cp.async.bulk.prefetch.tensor.2d.L2.global.tile [%0, {%1, %2}];"
+                 ::"l"(map), "r"(c_inner), "r"(c_outer) : "memory");
 }
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int c_inner, int c_outer, uint32_t bar) {
     asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
@@ -127,7 +133,7 @@ __device__ __forceinline__ void tmem_ld16(uint32_t taddr, float* v) {
 // loads and MMAs of the next.  Warp 0: TMA producer, warp 1: MMA issuer, warps 2-5: epilogue.
 __global__ void __launch_bounds__(TC_THREADS, 2) gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w,
                                                                 const __grid_constant__ CUtensorMap map_x,
-                                                                const __grid_constant__ CUtensorMap map_xlo,
+                                                                const __grid_constant__ CUtensorMap map_xlo, const __grid_constant__ CUtensorMap map_ahead,
                                                                 const TcParams p) {
     extern __shared__ uint8_t smem_raw[];
     __shared__ __align__(8) uint64_t bars[2 * TC_MAX_STAGES + 4];
@@ -201,7 +207,13 @@ __global__ void __launch_bounds__(TC_THREADS, 2) gemm_tc_kernel(const __grid_con
                     }
                     if (pass == 0 && fill >= p.stages) break;
                 }
-                if (pass == 0) pdl_wait();                   // activations come from the previous kernel
+                if (pass == 0) {
+                    // CTAs that run while the previous kernel still does: a later projection's weights into L2
+                    if ((int)blockIdx.x < p.ahead_ctas)
+                        for (int i = blockIdx.x; i < p.ahead_boxes; i += p.ahead_ctas)
+                            tma_prefetch_l2_2d(&map_ahead, (i % p.ahead_kblocks) * TC_BK, (i / p.ahead_kblocks) * TC_BM);
+                    pdl_wait();                              // activations come from the previous kernel
+                }
             }
         }
     } else if (warp == 1) {
@@ -354,7 +366,7 @@ size_t gemm_tc_workspace(int32_t M, int32_t N, int32_t K) {
 }
 
 cudaError_t launch_gemm_tc(const void* x, const void* x_lo, const void* w, float* y, int32_t M, int32_t N, int32_t K,
-                           void* workspace, cudaStream_t st, Parts* parts) {
+                           void* workspace, cudaStream_t st, Parts* parts, const WeightPrefetch* ahead) {
     int* status = (int*)workspace;
     workspace = (char*)workspace + 256;
     static std::once_flag once;
@@ -383,14 +395,26 @@ cudaError_t launch_gemm_tc(const void* x, const void* x_lo, const void* w, float
     if (p.stages < 2) return cudaErrorInvalidConfiguration;
     p.out = p.splits > 1 ? (float*)workspace : y;
     p.status = status;
-    CUtensorMap map_w, map_x, map_xlo;
+    CUtensorMap map_w, map_x, map_xlo, map_ahead;
+    p.ahead_boxes = 0; p.ahead_kblocks = 1; p.ahead_ctas = 0;
+    const bool want_ahead = ahead && ahead->ctas > 0 && ahead->w && ahead->K % TC_BK == 0 && ahead->K >= TC_BK &&
+                            ((uintptr_t)ahead->w % 16) == 0;
+    if (want_ahead) {
+        if (!make_map(&map_ahead, ahead->w, ahead->N, ahead->K, TC_BM)) return cudaErrorInvalidValue;
+        const size_t all = (size_t)((ahead->N + TC_BM - 1) / TC_BM) * (ahead->K / TC_BK);
+        const size_t asked = ahead->bytes / TC_A_BYTES;
+        p.ahead_kblocks = ahead->K / TC_BK;
+        p.ahead_boxes = (int)(asked < all ? asked : all);
+        p.ahead_ctas = ahead->ctas;
+    }
     if (!make_map(&map_w, w, N, K, TC_BM) || !make_map(&map_x, x, M, K, p.m_pad) ||
         !make_map(&map_xlo, x_lo ? x_lo : x, M, K, p.m_pad))
         return cudaErrorInvalidValue;
+    if (!want_ahead) map_ahead = map_w;                      // never used: no CTA asks
     count_launch();
     const int items = p.tiles * p.splits;
     cudaError_t e = launch_chain(gemm_tc_kernel, dim3(items < TC_GRID ? items : TC_GRID), dim3(TC_THREADS),
-                                 p.stages * stage + 1024, st, map_w, map_x, map_xlo, p);
+                                 p.stages * stage + 1024, st, map_w, map_x, map_xlo, map_ahead, p);
     if (e == cudaSuccess) e = cudaGetLastError();
     if (parts) *parts = Parts{p.out, p.splits, (size_t)M * N};
     if (e != cudaSuccess || p.splits == 1 || parts) return e;
@@ -402,10 +426,11 @@ cudaError_t launch_gemm_tc(const void* x, const void* x_lo, const void* w, float
 }
 
 cudaError_t launch_gemm(const void* x, const void* x_lo, const void* w, float* y, int32_t M, int32_t N, int32_t K,
-                        int32_t dtype, void* workspace, size_t workspace_bytes, cudaStream_t st, Parts* parts) {
+                        int32_t dtype, void* workspace, size_t workspace_bytes, cudaStream_t st, Parts* parts,
+                        const WeightPrefetch* ahead) {
     if (workspace && workspace_bytes >= gemm_tc_workspace(M, N, K) && ((uintptr_t)workspace % 256) == 0 &&
         gemm_tc_supported(x, x_lo, w, y, M, N, K, dtype))
-        return launch_gemm_tc(x, x_lo, w, y, M, N, K, workspace, st, parts);
+        return launch_gemm_tc(x, x_lo, w, y, M, N, K, workspace, st, parts, ahead);
     if (parts) *parts = whole(y);
     return launch_gemm_simt(x, x_lo, w, y, M, N, K, dtype, st);
 }

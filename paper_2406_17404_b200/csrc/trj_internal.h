@@ -79,6 +79,12 @@ struct Batch {
     int32_t B, rows_total, max_rows, max_len;
 };
 
+// Weights of a LATER projection that a projection kernel may ask for ahead of time.  When the kernel before a
+// projection leaves SMs free and HBM idle (the attention kernel of a decoding step does both), the projection's
+// first `ctas` CTAs get those SMs at once and spend their wait requesting the first `bytes` of `w` ([N][K] bf16)
+// into L2, so that the later projection starts from L2 instead of HBM.  ctas = 0: nothing is requested.
+struct WeightPrefetch { const void* w; int32_t N, K; size_t bytes; int32_t ctas; };
+
 // A projection result that may still be in split-K pieces: value(i) = sum over s < splits of ptr[s * stride + i].
 struct Parts { const float* ptr; int32_t splits; size_t stride; };
 inline Parts whole(const float* p) { return Parts{p, 1, 0}; }
@@ -99,12 +105,12 @@ bool gemm_tc_supported(const void* x, const void* x_lo, const void* w, const flo
                        int32_t dtype);
 size_t gemm_tc_workspace(int32_t M, int32_t N, int32_t K);
 cudaError_t launch_gemm_tc(const void* x, const void* x_lo, const void* w, float* y, int32_t M, int32_t N, int32_t K,
-                           void* workspace, cudaStream_t st, Parts* parts);
+                           void* workspace, cudaStream_t st, Parts* parts, const WeightPrefetch* ahead = nullptr);
 // Picks the tcgen05 kernel when the shape allows it, the plain kernel otherwise.  With `parts` non-null the
 // split-K pieces are left unreduced in the workspace for the consumer to add (*parts says where); otherwise
 // y holds the finished result.
 cudaError_t launch_gemm(const void* x, const void* x_lo, const void* w, float* y, int32_t M, int32_t N, int32_t K,
-                        int32_t dtype, void* workspace, size_t workspace_bytes, cudaStream_t st, Parts* parts = nullptr);
+                        int32_t dtype, void* workspace, size_t workspace_bytes, cudaStream_t st, Parts* parts = nullptr, const WeightPrefetch* ahead = nullptr);
 
 // Rotary embedding of q and k at position seq_len[b] + depth[row]; q -> q_out [rows][H][D];
 // k, v -> cache rows seq_len[b] + local row of the layer slab [B][H][max_seq][D].
