@@ -443,6 +443,40 @@ def run_ours(args, rank, world, local_rank):
         mat.append(k + 1)
     torch.cuda.synchronize()
     e2e_s = time.perf_counter() - t0
+
+    # ---- the same loop resident on the device (trj_decode_device): the host uploads the random draws of all steps,
+    #      enqueues the steps and reads the generated tokens back at the end; wall clock around all of it
+    n_loop = args.steps
+    cap = n_ctx + n_loop * (max(WIDTH, BRANCH_LEN) + 1)
+    host_ctx = np.zeros(cap, np.int32)
+    host_ctx[:n_ctx] = ctx_buf[:n_ctx]
+    host_ctx_t, host_n_t = torch.from_numpy(host_ctx).pin_memory(), torch.tensor([n_ctx], dtype=torch.int32).pin_memory()
+    host_window_t = torch.from_numpy(np.ascontiguousarray(window, dtype=np.int32)).pin_memory()
+    loop_draws = torch.from_numpy(np.stack([np.asarray(draw(10_000 + s, WIDTH + N_BRANCHES * BRANCH_LEN), np.int64)
+                                            for s in range(n_loop)])).pin_memory()
+    d_ctx, d_n = torch.empty(cap, dtype=torch.int32, device=dev), torch.empty(1, dtype=torch.int32, device=dev)
+    d_window, d_draws = torch.empty(WIDTH, dtype=torch.int32, device=dev), torch.empty_like(loop_draws, device=dev)
+    out_tokens, out_n = torch.empty(cap, dtype=torch.int32).pin_memory(), torch.empty(1, dtype=torch.int32).pin_memory()
+
+    def device_loop():
+        t1 = time.perf_counter()
+        d_ctx.copy_(host_ctx_t, non_blocking=True); d_n.copy_(host_n_t, non_blocking=True)
+        d_window.copy_(host_window_t, non_blocking=True); d_draws.copy_(loop_draws, non_blocking=True)
+        model.decode_device(d_ctx, d_n, n_ctx, d_window, N_BRANCHES, BRANCH_LEN, d_draws, n_loop)
+        out_tokens.copy_(d_ctx, non_blocking=True); out_n.copy_(d_n, non_blocking=True)
+        torch.cuda.synchronize()
+        dt = time.perf_counter() - t1
+        assert int(out_n[0]) - n_ctx >= n_loop
+        return dt
+    device_loop()                                            # warm-up: same sizes and buffers, so its step graph is reused
+    model.seq_len.fill_(n_ctx - 1)                           # rewind the cache to the state before the warm-up loop
+    loop_s = device_loop()
+    loop_h2d = int(host_ctx.nbytes + 4 + host_window_t.numel() * 4 + loop_draws.numel() * 8)
+    loop_d2h = int(cap * 4 + 4)
+    if world > 1:                                            # replicas: the slowest rank's loop
+        t_loop = torch.tensor([loop_s], dtype=torch.float64, device=dev)
+        dist.all_reduce(t_loop, op=dist.ReduceOp.MAX)
+        loop_s = float(t_loop[0])
     barrier()
     clocks = sampler.stop()
 
@@ -499,6 +533,10 @@ def run_ours(args, rank, world, local_rank):
             "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": trj.STEP_H2D_BYTES,
                     "d2h_bytes_per_step": trj.STEP_D2H_BYTES, "ms_per_step": 1e3 * e2e_s / args.steps,
                     "tokens_committed_per_step": sum(mat[-args.steps:]) / args.steps},
+            "device_loop": {"value": whole_job_rate(world, DRAFTS * args.steps, loop_s), "unit": UNIT,
+                            "ms_per_step": 1e3 * loop_s / args.steps, "h2d_bytes_total": loop_h2d, "d2h_bytes_total": loop_d2h,
+                            "what": "trj_decode_device: %d steps enqueued at once, drafting and refill on the device; "
+                                    "wall clock incl. uploading the draws and reading the tokens back" % args.steps},
             "roofline": roofline, "kernel_breakdown": breakdown, "profiled_step_ms": step_ms_prof}
     if world == 1:
         if not args.no_attention:

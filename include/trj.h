@@ -291,6 +291,51 @@ trj_status trj_step_host(trj_ctx* ctx, void* k_cache, void* v_cache, int32_t* se
                          int32_t* k_acc, int32_t* path, int32_t* bonus, void* stream);
 
 /* ------------------------------------------------------------------------
+ * Drafting and refill on the device: the integer work between two verification
+ * steps, so that a decode loop needs no host round trip per step.  Same rules
+ * as trj_retrieve / trj_build_tree / trj_refill_window (Section 3.3: drafts are
+ * retrieved from the tokens seen so far and the window is refilled from the
+ * chosen path's own predictions; Eq. 4: ahead noise), on device buffers.
+ * All pointers dev; launches only, nothing is synchronised.
+ *
+ * trj_draft_tokens: tokens [1 + W + R*branch_len] of the next tree in the fixed
+ * layout of trj_build_tree: root = context[n_ctx - 1], then window [W], then R
+ * retrieved branches.  draws [W + R*branch_len] int64 >= 0; slots [W, ...) feed
+ * the branches' ahead noise (context[draw % n_ctx]).  R <= 64.
+ *
+ * trj_commit_refill: appends tokens[path[1..k]] and *bonus to context
+ * (capacity ints; *n_ctx += k + 1), then writes the next window [W]:
+ * node_argmax of the lowest-index child, level by level, below path[k], then
+ * ahead noise context[draws[i] % n_ctx] on the grown context.  A context that
+ * would overflow is left untouched and *overflow (may be null) is set to 1. */
+trj_status trj_draft_tokens(const int32_t* context, const int32_t* n_ctx, const int32_t* window, int32_t W,
+                            int32_t R, int32_t branch_len, const int64_t* draws, int32_t* tokens, void* stream);
+trj_status trj_commit_refill(const int32_t* tokens, const int32_t* parent, const int32_t* node_argmax, int32_t M,
+                             const int32_t* k_acc, const int32_t* path, const int32_t* bonus, int32_t* context,
+                             int32_t capacity, int32_t* n_ctx, int32_t W, const int64_t* draws, int32_t* window,
+                             int32_t* overflow, void* stream);
+
+/* n_steps whole decode steps for batch 1 with everything resident on the device
+ * (Section 3.3: draft, verify, accept, commit, refill): per step trj_draft_tokens, the verification forward, arg-max +
+ * acceptance, KV compaction and trj_commit_refill are enqueued on `stream`; the
+ * host is not involved between steps and the call does not wait for them.
+ *   dev in/out: k_cache, v_cache, seq_len [1]; context [capacity] with *n_ctx
+ *               valid tokens (prompt + generated; the last one is the next root,
+ *               so seq_len[0] == *n_ctx - 1); window [W] (the next window)
+ *   dev in    : draws [n_steps][W + R*branch_len] int64 >= 0 (step i uses row i:
+ *               slots [W, ...) for its retrieval, slots [0, W) for its refill)
+ *   dev out   : k_log [n_steps] accepted draft tokens per step (may be null)
+ *   host      : n_ctx_now = the value of *n_ctx at the time of the call (used for
+ *               the capacity checks: every step commits at most
+ *               max(W, branch_len) + 1 tokens)
+ * TRJ_ECAPACITY if the context buffer, cfg.max_seq or cfg.max_rows cannot take
+ * the worst case; nothing is enqueued then. */
+trj_status trj_decode_device(trj_ctx* ctx, void* k_cache, void* v_cache, int32_t* seq_len, int32_t* context,
+                             int32_t capacity, int32_t* n_ctx, int32_t n_ctx_now, int32_t* window, int32_t W,
+                             int32_t R, int32_t branch_len, const int64_t* draws, int32_t n_steps,
+                             int32_t* k_log, void* stream);
+
+/* ------------------------------------------------------------------------
  * The projections as a stand-alone op: y[M][N] (fp32) = x[M][K] . w[N][K]^T,
  * x and w of `dtype`, all dev.  Used by the model path for every projection
  * and exposed for measurement.  workspace: dev, >= trj_gemm_workspace(M, N, K)

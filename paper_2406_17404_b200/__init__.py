@@ -74,6 +74,9 @@ _SIGNATURES = {
     "trj_prefill": (_I, [_VP, _VP, _VP, _VP, _I, _VP, _I, _VP, _VP]),
     "trj_step_host": (_I, [_VP, _VP, _VP, _VP, _I, _I, _I32P, _I, _I32P, _I, _I, _I32P, _I32P, _I32P, _I32P,
                            _I32P, _I32P, _I32P, _VP]),
+    "trj_draft_tokens": (_I, [_VP, _VP, _VP, _I, _I, _I, _VP, _VP, _VP]),
+    "trj_commit_refill": (_I, [_VP, _VP, _VP, _I, _VP, _VP, _VP, _VP, _I, _VP, _I, _VP, _VP, _VP, _VP]),
+    "trj_decode_device": (_I, [_VP, _VP, _VP, _VP, _VP, _I, _VP, _I, _VP, _I, _I, _I, _VP, _I, _VP, _VP]),
     "trj_gemm_workspace": (_SZ, [_I, _I, _I]),
     "trj_gemm": (_I, [_VP, _VP, _VP, _I, _I, _I, _I, _VP, _SZ, _VP]),
     "trj_launch_count": (C.c_uint64, []),
@@ -309,6 +312,34 @@ def gemm(x, w, *, out=None, workspace=None, stream=None):
     return out
 
 
+def draft_tokens(context, n_ctx, window, n_branches: int, branch_len: int, draws, stream=None):
+    """trj_draft_tokens: the next tree's tokens [1 + W + R*Lr] (int32, device) from device buffers.
+
+    context: int32 [capacity], n_ctx: int32 [1], window: int32 [W], draws: int64 [W + R*Lr], all CUDA tensors."""
+    torch = _torch()
+    w = int(window.numel())
+    out = torch.empty(1 + w + n_branches * branch_len, dtype=torch.int32, device=context.device)
+    _check(lib().trj_draft_tokens(_dev(context, torch.int32, "context"), _dev(n_ctx, torch.int32, "n_ctx"),
+                                  _dev(window, torch.int32, "window") if w else None, w, n_branches, branch_len,
+                                  _dev(draws, torch.int64, "draws"), _dev(out), _stream(stream)))
+    return out
+
+
+def commit_refill(tokens, parent, node_argmax, k_acc, path, bonus, context, n_ctx, width: int, draws, stream=None):
+    """trj_commit_refill: appends the accepted tokens and the bonus to ``context`` (in place, ``n_ctx`` advanced) and
+    returns (next window [width] int32, overflow flag [1] int32), both on the device."""
+    torch = _torch()
+    window = torch.empty(max(width, 1), dtype=torch.int32, device=context.device)
+    overflow = torch.zeros(1, dtype=torch.int32, device=context.device)
+    _check(lib().trj_commit_refill(_dev(tokens, torch.int32, "tokens"), _dev(parent, torch.int32, "parent"),
+                                   _dev(node_argmax, torch.int32, "node_argmax"), int(tokens.numel()),
+                                   _dev(k_acc, torch.int32, "k_acc"), _dev(path, torch.int32, "path"),
+                                   _dev(bonus, torch.int32, "bonus"), _dev(context, torch.int32, "context"),
+                                   int(context.numel()), _dev(n_ctx, torch.int32, "n_ctx"), width,
+                                   _dev(draws, torch.int64, "draws"), _dev(window), _dev(overflow), _stream(stream)))
+    return window[:width], overflow
+
+
 class Model:
     """A decoder context (trj_create) plus its KV cache; methods map one to one onto the C ABI."""
 
@@ -415,6 +446,20 @@ class Model:
         torch = _torch()
         _check(lib().trj_compact_kv(self._handle, _dev(self.k_cache), _dev(self.v_cache), _dev(self.seq_len), batch,
                                     _dev(k_acc, torch.int32), _dev(path, torch.int32), _stream(stream)))
+
+    def decode_device(self, context, n_ctx, n_ctx_now: int, window, n_branches: int, branch_len: int, draws,
+                      n_steps: int, k_log=None, stream=None) -> None:
+        """trj_decode_device: ``n_steps`` decode steps of sequence 0 without the host in between (nothing is
+        synchronised).  context int32 [capacity], n_ctx int32 [1], window int32 [W], draws int64
+        [n_steps, W + R*Lr], k_log int32 [n_steps] or None: CUDA tensors, updated in place."""
+        torch = _torch()
+        w = int(window.numel())
+        _check(lib().trj_decode_device(self._handle, _dev(self.k_cache), _dev(self.v_cache), _dev(self.seq_len),
+                                       _dev(context, torch.int32, "context"), int(context.numel()),
+                                       _dev(n_ctx, torch.int32, "n_ctx"), int(n_ctx_now),
+                                       _dev(window, torch.int32, "window") if w else None, w, n_branches, branch_len,
+                                       _dev(draws, torch.int64, "draws"), int(n_steps),
+                                       _dev(k_log, torch.int32, "k_log") if k_log is not None else None, _stream(stream)))
 
     def step_host(self, root: int, window, branches, max_len: int, stream=None) -> Dict[str, object]:
         """trj_step_host: one whole decode step from host integers; returns host results."""

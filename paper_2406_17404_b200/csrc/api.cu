@@ -140,6 +140,7 @@ struct trj_ctx {
     void* argmax_ws; void* attn_ws; size_t attn_ws_bytes; void* gemm_ws; size_t gemm_ws_bytes;
     // chain-tree tables for prefill and the staging area of trj_step_host (device)
     int32_t* chain_depth; uint64_t* chain_anc; int32_t* chunk_row_off; int32_t* unit_row_off;
+    int32_t* loop_state;   // device: [0] step counter, [1] context-overflow flag of trj_decode_device
     int32_t* step_in;      // tokens | parent | depth | row_off(2) | pad -> anc
     int32_t* step_out;     // node_argmax | k_acc | bonus | path
     int32_t* pin_in; int32_t* pin_out;   // pinned host mirrors
@@ -148,6 +149,9 @@ struct trj_ctx {
     // CUDA graphs of trj_step_host, one per (tree rows, attention grid, buffers)
     struct GraphEntry { int32_t M; int grid; void* k; void* v; void* len; cudaGraphExec_t exec; };
     std::vector<GraphEntry> graphs;
+    // CUDA graphs of one step of trj_decode_device, keyed by every pointer and size the step depends on
+    struct LoopGraph { std::vector<uint64_t> key; cudaGraphExec_t exec; };
+    std::vector<LoopGraph> loop_graphs;
     cudaStream_t cap_stream = nullptr; cudaEvent_t order_ev = nullptr; uint64_t steps_done = 0;
 };
 
@@ -186,6 +190,7 @@ size_t carve(const trj_model_cfg& c, void* ws, trj_ctx* ctx) {
     int32_t* unit_row_off = cv.take<int32_t>(2);
     int32_t* step_in = (int32_t*)cv.take<char>(STEP_IN_BYTES);
     int32_t* step_out = cv.take<int32_t>(STEP_OUT_INTS);
+    int32_t* loop_state = cv.take<int32_t>(64);
     if (ctx) {
         ctx->h = h; ctx->y = y; ctx->logits = logits; ctx->x = x; ctx->q = q; ctx->act = act;
         ctx->x_lo = c.dtype == TRJ_BF16 ? x_lo : nullptr; ctx->act_lo = c.dtype == TRJ_BF16 ? act_lo : nullptr;
@@ -193,7 +198,7 @@ size_t carve(const trj_model_cfg& c, void* ws, trj_ctx* ctx) {
         ctx->gemm_ws = gemm_ws; ctx->gemm_ws_bytes = gemm_bytes;
         ctx->chain_depth = chain_depth; ctx->chain_anc = chain_anc;
         ctx->chunk_row_off = chunk_row_off; ctx->unit_row_off = unit_row_off;
-        ctx->step_in = step_in; ctx->step_out = step_out;
+        ctx->step_in = step_in; ctx->step_out = step_out; ctx->loop_state = loop_state;
     }
     return cv.off;
 }
@@ -236,6 +241,14 @@ void prof_end(trj_ctx* ctx, cudaStream_t st) {
         prof_begin(ctx, cat, st);          \
         cudaError_t le__ = (expr);         \
         prof_end(ctx, st);                 \
+        if (le__ != cudaSuccess) return fail(TRJ_ECUDA, "%s: %s", #expr, cudaGetErrorString(le__)); \
+    } while (0)
+
+#define LAUNCH_ON(stream_, cat, expr)      \
+    do {                                   \
+        prof_begin(ctx, cat, stream_);     \
+        cudaError_t le__ = (expr);         \
+        prof_end(ctx, stream_);            \
         if (le__ != cudaSuccess) return fail(TRJ_ECUDA, "%s: %s", #expr, cudaGetErrorString(le__)); \
     } while (0)
 
@@ -380,6 +393,7 @@ extern "C" trj_status trj_destroy(trj_ctx* ctx) {
     if (ctx->pin_out) cudaFreeHost(ctx->pin_out);
     for (cudaEvent_t e : ctx->prof_ev) cudaEventDestroy(e);
     for (const trj_ctx::GraphEntry& g : ctx->graphs) cudaGraphExecDestroy(g.exec);
+    for (const trj_ctx::LoopGraph& g : ctx->loop_graphs) cudaGraphExecDestroy(g.exec);
     if (ctx->cap_stream) cudaStreamDestroy(ctx->cap_stream);
     if (ctx->order_ev) cudaEventDestroy(ctx->order_ev);
     delete ctx;
@@ -579,5 +593,131 @@ extern "C" trj_status trj_step_host(trj_ctx* ctx, void* k_cache, void* v_cache, 
     *k_acc = ctx->pin_out[TRJ_MAX_ROWS];
     *bonus = ctx->pin_out[TRJ_MAX_ROWS + 1];
     std::memcpy(path, ctx->pin_out + TRJ_MAX_ROWS + 2, sizeof(int32_t) * TRJ_PATH_STRIDE);
+    return TRJ_OK;
+}
+
+
+// ---------------------------------------------------------------- device-resident drafting, commit and decode loop
+extern "C" trj_status trj_draft_tokens(const int32_t* context, const int32_t* n_ctx, const int32_t* window, int32_t W,
+                                       int32_t R, int32_t branch_len, const int64_t* draws, int32_t* tokens, void* stream) {
+    TRJ_REQUIRE(context && n_ctx && tokens, TRJ_EINVAL, "draft_tokens: null pointer");
+    TRJ_REQUIRE(W >= 0 && R >= 0 && branch_len >= 0, TRJ_EINVAL, "draft_tokens: negative size");
+    TRJ_REQUIRE(W == 0 || window, TRJ_EINVAL, "draft_tokens: null window");
+    TRJ_REQUIRE(R * branch_len == 0 || draws, TRJ_EINVAL, "draft_tokens: null draws");
+    TRJ_REQUIRE(R <= 64 && 1 + (int64_t)W + (int64_t)R * branch_len <= TRJ_MAX_ROWS, TRJ_ECAPACITY,
+                "draft_tokens: %d + %d x %d draft rows exceed the limits (64 branches, %d rows)", W, R, branch_len, TRJ_MAX_ROWS);
+    TRJ_CHECK_CUDA(launch_draft_tokens(context, n_ctx, window, W, R, branch_len, draws, nullptr, tokens, (cudaStream_t)stream));
+    return TRJ_OK;
+}
+
+extern "C" trj_status trj_commit_refill(const int32_t* tokens, const int32_t* parent, const int32_t* node_argmax, int32_t M,
+                                        const int32_t* k_acc, const int32_t* path, const int32_t* bonus, int32_t* context,
+                                        int32_t capacity, int32_t* n_ctx, int32_t W, const int64_t* draws, int32_t* window,
+                                        int32_t* overflow, void* stream) {
+    TRJ_REQUIRE(tokens && parent && node_argmax && k_acc && path && bonus && context && n_ctx, TRJ_EINVAL, "commit_refill: null pointer");
+    TRJ_REQUIRE(M >= 1 && M <= TRJ_MAX_ROWS, TRJ_ECAPACITY, "commit_refill: %d rows outside 1..%d", M, TRJ_MAX_ROWS);
+    TRJ_REQUIRE(W >= 0 && (W == 0 || (window && draws)), TRJ_EINVAL, "commit_refill: null window or draws");
+    TRJ_REQUIRE(capacity >= 1, TRJ_EINVAL, "commit_refill: empty context buffer");
+    TRJ_CHECK_CUDA(launch_commit_refill(tokens, parent, node_argmax, M, k_acc, path, bonus, context, capacity, n_ctx, W, W,
+                                        draws, nullptr, window, nullptr, overflow, (cudaStream_t)stream));
+    return TRJ_OK;
+}
+
+extern "C" trj_status trj_decode_device(trj_ctx* ctx, void* k_cache, void* v_cache, int32_t* seq_len, int32_t* context,
+                                        int32_t capacity, int32_t* n_ctx, int32_t n_ctx_now, int32_t* window, int32_t W,
+                                        int32_t R, int32_t branch_len, const int64_t* draws, int32_t n_steps,
+                                        int32_t* k_log, void* stream) {
+    TRJ_REQUIRE(ctx, TRJ_EINVAL, "decode_device: null context");
+    TRJ_REQUIRE(k_cache && v_cache && seq_len && context && n_ctx && draws, TRJ_EINVAL, "decode_device: null pointer");
+    TRJ_REQUIRE(W >= 0 && R >= 0 && branch_len >= 0 && n_steps >= 0 && (W == 0 || window), TRJ_EINVAL, "decode_device: bad sizes");
+    const trj_model_cfg& c = ctx->cfg;
+    const int64_t M64 = 1 + (int64_t)W + (int64_t)R * branch_len;
+    TRJ_REQUIRE(R <= 64 && M64 <= c.max_rows, TRJ_ECAPACITY, "decode_device: %lld tree rows exceed max_rows %d (or more than 64 branches)",
+                (long long)M64, c.max_rows);
+    const int32_t M = (int32_t)M64;
+    // a step commits at most depth + 1 tokens; the deepest node is the end of the window chain or of a branch
+    const int32_t per_step = std::max(W, branch_len) + 1;
+    TRJ_REQUIRE(n_ctx_now >= 1, TRJ_EINVAL, "decode_device: empty context");
+    TRJ_REQUIRE((int64_t)n_ctx_now + (int64_t)n_steps * per_step <= capacity, TRJ_ECAPACITY,
+                "decode_device: context buffer of %d cannot take %d steps of up to %d tokens after %d", capacity, n_steps, per_step, n_ctx_now);
+    // the cache holds every committed token but the last one (the next root) and, during a step, the tree rows
+    const int64_t max_len = (int64_t)n_ctx_now - 1 + (int64_t)n_steps * per_step + M;
+    TRJ_REQUIRE(max_len <= c.max_seq, TRJ_ECAPACITY, "decode_device: up to %lld cache rows exceed max_seq %d", (long long)max_len, c.max_seq);
+    trj_status s = check_step_args(ctx, 1, M, M, (int32_t)max_len, 2);
+    if (s != TRJ_OK) return s;
+    if (n_steps == 0) return TRJ_OK;
+    cudaStream_t st = (cudaStream_t)stream;
+    // the tree's shape is static: parents, depths, ancestor masks and row offsets go to the device once
+    int32_t* in = ctx->pin_in;
+    int32_t* h_tokens = in, *h_parent = in + TRJ_MAX_ROWS, *h_depth = in + 2 * TRJ_MAX_ROWS, *h_off = in + 3 * TRJ_MAX_ROWS;
+    uint64_t* h_anc = (uint64_t*)(in + STEP_IN_INTS);
+    {
+        std::vector<int32_t> zeros((size_t)std::max(W, R * branch_len) + 1, 0);
+        int32_t m_built = 0;
+        s = trj_build_tree(0, zeros.data(), W, zeros.data(), R, branch_len, c.max_rows, 2, h_tokens, h_parent, h_depth, h_anc, &m_built);
+        if (s != TRJ_OK) return s;
+    }
+    h_off[0] = 0; h_off[1] = M;
+    TRJ_CHECK_CUDA(cudaMemcpyAsync(ctx->step_in, ctx->pin_in, STEP_IN_BYTES, cudaMemcpyHostToDevice, st));
+    TRJ_CHECK_CUDA(cudaMemsetAsync(ctx->loop_state, 0, sizeof(int32_t) * 64, st));
+    // the pinned staging area is shared with trj_step_host: the copy must have left it before this call returns
+    TRJ_CHECK_CUDA(cudaEventRecord(ctx->order_ev, st));
+    TRJ_CHECK_CUDA(cudaEventSynchronize(ctx->order_ev));
+    int32_t* d_tokens = ctx->step_in, *d_parent = d_tokens + TRJ_MAX_ROWS, *d_depth = d_tokens + 2 * TRJ_MAX_ROWS;
+    int32_t* d_off = d_tokens + 3 * TRJ_MAX_ROWS;
+    uint64_t* d_anc = (uint64_t*)(d_tokens + STEP_IN_INTS);
+    int32_t* d_pred = ctx->step_out, *d_k = d_pred + TRJ_MAX_ROWS, *d_bonus = d_k + 1, *d_path = d_k + 2;
+    int32_t* d_step = ctx->loop_state, *d_overflow = ctx->loop_state + 1;
+    Batch bt{seq_len, d_off, 1, M, M, (int32_t)max_len};
+    auto enqueue_one = [&](cudaStream_t on) -> trj_status {
+        ChainScope chain;
+        LAUNCH_ON(on, PROF_ELEMENTWISE, launch_draft_tokens(context, n_ctx, window, W, R, branch_len, draws, d_step, d_tokens, on));
+        trj_status fs = forward(ctx, k_cache, v_cache, 0, bt, d_tokens, d_depth, d_anc, 2, 0, M, on);
+        if (fs != TRJ_OK) return fs;
+        LAUNCH_ON(on, PROF_ARGMAX, launch_argmax_accept(ctx->logits, TRJ_F32, c.vocab, d_tokens, d_parent, d_depth, d_off, 1, M, d_pred,
+                                                        nullptr, d_k, d_path, d_bonus, true, true, ctx->argmax_ws, on));
+        LAUNCH_ON(on, PROF_COMPACT, launch_compact(k_cache, v_cache, c.n_layers, c.max_batch, 1, c.n_heads, c.max_seq, c.head_dim,
+                                                   c.dtype, seq_len, d_k, d_path, on));
+        LAUNCH_ON(on, PROF_ELEMENTWISE, launch_commit_refill(d_tokens, d_parent, d_pred, M, d_k, d_path, d_bonus, context, capacity,
+                                                             n_ctx, W, W + R * branch_len, draws, d_step, window, k_log, d_overflow, on));
+        return TRJ_OK;
+    };
+    int32_t done = 0;
+    // The first step a context ever runs is enqueued plainly (one-time set-up of the kernels happens outside any
+    // capture); so is everything while profiling or without a capture stream.  Otherwise one step is captured once
+    // per key and the graph is launched once per step: the device step counter makes the steps differ.
+    const bool plain = ctx->prof_on || !ctx->cap_stream;
+    if (ctx->steps_done == 0 || plain) {
+        const int32_t n_plain = plain ? n_steps : 1;
+        for (; done < n_plain; ++done) {
+            s = enqueue_one(st);
+            if (s != TRJ_OK) return s;
+        }
+    }
+    if (done < n_steps) {
+        const std::vector<uint64_t> key = {(uint64_t)M, (uint64_t)tree_attention_grid(1, c.n_heads, (int32_t)max_len),
+                                           (uint64_t)(uintptr_t)k_cache, (uint64_t)(uintptr_t)v_cache, (uint64_t)(uintptr_t)seq_len,
+                                           (uint64_t)(uintptr_t)context, (uint64_t)capacity, (uint64_t)(uintptr_t)n_ctx,
+                                           (uint64_t)(uintptr_t)window, (uint64_t)W, (uint64_t)R, (uint64_t)branch_len,
+                                           (uint64_t)(uintptr_t)draws, (uint64_t)(uintptr_t)k_log, (uint64_t)max_len};
+        cudaGraphExec_t exec = nullptr;
+        for (const trj_ctx::LoopGraph& g : ctx->loop_graphs)
+            if (g.key == key) exec = g.exec;
+        if (!exec) {
+            cudaGraph_t graph = nullptr;
+            TRJ_CHECK_CUDA(cudaStreamBeginCapture(ctx->cap_stream, cudaStreamCaptureModeThreadLocal));
+            s = enqueue_one(ctx->cap_stream);
+            cudaError_t e = cudaStreamEndCapture(ctx->cap_stream, &graph);
+            if (s != TRJ_OK) { if (graph) cudaGraphDestroy(graph); return s; }
+            if (e != cudaSuccess) return fail(TRJ_ECUDA, "decode_device: graph capture: %s", cudaGetErrorString(e));
+            e = cudaGraphInstantiate(&exec, graph, 0);
+            cudaGraphDestroy(graph);
+            if (e != cudaSuccess) return fail(TRJ_ECUDA, "decode_device: graph instantiate: %s", cudaGetErrorString(e));
+            if (ctx->loop_graphs.size() >= 8) { cudaGraphExecDestroy(ctx->loop_graphs.front().exec); ctx->loop_graphs.erase(ctx->loop_graphs.begin()); }
+            ctx->loop_graphs.push_back({key, exec});
+        }
+        for (; done < n_steps; ++done) TRJ_CHECK_CUDA(cudaGraphLaunch(exec, st));
+    }
+    ctx->steps_done += n_steps;
     return TRJ_OK;
 }

@@ -1,0 +1,118 @@
+// Device-side drafting and refill: the integer bookkeeping between two verification steps (prompt-lookup
+// retrieval, tree tokens, commit of the accepted tokens, next Jacobi window), so that a decode loop needs no
+// host round trip per step.  Each kernel is one warp; the work is a few hundred integer operations.
+// Semantics are those of the host functions trj_retrieve / trj_build_tree / trj_refill_window (Section 3.3:
+// retrieval from the tokens seen so far, refill from the chosen path's own predictions; Eq. 4: ahead noise).
+#include <cstdint>
+#include "trj_internal.h"
+
+namespace trj {
+namespace {
+
+constexpr int MAX_BRANCHES = 64;          // R is bounded by the tree size (R * Lr < TRJ_MAX_ROWS)
+
+// tokens[0] = root (last committed token), tokens[1..W] = window, then R branches of Lr tokens: for each of the R
+// most recent earlier occurrences of the context's last two tokens (then of its last token), the Lr tokens that
+// followed; missing slots are ahead noise, context[draw % n].  `step` (may be null) selects this step's draws.
+__global__ void __launch_bounds__(32) draft_tokens_kernel(const int32_t* __restrict__ context, const int32_t* __restrict__ n_ctx,
+                                                          const int32_t* __restrict__ window, int W, int R, int Lr,
+                                                          const int64_t* __restrict__ draws, const int32_t* __restrict__ step,
+                                                          int32_t* __restrict__ tokens) {
+    pdl_prologue();
+    const int lane = threadIdx.x;
+    const int n = *n_ctx;
+    const int64_t* my_draws = draws + (step ? (size_t)*step * (size_t)(W + R * Lr) : 0);
+    if (lane == 0) tokens[0] = context[n - 1];
+    for (int i = lane; i < W; i += 32) tokens[1 + i] = window[i];
+    // every lane keeps the same list of follow positions (first index after a match), most recent match first
+    int follow[MAX_BRANCHES];
+    int nf = 0;
+    for (int g = 2; g >= 1 && nf < R; --g) {
+        if (n <= g) continue;
+        const int t0 = context[n - g], t1 = context[n - 1];          // g == 1: t0 == t1
+        for (int base = n - g - 1; base >= 0 && nf < R; base -= 32) {
+            const int p = base - lane;
+            bool match = false;
+            if (p >= 0) match = context[p] == t0 && (g == 1 || context[p + 1] == t1);
+            unsigned m = __ballot_sync(0xffffffffu, match);
+            while (m && nf < R) {                            // lane 0 holds the largest p: ascending lanes = descending p
+                const int l = __ffs(m) - 1;
+                m &= m - 1;
+                const int f = base - l + g;
+                bool seen = false;
+                for (int i = 0; i < nf; ++i) seen |= follow[i] == f;
+                if (!seen) follow[nf++] = f;
+            }
+        }
+    }
+    for (int slot = lane; slot < R * Lr; slot += 32) {
+        const int r = slot / Lr, j = slot % Lr;
+        int32_t tok;
+        if (r < nf && follow[r] + j < n) tok = context[follow[r] + j];
+        else tok = context[(uint64_t)my_draws[W + slot] % (uint64_t)n];
+        tokens[1 + W + slot] = tok;
+    }
+}
+
+// Appends the accepted draft tokens and the bonus token to the context, refills the window from the predictions
+// below the winning node (lowest-index child at every level, then ahead noise on the grown context), and advances
+// the step counter.  A context that would overflow `capacity` is left untouched and flagged in *overflow.
+__global__ void __launch_bounds__(32) commit_refill_kernel(const int32_t* __restrict__ tokens, const int32_t* __restrict__ parent,
+                                                           const int32_t* __restrict__ node_argmax, int M,
+                                                           const int32_t* __restrict__ k_acc, const int32_t* __restrict__ path,
+                                                           const int32_t* __restrict__ bonus, int32_t* __restrict__ context,
+                                                           int capacity, int32_t* __restrict__ n_ctx, int W, int draws_per_step,
+                                                           const int64_t* __restrict__ draws, int32_t* __restrict__ step,
+                                                           int32_t* __restrict__ window, int32_t* __restrict__ k_log,
+                                                           int32_t* __restrict__ overflow) {
+    pdl_prologue();
+    const int lane = threadIdx.x;
+    const int n = *n_ctx, k = *k_acc;
+    const int s = step ? *step : 0;
+    const int64_t* my_draws = draws + (size_t)s * (size_t)draws_per_step;
+    if (n + k + 1 > capacity) {
+        if (lane == 0 && overflow) *overflow = 1;
+        return;
+    }
+    for (int j = lane; j < k; j += 32) context[n + j] = tokens[path[j + 1]];
+    if (lane == 0) context[n + k] = *bonus;
+    __syncwarp();
+    if (lane == 0) {
+        const int n_new = n + k + 1;
+        int filled = 0, cur = path[k];
+        while (filled < W) {
+            int child = -1;
+            for (int c = cur + 1; c < M; ++c)
+                if (parent[c] == cur) { child = c; break; }
+            if (child < 0) break;
+            window[filled++] = node_argmax[child];
+            cur = child;
+        }
+        for (; filled < W; ++filled) window[filled] = context[(uint64_t)my_draws[filled] % (uint64_t)n_new];
+        *n_ctx = n_new;
+        if (k_log) k_log[s] = k;
+        if (step) *step = s + 1;
+    }
+}
+
+}  // namespace
+
+cudaError_t launch_draft_tokens(const int32_t* context, const int32_t* n_ctx, const int32_t* window, int32_t W, int32_t R,
+                                int32_t Lr, const int64_t* draws, const int32_t* step, int32_t* tokens, cudaStream_t st) {
+    if (R > MAX_BRANCHES) return cudaErrorInvalidValue;
+    count_launch();
+    cudaError_t e = launch_chain(draft_tokens_kernel, dim3(1), dim3(32), 0, st, context, n_ctx, window, W, R, Lr, draws, step, tokens);
+    return e != cudaSuccess ? e : cudaGetLastError();
+}
+
+cudaError_t launch_commit_refill(const int32_t* tokens, const int32_t* parent, const int32_t* node_argmax, int32_t M,
+                                 const int32_t* k_acc, const int32_t* path, const int32_t* bonus, int32_t* context,
+                                 int32_t capacity, int32_t* n_ctx, int32_t W, int32_t draws_per_step, const int64_t* draws,
+                                 int32_t* step, int32_t* window, int32_t* k_log, int32_t* overflow, cudaStream_t st) {
+    count_launch();
+    cudaError_t e = launch_chain(commit_refill_kernel, dim3(1), dim3(32), 0, st, tokens, parent, node_argmax, M, k_acc, path, bonus,
+                                 context, capacity, n_ctx, W, draws_per_step, draws, step, window, k_log, overflow);
+    return e != cudaSuccess ? e : cudaGetLastError();
+}
+
+}  // namespace trj

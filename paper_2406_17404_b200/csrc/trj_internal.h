@@ -136,6 +136,15 @@ cudaError_t launch_tree_attention(const void* q, const void* k_slab, const void*
                                   int32_t dtype, void* out, void* out_lo, void* workspace, size_t workspace_bytes,
                                   cudaStream_t st);
 
+// Device-side drafting and refill (device_loop.cu); all pointers are device pointers.  `step` (may be null: step 0)
+// is a device counter that selects the step's slice of `draws` ([steps][W + R * Lr]) and is advanced by the commit.
+cudaError_t launch_draft_tokens(const int32_t* context, const int32_t* n_ctx, const int32_t* window, int32_t W, int32_t R,
+                                int32_t Lr, const int64_t* draws, const int32_t* step, int32_t* tokens, cudaStream_t st);
+cudaError_t launch_commit_refill(const int32_t* tokens, const int32_t* parent, const int32_t* node_argmax, int32_t M,
+                                 const int32_t* k_acc, const int32_t* path, const int32_t* bonus, int32_t* context,
+                                 int32_t capacity, int32_t* n_ctx, int32_t W, int32_t draws_per_step, const int64_t* draws,
+                                 int32_t* step, int32_t* window, int32_t* k_log, int32_t* overflow, cudaStream_t st);
+
 // act[M][f] (dtype) = silu(gu[:, :f]) * gu[:, f:]
 cudaError_t launch_swiglu(const Parts& gu, void* act, void* act_lo, int32_t dtype, int32_t rows, int32_t f,
                           cudaStream_t st);

@@ -112,6 +112,14 @@ def test_device_entry_points_reject_bad_arguments_before_any_launch(trj):
     assert lib.trj_tree_attention(fake, fake, fake, fake, fake, fake, 1, 1, 1, 8, 1, 128, 16, 32, 1, fake, fake, 256, nul) == 2
     assert lib.trj_tree_attention(fake, fake, fake, fake, fake, fake, 1, 1, 1, 8, 1, 128, 16, 16, 7, fake, fake, 256, nul) == 1
     assert lib.trj_argmax_accept(fake, 1, 10, fake, fake, fake, fake, 100, 100, fake, nul, fake, fake, fake, fake, 1 << 20, nul) == 2
+    # device-side drafting / commit / decode loop: pointers and sizes are checked before anything is launched
+    assert lib.trj_draft_tokens(nul, nul, nul, 4, 2, 3, nul, nul, nul) == 1
+    assert lib.trj_draft_tokens(fake, fake, fake, 4, 65, 1, fake, fake, nul) == 2          # more than 64 branches
+    assert lib.trj_draft_tokens(fake, fake, fake, 100, 10, 3, fake, fake, nul) == 2        # 131 rows
+    assert lib.trj_draft_tokens(fake, fake, nul, 4, 2, 3, fake, fake, nul) == 1            # window missing
+    assert lib.trj_commit_refill(nul, nul, nul, 4, nul, nul, nul, nul, 10, nul, 2, nul, nul, nul, nul) == 1
+    assert lib.trj_commit_refill(fake, fake, fake, 500, fake, fake, fake, fake, 10, fake, 2, fake, fake, nul, nul) == 2
+    assert lib.trj_decode_device(nul, fake, fake, fake, fake, 10, fake, 1, fake, 4, 2, 3, fake, 1, nul, nul) == 1
     cfg = trj.ModelCfg(2, 256, 4, 48, 688, 1024, 1e-5, 1e4, 0, 1, 256, 16)
     assert lib.trj_workspace_bytes(ctypes.byref(cfg)) == 0
     cfg = trj.ModelCfg(2, 256, 4, 64, 688, 1024, 1e-5, 1e4, 0, 1, 256, 300)
