@@ -305,8 +305,11 @@ __device__ __forceinline__ void build_sched(Sched& s, const AtParams& p) {
 __device__ __forceinline__ void build_range(Sched& s, const AtParams& p) {
     if (p.cluster > 1) {
         const int head = blockIdx.x / p.cluster, rank = blockIdx.x % p.cluster, T = s.tiles[0];
-        s.u_begin = head * T + T * rank / p.cluster;
-        s.u_end = head * T + T * (rank + 1) / p.cluster;
+        // shares rounded so that the extra tiles go to the FIRST CTAs: their tiles are cached rows that are already
+        // on their way when the previous kernel ends, while the last CTA has the tile with this step's rows, the
+        // masks and the padding to deal with
+        s.u_begin = head * T + (T * rank + p.cluster - 1) / p.cluster;
+        s.u_end = head * T + (T * (rank + 1) + p.cluster - 1) / p.cluster;
     } else {
         const long long U = s.first[p.B];
         s.u_begin = (int)(U * blockIdx.x / gridDim.x);
