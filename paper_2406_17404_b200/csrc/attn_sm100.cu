@@ -6,7 +6,7 @@
 //   * one thread streams Q (per segment) and the K/V tiles with TMA into 128-byte-swizzled shared memory;
 //   * one thread issues tcgen05.mma: S = Q.K^T into TMEM (two S buffers), then O += P.V with P read from
 //     TMEM as well (two P buffers) and the accumulator resident in TMEM for the whole segment;
-//   * eight warps do the softmax: a thread owns half of one query row (TMEM lane = row, 64 of the 128
+//   * eight (or sixteen) warps do the softmax: a thread owns half (a quarter) of one query row (TMEM lane = row, 64 of the 128
 //     columns); they read S once into registers, apply the ancestor bitmask on tiles that reach the tree
 //     rows, keep an online softmax whose running maximum is only raised when a tile exceeds it by more
 //     than 2^8 (then O is rescaled in TMEM), and store P as bf16 pairs back into TMEM, where the second
@@ -24,7 +24,10 @@ namespace {
 constexpr int AT_ROWS = 128;                 // query rows per CTA = UMMA M = TMEM lanes
 constexpr int AT_KEYS = 128;                 // keys per tile
 constexpr int AT_D = 128;                    // head_dim
-constexpr int AT_THREADS = 320;              // 8 softmax warps + TMA warp + MMA warp
+// The softmax is done by 4 * SPLIT warps: SPLIT threads share a query row, each taking a column group of a tile
+// (template parameter of the kernel: 2 for one sequence with full row groups, 4 for batches of small trees, where
+// half of the row groups are empty and more threads per row pay off).
+__host__ __device__ constexpr int at_threads(int split) { return 32 * 4 * split + 64; }   // softmax warps + TMA warp + MMA warp
 constexpr uint32_t AT_SUB = 128 * 128;       // one [128 x 64 bf16] swizzled sub-tile: 16 KB
 constexpr uint32_t AT_TILE = 2 * AT_SUB;     // Q, P, a K tile or a V tile: 32 KB
 constexpr int AT_RING = 5;                   // K/V ring slots; load n = 2g + (0: K, 1: V) of tile g goes to slot n % 5
@@ -204,6 +207,14 @@ __device__ __forceinline__ void tmem_st32u(uint32_t taddr, const uint32_t* v) {
                  : "memory");
     asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
 }
+__device__ __forceinline__ void tmem_st16u(uint32_t taddr, const uint32_t* v) {
+    asm volatile("tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], "
+                 "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16};"
+                 ::"r"(taddr), "r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3]), "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7]),
+                   "r"(v[8]), "r"(v[9]), "r"(v[10]), "r"(v[11]), "r"(v[12]), "r"(v[13]), "r"(v[14]), "r"(v[15])
+                 : "memory");
+    asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
+}
 __device__ __forceinline__ uint32_t pack_bf16(float a, float b) {
     const __nv_bfloat162 h = __floats2bfloat162_rn(a, b);      // .x (low half) = a
     return *reinterpret_cast<const uint32_t*>(&h);
@@ -317,16 +328,23 @@ __device__ __forceinline__ void build_range(Sched& s, const AtParams& p) {
     }
 }
 
-__global__ void __launch_bounds__(AT_THREADS, 1) tree_attention_tc_kernel(const __grid_constant__ CUtensorMap map_q,
+template <int AT_SPLIT>
+__global__ void __launch_bounds__(at_threads(AT_SPLIT), 1) tree_attention_tc_kernel(const __grid_constant__ CUtensorMap map_q,
                                                                           const __grid_constant__ CUtensorMap map_k,
                                                                           const __grid_constant__ CUtensorMap map_v,
                                                                           const AtParams p) {
+    constexpr int AT_KPT = 128 / AT_SPLIT;        // keys of a tile, and head_dim columns of O, per thread
+    constexpr int AT_SM_WARPS = 4 * AT_SPLIT;     // warp w owns TMEM lanes 32*(w%4).. and column group w/4
+    constexpr int AT_SM_THREADS = 32 * AT_SM_WARPS;
+    constexpr int AT_W_COPY = AT_SM_WARPS, AT_W_MMA = AT_SM_WARPS + 1;
+    constexpr int AT_THREADS = at_threads(AT_SPLIT);
+    static_assert(AT_KPT == 32 || AT_KPT == 64, "column groups are read with 32- or 64-column tensor-memory loads");
     extern __shared__ uint8_t smem_raw[];
     __shared__ __align__(8) uint64_t bars[B_COUNT];
     __shared__ uint32_t tmem_base_slot;
     __shared__ int abort_flag;
     __shared__ Sched sched;
-    __shared__ float pair_max[2][2][AT_ROWS], pair_sum[2][2][AT_ROWS];      // [parity][half][row]
+    __shared__ float pair_max[2][AT_SPLIT][AT_ROWS], pair_sum[2][AT_SPLIT][AT_ROWS];      // [parity][column group][row]
     __shared__ float piece_m[AT_ROWS], piece_l[AT_ROWS];                     // this CTA's piece of a head shared by a cluster
 
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -344,10 +362,11 @@ __global__ void __launch_bounds__(AT_THREADS, 1) tree_attention_tc_kernel(const 
     }
     if (threadIdx.x == 0) {
         abort_flag = 0;
-        for (int i = 0; i < B_COUNT; ++i) mbar_init(bar(i), (i == B_P_READY || i == B_P_READY + 1 || i == B_O_FREE) ? 256 : 1);
+        for (int i = 0; i < B_COUNT; ++i)
+            mbar_init(bar(i), (i == B_P_READY || i == B_P_READY + 1 || i == B_O_FREE) ? AT_SM_THREADS : 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
-    if (warp == 9) {
+    if (warp == AT_W_MMA) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
                      ::"r"(smem_u32(&tmem_base_slot)), "r"(512u) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
@@ -370,7 +389,7 @@ __global__ void __launch_bounds__(AT_THREADS, 1) tree_attention_tc_kernel(const 
     // merges a slice of head_dim from all pieces.
     float* piece_o = reinterpret_cast<float*>(base_ptr + AT_TILE);          // [row][AT_PIECE_STRIDE], over the K/V ring once it is idle
 
-    if (warp == 8) {
+    if (warp == AT_W_COPY) {
         if (lane == 0) {
             // ------------------------------------------------ TMA producer
             int g = 0, e = 0;
@@ -415,7 +434,7 @@ __global__ void __launch_bounds__(AT_THREADS, 1) tree_attention_tc_kernel(const 
             }
             if (!waited) pdl_wait();
         }
-    } else if (warp == 9) {
+    } else if (warp == AT_W_MMA) {
         if (lane == 0) {
             // ------------------------------------------------ MMA issuer
             // S = Q.K^T: both K-major from shared memory, 128 x 128.  O += P.V: P from TMEM, V MN-major, 128 x 128.
@@ -473,13 +492,13 @@ __global__ void __launch_bounds__(AT_THREADS, 1) tree_attention_tc_kernel(const 
         }
     } else {
         // ------------------------------------------------ softmax + epilogue
-        // Eight warps: warp w owns rows 32*(w%4) .. +31 (its TMEM lanes) and key / head_dim columns
-        // 64*(w/4) .. +63, so two threads share a row and exchange their maxima and sums through shared memory.
-        const int rg = warp & 3, half = warp >> 2;
+        // Warp w owns rows 32*(w%4) .. +31 (its TMEM lanes) and key / head_dim columns AT_KPT*(w/4) .. +AT_KPT-1, so
+        // AT_SPLIT threads share a row and exchange their maxima and sums through shared memory.
+        const int rg = warp & 3, part = warp >> 2;
         const int row = rg * 32 + lane;
         const uint32_t lane_addr = (uint32_t)(rg * 32) << 16;
-        const uint32_t col0 = (uint32_t)half * 64;
-        const uint32_t pair_bar = 1 + rg;                    // named barrier of the two warps of a row group
+        const uint32_t col0 = (uint32_t)part * AT_KPT;
+        const uint32_t pair_bar = 1 + rg;                    // named barrier of the warps of a row group
         int g = 0, e = 0;
         bool ok = true;
         for (int u = u_begin; u < u_end && ok;) {
@@ -500,35 +519,38 @@ __global__ void __launch_bounds__(AT_THREADS, 1) tree_attention_tc_kernel(const 
             for (g = g0; g < g1 && ok; ++g) {
                 const int key0 = (w.t + (g - g0)) * AT_KEYS;
                 const bool edge = key0 + AT_KEYS > w.S;      // the tile reaches tree rows or the end of the keys
-                float s[64];
+                float s[AT_KPT];
                 float mt = -INFINITY;
                 if (group_live) {
                     ok = __all_sync(0xffffffffu, mbar_wait(bar(B_S_FULL + (g & 1)), (uint32_t)(g >> 1) & 1u, &abort_flag, p.status));
                     if (!ok) break;
                     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-                    tmem_ld64(tmem_s[g & 1] + lane_addr + col0, s);
+                    if constexpr (AT_KPT == 64) tmem_ld64(tmem_s[g & 1] + lane_addr + col0, s);
+                    else tmem_ld32(tmem_s[g & 1] + lane_addr + col0, s);
                     if (edge) {
                         // bit c of (vis0, vis1) = visibility of key key0 + c for this row: tree row tt = key0 + c - S
                         // is visible if tt < 0 (prefix) or if bit tt of the row's ancestor mask is set
                         uint64_t vis0 = m0, vis1 = m1;
                         const int d = key0 - w.S;            // -127 .. 127 on an edge tile
                         if (d >= 0) shr128(vis0, vis1, d); else shl128_fill(vis0, vis1, -d);
-                        const uint64_t vis = half ? vis1 : vis0;
+                        const uint64_t vis = (col0 < 64 ? vis0 : vis1) >> (col0 & 63u);      // this thread's AT_KPT keys
 #pragma unroll
-                        for (int i = 0; i < 64; ++i) if (!((vis >> i) & 1ull)) s[i] = -INFINITY;
+                        for (int i = 0; i < AT_KPT; ++i) if (!((vis >> i) & 1ull)) s[i] = -INFINITY;
                     }
                     {   // four independent chains instead of one 64-long dependency chain
                         float mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
 #pragma unroll
-                        for (int i = 0; i < 64; i += 4) {
+                        for (int i = 0; i < AT_KPT; i += 4) {
                             mx[0] = fmaxf(mx[0], s[i]); mx[1] = fmaxf(mx[1], s[i + 1]);
                             mx[2] = fmaxf(mx[2], s[i + 2]); mx[3] = fmaxf(mx[3], s[i + 3]);
                         }
                         mt = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3]));
                     }
-                    pair_max[g & 1][half][row] = mt;
-                    asm volatile("bar.sync %0, 64;" ::"r"(pair_bar) : "memory");
-                    mt = fmaxf(mt, pair_max[g & 1][half ^ 1][row]) * p.scale_log2;
+                    pair_max[g & 1][part][row] = mt;
+                    asm volatile("bar.sync %0, %1;" ::"r"(pair_bar), "n"(32 * AT_SPLIT) : "memory");
+#pragma unroll
+                    for (int q = 0; q < AT_SPLIT; ++q) mt = fmaxf(mt, pair_max[g & 1][q][row]);
+                    mt *= p.scale_log2;
                 }
                 // this tile's P buffer was last read by the P.V product of two tiles ago
                 if (g > 1) ok = __all_sync(0xffffffffu, mbar_wait(bar(B_P_FREE + (g & 1)), ((uint32_t)(g >> 1) & 1u) ^ 1u, &abort_flag, p.status));
@@ -547,7 +569,7 @@ __global__ void __launch_bounds__(AT_THREADS, 1) tree_attention_tc_kernel(const 
                         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                         l_sum *= factor;
 #pragma unroll 1
-                        for (int c0 = 0; c0 < 64; c0 += 32) {
+                        for (int c0 = 0; c0 < AT_KPT; c0 += 32) {
                             float o[32];
                             tmem_ld32(tmem_o + lane_addr + col0 + c0, o);
 #pragma unroll
@@ -558,11 +580,11 @@ __global__ void __launch_bounds__(AT_THREADS, 1) tree_attention_tc_kernel(const 
                     // P = 2^(s * c - m_ref) as bf16 pairs into this tile's P buffer in TMEM (lane = row, one column
                     // per two keys); masked scores are -inf and give exactly 0.  Rows past the tree store zeros.
                     const float m_use = (m_ref == -INFINITY) ? 0.f : m_ref;
-                    uint32_t packed[32];
+                    uint32_t packed[AT_KPT / 2];
                     if (live) {
                         float ls[4] = {0.f, 0.f, 0.f, 0.f};  // independent partial sums
 #pragma unroll
-                        for (int i = 0; i < 64; i += 4) {
+                        for (int i = 0; i < AT_KPT; i += 4) {
                             const float a = fast_exp2(fmaf(s[i], p.scale_log2, -m_use));
                             const float b = fast_exp2(fmaf(s[i + 1], p.scale_log2, -m_use));
                             const float c = fast_exp2(fmaf(s[i + 2], p.scale_log2, -m_use));
@@ -574,9 +596,10 @@ __global__ void __launch_bounds__(AT_THREADS, 1) tree_attention_tc_kernel(const 
                         l_sum += (ls[0] + ls[1]) + (ls[2] + ls[3]);
                     } else {
 #pragma unroll
-                        for (int i = 0; i < 32; ++i) packed[i] = 0u;
+                        for (int i = 0; i < AT_KPT / 2; ++i) packed[i] = 0u;
                     }
-                    tmem_st32u(tmem_p[g & 1] + lane_addr + 32 * half, packed);
+                    if constexpr (AT_KPT == 64) tmem_st32u(tmem_p[g & 1] + lane_addr + (AT_KPT / 2) * part, packed);
+                    else tmem_st16u(tmem_p[g & 1] + lane_addr + (AT_KPT / 2) * part, packed);
                 }
                 // keys past the end of the sequence hold whatever the cache holds: clear those V rows so
                 // that 0 * garbage cannot poison the product
@@ -586,7 +609,7 @@ __global__ void __launch_bounds__(AT_THREADS, 1) tree_attention_tc_kernel(const 
                     if (!ok) break;
                     uint8_t* v_ptr = base_ptr + AT_TILE + slot * AT_TILE;
                     const int first_bad = max(total - key0, 0);
-                    for (int i = first_bad * 8 + (int)threadIdx.x; i < AT_KEYS * 8; i += 256) {      // 16-byte chunks, both sub-tiles
+                    for (int i = first_bad * 8 + (int)threadIdx.x; i < AT_KEYS * 8; i += AT_SM_THREADS) {      // 16-byte chunks, both sub-tiles
                         *reinterpret_cast<uint4*>(v_ptr + i * 16) = make_uint4(0, 0, 0, 0);
                         *reinterpret_cast<uint4*>(v_ptr + AT_SUB + i * 16) = make_uint4(0, 0, 0, 0);
                     }
@@ -601,14 +624,16 @@ __global__ void __launch_bounds__(AT_THREADS, 1) tree_attention_tc_kernel(const 
             if (!ok) break;
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
             if (group_live) {
-                pair_sum[e & 1][half][row] = l_sum;
-                asm volatile("bar.sync %0, 64;" ::"r"(pair_bar) : "memory");
-                const float l_row = l_sum + pair_sum[e & 1][half ^ 1][row];
+                pair_sum[e & 1][part][row] = l_sum;
+                asm volatile("bar.sync %0, %1;" ::"r"(pair_bar), "n"(32 * AT_SPLIT) : "memory");
+                float l_row = 0.f;
+#pragma unroll
+                for (int q = 0; q < AT_SPLIT; ++q) l_row += pair_sum[e & 1][q][row];     // the same order in every thread
                 const bool whole_seg = (w.t == 0 && n_tiles == w.tiles);
                 if (p.cluster > 1) {
                     // all products that read the ring have finished (B_O_READY), and this CTA loads nothing more
 #pragma unroll 1
-                    for (int c0 = 0; c0 < 64; c0 += 32) {
+                    for (int c0 = 0; c0 < AT_KPT; c0 += 32) {
                         float o[32];
                         tmem_ld32(tmem_o + lane_addr + col0 + c0, o);
                         if (live) {
@@ -617,12 +642,12 @@ __global__ void __launch_bounds__(AT_THREADS, 1) tree_attention_tc_kernel(const 
                             for (int i = 0; i < 8; ++i) dst[i] = make_float4(o[4 * i], o[4 * i + 1], o[4 * i + 2], o[4 * i + 3]);
                         }
                     }
-                    if (live && half == 0) { piece_m[row] = m_ref; piece_l[row] = l_row; }
+                    if (live && part == 0) { piece_m[row] = m_ref; piece_l[row] = l_row; }
                 } else if (whole_seg) {
                     const float inv = live ? 1.f / l_row : 0.f;
                     const size_t off = ((size_t)grow * p.H + w.h) * AT_D + col0;
 #pragma unroll 1
-                    for (int c0 = 0; c0 < 64; c0 += 32) {
+                    for (int c0 = 0; c0 < AT_KPT; c0 += 32) {
                         float o[32];
                         tmem_ld32(tmem_o + lane_addr + col0 + c0, o);
                         if (live) {
@@ -636,7 +661,7 @@ __global__ void __launch_bounds__(AT_THREADS, 1) tree_attention_tc_kernel(const 
                 } else {
                     float* slot = p.slots + (size_t)(w.bh + (int)blockIdx.x) * AT_SLOT_FLOATS;
 #pragma unroll 1
-                    for (int c0 = 0; c0 < 64; c0 += 32) {
+                    for (int c0 = 0; c0 < AT_KPT; c0 += 32) {
                         float o[32];
                         tmem_ld32(tmem_o + lane_addr + col0 + c0, o);
                         if (live) {
@@ -644,7 +669,7 @@ __global__ void __launch_bounds__(AT_THREADS, 1) tree_attention_tc_kernel(const 
                             for (int i = 0; i < 32; ++i) slot[(size_t)(col0 + c0 + i) * AT_ROWS + row] = o[i];
                         }
                     }
-                    if (live && half == 0) { slot[AT_D * AT_ROWS + row] = m_ref; slot[AT_D * AT_ROWS + AT_ROWS + row] = l_row; }
+                    if (live && part == 0) { slot[AT_D * AT_ROWS + row] = m_ref; slot[AT_D * AT_ROWS + AT_ROWS + row] = l_row; }
                 }
             }
             asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
@@ -700,7 +725,7 @@ __global__ void __launch_bounds__(AT_THREADS, 1) tree_attention_tc_kernel(const 
         }
         cluster_sync_all();                                  // nobody leaves while its piece may still be read
     }
-    if (warp == 9)
+    if (warp == AT_W_MMA)
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(512u) : "memory");
 }
 
@@ -799,17 +824,17 @@ int at_cluster_size(int H) {
     std::lock_guard<std::mutex> lock(mu);
     if (cached_h == H) return cached_c;
     int pick = 1;
-    if (cudaFuncSetAttribute(tree_attention_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)AT_SMEM) == cudaSuccess) {
+    if (cudaFuncSetAttribute(tree_attention_tc_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)AT_SMEM) == cudaSuccess) {
         for (int c = 4; c >= 2 && pick == 1; c /= 2) {
             if (H * c > AT_MAX_GRID) continue;
             cudaLaunchConfig_t cfg = {};
-            cfg.gridDim = dim3(H * c); cfg.blockDim = dim3(AT_THREADS); cfg.dynamicSmemBytes = AT_SMEM;
+            cfg.gridDim = dim3(H * c); cfg.blockDim = dim3(at_threads(2)); cfg.dynamicSmemBytes = AT_SMEM;
             cudaLaunchAttribute attr[1];
             attr[0].id = cudaLaunchAttributeClusterDimension;
             attr[0].val.clusterDim.x = c; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
             cfg.attrs = attr; cfg.numAttrs = 1;
             int n = 0;
-            if (cudaOccupancyMaxActiveClusters(&n, tree_attention_tc_kernel, &cfg) == cudaSuccess && n >= H) pick = c;
+            if (cudaOccupancyMaxActiveClusters(&n, tree_attention_tc_kernel<2>, &cfg) == cudaSuccess && n >= H) pick = c;
         }
     }
     (void)cudaGetLastError();                                // a refused query is not an error of the caller
@@ -818,7 +843,7 @@ int at_cluster_size(int H) {
 }
 
 // Launch shape.  The host only knows an upper bound of the key count; CTAs whose range turns out empty do no work.
-struct AtPlan { int grid, cluster; bool merge_kernel; };
+struct AtPlan { int grid, cluster; bool merge_kernel; int split; };   // split: threads per query row in the softmax
 AtPlan at_plan(int32_t B, int32_t H, int32_t max_len) {
     const int tiles_bound = (max_len + AT_KEYS - 1) / AT_KEYS;
     const long long units_bound = (long long)B * H * tiles_bound;
@@ -827,9 +852,10 @@ AtPlan at_plan(int32_t B, int32_t H, int32_t max_len) {
     // Where clusters do not fit, one CTA takes a whole head of up to AT_WHOLE_HEAD_TILES tiles.
     if (B == 1 && H <= AT_MAX_GRID) {
         const int c = tiles_bound >= 2 ? at_cluster_size(H) : 1;
-        if (c > 1 || tiles_bound <= AT_WHOLE_HEAD_TILES) return AtPlan{H * c, c, false};
+        if (c > 1 || tiles_bound <= AT_WHOLE_HEAD_TILES) return AtPlan{H * c, c, false, 2};
     }
-    return AtPlan{(int)(units_bound < AT_MAX_GRID ? units_bound : AT_MAX_GRID), 1, true};
+    // contiguous ranges + merge kernel; batches of small trees leave row groups empty, so four threads share a row
+    return AtPlan{(int)(units_bound < AT_MAX_GRID ? units_bound : AT_MAX_GRID), 1, true, B > 1 ? 4 : 2};
 }
 
 }  // namespace
@@ -852,7 +878,9 @@ cudaError_t launch_tree_attention_tc(const void* q, const void* k_slab, const vo
     static std::once_flag once;
     static cudaError_t attr_err = cudaSuccess;
     std::call_once(once, [] {
-        attr_err = cudaFuncSetAttribute(tree_attention_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)AT_SMEM);
+        attr_err = cudaFuncSetAttribute(tree_attention_tc_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)AT_SMEM);
+        if (attr_err == cudaSuccess)
+            attr_err = cudaFuncSetAttribute(tree_attention_tc_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)AT_SMEM);
     });
     if (attr_err != cudaSuccess) return attr_err;
     CUtensorMap map_q, map_k, map_v;
@@ -873,7 +901,7 @@ cudaError_t launch_tree_attention_tc(const void* q, const void* k_slab, const vo
     p.cluster = plan.cluster;
     count_launch();
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(plan.grid); cfg.blockDim = dim3(AT_THREADS); cfg.dynamicSmemBytes = AT_SMEM; cfg.stream = st;
+    cfg.gridDim = dim3(plan.grid); cfg.blockDim = dim3(at_threads(plan.split)); cfg.dynamicSmemBytes = AT_SMEM; cfg.stream = st;
     cudaLaunchAttribute attr[2];
     int n_attr = 0;
     if (chain_active()) {
@@ -887,7 +915,8 @@ cudaError_t launch_tree_attention_tc(const void* q, const void* k_slab, const vo
         ++n_attr;
     }
     cfg.attrs = attr; cfg.numAttrs = n_attr;
-    cudaError_t e = cudaLaunchKernelEx(&cfg, tree_attention_tc_kernel, map_q, map_k, map_v, p);
+    cudaError_t e = plan.split == 4 ? cudaLaunchKernelEx(&cfg, tree_attention_tc_kernel<4>, map_q, map_k, map_v, p)
+                                    : cudaLaunchKernelEx(&cfg, tree_attention_tc_kernel<2>, map_q, map_k, map_v, p);
     if (e == cudaSuccess) e = cudaGetLastError();
     if (e != cudaSuccess || !plan.merge_kernel) return e;
     count_launch();
