@@ -467,12 +467,26 @@ class Model:
         br = _i32(branches)
         br = br.reshape(br.shape[0], -1) if br.size else np.zeros((0, 0), np.int32)
         r, bl = (br.shape[0], br.shape[1]) if br.size else (0, 0)
-        tokens, parent, pred = (np.zeros(MAX_ROWS, np.int32) for _ in range(3))
-        path = np.zeros(PATH_STRIDE, np.int32)
-        n, k, bonus = C.c_int32(0), C.c_int32(0), C.c_int32(0)
-        _check(lib().trj_step_host(self._handle, _dev(self.k_cache), _dev(self.v_cache), _dev(self.seq_len), max_len,
-                                   int(root), _p32(window), len(window), _p32(br), r, bl, _p32(tokens), _p32(parent),
-                                   C.byref(n), _p32(pred), C.byref(k), _p32(path), C.byref(bonus), _stream(stream)))
+        hb = self._step_host_buffers()                       # marshalling state that does not change between calls
+        tokens, parent, pred, path = hb["tokens"], hb["parent"], hb["pred"], hb["path"]
+        n, k, bonus = hb["n"], hb["k"], hb["bonus"]
+        _check(hb["fn"](self._handle, hb["kc"], hb["vc"], hb["len"], max_len,
+                        int(root), _p32(window), len(window), _p32(br), r, bl, hb["p_tokens"], hb["p_parent"],
+                        hb["r_n"], hb["p_pred"], hb["r_k"], hb["p_path"], hb["r_bonus"], _stream(stream)))
         m = n.value
-        return {"tokens": tokens[:m], "parent": parent[:m], "node_argmax": pred[:m], "k_acc": k.value,
-                "path": path[:k.value + 1], "bonus": bonus.value}
+        return {"tokens": tokens[:m].copy(), "parent": parent[:m].copy(), "node_argmax": pred[:m].copy(), "k_acc": k.value,
+                "path": path[:k.value + 1].copy(), "bonus": bonus.value}
+
+    def _step_host_buffers(self):
+        hb = getattr(self, "_hb", None)
+        if hb is None or hb["ptrs"] != (self.k_cache.data_ptr(), self.v_cache.data_ptr(), self.seq_len.data_ptr()):
+            tokens, parent, pred = (np.zeros(MAX_ROWS, np.int32) for _ in range(3))
+            path = np.zeros(PATH_STRIDE, np.int32)
+            n, k, bonus = C.c_int32(0), C.c_int32(0), C.c_int32(0)
+            hb = {"ptrs": (self.k_cache.data_ptr(), self.v_cache.data_ptr(), self.seq_len.data_ptr()),
+                  "fn": lib().trj_step_host, "kc": _dev(self.k_cache), "vc": _dev(self.v_cache), "len": _dev(self.seq_len),
+                  "tokens": tokens, "parent": parent, "pred": pred, "path": path, "n": n, "k": k, "bonus": bonus,
+                  "p_tokens": _p32(tokens), "p_parent": _p32(parent), "p_pred": _p32(pred), "p_path": _p32(path),
+                  "r_n": C.byref(n), "r_k": C.byref(k), "r_bonus": C.byref(bonus)}
+            self._hb = hb
+        return hb
