@@ -136,3 +136,37 @@ def test_llama7b_shape_two_layers_bf16(trj):
     stats = drive_with_oracle_trace(trj, model, prompt, trace, tol=2e-2)
     assert stats["rows"] > 100
     model.close()
+
+
+def test_programmatic_launch_does_not_change_results(trj):
+    """The chain's kernels start on chain-invariant data before their predecessor has finished (tensor maps, weights,
+    batch geometry, cached K/V rows).  If any of that were data the predecessor still writes, the result would
+    depend on timing: the same verification step must give bit-identical logits and caches with programmatic
+    launches on, repeatedly, and with every launch fully serialised."""
+    cfg = synth.LLAMA7B.with_layers(2)
+    model, _ = make_models(trj, cfg, 4, max_seq=512, max_rows=128)
+    prompt = synth.prompt(11, 300, cfg.vocab)
+    model.prefill(i32(prompt))
+    base_len = model.seq_len.clone()
+    parent = synth.random_tree(5, 33, 6, 3)
+    depth, anc = trj.tree_from_parents(parent)
+    tokens = synth.prompt(12, 33, cfg.vocab)
+    args = (i32(tokens), i32(parent), i32(depth), anc_dev(anc), i32([0, 33]))
+
+    def run():
+        model.seq_len.copy_(base_len)
+        out = model.verify_step(*args, max_rows=33, max_len=300 + 33, want_logits=True)
+        torch.cuda.synchronize()
+        rows = slice(300, 333)
+        return out["logits"].clone(), model.k_cache[:, 0, :, rows].clone(), model.v_cache[:, 0, :, rows].clone()
+    try:
+        ref = run()
+        for _ in range(3):
+            for a, b in zip(ref, run()):
+                assert torch.equal(a, b)
+        trj.set_pdl(False)
+        for a, b in zip(ref, run()):
+            assert torch.equal(a, b)
+    finally:
+        trj.set_pdl(True)
+    model.close()
