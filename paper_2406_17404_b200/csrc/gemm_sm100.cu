@@ -13,6 +13,7 @@
 // order, so results do not depend on scheduling.
 #include <cuda.h>
 #include <mutex>
+#include <algorithm>
 #include "trj_internal.h"
 
 namespace trj {
@@ -344,9 +345,12 @@ bool gemm_tc_supported(const void* x, const void* x_lo, const void* w, const flo
 
 // Number of K ranges per weight tile.  Items (tiles x splits) are dealt round-robin to a grid of at most 296
 // CTAs, so the choice trades balance (items close to a multiple of 148) against the extra traffic of the
-// partial sums, about 2*splits*M/K of the weight bytes.
-int gemm_tc_splits(int32_t M, int32_t N, int32_t K) {
+// partial sums, about 2*splits*M/K of the weight bytes.  When no consumer kernel adds the pieces (`finished`:
+// the caller wants y itself) a reduce kernel has to read them again and is one more launch: then a single
+// K range is taken as soon as the tiles alone fill most of the grid.
+int gemm_tc_splits(int32_t M, int32_t N, int32_t K, bool finished) {
     const int tiles = (N + TC_BM - 1) / TC_BM, kblocks = K / TC_BK;
+    if (finished && tiles * 5 >= TC_GRID * 4) return 1;
     int best = 1;
     double best_score = 0.0;
     for (int s = 1; s <= 16 && s <= (kblocks >= 4 ? kblocks / 4 : 1); ++s) {
@@ -361,7 +365,7 @@ int gemm_tc_splits(int32_t M, int32_t N, int32_t K) {
 // Workspace: a 256-byte header whose first word is the device status, then the split-K partial sums.
 size_t gemm_tc_workspace(int32_t M, int32_t N, int32_t K) {
     if (K % TC_BK != 0 || K < TC_BK) return 256;
-    const int s = gemm_tc_splits(M, N, K);
+    const int s = std::max(gemm_tc_splits(M, N, K, false), gemm_tc_splits(M, N, K, true));
     return 256 + (s > 1 ? align_up((size_t)s * M * N * sizeof(float), 256) : 0);
 }
 
@@ -386,7 +390,7 @@ cudaError_t launch_gemm_tc(const void* x, const void* x_lo, const void* w, float
     while (p.acc_cols < reach) p.acc_cols *= 2;
     p.kblocks = K / TC_BK;
     p.tiles = (N + TC_BM - 1) / TC_BM;
-    p.splits = gemm_tc_splits(M, N, K);
+    p.splits = gemm_tc_splits(M, N, K, parts == nullptr);
     const size_t stage = TC_A_BYTES + (size_t)p.n_mma * TC_BK * 2;
     // four stages in at most ~108 KB let two CTAs share an SM; wider activation tiles get one CTA per SM
     p.stages = (int)((108 * 1024) / stage);
