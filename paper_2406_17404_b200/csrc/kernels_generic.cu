@@ -305,13 +305,22 @@ __global__ void rope_kv_write_vec_kernel(const Parts qkv, const double* __restri
     float4 acc[6];                                           // q, k, v: first and second half of the head
 #pragma unroll
     for (int e = 0; e < 6; ++e) acc[e] = make_float4(0.f, 0.f, 0.f, 0.f);
-    for (int s = 0; s < qkv.splits; ++s) {                   // six independent loads per split-K piece
-        const float* piece = qkv.ptr + (size_t)s * qkv.stride + src;
-        float4 t[6];
+    // the pieces are requested three at a time (18 loads in flight) and added in ascending order
+    for (int s0 = 0; s0 < qkv.splits; s0 += 3) {
+        float4 t[3][6];
 #pragma unroll
-        for (int e = 0; e < 6; ++e) t[e] = *reinterpret_cast<const float4*>(piece + (e >> 1) * HD + (e & 1) * half);
+        for (int j = 0; j < 3; ++j)
+            if (s0 + j < qkv.splits) {
+                const float* piece = qkv.ptr + (size_t)(s0 + j) * qkv.stride + src;
 #pragma unroll
-        for (int e = 0; e < 6; ++e) { acc[e].x += t[e].x; acc[e].y += t[e].y; acc[e].z += t[e].z; acc[e].w += t[e].w; }
+                for (int e = 0; e < 6; ++e) t[j][e] = *reinterpret_cast<const float4*>(piece + (e >> 1) * HD + (e & 1) * half);
+            }
+#pragma unroll
+        for (int j = 0; j < 3; ++j)
+            if (s0 + j < qkv.splits) {
+#pragma unroll
+                for (int e = 0; e < 6; ++e) { acc[e].x += t[j][e].x; acc[e].y += t[j][e].y; acc[e].z += t[j][e].z; acc[e].w += t[j][e].w; }
+            }
     }
     auto rot_lo = [&](const float4& a, const float4& bb) {
         return make_float4(a.x * cs[0] - bb.x * sn[0], a.y * cs[1] - bb.y * sn[1], a.z * cs[2] - bb.z * sn[2], a.w * cs[3] - bb.w * sn[3]);
