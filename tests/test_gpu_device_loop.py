@@ -120,6 +120,39 @@ def test_device_decode_loop_commits_the_oracle_tokens(trj):
     model.close()
 
 
+@pytest.mark.parametrize("width,r,lr", [(0, 3, 2), (3, 0, 0), (1, 1, 1)])
+def test_device_decode_loop_degenerate_tree_shapes(trj, width, r, lr):
+    """No window, no retrieved branches, a single-token window and branch: the loop still commits the oracle's tokens."""
+    cfg = synth.TINY
+    n_steps = 10
+    model, dec = make_models(trj, cfg, 1, max_seq=40 + n_steps * 4 + 16, max_rows=16)
+    prompt = synth.prompt(3, 40, cfg.vocab)
+    draw = lambda s, n: synth.noise_draws(5, s, n)
+    trace = []
+    oracle.tr_jacobi_generate(dec, prompt, 60, width, r, lr, draw, trace=trace)
+    trace = trace[:n_steps]
+    want = oracle.tr_jacobi_generate(dec, prompt, sum(rec["k"] + 1 for rec in trace), width, r, lr, draw)
+    model.seq_len.zero_()
+    first = int(model.prefill(i32(prompt)).item())
+    committed = [int(t) for t in prompt] + [first]
+    buf = np.zeros(len(committed) + n_steps * (max(width, lr) + 1), np.int32); buf[:len(committed)] = committed
+    d_ctx, d_n = i32(buf), i32([len(committed)])
+    window = i32([committed[int(d) % len(committed)] for d in draw(0, width)]) if width else torch.empty(0, dtype=torch.int32, device="cuda")
+    per = max(width + r * lr, 1)
+    draws = i64(np.stack([np.resize(np.asarray(draw(s, width + r * lr), np.int64), per) for s in range(1, n_steps + 1)]))
+    if width + r * lr == 0:
+        pytest.skip("a tree of the root alone needs no draws")
+    model.decode_device(d_ctx, d_n, len(committed), window, r, lr, draws, n_steps)
+    torch.cuda.synchronize()
+    got = d_ctx.cpu().numpy()[len(prompt):int(d_n[0])].tolist()
+    first_bad = next((i for i, (a, b) in enumerate(zip(got, want)) if a != b), None)
+    if first_bad is not None:
+        assert min(oracle.top2_margin(rec["logits"]).min() for rec in trace) < MARGIN
+    else:
+        assert len(got) == len(want) + 1
+    model.close()
+
+
 def test_device_decode_loop_7b_shape_equals_the_host_driven_loop(trj):
     """7B layer shape, 2 layers, bf16 (the tcgen05 kernels): the device-resident loop and the host-driven loop run the
     same kernels on the same inputs, so their committed tokens must be identical.  This checks the loop's plumbing on
