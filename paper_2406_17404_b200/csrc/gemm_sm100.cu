@@ -118,14 +118,13 @@ __device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t a_desc, uint
 __device__ __forceinline__ void umma_commit(uint32_t bar) {
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
 }
-__device__ __forceinline__ void tmem_ld16(uint32_t taddr, float* v) {
-    uint32_t r[16];
-    asm volatile("tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
-                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
-                   "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+__device__ __forceinline__ void tmem_ld8(uint32_t taddr, float* v) {
+    uint32_t r[8];
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7])
                  : "r"(taddr) : "memory");
 #pragma unroll
-    for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]);
+    for (int i = 0; i < 8; ++i) v[i] = __uint_as_float(r[i]);
 }
 
 // Persistent kernel: CTA c works on items c, c + grid, c + 2*grid, ... where an item is one 128-row weight tile
@@ -263,13 +262,14 @@ __global__ void __launch_bounds__(TC_THREADS, 2) gemm_tc_kernel(const __grid_con
             const int n = tile * TC_BM + q * 32 + lane;
             const uint32_t taddr = tmem_base + (uint32_t)(buf * p.acc_cols) + ((uint32_t)(q * 32) << 16);
             float* out = p.out + (size_t)split * p.M * p.N;
-            for (int c0 = 0; c0 < p.m_pad; c0 += 16) {
-                float hi[16], lo[16];
-                tmem_ld16(taddr + c0, hi);
-                if (p.halves == 2) tmem_ld16(taddr + p.m_pad + c0, lo);
+            // eight columns (activation rows) of each half per round trip: measured faster than 16 or 32 at a time
+            for (int c0 = 0; c0 < p.m_pad; c0 += 8) {
+                float hi[8], lo[8];
+                tmem_ld8(taddr + c0, hi);
+                if (p.halves == 2) tmem_ld8(taddr + p.m_pad + c0, lo);
                 asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 #pragma unroll
-                for (int jj = 0; jj < 16; ++jj) {
+                for (int jj = 0; jj < 8; ++jj) {
                     const int m = c0 + jj;
                     if (m < p.M && n < p.N) out[(size_t)m * p.N + n] = p.halves == 2 ? hi[jj] + lo[jj] : hi[jj];
                 }
