@@ -39,7 +39,7 @@ UNIT = "tokens/s"
 # DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) of ALL 129 projection launches of one step, from
 # an ncu capture of the current projection kernel (profiles/gemm_tc_traffic_llama7b_33rows.md); set to None
 # whenever that kernel changes.
-GEMM_TRAFFIC_BYTES_PER_STEP = 13736045312 + 71997696
+GEMM_TRAFFIC_BYTES_PER_STEP = 13720706048 + 85961728
 
 
 def measured_peaks():
