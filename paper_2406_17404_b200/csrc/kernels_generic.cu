@@ -3,6 +3,7 @@
 // sizes) and all the small element-wise steps between the projections.
 #include <atomic>
 #include <mutex>
+#include <algorithm>
 #include "trj_internal.h"
 
 namespace trj {
@@ -273,17 +274,18 @@ __global__ void rope_kv_write_kernel(const Parts qkv, const double* __restrict__
 }
 
 // Four consecutive dimensions per thread (head_dim / 2 a multiple of 4): 16-byte loads of the projection pieces,
-// 8-byte (bf16) or 16-byte (fp32) stores.  One CTA covers ROPE_HEADS heads of a row.
-constexpr int ROPE_HEADS = 8;
+// 8-byte (bf16) or 16-byte (fp32) stores.  One CTA covers heads_per_cta heads of a row (at most ROPE_THREADS threads).
+constexpr int ROPE_THREADS = 256;           // a few fat CTAs (16 heads of 128 each) measured faster than many thin ones
 template <typename T>
-__global__ void rope_kv_write_vec_kernel(const Parts qkv, const double* __restrict__ inv_freq,
+__global__ void __launch_bounds__(ROPE_THREADS) rope_kv_write_vec_kernel(const Parts qkv, const double* __restrict__ inv_freq,
                                          const int32_t* __restrict__ depth, const int32_t* __restrict__ seq_len,
                                          const int32_t* __restrict__ row_off, int B, T* __restrict__ q_out,
-                                         T* __restrict__ k_slab, T* __restrict__ v_slab, int H, int D, int max_seq) {
+                                         T* __restrict__ k_slab, T* __restrict__ v_slab, int H, int D, int max_seq,
+                                         int heads_per_cta) {
     pdl_launch_dependents();
     // geometry and rotations do not depend on the projection: have them ready before waiting for it
     const int half = D >> 1, HD = H * D, per_head = half >> 2;
-    const int row = blockIdx.x, hh = blockIdx.y * ROPE_HEADS + (int)threadIdx.x / per_head;
+    const int row = blockIdx.x, hh = blockIdx.y * heads_per_cta + (int)threadIdx.x / per_head;
     const int i = ((int)threadIdx.x % per_head) * 4;
     if (hh >= H) return;
     const int b = seq_of_row(row_off, B, row);
@@ -662,11 +664,12 @@ cudaError_t launch_rope_kv_write(const Parts& qkv, const double* inv_freq, const
     count_launch();
     cudaError_t launch_err = cudaSuccess;
     const int per_head = D / 8;                              // threads per head in the vector kernel
-    const bool vec = D % 8 == 0 && per_head * ROPE_HEADS <= 1024 && qkv.stride % 4 == 0 && ((uintptr_t)qkv.ptr % 16) == 0;
+    const int hpc = per_head > 0 ? std::max(1, std::min(H, ROPE_THREADS / per_head)) : 1;
+    const bool vec = D % 8 == 0 && per_head <= ROPE_THREADS && qkv.stride % 4 == 0 && ((uintptr_t)qkv.ptr % 16) == 0;
     if (vec) {
-        dim3 grid(bt.rows_total, (H + ROPE_HEADS - 1) / ROPE_HEADS);
-        DISPATCH_T(dtype, launch_err = launch_chain(rope_kv_write_vec_kernel<T>, grid, dim3(per_head * ROPE_HEADS), 0, st, qkv, inv_freq, depth,
-                                                    bt.seq_len, bt.row_off, bt.B, (T*)q_out, (T*)k_slab, (T*)v_slab, H, D, max_seq));
+        dim3 grid(bt.rows_total, (H + hpc - 1) / hpc);
+        DISPATCH_T(dtype, launch_err = launch_chain(rope_kv_write_vec_kernel<T>, grid, dim3(per_head * hpc), 0, st, qkv, inv_freq, depth,
+                                                    bt.seq_len, bt.row_off, bt.B, (T*)q_out, (T*)k_slab, (T*)v_slab, H, D, max_seq, hpc));
     } else {
         dim3 grid(bt.rows_total, H);
         DISPATCH_T(dtype, launch_err = launch_chain(rope_kv_write_kernel<T>, grid, dim3(64), 0, st, qkv, inv_freq, depth, bt.seq_len, bt.row_off,
