@@ -357,7 +357,12 @@ def run_ours(args, rank, world, local_rank):
     peaks = measured_peaks()
     cfg = synth.LLAMA7B if not args.layers else synth.LLAMA7B.with_layers(args.layers)
     layers, glob = device_weights(cfg, 1234 + rank, dev)
-    model = trj.Model(cfg, layers, glob, max_batch=1, max_seq=PROMPT + 1024, max_rows=trj.MAX_ROWS)
+    # cache rows: the prompt, every step of the warm-up decode, of the end-to-end loop and of the two device loops in
+    # their worst case (a step commits at most depth + 1 tokens), plus one tree
+    per_step = max(WIDTH, BRANCH_LEN) + 1
+    n_decode_steps = (max(args.warmup, 3) + 1) + (max(args.warmup, 3) + args.steps + 1) + 2 * args.steps
+    max_seq = max(PROMPT + 1024, PROMPT + 1 + n_decode_steps * per_step + TREE_ROWS + 64)
+    model = trj.Model(cfg, layers, glob, max_batch=1, max_seq=max_seq, max_rows=trj.MAX_ROWS)
     prompt = synth.prompt(100 + rank, PROMPT, cfg.vocab)
     draw = lambda s, n: synth.noise_draws(rank, s, n)
 
