@@ -281,9 +281,9 @@ trj_status trj_prefill(trj_ctx* ctx, void* k_cache, void* v_cache, int32_t* seq_
  *   dev     : k_cache, v_cache, seq_len [1] (advanced by k_acc + 1)
  *   max_len : host-known bound of seq_len[0] + M
  * From the second call on a context the launch sequence is captured once per
- * (tree rows, launch geometry, buffer addresses) into a CUDA graph on a stream of
- * the context and replayed; it still runs after everything already enqueued on
- * `stream` and has completed when the call returns. */
+ * (tree rows, launch geometry, buffer addresses) into a CUDA graph (on a stream of
+ * the context) and that graph is launched on `stream`; it runs after everything
+ * already enqueued there and has completed when the call returns. */
 trj_status trj_step_host(trj_ctx* ctx, void* k_cache, void* v_cache, int32_t* seq_len, int32_t max_len,
                          int32_t root, const int32_t* window, int32_t W,
                          const int32_t* branches, int32_t R, int32_t branch_len,

@@ -554,11 +554,9 @@ trj_status run_step(trj_ctx* ctx, void* k_cache, void* v_cache, int32_t* seq_len
         if (ctx->graphs.size() >= 32) { cudaGraphExecDestroy(ctx->graphs.front().exec); ctx->graphs.erase(ctx->graphs.begin()); }
         ctx->graphs.push_back({M, grid, k_cache, v_cache, seq_len, exec});
     }
-    // keep the order of the caller's stream: the graph runs after everything already enqueued on it
-    TRJ_CHECK_CUDA(cudaEventRecord(ctx->order_ev, st));
-    TRJ_CHECK_CUDA(cudaStreamWaitEvent(ctx->cap_stream, ctx->order_ev, 0));
-    TRJ_CHECK_CUDA(cudaGraphLaunch(exec, ctx->cap_stream));
-    TRJ_CHECK_CUDA(cudaStreamSynchronize(ctx->cap_stream));
+    // launched on the caller's stream: the graph runs after everything already enqueued on it
+    TRJ_CHECK_CUDA(cudaGraphLaunch(exec, st));
+    TRJ_CHECK_CUDA(cudaStreamSynchronize(st));
     return TRJ_OK;
 }
 
