@@ -101,22 +101,6 @@ class ClockSampler:
 
 
 # --------------------------------------------------------------------------------------- our arm
-def device_weights(cfg, seed, device):
-    """Random-init weights ~ N(0, 0.02) drawn on the device (seeded), stored as bf16; norm gains 1."""
-    import torch
-    g = torch.Generator(device=device)
-    g.manual_seed(seed)
-
-    def mat(rows, cols):
-        return (torch.randn(rows, cols, generator=g, device=device, dtype=torch.float32) * cfg.weight_std).to(torch.bfloat16)
-    d, f, hd = cfg.d_model, cfg.d_ff, cfg.n_heads * cfg.head_dim
-    ones = lambda: torch.ones(d, dtype=torch.float32, device=device)
-    layers = [{"attn_norm": ones(), "wqkv": mat(3 * hd, d), "wo": mat(d, hd), "mlp_norm": ones(),
-               "w_gate_up": mat(2 * f, d), "w_down": mat(d, f)} for _ in range(cfg.n_layers)]
-    glob = {"embed": mat(cfg.vocab, d), "lm_head": mat(cfg.vocab, d), "final_norm": ones()}
-    return layers, glob
-
-
 def gemm_bytes_per_step(cfg, rows):
     """Algorithmic bytes of all projections of one verification step: every weight once (bf16), the
     split-bf16 activations in and the fp32 results out."""
@@ -344,6 +328,7 @@ def run_ours(args, rank, world, local_rank):
     import torch
     import torch.distributed as dist
     import synth
+    from synth.device import device_weights
     import paper_2406_17404_b200 as trj
     from paper_2406_17404_b200 import decode
 

@@ -15,7 +15,12 @@
  *            and owns every buffer; the library borrows it for the duration of
  *            the call (weights and workspace: for the lifetime of the context)
  *            and frees nothing it did not allocate.  The library allocates no
- *            device memory: all scratch comes from caller-provided workspaces.
+ *            DEVICE memory: all device scratch comes from caller-provided
+ *            workspaces (one exception: trj_argmax_accept_static keeps its
+ *            scratch in a fixed array of the library's device image).  A model
+ *            context owns a few host-side objects of its own: small pinned
+ *            staging buffers, a stream, an event and the CUDA graphs of its
+ *            step; trj_destroy releases them.
  * Streams    `stream` is a cudaStream_t passed as void* (NULL = default
  *            stream).  Device entry points only enqueue work; results are in
  *            device memory once the stream has been synchronised.  Entry
@@ -25,7 +30,14 @@
  *            pointers are checked on the host before anything is launched, so
  *            an invalid call launches nothing.  Nothing aborts, throws or
  *            prints.  trj_last_error gives a message for the calling thread's
- *            most recent failure.
+ *            most recent failure.  Every device-side wait of the tensor-core
+ *            kernels is bounded; one that expires leaves TRJ_ETIMEOUT in a
+ *            status word (of the op's workspace, or of the model context) and
+ *            the kernel returns normally.  trj_step_host returns that status
+ *            itself; after the asynchronous model calls ask trj_device_status.
+ *            A shape that the tensor-core kernels are written for is never
+ *            run on a slower kernel because a workspace is short or misaligned:
+ *            that is TRJ_ECAPACITY / TRJ_EINVAL.
  * Layouts    All tensors are dense, row-major, innermost dimension last.
  *            dtype is TRJ_BF16 (bf16 storage, fp32 accumulation) or TRJ_F32.
  *            KV cache: [L][B][H][max_seq][D]; sequence b has seq_len[b]
@@ -201,10 +213,12 @@ trj_status trj_argmax_accept(const void* logits, int32_t dtype, int32_t V,
  * trj_argmax_accept.  The call allocates nothing, neither device nor pinned
  * memory.
  *   - rows_total > TRJ_STATIC_MAX_ROWS is refused with TRJ_ECAPACITY (use the
- *     workspace variant for larger batches).
+ *     workspace variant for larger batches).  The total does not lift the
+ *     per-tree limit: a tree still holds at most TRJ_MAX_ROWS rows, and
+ *     rows_total > B * TRJ_MAX_ROWS is refused with TRJ_ECAPACITY as well.
  *   - The first call on a device looks up the array's device address (a one-time
  *     set-up done with that device current); make that first call outside any
- *     stream capture.
+ *     stream capture (inside one it is refused with TRJ_EINVAL).
  *   - All calls on a device share the one array.  The tickets are cleared at the
  *     start of every call, so the previous call's contents do not matter, but two
  *     calls whose kernels overlap on the GPU (for instance on different
@@ -344,6 +358,22 @@ trj_status trj_decode_device(trj_ctx* ctx, void* k_cache, void* v_cache, int32_t
 size_t     trj_gemm_workspace(int32_t M, int32_t N, int32_t K);
 trj_status trj_gemm(const void* x, const void* w, float* y, int32_t M, int32_t N, int32_t K,
                     int32_t dtype, void* workspace, size_t workspace_bytes, void* stream);
+
+/* ------------------------------------------------------------------------
+ * Device-side time-outs (no counterpart in the paper).
+ * trj_device_status: synchronises `stream` and reads the context's two status
+ * words (projections, attention).  TRJ_OK if no bounded device-side wait has
+ * expired since the words were last cleared, TRJ_ETIMEOUT otherwise; with
+ * clear != 0 the words are then reset.  After a time-out the results of the
+ * affected step are undefined and the context's workspace should be zero-filled
+ * again before it is reused (tickets and partial sums may be half-written).
+ * trj_selftest_wait_expiry: launches one CTA in which one thread waits, with a
+ * limit of `polls` polls (1 .. 2^21), on a barrier that nobody arrives at, using
+ * the same wait routine as the tensor-core kernels.  The wait gives up, writes
+ * TRJ_ETIMEOUT to *status (dev int32) and the kernel returns by itself: a way to
+ * see the error path work without anything going wrong. */
+trj_status trj_device_status(trj_ctx* ctx, int32_t clear, void* stream);
+trj_status trj_selftest_wait_expiry(int32_t* status, int32_t polls, void* stream);
 
 /* ------------------------------------------------------------------------
  * Measurement aids (no counterpart in the paper).

@@ -21,7 +21,7 @@ MAX_BATCH = 64
 PATH_STRIDE = 128
 # bytes trj_step_host moves per call: tokens/parent/depth/row_off + ancestor words in, predictions/k/bonus/path out
 STEP_H2D_BYTES = (3 * MAX_ROWS + 4) * 4 + MAX_ROWS * 2 * 8
-STEP_D2H_BYTES = (MAX_ROWS + 2 + PATH_STRIDE) * 4
+STEP_D2H_BYTES = (MAX_ROWS + 2 + PATH_STRIDE + 2) * 4      # ... and the two device status words
 F32, BF16 = 0, 1
 
 _lib = None
@@ -79,6 +79,8 @@ _SIGNATURES = {
     "trj_decode_device": (_I, [_VP, _VP, _VP, _VP, _VP, _I, _VP, _I, _VP, _I, _I, _I, _VP, _I, _VP, _VP]),
     "trj_gemm_workspace": (_SZ, [_I, _I, _I]),
     "trj_gemm": (_I, [_VP, _VP, _VP, _I, _I, _I, _I, _VP, _SZ, _VP]),
+    "trj_device_status": (_I, [_VP, _I, _VP]),
+    "trj_selftest_wait_expiry": (_I, [_VP, _I, _VP]),
     "trj_launch_count": (C.c_uint64, []),
     "trj_set_pdl": (None, [_I]),
     "trj_profile_enable": (_I, [_VP, _I]),
@@ -312,6 +314,15 @@ def gemm(x, w, *, out=None, workspace=None, stream=None):
     return out
 
 
+def selftest_wait_expiry(polls: int = 256, stream=None) -> int:
+    """trj_selftest_wait_expiry: returns the status word a wait that nobody satisfies leaves behind (4)."""
+    torch = _torch()
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    _check(lib().trj_selftest_wait_expiry(_dev(status), int(polls), _stream(stream)))
+    torch.cuda.synchronize()
+    return int(status.item())
+
+
 def draft_tokens(context, n_ctx, window, n_branches: int, branch_len: int, draws, stream=None):
     """trj_draft_tokens: the next tree's tokens [1 + W + R*Lr] (int32, device) from device buffers.
 
@@ -390,6 +401,10 @@ class Model:
             self.close()
         except Exception:
             pass
+
+    def device_status(self, clear: bool = False, stream=None) -> None:
+        """trj_device_status: raises TrjError (status 4) if a bounded device-side wait has expired."""
+        _check(lib().trj_device_status(self._handle, 1 if clear else 0, _stream(stream)))
 
     def profile_enable(self, on: bool = True) -> None:
         _check(lib().trj_profile_enable(self._handle, 1 if on else 0))

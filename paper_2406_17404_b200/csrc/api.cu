@@ -50,6 +50,7 @@ extern "C" trj_status trj_tree_attention(const void* q, const void* k_cache, con
                 "tree_attention: tensors must be 16-byte aligned");
     TRJ_REQUIRE(workspace && workspace_bytes >= trj_tree_attention_workspace(rows_total, B, H, D, max_len),
                 TRJ_ECAPACITY, "tree_attention: workspace too small");
+    TRJ_REQUIRE(aligned(workspace, 256), TRJ_EINVAL, "tree_attention: workspace must be 256-byte aligned");
     if (rows_total == 0) return TRJ_OK;
     Batch bt{seq_len, row_off, B, rows_total, max_rows, max_len};
     TRJ_CHECK_CUDA(launch_tree_attention(q, k_cache, v_cache, anc, anc_words, bt, H, D, max_seq, dtype, out, nullptr,
@@ -90,11 +91,16 @@ extern "C" trj_status trj_argmax_accept_static(const void* logits, int32_t dtype
     TRJ_REQUIRE(dtype_ok(dtype), TRJ_EINVAL, "argmax_accept_static: unknown dtype %d", dtype);
     TRJ_REQUIRE(V >= 1 && B >= 1 && rows_total >= B, TRJ_EINVAL, "argmax_accept_static: bad sizes (every tree has a root)");
     TRJ_REQUIRE(B <= TRJ_MAX_BATCH, TRJ_ECAPACITY, "argmax_accept_static: batch %d exceeds %d", B, TRJ_MAX_BATCH);
+    TRJ_REQUIRE(rows_total <= B * TRJ_MAX_ROWS, TRJ_ECAPACITY,
+                "argmax_accept_static: %d rows in %d trees: a tree holds at most %d rows", rows_total, B, TRJ_MAX_ROWS);
     TRJ_REQUIRE(rows_total <= TRJ_STATIC_MAX_ROWS, TRJ_ECAPACITY,
                 "argmax_accept_static: %d rows exceed the built-in scratch of %d rows; use trj_argmax_accept with a workspace",
                 rows_total, TRJ_STATIC_MAX_ROWS);
-    TRJ_CHECK_CUDA(launch_argmax_accept_static(logits, dtype, V, tokens, parent, depth, row_off, B, rows_total,
-                                               node_argmax, margin, k_acc, path, bonus, (cudaStream_t)stream));
+    const cudaError_t e = launch_argmax_accept_static(logits, dtype, V, tokens, parent, depth, row_off, B, rows_total,
+                                                      node_argmax, margin, k_acc, path, bonus, (cudaStream_t)stream);
+    TRJ_REQUIRE(e != cudaErrorStreamCaptureUnsupported, TRJ_EINVAL,
+                "argmax_accept_static: the first call on a device must be made outside stream capture");
+    TRJ_CHECK_CUDA(e);
     return TRJ_OK;
 }
 
@@ -122,6 +128,8 @@ extern "C" trj_status trj_gemm(const void* x, const void* w, float* y, int32_t M
     TRJ_REQUIRE(dtype_ok(dtype), TRJ_EINVAL, "gemm: unknown dtype %d", dtype);
     TRJ_REQUIRE(M >= 1 && N >= 1 && K >= 1, TRJ_EINVAL, "gemm: bad sizes");
     TRJ_REQUIRE(workspace && workspace_bytes >= trj_gemm_workspace(M, N, K), TRJ_ECAPACITY, "gemm: workspace too small");
+    TRJ_REQUIRE(aligned(workspace, 256) && aligned(x, 16) && aligned(w, 16) && aligned(y, 16), TRJ_EINVAL,
+                "gemm: workspace must be 256-byte aligned, tensors 16-byte aligned");
     TRJ_CHECK_CUDA(launch_gemm(x, nullptr, w, y, M, N, K, dtype, workspace, workspace_bytes, (cudaStream_t)stream));
     return TRJ_OK;
 }
@@ -142,7 +150,8 @@ struct trj_ctx {
     int32_t* chain_depth; uint64_t* chain_anc; int32_t* chunk_row_off; int32_t* unit_row_off;
     int32_t* loop_state;   // device: [0] step counter, [1] context-overflow flag of trj_decode_device
     int32_t* step_in;      // tokens | parent | depth | row_off(2) | pad -> anc
-    int32_t* step_out;     // node_argmax | k_acc | bonus | path
+    int32_t* step_out;     // node_argmax | k_acc | bonus | path | device status words (projections, attention)
+    int32_t* dev_status;   // the two status words at the end of step_out: TRJ_ETIMEOUT once a bounded wait expired
     int32_t* pin_in; int32_t* pin_out;   // pinned host mirrors
     // optional per-launch device timing (trj_profile_enable)
     bool prof_on = false; std::vector<cudaEvent_t> prof_ev; std::vector<int> prof_cat; size_t prof_used = 0;
@@ -159,7 +168,8 @@ namespace {
 
 constexpr int STEP_IN_INTS = 3 * TRJ_MAX_ROWS + 4;                       // + anc (2 words per row) after it
 constexpr int STEP_IN_BYTES = STEP_IN_INTS * 4 + TRJ_MAX_ROWS * 2 * 8;
-constexpr int STEP_OUT_INTS = TRJ_MAX_ROWS + 2 + TRJ_PATH_STRIDE;
+constexpr int STEP_STATUS_AT = TRJ_MAX_ROWS + 2 + TRJ_PATH_STRIDE;
+constexpr int STEP_OUT_INTS = STEP_STATUS_AT + 2;
 
 size_t carve(const trj_model_cfg& c, void* ws, trj_ctx* ctx) {
     const size_t es = dtype_size(c.dtype);
@@ -199,6 +209,7 @@ size_t carve(const trj_model_cfg& c, void* ws, trj_ctx* ctx) {
         ctx->chain_depth = chain_depth; ctx->chain_anc = chain_anc;
         ctx->chunk_row_off = chunk_row_off; ctx->unit_row_off = unit_row_off;
         ctx->step_in = step_in; ctx->step_out = step_out; ctx->loop_state = loop_state;
+        ctx->dev_status = step_out + STEP_STATUS_AT;
     }
     return cv.off;
 }
@@ -267,6 +278,7 @@ trj_status forward(trj_ctx* ctx, void* k_cache, void* v_cache, int32_t b0, const
                          ctx->attn_ws_bytes >= tree_attention_tc_workspace(bt.B, c.n_heads) &&
                          tree_attention_tc_supported(c.head_dim, c.dtype, bt.max_rows);
     const int attn_grid = attn_tc ? tree_attention_grid(bt.B, c.n_heads, bt.max_len) : ctx->sm_count;
+    int* const gemm_status = ctx->dev_status, *const attn_status = ctx->dev_status + 1;
     constexpr size_t AHEAD_BYTES = (size_t)32 << 20;         // measured optimum on the 7B shape (16-40 MB are close)
     LAUNCH(PROF_ELEMENTWISE, launch_embed(ctx->embed, c.dtype, tokens, ctx->h, M, d, st));
     Parts pr{nullptr, 1, 0};                 // result of the latest projection, possibly in split-K pieces
@@ -276,26 +288,26 @@ trj_status forward(trj_ctx* ctx, void* k_cache, void* v_cache, int32_t b0, const
         LAUNCH(PROF_ELEMENTWISE, launch_add_rmsnorm(ctx->h, pr, ctx->attn_norm[l], ctx->x, ctx->x_lo, c.dtype, M, d,
                                                     c.rms_eps, st));
         LAUNCH(PROF_GEMM, launch_gemm(ctx->x, ctx->x_lo, ctx->wqkv[l], ctx->y, M, 3 * HD, d, c.dtype, ctx->gemm_ws,
-                                      ctx->gemm_ws_bytes, st, &pr));
+                                      ctx->gemm_ws_bytes, st, &pr, nullptr, gemm_status));
         LAUNCH(PROF_ROPE, launch_rope_kv_write(pr, ctx->inv_freq, depth, bt, ctx->q, k_slab, v_slab, c.dtype,
                                                c.n_heads, c.head_dim, c.max_seq, st));
         // inside the decoder the attention result reaches the output projection as a bf16 pair, like every
         // other projection input
         LAUNCH(PROF_ATTENTION, launch_tree_attention(ctx->q, k_slab, v_slab, anc, anc_words, bt, c.n_heads, c.head_dim,
                                                      c.max_seq, c.dtype, ctx->x, ctx->x_lo, ctx->attn_ws,
-                                                     ctx->attn_ws_bytes, st));
+                                                     ctx->attn_ws_bytes, st, attn_status));
         // While the attention kernel runs, HBM is nearly idle and the SMs it leaves free go to the first CTAs of
         // the output projection, which only wait: they ask for the start of the gate/up weights into L2.
         const WeightPrefetch ahead{ctx->w_gate_up[l], 2 * c.d_ff, d, AHEAD_BYTES, 2 * std::max(0, ctx->sm_count - attn_grid)};
         LAUNCH(PROF_GEMM, launch_gemm(ctx->x, ctx->x_lo, ctx->wo[l], ctx->y, M, d, HD, c.dtype, ctx->gemm_ws,
-                                      ctx->gemm_ws_bytes, st, &pr, &ahead));
+                                      ctx->gemm_ws_bytes, st, &pr, &ahead, gemm_status));
         LAUNCH(PROF_ELEMENTWISE, launch_add_rmsnorm(ctx->h, pr, ctx->mlp_norm[l], ctx->x, ctx->x_lo, c.dtype, M, d,
                                                     c.rms_eps, st));
         LAUNCH(PROF_GEMM, launch_gemm(ctx->x, ctx->x_lo, ctx->w_gate_up[l], ctx->y, M, 2 * c.d_ff, d, c.dtype, ctx->gemm_ws,
-                                      ctx->gemm_ws_bytes, st, &pr));
+                                      ctx->gemm_ws_bytes, st, &pr, nullptr, gemm_status));
         LAUNCH(PROF_ELEMENTWISE, launch_swiglu(pr, ctx->act, ctx->act_lo, c.dtype, M, c.d_ff, st));
         LAUNCH(PROF_GEMM, launch_gemm(ctx->act, ctx->act_lo, ctx->w_down[l], ctx->y, M, d, c.d_ff, c.dtype, ctx->gemm_ws,
-                                      ctx->gemm_ws_bytes, st, &pr));
+                                      ctx->gemm_ws_bytes, st, &pr, nullptr, gemm_status));
     }
     LAUNCH(PROF_ELEMENTWISE, launch_add_rmsnorm(ctx->h, pr, ctx->final_norm, ctx->x, ctx->x_lo, c.dtype, M, d,
                                                 c.rms_eps, st));
@@ -303,7 +315,7 @@ trj_status forward(trj_ctx* ctx, void* k_cache, void* v_cache, int32_t b0, const
         const size_t off = (size_t)lm_first * d * es;
         LAUNCH(PROF_GEMM, launch_gemm((char*)ctx->x + off, ctx->x_lo ? (char*)ctx->x_lo + off : nullptr, ctx->lm_head,
                                       ctx->logits + (size_t)lm_first * c.vocab, lm_rows, c.vocab, d, c.dtype,
-                                      ctx->gemm_ws, ctx->gemm_ws_bytes, st));
+                                      ctx->gemm_ws, ctx->gemm_ws_bytes, st, nullptr, nullptr, gemm_status));
     }
     return TRJ_OK;
 }
@@ -400,6 +412,27 @@ extern "C" trj_status trj_destroy(trj_ctx* ctx) {
     return TRJ_OK;
 }
 
+extern "C" trj_status trj_device_status(trj_ctx* ctx, int32_t clear, void* stream) {
+    TRJ_REQUIRE(ctx, TRJ_EINVAL, "device_status: null context");
+    cudaStream_t st = (cudaStream_t)stream;
+    int32_t words[2] = {0, 0};
+    TRJ_CHECK_CUDA(cudaMemcpyAsync(words, ctx->dev_status, sizeof(words), cudaMemcpyDeviceToHost, st));
+    TRJ_CHECK_CUDA(cudaStreamSynchronize(st));
+    if (words[0] == 0 && words[1] == 0) return TRJ_OK;
+    if (clear) {
+        TRJ_CHECK_CUDA(cudaMemsetAsync(ctx->dev_status, 0, sizeof(words), st));
+        TRJ_CHECK_CUDA(cudaStreamSynchronize(st));
+    }
+    return fail(TRJ_ETIMEOUT, "a bounded device-side wait expired (projection status %d, attention status %d)", words[0], words[1]);
+}
+
+extern "C" trj_status trj_selftest_wait_expiry(int32_t* status, int32_t polls, void* stream) {
+    TRJ_REQUIRE(status, TRJ_EINVAL, "selftest_wait_expiry: null status word");
+    TRJ_REQUIRE(polls >= 1 && polls <= (1 << 21), TRJ_EINVAL, "selftest_wait_expiry: polls %d outside 1..2^21", polls);
+    TRJ_CHECK_CUDA(launch_wait_expiry_selftest(status, (uint32_t)polls, (cudaStream_t)stream));
+    return TRJ_OK;
+}
+
 extern "C" uint64_t trj_launch_count(void) { return launches_so_far(); }
 extern "C" void trj_set_pdl(int32_t on) { set_pdl(on != 0); }
 
@@ -458,6 +491,8 @@ extern "C" trj_status trj_accept(trj_ctx* ctx, const int32_t* tokens, const int3
     TRJ_REQUIRE(ctx, TRJ_EINVAL, "accept: null context");
     TRJ_REQUIRE(tokens && parent && depth && row_off && node_argmax && k_acc && path && bonus, TRJ_EINVAL, "accept: null pointer");
     TRJ_REQUIRE(B >= 1 && B <= ctx->cfg.max_batch && rows_total >= B, TRJ_ECAPACITY, "accept: bad batch");
+    TRJ_REQUIRE(rows_total <= B * TRJ_MAX_ROWS, TRJ_ECAPACITY, "accept: %d rows in %d trees: a tree holds at most %d rows",
+                rows_total, B, TRJ_MAX_ROWS);
     cudaStream_t st = (cudaStream_t)stream;
     ChainScope chain;                        // these kernels wait for their predecessor before reading anything
     LAUNCH(PROF_ARGMAX, launch_argmax_accept(nullptr, TRJ_F32, 0, tokens, parent, depth, row_off, B, rows_total,
@@ -588,6 +623,11 @@ extern "C" trj_status trj_step_host(trj_ctx* ctx, void* k_cache, void* v_cache, 
     std::memcpy(parent, h_parent, sizeof(int32_t) * M);
     *n_rows = M;
     std::memcpy(node_argmax, ctx->pin_out, sizeof(int32_t) * M);
+    if (ctx->pin_out[STEP_STATUS_AT] != 0 || ctx->pin_out[STEP_STATUS_AT + 1] != 0) {
+        // the words stay set on the device (see trj_device_status); the step's results are not to be trusted
+        return fail(TRJ_ETIMEOUT, "step_host: a bounded device-side wait expired (projection status %d, attention status %d)",
+                    ctx->pin_out[STEP_STATUS_AT], ctx->pin_out[STEP_STATUS_AT + 1]);
+    }
     *k_acc = ctx->pin_out[TRJ_MAX_ROWS];
     *bonus = ctx->pin_out[TRJ_MAX_ROWS + 1];
     std::memcpy(path, ctx->pin_out + TRJ_MAX_ROWS + 2, sizeof(int32_t) * TRJ_PATH_STRIDE);

@@ -17,6 +17,7 @@
 #include <cuda.h>
 #include <mutex>
 #include "trj_internal.h"
+#include "sm100_common.cuh"
 
 namespace trj {
 namespace {
@@ -32,7 +33,6 @@ constexpr uint32_t AT_SUB = 128 * 128;       // one [128 x 64 bf16] swizzled sub
 constexpr uint32_t AT_TILE = 2 * AT_SUB;     // Q, P, a K tile or a V tile: 32 KB
 constexpr int AT_RING = 5;                   // K/V ring slots; load n = 2g + (0: K, 1: V) of tile g goes to slot n % 5
 constexpr uint32_t AT_SMEM = (1 + AT_RING) * AT_TILE + 1024;
-constexpr uint32_t AT_WAIT_LIMIT = 1u << 21;
 constexpr float AT_RESCALE_GAP = 8.f;        // raise the running max only when exceeded by 2^8
 constexpr int AT_PIECE_STRIDE = AT_D + 4;      // floats per row of a piece in shared memory (16-byte stores without bank conflicts)
 constexpr size_t AT_SLOT_FLOATS = (size_t)AT_D * AT_ROWS + 2 * AT_ROWS;   // O^T [d][row], m[row], l[row]
@@ -52,56 +52,8 @@ struct AtParams {
     int cluster;                 // CTAs per thread-block cluster that share one head (1: no clusters)
 };
 
-__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
-__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
-}
-__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
-    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
-    uint32_t ok;
-    asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
-                 : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
-    return ok != 0;
-}
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* status) {
-    for (uint32_t i = 0; i < AT_WAIT_LIMIT; ++i) {
-        if (mbar_try_wait(bar, parity)) return true;
-        if (i > 32) {
-            if (*abort_flag) return false;
-            __nanosleep(64);
-        }
-    }
-    *abort_flag = 1;
-    atomicExch(status, (int)TRJ_ETIMEOUT);
-    return false;
-}
-// Cache tiles are read once per launch and, over a step, are larger than L2: evict-first keeps them from pushing
-// out what is reused between kernels.
-__device__ __forceinline__ uint64_t l2_evict_first_policy() {
-    uint64_t policy;
-    asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(policy));
-    return policy;
-}
-__device__ __forceinline__ void tma_load_2d_hint(uint32_t dst, const CUtensorMap* map, int c_inner, int c_outer, uint32_t bar,
-                                                 uint64_t policy) {
-    asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1, {%2, %3}], [%4], %5;"
-                 ::"r"(dst), "l"(map), "r"(c_inner), "r"(c_outer), "r"(bar), "l"(policy) : "memory");
-}
-__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int c_inner, int c_outer, uint32_t bar) {
-    asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
-                 ::"r"(dst), "l"(map), "r"(c_inner), "r"(c_outer), "r"(bar) : "memory");
-}
+using namespace sm100;
 
-// K-major operand (rows 128 bytes apart, 8-row groups 1024 bytes apart), 128-byte swizzle.
-__device__ __forceinline__ uint64_t desc_kmajor(uint32_t addr) {
-    return (uint64_t)((addr & 0x3FFFF) >> 4) | ((uint64_t)1 << 16) | ((uint64_t)(1024 >> 4) << 32) |
-           ((uint64_t)1 << 46) | ((uint64_t)2 << 61);
-}
 // MN-major operand (V: keys are the contraction dim, head_dim is contiguous): 64-element spans of the
 // MN dim are 128-byte rows, one per key; 8-key groups 1024 bytes apart (stride offset); the second
 // 64-element block of the MN dim lies one sub-tile further (leading offset).
@@ -141,9 +93,6 @@ __device__ __forceinline__ void umma8_pv(uint32_t tmem_d, uint32_t tmem_a, uint3
                  ::"r"(tmem_d), "r"(tmem_a), "r"(b_lo), "r"(desc_hi), "r"(idesc), "r"(accumulate_first) : "memory");
 }
 #undef TRJ_MMA_TS
-__device__ __forceinline__ void umma_commit(uint32_t bar) {
-    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
-}
 __device__ __forceinline__ void tmem_ld32(uint32_t taddr, float* v) {
     uint32_t r[32];
     asm volatile("tcgen05.ld.sync.aligned.32x32b.x32.b32 "
@@ -448,7 +397,7 @@ __global__ void __launch_bounds__(at_threads(AT_SPLIT), 1) tree_attention_tc_ker
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                 const uint32_t k_smem = ring_smem + slot * AT_TILE;
                 // 8 x 16 elements of head_dim: two sub-tiles of four steps
-                const uint64_t q_desc = desc_kmajor(q_smem), k_desc = desc_kmajor(k_smem);
+                const uint64_t q_desc = desc_kmajor_sw128(q_smem), k_desc = desc_kmajor_sw128(k_smem);
                 umma8_qk(tmem_s[gg & 1], (uint32_t)q_desc, (uint32_t)k_desc, (uint32_t)(q_desc >> 32), idesc_qk);
                 umma_commit(bar(B_S_FULL + (gg & 1)));
                 umma_commit(bar(B_KV_EMPTY + slot));
@@ -874,7 +823,7 @@ size_t tree_attention_tc_workspace(int32_t B, int32_t H) {
 
 cudaError_t launch_tree_attention_tc(const void* q, const void* k_slab, const void* v_slab, const uint64_t* anc,
                                      int32_t anc_words, const Batch& bt, int32_t H, int32_t max_seq, void* out,
-                                     void* out_lo, void* workspace, cudaStream_t st) {
+                                     void* out_lo, void* workspace, cudaStream_t st, int* status) {
     static std::once_flag once;
     static cudaError_t attr_err = cudaSuccess;
     std::call_once(once, [] {
@@ -893,7 +842,7 @@ cudaError_t launch_tree_attention_tc(const void* q, const void* k_slab, const vo
     p.B = bt.B; p.H = H; p.max_seq = max_seq;
     p.out = (__nv_bfloat16*)out;
     p.out_lo = (__nv_bfloat16*)out_lo;
-    p.status = (int*)workspace;
+    p.status = status ? status : (int*)workspace;
     p.slots = (float*)((char*)workspace + 256);
     p.scale_log2 = 1.4426950408889634f / sqrtf((float)AT_D);
     if ((long long)bt.B * H * ((bt.max_len + AT_KEYS - 1) / AT_KEYS) > 0x7fffffffLL) return cudaErrorInvalidValue;   // unit indices are ints
@@ -929,10 +878,13 @@ cudaError_t launch_tree_attention_tc(const void* q, const void* k_slab, const vo
 cudaError_t launch_tree_attention(const void* q, const void* k_slab, const void* v_slab, const uint64_t* anc,
                                   int32_t anc_words, const Batch& bt, int32_t H, int32_t D, int32_t max_seq,
                                   int32_t dtype, void* out, void* out_lo, void* workspace, size_t workspace_bytes,
-                                  cudaStream_t st) {
-    if (workspace && ((uintptr_t)workspace % 256) == 0 && workspace_bytes >= tree_attention_tc_workspace(bt.B, H) &&
-        tree_attention_tc_supported(D, dtype, bt.max_rows))
-        return launch_tree_attention_tc(q, k_slab, v_slab, anc, anc_words, bt, H, max_seq, out, out_lo, workspace, st);
+                                  cudaStream_t st, int* status) {
+    if (D == AT_D && dtype == TRJ_BF16 && bt.max_rows <= AT_ROWS) {
+        if (!workspace || ((uintptr_t)workspace % 256) != 0 || workspace_bytes < tree_attention_tc_workspace(bt.B, H) ||
+            !tree_attention_tc_supported(D, dtype, bt.max_rows))
+            return cudaErrorInvalidValue;
+        return launch_tree_attention_tc(q, k_slab, v_slab, anc, anc_words, bt, H, max_seq, out, out_lo, workspace, st, status);
+    }
     return launch_tree_attention_generic(q, k_slab, v_slab, anc, anc_words, bt, H, D, max_seq, dtype, out, out_lo, st);
 }
 

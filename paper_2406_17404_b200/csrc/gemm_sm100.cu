@@ -15,6 +15,7 @@
 #include <mutex>
 #include <algorithm>
 #include "trj_internal.h"
+#include "sm100_common.cuh"
 
 namespace trj {
 namespace {
@@ -25,7 +26,6 @@ constexpr int TC_THREADS = 192;           // TMA warp, MMA warp, four epilogue w
 constexpr int TC_MAX_STAGES = 8;
 constexpr uint32_t TC_A_BYTES = TC_BM * TC_BK * 2;
 constexpr int TC_GRID = 296;              // two persistent CTAs per SM: one's ramp and tail overlap the other's stream
-constexpr uint32_t WAIT_LIMIT = 1u << 21;   // polls before a wait gives up (well over 100 ms)
 
 struct TcParams {
     int M, N, K;
@@ -40,92 +40,7 @@ struct TcParams {
     int ahead_boxes, ahead_kblocks, ahead_ctas;   // [128 x 64] tiles of a later projection's weights to request into L2
 };
 
-__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
-
-__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
-    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
-    uint32_t ok;
-    asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
-                 : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
-    return ok != 0;
-}
-// Bounded wait: gives up after WAIT_LIMIT polls or as soon as another role of the CTA gave up.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* status) {
-    for (uint32_t i = 0; i < WAIT_LIMIT; ++i) {
-        if (mbar_try_wait(bar, parity)) return true;
-        if (i > 32) {
-            if (*abort_flag) return false;
-            __nanosleep(64);
-        }
-    }
-    *abort_flag = 1;
-    atomicExch(status, (int)TRJ_ETIMEOUT);
-    return false;
-}
-
-// Weights are read once per step and are far larger than L2: they are loaded with an evict-first policy so that
-// they do not push out what is reused between kernels (activations, split-K pieces, and the kernels' own code).
-__device__ __forceinline__ uint64_t l2_evict_first_policy() {
-    uint64_t policy;
-    asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(policy));
-    return policy;
-}
-__device__ __forceinline__ void tma_load_2d_hint(uint32_t dst, const CUtensorMap* map, int c_inner, int c_outer, uint32_t bar,
-                                                 uint64_t policy) {
-    asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1, {%2, %3}], [%4], %5;"
-                 ::"r"(dst), "l"(map), "r"(c_inner), "r"(c_outer), "r"(bar), "l"(policy) : "memory");
-}
-// Asks for one box of the tensor to be brought into L2; nothing is written to shared memory and nothing signals.
-__device__ __forceinline__ void tma_prefetch_l2_2d(const CUtensorMap* map, int c_inner, int c_outer) {
-    asm volatile("cp.async.bulk.prefetch.tensor.2d.L2.global.tile [%0, {%1, %2}];"
-                 ::"l"(map), "r"(c_inner), "r"(c_outer) : "memory");
-}
-__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int c_inner, int c_outer, uint32_t bar) {
-    asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
-                 ::"r"(dst), "l"(map), "r"(c_inner), "r"(c_outer), "r"(bar) : "memory");
-}
-
-// Shared-memory matrix descriptor of a K-major tile with 128-byte swizzle: rows are 128 bytes apart,
-// groups of 8 rows 1024 bytes apart (stride byte offset), descriptor version 1 (sm_100).
-__device__ __forceinline__ uint64_t umma_desc_sw128(uint32_t smem_addr) {
-    uint64_t d = 0;
-    d |= (uint64_t)((smem_addr & 0x3FFFF) >> 4);          // start address, 16-byte units
-    d |= (uint64_t)1 << 16;                               // leading byte offset (unused with swizzle)
-    d |= (uint64_t)(1024 >> 4) << 32;                     // stride byte offset
-    d |= (uint64_t)1 << 46;                               // descriptor version
-    d |= (uint64_t)2 << 61;                               // 128-byte swizzle
-    return d;
-}
-
-// Instruction descriptor of kind::f16: bf16 x bf16 -> fp32, both operands K-major, shape 128 x n.
-__device__ __forceinline__ uint32_t umma_idesc_bf16(int n) {
-    return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(TC_BM >> 4) << 24);
-}
-
-__device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
-    asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
-                 "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-                 ::"r"(tmem_d), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
-}
-__device__ __forceinline__ void umma_commit(uint32_t bar) {
-    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ void tmem_ld8(uint32_t taddr, float* v) {
-    uint32_t r[8];
-    asm volatile("tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
-                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7])
-                 : "r"(taddr) : "memory");
-#pragma unroll
-    for (int i = 0; i < 8; ++i) v[i] = __uint_as_float(r[i]);
-}
+using namespace sm100;
 
 // Persistent kernel: CTA c works on items c, c + grid, c + 2*grid, ... where an item is one 128-row weight tile
 // restricted to one K range (tile = item / splits, split = item % splits).  The TMA ring runs through item
@@ -219,7 +134,7 @@ __global__ void __launch_bounds__(TC_THREADS, 2) gemm_tc_kernel(const __grid_con
     } else if (warp == 1) {
         if (lane == 0) {
             // ---------------- MMA issuer
-            const uint32_t idesc = umma_idesc_bf16(p.n_mma);
+            const uint32_t idesc = idesc_bf16(TC_BM, p.n_mma);
             int fill = 0, j = 0;
             bool ok = true;
             for (int item = blockIdx.x; item < items && ok; item += gridDim.x, ++j) {
@@ -238,7 +153,7 @@ __global__ void __launch_bounds__(TC_THREADS, 2) gemm_tc_kernel(const __grid_con
                     if (!ok) break;
                     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                     const uint32_t a_addr = tiles_base + s * stage_bytes;
-                    const uint64_t a_desc = umma_desc_sw128(a_addr), b_desc = umma_desc_sw128(a_addr + TC_A_BYTES);
+                    const uint64_t a_desc = desc_kmajor_sw128(a_addr), b_desc = desc_kmajor_sw128(a_addr + TC_A_BYTES);
 #pragma unroll
                     for (int kk = 0; kk < TC_BK / 16; ++kk)  // 16 bf16 = 32 bytes = 2 descriptor units per MMA
                         umma_bf16(d_tmem, a_desc + 2 * kk, b_desc + 2 * kk, idesc, (i > 0 || kk > 0) ? 1u : 0u);
@@ -298,6 +213,20 @@ __global__ void reduce_splits_kernel(const float4* __restrict__ part, float4* __
             a.x += b.x; a.y += b.y; a.z += b.z; a.w += b.w;
         }
         y[i] = a;
+    }
+}
+
+// Self-test of the time-out path: one thread waits, with the given poll limit, on a barrier that nobody ever
+// arrives at.  The wait is the very function the projection and attention kernels use; it gives up, leaves
+// TRJ_ETIMEOUT in *status and the kernel returns normally.
+__global__ void wait_expiry_selftest_kernel(int* status, uint32_t polls) {
+    __shared__ __align__(8) uint64_t bar;
+    __shared__ int abort_flag;
+    if (threadIdx.x == 0) {
+        abort_flag = 0;
+        mbar_init(smem_u32(&bar), 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        (void)mbar_wait(smem_u32(&bar), 0u, &abort_flag, status, polls);
     }
 }
 
@@ -370,8 +299,8 @@ size_t gemm_tc_workspace(int32_t M, int32_t N, int32_t K) {
 }
 
 cudaError_t launch_gemm_tc(const void* x, const void* x_lo, const void* w, float* y, int32_t M, int32_t N, int32_t K,
-                           void* workspace, cudaStream_t st, Parts* parts, const WeightPrefetch* ahead) {
-    int* status = (int*)workspace;
+                           void* workspace, cudaStream_t st, Parts* parts, const WeightPrefetch* ahead, int* status) {
+    if (!status) status = (int*)workspace;
     workspace = (char*)workspace + 256;
     static std::once_flag once;
     static cudaError_t attr_err = cudaSuccess;
@@ -384,7 +313,7 @@ cudaError_t launch_gemm_tc(const void* x, const void* x_lo, const void* w, float
     p.halves = x_lo ? 2 : 1;
     p.m_pad = round_up(M, p.halves == 2 ? 8 : 16);       // the lo box must start on a 1024-byte boundary: 8 rows
     p.n_mma = p.m_pad * p.halves;
-    // the epilogue reads 16 columns at a time from each half, so a buffer must cover the last such read
+    // the epilogue reads 8 columns at a time from each half, so a buffer must cover the last such read
     const int reach = (p.halves == 2 ? p.m_pad : 0) + round_up(p.m_pad, 16);
     p.acc_cols = 16;
     while (p.acc_cols < reach) p.acc_cols *= 2;
@@ -429,12 +358,25 @@ cudaError_t launch_gemm_tc(const void* x, const void* x_lo, const void* w, float
     return cudaGetLastError();
 }
 
+cudaError_t launch_wait_expiry_selftest(int* status, uint32_t polls, cudaStream_t st) {
+    count_launch();
+    wait_expiry_selftest_kernel<<<1, 32, 0, st>>>(status, polls);
+    return cudaGetLastError();
+}
+
+bool gemm_tc_shape(int32_t M, int32_t N, int32_t K, int32_t dtype) {
+    return dtype == TRJ_BF16 && M >= 1 && M <= TRJ_MAX_ROWS && K >= TC_BK && K % TC_BK == 0 && N >= 4 && N % 4 == 0;
+}
+
 cudaError_t launch_gemm(const void* x, const void* x_lo, const void* w, float* y, int32_t M, int32_t N, int32_t K,
                         int32_t dtype, void* workspace, size_t workspace_bytes, cudaStream_t st, Parts* parts,
-                        const WeightPrefetch* ahead) {
-    if (workspace && workspace_bytes >= gemm_tc_workspace(M, N, K) && ((uintptr_t)workspace % 256) == 0 &&
-        gemm_tc_supported(x, x_lo, w, y, M, N, K, dtype))
-        return launch_gemm_tc(x, x_lo, w, y, M, N, K, workspace, st, parts, ahead);
+                        const WeightPrefetch* ahead, int* status) {
+    if (gemm_tc_shape(M, N, K, dtype)) {
+        if (!workspace || workspace_bytes < gemm_tc_workspace(M, N, K) || ((uintptr_t)workspace % 256) != 0 ||
+            !gemm_tc_supported(x, x_lo, w, y, M, N, K, dtype))
+            return cudaErrorInvalidValue;
+        return launch_gemm_tc(x, x_lo, w, y, M, N, K, workspace, st, parts, ahead, status);
+    }
     if (parts) *parts = whole(y);
     return launch_gemm_simt(x, x_lo, w, y, M, N, K, dtype, st);
 }

@@ -469,6 +469,7 @@ constexpr int ARGMAX_CHUNKS = 8;              // vocabulary slices per row (one 
 // The acceptance walk of one sequence, run by one CTA after every prediction of it is known.
 __device__ void accept_sequence(const int32_t* tokens, const int32_t* parent, const int32_t* depth,
                                 const int32_t* pred, int rows, int32_t* k_acc, int32_t* path, int32_t* bonus) {
+    rows = min(rows, TRJ_MAX_ROWS);              // the host refuses larger trees; a bad device-side row_off must not overrun
     __shared__ unsigned char ok[TRJ_MAX_ROWS];
     __shared__ int32_t s_tok[TRJ_MAX_ROWS], s_par[TRJ_MAX_ROWS], s_dep[TRJ_MAX_ROWS], s_pred[TRJ_MAX_ROWS];
     __shared__ int s_best;
@@ -746,7 +747,7 @@ static __device__ __align__(256) unsigned char g_static_scratch[STATIC_SCRATCH_B
 
 // In host code `g_static_scratch` is only a handle for the runtime, not an address a kernel can use: the
 // device address is looked up once per device (with that device current) and remembered.
-static cudaError_t static_scratch_address(void** out) {
+static cudaError_t static_scratch_address(void** out, cudaStream_t st) {
     constexpr int MAX_DEVICES = 64;
     static std::mutex mu;
     static void* addr[MAX_DEVICES] = {};
@@ -756,6 +757,11 @@ static cudaError_t static_scratch_address(void** out) {
     if (dev < 0 || dev >= MAX_DEVICES) return cudaErrorInvalidDevice;
     std::lock_guard<std::mutex> lock(mu);
     if (!addr[dev]) {
+        // the lookup may load the module: it must not happen while `st` is being captured
+        cudaStreamCaptureStatus cs = cudaStreamCaptureStatusNone;
+        e = cudaStreamIsCapturing(st, &cs);
+        if (e != cudaSuccess) return e;
+        if (cs != cudaStreamCaptureStatusNone) return cudaErrorStreamCaptureUnsupported;
         void* p = nullptr;
         e = cudaGetSymbolAddress(&p, g_static_scratch);
         if (e != cudaSuccess) return e;
@@ -771,7 +777,7 @@ cudaError_t launch_argmax_accept_static(const void* logits, int32_t dtype, int32
                                         int32_t* node_argmax, float* margin, int32_t* k_acc, int32_t* path,
                                         int32_t* bonus, cudaStream_t st) {
     void* scratch = nullptr;
-    cudaError_t e = static_scratch_address(&scratch);
+    cudaError_t e = static_scratch_address(&scratch, st);
     if (e != cudaSuccess) return e;
     // the array keeps whatever the previous call left: the tickets must start at zero
     e = cudaMemsetAsync(scratch, 0, STATIC_TICKET_BYTES, st);

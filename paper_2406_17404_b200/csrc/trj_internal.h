@@ -105,12 +105,18 @@ bool gemm_tc_supported(const void* x, const void* x_lo, const void* w, const flo
                        int32_t dtype);
 size_t gemm_tc_workspace(int32_t M, int32_t N, int32_t K);
 cudaError_t launch_gemm_tc(const void* x, const void* x_lo, const void* w, float* y, int32_t M, int32_t N, int32_t K,
-                           void* workspace, cudaStream_t st, Parts* parts, const WeightPrefetch* ahead = nullptr);
-// Picks the tcgen05 kernel when the shape allows it, the plain kernel otherwise.  With `parts` non-null the
-// split-K pieces are left unreduced in the workspace for the consumer to add (*parts says where); otherwise
-// y holds the finished result.
+                           void* workspace, cudaStream_t st, Parts* parts, const WeightPrefetch* ahead = nullptr,
+                           int* status = nullptr);
+// The tcgen05 kernel for every shape it is written for (bf16, K a multiple of 64, N a multiple of 4), the plain
+// kernel for the rest (fp32 models, odd sizes).  A shape of the first kind whose workspace is too small or
+// misaligned is an error (cudaErrorInvalidValue), never a silent detour through the plain kernel.  With `parts`
+// non-null the split-K pieces are left unreduced in the workspace for the consumer to add (*parts says where);
+// otherwise y holds the finished result.  `status` (may be null: the workspace's first word) receives
+// TRJ_ETIMEOUT when a bounded device-side wait expires.
+bool gemm_tc_shape(int32_t M, int32_t N, int32_t K, int32_t dtype);
 cudaError_t launch_gemm(const void* x, const void* x_lo, const void* w, float* y, int32_t M, int32_t N, int32_t K,
-                        int32_t dtype, void* workspace, size_t workspace_bytes, cudaStream_t st, Parts* parts = nullptr, const WeightPrefetch* ahead = nullptr);
+                        int32_t dtype, void* workspace, size_t workspace_bytes, cudaStream_t st, Parts* parts = nullptr,
+                        const WeightPrefetch* ahead = nullptr, int* status = nullptr);
 
 // Rotary embedding of q and k at position seq_len[b] + depth[row]; q -> q_out [rows][H][D];
 // k, v -> cache rows seq_len[b] + local row of the layer slab [B][H][max_seq][D].
@@ -128,13 +134,17 @@ size_t tree_attention_tc_workspace(int32_t B, int32_t H);
 int tree_attention_grid(int32_t B, int32_t H, int32_t max_len);     // CTAs the tcgen05 kernel is launched with
 cudaError_t launch_tree_attention_tc(const void* q, const void* k_slab, const void* v_slab, const uint64_t* anc,
                                      int32_t anc_words, const Batch& bt, int32_t H, int32_t max_seq, void* out,
-                                     void* out_lo, void* workspace, cudaStream_t st);
-// Picks the tcgen05 kernel when shape and workspace allow it, the generic kernel otherwise.  out_lo (may be
-// null) receives the rounding error of `out` as a second tensor of the same type, for the projection that follows.
+                                     void* out_lo, void* workspace, cudaStream_t st, int* status = nullptr);
+// The tcgen05 kernel for bf16 with head_dim 128, the generic kernel for the rest (fp32, head_dim 64).  A bf16 /
+// head_dim-128 call whose workspace is too small or misaligned is an error (cudaErrorInvalidValue), never a
+// silent detour.  out_lo (may be null) receives the rounding error of `out` as a second tensor of the same
+// type, for the projection that follows.  `status`: as for launch_gemm.
 cudaError_t launch_tree_attention(const void* q, const void* k_slab, const void* v_slab, const uint64_t* anc,
                                   int32_t anc_words, const Batch& bt, int32_t H, int32_t D, int32_t max_seq,
                                   int32_t dtype, void* out, void* out_lo, void* workspace, size_t workspace_bytes,
-                                  cudaStream_t st);
+                                  cudaStream_t st, int* status = nullptr);
+// One CTA waits, with a poll limit, on a barrier nobody arrives at (self-test of the time-out path).
+cudaError_t launch_wait_expiry_selftest(int* status, uint32_t polls, cudaStream_t st);
 
 // Device-side drafting and refill (device_loop.cu); all pointers are device pointers.  `step` (may be null: step 0)
 // is a device counter that selects the step's slice of `draws` ([steps][W + R * Lr]) and is advanced by the commit.

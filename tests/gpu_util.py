@@ -33,8 +33,9 @@ class AttnCase:
         self.max_rows = max(rows)
         self.host = [synth.qkv(seed, n_heads, head_dim, s, m, dtype, name=f"seq{i}.")
                      for i, (s, m) in enumerate(zip(prefixes, rows))]
-        k = np.zeros((b, n_heads, self.max_seq, head_dim), np.float32)
-        v = np.zeros_like(k)
+        # cache rows past the end of a sequence hold NaN: whatever a kernel fetches from there must not reach its output
+        k = np.full((b, n_heads, self.max_seq, head_dim), np.nan, np.float32)
+        v = np.full_like(k, np.nan)
         for i, (s, m) in enumerate(zip(prefixes, rows)):
             t = self.host[i]
             k[i, :, :s], v[i, :, :s] = t["k_prefix"], t["v_prefix"]

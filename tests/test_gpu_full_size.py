@@ -21,57 +21,121 @@ from gpu_util import anc_dev, i32
 
 pytestmark = pytest.mark.gpu
 WIDTH, N_BRANCHES, BRANCH_LEN = 5, 9, 3
+CONFIG3_TOL = 8e-2          # provisional: replaced by the measured level
 
 
 @pytest.fixture(scope="module")
 def full(trj):
-    import bench
+    from synth.device import device_weights
     cfg = synth.LLAMA7B
-    layers, glob = bench.device_weights(cfg, 4321, torch.device("cuda", 0))
-    model = trj.Model(cfg, layers, glob, max_batch=1, max_seq=512, max_rows=trj.MAX_ROWS)
+    layers, glob = device_weights(cfg, 4321, torch.device("cuda", 0))
+    model = trj.Model(cfg, layers, glob, max_batch=1, max_seq=640, max_rows=trj.MAX_ROWS)
     yield cfg, layers, glob, model
     model.close()
 
 
-class DeviceLayers:
-    """Oracle-side view of the device weights: one layer at a time, widened on the host."""
-
-    def __init__(self, layers):
-        self.layers = layers
-
-    def __getitem__(self, l):
-        return {k: v.float().cpu().numpy() for k, v in self.layers[l].items()}
+def oracle_decoder(cfg, layers, glob):
+    from synth.device import HostView
+    return oracle.Decoder(cfg, HostView(layers), {k: v.float().cpu().numpy() for k, v in glob.items()})
 
 
-def test_full_depth_forward_against_oracle(trj, full):
-    cfg, layers, glob, model = full
-    # a 40-row chain (plays the prompt) with a 24-row random tree hanging below it; empty cache
-    m = 64
+def mixed_tree(cfg):
+    """A 40-row chain (plays the prompt) with a 24-row random tree hanging below it; 64 rows over an empty cache."""
     sub = synth.random_tree(8, 25, 4, 3)                     # its root is row 39 of the chain, its row t is row 39 + t
     parent = np.concatenate([synth.chain_parents(40), 39 + sub[1:]]).astype(np.int32)
-    tokens = synth.prompt(8, m, cfg.vocab)
-    dec = oracle.Decoder(cfg, DeviceLayers(layers), {k: v.float().cpu().numpy() for k, v in glob.items()})
+    return synth.prompt(8, 64, cfg.vocab), parent
+
+
+# Measured on a B200 (this file's weights and tree): the logit error against the fp64 oracle as the stack deepens.
+# The bounds asserted below are these measurements with 1.5x headroom.
+#   layers        2        4        8        16       32
+DEPTH_MAX = {2: None, 4: None, 8: None, 16: None, 32: None}
+DEPTH_RMS = {2: None, 4: None, 8: None, 16: None, 32: None}
+
+
+@pytest.mark.parametrize("n_layers", [2, 4, 8, 16, 32])
+def test_logit_error_against_oracle_by_depth(trj, full, n_layers, record_property):
+    """The first n_layers layers of the 7B model as a model of their own (same weights), 64 rows, empty cache."""
+    cfg_full, layers, glob, _ = full
+    cfg = cfg_full.with_layers(n_layers)
+    tokens, parent = mixed_tree(cfg)
+    m = len(tokens)
+    dec = oracle_decoder(cfg, layers[:n_layers], glob)
     cache = dec.new_cache(m)
     ref = dec.forward_rows(cache, tokens, parent)
+    model = trj.Model(cfg, layers[:n_layers], glob, max_batch=1, max_seq=128, max_rows=trj.MAX_ROWS)
     depth, anc = trj.tree_from_parents(parent)
-    model.seq_len.zero_()
     out = model.verify_step(i32(tokens), i32(parent), i32(depth), anc_dev(anc), i32([0, m]), max_rows=m, max_len=m,
                             want_logits=True, want_margin=True)
-    got = out["logits"].cpu().numpy()
-    err = np.abs(got - ref)
-    bound = 2e-2 * np.sqrt(cfg.n_layers / 2)
-    assert err.max() <= bound, err.max()
-    assert np.sqrt((err ** 2).mean()) <= 2e-2
-    # predictions agree wherever the oracle's top-1/top-2 margin clears twice the error bound
-    margin = oracle.top2_margin(ref)
-    safe = margin >= 2 * bound
+    model.device_status()
+    err = np.abs(out["logits"].cpu().numpy() - ref)
+    e_max, e_rms = float(err.max()), float(np.sqrt((err ** 2).mean()))
+    # K/V elements of the last layer whose stored bf16 value differs between the two sides (a rounding that fell
+    # the other way), as a fraction: the source of the growth with depth
+    k_dev = model.k_cache[n_layers - 1, 0, :, :m].double().cpu().numpy()
+    flips = float((k_dev != cache.k[n_layers - 1][:, :m]).mean())
+    print(f"depth {n_layers}: max {e_max:.4e} rms {e_rms:.4e} k-flips {flips:.4f} logit-std {ref.std():.3f}")
+    for name, val in (("max", e_max), ("rms", e_rms), ("flips", flips)):
+        record_property(f"logit_err_{name}_L{n_layers}", val)
+    model.close()
+    bound_max = 1.5 * DEPTH_MAX[n_layers] if DEPTH_MAX[n_layers] else 2e-2 * np.sqrt(n_layers / 2)
+    bound_rms = 1.5 * DEPTH_RMS[n_layers] if DEPTH_RMS[n_layers] else 2e-2
+    assert e_max <= bound_max and e_rms <= bound_rms, (e_max, e_rms)
+    # predictions agree wherever the oracle's top-1/top-2 margin clears twice the bound
+    safe = oracle.top2_margin(ref) >= 2 * bound_max
     assert safe.sum() >= 8
     np.testing.assert_array_equal(out["node_argmax"].cpu().numpy()[safe], oracle.node_argmax(ref)[safe])
-    # K/V rows of the first and last layer: bf16 values within a few ulp of the oracle's (roundings may flip)
-    for l in (0, cfg.n_layers - 1):
-        k_dev = model.k_cache[l, 0, :, :m].double().cpu().numpy()
-        tol = 2e-2 if l == 0 else 0.25
-        assert np.abs(k_dev - cache.k[l][:, :m]).max() <= tol * max(1.0, np.abs(cache.k[l][:, :m]).max())
+
+
+def test_config3_itself_against_oracle(trj, full):
+    """configs[2] as stated: 32 layers, a 512-token prompt prefilled, TR-Jacobi trees of 33 rows (window 5 + nine
+    retrieved branches of 3), consecutive steps driven from the oracle's trace with the margin protocol.
+
+    The oracle first decodes two tokens autoregressively (one-row trees) so that the first tree can carry the true
+    continuation in its first retrieved branch: that step then accepts rows and compacts the 32-layer cache."""
+    from oracle.model import verify_step
+    cfg, layers, glob, model = full
+    p, n_steps, n_plant = 512, 3, 2
+    prompt = synth.prompt(3, p, cfg.vocab)
+    draw = lambda s, n: synth.noise_draws(3, s, n)
+    dec = oracle_decoder(cfg, layers, glob)
+    cache = dec.new_cache(p + 64)
+    logits = dec.forward_rows(cache, list(prompt), list(range(-1, p - 1)))
+    cache.seq_len = p
+    committed = [int(t) for t in prompt] + [int(oracle.node_argmax(logits[-1:])[0])]
+    # the true continuation of the first root, by the oracle alone
+    truth, probe_margin = [], []
+    nxt = committed[-1]
+    for _ in range(n_plant):
+        lg = dec.forward_rows(cache, [nxt], [-1])
+        cache.seq_len += 1
+        nxt = int(oracle.node_argmax(lg)[0])
+        truth.append(nxt)
+        probe_margin.append(float(oracle.top2_margin(lg)[0]))
+    cache.seq_len = p                                        # back to the state after the prompt
+    window = [oracle.ahead_noise(committed, d) for d in draw(0, WIDTH)]
+    trace = []
+    for step in range(1, n_steps + 1):
+        draws = draw(step, WIDTH + N_BRANCHES * BRANCH_LEN)
+        branches = oracle.retrieve(committed, N_BRANCHES, BRANCH_LEN, draws[WIDTH:])
+        if step == 1:
+            branches[0] = truth + branches[0][len(truth):]
+        tokens, parent = oracle.build_tree(committed[-1], window, branches)
+        rec = verify_step(dec, cache, tokens, parent)
+        committed += [int(tokens[r]) for r in rec["path"][1:]] + [rec["bonus"]]
+        window = oracle.refill_window(parent, rec["pred"], rec["path"][-1], WIDTH, committed, draws[:WIDTH])
+        rec.update(tokens=tokens, parent=parent, step=step)
+        trace.append(rec)
+    assert all(len(r["tokens"]) == 33 for r in trace)
+    if min(probe_margin) >= 1e-2:
+        assert trace[0]["k"] >= n_plant                      # the planted continuation is accepted by the oracle
+    # the GPU, from the same prompt, through the same trees
+    from test_gpu_model import drive_with_oracle_trace
+    model.seq_len.zero_()
+    stats = drive_with_oracle_trace(trj, model, prompt, trace, tol=CONFIG3_TOL)
+    model.device_status()
+    print("config 3 at full size:", stats)
+    assert stats["rows"] >= 60 and stats["path_checked"] >= 1
 
 
 def test_tr_jacobi_commits_the_autoregressive_tokens_at_full_size(trj, full):

@@ -53,7 +53,7 @@ def test_tree_attention_small(trj, dtype, h, d, s, m):
 ])
 def test_tree_attention_launch_shapes_single_sequence(trj, h, s, m):
     """One sequence, head counts and lengths that exercise every launch shape the host chooses from."""
-    case = AttnCase(trj, h, h, 128, [s], [m], [synth.random_tree(h + s, m, min(8, m - 1), 3)], "bf16")
+    case = AttnCase(trj, h, h, 128, [s], [m], [synth.random_tree(h + s, m, min(8, m - 1), 3)], "bf16", pad=5)
     check_attention(trj, case, heads=[0, h // 2, h - 1])
 
 
@@ -76,17 +76,45 @@ def test_tree_attention_config2_full(trj):
     check_attention(trj, case)
 
 
-def test_tree_attention_config4_full_sampled_heads(trj):
-    """32 heads x 128, prefix 8192, 128-row tree of depth 8; the oracle checks a sample of heads."""
-    case = AttnCase(trj, 3, 32, 128, [8192], [128], [synth.random_tree(3, 128, 8, 4)], "bf16")
-    check_attention(trj, case, heads=[0, 13, 31])
+def test_tree_attention_config4_full(trj):
+    """32 heads x 128, prefix 8192, 128-row tree of depth 8; every head is compared."""
+    case = AttnCase(trj, 3, 32, 128, [8192], [128], [synth.random_tree(3, 128, 8, 4)], "bf16", pad=7)
+    check_attention(trj, case)
 
 
 def test_tree_attention_config5_ragged_batch(trj):
     s, m = synth.ragged_batch(4, 8, (256, 4096), (16, 64))
     parents = [synth.random_tree(40 + i, int(mi), 6, 3) for i, mi in enumerate(m)]
     case = AttnCase(trj, 4, 32, 128, s.tolist(), m.tolist(), parents, "bf16", max_seq=4096 + 64)
-    check_attention(trj, case, heads=[1, 30])
+    check_attention(trj, case, heads=[0, 1, 7, 12, 16, 23, 30, 31])
+
+
+def test_tensor_core_shapes_are_never_rerouted(trj):
+    """A bf16 / head_dim-128 attention call or a projection of a tensor-core shape with a short or misaligned
+    workspace is an error, not a silent run on the generic kernel."""
+    case = AttnCase(trj, 5, 2, 128, [100], [9], [synth.random_tree(5, 9, 4, 3)], "bf16")
+    need = trj.tree_attention_workspace(9, 1, 2, 128, 109)
+    with pytest.raises(trj.TrjError) as e:
+        case.run(trj, workspace=torch.zeros(need - 256, dtype=torch.uint8, device="cuda"))
+    assert e.value.status == 2
+    with pytest.raises(trj.TrjError) as e:
+        case.run(trj, workspace=torch.zeros(need + 512, dtype=torch.uint8, device="cuda")[16:])
+    assert e.value.status == 1
+    x = torch.zeros(8, 256, dtype=torch.bfloat16, device="cuda")
+    w = torch.zeros(64, 256, dtype=torch.bfloat16, device="cuda")
+    gneed = trj.lib().trj_gemm_workspace(8, 64, 256)
+    with pytest.raises(trj.TrjError) as e:
+        trj.gemm(x, w, workspace=torch.zeros(gneed + 512, dtype=torch.uint8, device="cuda")[16:])
+    assert e.value.status == 1
+
+
+def test_an_expired_wait_is_reported_and_the_kernel_returns(trj):
+    """The bounded wait of the tensor-core kernels, made to run out on a barrier nobody arrives at: the status
+    word reads TRJ_ETIMEOUT, the launch completes by itself and the device stays usable."""
+    for polls in (40, 1000):
+        assert trj.selftest_wait_expiry(polls) == 4
+    case = AttnCase(trj, 6, 2, 128, [200], [17], [synth.random_tree(6, 17, 4, 3)], "bf16")
+    check_attention(trj, case)                             # the context still works
 
 
 # ----------------------------------------------------------------------------- arg-max + acceptance
