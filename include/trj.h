@@ -349,6 +349,15 @@ trj_status trj_decode_device(trj_ctx* ctx, void* k_cache, void* v_cache, int32_t
                              int32_t R, int32_t branch_len, const int64_t* draws, int32_t n_steps,
                              int32_t* k_log, void* stream);
 
+/* An external source of drafts for trj_decode_device (Section 3.3: retrieved drafts get a path of their own; where
+ * they are retrieved from is open).  stream [n] (dev int32) holds the source's guess for the token at context
+ * position i in stream[i]; in step s of a later trj_decode_device call the first take[s] (dev int32 [n_steps],
+ * clipped to branch_len and to n) tokens of retrieved branch 0 come from stream, starting at the position after
+ * the root, instead of from prompt lookup.  Borrowed until replaced; stream == NULL removes the source.  With
+ * guesses of a known quality this sets how many drafts a step accepts: the benchmark uses it to run the loop at
+ * the acceptance lengths the paper reports instead of the zero of random drafts on random weights. */
+trj_status trj_set_draft_source(trj_ctx* ctx, const int32_t* stream, int32_t n, const int32_t* take, int32_t n_steps);
+
 /* ------------------------------------------------------------------------
  * The projections as a stand-alone op: y[M][N] (fp32) = x[M][K] . w[N][K]^T,
  * x and w of `dtype`, all dev.  Used by the model path for every projection

@@ -77,6 +77,7 @@ _SIGNATURES = {
     "trj_draft_tokens": (_I, [_VP, _VP, _VP, _I, _I, _I, _VP, _VP, _VP]),
     "trj_commit_refill": (_I, [_VP, _VP, _VP, _I, _VP, _VP, _VP, _VP, _I, _VP, _I, _VP, _VP, _VP, _VP]),
     "trj_decode_device": (_I, [_VP, _VP, _VP, _VP, _VP, _I, _VP, _I, _VP, _I, _I, _I, _VP, _I, _VP, _VP]),
+    "trj_set_draft_source": (_I, [_VP, _VP, _I, _VP, _I]),
     "trj_gemm_workspace": (_SZ, [_I, _I, _I]),
     "trj_gemm": (_I, [_VP, _VP, _VP, _I, _I, _I, _I, _VP, _SZ, _VP]),
     "trj_device_status": (_I, [_VP, _I, _VP]),
@@ -265,6 +266,21 @@ def argmax_accept(logits, tokens, parent, depth, row_off, *, want_margin: bool =
         batch, rows, _dev(node_argmax), _dev(margin) if want_margin else None, _dev(k_acc), _dev(path), _dev(bonus),
         _dev(workspace, torch.uint8, "workspace"), workspace.numel(), _stream(stream)))
     return {"node_argmax": node_argmax, "margin": margin, "k_acc": k_acc, "path": path, "bonus": bonus}
+
+
+def argmax_accept_into(logits, tokens, parent, depth, row_off, out, workspace, *, stream=None) -> None:
+    """trj_argmax_accept into preallocated outputs (``out`` as for :func:`argmax_accept_static`) with a caller-held,
+    zero-initialised workspace: nothing is allocated, so the call can be captured in a CUDA graph."""
+    torch = _torch()
+    rows, vocab = logits.shape
+    batch = row_off.numel() - 1
+    margin = out.get("margin")
+    _check(lib().trj_argmax_accept(
+        _dev(logits, name="logits"), _dtype_code(logits), vocab, _dev(tokens, torch.int32, "tokens"),
+        _dev(parent, torch.int32, "parent"), _dev(depth, torch.int32, "depth"), _dev(row_off, torch.int32, "row_off"),
+        batch, rows, _dev(out["node_argmax"], torch.int32), _dev(margin, torch.float32) if margin is not None else None,
+        _dev(out["k_acc"], torch.int32), _dev(out["path"], torch.int32), _dev(out["bonus"], torch.int32),
+        _dev(workspace, torch.uint8, "workspace"), workspace.numel(), _stream(stream)))
 
 
 STATIC_MAX_ROWS = 1024
@@ -475,6 +491,18 @@ class Model:
                                        _dev(window, torch.int32, "window") if w else None, w, n_branches, branch_len,
                                        _dev(draws, torch.int64, "draws"), int(n_steps),
                                        _dev(k_log, torch.int32, "k_log") if k_log is not None else None, _stream(stream)))
+
+    def set_draft_source(self, stream=None, take=None) -> None:
+        """trj_set_draft_source: ``stream`` int32 [n] guesses by context position, ``take`` int32 [n_steps] how many
+        of them each step of the next decode_device call plants into branch 0 (CUDA tensors, kept alive here);
+        ``None`` removes the source."""
+        torch = _torch()
+        self._draft_src = (stream, take)
+        if stream is None:
+            _check(lib().trj_set_draft_source(self._handle, None, 0, None, 0))
+        else:
+            _check(lib().trj_set_draft_source(self._handle, _dev(stream, torch.int32, "stream"), int(stream.numel()),
+                                              _dev(take, torch.int32, "take"), int(take.numel())))
 
     def step_host(self, root: int, window, branches, max_len: int, stream=None) -> Dict[str, object]:
         """trj_step_host: one whole decode step from host integers; returns host results."""

@@ -162,6 +162,7 @@ struct trj_ctx {
     struct LoopGraph { std::vector<uint64_t> key; cudaGraphExec_t exec; };
     std::vector<LoopGraph> loop_graphs;
     cudaStream_t cap_stream = nullptr; cudaEvent_t order_ev = nullptr; uint64_t steps_done = 0;
+    DraftSource draft_src{nullptr, 0, nullptr}; int32_t draft_src_steps = 0;   // trj_set_draft_source
 };
 
 namespace {
@@ -661,6 +662,15 @@ extern "C" trj_status trj_commit_refill(const int32_t* tokens, const int32_t* pa
     return TRJ_OK;
 }
 
+extern "C" trj_status trj_set_draft_source(trj_ctx* ctx, const int32_t* stream, int32_t n, const int32_t* take, int32_t n_steps) {
+    TRJ_REQUIRE(ctx, TRJ_EINVAL, "set_draft_source: null context");
+    if (!stream) { ctx->draft_src = DraftSource{nullptr, 0, nullptr}; ctx->draft_src_steps = 0; return TRJ_OK; }
+    TRJ_REQUIRE(take && n >= 0 && n_steps >= 0, TRJ_EINVAL, "set_draft_source: null take or negative size");
+    ctx->draft_src = DraftSource{stream, n, take};
+    ctx->draft_src_steps = n_steps;
+    return TRJ_OK;
+}
+
 extern "C" trj_status trj_decode_device(trj_ctx* ctx, void* k_cache, void* v_cache, int32_t* seq_len, int32_t* context,
                                         int32_t capacity, int32_t* n_ctx, int32_t n_ctx_now, int32_t* window, int32_t W,
                                         int32_t R, int32_t branch_len, const int64_t* draws, int32_t n_steps,
@@ -681,6 +691,8 @@ extern "C" trj_status trj_decode_device(trj_ctx* ctx, void* k_cache, void* v_cac
     // the cache holds every committed token but the last one (the next root) and, during a step, the tree rows
     const int64_t max_len = (int64_t)n_ctx_now - 1 + (int64_t)n_steps * per_step + M;
     TRJ_REQUIRE(max_len <= c.max_seq, TRJ_ECAPACITY, "decode_device: up to %lld cache rows exceed max_seq %d", (long long)max_len, c.max_seq);
+    TRJ_REQUIRE(!ctx->draft_src.stream || ctx->draft_src_steps >= n_steps, TRJ_ECAPACITY,
+                "decode_device: the draft source covers %d steps, %d asked", ctx->draft_src_steps, n_steps);
     trj_status s = check_step_args(ctx, 1, M, M, (int32_t)max_len, 2);
     if (s != TRJ_OK) return s;
     if (n_steps == 0) return TRJ_OK;
@@ -709,7 +721,8 @@ extern "C" trj_status trj_decode_device(trj_ctx* ctx, void* k_cache, void* v_cac
     Batch bt{seq_len, d_off, 1, M, M, (int32_t)max_len};
     auto enqueue_one = [&](cudaStream_t on) -> trj_status {
         ChainScope chain;
-        LAUNCH_ON(on, PROF_ELEMENTWISE, launch_draft_tokens(context, n_ctx, window, W, R, branch_len, draws, d_step, d_tokens, on));
+        LAUNCH_ON(on, PROF_ELEMENTWISE, launch_draft_tokens(context, n_ctx, window, W, R, branch_len, draws, d_step, d_tokens, on,
+                                                            ctx->draft_src));
         trj_status fs = forward(ctx, k_cache, v_cache, 0, bt, d_tokens, d_depth, d_anc, 2, 0, M, on);
         if (fs != TRJ_OK) return fs;
         LAUNCH_ON(on, PROF_ARGMAX, launch_argmax_accept(ctx->logits, TRJ_F32, c.vocab, d_tokens, d_parent, d_depth, d_off, 1, M, d_pred,
@@ -737,7 +750,9 @@ extern "C" trj_status trj_decode_device(trj_ctx* ctx, void* k_cache, void* v_cac
                                            (uint64_t)(uintptr_t)k_cache, (uint64_t)(uintptr_t)v_cache, (uint64_t)(uintptr_t)seq_len,
                                            (uint64_t)(uintptr_t)context, (uint64_t)capacity, (uint64_t)(uintptr_t)n_ctx,
                                            (uint64_t)(uintptr_t)window, (uint64_t)W, (uint64_t)R, (uint64_t)branch_len,
-                                           (uint64_t)(uintptr_t)draws, (uint64_t)(uintptr_t)k_log, (uint64_t)max_len};
+                                           (uint64_t)(uintptr_t)draws, (uint64_t)(uintptr_t)k_log, (uint64_t)max_len,
+                                           (uint64_t)(uintptr_t)ctx->draft_src.stream, (uint64_t)ctx->draft_src.n,
+                                           (uint64_t)(uintptr_t)ctx->draft_src.take};
         cudaGraphExec_t exec = nullptr;
         for (const trj_ctx::LoopGraph& g : ctx->loop_graphs)
             if (g.key == key) exec = g.exec;

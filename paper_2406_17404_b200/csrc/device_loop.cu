@@ -14,10 +14,12 @@ constexpr int MAX_BRANCHES = 64;          // R is bounded by the tree size (R * 
 // tokens[0] = root (last committed token), tokens[1..W] = window, then R branches of Lr tokens: for each of the R
 // most recent earlier occurrences of the context's last two tokens (then of its last token), the Lr tokens that
 // followed; missing slots are ahead noise, context[draw % n].  `step` (may be null) selects this step's draws.
+// An external draft source (may be absent) overrides the start of branch 0: src.stream[i] is its guess for the token
+// at context position i, and step s takes src.take[s] of them, from position n on.
 __global__ void __launch_bounds__(32) draft_tokens_kernel(const int32_t* __restrict__ context, const int32_t* __restrict__ n_ctx,
                                                           const int32_t* __restrict__ window, int W, int R, int Lr,
                                                           const int64_t* __restrict__ draws, const int32_t* __restrict__ step,
-                                                          int32_t* __restrict__ tokens) {
+                                                          int32_t* __restrict__ tokens, const DraftSource src) {
     pdl_prologue();
     const int lane = threadIdx.x;
     const int n = *n_ctx;
@@ -50,6 +52,7 @@ __global__ void __launch_bounds__(32) draft_tokens_kernel(const int32_t* __restr
         int32_t tok;
         if (r < nf && follow[r] + j < n) tok = context[follow[r] + j];
         else tok = context[(uint64_t)my_draws[W + slot] % (uint64_t)n];
+        if (src.stream && r == 0 && j < src.take[step ? *step : 0] && n + j < src.n) tok = src.stream[n + j];
         tokens[1 + W + slot] = tok;
     }
 }
@@ -98,10 +101,11 @@ __global__ void __launch_bounds__(32) commit_refill_kernel(const int32_t* __rest
 }  // namespace
 
 cudaError_t launch_draft_tokens(const int32_t* context, const int32_t* n_ctx, const int32_t* window, int32_t W, int32_t R,
-                                int32_t Lr, const int64_t* draws, const int32_t* step, int32_t* tokens, cudaStream_t st) {
+                                int32_t Lr, const int64_t* draws, const int32_t* step, int32_t* tokens, cudaStream_t st,
+                                const DraftSource& src) {
     if (R > MAX_BRANCHES) return cudaErrorInvalidValue;
     count_launch();
-    cudaError_t e = launch_chain(draft_tokens_kernel, dim3(1), dim3(32), 0, st, context, n_ctx, window, W, R, Lr, draws, step, tokens);
+    cudaError_t e = launch_chain(draft_tokens_kernel, dim3(1), dim3(32), 0, st, context, n_ctx, window, W, R, Lr, draws, step, tokens, src);
     return e != cudaSuccess ? e : cudaGetLastError();
 }
 

@@ -148,8 +148,12 @@ cudaError_t launch_wait_expiry_selftest(int* status, uint32_t polls, cudaStream_
 
 // Device-side drafting and refill (device_loop.cu); all pointers are device pointers.  `step` (may be null: step 0)
 // is a device counter that selects the step's slice of `draws` ([steps][W + R * Lr]) and is advanced by the commit.
+// An external source of drafts for the decode loop: stream[i] (i < n) is its guess for the token at context position
+// i; take[s] is how many of them step s puts at the start of retrieved branch 0.  stream == nullptr: none.
+struct DraftSource { const int32_t* stream; int32_t n; const int32_t* take; };
 cudaError_t launch_draft_tokens(const int32_t* context, const int32_t* n_ctx, const int32_t* window, int32_t W, int32_t R,
-                                int32_t Lr, const int64_t* draws, const int32_t* step, int32_t* tokens, cudaStream_t st);
+                                int32_t Lr, const int64_t* draws, const int32_t* step, int32_t* tokens, cudaStream_t st,
+                                const DraftSource& src = DraftSource{nullptr, 0, nullptr});
 cudaError_t launch_commit_refill(const int32_t* tokens, const int32_t* parent, const int32_t* node_argmax, int32_t M,
                                  const int32_t* k_acc, const int32_t* path, const int32_t* bonus, int32_t* context,
                                  int32_t capacity, int32_t* n_ctx, int32_t W, int32_t draws_per_step, const int64_t* draws,
