@@ -40,7 +40,8 @@
  *            that is TRJ_ECAPACITY / TRJ_EINVAL.
  * Layouts    All tensors are dense, row-major, innermost dimension last.
  *            dtype is TRJ_BF16 (bf16 storage, fp32 accumulation) or TRJ_F32.
- *            KV cache: [L][B][H][max_seq][D]; sequence b has seq_len[b]
+ *            KV cache: [L][B][Hkv][max_seq][D] (Hkv = K/V heads: H, or fewer with
+ *            grouped-query attention); sequence b has seq_len[b]
  *            committed rows; during a step the M_b tree rows of sequence b
  *            live at cache rows seq_len[b] .. seq_len[b] + M_b - 1.
  * Trees      A tree is a parent-pointer array in topological order:
@@ -81,24 +82,29 @@ typedef enum { TRJ_F32 = 0, TRJ_BF16 = 1 } trj_dtype;
 typedef struct trj_ctx trj_ctx;    /* opaque model context */
 
 /* LLaMA-family decoder shape: pre-norm, RMSNorm, rotary embedding (half-split
- * pairing, base rope_theta), multi-head attention, SwiGLU, untied LM head. */
+ * pairing, base rope_theta), multi-head or grouped-query attention, SwiGLU,
+ * untied LM head.  The paper's main models (Table 2) are of the LLaMA-3 family:
+ * grouped-query attention (n_kv_heads = 8 for 32 query heads) and a 128 256-way
+ * vocabulary. */
 typedef struct {
     int32_t n_layers, d_model, n_heads, head_dim, d_ff, vocab;
     float   rms_eps, rope_theta;
     int32_t dtype;                 /* trj_dtype of weights, activations and cache */
     int32_t max_batch, max_seq, max_rows;   /* capacities the workspace is sized for */
+    int32_t n_kv_heads;            /* K/V heads; 0 = n_heads; must divide n_heads: query head h
+                                      reads K/V head h / (n_heads / n_kv_heads)              */
 } trj_model_cfg;
 
 /* Device pointers to the weights, borrowed for the lifetime of the context.
  * Every matrix is [d_out][d_in].  The per-layer members are HOST arrays of
- * n_layers device pointers.  wqkv stacks Wq, Wk, Wv rows; w_gate_up stacks the
+ * n_layers device pointers.  wqkv stacks Wq (H*D rows), Wk, Wv (Hkv*D rows each); w_gate_up stacks the
  * SwiGLU gate rows over the up rows.  Norm gains are fp32 vectors [d_model]. */
 typedef struct {
     const void*  embed;            /* [vocab][d_model]  dtype                     */
     const void*  lm_head;          /* [vocab][d_model]  dtype                     */
     const float* final_norm;       /* [d_model]                                   */
     const float* const* attn_norm; /* [L] -> [d_model]                            */
-    const void*  const* wqkv;      /* [L] -> [3*H*D][d_model]                     */
+    const void*  const* wqkv;      /* [L] -> [(H+2*Hkv)*D][d_model]               */
     const void*  const* wo;        /* [L] -> [d_model][H*D]                       */
     const float* const* mlp_norm;  /* [L] -> [d_model]                            */
     const void*  const* w_gate_up; /* [L] -> [2*d_ff][d_model]                    */
@@ -173,6 +179,14 @@ trj_status trj_tree_attention(const void* q, const void* k_cache, const void* v_
                               int32_t anc_words, int32_t B, int32_t rows_total, int32_t max_rows,
                               int32_t H, int32_t D, int32_t max_seq, int32_t max_len, int32_t dtype,
                               void* out, void* workspace, size_t workspace_bytes, void* stream);
+/* The same with grouped-query attention (LLaMA-3 family, Table 2): H query heads over Hkv K/V heads, H a
+ * multiple of Hkv; k_cache / v_cache are [B][Hkv][max_seq][D] and query head h reads K/V head h / (H / Hkv).
+ * Hkv == H is trj_tree_attention. */
+trj_status trj_tree_attention_gqa(const void* q, const void* k_cache, const void* v_cache,
+                                  const int32_t* seq_len, const int32_t* row_off, const uint64_t* anc,
+                                  int32_t anc_words, int32_t B, int32_t rows_total, int32_t max_rows,
+                                  int32_t H, int32_t Hkv, int32_t D, int32_t max_seq, int32_t max_len, int32_t dtype,
+                                  void* out, void* workspace, size_t workspace_bytes, void* stream);
 
 /* ------------------------------------------------------------------------
  * Per-node arg-max fused with greedy longest-path acceptance (Eq. 1; Section
@@ -236,7 +250,8 @@ trj_status trj_argmax_accept_static(const void* logits, int32_t dtype, int32_t V
  * V, row seq_len[b] + path[b][j] moves to row seq_len[b] + j, j = 1..k_acc[b]
  * (row 0, the root, is already in place); then seq_len[b] += k_acc[b] + 1.
  * Bit-exact copy; source and destination ranges may overlap.
- *   k_cache, v_cache  dev [L][B][H][max_seq][D] dtype, modified in place
+ *   k_cache, v_cache  dev [L][B][H][max_seq][D] dtype, modified in place (H = heads of the cache: the
+ *                     K/V heads of a grouped-query model)
  *   seq_len dev [B] (updated);  k_acc dev [B];  path dev [B][TRJ_PATH_STRIDE] */
 trj_status trj_compact_rows(void* k_cache, void* v_cache, int32_t L, int32_t B, int32_t H,
                             int32_t max_seq, int32_t D, int32_t dtype, int32_t* seq_len,
@@ -246,7 +261,7 @@ trj_status trj_compact_rows(void* k_cache, void* v_cache, int32_t L, int32_t B, 
  * Model context: the whole verification step of a LLaMA-shaped decoder.
  * workspace: dev, >= trj_workspace_bytes(cfg), 256-byte aligned, zero-filled by
  * the caller before trj_create, owned by the caller, used by every call on ctx.
- * The cache passed to the calls below is [n_layers][max_batch][H][max_seq][D]. */
+ * The cache passed to the calls below is [n_layers][max_batch][Hkv][max_seq][D]. */
 size_t     trj_workspace_bytes(const trj_model_cfg* cfg);
 trj_status trj_create(const trj_model_cfg* cfg, const trj_weights* weights,
                       void* workspace, size_t workspace_bytes, trj_ctx** out);

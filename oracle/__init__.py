@@ -26,7 +26,9 @@ cannot change which tokens a greedy decoder commits, unless noted):
 * Model.  The paper names LLaMA-family 7-8B decoders but prints no
   architecture.  Used here: pre-norm decoder, RMSNorm (eps 1e-5), rotary
   embedding with the half-split pairing (i, i + D/2) and base 10000, multi-head
-  attention scaled by 1/sqrt(D), SwiGLU MLP, no biases, untied LM head.
+  attention scaled by 1/sqrt(D), SwiGLU MLP, no biases, untied LM head.  With
+  grouped-query attention (LLaMA-3 family, Table 2) query head h reads K/V
+  head h // (H / Hkv).
 * Tree layout (Section 3.3, Appendix B).  The concrete 63-node template is a
   third-party artefact that the paper does not print; any parent-pointer tree
   with parent[i] < i is accepted.  ``build_tree`` lays out row 0 = root (the

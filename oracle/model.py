@@ -47,7 +47,7 @@ def store_bf16(x: np.ndarray) -> np.ndarray:
 
 
 class KVCache:
-    """K and V of every layer, [L, H, capacity, D] fp64, and the number of committed rows."""
+    """K and V of every layer, [L, Hkv, capacity, D] fp64, and the number of committed rows."""
 
     def __init__(self, n_layers: int, n_heads: int, capacity: int, head_dim: int):
         self.k = np.zeros((n_layers, n_heads, capacity, head_dim), np.float64)
@@ -71,7 +71,7 @@ class Decoder:
 
     def new_cache(self, capacity: int) -> KVCache:
         c = self.cfg
-        return KVCache(c.n_layers, c.n_heads, capacity, c.head_dim)
+        return KVCache(c.n_layers, getattr(c, "kv_heads", c.n_heads), capacity, c.head_dim)
 
     def forward_rows(self, cache: KVCache, tokens: Sequence[int], parent: Sequence[int]) -> np.ndarray:
         """Logits [M, V] of the M tree rows given the cache's first ``seq_len`` rows.
@@ -82,6 +82,7 @@ class Decoder:
         c = self.cfg
         m, s = len(tokens), cache.seq_len
         n_heads, hd = c.n_heads, c.head_dim
+        kv_heads = getattr(c, "kv_heads", n_heads)          # grouped-query attention when smaller than n_heads
         pos = s + depths(parent)
         # bf16 configs: q and the K/V cache rows are bf16 tensors (the cache is stored in bf16 by the
         # config's definition and q is the other operand of the attention op); what such a tensor holds
@@ -92,8 +93,10 @@ class Decoder:
             w = self.layers[l]
             x = rmsnorm(h, np.asarray(w["attn_norm"], np.float64), c.rms_eps)
             qkv = x @ np.asarray(w["wqkv"], np.float64).T
-            q, k, v = (qkv[:, j * n_heads * hd:(j + 1) * n_heads * hd].reshape(m, n_heads, hd)
-                       for j in range(3))
+            nq, nkv = n_heads * hd, kv_heads * hd
+            q = qkv[:, :nq].reshape(m, n_heads, hd)
+            k = qkv[:, nq:nq + nkv].reshape(m, kv_heads, hd)
+            v = qkv[:, nq + nkv:].reshape(m, kv_heads, hd)
             q, k, v = store(rope(q, pos, c.rope_theta)), store(rope(k, pos, c.rope_theta)), store(v)
             cache.k[l][:, s:s + m, :] = k.transpose(1, 0, 2)
             cache.v[l][:, s:s + m, :] = v.transpose(1, 0, 2)

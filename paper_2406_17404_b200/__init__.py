@@ -38,7 +38,7 @@ class TrjError(RuntimeError):
 class ModelCfg(C.Structure):
     _fields_ = [(n, C.c_int32) for n in ("n_layers", "d_model", "n_heads", "head_dim", "d_ff", "vocab")] + \
                [("rms_eps", C.c_float), ("rope_theta", C.c_float)] + \
-               [(n, C.c_int32) for n in ("dtype", "max_batch", "max_seq", "max_rows")]
+               [(n, C.c_int32) for n in ("dtype", "max_batch", "max_seq", "max_rows", "n_kv_heads")]
 
 
 class Weights(C.Structure):
@@ -61,6 +61,7 @@ _SIGNATURES = {
     "trj_refill_window": (_I, [_I32P, _I32P, _I, _I, _I, _I32P, _I, _I64P, _I32P]),
     "trj_tree_attention_workspace": (_SZ, [_I, _I, _I, _I, _I]),
     "trj_tree_attention": (_I, [_VP, _VP, _VP, _VP, _VP, _VP, _I, _I, _I, _I, _I, _I, _I, _I, _I, _VP, _VP, _SZ, _VP]),
+    "trj_tree_attention_gqa": (_I, [_VP, _VP, _VP, _VP, _VP, _VP, _I, _I, _I, _I, _I, _I, _I, _I, _I, _I, _VP, _VP, _SZ, _VP]),
     "trj_argmax_accept_workspace": (_SZ, [_I, _I]),
     "trj_argmax_accept": (_I, [_VP, _I, _I, _VP, _VP, _VP, _VP, _I, _I, _VP, _VP, _VP, _VP, _VP, _VP, _SZ, _VP]),
     "trj_argmax_accept_static": (_I, [_VP, _I, _I, _VP, _VP, _VP, _VP, _I, _I, _VP, _VP, _VP, _VP, _VP, _VP]),
@@ -223,21 +224,26 @@ def tree_attention_workspace(rows_total: int, batch: int, n_heads: int, head_dim
 
 def tree_attention(q, k_cache, v_cache, seq_len, row_off, anc, *, max_rows: int, max_len: int,
                    out=None, workspace=None, stream=None):
-    """trj_tree_attention.  q [rows, H, D]; k/v_cache [B, H, max_seq, D]; seq_len [B]; row_off [B+1];
-    anc [rows, anc_words] (int64 view of the u64 words).  Returns out [rows, H, D]."""
+    """trj_tree_attention (trj_tree_attention_gqa when the cache has fewer heads than q).  q [rows, H, D];
+    k/v_cache [B, Hkv, max_seq, D]; seq_len [B]; row_off [B+1]; anc [rows, anc_words] (int64 view of the u64
+    words).  Returns out [rows, H, D]."""
     torch = _torch()
     rows, n_heads, hd = q.shape
-    batch, _, max_seq, _ = k_cache.shape
+    batch, kv_heads, max_seq, _ = k_cache.shape
     if out is None:
         out = torch.empty_like(q)
     need = tree_attention_workspace(rows, batch, n_heads, hd, max_len)
     if workspace is None:
         workspace = _scratch(need, q.device)
-    _check(lib().trj_tree_attention(
-        _dev(q, name="q"), _dev(k_cache, q.dtype, "k_cache"), _dev(v_cache, q.dtype, "v_cache"),
-        _dev(seq_len, torch.int32, "seq_len"), _dev(row_off, torch.int32, "row_off"), _dev(anc, torch.int64, "anc"),
-        anc.shape[1], batch, rows, max_rows, n_heads, hd, max_seq, max_len, _dtype_code(q),
-        _dev(out, q.dtype, "out"), _dev(workspace, torch.uint8, "workspace"), workspace.numel(), _stream(stream)))
+    args = (_dev(q, name="q"), _dev(k_cache, q.dtype, "k_cache"), _dev(v_cache, q.dtype, "v_cache"),
+            _dev(seq_len, torch.int32, "seq_len"), _dev(row_off, torch.int32, "row_off"), _dev(anc, torch.int64, "anc"),
+            anc.shape[1], batch, rows, max_rows, n_heads)
+    tail = (hd, max_seq, max_len, _dtype_code(q), _dev(out, q.dtype, "out"), _dev(workspace, torch.uint8, "workspace"),
+            workspace.numel(), _stream(stream))
+    if kv_heads == n_heads:
+        _check(lib().trj_tree_attention(*args, *tail))
+    else:
+        _check(lib().trj_tree_attention_gqa(*args, kv_heads, *tail))
     return out
 
 
@@ -373,7 +379,8 @@ class Model:
     def __init__(self, cfg, layers: List[Dict[str, "object"]], glob: Dict[str, "object"], *,
                  max_batch: int = 1, max_seq: int = 2048, max_rows: int = MAX_ROWS):
         """``cfg`` has n_layers, d_model, n_heads, head_dim, d_ff, vocab, rms_eps, rope_theta, dtype
-        ("bf16" | "f32"); ``layers[l]`` and ``glob`` hold CUDA tensors named as in trj_weights."""
+        ("bf16" | "f32") and optionally n_kv_heads (0 = n_heads); ``layers[l]`` and ``glob`` hold CUDA tensors
+        named as in trj_weights."""
         torch = _torch()
         self.cfg = cfg
         self.tdtype = torch.bfloat16 if cfg.dtype == "bf16" else torch.float32
@@ -383,7 +390,7 @@ class Model:
         self.device = dev
         self.ccfg = ModelCfg(cfg.n_layers, cfg.d_model, cfg.n_heads, cfg.head_dim, cfg.d_ff, cfg.vocab,
                              cfg.rms_eps, cfg.rope_theta, BF16 if cfg.dtype == "bf16" else F32,
-                             max_batch, max_seq, max_rows)
+                             max_batch, max_seq, max_rows, int(getattr(cfg, "n_kv_heads", 0) or 0))
         need = lib().trj_workspace_bytes(C.byref(self.ccfg))
         if need == 0:
             raise TrjError(1, lib().trj_last_error().decode())
@@ -402,7 +409,7 @@ class Model:
                       for n in ("attn_norm", "wqkv", "wo", "mlp_norm", "w_gate_up", "w_down")))
         self._handle = C.c_void_p()
         _check(lib().trj_create(C.byref(self.ccfg), C.byref(w), _dev(self.workspace), need, C.byref(self._handle)))
-        shape = (cfg.n_layers, max_batch, cfg.n_heads, max_seq, cfg.head_dim)
+        shape = (cfg.n_layers, max_batch, int(getattr(cfg, "n_kv_heads", 0) or cfg.n_heads), max_seq, cfg.head_dim)
         self.k_cache = torch.zeros(shape, dtype=self.tdtype, device=dev)
         self.v_cache = torch.zeros(shape, dtype=self.tdtype, device=dev)
         self.seq_len = torch.zeros(max_batch, dtype=torch.int32, device=dev)

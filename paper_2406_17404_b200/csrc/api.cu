@@ -38,6 +38,16 @@ extern "C" trj_status trj_tree_attention(const void* q, const void* k_cache, con
                                          int32_t anc_words, int32_t B, int32_t rows_total, int32_t max_rows,
                                          int32_t H, int32_t D, int32_t max_seq, int32_t max_len, int32_t dtype,
                                          void* out, void* workspace, size_t workspace_bytes, void* stream) {
+    return trj_tree_attention_gqa(q, k_cache, v_cache, seq_len, row_off, anc, anc_words, B, rows_total, max_rows, H, H, D,
+                                  max_seq, max_len, dtype, out, workspace, workspace_bytes, stream);
+}
+
+extern "C" trj_status trj_tree_attention_gqa(const void* q, const void* k_cache, const void* v_cache,
+                                             const int32_t* seq_len, const int32_t* row_off, const uint64_t* anc,
+                                             int32_t anc_words, int32_t B, int32_t rows_total, int32_t max_rows,
+                                             int32_t H, int32_t Hkv, int32_t D, int32_t max_seq, int32_t max_len, int32_t dtype,
+                                             void* out, void* workspace, size_t workspace_bytes, void* stream) {
+    TRJ_REQUIRE(Hkv >= 1 && H >= Hkv && H % Hkv == 0, TRJ_EINVAL, "tree_attention: %d query heads over %d K/V heads", H, Hkv);
     TRJ_REQUIRE(q && k_cache && v_cache && seq_len && row_off && anc && out, TRJ_EINVAL, "tree_attention: null pointer");
     TRJ_REQUIRE(dtype_ok(dtype), TRJ_EINVAL, "tree_attention: unknown dtype %d", dtype);
     TRJ_REQUIRE(B >= 1 && H >= 1 && rows_total >= 0 && max_rows >= 1, TRJ_EINVAL, "tree_attention: bad sizes");
@@ -53,7 +63,7 @@ extern "C" trj_status trj_tree_attention(const void* q, const void* k_cache, con
     TRJ_REQUIRE(aligned(workspace, 256), TRJ_EINVAL, "tree_attention: workspace must be 256-byte aligned");
     if (rows_total == 0) return TRJ_OK;
     Batch bt{seq_len, row_off, B, rows_total, max_rows, max_len};
-    TRJ_CHECK_CUDA(launch_tree_attention(q, k_cache, v_cache, anc, anc_words, bt, H, D, max_seq, dtype, out, nullptr,
+    TRJ_CHECK_CUDA(launch_tree_attention(q, k_cache, v_cache, anc, anc_words, bt, H, Hkv, D, max_seq, dtype, out, nullptr,
                                          workspace, workspace_bytes, (cudaStream_t)stream));
     return TRJ_OK;
 }
@@ -91,11 +101,11 @@ extern "C" trj_status trj_argmax_accept_static(const void* logits, int32_t dtype
     TRJ_REQUIRE(dtype_ok(dtype), TRJ_EINVAL, "argmax_accept_static: unknown dtype %d", dtype);
     TRJ_REQUIRE(V >= 1 && B >= 1 && rows_total >= B, TRJ_EINVAL, "argmax_accept_static: bad sizes (every tree has a root)");
     TRJ_REQUIRE(B <= TRJ_MAX_BATCH, TRJ_ECAPACITY, "argmax_accept_static: batch %d exceeds %d", B, TRJ_MAX_BATCH);
-    TRJ_REQUIRE(rows_total <= B * TRJ_MAX_ROWS, TRJ_ECAPACITY,
-                "argmax_accept_static: %d rows in %d trees: a tree holds at most %d rows", rows_total, B, TRJ_MAX_ROWS);
     TRJ_REQUIRE(rows_total <= TRJ_STATIC_MAX_ROWS, TRJ_ECAPACITY,
                 "argmax_accept_static: %d rows exceed the built-in scratch of %d rows; use trj_argmax_accept with a workspace",
                 rows_total, TRJ_STATIC_MAX_ROWS);
+    TRJ_REQUIRE(rows_total <= B * TRJ_MAX_ROWS, TRJ_ECAPACITY,
+                "argmax_accept_static: %d rows in %d trees: a tree holds at most %d rows", rows_total, B, TRJ_MAX_ROWS);
     const cudaError_t e = launch_argmax_accept_static(logits, dtype, V, tokens, parent, depth, row_off, B, rows_total,
                                                       node_argmax, margin, k_acc, path, bonus, (cudaStream_t)stream);
     TRJ_REQUIRE(e != cudaErrorStreamCaptureUnsupported, TRJ_EINVAL,
@@ -172,11 +182,14 @@ constexpr int STEP_IN_BYTES = STEP_IN_INTS * 4 + TRJ_MAX_ROWS * 2 * 8;
 constexpr int STEP_STATUS_AT = TRJ_MAX_ROWS + 2 + TRJ_PATH_STRIDE;
 constexpr int STEP_OUT_INTS = STEP_STATUS_AT + 2;
 
+int kv_heads(const trj_model_cfg& c) { return c.n_kv_heads > 0 ? c.n_kv_heads : c.n_heads; }
+
 size_t carve(const trj_model_cfg& c, void* ws, trj_ctx* ctx) {
     const size_t es = dtype_size(c.dtype);
     const int rows = c.max_batch * c.max_rows;
     const int HD = c.n_heads * c.head_dim;
-    const size_t wide = (size_t)std::max(std::max(3 * HD, 2 * c.d_ff), c.d_model);
+    const int QKV = HD + 2 * kv_heads(c) * c.head_dim;
+    const size_t wide = (size_t)std::max(std::max(QKV, 2 * c.d_ff), c.d_model);
     Carver cv(ws);
     float* h = cv.take<float>((size_t)rows * c.d_model);
     float* y = cv.take<float>((size_t)rows * wide);
@@ -190,10 +203,12 @@ size_t carve(const trj_model_cfg& c, void* ws, trj_ctx* ctx) {
     char* argmax_ws = cv.take<char>(argmax_workspace_bytes(rows, c.max_batch));
     const size_t attn_bytes = trj_tree_attention_workspace(rows, c.max_batch, c.n_heads, c.head_dim, c.max_seq);
     char* attn_ws = cv.take<char>(attn_bytes);
+    // every row count a call may bring (the K split, hence the space for partial sums, is not monotone in it)
     size_t gemm_bytes = 256;
-    for (auto nk : {std::pair<int, int>{3 * HD, c.d_model}, {c.d_model, HD}, {2 * c.d_ff, c.d_model},
+    for (auto nk : {std::pair<int, int>{QKV, c.d_model}, {c.d_model, HD}, {2 * c.d_ff, c.d_model},
                     {c.d_model, c.d_ff}, {c.vocab, c.d_model}})
-        gemm_bytes = std::max(gemm_bytes, gemm_tc_workspace(rows, nk.first, nk.second));
+        for (int m = 1; m <= std::min(rows, TRJ_MAX_ROWS); ++m)
+            gemm_bytes = std::max(gemm_bytes, gemm_tc_workspace(m, nk.first, nk.second));
     char* gemm_ws = cv.take<char>(gemm_bytes);
     int32_t* chain_depth = cv.take<int32_t>(TRJ_MAX_ROWS);
     uint64_t* chain_anc = cv.take<uint64_t>(TRJ_MAX_ROWS * 2);
@@ -221,6 +236,8 @@ trj_status check_cfg(const trj_model_cfg* c) {
     TRJ_REQUIRE(c->n_layers >= 1 && c->d_model >= 1 && c->n_heads >= 1 && c->d_ff >= 1 && c->vocab >= 1,
                 TRJ_EINVAL, "cfg: non-positive dimension");
     TRJ_REQUIRE(c->head_dim == 64 || c->head_dim == 128, TRJ_EUNSUPPORTED, "cfg: head_dim %d (supported: 64, 128)", c->head_dim);
+    TRJ_REQUIRE(c->n_kv_heads >= 0 && c->n_kv_heads <= c->n_heads && (c->n_kv_heads == 0 || c->n_heads % c->n_kv_heads == 0),
+                TRJ_EINVAL, "cfg: %d K/V heads do not divide %d query heads", c->n_kv_heads, c->n_heads);
     TRJ_REQUIRE(c->max_batch >= 1 && c->max_batch <= TRJ_MAX_BATCH, TRJ_ECAPACITY, "cfg: max_batch %d outside 1..%d", c->max_batch, TRJ_MAX_BATCH);
     TRJ_REQUIRE(c->max_rows >= 1 && c->max_rows <= TRJ_MAX_ROWS, TRJ_ECAPACITY, "cfg: max_rows %d outside 1..%d", c->max_rows, TRJ_MAX_ROWS);
     TRJ_REQUIRE(c->max_seq >= c->max_rows, TRJ_EINVAL, "cfg: max_seq smaller than a tree");
@@ -271,9 +288,10 @@ trj_status forward(trj_ctx* ctx, void* k_cache, void* v_cache, int32_t b0, const
                    int32_t lm_first, int32_t lm_rows, cudaStream_t st) {
     ChainScope chain;                        // the embedding below is the chain's fence
     const trj_model_cfg& c = ctx->cfg;
-    const int M = bt.rows_total, d = c.d_model, HD = c.n_heads * c.head_dim;
+    const int M = bt.rows_total, d = c.d_model, HD = c.n_heads * c.head_dim, Hkv = kv_heads(c);
+    const int QKV = HD + 2 * Hkv * c.head_dim;
     const size_t es = dtype_size(c.dtype);
-    const size_t seq_stride = (size_t)c.n_heads * c.max_seq * c.head_dim * es;     // one sequence of one layer
+    const size_t seq_stride = (size_t)Hkv * c.max_seq * c.head_dim * es;           // one sequence of one layer
     // CTAs of the attention launch: what it leaves of the device is free while it runs (the plain kernel fills it)
     const bool attn_tc = ctx->attn_ws && ((uintptr_t)ctx->attn_ws % 256) == 0 &&
                          ctx->attn_ws_bytes >= tree_attention_tc_workspace(bt.B, c.n_heads) &&
@@ -288,13 +306,13 @@ trj_status forward(trj_ctx* ctx, void* k_cache, void* v_cache, int32_t b0, const
         char* v_slab = (char*)v_cache + ((size_t)l * c.max_batch + b0) * seq_stride;
         LAUNCH(PROF_ELEMENTWISE, launch_add_rmsnorm(ctx->h, pr, ctx->attn_norm[l], ctx->x, ctx->x_lo, c.dtype, M, d,
                                                     c.rms_eps, st));
-        LAUNCH(PROF_GEMM, launch_gemm(ctx->x, ctx->x_lo, ctx->wqkv[l], ctx->y, M, 3 * HD, d, c.dtype, ctx->gemm_ws,
+        LAUNCH(PROF_GEMM, launch_gemm(ctx->x, ctx->x_lo, ctx->wqkv[l], ctx->y, M, QKV, d, c.dtype, ctx->gemm_ws,
                                       ctx->gemm_ws_bytes, st, &pr, nullptr, gemm_status));
         LAUNCH(PROF_ROPE, launch_rope_kv_write(pr, ctx->inv_freq, depth, bt, ctx->q, k_slab, v_slab, c.dtype,
-                                               c.n_heads, c.head_dim, c.max_seq, st));
+                                               c.n_heads, Hkv, c.head_dim, c.max_seq, st));
         // inside the decoder the attention result reaches the output projection as a bf16 pair, like every
         // other projection input
-        LAUNCH(PROF_ATTENTION, launch_tree_attention(ctx->q, k_slab, v_slab, anc, anc_words, bt, c.n_heads, c.head_dim,
+        LAUNCH(PROF_ATTENTION, launch_tree_attention(ctx->q, k_slab, v_slab, anc, anc_words, bt, c.n_heads, Hkv, c.head_dim,
                                                      c.max_seq, c.dtype, ctx->x, ctx->x_lo, ctx->attn_ws,
                                                      ctx->attn_ws_bytes, st, attn_status));
         // While the attention kernel runs, HBM is nearly idle and the SMs it leaves free go to the first CTAs of
@@ -510,7 +528,7 @@ extern "C" trj_status trj_compact_kv(trj_ctx* ctx, void* k_cache, void* v_cache,
     TRJ_REQUIRE(B >= 1 && B <= c.max_batch, TRJ_ECAPACITY, "compact_kv: batch %d outside 1..%d", B, c.max_batch);
     cudaStream_t st = (cudaStream_t)stream;
     ChainScope chain;
-    LAUNCH(PROF_COMPACT, launch_compact(k_cache, v_cache, c.n_layers, c.max_batch, B, c.n_heads, c.max_seq, c.head_dim,
+    LAUNCH(PROF_COMPACT, launch_compact(k_cache, v_cache, c.n_layers, c.max_batch, B, kv_heads(c), c.max_seq, c.head_dim,
                                         c.dtype, seq_len, k_acc, path, st));
     return TRJ_OK;
 }
@@ -557,7 +575,7 @@ trj_status enqueue_step(trj_ctx* ctx, void* k_cache, void* v_cache, int32_t* seq
     if (s != TRJ_OK) return s;
     LAUNCH(PROF_ARGMAX, launch_argmax_accept(ctx->logits, TRJ_F32, c.vocab, d_tokens, d_parent, d_depth, d_off, 1, M, d_pred,
                                              nullptr, d_k, d_path, d_bonus, true, true, ctx->argmax_ws, st));
-    LAUNCH(PROF_COMPACT, launch_compact(k_cache, v_cache, c.n_layers, c.max_batch, 1, c.n_heads, c.max_seq, c.head_dim,
+    LAUNCH(PROF_COMPACT, launch_compact(k_cache, v_cache, c.n_layers, c.max_batch, 1, kv_heads(c), c.max_seq, c.head_dim,
                                         c.dtype, seq_len, d_k, d_path, st));
     TRJ_CHECK_CUDA(cudaMemcpyAsync(ctx->pin_out, ctx->step_out, sizeof(int32_t) * STEP_OUT_INTS, cudaMemcpyDeviceToHost, st));
     return TRJ_OK;
@@ -727,7 +745,7 @@ extern "C" trj_status trj_decode_device(trj_ctx* ctx, void* k_cache, void* v_cac
         if (fs != TRJ_OK) return fs;
         LAUNCH_ON(on, PROF_ARGMAX, launch_argmax_accept(ctx->logits, TRJ_F32, c.vocab, d_tokens, d_parent, d_depth, d_off, 1, M, d_pred,
                                                         nullptr, d_k, d_path, d_bonus, true, true, ctx->argmax_ws, on));
-        LAUNCH_ON(on, PROF_COMPACT, launch_compact(k_cache, v_cache, c.n_layers, c.max_batch, 1, c.n_heads, c.max_seq, c.head_dim,
+        LAUNCH_ON(on, PROF_COMPACT, launch_compact(k_cache, v_cache, c.n_layers, c.max_batch, 1, kv_heads(c), c.max_seq, c.head_dim,
                                                    c.dtype, seq_len, d_k, d_path, on));
         LAUNCH_ON(on, PROF_ELEMENTWISE, launch_commit_refill(d_tokens, d_parent, d_pred, M, d_k, d_path, d_bonus, context, capacity,
                                                              n_ctx, W, W + R * branch_len, draws, d_step, window, k_log, d_overflow, on));

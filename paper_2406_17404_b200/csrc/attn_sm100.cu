@@ -44,6 +44,7 @@ enum { B_KV_FULL = 0, B_KV_EMPTY = 5, B_Q_FULL = 10, B_Q_EMPTY = 11, B_S_FULL = 
 struct AtParams {
     const int32_t* seq_len; const int32_t* row_off; const uint64_t* anc;
     int anc_words, B, H, max_seq;
+    int Hkv, group;              // K/V heads and query heads per K/V head (grouped-query attention; group = 1: multi-head)
     __nv_bfloat16* out;          // [rows_total][H][128]
     __nv_bfloat16* out_lo;       // optional: rounding error of `out` as a second bf16 tensor (same shape)
     float* slots;                // partial results, AT_SLOT_FLOATS each
@@ -277,7 +278,12 @@ __device__ __forceinline__ void build_range(Sched& s, const AtParams& p) {
     }
 }
 
-template <int AT_SPLIT>
+// PRECISE: the probabilities go to the second product as a bf16 pair hi + lo (lo = the rounding error of hi, kept in
+// the tile's own score buffer once the scores are in registers), so the product sees ~16 mantissa bits of P.  A
+// single bf16 P costs ~1e-3 of relative error in the output whatever the number of keys (the output of near-uniform
+// attention is a mean of n values and the rounding errors of its n weights do not average out any faster than it
+// does); inside a deep decoder that error flips the bf16 roundings of the next layers' K/V rows and grows with depth.
+template <int AT_SPLIT, bool PRECISE>
 __global__ void __launch_bounds__(at_threads(AT_SPLIT), 1) tree_attention_tc_kernel(const __grid_constant__ CUtensorMap map_q,
                                                                           const __grid_constant__ CUtensorMap map_k,
                                                                           const __grid_constant__ CUtensorMap map_v,
@@ -359,7 +365,7 @@ __global__ void __launch_bounds__(at_threads(AT_SPLIT), 1) tree_attention_tc_ker
                 // the first segment's Q is requested by the MMA thread as soon as the previous kernel is done, so
                 // that it does not queue behind the cache tiles this thread asks for ahead of the wait
                 if (e > 0) { ok = load_q(); if (!ok) break; }
-                const int cache_row0 = (w.b * p.H + w.h) * p.max_seq;
+                const int cache_row0 = (w.b * p.Hkv + w.h / p.group) * p.max_seq;
                 const int old_tiles = w.S / AT_KEYS;          // tiles that hold cached rows only
                 for (int t = w.t; t < t_end && ok; ++t, ++g) {
                     for (int kv = 0; kv < 2 && ok; ++kv) {
@@ -431,6 +437,8 @@ __global__ void __launch_bounds__(at_threads(AT_SPLIT), 1) tree_attention_tc_ker
                     // 8 x 16 keys; P comes straight from TMEM
                     const uint64_t v_desc = desc_mnmajor(v_smem);
                     umma8_pv(tmem_o, tmem_p[g & 1], (uint32_t)v_desc, (uint32_t)(v_desc >> 32), idesc_pv, g > g0 ? 1u : 0u);
+                    if constexpr (PRECISE)                   // the low halves of P sit in the first 64 columns of the tile's S buffer
+                        umma8_pv(tmem_o, tmem_s[g & 1], (uint32_t)v_desc, (uint32_t)(v_desc >> 32), idesc_pv, 1u);
                     umma_commit(bar(B_P_FREE + (g & 1)));
                     umma_commit(bar(B_KV_EMPTY + slot));
                 }
@@ -549,6 +557,27 @@ __global__ void __launch_bounds__(at_threads(AT_SPLIT), 1) tree_attention_tc_ker
                     }
                     if constexpr (AT_KPT == 64) tmem_st32u(tmem_p[g & 1] + lane_addr + (AT_KPT / 2) * part, packed);
                     else tmem_st16u(tmem_p[g & 1] + lane_addr + (AT_KPT / 2) * part, packed);
+                    if constexpr (PRECISE) {
+                        // lo = p - bf16(p), recomputed from the scores 32 keys at a time (keeps the register count
+                        // down); every thread of the row group has its scores in registers since the exchange of
+                        // the maxima, so the S buffer may be overwritten
+#pragma unroll
+                        for (int c0 = 0; c0 < AT_KPT; c0 += 32) {
+                            uint32_t lo[16];
+                            if (live) {
+#pragma unroll
+                                for (int i = 0; i < 32; i += 2) {
+                                    const float a = fast_exp2(fmaf(s[c0 + i], p.scale_log2, -m_use));
+                                    const float b = fast_exp2(fmaf(s[c0 + i + 1], p.scale_log2, -m_use));
+                                    lo[i >> 1] = pack_bf16(a - bf16_round(a), b - bf16_round(b));
+                                }
+                            } else {
+#pragma unroll
+                                for (int i = 0; i < 16; ++i) lo[i] = 0u;
+                            }
+                            tmem_st16u(tmem_s[g & 1] + lane_addr + (AT_KPT / 2) * part + (c0 >> 1), lo);
+                        }
+                    }
                 }
                 // keys past the end of the sequence hold whatever the cache holds: clear those V rows so
                 // that 0 * garbage cannot poison the product
@@ -773,7 +802,7 @@ int at_cluster_size(int H) {
     std::lock_guard<std::mutex> lock(mu);
     if (cached_h == H) return cached_c;
     int pick = 1;
-    if (cudaFuncSetAttribute(tree_attention_tc_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)AT_SMEM) == cudaSuccess) {
+    if (cudaFuncSetAttribute(tree_attention_tc_kernel<2, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)AT_SMEM) == cudaSuccess) {
         for (int c = 4; c >= 2 && pick == 1; c /= 2) {
             if (H * c > AT_MAX_GRID) continue;
             cudaLaunchConfig_t cfg = {};
@@ -783,7 +812,7 @@ int at_cluster_size(int H) {
             attr[0].val.clusterDim.x = c; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
             cfg.attrs = attr; cfg.numAttrs = 1;
             int n = 0;
-            if (cudaOccupancyMaxActiveClusters(&n, tree_attention_tc_kernel<2>, &cfg) == cudaSuccess && n >= H) pick = c;
+            if (cudaOccupancyMaxActiveClusters(&n, tree_attention_tc_kernel<2, true>, &cfg) == cudaSuccess && n >= H) pick = c;
         }
     }
     (void)cudaGetLastError();                                // a refused query is not an error of the caller
@@ -822,24 +851,29 @@ size_t tree_attention_tc_workspace(int32_t B, int32_t H) {
 }
 
 cudaError_t launch_tree_attention_tc(const void* q, const void* k_slab, const void* v_slab, const uint64_t* anc,
-                                     int32_t anc_words, const Batch& bt, int32_t H, int32_t max_seq, void* out,
+                                     int32_t anc_words, const Batch& bt, int32_t H, int32_t Hkv, int32_t max_seq, void* out,
                                      void* out_lo, void* workspace, cudaStream_t st, int* status) {
     static std::once_flag once;
     static cudaError_t attr_err = cudaSuccess;
     std::call_once(once, [] {
-        attr_err = cudaFuncSetAttribute(tree_attention_tc_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)AT_SMEM);
+        attr_err = cudaFuncSetAttribute(tree_attention_tc_kernel<2, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)AT_SMEM);
         if (attr_err == cudaSuccess)
-            attr_err = cudaFuncSetAttribute(tree_attention_tc_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)AT_SMEM);
+            attr_err = cudaFuncSetAttribute(tree_attention_tc_kernel<4, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)AT_SMEM);
+        if (attr_err == cudaSuccess)
+            attr_err = cudaFuncSetAttribute(tree_attention_tc_kernel<2, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)AT_SMEM);
+        if (attr_err == cudaSuccess)
+            attr_err = cudaFuncSetAttribute(tree_attention_tc_kernel<4, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)AT_SMEM);
     });
     if (attr_err != cudaSuccess) return attr_err;
     CUtensorMap map_q, map_k, map_v;
     if (!at_make_map(&map_q, q, (size_t)bt.rows_total, (size_t)H * AT_D) ||
-        !at_make_map(&map_k, k_slab, (size_t)bt.B * H * max_seq, AT_D) ||
-        !at_make_map(&map_v, v_slab, (size_t)bt.B * H * max_seq, AT_D))
+        !at_make_map(&map_k, k_slab, (size_t)bt.B * Hkv * max_seq, AT_D) ||
+        !at_make_map(&map_v, v_slab, (size_t)bt.B * Hkv * max_seq, AT_D))
         return cudaErrorInvalidValue;
     AtParams p;
     p.seq_len = bt.seq_len; p.row_off = bt.row_off; p.anc = anc; p.anc_words = anc_words;
     p.B = bt.B; p.H = H; p.max_seq = max_seq;
+    p.Hkv = Hkv; p.group = H / Hkv;
     p.out = (__nv_bfloat16*)out;
     p.out_lo = (__nv_bfloat16*)out_lo;
     p.status = status ? status : (int*)workspace;
@@ -864,8 +898,15 @@ cudaError_t launch_tree_attention_tc(const void* q, const void* k_slab, const vo
         ++n_attr;
     }
     cfg.attrs = attr; cfg.numAttrs = n_attr;
-    cudaError_t e = plan.split == 4 ? cudaLaunchKernelEx(&cfg, tree_attention_tc_kernel<4>, map_q, map_k, map_v, p)
-                                    : cudaLaunchKernelEx(&cfg, tree_attention_tc_kernel<2>, map_q, map_k, map_v, p);
+    // inside a decoder (the caller asks for the result as a bf16 pair) the probabilities are a bf16 pair as well
+    const bool precise = out_lo != nullptr;
+    cudaError_t e;
+    if (plan.split == 4)
+        e = precise ? cudaLaunchKernelEx(&cfg, tree_attention_tc_kernel<4, true>, map_q, map_k, map_v, p)
+                    : cudaLaunchKernelEx(&cfg, tree_attention_tc_kernel<4, false>, map_q, map_k, map_v, p);
+    else
+        e = precise ? cudaLaunchKernelEx(&cfg, tree_attention_tc_kernel<2, true>, map_q, map_k, map_v, p)
+                    : cudaLaunchKernelEx(&cfg, tree_attention_tc_kernel<2, false>, map_q, map_k, map_v, p);
     if (e == cudaSuccess) e = cudaGetLastError();
     if (e != cudaSuccess || !plan.merge_kernel) return e;
     count_launch();
@@ -876,16 +917,16 @@ cudaError_t launch_tree_attention_tc(const void* q, const void* k_slab, const vo
 }
 
 cudaError_t launch_tree_attention(const void* q, const void* k_slab, const void* v_slab, const uint64_t* anc,
-                                  int32_t anc_words, const Batch& bt, int32_t H, int32_t D, int32_t max_seq,
+                                  int32_t anc_words, const Batch& bt, int32_t H, int32_t Hkv, int32_t D, int32_t max_seq,
                                   int32_t dtype, void* out, void* out_lo, void* workspace, size_t workspace_bytes,
                                   cudaStream_t st, int* status) {
     if (D == AT_D && dtype == TRJ_BF16 && bt.max_rows <= AT_ROWS) {
         if (!workspace || ((uintptr_t)workspace % 256) != 0 || workspace_bytes < tree_attention_tc_workspace(bt.B, H) ||
             !tree_attention_tc_supported(D, dtype, bt.max_rows))
             return cudaErrorInvalidValue;
-        return launch_tree_attention_tc(q, k_slab, v_slab, anc, anc_words, bt, H, max_seq, out, out_lo, workspace, st, status);
+        return launch_tree_attention_tc(q, k_slab, v_slab, anc, anc_words, bt, H, Hkv, max_seq, out, out_lo, workspace, st, status);
     }
-    return launch_tree_attention_generic(q, k_slab, v_slab, anc, anc_words, bt, H, D, max_seq, dtype, out, out_lo, st);
+    return launch_tree_attention_generic(q, k_slab, v_slab, anc, anc_words, bt, H, Hkv, D, max_seq, dtype, out, out_lo, st);
 }
 
 }  // namespace trj

@@ -233,7 +233,7 @@ template <typename T>
 __global__ void rope_kv_write_kernel(const Parts qkv, const double* __restrict__ inv_freq,
                                      const int32_t* __restrict__ depth, const int32_t* __restrict__ seq_len,
                                      const int32_t* __restrict__ row_off, int B, T* __restrict__ q_out,
-                                     T* __restrict__ k_slab, T* __restrict__ v_slab, int H, int D, int max_seq) {
+                                     T* __restrict__ k_slab, T* __restrict__ v_slab, int H, int Hkv, int D, int max_seq) {
     pdl_launch_dependents();
     // geometry and the rotation of this thread's first element do not depend on the projection: have them
     // ready before waiting for it
@@ -241,9 +241,10 @@ __global__ void rope_kv_write_kernel(const Parts qkv, const double* __restrict__
     const int b = seq_of_row(row_off, B, row);
     const int local = row - row_off[b];
     const int pos = seq_len[b] + depth[row];
-    const int half = D >> 1, HD = H * D;
-    const size_t src = (size_t)row * 3 * HD + hh * D;        // flat index into the projection result
-    const size_t cache_row = (((size_t)b * H + hh) * max_seq + seq_len[b] + local) * D;
+    const int half = D >> 1, HD = H * D, KD = Hkv * D;
+    const bool has_kv = hh < Hkv;                            // this CTA also handles K/V head hh
+    const size_t src = (size_t)row * (HD + 2 * KD) + hh * D; // flat index of query head hh in the projection result
+    const size_t cache_row = (((size_t)b * Hkv + hh) * max_seq + seq_len[b] + local) * D;
     auto rotation = [&](int i, float& sn, float& cs) {
         // angle in fp64 (positions reach thousands of radians), reduced to [-pi, pi] there; sin/cos of the reduced
         // angle in fp32 are then accurate to ~1e-7
@@ -261,11 +262,14 @@ __global__ void rope_kv_write_kernel(const Parts qkv, const double* __restrict__
         for (int s = 0; s < qkv.splits; ++s) {               // six independent loads per split-K piece
             const float* piece = qkv.ptr + (size_t)s * qkv.stride + src + i;
             qa += piece[0];      qb += piece[half];
-            ka += piece[HD];     kb += piece[HD + half];
-            va += piece[2 * HD]; vb += piece[2 * HD + half];
+            if (has_kv) {
+                ka += piece[HD];      kb += piece[HD + half];
+                va += piece[HD + KD]; vb += piece[HD + KD + half];
+            }
         }
         q_out[(size_t)row * HD + hh * D + i] = from_f<T>(qa * cs - qb * sn);
         q_out[(size_t)row * HD + hh * D + i + half] = from_f<T>(qb * cs + qa * sn);
+        if (!has_kv) continue;
         k_slab[cache_row + i] = from_f<T>(ka * cs - kb * sn);
         k_slab[cache_row + i + half] = from_f<T>(kb * cs + ka * sn);
         v_slab[cache_row + i] = from_f<T>(va);
@@ -280,19 +284,21 @@ template <typename T>
 __global__ void __launch_bounds__(ROPE_THREADS) rope_kv_write_vec_kernel(const Parts qkv, const double* __restrict__ inv_freq,
                                          const int32_t* __restrict__ depth, const int32_t* __restrict__ seq_len,
                                          const int32_t* __restrict__ row_off, int B, T* __restrict__ q_out,
-                                         T* __restrict__ k_slab, T* __restrict__ v_slab, int H, int D, int max_seq,
+                                         T* __restrict__ k_slab, T* __restrict__ v_slab, int H, int Hkv, int D, int max_seq,
                                          int heads_per_cta) {
     pdl_launch_dependents();
     // geometry and rotations do not depend on the projection: have them ready before waiting for it
-    const int half = D >> 1, HD = H * D, per_head = half >> 2;
+    const int half = D >> 1, HD = H * D, KD = Hkv * D, per_head = half >> 2;
     const int row = blockIdx.x, hh = blockIdx.y * heads_per_cta + (int)threadIdx.x / per_head;
     const int i = ((int)threadIdx.x % per_head) * 4;
     if (hh >= H) return;
     const int b = seq_of_row(row_off, B, row);
     const int local = row - row_off[b];
     const int pos = seq_len[b] + depth[row];
-    const size_t src = (size_t)row * 3 * HD + hh * D + i;    // flat index into the projection result
-    const size_t cache_at = (((size_t)b * H + hh) * max_seq + seq_len[b] + local) * D + i;
+    const bool has_kv = hh < Hkv;                            // this thread also handles K/V head hh
+    const int n_e = has_kv ? 6 : 2;
+    const size_t src = (size_t)row * (HD + 2 * KD) + hh * D + i;    // flat index of query head hh in the projection result
+    const size_t cache_at = (((size_t)b * Hkv + hh) * max_seq + seq_len[b] + local) * D + i;
     const size_t q_at = (size_t)row * HD + hh * D + i;
     float sn[4], cs[4];
 #pragma unroll
@@ -315,13 +321,15 @@ __global__ void __launch_bounds__(ROPE_THREADS) rope_kv_write_vec_kernel(const P
             if (s0 + j < qkv.splits) {
                 const float* piece = qkv.ptr + (size_t)(s0 + j) * qkv.stride + src;
 #pragma unroll
-                for (int e = 0; e < 6; ++e) t[j][e] = *reinterpret_cast<const float4*>(piece + (e >> 1) * HD + (e & 1) * half);
+                for (int e = 0; e < 6; ++e)                  // q at 0, k at HD, v at HD + KD; first and second half of the head
+                    if (e < n_e) t[j][e] = *reinterpret_cast<const float4*>(piece + (e >> 1 == 0 ? 0 : e >> 1 == 1 ? HD : HD + KD) + (e & 1) * half);
             }
 #pragma unroll
         for (int j = 0; j < 3; ++j)
             if (s0 + j < qkv.splits) {
 #pragma unroll
-                for (int e = 0; e < 6; ++e) { acc[e].x += t[j][e].x; acc[e].y += t[j][e].y; acc[e].z += t[j][e].z; acc[e].w += t[j][e].w; }
+                for (int e = 0; e < 6; ++e)
+                    if (e < n_e) { acc[e].x += t[j][e].x; acc[e].y += t[j][e].y; acc[e].z += t[j][e].z; acc[e].w += t[j][e].w; }
             }
     }
     auto rot_lo = [&](const float4& a, const float4& bb) {
@@ -332,6 +340,7 @@ __global__ void __launch_bounds__(ROPE_THREADS) rope_kv_write_vec_kernel(const P
     };
     store_split4<T>(q_out, nullptr, q_at, rot_lo(acc[0], acc[1]));
     store_split4<T>(q_out, nullptr, q_at + half, rot_hi(acc[0], acc[1]));
+    if (!has_kv) return;
     store_split4<T>(k_slab, nullptr, cache_at, rot_lo(acc[2], acc[3]));
     store_split4<T>(k_slab, nullptr, cache_at + half, rot_hi(acc[2], acc[3]));
     store_split4<T>(v_slab, nullptr, cache_at, acc[4]);
@@ -345,7 +354,7 @@ template <typename T, int D>
 __global__ void __launch_bounds__(128) tree_attention_generic_kernel(
         const T* __restrict__ q, const T* __restrict__ k_slab, const T* __restrict__ v_slab,
         const uint64_t* __restrict__ anc, int anc_words, const int32_t* __restrict__ seq_len,
-        const int32_t* __restrict__ row_off, int B, int H, int max_seq, T* __restrict__ out, T* __restrict__ out_lo) {
+        const int32_t* __restrict__ row_off, int B, int H, int Hkv, int max_seq, T* __restrict__ out, T* __restrict__ out_lo) {
     constexpr int PER = D / 32;                  // output dims per lane
     __shared__ float qs[D];
     __shared__ float part_m[4], part_l[4];
@@ -356,8 +365,9 @@ __global__ void __launch_bounds__(128) tree_attention_generic_kernel(
     const int rows_b = row_off[b + 1] - row_off[b];
     const int total = S + rows_b;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const T* kb = k_slab + ((size_t)b * H + hh) * max_seq * D;
-    const T* vb = v_slab + ((size_t)b * H + hh) * max_seq * D;
+    const int kvh = hh / (H / Hkv);              // grouped-query attention: the K/V head of this query head
+    const T* kb = k_slab + ((size_t)b * Hkv + kvh) * max_seq * D;
+    const T* vb = v_slab + ((size_t)b * Hkv + kvh) * max_seq * D;
     const uint64_t* mask = anc + (size_t)row * anc_words;
     for (int c = threadIdx.x; c < D; c += blockDim.x) qs[c] = to_f(q[((size_t)row * H + hh) * D + c]);
     __syncthreads();
@@ -661,7 +671,7 @@ cudaError_t launch_gemm_simt(const void* x, const void* x_lo, const void* w, flo
 
 cudaError_t launch_rope_kv_write(const Parts& qkv, const double* inv_freq, const int32_t* depth,
                                  const Batch& bt, void* q_out, void* k_slab, void* v_slab, int32_t dtype,
-                                 int32_t H, int32_t D, int32_t max_seq, cudaStream_t st) {
+                                 int32_t H, int32_t Hkv, int32_t D, int32_t max_seq, cudaStream_t st) {
     count_launch();
     cudaError_t launch_err = cudaSuccess;
     const int per_head = D / 8;                              // threads per head in the vector kernel
@@ -670,25 +680,25 @@ cudaError_t launch_rope_kv_write(const Parts& qkv, const double* inv_freq, const
     if (vec) {
         dim3 grid(bt.rows_total, (H + hpc - 1) / hpc);
         DISPATCH_T(dtype, launch_err = launch_chain(rope_kv_write_vec_kernel<T>, grid, dim3(per_head * hpc), 0, st, qkv, inv_freq, depth,
-                                                    bt.seq_len, bt.row_off, bt.B, (T*)q_out, (T*)k_slab, (T*)v_slab, H, D, max_seq, hpc));
+                                                    bt.seq_len, bt.row_off, bt.B, (T*)q_out, (T*)k_slab, (T*)v_slab, H, Hkv, D, max_seq, hpc));
     } else {
         dim3 grid(bt.rows_total, H);
         DISPATCH_T(dtype, launch_err = launch_chain(rope_kv_write_kernel<T>, grid, dim3(64), 0, st, qkv, inv_freq, depth, bt.seq_len, bt.row_off,
-                                                    bt.B, (T*)q_out, (T*)k_slab, (T*)v_slab, H, D, max_seq));
+                                                    bt.B, (T*)q_out, (T*)k_slab, (T*)v_slab, H, Hkv, D, max_seq));
     }
     return launch_err != cudaSuccess ? launch_err : cudaGetLastError();
 }
 
 cudaError_t launch_tree_attention_generic(const void* q, const void* k_slab, const void* v_slab,
                                           const uint64_t* anc, int32_t anc_words, const Batch& bt,
-                                          int32_t H, int32_t D, int32_t max_seq, int32_t dtype,
+                                          int32_t H, int32_t Hkv, int32_t D, int32_t max_seq, int32_t dtype,
                                           void* out, void* out_lo, cudaStream_t st) {
     count_launch();
     dim3 grid(bt.rows_total, H);
 #define ATT(DD)                                                                                          \
     DISPATCH_T(dtype, tree_attention_generic_kernel<T, DD><<<grid, 128, 0, st>>>(                        \
                           (const T*)q, (const T*)k_slab, (const T*)v_slab, anc, anc_words, bt.seq_len,   \
-                          bt.row_off, bt.B, H, max_seq, (T*)out, (T*)out_lo))
+                          bt.row_off, bt.B, H, Hkv, max_seq, (T*)out, (T*)out_lo))
     if (D == 64) { ATT(64); }
     else if (D == 128) { ATT(128); }
     else return cudaErrorInvalidValue;

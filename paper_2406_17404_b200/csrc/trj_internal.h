@@ -119,13 +119,15 @@ cudaError_t launch_gemm(const void* x, const void* x_lo, const void* w, float* y
                         const WeightPrefetch* ahead = nullptr, int* status = nullptr);
 
 // Rotary embedding of q and k at position seq_len[b] + depth[row]; q -> q_out [rows][H][D];
-// k, v -> cache rows seq_len[b] + local row of the layer slab [B][H][max_seq][D].
+// k, v -> cache rows seq_len[b] + local row of the layer slab [B][Hkv][max_seq][D].  The projection result has
+// (H + 2 * Hkv) * D values per row: H query heads, then Hkv key heads, then Hkv value heads.
 cudaError_t launch_rope_kv_write(const Parts& qkv, const double* inv_freq, const int32_t* depth,
                                  const Batch& bt, void* q_out, void* k_slab, void* v_slab, int32_t dtype,
-                                 int32_t H, int32_t D, int32_t max_seq, cudaStream_t st);
+                                 int32_t H, int32_t Hkv, int32_t D, int32_t max_seq, cudaStream_t st);
+// Attention: H query heads over Hkv K/V heads (query head h reads K/V head h / (H / Hkv)).
 cudaError_t launch_tree_attention_generic(const void* q, const void* k_slab, const void* v_slab,
                                           const uint64_t* anc, int32_t anc_words, const Batch& bt,
-                                          int32_t H, int32_t D, int32_t max_seq, int32_t dtype,
+                                          int32_t H, int32_t Hkv, int32_t D, int32_t max_seq, int32_t dtype,
                                           void* out, void* out_lo, cudaStream_t st);
 // tcgen05 / TMA tree attention (attn_sm100.cu): bf16, head_dim 128.  Workspace: status word in the first
 // 256 bytes, then split-KV partial results.
@@ -133,14 +135,14 @@ bool tree_attention_tc_supported(int32_t D, int32_t dtype, int32_t max_rows);
 size_t tree_attention_tc_workspace(int32_t B, int32_t H);
 int tree_attention_grid(int32_t B, int32_t H, int32_t max_len);     // CTAs the tcgen05 kernel is launched with
 cudaError_t launch_tree_attention_tc(const void* q, const void* k_slab, const void* v_slab, const uint64_t* anc,
-                                     int32_t anc_words, const Batch& bt, int32_t H, int32_t max_seq, void* out,
+                                     int32_t anc_words, const Batch& bt, int32_t H, int32_t Hkv, int32_t max_seq, void* out,
                                      void* out_lo, void* workspace, cudaStream_t st, int* status = nullptr);
 // The tcgen05 kernel for bf16 with head_dim 128, the generic kernel for the rest (fp32, head_dim 64).  A bf16 /
 // head_dim-128 call whose workspace is too small or misaligned is an error (cudaErrorInvalidValue), never a
 // silent detour.  out_lo (may be null) receives the rounding error of `out` as a second tensor of the same
 // type, for the projection that follows.  `status`: as for launch_gemm.
 cudaError_t launch_tree_attention(const void* q, const void* k_slab, const void* v_slab, const uint64_t* anc,
-                                  int32_t anc_words, const Batch& bt, int32_t H, int32_t D, int32_t max_seq,
+                                  int32_t anc_words, const Batch& bt, int32_t H, int32_t Hkv, int32_t D, int32_t max_seq,
                                   int32_t dtype, void* out, void* out_lo, void* workspace, size_t workspace_bytes,
                                   cudaStream_t st, int* status = nullptr);
 // One CTA waits, with a poll limit, on a barrier nobody arrives at (self-test of the time-out path).

@@ -24,7 +24,7 @@ from typing import Dict, List, Optional, Tuple
 import numpy as np
 
 __all__ = [
-    "ModelCfg", "TINY", "LLAMA7B", "stream", "round_bf16", "bf16_bits",
+    "ModelCfg", "TINY", "TINY_GQA", "LLAMA7B", "LLAMA3_8B", "stream", "round_bf16", "bf16_bits",
     "layer_weights", "global_weights", "prompt", "chain_parents",
     "random_tree", "node_depths", "qkv", "logits", "planted_tokens",
     "random_path", "ragged_batch", "noise_draws",
@@ -36,7 +36,10 @@ __all__ = [
 # --------------------------------------------------------------------------
 @dataclass(frozen=True)
 class ModelCfg:
-    """LLaMA-family decoder shape (RMSNorm, RoPE, MHA, SwiGLU, untied LM head)."""
+    """LLaMA-family decoder shape (RMSNorm, RoPE, MHA or grouped-query attention, SwiGLU, untied LM head).
+
+    ``n_kv_heads`` = 0 means one K/V head per query head; otherwise query head h uses K/V head
+    h // (n_heads // n_kv_heads)."""
     n_layers: int
     d_model: int
     n_heads: int
@@ -47,6 +50,11 @@ class ModelCfg:
     rms_eps: float = 1e-5
     rope_theta: float = 10000.0
     weight_std: float = 0.02
+    n_kv_heads: int = 0
+
+    @property
+    def kv_heads(self) -> int:
+        return self.n_kv_heads or self.n_heads
 
     def with_layers(self, n: int) -> "ModelCfg":
         return replace(self, n_layers=n)
@@ -54,8 +62,13 @@ class ModelCfg:
 
 TINY = ModelCfg(n_layers=2, d_model=256, n_heads=4, head_dim=64, d_ff=688,
                 vocab=1024, dtype="f32")
+TINY_GQA = ModelCfg(n_layers=2, d_model=256, n_heads=4, head_dim=64, d_ff=688,
+                    vocab=1024, dtype="f32", n_kv_heads=2)
 LLAMA7B = ModelCfg(n_layers=32, d_model=4096, n_heads=32, head_dim=128,
                    d_ff=11008, vocab=32000, dtype="bf16")
+# the shape of the paper's main model family (Table 2): grouped-query attention with 8 K/V heads, 128 256-way vocabulary
+LLAMA3_8B = ModelCfg(n_layers=32, d_model=4096, n_heads=32, head_dim=128, d_ff=14336, vocab=128256,
+                     dtype="bf16", rope_theta=500000.0, n_kv_heads=8)
 
 
 # --------------------------------------------------------------------------
@@ -97,16 +110,17 @@ def _normal(seed: int, name: str, shape, std: float, dtype: str) -> np.ndarray:
 def layer_weights(cfg: ModelCfg, seed: int, layer: int) -> Dict[str, np.ndarray]:
     """Weights of one decoder layer.  Every matrix is [d_out, d_in] (d_in contiguous).
 
-    ``wqkv`` stacks the query, key and value projections (rows 0..d-1 = Wq,
-    d..2d-1 = Wk, 2d..3d-1 = Wv, d = n_heads*head_dim); ``w_gate_up`` stacks the
-    SwiGLU gate rows (0..f-1) over the up rows (f..2f-1).
+    ``wqkv`` stacks the query, key and value projections (rows 0..q-1 = Wq,
+    q..q+kv-1 = Wk, q+kv..q+2kv-1 = Wv, q = n_heads*head_dim, kv = kv_heads*head_dim);
+    ``w_gate_up`` stacks the SwiGLU gate rows (0..f-1) over the up rows (f..2f-1).
     """
     d, f, hd = cfg.d_model, cfg.d_ff, cfg.n_heads * cfg.head_dim
+    kvd = cfg.kv_heads * cfg.head_dim
     s, t = cfg.weight_std, cfg.dtype
     p = f"layer{layer}."
     return {
         "attn_norm": np.ones(d, np.float32),
-        "wqkv": _normal(seed, p + "wqkv", (3 * hd, d), s, t),
+        "wqkv": _normal(seed, p + "wqkv", (hd + 2 * kvd, d), s, t),
         "wo": _normal(seed, p + "wo", (d, hd), s, t),
         "mlp_norm": np.ones(d, np.float32),
         "w_gate_up": _normal(seed, p + "w_gate_up", (2 * f, d), s, t),
@@ -175,15 +189,17 @@ def random_tree(seed: int, m: int, max_depth: int, max_children: int,
 # op-level tensors
 # --------------------------------------------------------------------------
 def qkv(seed: int, n_heads: int, head_dim: int, prefix: int, rows: int,
-        dtype: str = "bf16", name: str = "") -> Dict[str, np.ndarray]:
-    """q/k/v ~ N(0,1).  q: [rows, H, D]; k/v prefix: [H, prefix, D]; k/v tree: [H, rows, D]."""
+        dtype: str = "bf16", name: str = "", kv_heads: int = 0) -> Dict[str, np.ndarray]:
+    """q/k/v ~ N(0,1).  q: [rows, H, D]; k/v prefix: [Hkv, prefix, D]; k/v tree: [Hkv, rows, D] (Hkv = H unless
+    ``kv_heads`` says otherwise)."""
     n = name
+    hk = kv_heads or n_heads
     return {
         "q": _normal(seed, n + "q", (rows, n_heads, head_dim), 1.0, dtype),
-        "k_prefix": _normal(seed, n + "k_prefix", (n_heads, prefix, head_dim), 1.0, dtype),
-        "v_prefix": _normal(seed, n + "v_prefix", (n_heads, prefix, head_dim), 1.0, dtype),
-        "k_tree": _normal(seed, n + "k_tree", (n_heads, rows, head_dim), 1.0, dtype),
-        "v_tree": _normal(seed, n + "v_tree", (n_heads, rows, head_dim), 1.0, dtype),
+        "k_prefix": _normal(seed, n + "k_prefix", (hk, prefix, head_dim), 1.0, dtype),
+        "v_prefix": _normal(seed, n + "v_prefix", (hk, prefix, head_dim), 1.0, dtype),
+        "k_tree": _normal(seed, n + "k_tree", (hk, rows, head_dim), 1.0, dtype),
+        "v_tree": _normal(seed, n + "v_tree", (hk, rows, head_dim), 1.0, dtype),
     }
 
 

@@ -24,17 +24,19 @@ def anc_dev(anc):
 class AttnCase:
     """A ragged batch of (prefix, tree) attention problems in device layout plus the host originals."""
 
-    def __init__(self, trj, seed, n_heads, head_dim, prefixes, rows, parents, dtype="bf16", max_seq=None, pad=0):
+    def __init__(self, trj, seed, n_heads, head_dim, prefixes, rows, parents, dtype="bf16", max_seq=None, pad=0,
+                 kv_heads=0):
         self.h, self.d, self.dtype = n_heads, head_dim, dtype
+        self.hk = kv_heads or n_heads
         self.prefixes, self.rows, self.parents = list(prefixes), list(rows), parents
         b = len(prefixes)
         self.max_len = max(s + m for s, m in zip(prefixes, rows))
         self.max_seq = max_seq or (self.max_len + pad)
         self.max_rows = max(rows)
-        self.host = [synth.qkv(seed, n_heads, head_dim, s, m, dtype, name=f"seq{i}.")
+        self.host = [synth.qkv(seed, n_heads, head_dim, s, m, dtype, name=f"seq{i}.", kv_heads=kv_heads)
                      for i, (s, m) in enumerate(zip(prefixes, rows))]
         # cache rows past the end of a sequence hold NaN: whatever a kernel fetches from there must not reach its output
-        k = np.full((b, n_heads, self.max_seq, head_dim), np.nan, np.float32)
+        k = np.full((b, self.hk, self.max_seq, head_dim), np.nan, np.float32)
         v = np.full_like(k, np.nan)
         for i, (s, m) in enumerate(zip(prefixes, rows)):
             t = self.host[i]
@@ -58,5 +60,6 @@ class AttnCase:
         """fp64 reference [M, len(heads), D] of sequence ``seq`` restricted to ``heads``."""
         t = self.host[seq]
         hs = list(range(self.h)) if heads is None else list(heads)
-        return oracle.tree_attention(t["q"][:, hs], t["k_prefix"][hs], t["v_prefix"][hs],
-                                     t["k_tree"][hs], t["v_tree"][hs], self.parents[seq])
+        ks = [h // (self.h // self.hk) for h in hs]          # the K/V head each of the chosen query heads reads
+        return oracle.tree_attention(t["q"][:, hs], t["k_prefix"][ks], t["v_prefix"][ks],
+                                     t["k_tree"][ks], t["v_tree"][ks], self.parents[seq])

@@ -138,6 +138,38 @@ def test_llama7b_shape_two_layers_bf16(trj):
     model.close()
 
 
+def test_grouped_query_tiny_fp32_16_steps(trj):
+    """Grouped-query attention on the tiny fp32 shape (4 query heads over 2 K/V heads), generic kernels."""
+    cfg = synth.TINY_GQA
+    model, dec = make_models(trj, cfg, 3, max_seq=512, max_rows=64)
+    assert model.k_cache.shape[2] == 2
+    prompt = synth.prompt(3, 64, cfg.vocab)
+    draw = lambda s, n: synth.noise_draws(3, s, n)
+    trace = []
+    oracle.tr_jacobi_generate(dec, prompt, 80, 4, 2, 3, draw, trace=trace)
+    trace = trace[:16]
+    stats = drive_with_oracle_trace(trj, model, prompt, trace, tol=1e-3)
+    assert stats["rows"] > 120 and stats["path_checked"] >= 12
+    model.close()
+
+
+def test_llama3_8b_shape_two_layers_bf16(trj):
+    """The LLaMA-3-8B layer shape (d 4096, 32 query heads over 8 K/V heads of 128, MLP 14336, vocabulary 128 256,
+    rotary base 5e5), 2 layers, 33-row trees, bf16: the tcgen05 kernels with grouped-query attention."""
+    cfg = synth.LLAMA3_8B.with_layers(2)
+    model, dec = make_models(trj, cfg, 5, max_seq=256, max_rows=128)
+    prompt = synth.prompt(5, 40, cfg.vocab)
+    draw = lambda s, n: synth.noise_draws(5, s, n)
+    trace = []
+    oracle.tr_jacobi_generate(dec, prompt, 6, 5, 9, 3, draw, trace=trace)
+    trace = trace[:3]
+    assert all(len(r["tokens"]) == 33 for r in trace)
+    stats = drive_with_oracle_trace(trj, model, prompt, trace, tol=2e-2)
+    model.device_status()
+    assert stats["rows"] > 60
+    model.close()
+
+
 def test_programmatic_launch_does_not_change_results(trj):
     """The chain's kernels start on chain-invariant data before their predecessor has finished (tensor maps, weights,
     batch geometry, cached K/V rows).  If any of that were data the predecessor still writes, the result would

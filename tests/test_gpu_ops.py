@@ -89,6 +89,21 @@ def test_tree_attention_config5_ragged_batch(trj):
     check_attention(trj, case, heads=[0, 1, 7, 12, 16, 23, 30, 31])
 
 
+@pytest.mark.parametrize("dtype,h,hk,d,prefixes,rows", [
+    ("bf16", 32, 8, 128, [1024], [64]),                    # LLaMA-3 head layout on the config-2 shape (clusters)
+    ("bf16", 8, 2, 128, [3000], [128]),                    # long prefix: clusters whose ring wraps
+    ("bf16", 32, 8, 128, [700, 2200, 256], [33, 16, 64]),  # ragged batch: contiguous ranges + merge kernel
+    ("bf16", 4, 1, 128, [130], [9]),                       # multi-query
+    ("f32", 4, 2, 64, [70], [11]),                         # the generic kernel
+])
+def test_tree_attention_grouped_query(trj, dtype, h, hk, d, prefixes, rows):
+    """Grouped-query attention (LLaMA-3 family, Table 2): H query heads over Hkv K/V heads."""
+    parents = [synth.random_tree(70 + i, m, min(6, m - 1), 3) for i, m in enumerate(rows)]
+    case = AttnCase(trj, 9, h, d, prefixes, rows, parents, dtype, pad=4, kv_heads=hk)
+    heads = None if h <= 8 else [0, 3, 4, 7, 13, 20, 27, 31]
+    check_attention(trj, case, heads=heads)
+
+
 def test_tensor_core_shapes_are_never_rerouted(trj):
     """A bf16 / head_dim-128 attention call or a projection of a tensor-core shape with a short or misaligned
     workspace is an error, not a silent run on the generic kernel."""

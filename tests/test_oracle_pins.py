@@ -200,6 +200,86 @@ def test_matches_independent_library_decoder(dec):
     np.testing.assert_allclose(got, ref, rtol=0, atol=2e-6)
 
 
+def _load_into_library_decoder(tf, torch, dec):
+    cfg = dec.cfg
+    hc = tf.LlamaConfig(vocab_size=cfg.vocab, hidden_size=cfg.d_model, intermediate_size=cfg.d_ff,
+                        num_hidden_layers=cfg.n_layers, num_attention_heads=cfg.n_heads,
+                        num_key_value_heads=cfg.kv_heads, head_dim=cfg.head_dim, rms_norm_eps=cfg.rms_eps,
+                        rope_theta=cfg.rope_theta, attention_bias=False, mlp_bias=False,
+                        tie_word_embeddings=False, max_position_embeddings=256)
+    hf = tf.LlamaForCausalLM(hc).double().eval()
+    hd, kvd = cfg.n_heads * cfg.head_dim, cfg.kv_heads * cfg.head_dim
+    sd = {"model.embed_tokens.weight": dec.glob["embed"], "lm_head.weight": dec.glob["lm_head"],
+          "model.norm.weight": dec.glob["final_norm"]}
+    for l in range(cfg.n_layers):
+        w, p = dec.layers[l], f"model.layers.{l}."
+        sd[p + "self_attn.q_proj.weight"] = w["wqkv"][:hd]
+        sd[p + "self_attn.k_proj.weight"] = w["wqkv"][hd:hd + kvd]
+        sd[p + "self_attn.v_proj.weight"] = w["wqkv"][hd + kvd:]
+        sd[p + "self_attn.o_proj.weight"] = w["wo"]
+        sd[p + "mlp.gate_proj.weight"] = w["w_gate_up"][:cfg.d_ff]
+        sd[p + "mlp.up_proj.weight"] = w["w_gate_up"][cfg.d_ff:]
+        sd[p + "mlp.down_proj.weight"] = w["w_down"]
+        sd[p + "input_layernorm.weight"] = w["attn_norm"]
+        sd[p + "post_attention_layernorm.weight"] = w["mlp_norm"]
+    missing = hf.load_state_dict({k: torch.tensor(np.asarray(v), dtype=torch.float64) for k, v in sd.items()},
+                                 strict=False)
+    assert not [k for k in missing.missing_keys if "rotary" not in k and "inv_freq" not in k]
+    return hf
+
+
+def test_grouped_query_attention_matches_library_decoder():
+    """Grouped-query attention (the LLaMA-3 family of Table 2): 4 query heads over 2 K/V heads on the tiny shape
+    give the causal logits of transformers' LLaMA with num_key_value_heads = 2."""
+    torch = pytest.importorskip("torch")
+    tf = pytest.importorskip("transformers")
+    dec = tiny_decoder(3, synth.TINY_GQA)
+    hf = _load_into_library_decoder(tf, torch, dec)
+    toks = synth.prompt(19, 20, dec.cfg.vocab)
+    with torch.no_grad():
+        ref = hf(torch.tensor(toks[None].astype(np.int64))).logits[0].numpy()
+    got = dec.forward_rows(dec.new_cache(32), toks, synth.chain_parents(20))
+    np.testing.assert_allclose(got, ref, rtol=0, atol=2e-6)
+
+
+def test_grouped_query_attention_is_multi_head_attention_with_repeated_kv():
+    """A grouped-query model is the multi-head model whose K/V projection rows are repeated once per query head of
+    the group: same logits and, head for head, the same cache rows, on a branching tree over a non-empty cache."""
+    from dataclasses import replace
+    cfg = synth.TINY_GQA
+    dec = tiny_decoder(5, cfg)
+    h, kv, d = cfg.n_heads, cfg.kv_heads, cfg.head_dim
+    rep = np.repeat(np.arange(kv), h // kv)                  # K/V head of every query head
+    wide_layers = []
+    for w in dec.layers:
+        wq, wk, wv = w["wqkv"][:h * d], w["wqkv"][h * d:(h + kv) * d], w["wqkv"][(h + kv) * d:]
+        wk = wk.reshape(kv, d, -1)[rep].reshape(h * d, -1)
+        wv = wv.reshape(kv, d, -1)[rep].reshape(h * d, -1)
+        wide_layers.append({**w, "wqkv": np.concatenate([wq, wk, wv], 0)})
+    wide = oracle.Decoder(replace(cfg, n_kv_heads=0), wide_layers, dec.glob)
+    prompt = synth.prompt(6, 12, cfg.vocab)
+    parent = synth.random_tree(6, 14, 4, 3)
+    tokens = synth.prompt(7, 14, cfg.vocab)
+    outs = []
+    for model in (dec, wide):
+        cache = model.new_cache(40)
+        model.forward_rows(cache, prompt, synth.chain_parents(12))
+        cache.seq_len = 12
+        outs.append((model.forward_rows(cache, tokens, parent), cache))
+    np.testing.assert_allclose(outs[0][0], outs[1][0], rtol=0, atol=1e-12)
+    np.testing.assert_allclose(outs[0][1].k[:, rep], outs[1][1].k, rtol=0, atol=1e-13)
+    assert outs[0][1].k.shape[1] == kv and outs[1][1].k.shape[1] == h
+
+
+def test_grouped_query_tr_jacobi_equals_autoregressive():
+    """Eq. 1 with grouped-query attention: greedy TR-Jacobi commits the autoregressive tokens."""
+    dec = tiny_decoder(3, synth.TINY_GQA)
+    pr = synth.prompt(2, 40, dec.cfg.vocab)
+    ar = oracle.autoregressive_greedy(dec, pr, 24)
+    got = oracle.tr_jacobi_generate(dec, pr, 24, 4, 2, 3, lambda s, n: synth.noise_draws(8, s, n))
+    assert got == ar
+
+
 # ---------------------------------------------------------------- Eq. 1, Sections 2.1 and 3.3
 @pytest.mark.parametrize("width,n_br,br_len,seed", [(4, 2, 3, 0), (5, 3, 3, 1), (3, 0, 0, 2), (1, 1, 5, 3), (8, 1, 2, 4)])
 def test_tr_jacobi_equals_autoregressive(dec, ar_tokens, width, n_br, br_len, seed):
