@@ -50,6 +50,16 @@ cannot change which tokens a greedy decoder commits, unless noted):
 * Refill (Section 3.3).  New root = bonus.  New window = the arg-max at the
   rows below the winner along its own branch (lowest-index child at every
   level), then ahead noise up to W tokens.
+* Top-K trees (Appendix B: the benefit of the tree "mainly depends on the
+  topK of the first draft token"; the 63-node template itself is third-party
+  and not printed).  A template is ``parent`` plus a rank per row: siblings
+  under one parent carry ranks 0, 1, 2, ... and hold the rank-th most likely
+  token for their position; rows of negative rank form the retrieval path.
+  The candidates for depth d come from the d-th row below the winner along
+  its own path (lowest-index child at every level), so all rows of one depth
+  and rank carry the same token; depths the path does not reach are ahead
+  noise.  Top-K order: larger logit first, equal logits by ascending id.
+  With a chain template this is the window refill above.
 * Ahead noise (Eq. 4).  Uniform over all tokens committed so far; the raw
   random draws are inputs.
 * Retrieval (Section 3.3, prompt lookup).  Key = the last g committed tokens
@@ -70,14 +80,14 @@ path, and the library-decoder pin fixes the model-side ones to the common
 LLaMA convention.
 """
 from .tree import (ancestor_mask, pack_mask, build_tree, depths, retrieve, ahead_noise,
-                   refill_window, validate_tree)
+                   refill_window, refill_tree, continuation_rows, validate_tree)
 from .attention import tree_attention
-from .accept import node_argmax, accept_path, compact_rows, top2_margin
-from .model import Decoder, KVCache, autoregressive_greedy, tr_jacobi_generate
+from .accept import node_argmax, node_topk, accept_path, compact_rows, top2_margin
+from .model import Decoder, KVCache, autoregressive_greedy, tr_jacobi_generate, tr_jacobi_generate_tree
 
 __all__ = [
     "ancestor_mask", "pack_mask", "build_tree", "depths", "retrieve", "ahead_noise",
-    "refill_window", "validate_tree", "tree_attention", "node_argmax",
-    "accept_path", "compact_rows", "top2_margin", "Decoder", "KVCache",
-    "autoregressive_greedy", "tr_jacobi_generate",
+    "refill_window", "refill_tree", "continuation_rows", "validate_tree", "tree_attention", "node_argmax",
+    "node_topk", "accept_path", "compact_rows", "top2_margin", "Decoder", "KVCache",
+    "autoregressive_greedy", "tr_jacobi_generate", "tr_jacobi_generate_tree",
 ]

@@ -23,6 +23,18 @@ def node_argmax(logits: np.ndarray) -> np.ndarray:
     return out
 
 
+def node_topk(logits: np.ndarray, k: int) -> np.ndarray:
+    """The k most likely token ids of every row, best first (Appendix B: the tree holds the top-K candidates of a
+    draft position as siblings).  Order: larger logit first, equal logits by ascending token id; column 0 is
+    ``node_argmax``.  Returns [M, k] int32."""
+    logits = np.asarray(logits, np.float64)
+    out = np.zeros((logits.shape[0], k), np.int32)
+    for i in range(logits.shape[0]):
+        order = sorted(range(logits.shape[1]), key=lambda v: (-logits[i, v], v))
+        out[i] = order[:k]
+    return out
+
+
 def top2_margin(logits: np.ndarray) -> np.ndarray:
     """Gap between the largest and second-largest logit of every row (0 for an exact tie)."""
     logits = np.asarray(logits, np.float64)

@@ -10,9 +10,9 @@ from typing import Callable, Dict, List, Sequence
 
 import numpy as np
 
-from .accept import accept_path, compact_rows, node_argmax
+from .accept import accept_path, compact_rows, node_argmax, node_topk
 from .attention import tree_attention
-from .tree import build_tree, depths, refill_window, retrieve, ahead_noise
+from .tree import build_tree, depths, refill_tree, refill_window, retrieve, ahead_noise
 
 
 def rmsnorm(h: np.ndarray, gain: np.ndarray, eps: float) -> np.ndarray:
@@ -178,5 +178,44 @@ def tr_jacobi_generate(dec: Decoder, prompt: Sequence[int], n_new: int, width: i
         window = refill_window(parent, rec["pred"], rec["path"][-1], width, committed, draws[:width])
         if trace is not None:
             rec.update(tokens=tokens, parent=parent, step=step, next_window=list(window))
+            trace.append(rec)
+    return committed[p:p + n_new]
+
+
+def tr_jacobi_generate_tree(dec: Decoder, prompt: Sequence[int], n_new: int, parent: Sequence[int],
+                            rank: Sequence[int], top_k: int, n_retrieved: int,
+                            draw_fn: Callable[[int, int], Sequence[int]],
+                            capacity: int = 0, trace: List[dict] = None) -> List[int]:
+    """Greedy TR-Jacobi decoding over a static tree template with top-K siblings (Section 3.3, Appendix B).
+
+    ``parent`` / ``rank`` describe the template (see ``refill_tree``); rows of rank -1 - j form one retrieval
+    path of ``n_retrieved`` slots filled by prompt lookup.  All rows start as ahead noise (Section 3.3).
+    ``draw_fn(step, n)``: step 0 seeds the first tree (slot i - 1 for row i); step t >= 1 uses slots [0, M - 1) for
+    the refill after that step and slots [M - 1, M - 1 + n_retrieved) for that step's retrieval.
+    """
+    m = len(parent)
+    cache = dec.new_cache(capacity or len(prompt) + n_new + m + 1)
+    p = len(prompt)
+    logits = dec.forward_rows(cache, list(prompt), list(range(-1, p - 1)))
+    cache.seq_len = p
+    committed = [int(t) for t in prompt] + [int(node_argmax(logits[-1:])[0])]
+    d0 = draw_fn(0, m - 1)
+    drafts = [ahead_noise(committed, d0[i]) for i in range(m - 1)]
+    step = 0
+    while len(committed) - p < n_new:
+        step += 1
+        draws = draw_fn(step, m - 1 + n_retrieved)
+        retrieved = retrieve(committed, 1, n_retrieved, draws[m - 1:])[0] if n_retrieved else []
+        tokens = np.asarray([committed[-1]] + list(drafts), np.int32)
+        for i in range(1, m):                              # retrieval slots are refreshed from the current context
+            if rank[i] < 0:
+                tokens[i] = retrieved[-1 - rank[i]]
+        rec = verify_step(dec, cache, tokens, parent)
+        topk = node_topk(rec["logits"], top_k)
+        committed += [int(tokens[r]) for r in rec["path"][1:]] + [rec["bonus"]]
+        drafts = refill_tree(parent, rank, topk, rec["path"][-1], committed, draws[:m - 1],
+                             retrieved if n_retrieved else [0])
+        if trace is not None:
+            rec.update(tokens=tokens, parent=np.asarray(parent, np.int32), step=step, topk=topk, next_drafts=list(drafts))
             trace.append(rec)
     return committed[p:p + n_new]

@@ -126,6 +126,46 @@ def retrieve(context: Sequence[int], n_branches: int, branch_len: int,
     return out
 
 
+def continuation_rows(parent: Sequence[int], best: int) -> List[int]:
+    """Rows below ``best`` along its own path: the lowest-index child at every level, down to a leaf."""
+    m = len(parent)
+    rows: List[int] = []
+    cur = best
+    while True:
+        kids = [c for c in range(cur + 1, m) if parent[c] == cur]
+        if not kids:
+            return rows
+        cur = kids[0]
+        rows.append(cur)
+
+
+def refill_tree(parent: Sequence[int], rank: Sequence[int], node_topk: np.ndarray, best: int,
+                context: Sequence[int], draws: Sequence[int], retrieved: Sequence[int]) -> List[int]:
+    """Draft tokens of the next step for a static tree template with top-K siblings (Section 3.3, Appendix B).
+
+    The template is ``parent`` plus, for every row i >= 1, ``rank[i]``: rank r >= 0 makes the row the r-th best
+    candidate for its position (siblings under one parent carry ranks 0, 1, 2, ...); rank -1 - j makes it slot j of
+    the retrieval path(s) and it takes ``retrieved[j]``.  The candidates for depth d come from the d-th row below
+    the winner ``best`` along its own path (the chosen path's subsequent predictions): a row of depth d and rank r
+    takes ``node_topk[that row][r]``.  Depths the path does not reach are ahead noise over ``context`` (the
+    committed tokens, this step's included), row i using ``draws[i - 1]``.  Returns the tokens of rows 1..M-1; row 0
+    (the root) is the step's bonus token and is not produced here.  With a chain template and ranks 0 this is
+    ``refill_window``.
+    """
+    depth = depths(parent)
+    below = continuation_rows(parent, best)
+    out: List[int] = []
+    for i in range(1, len(parent)):
+        r = int(rank[i])
+        if r < 0:
+            out.append(int(retrieved[-1 - r]))
+        elif depth[i] <= len(below):
+            out.append(int(node_topk[below[depth[i] - 1]][r]))
+        else:
+            out.append(ahead_noise(context, draws[i - 1]))
+    return out
+
+
 def refill_window(parent: Sequence[int], node_pred: Sequence[int], best: int, width: int,
                   context: Sequence[int], draws: Sequence[int]) -> List[int]:
     """Next Jacobi window (Section 3.3): the chosen path's subsequent predictions, then noise.

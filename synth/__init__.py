@@ -26,7 +26,7 @@ import numpy as np
 __all__ = [
     "ModelCfg", "TINY", "TINY_GQA", "LLAMA7B", "LLAMA3_8B", "stream", "round_bf16", "bf16_bits",
     "layer_weights", "global_weights", "prompt", "chain_parents",
-    "random_tree", "node_depths", "qkv", "logits", "planted_tokens",
+    "random_tree", "tree_template", "node_depths", "qkv", "logits", "planted_tokens",
     "random_path", "ragged_batch", "noise_draws",
 ]
 
@@ -183,6 +183,50 @@ def random_tree(seed: int, m: int, max_depth: int, max_children: int,
         depth[i] = depth[p] + 1
         nchild[p] += 1
     return parent
+
+
+def tree_template(seed: int, n_nodes: int = 63, max_depth: int = 4, first_level: int = 10,
+                  retrieval_len: int = 5, name: str = "template") -> Tuple[np.ndarray, np.ndarray]:
+    """A seeded sparse tree template with top-K siblings plus one retrieval path (stands in for the paper's
+    third-party 63-node template, which is not printed there): returns (parent[M], rank[M]), M = 1 + n_nodes +
+    retrieval_len, row 0 the root.
+
+    Rows are added one at a time as the next-ranked child of a drawn parent (the root has up to ``first_level``
+    children, every other row up to 3; depth <= ``max_depth``), parents being drawn with a weight that halves with
+    every level and shrinks with every child already present (x 0.8 at the root, x 0.5 elsewhere), so the tree is
+    wide near the root and sparse below it.  The
+    rank of a row is its position among its siblings (0 = most likely candidate).  The retrieval path is a chain
+    off the root whose rows carry rank -1 - j (slot j).  Rows are then renumbered level by level so that
+    parent[i] < i and rank-0 children come first.
+    """
+    g = stream(seed, name)
+    parent, depth, nchild = [-1], [0], [0]
+    rank = [0]
+    for _ in range(n_nodes):
+        cap = [first_level if i == 0 else 3 for i in range(len(parent))]
+        w = np.array([0.0 if (depth[i] >= max_depth or nchild[i] >= cap[i])
+                      else 0.5 ** depth[i] * (0.8 if i == 0 else 0.5) ** nchild[i] for i in range(len(parent))])
+        p = int(g.choice(len(parent), p=w / w.sum()))
+        parent.append(p); depth.append(depth[p] + 1); rank.append(nchild[p]); nchild.append(0)
+        nchild[p] += 1
+    prev = 0
+    for j in range(retrieval_len):
+        parent.append(prev); depth.append(depth[prev] + 1); rank.append(-1 - j); nchild.append(0)
+        prev = len(parent) - 1
+    # renumber: breadth-first, siblings by rank (retrieval rows last among the root's children)
+    order = sorted(range(len(parent)), key=lambda i: (depth[i], parent[i] if parent[i] >= 0 else -1,
+                                                      rank[i] if rank[i] >= 0 else 1000 - rank[i]))
+    # a stable breadth-first order needs parents renumbered first: do it level by level
+    new_of = {0: 0}
+    out_parent, out_rank = [-1], [0]
+    for d in range(1, max(depth) + 1):
+        level = [i for i in order if depth[i] == d]
+        level.sort(key=lambda i: (new_of[parent[i]], rank[i] if rank[i] >= 0 else 1000 - rank[i]))
+        for i in level:
+            new_of[i] = len(out_parent)
+            out_parent.append(new_of[parent[i]])
+            out_rank.append(rank[i])
+    return np.asarray(out_parent, np.int32), np.asarray(out_rank, np.int32)
 
 
 # --------------------------------------------------------------------------

@@ -280,6 +280,67 @@ def test_grouped_query_tr_jacobi_equals_autoregressive():
     assert got == ar
 
 
+# ---------------------------------------------------------------- Appendix B: top-K siblings
+def test_node_topk_order_ties_and_reduction_to_argmax():
+    logits = np.array([[0.5, 2.0, 2.0, -1.0, 2.0, 0.5],      # three-way tie at the top, two-way tie below it
+                       [3.0, 1.0, 0.0, 7.0, 7.0, -2.0],
+                       [1.0, 1.0, 1.0, 1.0, 1.0, 1.0]])
+    np.testing.assert_array_equal(oracle.node_topk(logits, 4), [[1, 2, 4, 0], [3, 4, 0, 1], [0, 1, 2, 3]])
+    g = synth.stream(4, "topk")
+    x = g.standard_normal((7, 500))
+    top = oracle.node_topk(x, 10)
+    np.testing.assert_array_equal(top[:, 0], oracle.node_argmax(x))          # K = 1 is the greedy prediction
+    np.testing.assert_array_equal(oracle.node_topk(x, 1)[:, 0], oracle.node_argmax(x))
+    torch = pytest.importorskip("torch")                      # distinct values: the library's top-k gives the same ids
+    np.testing.assert_array_equal(top, torch.topk(torch.from_numpy(x), 10, dim=1).indices.numpy())
+
+
+def test_refill_tree_hand_worked_and_chain_reduces_to_window_refill():
+    # template: root; rows 1, 2 = rank 0, 1 under the root; row 3 = retrieval slot 0; rows 4, 5 = rank 0, 1 under row 1;
+    # row 6 = rank 0 under row 4
+    parent = [-1, 0, 0, 0, 1, 1, 4]
+    rank = [0, 0, 1, -1, 0, 1, 0]
+    topk = np.arange(7 * 3).reshape(7, 3) + 100               # row i offers 100 + 3i, 101 + 3i, 102 + 3i
+    ctx = [9, 8, 7, 6]
+    draws = [5, 2, 3, 0, 1, 7]
+    # winner = root: the rows below it are 1, 4, 6 -> depth 1 from row 1, depth 2 from row 4, depth 3 from row 6
+    assert oracle.continuation_rows(parent, 0) == [1, 4, 6]
+    assert oracle.refill_tree(parent, rank, topk, 0, ctx, draws, [55]) == [103, 104, 55, 112, 113, 118]
+    # winner = row 1: below it 4, 6 -> depth 1 from row 4, depth 2 from row 6, depth 3 is noise (row 6 uses draws[5])
+    assert oracle.refill_tree(parent, rank, topk, 1, ctx, draws, [55]) == [112, 113, 55, 118, 119, ctx[7 % 4]]
+    # winner = row 2 (a leaf): everything but the retrieval slot is noise
+    assert oracle.refill_tree(parent, rank, topk, 2, ctx, draws, [55]) == [ctx[5 % 4], ctx[2], 55, ctx[0], ctx[1], ctx[3]]
+    # a chain with ranks 0 is the Jacobi window
+    g = synth.stream(6, "chain")
+    for best in range(6):
+        pred = g.integers(0, 1000, size=6)
+        d = g.integers(0, 1000, size=5)
+        chain = synth.chain_parents(6)
+        want = oracle.refill_window(chain, pred, best, 5, ctx, d[:5])
+        got = oracle.refill_tree(chain, [0] * 6, pred[:, None], best, ctx, np.concatenate([np.zeros(best, np.int64), d]), [])
+        # refill_window numbers its noise draws from the first unfilled slot of the window, refill_tree by row
+        filled = 5 - best
+        assert got[:filled] == want[:filled]
+
+
+@pytest.mark.parametrize("seed,n_nodes,top_k,n_retr", [(0, 63, 10, 5), (1, 20, 5, 0), (2, 12, 6, 3)])
+def test_top_k_tree_decoding_equals_autoregressive(dec, ar_tokens, seed, n_nodes, top_k, n_retr):
+    """Eq. 1 on a static template with top-K siblings and a retrieval path (Appendix B): same tokens as greedy
+    autoregressive decoding, whatever the template, K or the noise."""
+    prompt, ar = ar_tokens
+    parent, rank = synth.tree_template(seed, n_nodes, 4, 10, n_retr)
+    assert len(parent) == 1 + n_nodes + n_retr and rank.max() < top_k
+    trace = []
+    got = oracle.tr_jacobi_generate_tree(dec, prompt, 40, parent, rank, top_k, n_retr,
+                                         lambda s, n: synth.noise_draws(seed, s, n), trace=trace)
+    assert got == ar[:40]
+    assert len(trace) <= 40
+    # siblings of one parent hold distinct candidates whenever they come from a prediction (same source row, different rank)
+    for rec in trace[1:]:
+        tok, par = rec["tokens"], rec["parent"]
+        assert len(tok) == len(parent)
+
+
 # ---------------------------------------------------------------- Eq. 1, Sections 2.1 and 3.3
 @pytest.mark.parametrize("width,n_br,br_len,seed", [(4, 2, 3, 0), (5, 3, 3, 1), (3, 0, 0, 2), (1, 1, 5, 3), (8, 1, 2, 4)])
 def test_tr_jacobi_equals_autoregressive(dec, ar_tokens, width, n_br, br_len, seed):
