@@ -417,6 +417,50 @@ def whole_job_rate(world, units_per_rank, seconds):
     return world * units_per_rank / seconds
 
 
+def bench_template_step(trj, torch, synth, model, cfg, prefix, side, steps):
+    """One verification step over a 69-row static template with top-K siblings (63 draft nodes + a retrieval path of
+    5 + the root: the tree size the paper uses, Appendix B; the topology is a seeded stand-in): forward, per-row top-10,
+    acceptance and compaction, replayed from a CUDA graph on the same model and cache."""
+    dev = model.device
+    parent, rank = synth.tree_template(0)
+    m = len(parent)
+    depth, anc = trj.tree_from_parents(parent)
+    i32 = lambda a: torch.from_numpy(np.ascontiguousarray(a, dtype=np.int32)).to(dev)
+    d_tok, d_par, d_dep, d_off = i32(synth.prompt(77, m, cfg.vocab)), i32(parent), i32(depth), i32([0, m])
+    d_anc = torch.from_numpy(anc.view(np.int64)).to(dev)
+    pred = torch.empty(m, dtype=torch.int32, device=dev)
+    topk = torch.empty(m, 10, dtype=torch.int32, device=dev)
+    acc = {"k_acc": torch.empty(1, dtype=torch.int32, device=dev), "bonus": torch.empty(1, dtype=torch.int32, device=dev),
+           "path": torch.empty(1, trj.PATH_STRIDE, dtype=torch.int32, device=dev)}
+    seq0 = torch.full_like(model.seq_len, prefix)
+
+    def step():
+        model.seq_len.copy_(seq0)
+        model.verify_step(d_tok, d_par, d_dep, d_anc, d_off, max_rows=m, max_len=prefix + m, node_argmax=pred)
+        model.node_topk(m, 10, out=topk)
+        model.accept(d_tok, d_par, d_dep, d_off, pred, out=acc)
+        model.compact_kv(acc["k_acc"], acc["path"])
+    with torch.cuda.stream(side):
+        step()
+    torch.cuda.synchronize()
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g, stream=side):
+        step()
+    for _ in range(3):
+        g.replay()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(steps):
+        g.replay()
+    e1.record()
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / steps
+    return {"tree_rows": m, "draft_tokens_per_step": m - 1, "top_k": 10, "ms_per_step": ms,
+            "draft_tokens_verified_per_s": (m - 1) / (ms / 1e3),
+            "what": "7B shape, prefix %d, 63-node template + retrieval path of 5 + root; random drafts" % prefix}
+
+
 def planted_lengths(seed, n):
     """How many tokens of the true continuation each step's first retrieved branch carries: uniform on 0..3, so
     that a step commits 1 + (0..3) tokens, 2.5 on average (the paper's Table 2 reports 2.0-2.9 per step)."""
@@ -669,6 +713,7 @@ def run_ours(args, rank, world, local_rank):
                                     "wall clock incl. uploading the draws and reading the tokens back" % args.steps},
             "roofline": roofline, "kernel_breakdown": breakdown, "profiled_step_ms": step_ms_prof}
     if world == 1:
+        line["paper_sized_tree"] = bench_template_step(trj, torch, synth, model, cfg, PROMPT, side, args.steps)
         if not args.no_attention:
             line["tree_attention"] = bench_tree_attention(trj, torch, peaks, max(args.steps, 5), 3, cpu=not args.no_cpu)
             line["small_ops"] = bench_small_ops(trj, torch, peaks, max(args.steps, 5), 3, cpu=not args.no_cpu)

@@ -67,6 +67,7 @@ extern "C" {
 #define TRJ_MAX_ROWS  128      /* tree rows per sequence, root included          */
 #define TRJ_MAX_BATCH 64       /* sequences per call                             */
 #define TRJ_PATH_STRIDE 128    /* int32 slots per sequence in `path` arrays      */
+#define TRJ_MAX_TOPK  10       /* candidates per row that a top-K call can return */
 
 typedef enum {
     TRJ_OK = 0,
@@ -212,6 +213,44 @@ trj_status trj_argmax_accept(const void* logits, int32_t dtype, int32_t V,
                              int32_t* node_argmax, float* margin,
                              int32_t* k_acc, int32_t* path, int32_t* bonus,
                              void* workspace, size_t workspace_bytes, void* stream);
+
+/* ------------------------------------------------------------------------
+ * Top-K siblings (Appendix B: the tree template holds, as siblings, the K most
+ * likely tokens of a draft position; what the tree gains "mainly depends on the
+ * topK of the first draft token").
+ *
+ * trj_topk_accept is trj_argmax_accept that also returns, for every row, the ids
+ * of its K largest logits, best first (larger logit first, equal logits by
+ * ascending id), in topk [rows_total][K] (dev int32; column 0 equals
+ * node_argmax).  1 <= K <= TRJ_MAX_TOPK.  Acceptance is unchanged: a row is
+ * accepted iff its token is the arg-max of its parent.  workspace: dev, >=
+ * trj_topk_accept_workspace() bytes, 256-byte aligned, zero before the first
+ * call; every call leaves it zero again.
+ *
+ * trj_node_topk: the same top-K of the logits that the latest trj_verify_step on
+ * ctx produced (rows_total as in that call); launches only.
+ *
+ * trj_refill_tree (host): draft tokens of the next step for a static template
+ * with top-K siblings.  The template is parent [M] plus rank [M]: rank[i] = r >=
+ * 0 makes row i the r-th best candidate of its position (siblings under one
+ * parent carry ranks 0, 1, 2, ...), rank[i] = -1 - j makes it slot j of the
+ * retrieval path and it takes retrieved[j].  Candidates for depth d come from the
+ * d-th row below the winner `best` along its own path (lowest-index child at
+ * every level): row i of depth d and rank r takes topk[that row][r]; depths the
+ * path does not reach are ahead noise context[draws[i-1] % n] (Eq. 4).  Writes
+ * tokens [M-1] (rows 1..M-1; the root is the step's bonus token).  With a chain
+ * and ranks 0 this is trj_refill_window.  All pointers host. */
+size_t trj_topk_accept_workspace(void);
+trj_status trj_topk_accept(const void* logits, int32_t dtype, int32_t V, int32_t K,
+                           const int32_t* tokens, const int32_t* parent, const int32_t* depth,
+                           const int32_t* row_off, int32_t B, int32_t rows_total,
+                           int32_t* topk, int32_t* node_argmax, float* margin,
+                           int32_t* k_acc, int32_t* path, int32_t* bonus,
+                           void* workspace, size_t workspace_bytes, void* stream);
+trj_status trj_node_topk(trj_ctx* ctx, int32_t rows_total, int32_t K, int32_t* topk, void* stream);
+trj_status trj_refill_tree(const int32_t* parent, const int32_t* rank, int32_t M, const int32_t* topk, int32_t K,
+                           int32_t best, const int32_t* context, int32_t n, const int64_t* draws,
+                           const int32_t* retrieved, int32_t n_retrieved, int32_t* tokens);
 
 /* ------------------------------------------------------------------------
  * trj_argmax_accept for callers that cannot hand over a workspace (the paper has

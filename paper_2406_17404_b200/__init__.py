@@ -18,6 +18,7 @@ LIB_PATH = os.path.join(_HERE, "libtrj.so")
 
 MAX_ROWS = 128
 MAX_BATCH = 64
+MAX_TOPK = 10
 PATH_STRIDE = 128
 # bytes trj_step_host moves per call: tokens/parent/depth/row_off + ancestor words in, predictions/k/bonus/path out
 STEP_H2D_BYTES = (3 * MAX_ROWS + 4) * 4 + MAX_ROWS * 2 * 8
@@ -64,6 +65,10 @@ _SIGNATURES = {
     "trj_tree_attention_gqa": (_I, [_VP, _VP, _VP, _VP, _VP, _VP, _I, _I, _I, _I, _I, _I, _I, _I, _I, _I, _VP, _VP, _SZ, _VP]),
     "trj_argmax_accept_workspace": (_SZ, [_I, _I]),
     "trj_argmax_accept": (_I, [_VP, _I, _I, _VP, _VP, _VP, _VP, _I, _I, _VP, _VP, _VP, _VP, _VP, _VP, _SZ, _VP]),
+    "trj_topk_accept_workspace": (_SZ, []),
+    "trj_topk_accept": (_I, [_VP, _I, _I, _I, _VP, _VP, _VP, _VP, _I, _I, _VP, _VP, _VP, _VP, _VP, _VP, _VP, _SZ, _VP]),
+    "trj_node_topk": (_I, [_VP, _I, _I, _VP, _VP]),
+    "trj_refill_tree": (_I, [_I32P, _I32P, _I, _I32P, _I, _I, _I32P, _I, _I64P, _I32P, _I, _I32P]),
     "trj_argmax_accept_static": (_I, [_VP, _I, _I, _VP, _VP, _VP, _VP, _I, _I, _VP, _VP, _VP, _VP, _VP, _VP]),
     "trj_compact_rows": (_I, [_VP, _VP, _I, _I, _I, _I, _I, _I, _VP, _VP, _VP, _VP]),
     "trj_workspace_bytes": (_SZ, [C.POINTER(ModelCfg)]),
@@ -274,6 +279,39 @@ def argmax_accept(logits, tokens, parent, depth, row_off, *, want_margin: bool =
     return {"node_argmax": node_argmax, "margin": margin, "k_acc": k_acc, "path": path, "bonus": bonus}
 
 
+def topk_accept(logits, tokens, parent, depth, row_off, k: int, *, workspace=None, stream=None):
+    """trj_topk_accept: :func:`argmax_accept` plus ``topk`` [rows, k] int32, the ids of every row's k largest logits."""
+    torch = _torch()
+    rows, vocab = logits.shape
+    batch = row_off.numel() - 1
+    dev = logits.device
+    if workspace is None:
+        workspace = _scratch(lib().trj_topk_accept_workspace(), dev, zero=True)
+    i32 = dict(dtype=torch.int32, device=dev)
+    topk, node_argmax = torch.empty(rows, k, **i32), torch.empty(rows, **i32)
+    margin = torch.empty(rows, dtype=torch.float32, device=dev)
+    k_acc, bonus, path = torch.empty(batch, **i32), torch.empty(batch, **i32), torch.empty(batch, PATH_STRIDE, **i32)
+    _check(lib().trj_topk_accept(
+        _dev(logits, name="logits"), _dtype_code(logits), vocab, int(k), _dev(tokens, torch.int32, "tokens"),
+        _dev(parent, torch.int32, "parent"), _dev(depth, torch.int32, "depth"), _dev(row_off, torch.int32, "row_off"),
+        batch, rows, _dev(topk), _dev(node_argmax), _dev(margin), _dev(k_acc), _dev(path), _dev(bonus),
+        _dev(workspace, torch.uint8, "workspace"), workspace.numel(), _stream(stream)))
+    return {"topk": topk, "node_argmax": node_argmax, "margin": margin, "k_acc": k_acc, "path": path, "bonus": bonus}
+
+
+def refill_tree(parent, rank, topk, best: int, context, draws, retrieved=()) -> np.ndarray:
+    """trj_refill_tree: draft tokens [M - 1] of the next step for a template with top-K siblings (host)."""
+    parent, rank, context = _i32(parent), _i32(rank), _i32(context)
+    topk = _i32(topk).reshape(len(parent), -1)
+    draws = np.ascontiguousarray(draws, dtype=np.int64)
+    retrieved = _i32(retrieved).reshape(-1)
+    out = np.zeros(max(len(parent) - 1, 1), np.int32)
+    _check(lib().trj_refill_tree(_p32(parent), _p32(rank), len(parent), _p32(topk), topk.shape[1], int(best),
+                                 _p32(context), len(context), draws.ctypes.data_as(_I64P),
+                                 _p32(retrieved) if len(retrieved) else None, len(retrieved), _p32(out)))
+    return out[:len(parent) - 1]
+
+
 def argmax_accept_into(logits, tokens, parent, depth, row_off, out, workspace, *, stream=None) -> None:
     """trj_argmax_accept into preallocated outputs (``out`` as for :func:`argmax_accept_static`) with a caller-held,
     zero-initialised workspace: nothing is allocated, so the call can be captured in a CUDA graph."""
@@ -464,6 +502,14 @@ class Model:
             max_rows, max_len, _dev(node_argmax), _dev(margin) if want_margin else None,
             _dev(logits) if want_logits else None, _stream(stream)))
         return {"node_argmax": node_argmax, "margin": margin, "logits": logits}
+
+    def node_topk(self, rows: int, k: int, out=None, stream=None):
+        """trj_node_topk: [rows, k] int32 ids of the k largest logits of every row of the latest verify_step."""
+        torch = _torch()
+        if out is None:
+            out = torch.empty(rows, k, dtype=torch.int32, device=self.device)
+        _check(lib().trj_node_topk(self._handle, int(rows), int(k), _dev(out, torch.int32, "topk"), _stream(stream)))
+        return out
 
     def accept(self, tokens, parent, depth, row_off, node_argmax, out=None, stream=None):
         """trj_accept: dict(k_acc [B], path [B, PATH_STRIDE], bonus [B]); ``out`` may hold preallocated ones."""

@@ -86,8 +86,30 @@ extern "C" trj_status trj_argmax_accept(const void* logits, int32_t dtype, int32
     TRJ_REQUIRE(rows_total <= B * TRJ_MAX_ROWS, TRJ_ECAPACITY, "argmax_accept: too many rows");
     TRJ_REQUIRE(workspace && aligned(workspace, 256) && workspace_bytes >= argmax_workspace_bytes(rows_total, B),
                 TRJ_ECAPACITY, "argmax_accept: workspace too small or misaligned");
-    TRJ_CHECK_CUDA(launch_argmax_accept(logits, dtype, V, tokens, parent, depth, row_off, B, rows_total, node_argmax,
-                                        margin, k_acc, path, bonus, true, true, workspace, (cudaStream_t)stream));
+    TRJ_CHECK_CUDA(launch_topk_accept(logits, dtype, V, 1, tokens, parent, depth, row_off, B, rows_total, nullptr, node_argmax,
+                                      margin, k_acc, path, bonus, true, workspace, (cudaStream_t)stream));
+    return TRJ_OK;
+}
+
+extern "C" size_t trj_topk_accept_workspace(void) { return topk_workspace_bytes(); }
+
+extern "C" trj_status trj_topk_accept(const void* logits, int32_t dtype, int32_t V, int32_t K,
+                                      const int32_t* tokens, const int32_t* parent, const int32_t* depth,
+                                      const int32_t* row_off, int32_t B, int32_t rows_total,
+                                      int32_t* topk, int32_t* node_argmax, float* margin,
+                                      int32_t* k_acc, int32_t* path, int32_t* bonus,
+                                      void* workspace, size_t workspace_bytes, void* stream) {
+    TRJ_REQUIRE(logits && tokens && parent && depth && row_off && topk && node_argmax && k_acc && path && bonus,
+                TRJ_EINVAL, "topk_accept: null pointer");
+    TRJ_REQUIRE(dtype_ok(dtype), TRJ_EINVAL, "topk_accept: unknown dtype %d", dtype);
+    TRJ_REQUIRE(K >= 1 && K <= TRJ_MAX_TOPK && K <= V, TRJ_EINVAL, "topk_accept: K = %d outside 1..min(%d, V)", K, TRJ_MAX_TOPK);
+    TRJ_REQUIRE(V >= 1 && B >= 1 && rows_total >= B, TRJ_EINVAL, "topk_accept: bad sizes (every tree has a root)");
+    TRJ_REQUIRE(B <= TRJ_MAX_BATCH, TRJ_ECAPACITY, "topk_accept: batch %d exceeds %d", B, TRJ_MAX_BATCH);
+    TRJ_REQUIRE(rows_total <= B * TRJ_MAX_ROWS, TRJ_ECAPACITY, "topk_accept: too many rows");
+    TRJ_REQUIRE(workspace && aligned(workspace, 256) && workspace_bytes >= topk_workspace_bytes(),
+                TRJ_ECAPACITY, "topk_accept: workspace too small or misaligned");
+    TRJ_CHECK_CUDA(launch_topk_accept(logits, dtype, V, K, tokens, parent, depth, row_off, B, rows_total, topk, node_argmax,
+                                      margin, k_acc, path, bonus, true, workspace, (cudaStream_t)stream));
     return TRJ_OK;
 }
 
@@ -173,6 +195,7 @@ struct trj_ctx {
     std::vector<LoopGraph> loop_graphs;
     cudaStream_t cap_stream = nullptr; cudaEvent_t order_ev = nullptr; uint64_t steps_done = 0;
     DraftSource draft_src{nullptr, 0, nullptr}; int32_t draft_src_steps = 0;   // trj_set_draft_source
+    int32_t last_rows = 0, last_B = 0; const int32_t* last_row_off = nullptr;  // geometry of the latest trj_verify_step
 };
 
 namespace {
@@ -495,12 +518,28 @@ extern "C" trj_status trj_verify_step(trj_ctx* ctx, void* k_cache, void* v_cache
     Batch bt{seq_len, row_off, B, rows_total, max_rows, max_len};
     s = forward(ctx, k_cache, v_cache, 0, bt, tokens, depth, anc, anc_words, 0, rows_total, st);
     if (s != TRJ_OK) return s;
-    LAUNCH(PROF_ARGMAX, launch_argmax_accept(ctx->logits, TRJ_F32, ctx->cfg.vocab, tokens, parent, depth, row_off, B,
-                                             rows_total, node_argmax, margin, nullptr, nullptr, nullptr, true, false,
-                                             ctx->argmax_ws, st));
+    LAUNCH(PROF_ARGMAX, launch_topk_accept(ctx->logits, TRJ_F32, ctx->cfg.vocab, 1, tokens, parent, depth, row_off, B,
+                                           rows_total, nullptr, node_argmax, margin, nullptr, nullptr, nullptr, false,
+                                           ctx->argmax_ws, st));
+    ctx->last_rows = rows_total; ctx->last_row_off = row_off; ctx->last_B = B;
     if (logits)
         TRJ_CHECK_CUDA(cudaMemcpyAsync(logits, ctx->logits, sizeof(float) * (size_t)rows_total * ctx->cfg.vocab,
                                        cudaMemcpyDeviceToDevice, st));
+    return TRJ_OK;
+}
+
+extern "C" trj_status trj_node_topk(trj_ctx* ctx, int32_t rows_total, int32_t K, int32_t* topk, void* stream) {
+    TRJ_REQUIRE(ctx && topk, TRJ_EINVAL, "node_topk: null pointer");
+    TRJ_REQUIRE(K >= 1 && K <= TRJ_MAX_TOPK && K <= ctx->cfg.vocab, TRJ_EINVAL, "node_topk: K = %d outside 1..%d", K, TRJ_MAX_TOPK);
+    TRJ_REQUIRE(ctx->last_rows > 0 && rows_total == ctx->last_rows, TRJ_EINVAL,
+                "node_topk: %d rows asked, the latest verify_step scored %d", rows_total, ctx->last_rows);
+    cudaStream_t st = (cudaStream_t)stream;
+    ChainScope chain;
+    // predictions and margins are recomputed into scratch of the context (the caller already has them)
+    int32_t* scratch_pred = (int32_t*)ctx->y;
+    LAUNCH(PROF_ARGMAX, launch_topk_accept(ctx->logits, TRJ_F32, ctx->cfg.vocab, K, nullptr, nullptr, nullptr, ctx->last_row_off,
+                                           ctx->last_B, rows_total, topk, scratch_pred, nullptr, nullptr, nullptr, nullptr, false,
+                                           ctx->argmax_ws, st));
     return TRJ_OK;
 }
 
@@ -550,9 +589,9 @@ extern "C" trj_status trj_prefill(trj_ctx* ctx, void* k_cache, void* v_cache, in
                                m - 1, last ? 1 : 0, st);
         if (s != TRJ_OK) return s;
         if (last)   // greedy prediction after the last prompt token: a one-row arg-max
-            TRJ_CHECK_CUDA(launch_argmax_accept(ctx->logits + (size_t)(m - 1) * c.vocab, TRJ_F32, c.vocab, nullptr, nullptr,
-                                                nullptr, ctx->unit_row_off, 1, 1, first_token, nullptr, nullptr,
-                                                nullptr, nullptr, true, false, ctx->argmax_ws, st));
+            TRJ_CHECK_CUDA(launch_topk_accept(ctx->logits + (size_t)(m - 1) * c.vocab, TRJ_F32, c.vocab, 1, nullptr, nullptr,
+                                              nullptr, ctx->unit_row_off, 1, 1, nullptr, first_token, nullptr, nullptr,
+                                              nullptr, nullptr, false, ctx->argmax_ws, st));
         TRJ_CHECK_CUDA(launch_bump_len(seq_len + b, m, st));
     }
     return TRJ_OK;
@@ -573,8 +612,8 @@ trj_status enqueue_step(trj_ctx* ctx, void* k_cache, void* v_cache, int32_t* seq
     Batch bt{seq_len, d_off, 1, M, M, max_len};
     trj_status s = forward(ctx, k_cache, v_cache, 0, bt, d_tokens, d_depth, d_anc, 2, 0, M, st);
     if (s != TRJ_OK) return s;
-    LAUNCH(PROF_ARGMAX, launch_argmax_accept(ctx->logits, TRJ_F32, c.vocab, d_tokens, d_parent, d_depth, d_off, 1, M, d_pred,
-                                             nullptr, d_k, d_path, d_bonus, true, true, ctx->argmax_ws, st));
+    LAUNCH(PROF_ARGMAX, launch_topk_accept(ctx->logits, TRJ_F32, c.vocab, 1, d_tokens, d_parent, d_depth, d_off, 1, M, nullptr, d_pred,
+                                           nullptr, d_k, d_path, d_bonus, true, ctx->argmax_ws, st));
     LAUNCH(PROF_COMPACT, launch_compact(k_cache, v_cache, c.n_layers, c.max_batch, 1, kv_heads(c), c.max_seq, c.head_dim,
                                         c.dtype, seq_len, d_k, d_path, st));
     TRJ_CHECK_CUDA(cudaMemcpyAsync(ctx->pin_out, ctx->step_out, sizeof(int32_t) * STEP_OUT_INTS, cudaMemcpyDeviceToHost, st));
@@ -743,8 +782,8 @@ extern "C" trj_status trj_decode_device(trj_ctx* ctx, void* k_cache, void* v_cac
                                                             ctx->draft_src));
         trj_status fs = forward(ctx, k_cache, v_cache, 0, bt, d_tokens, d_depth, d_anc, 2, 0, M, on);
         if (fs != TRJ_OK) return fs;
-        LAUNCH_ON(on, PROF_ARGMAX, launch_argmax_accept(ctx->logits, TRJ_F32, c.vocab, d_tokens, d_parent, d_depth, d_off, 1, M, d_pred,
-                                                        nullptr, d_k, d_path, d_bonus, true, true, ctx->argmax_ws, on));
+        LAUNCH_ON(on, PROF_ARGMAX, launch_topk_accept(ctx->logits, TRJ_F32, c.vocab, 1, d_tokens, d_parent, d_depth, d_off, 1, M, nullptr,
+                                                      d_pred, nullptr, d_k, d_path, d_bonus, true, ctx->argmax_ws, on));
         LAUNCH_ON(on, PROF_COMPACT, launch_compact(k_cache, v_cache, c.n_layers, c.max_batch, 1, kv_heads(c), c.max_seq, c.head_dim,
                                                    c.dtype, seq_len, d_k, d_path, on));
         LAUNCH_ON(on, PROF_ELEMENTWISE, launch_commit_refill(d_tokens, d_parent, d_pred, M, d_k, d_path, d_bonus, context, capacity,

@@ -125,3 +125,44 @@ extern "C" trj_status trj_refill_window(const int32_t* parent, const int32_t* no
     }
     return TRJ_OK;
 }
+
+extern "C" trj_status trj_refill_tree(const int32_t* parent, const int32_t* rank, int32_t M, const int32_t* topk, int32_t K,
+                                      int32_t best, const int32_t* context, int32_t n, const int64_t* draws,
+                                      const int32_t* retrieved, int32_t n_retrieved, int32_t* tokens) {
+    TRJ_REQUIRE(parent && rank && topk && M >= 1, TRJ_EINVAL, "refill_tree: null tree");
+    TRJ_REQUIRE(M <= TRJ_MAX_ROWS, TRJ_ECAPACITY, "refill_tree: %d rows exceed the limit of %d", M, TRJ_MAX_ROWS);
+    TRJ_REQUIRE(K >= 1 && K <= TRJ_MAX_TOPK, TRJ_EINVAL, "refill_tree: K = %d outside 1..%d", K, TRJ_MAX_TOPK);
+    TRJ_REQUIRE(best >= 0 && best < M, TRJ_EINVAL, "refill_tree: winner %d outside the tree", best);
+    TRJ_REQUIRE(M == 1 || (tokens && draws && context && n >= 1), TRJ_EINVAL, "refill_tree: null pointer");
+    TRJ_REQUIRE(n_retrieved >= 0 && (n_retrieved == 0 || retrieved), TRJ_EINVAL, "refill_tree: null retrieved tokens");
+    // depth of every row, and the rows below the winner along its own path (lowest-index child at every level)
+    int32_t depth[TRJ_MAX_ROWS], below[TRJ_MAX_ROWS];
+    depth[0] = 0;
+    for (int32_t i = 1; i < M; ++i) {
+        TRJ_REQUIRE(parent[i] >= 0 && parent[i] < i, TRJ_EINVAL, "refill_tree: parent[%d] = %d is not an earlier row", i, parent[i]);
+        depth[i] = depth[parent[i]] + 1;
+    }
+    int32_t n_below = 0;
+    for (int32_t cur = best;;) {
+        int32_t child = -1;
+        for (int32_t c = cur + 1; c < M; ++c)
+            if (parent[c] == cur) { child = c; break; }
+        if (child < 0) break;
+        below[n_below++] = child;
+        cur = child;
+    }
+    for (int32_t i = 1; i < M; ++i) {
+        const int32_t r = rank[i];
+        if (r < 0) {
+            TRJ_REQUIRE(-1 - r < n_retrieved, TRJ_EINVAL, "refill_tree: row %d wants retrieval slot %d of %d", i, -1 - r, n_retrieved);
+            tokens[i - 1] = retrieved[-1 - r];
+        } else if (depth[i] <= n_below) {
+            TRJ_REQUIRE(r < K, TRJ_EINVAL, "refill_tree: row %d has rank %d but K = %d", i, r, K);
+            tokens[i - 1] = topk[(size_t)below[depth[i] - 1] * K + r];
+        } else {
+            TRJ_REQUIRE(draws[i - 1] >= 0, TRJ_EINVAL, "refill_tree: negative random draw");
+            tokens[i - 1] = context[draws[i - 1] % n];
+        }
+    }
+    return TRJ_OK;
+}

@@ -485,7 +485,8 @@ __device__ void accept_sequence(const int32_t* tokens, const int32_t* parent, co
     __shared__ int s_best;
     // all threads fetch the tree, then one thread walks it out of shared memory
     for (int i = threadIdx.x; i < rows; i += blockDim.x) {
-        s_tok[i] = tokens[i]; s_par[i] = parent[i]; s_dep[i] = depth[i]; s_pred[i] = pred[i];
+        s_tok[i] = tokens[i]; s_par[i] = parent[i]; s_dep[i] = depth[i];
+        s_pred[i] = __ldcg(pred + i);            // possibly written by other CTAs of this launch: read it from L2
     }
     __syncthreads();
     if (threadIdx.x == 0) {
@@ -565,6 +566,112 @@ __global__ void __launch_bounds__(ARGMAX_THREADS) argmax_accept_kernel(
     if (do_accept)
         accept_sequence(tokens + r0, parent + r0, depth + r0, node_argmax + r0, rows,
                         k_acc + b, path + (size_t)b * TRJ_PATH_STRIDE, bonus + b);
+}
+
+// ---------------------------------------------------------------- per-row top-K (K = 1: arg-max) + acceptance
+// One CTA per row.  Every thread keeps the KMAX best of its share of the row as a sorted list in registers (order:
+// larger value first, equal values by ascending id); each warp then merges its 32 lists into one by KMAX rounds of a
+// warp-wide arg-max over the lists' heads, and the first warp merges the 32 warp lists the same way.  The CTA that
+// finishes the last row of a sequence walks that sequence's tree.
+constexpr int TOPK_THREADS = 1024;
+template <int KMAX>
+struct TopList {
+    float v[KMAX]; int id[KMAX];
+    __device__ __forceinline__ void clear() {
+#pragma unroll
+        for (int i = 0; i < KMAX; ++i) { v[i] = -INFINITY; id[i] = 0x7fffffff; }
+    }
+    __device__ __forceinline__ void push(float x, int i) {
+        if (!(x > v[KMAX - 1] || (x == v[KMAX - 1] && i < id[KMAX - 1]))) return;
+#pragma unroll
+        for (int s = KMAX - 1; s >= 1; --s) {
+            const bool above = x > v[s - 1] || (x == v[s - 1] && i < id[s - 1]);    // the new entry goes above slot s - 1
+            if (above) { v[s] = v[s - 1]; id[s] = id[s - 1]; }
+            else { v[s] = x; id[s] = i; return; }
+        }
+        v[0] = x; id[0] = i;
+    }
+    __device__ __forceinline__ void pop() {
+#pragma unroll
+        for (int s = 0; s + 1 < KMAX; ++s) { v[s] = v[s + 1]; id[s] = id[s + 1]; }
+        v[KMAX - 1] = -INFINITY; id[KMAX - 1] = 0x7fffffff;
+    }
+};
+// KMAX rounds: the best head of the warp's 32 lists is taken out (ids are unique, so exactly one lane pops) and
+// handed to lane `round`; afterwards lane r < KMAX holds the warp's r-th best entry.
+template <int KMAX>
+__device__ __forceinline__ void warp_merge(TopList<KMAX>& t, float& out_v, int& out_id) {
+    const int lane = threadIdx.x & 31;
+    out_v = -INFINITY; out_id = 0x7fffffff;
+#pragma unroll 1
+    for (int r = 0; r < KMAX; ++r) {
+        float bv = t.v[0]; int bi = t.id[0];
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+            const float ov = __shfl_xor_sync(0xffffffffu, bv, o);
+            const int oi = __shfl_xor_sync(0xffffffffu, bi, o);
+            if (ov > bv || (ov == bv && oi < bi)) { bv = ov; bi = oi; }
+        }
+        if (bi != 0x7fffffff && t.id[0] == bi) t.pop();
+        if (lane == r) { out_v = bv; out_id = bi; }
+    }
+}
+
+template <typename T, int KMAX>
+__global__ void __launch_bounds__(TOPK_THREADS) topk_accept_kernel(
+        const T* __restrict__ logits, int V, int K, const int32_t* __restrict__ tokens,
+        const int32_t* __restrict__ parent, const int32_t* __restrict__ depth,
+        const int32_t* __restrict__ row_off, int B, int32_t* __restrict__ topk, int32_t* node_argmax,
+        float* __restrict__ margin, int32_t* __restrict__ k_acc, int32_t* __restrict__ path,
+        int32_t* __restrict__ bonus, int do_accept, unsigned int* tickets) {
+    pdl_prologue();
+    __shared__ float warp_v[TOPK_THREADS / 32][KMAX];
+    __shared__ int warp_id[TOPK_THREADS / 32][KMAX];
+    __shared__ int last_flag;
+    const int row = blockIdx.x, warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const T* lr = logits + (size_t)row * V;
+    TopList<KMAX> t;
+    t.clear();
+    constexpr int VEC = 16 / (int)sizeof(T);                 // elements per 16-byte load
+    if (V % VEC == 0 && ((uintptr_t)logits % 16) == 0) {
+        for (int v = threadIdx.x * VEC; v < V; v += TOPK_THREADS * VEC) {
+            const uint4 raw = *reinterpret_cast<const uint4*>(lr + v);
+            const T* e = reinterpret_cast<const T*>(&raw);
+#pragma unroll
+            for (int i = 0; i < VEC; ++i) t.push(to_f(e[i]), v + i);
+        }
+    } else {
+        for (int v = threadIdx.x; v < V; v += TOPK_THREADS) t.push(to_f(lr[v]), v);
+    }
+    float cv; int ci;
+    warp_merge<KMAX>(t, cv, ci);
+    if (lane < KMAX) { warp_v[warp][lane] = cv; warp_id[warp][lane] = ci; }
+    __syncthreads();
+    if (warp == 0) {
+        // lane w's list = warp w's merged list (already sorted)
+#pragma unroll
+        for (int i = 0; i < KMAX; ++i) { t.v[i] = warp_v[lane][i]; t.id[i] = warp_id[lane][i]; }
+        warp_merge<KMAX>(t, cv, ci);
+        if (lane < K && topk) topk[(size_t)row * K + lane] = ci;
+        const float second = __shfl_sync(0xffffffffu, cv, 1);
+        if (lane == 0) {
+            node_argmax[row] = ci;
+            if (margin) margin[row] = cv - second;
+            __threadfence();
+            const int b = seq_of_row(row_off, B, row);
+            const unsigned int need = (unsigned int)(row_off[b + 1] - row_off[b]);
+            const unsigned int got = atomicAdd(&tickets[b], 1u);
+            last_flag = (got + 1 == need) ? b : -1;
+            if (got + 1 == need) tickets[b] = 0;             // ready for the next call
+        }
+    }
+    __syncthreads();
+    const int b = last_flag;
+    if (b < 0 || !do_accept) return;
+    __threadfence();                                         // the other rows' predictions were written by other CTAs
+    const int r0 = row_off[b], rows = row_off[b + 1] - r0;
+    accept_sequence(tokens + r0, parent + r0, depth + r0, node_argmax + r0, rows,
+                    k_acc + b, path + (size_t)b * TRJ_PATH_STRIDE, bonus + b);
 }
 
 __global__ void accept_only_kernel(const int32_t* __restrict__ tokens, const int32_t* __restrict__ parent,
@@ -743,6 +850,30 @@ cudaError_t launch_argmax_accept(const void* logits, int32_t dtype, int32_t V,
     } else if (do_accept) {
         launch_err = launch_chain(accept_only_kernel, dim3(B), dim3(32), 0, st, tokens, parent, depth, row_off,
                                   (const int32_t*)node_argmax, k_acc, path, bonus);
+    }
+    return launch_err != cudaSuccess ? launch_err : cudaGetLastError();
+}
+
+size_t topk_workspace_bytes() { return align_up(sizeof(unsigned int) * TRJ_MAX_BATCH, 256); }
+
+cudaError_t launch_topk_accept(const void* logits, int32_t dtype, int32_t V, int32_t K,
+                               const int32_t* tokens, const int32_t* parent, const int32_t* depth,
+                               const int32_t* row_off, int32_t B, int32_t rows_total, int32_t* topk,
+                               int32_t* node_argmax, float* margin, int32_t* k_acc, int32_t* path,
+                               int32_t* bonus, bool do_accept, void* ws, cudaStream_t st) {
+    if (K < 1 || K > TRJ_MAX_TOPK) return cudaErrorInvalidValue;
+    count_launch();
+    cudaError_t launch_err = cudaSuccess;
+    unsigned int* tickets = (unsigned int*)ws;
+    // the margin needs the runner-up, so the shortest list holds two entries
+    if (K <= 2) {
+        DISPATCH_T(dtype, launch_err = launch_chain(topk_accept_kernel<T, 2>, dim3(rows_total), dim3(TOPK_THREADS), 0, st,
+                                                    (const T*)logits, V, K, tokens, parent, depth, row_off, B, topk, node_argmax,
+                                                    margin, k_acc, path, bonus, do_accept ? 1 : 0, tickets));
+    } else {
+        DISPATCH_T(dtype, launch_err = launch_chain(topk_accept_kernel<T, TRJ_MAX_TOPK>, dim3(rows_total), dim3(TOPK_THREADS), 0, st,
+                                                    (const T*)logits, V, K, tokens, parent, depth, row_off, B, topk, node_argmax,
+                                                    margin, k_acc, path, bonus, do_accept ? 1 : 0, tickets));
     }
     return launch_err != cudaSuccess ? launch_err : cudaGetLastError();
 }

@@ -174,6 +174,16 @@ cudaError_t launch_argmax_accept(const void* logits, int32_t dtype, int32_t V,
                                  int32_t* node_argmax, float* margin, int32_t* k_acc, int32_t* path,
                                  int32_t* bonus, bool do_argmax, bool do_accept, void* ws, cudaStream_t st);
 
+// Per-row top-K (K = 1: arg-max; ids best first into topk [rows][K] when not null; node_argmax and margin as above)
+// and, with do_accept, the acceptance walk.  One CTA per row; ws: one ticket per sequence (topk_workspace_bytes, zero
+// before the first call, left zero by every call).
+size_t topk_workspace_bytes();
+cudaError_t launch_topk_accept(const void* logits, int32_t dtype, int32_t V, int32_t K,
+                               const int32_t* tokens, const int32_t* parent, const int32_t* depth,
+                               const int32_t* row_off, int32_t B, int32_t rows_total, int32_t* topk,
+                               int32_t* node_argmax, float* margin, int32_t* k_acc, int32_t* path,
+                               int32_t* bonus, bool do_accept, void* ws, cudaStream_t st);
+
 // Same kernel with its scratch in a file-scope device array of the library (no workspace argument).
 cudaError_t launch_argmax_accept_static(const void* logits, int32_t dtype, int32_t V,
                                         const int32_t* tokens, const int32_t* parent, const int32_t* depth,

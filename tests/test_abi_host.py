@@ -129,3 +129,26 @@ def test_device_entry_points_reject_bad_arguments_before_any_launch(trj):
     out = ctypes.c_void_p()
     assert lib.trj_create(ctypes.byref(cfg), None, fake, 1 << 30, ctypes.byref(out)) == 1
     assert lib.trj_destroy(None) == 0
+
+
+def test_refill_tree_matches_oracle(trj):
+    """trj_refill_tree against the oracle on seeded templates, every possible winner, random top-K tables."""
+    for seed, (n_nodes, n_retr, k) in enumerate([(63, 5, 10), (20, 0, 5), (12, 3, 6), (0, 2, 1)]):
+        parent, rank = synth.tree_template(seed, n_nodes, 4, 10, n_retr)
+        m = len(parent)
+        g = synth.stream(seed, "refill_tree")
+        topk = g.integers(0, 5000, size=(m, k)).astype(np.int32)
+        context = g.integers(0, 5000, size=37).astype(np.int32)
+        retrieved = g.integers(0, 5000, size=n_retr).astype(np.int32)
+        for best in range(m):
+            draws = g.integers(0, 2 ** 31 - 1, size=max(m - 1, 1))
+            want = oracle.refill_tree(parent, rank, topk, best, context, draws, retrieved)
+            got = trj.refill_tree(parent, rank, topk, best, context, draws, retrieved)
+            assert got.tolist() == want
+    # chain + ranks 0 = the Jacobi window refill
+    chain = synth.chain_parents(7)
+    pred = np.arange(7, dtype=np.int32) + 50
+    got = trj.refill_tree(chain, np.zeros(7, np.int32), pred[:, None], 2, [1, 2, 3], np.zeros(6, np.int64))
+    assert got.tolist()[:4] == trj.refill_window(chain, pred, 2, 4, [1, 2, 3], np.zeros(4, np.int64)).tolist()
+    with pytest.raises(trj.TrjError):
+        trj.refill_tree([-1, 0], [0, 3], np.zeros((2, 2), np.int32), 0, [1], [0])       # rank 3 with K = 2

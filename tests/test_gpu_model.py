@@ -170,6 +170,42 @@ def test_llama3_8b_shape_two_layers_bf16(trj):
     model.close()
 
 
+def test_top_k_tree_template_decoding(trj):
+    """A static 69-row template with top-K siblings and a retrieval path (Appendix B; seeded stand-in for the paper's
+    63-node template + retrieval path of 5) on the tiny fp32 decoder: every step's top-K table, predictions and
+    accepted path equal the oracle's, and the loop commits the greedy autoregressive tokens (Eq. 1)."""
+    from paper_2406_17404_b200.decode import tr_jacobi_generate_tree
+    cfg = synth.TINY
+    model, dec = make_models(trj, cfg, 0, max_seq=512, max_rows=128)
+    prompt = synth.prompt(0, 64, cfg.vocab)
+    parent, rank = synth.tree_template(0)
+    assert len(parent) == 69
+    draw = lambda s, n: synth.noise_draws(4, s, n)
+    n_new = 40
+    trace, gtrace = [], []
+    want = oracle.tr_jacobi_generate_tree(dec, prompt, n_new, parent, rank, 10, 5, draw, trace=trace)
+    assert want == oracle.autoregressive_greedy(dec, prompt, n_new)
+    got = tr_jacobi_generate_tree(model, prompt, n_new, parent, rank, 10, 5, draw, trace=gtrace)
+    # the oracle's logits say where an id may legitimately differ: ranks whose logits lie within 1e-3 of a neighbour
+    diverged = False
+    for rec, grec in zip(trace, gtrace):
+        np.testing.assert_array_equal(rec["tokens"], grec["tokens"])
+        srt = -np.sort(-rec["logits"], axis=1)[:, :11]
+        gap = srt[:, :10] - srt[:, 1:11]                   # logit of rank r minus logit of rank r + 1
+        clear = gap >= 1e-3
+        clear[:, 1:] &= gap[:, :-1] >= 1e-3                # ... and rank r - 1 is clear of rank r
+        same = rec["topk"] == grec["topk"]
+        assert same[clear].all()
+        if not same.all() or (rec["k"], list(rec["path"])) != (grec["k_acc"], grec["path"].tolist()):
+            diverged = True                                # a near-tie fell the other way: later trees may differ
+            break
+    assert len(gtrace) >= 5
+    if not diverged:
+        assert got == want
+        assert max(r["k"] for r in trace) >= 1
+    model.close()
+
+
 def test_programmatic_launch_does_not_change_results(trj):
     """The chain's kernels start on chain-invariant data before their predecessor has finished (tensor maps, weights,
     batch geometry, cached K/V rows).  If any of that were data the predecessor still writes, the result would

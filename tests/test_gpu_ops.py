@@ -180,6 +180,29 @@ def test_argmax_accept_edges(trj, rows_list, vocab):
     check_argmax_accept(trj, 8, rows_list, vocab, "f32")
 
 
+@pytest.mark.parametrize("rows_list,vocab,k,dtype", [
+    ([69], 32000, 10, "f32"), ([64], 32000, 10, "bf16"), ([33], 128256, 4, "f32"), ([1], 11, 10, "f32"),
+    ([5, 128, 2], 4099, 3, "bf16"), ([16] * 8, 1001, 2, "f32"), ([7], 513, 1, "bf16"),
+])
+def test_topk_accept_against_oracle(trj, rows_list, vocab, k, dtype):
+    """Per-row top-K (Appendix B) bit-exact against the oracle, exact ties included (bf16 logits tie often), and the
+    acceptance results next to it."""
+    parents, logits, pred, off, tokens = accept_case(11, rows_list, vocab, dtype)
+    depth = np.concatenate([oracle.depths(p) for p in parents])
+    ws = torch.zeros(trj.lib().trj_topk_accept_workspace(), dtype=torch.uint8, device="cuda")
+    for _ in range(2):                                     # the workspace is left ready for the next call
+        res = trj.topk_accept(to_dev(logits, dtype), i32(tokens), i32(np.concatenate(parents)), i32(depth), i32(off), k, workspace=ws)
+        torch.cuda.synchronize()
+        np.testing.assert_array_equal(res["topk"].cpu().numpy(), oracle.node_topk(logits, k))
+        np.testing.assert_array_equal(res["node_argmax"].cpu().numpy(), pred)
+        if vocab > 1:
+            np.testing.assert_allclose(res["margin"].cpu().numpy(), oracle.top2_margin(logits), rtol=0, atol=1e-6)
+        for b, p in enumerate(parents):
+            kk, path, bonus = oracle.accept_path(tokens[off[b]:off[b + 1]], p, pred[off[b]:off[b + 1]])
+            assert int(res["k_acc"][b]) == kk and int(res["bonus"][b]) == bonus
+            assert res["path"][b, :kk + 1].tolist() == path and (res["path"][b, kk + 1:] == -1).all()
+
+
 def test_argmax_ties_go_to_the_smallest_id_and_workspace_is_reusable(trj):
     rows, vocab = 9, 4099
     logits = np.zeros((rows, vocab), np.float32)
