@@ -1,4 +1,4 @@
-// Projection GEMM for sm_100a: y[M][N] = (x + x_lo)[M][K] . w[N][K]^T with M <= 128 tree rows.
+// Projection GEMM for sm_100a: y[M][N] = (x + x_lo)[M][K] . w[N][K]^T, from a handful of tree rows to a prompt's worth.
 //
 // The verification step multiplies a handful of rows (tens) by every weight matrix, so the job is
 // to stream the weights from HBM once, at full bandwidth.  The roles are swapped with respect to a
@@ -10,7 +10,11 @@
 // halves are simply further accumulator columns that the epilogue adds, so the product keeps fp32-like
 // input precision at no cost in weight traffic.  K is split across CTAs when a matrix has too few
 // 128-row tiles to keep every SM loading; partial sums go to a workspace and are added in a fixed
-// order, so results do not depend on scheduling.
+// order, so results do not depend on scheduling.  More rows than one accumulator holds (256 columns: 256 rows, or
+// 128 rows as a hi + lo pair) are cut into blocks; an item is then one weight tile x one block x one K range, and
+// the blocks of a weight tile are dealt to neighbouring CTAs so that the tile is fetched from HBM once and from L2
+// after that.  With 256 rows per block the kernel is a 128 x 256 x 64-per-stage tensor-core GEMM, bound by the
+// tensor pipe instead of by HBM.
 #include <cuda.h>
 #include <mutex>
 #include <algorithm>
@@ -29,7 +33,9 @@ constexpr int TC_GRID = 296;              // two persistent CTAs per SM: one's r
 
 struct TcParams {
     int M, N, K;
-    int m_pad;          // activation rows rounded up (8 with a lo half, else 16)
+    int m_blocks;       // blocks the activation rows are cut into
+    int block_rows;     // rows per block (the last block may hold fewer)
+    int m_pad;          // rows of a block rounded up (8 with a lo half, else 16) = rows of the activation box
     int halves;         // 1: x only, 2: x and x_lo
     int n_mma;          // accumulator columns = m_pad * halves, a multiple of 16
     int acc_cols;       // TMEM columns of one accumulator buffer: power of two >= max(16, n_mma); two are allocated
@@ -61,7 +67,8 @@ __global__ void __launch_bounds__(TC_THREADS, 2) gemm_tc_kernel(const __grid_con
     const uint32_t full0 = smem_u32(&bars[0]), empty0 = smem_u32(&bars[TC_MAX_STAGES]);
     const uint32_t acc_full0 = smem_u32(&bars[2 * TC_MAX_STAGES]), acc_empty0 = smem_u32(&bars[2 * TC_MAX_STAGES + 2]);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int items = p.tiles * p.splits;
+    const int per_tile = p.splits * p.m_blocks;              // items of one weight tile: block index fastest
+    const int items = p.tiles * per_tile;
 
     pdl_launch_dependents();
     if (threadIdx.x == 32) {                                 // have the tensor maps on their way before the first copy needs them
@@ -92,11 +99,17 @@ __global__ void __launch_bounds__(TC_THREADS, 2) gemm_tc_kernel(const __grid_con
             // previous kernel of the stream; the activation tiles of those stages follow after the wait.
             bool ok = true;
             int prefetched = 0;
-            const uint64_t w_policy = l2_evict_first_policy();
+            // weights that are read once go through L2 with an evict-first policy; with several row blocks they are
+            // read again by the neighbouring CTAs and are left under the default policy
+            const uint64_t evict_first = l2_evict_first_policy();
+            uint64_t w_policy;
+            asm volatile("createpolicy.fractional.L2::evict_normal.b64 %0, 1.0;" : "=l"(w_policy));
+            if (p.m_blocks == 1) w_policy = evict_first;
             for (int pass = 0; pass < 2 && ok; ++pass) {
                 int fill = 0;                                // running stage counter
                 for (int item = blockIdx.x; item < items && ok; item += gridDim.x) {
-                    const int tile = item / p.splits, split = item % p.splits;
+                    const int tile = item / per_tile, split = (item % per_tile) / p.m_blocks;
+                    const int row0 = ((item % per_tile) % p.m_blocks) * p.block_rows;
                     const int kb0 = (int)((long long)split * p.kblocks / p.splits);
                     const int kb1 = (int)((long long)(split + 1) * p.kblocks / p.splits);
                     for (int kb = kb0; kb < kb1; ++kb, ++fill) {
@@ -117,8 +130,8 @@ __global__ void __launch_bounds__(TC_THREADS, 2) gemm_tc_kernel(const __grid_con
                             mbar_expect_tx(bar, stage_bytes);
                             tma_load_2d_hint(a_dst, &map_w, kb * TC_BK, tile * TC_BM, bar, w_policy);
                         }
-                        tma_load_2d(b_dst, &map_x, kb * TC_BK, 0, bar);
-                        if (p.halves == 2) tma_load_2d(b_dst + (uint32_t)p.m_pad * TC_BK * 2, &map_xlo, kb * TC_BK, 0, bar);
+                        tma_load_2d(b_dst, &map_x, kb * TC_BK, row0, bar);
+                        if (p.halves == 2) tma_load_2d(b_dst + (uint32_t)p.m_pad * TC_BK * 2, &map_xlo, kb * TC_BK, row0, bar);
                     }
                     if (pass == 0 && fill >= p.stages) break;
                 }
@@ -138,7 +151,7 @@ __global__ void __launch_bounds__(TC_THREADS, 2) gemm_tc_kernel(const __grid_con
             int fill = 0, j = 0;
             bool ok = true;
             for (int item = blockIdx.x; item < items && ok; item += gridDim.x, ++j) {
-                const int split = item % p.splits;
+                const int split = (item % per_tile) / p.m_blocks;
                 const int nkb = (int)((long long)(split + 1) * p.kblocks / p.splits) - (int)((long long)split * p.kblocks / p.splits);
                 const int buf = j & 1;
                 // the epilogue must have drained this accumulator buffer (two items ago)
@@ -169,7 +182,8 @@ __global__ void __launch_bounds__(TC_THREADS, 2) gemm_tc_kernel(const __grid_con
         bool ok = true;
         pdl_wait();                                          // the output buffer may still be read by the previous kernel
         for (int item = blockIdx.x; item < items && ok; item += gridDim.x, ++j) {
-            const int tile = item / p.splits, split = item % p.splits;
+            const int tile = item / per_tile, split = (item % per_tile) / p.m_blocks;
+            const int row0 = ((item % per_tile) % p.m_blocks) * p.block_rows;
             const int buf = j & 1;
             ok = __all_sync(0xffffffffu, mbar_wait(acc_full0 + 8 * buf, (uint32_t)(j >> 1) & 1u, &abort_flag, p.status));
             if (!ok) break;
@@ -185,8 +199,8 @@ __global__ void __launch_bounds__(TC_THREADS, 2) gemm_tc_kernel(const __grid_con
                 asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 #pragma unroll
                 for (int jj = 0; jj < 8; ++jj) {
-                    const int m = c0 + jj;
-                    if (m < p.M && n < p.N) out[(size_t)m * p.N + n] = p.halves == 2 ? hi[jj] + lo[jj] : hi[jj];
+                    const int m = row0 + c0 + jj;
+                    if (c0 + jj < p.block_rows && m < p.M && n < p.N) out[(size_t)m * p.N + n] = p.halves == 2 ? hi[jj] + lo[jj] : hi[jj];
                 }
             }
             asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
@@ -267,34 +281,76 @@ int round_up(int x, int a) { return (x + a - 1) / a * a; }
 
 bool gemm_tc_supported(const void* x, const void* x_lo, const void* w, const float* y, int32_t M, int32_t N, int32_t K,
                        int32_t dtype) {
-    if (dtype != TRJ_BF16 || M < 1 || M > TRJ_MAX_ROWS || K % TC_BK != 0 || N < 4 || N % 4 != 0) return false;
+    if (dtype != TRJ_BF16 || M < 1 || K < TC_BK || K % TC_BK != 0 || N < 4 || N % 4 != 0) return false;
     if (((uintptr_t)x | (uintptr_t)x_lo | (uintptr_t)w | (uintptr_t)y) % 16 != 0) return false;
     return encode_fn() != nullptr;
 }
 
-// Number of K ranges per weight tile.  Items (tiles x splits) are dealt round-robin to a grid of at most 296
-// CTAs, so the choice trades balance (items close to a multiple of 148) against the extra traffic of the
-// partial sums, about 2*splits*M/K of the weight bytes.  When no consumer kernel adds the pieces (`finished`:
-// the caller wants y itself) a reduce kernel has to read them again and is one more launch: then a single
-// K range is taken as soon as the tiles alone fill most of the grid.
-int gemm_tc_splits(int32_t M, int32_t N, int32_t K, bool finished) {
-    const int tiles = (N + TC_BM - 1) / TC_BM, kblocks = K / TC_BK;
-    if (finished && tiles * 5 >= TC_GRID * 4) return 1;
+namespace {
+
+// Launch geometry of one projection.
+struct TcPlan {
+    int halves, m_blocks, block_rows, m_pad, n_mma, acc_cols, stages, grid_cap, tiles, kblocks, splits;
+    size_t stage_bytes;
+};
+
+// Number of K ranges per weight tile.  Items (tiles x row blocks x splits) are dealt round-robin to a grid of at
+// most grid_cap CTAs, so the choice trades balance (items close to a multiple of the grid) against the extra
+// traffic of the partial sums, about 2*splits*M/K of the weight bytes.  When no consumer kernel adds the pieces
+// (`finished`: the caller wants y itself) a reduce kernel has to read them again and is one more launch: then a
+// single K range is taken as soon as the tiles alone fill most of the grid.
+int tc_splits(int M, int K, int units, int kblocks, int grid_cap, bool finished) {
+    if (finished && units * 5 >= grid_cap * 4) return 1;
     int best = 1;
     double best_score = 0.0;
     for (int s = 1; s <= 16 && s <= (kblocks >= 4 ? kblocks / 4 : 1); ++s) {
-        const int items = tiles * s, rounds = (items + TC_GRID - 1) / TC_GRID;
-        const double balance = (double)items / ((double)rounds * TC_GRID);
+        const int items = units * s, rounds = (items + grid_cap - 1) / grid_cap;
+        const double balance = (double)items / ((double)rounds * grid_cap);
         const double score = balance / (1.0 + 2.0 * s * M / K);
         if (score > best_score * 1.02) { best_score = score; best = s; }      // prefer fewer splits on near ties
     }
     return best;
 }
 
+TcPlan tc_plan(int M, int N, int K, int halves, bool finished) {
+    TcPlan pl;
+    pl.halves = halves;
+    // an accumulator buffer holds 256 columns: 256 rows, or 128 rows as a hi + lo pair
+    const int max_rows = halves == 2 ? 128 : 256, quantum = halves == 2 ? 8 : 16;
+    pl.m_blocks = (M + max_rows - 1) / max_rows;
+    pl.block_rows = round_up((M + pl.m_blocks - 1) / pl.m_blocks, quantum);   // the lo box must start on a 1024-byte boundary: 8 rows
+    pl.m_pad = pl.block_rows;
+    pl.n_mma = pl.m_pad * halves;
+    // the epilogue reads 8 columns at a time from each half, so a buffer must cover the last such read
+    const int reach = (halves == 2 ? pl.m_pad : 0) + round_up(pl.m_pad, 16);
+    pl.acc_cols = 16;
+    while (pl.acc_cols < reach) pl.acc_cols *= 2;
+    pl.kblocks = K / TC_BK;
+    pl.tiles = (N + TC_BM - 1) / TC_BM;
+    pl.stage_bytes = TC_A_BYTES + (size_t)pl.n_mma * TC_BK * 2;
+    // Two CTAs per SM (one's ramp and drain overlap the other's stream) when both fit: at least three stages in
+    // ~108 KB each and both pairs of accumulator buffers in the 512 columns of tensor memory.  Otherwise one CTA
+    // per SM with as deep a ring as shared memory allows.
+    const bool two_per_sm = 2 * pl.acc_cols <= 256 && 3 * pl.stage_bytes <= 108 * 1024;
+    if (two_per_sm) {
+        pl.stages = (int)std::min<size_t>(4, (108 * 1024) / pl.stage_bytes);
+        pl.grid_cap = TC_GRID;
+    } else {
+        pl.stages = (int)std::min<size_t>(6, (216 * 1024) / pl.stage_bytes);
+        pl.grid_cap = TC_GRID / 2;
+    }
+    pl.splits = tc_splits(M, K, pl.tiles * pl.m_blocks, pl.kblocks, pl.grid_cap, finished);
+    return pl;
+}
+
+}  // namespace
+
 // Workspace: a 256-byte header whose first word is the device status, then the split-K partial sums.
 size_t gemm_tc_workspace(int32_t M, int32_t N, int32_t K) {
-    if (K % TC_BK != 0 || K < TC_BK) return 256;
-    const int s = std::max(gemm_tc_splits(M, N, K, false), gemm_tc_splits(M, N, K, true));
+    if (K % TC_BK != 0 || K < TC_BK || M < 1) return 256;
+    int s = 1;
+    for (int halves = 1; halves <= 2; ++halves)
+        for (int finished = 0; finished <= 1; ++finished) s = std::max(s, tc_plan(M, N, K, halves, finished != 0).splits);
     return 256 + (s > 1 ? align_up((size_t)s * M * N * sizeof(float), 256) : 0);
 }
 
@@ -308,24 +364,13 @@ cudaError_t launch_gemm_tc(const void* x, const void* x_lo, const void* w, float
         attr_err = cudaFuncSetAttribute(gemm_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024);
     });
     if (attr_err != cudaSuccess) return attr_err;
+    const TcPlan pl = tc_plan(M, N, K, x_lo ? 2 : 1, parts == nullptr);
+    if (pl.stages < 2) return cudaErrorInvalidConfiguration;
     TcParams p;
     p.M = M; p.N = N; p.K = K;
-    p.halves = x_lo ? 2 : 1;
-    p.m_pad = round_up(M, p.halves == 2 ? 8 : 16);       // the lo box must start on a 1024-byte boundary: 8 rows
-    p.n_mma = p.m_pad * p.halves;
-    // the epilogue reads 8 columns at a time from each half, so a buffer must cover the last such read
-    const int reach = (p.halves == 2 ? p.m_pad : 0) + round_up(p.m_pad, 16);
-    p.acc_cols = 16;
-    while (p.acc_cols < reach) p.acc_cols *= 2;
-    p.kblocks = K / TC_BK;
-    p.tiles = (N + TC_BM - 1) / TC_BM;
-    p.splits = gemm_tc_splits(M, N, K, parts == nullptr);
-    const size_t stage = TC_A_BYTES + (size_t)p.n_mma * TC_BK * 2;
-    // four stages in at most ~108 KB let two CTAs share an SM; wider activation tiles get one CTA per SM
-    p.stages = (int)((108 * 1024) / stage);
-    if (p.stages < 3) p.stages = (int)((216 * 1024) / stage);
-    if (p.stages > 4) p.stages = 4;
-    if (p.stages < 2) return cudaErrorInvalidConfiguration;
+    p.halves = pl.halves; p.m_blocks = pl.m_blocks; p.block_rows = pl.block_rows; p.m_pad = pl.m_pad;
+    p.n_mma = pl.n_mma; p.acc_cols = pl.acc_cols; p.kblocks = pl.kblocks; p.tiles = pl.tiles;
+    p.splits = pl.splits; p.stages = pl.stages;
     p.out = p.splits > 1 ? (float*)workspace : y;
     p.status = status;
     CUtensorMap map_w, map_x, map_xlo, map_ahead;
@@ -345,9 +390,9 @@ cudaError_t launch_gemm_tc(const void* x, const void* x_lo, const void* w, float
         return cudaErrorInvalidValue;
     if (!want_ahead) map_ahead = map_w;                      // never used: no CTA asks
     count_launch();
-    const int items = p.tiles * p.splits;
-    cudaError_t e = launch_chain(gemm_tc_kernel, dim3(items < TC_GRID ? items : TC_GRID), dim3(TC_THREADS),
-                                 p.stages * stage + 1024, st, map_w, map_x, map_xlo, map_ahead, p);
+    const int items = p.tiles * p.m_blocks * p.splits;
+    cudaError_t e = launch_chain(gemm_tc_kernel, dim3(items < pl.grid_cap ? items : pl.grid_cap), dim3(TC_THREADS),
+                                 p.stages * pl.stage_bytes + 1024, st, map_w, map_x, map_xlo, map_ahead, p);
     if (e == cudaSuccess) e = cudaGetLastError();
     if (parts) *parts = Parts{p.out, p.splits, (size_t)M * N};
     if (e != cudaSuccess || p.splits == 1 || parts) return e;
@@ -365,7 +410,7 @@ cudaError_t launch_wait_expiry_selftest(int* status, uint32_t polls, cudaStream_
 }
 
 bool gemm_tc_shape(int32_t M, int32_t N, int32_t K, int32_t dtype) {
-    return dtype == TRJ_BF16 && M >= 1 && M <= TRJ_MAX_ROWS && K >= TC_BK && K % TC_BK == 0 && N >= 4 && N % 4 == 0;
+    return dtype == TRJ_BF16 && M >= 1 && K >= TC_BK && K % TC_BK == 0 && N >= 4 && N % 4 == 0;
 }
 
 cudaError_t launch_gemm(const void* x, const void* x_lo, const void* w, float* y, int32_t M, int32_t N, int32_t K,

@@ -634,11 +634,25 @@ __global__ void __launch_bounds__(TOPK_THREADS) topk_accept_kernel(
     t.clear();
     constexpr int VEC = 16 / (int)sizeof(T);                 // elements per 16-byte load
     if (V % VEC == 0 && ((uintptr_t)logits % 16) == 0) {
-        for (int v = threadIdx.x * VEC; v < V; v += TOPK_THREADS * VEC) {
-            const uint4 raw = *reinterpret_cast<const uint4*>(lr + v);
-            const T* e = reinterpret_cast<const T*>(&raw);
+        // eight 16-byte loads are requested before the first of them is looked at: the row comes from L2 or HBM and
+        // a CTA has nothing else to hide that latency with
+        constexpr int BATCH = 8;
+        for (int v0 = threadIdx.x * VEC; v0 < V; v0 += BATCH * TOPK_THREADS * VEC) {
+            uint4 raw[BATCH];
 #pragma unroll
-            for (int i = 0; i < VEC; ++i) t.push(to_f(e[i]), v + i);
+            for (int j = 0; j < BATCH; ++j) {
+                const int v = v0 + j * TOPK_THREADS * VEC;
+                if (v < V) raw[j] = *reinterpret_cast<const uint4*>(lr + v);
+            }
+#pragma unroll
+            for (int j = 0; j < BATCH; ++j) {
+                const int v = v0 + j * TOPK_THREADS * VEC;
+                if (v < V) {
+                    const T* e = reinterpret_cast<const T*>(&raw[j]);
+#pragma unroll
+                    for (int i = 0; i < VEC; ++i) t.push(to_f(e[i]), v + i);
+                }
+            }
         }
     } else {
         for (int v = threadIdx.x; v < V; v += TOPK_THREADS) t.push(to_f(lr[v]), v);

@@ -5,11 +5,12 @@ The CPU oracle cannot decode with the full model in test time, so this file chec
 any size, on the GPU alone, and (b) ONE full-depth forward against the oracle, whose weights are pulled from
 the device layer by layer.  Weights are drawn on the device (seeded torch Philox, N(0, 0.02), bf16), as in bench.py.
 
-Tolerance at full depth.  Both sides store q and K/V as bf16; after a few layers their pre-rounding values differ by
-~1e-4 relative, which flips a fraction of those roundings, and each flip is a bf16 ulp.  This is inherent to a bf16
-cache, not to a kernel, and makes the logit error a random walk in depth: measured rms 2.7e-3 at 2 layers, 5.6e-3 at
-8.  The stated 2e-2 bound (max |err| over ~1e6 logits) therefore applies to shallow stacks (tested at 2 layers); at
-L layers the bound used here is 2e-2 * sqrt(L / 2) for max |err|, and 2e-2 for the rms error.
+Tolerance at full depth.  Both sides store q and K/V as bf16.  Their values before that rounding agree to ~1e-5
+(fp32 arithmetic on bf16-pair activations against fp64), which is enough to make ~0.25 % of the roundings of the first
+layer fall the other way; each such flip is a whole bf16 step, the next layer sees it as an input error, flips more,
+and the logit error grows with depth (measured curve below).  This is a property of a bf16 cache compared against an
+fp64 computation, not of a kernel.  The stated 2e-2 bound on max |err| holds up to 8 layers; the full 32-layer
+stack reaches 3.2e-2 (rms 6e-3), and the bounds asserted here are the measured levels with 1.5x headroom.
 """
 import numpy as np
 import pytest
@@ -21,7 +22,7 @@ from gpu_util import anc_dev, i32
 
 pytestmark = pytest.mark.gpu
 WIDTH, N_BRANCHES, BRANCH_LEN = 5, 9, 3
-CONFIG3_TOL = 8e-2          # provisional: replaced by the measured level
+CONFIG3_TOL = 3.5e-2        # measured 2.33e-2 (worst of three steps over a 512-row prefix) x 1.5
 
 
 @pytest.fixture(scope="module")
@@ -49,8 +50,10 @@ def mixed_tree(cfg):
 # Measured on a B200 (this file's weights and tree): the logit error against the fp64 oracle as the stack deepens.
 # The bounds asserted below are these measurements with 1.5x headroom.
 #   layers        2        4        8        16       32
-DEPTH_MAX = {2: None, 4: None, 8: None, 16: None, 32: None}
-DEPTH_RMS = {2: None, 4: None, 8: None, 16: None, 32: None}
+DEPTH_MAX = {2: 5.8e-3, 4: 1.10e-2, 8: 1.52e-2, 16: 2.18e-2, 32: 3.23e-2}
+DEPTH_RMS = {2: 9.1e-4, 4: 1.69e-3, 8: 2.75e-3, 16: 4.22e-3, 32: 6.23e-3}
+# fraction of the last layer's K elements whose bf16 rounding fell the other way than the oracle's, same run:
+#                 0.12     0.32     0.46     0.58     0.68
 
 
 @pytest.mark.parametrize("n_layers", [2, 4, 8, 16, 32])
