@@ -461,7 +461,28 @@ def bench_template_step(trj, torch, synth, model, cfg, prefix, side, steps):
             "what": "7B shape, prefix %d, 63-node template + retrieval path of 5 + root; random drafts" % prefix}
 
 
-def planted_lengths(seed, n):
+def bench_prefill_gemm(trj, torch, peaks, steps):
+    """The four projections of the 7B shape on prompt-sized row counts (the tensor-bound side of the projection
+    kernel: 128 x 256 tiles), as a stand-alone op: TFLOP/s against the measured dense bf16 peak."""
+    out = []
+    g = torch.Generator(device="cuda"); g.manual_seed(5)
+    shapes = (("qkv", 12288, 4096), ("o", 4096, 4096), ("gate_up", 22016, 4096), ("down", 4096, 11008))
+    for m in (512, 2048):
+        for name, n, k in shapes:
+            x = torch.randn(m, k, generator=g, device="cuda").to(torch.bfloat16)
+            w = (torch.randn(n, k, generator=g, device="cuda") * 0.02).to(torch.bfloat16)
+            y = torch.empty(m, n, dtype=torch.float32, device="cuda")
+            ws = torch.zeros(trj.lib().trj_gemm_workspace(m, n, k), dtype=torch.uint8, device="cuda")
+            us = graph_us(torch, lambda: [trj.gemm(x, w, out=y, workspace=ws) for _ in range(4)], steps, 3) / 4
+            tf = 2.0 * m * n * k / us / 1e6
+            out.append({"shape": "%s: M=%d N=%d K=%d" % (name, m, n, k), "us": round(us, 2), "tflops": round(tf, 1),
+                        "frac_of_" + peaks["source"] + "_burst_peak": round(tf / peaks["bf16_tflops"], 4)})
+            assert int(ws[:4].view(torch.int32)[0]) == 0
+            del x, w, y, ws
+    return out
+
+
+def planted_lengths(seed, n):def planted_lengths(seed, n):
     """How many tokens of the true continuation each step's first retrieved branch carries: uniform on 0..3, so
     that a step commits 1 + (0..3) tokens, 2.5 on average (the paper's Table 2 reports 2.0-2.9 per step)."""
     import synth
@@ -714,6 +735,18 @@ def run_ours(args, rank, world, local_rank):
             "roofline": roofline, "kernel_breakdown": breakdown, "profiled_step_ms": step_ms_prof}
     if world == 1:
         line["paper_sized_tree"] = bench_template_step(trj, torch, synth, model, cfg, PROMPT, side, args.steps)
+        # prefill of the 512-token prompt: the weights are streamed once (projections over all 512 rows at a time)
+        model.seq_len.zero_()
+        model.prefill(i32(prompt)); torch.cuda.synchronize()
+        pe0, pe1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        model.seq_len.zero_()
+        pe0.record(); model.prefill(i32(prompt)); pe1.record(); torch.cuda.synchronize()
+        pf_ms = pe0.elapsed_time(pe1)
+        pf_flops = 2.0 * PROMPT * (gemm_bytes_per_step(cfg, 0) / 2)        # 2 x rows x weight parameters
+        line["prefill"] = {"prompt": PROMPT, "ms": pf_ms, "tflops": pf_flops / pf_ms / 1e9,
+                           "note": "projections take bf16-pair activations: two tensor-core products per weight tile"}
+        if not args.no_attention:
+            line["prefill_gemm"] = bench_prefill_gemm(trj, torch, peaks, max(args.steps // 2, 5))
         if not args.no_attention:
             line["tree_attention"] = bench_tree_attention(trj, torch, peaks, max(args.steps, 5), 3, cpu=not args.no_cpu)
             line["small_ops"] = bench_small_ops(trj, torch, peaks, max(args.steps, 5), 3, cpu=not args.no_cpu)

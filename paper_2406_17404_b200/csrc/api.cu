@@ -179,7 +179,7 @@ struct trj_ctx {
     int sm_count;          // SMs of the device the context lives on
     void* argmax_ws; void* attn_ws; size_t attn_ws_bytes; void* gemm_ws; size_t gemm_ws_bytes;
     // chain-tree tables for prefill and the staging area of trj_step_host (device)
-    int32_t* chain_depth; uint64_t* chain_anc; int32_t* chunk_row_off; int32_t* unit_row_off;
+    int32_t* chain_depth; uint64_t* chain_anc; int32_t* chunk_row_off; int32_t* unit_row_off; int32_t* prefill_geo;
     int32_t* loop_state;   // device: [0] step counter, [1] context-overflow flag of trj_decode_device
     int32_t* step_in;      // tokens | parent | depth | row_off(2) | pad -> anc
     int32_t* step_out;     // node_argmax | k_acc | bonus | path | device status words (projections, attention)
@@ -200,6 +200,12 @@ struct trj_ctx {
 
 namespace {
 
+// Prefill scores a prompt in chunks of this many rows (the projections see them all at once, so the weights are
+// streamed once per chunk); attention runs inside a chunk in pieces of at most TRJ_MAX_ROWS rows, at most 16 of them.
+constexpr int PREFILL_CHUNK = 512;
+constexpr int PREFILL_MAX_SUB = 16;
+struct SubChunks { int n, sub, last_rows; const int32_t* lens; const int32_t* off_full; const int32_t* off_last; };
+
 constexpr int STEP_IN_INTS = 3 * TRJ_MAX_ROWS + 4;                       // + anc (2 words per row) after it
 constexpr int STEP_IN_BYTES = STEP_IN_INTS * 4 + TRJ_MAX_ROWS * 2 * 8;
 constexpr int STEP_STATUS_AT = TRJ_MAX_ROWS + 2 + TRJ_PATH_STRIDE;
@@ -209,31 +215,33 @@ int kv_heads(const trj_model_cfg& c) { return c.n_kv_heads > 0 ? c.n_kv_heads : 
 
 size_t carve(const trj_model_cfg& c, void* ws, trj_ctx* ctx) {
     const size_t es = dtype_size(c.dtype);
-    const int rows = c.max_batch * c.max_rows;
+    const int step_rows = c.max_batch * c.max_rows;          // rows of a verification step
+    const int rows = std::max(step_rows, PREFILL_CHUNK);     // ... or of a prefill chunk
     const int HD = c.n_heads * c.head_dim;
     const int QKV = HD + 2 * kv_heads(c) * c.head_dim;
     const size_t wide = (size_t)std::max(std::max(QKV, 2 * c.d_ff), c.d_model);
     Carver cv(ws);
     float* h = cv.take<float>((size_t)rows * c.d_model);
     float* y = cv.take<float>((size_t)rows * wide);
-    float* logits = cv.take<float>((size_t)rows * c.vocab);
+    float* logits = cv.take<float>((size_t)step_rows * c.vocab);
     char* x = cv.take<char>((size_t)rows * std::max(c.d_model, HD) * es);
     char* x_lo = cv.take<char>((size_t)rows * std::max(c.d_model, HD) * es);
     char* q = cv.take<char>((size_t)rows * HD * es);
     char* act = cv.take<char>((size_t)rows * c.d_ff * es);
     char* act_lo = cv.take<char>((size_t)rows * c.d_ff * es);
     double* inv_freq = cv.take<double>(c.head_dim / 2);
-    char* argmax_ws = cv.take<char>(argmax_workspace_bytes(rows, c.max_batch));
-    const size_t attn_bytes = trj_tree_attention_workspace(rows, c.max_batch, c.n_heads, c.head_dim, c.max_seq);
+    char* argmax_ws = cv.take<char>(argmax_workspace_bytes(step_rows, c.max_batch));
+    const size_t attn_bytes = trj_tree_attention_workspace(step_rows, c.max_batch, c.n_heads, c.head_dim, c.max_seq);
     char* attn_ws = cv.take<char>(attn_bytes);
     // every row count a call may bring (the K split, hence the space for partial sums, is not monotone in it)
     size_t gemm_bytes = 256;
     for (auto nk : {std::pair<int, int>{QKV, c.d_model}, {c.d_model, HD}, {2 * c.d_ff, c.d_model},
                     {c.d_model, c.d_ff}, {c.vocab, c.d_model}})
-        for (int m = 1; m <= std::min(rows, TRJ_MAX_ROWS); ++m)
+        for (int m = 1; m <= rows; ++m)
             gemm_bytes = std::max(gemm_bytes, gemm_tc_workspace(m, nk.first, nk.second));
     char* gemm_ws = cv.take<char>(gemm_bytes);
-    int32_t* chain_depth = cv.take<int32_t>(TRJ_MAX_ROWS);
+    int32_t* chain_depth = cv.take<int32_t>(PREFILL_CHUNK);
+    int32_t* prefill_geo = cv.take<int32_t>(PREFILL_MAX_SUB + 6);   // piece lengths, then three {0, n} row-offset pairs
     uint64_t* chain_anc = cv.take<uint64_t>(TRJ_MAX_ROWS * 2);
     int32_t* chunk_row_off = cv.take<int32_t>(2);
     int32_t* unit_row_off = cv.take<int32_t>(2);
@@ -245,7 +253,7 @@ size_t carve(const trj_model_cfg& c, void* ws, trj_ctx* ctx) {
         ctx->x_lo = c.dtype == TRJ_BF16 ? x_lo : nullptr; ctx->act_lo = c.dtype == TRJ_BF16 ? act_lo : nullptr;
         ctx->inv_freq = inv_freq; ctx->argmax_ws = argmax_ws; ctx->attn_ws = attn_ws; ctx->attn_ws_bytes = attn_bytes;
         ctx->gemm_ws = gemm_ws; ctx->gemm_ws_bytes = gemm_bytes;
-        ctx->chain_depth = chain_depth; ctx->chain_anc = chain_anc;
+        ctx->chain_depth = chain_depth; ctx->chain_anc = chain_anc; ctx->prefill_geo = prefill_geo;
         ctx->chunk_row_off = chunk_row_off; ctx->unit_row_off = unit_row_off;
         ctx->step_in = step_in; ctx->step_out = step_out; ctx->loop_state = loop_state;
         ctx->dev_status = step_out + STEP_STATUS_AT;
@@ -306,9 +314,10 @@ void prof_end(trj_ctx* ctx, cudaStream_t st) {
 
 // One forward of the decoder over the rows of `bt`.  lm_first/lm_rows select which rows reach the
 // LM head (prefill only needs its last row).  b0 = first sequence of the cache the batch maps to.
+// `pieces` (prefill only): attention runs piece by piece, every piece a chain below all rows before it.
 trj_status forward(trj_ctx* ctx, void* k_cache, void* v_cache, int32_t b0, const Batch& bt,
                    const int32_t* tokens, const int32_t* depth, const uint64_t* anc, int32_t anc_words,
-                   int32_t lm_first, int32_t lm_rows, cudaStream_t st) {
+                   int32_t lm_first, int32_t lm_rows, cudaStream_t st, const SubChunks* pieces = nullptr) {
     ChainScope chain;                        // the embedding below is the chain's fence
     const trj_model_cfg& c = ctx->cfg;
     const int M = bt.rows_total, d = c.d_model, HD = c.n_heads * c.head_dim, Hkv = kv_heads(c);
@@ -335,9 +344,22 @@ trj_status forward(trj_ctx* ctx, void* k_cache, void* v_cache, int32_t b0, const
                                                c.n_heads, Hkv, c.head_dim, c.max_seq, st));
         // inside the decoder the attention result reaches the output projection as a bf16 pair, like every
         // other projection input
-        LAUNCH(PROF_ATTENTION, launch_tree_attention(ctx->q, k_slab, v_slab, anc, anc_words, bt, c.n_heads, Hkv, c.head_dim,
-                                                     c.max_seq, c.dtype, ctx->x, ctx->x_lo, ctx->attn_ws,
-                                                     ctx->attn_ws_bytes, st, attn_status));
+        if (!pieces) {
+            LAUNCH(PROF_ATTENTION, launch_tree_attention(ctx->q, k_slab, v_slab, anc, anc_words, bt, c.n_heads, Hkv, c.head_dim,
+                                                         c.max_seq, c.dtype, ctx->x, ctx->x_lo, ctx->attn_ws,
+                                                         ctx->attn_ws_bytes, st, attn_status));
+        } else {
+            for (int j = 0; j < pieces->n; ++j) {
+                const int mj = j + 1 < pieces->n ? pieces->sub : pieces->last_rows;
+                // piece j sees the rows of pieces 0..j-1 as cached rows, and those were written by this very chain
+                Batch bj{pieces->lens + j, j + 1 < pieces->n ? pieces->off_full : pieces->off_last, 1, mj, mj, bt.max_len, j == 0 ? 1 : 0};
+                const size_t off = (size_t)j * pieces->sub * HD * es;
+                LAUNCH(PROF_ATTENTION, launch_tree_attention((char*)ctx->q + off, k_slab, v_slab, anc, anc_words, bj, c.n_heads, Hkv,
+                                                             c.head_dim, c.max_seq, c.dtype, (char*)ctx->x + off,
+                                                             ctx->x_lo ? (char*)ctx->x_lo + off : nullptr, ctx->attn_ws,
+                                                             ctx->attn_ws_bytes, st, attn_status));
+            }
+        }
         // While the attention kernel runs, HBM is nearly idle and the SMs it leaves free go to the first CTAs of
         // the output projection, which only wait: they ask for the start of the gate/up weights into L2.
         const WeightPrefetch ahead{ctx->w_gate_up[l], 2 * c.d_ff, d, AHEAD_BYTES, 2 * std::max(0, ctx->sm_count - attn_grid)};
@@ -355,8 +377,10 @@ trj_status forward(trj_ctx* ctx, void* k_cache, void* v_cache, int32_t b0, const
                                                 c.rms_eps, st));
     if (lm_rows > 0) {
         const size_t off = (size_t)lm_first * d * es;
+        // a verification step keeps every row's logits in place; prefill wants one row and gets it in row 0
+        float* lm_out = pieces ? ctx->logits : ctx->logits + (size_t)lm_first * c.vocab;
         LAUNCH(PROF_GEMM, launch_gemm((char*)ctx->x + off, ctx->x_lo ? (char*)ctx->x_lo + off : nullptr, ctx->lm_head,
-                                      ctx->logits + (size_t)lm_first * c.vocab, lm_rows, c.vocab, d, c.dtype,
+                                      lm_out, lm_rows, c.vocab, d, c.dtype,
                                       ctx->gemm_ws, ctx->gemm_ws_bytes, st, nullptr, nullptr, gemm_status));
     }
     return TRJ_OK;
@@ -416,13 +440,14 @@ extern "C" trj_status trj_create(const trj_model_cfg* cfg, const trj_weights* w,
     const int half = cfg->head_dim / 2;
     std::vector<double> freq(half);
     for (int i = 0; i < half; ++i) freq[i] = std::pow((double)cfg->rope_theta, -2.0 * i / cfg->head_dim);
-    std::vector<int32_t> par(TRJ_MAX_ROWS), dep(TRJ_MAX_ROWS);
+    std::vector<int32_t> par(TRJ_MAX_ROWS), dep(TRJ_MAX_ROWS), long_dep(PREFILL_CHUNK);
+    for (int i = 0; i < PREFILL_CHUNK; ++i) long_dep[i] = i;
     std::vector<uint64_t> anc(TRJ_MAX_ROWS * 2);
     for (int i = 0; i < TRJ_MAX_ROWS; ++i) par[i] = i - 1;
     tree_from_parents_impl(par.data(), TRJ_MAX_ROWS, 2, dep.data(), anc.data());
     const int32_t unit[2] = {0, 1};
     cudaError_t e = cudaMemcpy(ctx->inv_freq, freq.data(), sizeof(double) * half, cudaMemcpyHostToDevice);
-    if (e == cudaSuccess) e = cudaMemcpy(ctx->chain_depth, dep.data(), sizeof(int32_t) * TRJ_MAX_ROWS, cudaMemcpyHostToDevice);
+    if (e == cudaSuccess) e = cudaMemcpy(ctx->chain_depth, long_dep.data(), sizeof(int32_t) * PREFILL_CHUNK, cudaMemcpyHostToDevice);
     if (e == cudaSuccess) e = cudaMemcpy(ctx->chain_anc, anc.data(), sizeof(uint64_t) * TRJ_MAX_ROWS * 2, cudaMemcpyHostToDevice);
     if (e == cudaSuccess) e = cudaMemcpy(ctx->unit_row_off, unit, sizeof(unit), cudaMemcpyHostToDevice);
     if (e == cudaSuccess) e = cudaMallocHost((void**)&ctx->pin_in, STEP_IN_BYTES);
@@ -580,16 +605,21 @@ extern "C" trj_status trj_prefill(trj_ctx* ctx, void* k_cache, void* v_cache, in
     TRJ_REQUIRE(b >= 0 && b < c.max_batch, TRJ_EINVAL, "prefill: sequence %d outside the cache", b);
     TRJ_REQUIRE(n >= 1 && n <= c.max_seq, TRJ_ECAPACITY, "prefill: %d tokens do not fit %d cache rows", n, c.max_seq);
     cudaStream_t st = (cudaStream_t)stream;
-    for (int32_t done = 0; done < n; done += c.max_rows) {
-        const int32_t m = std::min(c.max_rows, n - done);
+    const int32_t sub = std::min(c.max_rows, TRJ_MAX_ROWS);                  // rows of an attention piece
+    const int32_t chunk_cap = std::min(PREFILL_CHUNK, PREFILL_MAX_SUB * sub);
+    int32_t* lens = ctx->prefill_geo, *off_all = lens + PREFILL_MAX_SUB, *off_full = off_all + 2, *off_last = off_all + 4;
+    for (int32_t done = 0; done < n; done += chunk_cap) {
+        const int32_t m = std::min(chunk_cap, n - done);
         const bool last = done + m >= n;
-        TRJ_CHECK_CUDA(launch_set_chunk(ctx->chunk_row_off, m, st));
-        Batch bt{seq_len + b, ctx->chunk_row_off, 1, m, m, c.max_seq};
+        const int32_t n_sub = (m + sub - 1) / sub, last_rows = m - (n_sub - 1) * sub;
+        TRJ_CHECK_CUDA(launch_prefill_geometry(seq_len + b, lens, n_sub, sub, m, last_rows, off_all, off_full, off_last, st));
+        Batch bt{seq_len + b, off_all, 1, m, sub, c.max_seq};
+        const SubChunks pieces{n_sub, sub, last_rows, lens, off_full, off_last};
         trj_status s = forward(ctx, k_cache, v_cache, b, bt, tokens + done, ctx->chain_depth, ctx->chain_anc, 2,
-                               m - 1, last ? 1 : 0, st);
+                               m - 1, last ? 1 : 0, st, &pieces);
         if (s != TRJ_OK) return s;
         if (last)   // greedy prediction after the last prompt token: a one-row arg-max
-            TRJ_CHECK_CUDA(launch_topk_accept(ctx->logits + (size_t)(m - 1) * c.vocab, TRJ_F32, c.vocab, 1, nullptr, nullptr,
+            TRJ_CHECK_CUDA(launch_topk_accept(ctx->logits, TRJ_F32, c.vocab, 1, nullptr, nullptr,
                                               nullptr, ctx->unit_row_off, 1, 1, nullptr, first_token, nullptr, nullptr,
                                               nullptr, nullptr, false, ctx->argmax_ws, st));
         TRJ_CHECK_CUDA(launch_bump_len(seq_len + b, m, st));

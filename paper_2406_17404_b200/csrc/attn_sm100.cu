@@ -51,6 +51,7 @@ struct AtParams {
     int* status;
     float scale_log2;            // log2(e) / sqrt(D)
     int cluster;                 // CTAs per thread-block cluster that share one head (1: no clusters)
+    int early_ok;                // cache rows below seq_len are older than the chain: they may be fetched before the wait
 };
 
 using namespace sm100;
@@ -351,6 +352,7 @@ __global__ void __launch_bounds__(at_threads(AT_SPLIT), 1) tree_attention_tc_ker
             bool ok = true;
             bool waited = false;                             // for the previous kernel (see above)
             const uint64_t kv_policy = l2_evict_first_policy();
+            if (!p.early_ok) { pdl_wait(); waited = true; }
             for (int u = u_begin; u < u_end && ok;) {
                 Where w; sched.locate(u, w);
                 const int t_end = min(w.tiles, w.t + (u_end - u));
@@ -874,6 +876,7 @@ cudaError_t launch_tree_attention_tc(const void* q, const void* k_slab, const vo
     p.seq_len = bt.seq_len; p.row_off = bt.row_off; p.anc = anc; p.anc_words = anc_words;
     p.B = bt.B; p.H = H; p.max_seq = max_seq;
     p.Hkv = Hkv; p.group = H / Hkv;
+    p.early_ok = bt.cached_rows_final;
     p.out = (__nv_bfloat16*)out;
     p.out_lo = (__nv_bfloat16*)out_lo;
     p.status = status ? status : (int*)workspace;

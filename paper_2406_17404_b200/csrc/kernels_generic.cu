@@ -740,6 +740,13 @@ __global__ void advance_len_kernel(int32_t* seq_len, const int32_t* k_acc, int B
     if (b < B) seq_len[b] += k_acc[b] + 1;
 }
 __global__ void set_chunk_kernel(int32_t* row_off2, int m) { row_off2[0] = 0; row_off2[1] = m; }
+__global__ void prefill_geometry_kernel(const int32_t* seq_len_b, int32_t* lens, int n_sub, int sub, int m, int last_rows,
+                                        int32_t* off_all, int32_t* off_full, int32_t* off_last) {
+    for (int j = threadIdx.x; j < n_sub; j += blockDim.x) lens[j] = *seq_len_b + j * sub;
+    if (threadIdx.x == 0) {
+        off_all[0] = 0; off_all[1] = m; off_full[0] = 0; off_full[1] = sub; off_last[0] = 0; off_last[1] = last_rows;
+    }
+}
 __global__ void bump_len_kernel(int32_t* seq_len_b, int delta) { *seq_len_b += delta; }
 
 }  // namespace
@@ -964,6 +971,12 @@ cudaError_t launch_compact(void* k_cache, void* v_cache, int32_t L, int32_t B_ca
 cudaError_t launch_set_chunk(int32_t* row_off2, int32_t m, cudaStream_t st) {
     count_launch();
     set_chunk_kernel<<<1, 1, 0, st>>>(row_off2, m);
+    return cudaGetLastError();
+}
+cudaError_t launch_prefill_geometry(const int32_t* seq_len_b, int32_t* lens, int32_t n_sub, int32_t sub, int32_t m,
+                                    int32_t last_rows, int32_t* off_all, int32_t* off_full, int32_t* off_last, cudaStream_t st) {
+    count_launch();
+    prefill_geometry_kernel<<<1, 32, 0, st>>>(seq_len_b, lens, n_sub, sub, m, last_rows, off_all, off_full, off_last);
     return cudaGetLastError();
 }
 cudaError_t launch_bump_len(int32_t* seq_len_b, int32_t delta, cudaStream_t st) {

@@ -77,6 +77,9 @@ struct Batch {
     const int32_t* seq_len;   // [B] dev
     const int32_t* row_off;   // [B+1] dev
     int32_t B, rows_total, max_rows, max_len;
+    // 1: every cache row below seq_len was written before the chain of kernels this batch is launched in began, so a
+    // kernel may fetch such rows ahead of its wait for its predecessor; 0: some were written inside the chain
+    int32_t cached_rows_final = 1;
 };
 
 // Weights of a LATER projection that a projection kernel may ask for ahead of time.  When the kernel before a
@@ -196,6 +199,10 @@ cudaError_t launch_compact(void* k_cache, void* v_cache, int32_t L, int32_t B_ca
                            const int32_t* k_acc, const int32_t* path, cudaStream_t st);
 // row_off = {0, m} and seq_len[b] += delta: small bookkeeping used by prefill.
 cudaError_t launch_set_chunk(int32_t* row_off2, int32_t m, cudaStream_t st);
+// Geometry of a prefill chunk of m rows whose attention runs in n_sub pieces of `sub` rows (the last one of
+// last_rows): lens[j] = *seq_len_b + j * sub, off_all = {0, m}, off_full = {0, sub}, off_last = {0, last_rows}.
+cudaError_t launch_prefill_geometry(const int32_t* seq_len_b, int32_t* lens, int32_t n_sub, int32_t sub, int32_t m,
+                                    int32_t last_rows, int32_t* off_all, int32_t* off_full, int32_t* off_last, cudaStream_t st);
 cudaError_t launch_bump_len(int32_t* seq_len_b, int32_t delta, cudaStream_t st);
 
 }  // namespace trj
