@@ -482,7 +482,7 @@ def bench_prefill_gemm(trj, torch, peaks, steps):
     return out
 
 
-def planted_lengths(seed, n):def planted_lengths(seed, n):
+def planted_lengths(seed, n):
     """How many tokens of the true continuation each step's first retrieved branch carries: uniform on 0..3, so
     that a step commits 1 + (0..3) tokens, 2.5 on average (the paper's Table 2 reports 2.0-2.9 per step)."""
     import synth
