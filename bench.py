@@ -148,7 +148,7 @@ def oracle_attention_us(prefixes, rows_list, parents, n_heads, d):
     return 1e6 * t * n_heads
 
 
-def bench_tree_attention(trj, torch, peaks, steps, warmup, cpu=True):
+def bench_tree_attention(trj, torch, peaks, steps, warmup, cpu=True, only=""):
     """Op-level tree attention on the op-level shapes (configs 2, 4, 5), over distinct caches larger than L2."""
     import synth
     out = []
@@ -159,6 +159,8 @@ def bench_tree_attention(trj, torch, peaks, steps, warmup, cpu=True):
              ("cfg4: 32x128 heads, prefix 8192, 128-row tree", [8192], [128], 8, 4, 4),
              ("cfg5: 8 sequences, prefix 256-4096, 16-64-row trees", s5.tolist(), m5.tolist(), 6, 3, 2))
     for name, prefixes, rows_list, depth, kids, n_caches in cases:
+        if only and only not in name:
+            continue
         nb, rows_total = len(prefixes), sum(rows_list)
         max_seq = max(s + m for s, m in zip(prefixes, rows_list))
         g = torch.Generator(device="cuda"); g.manual_seed(7)
@@ -269,8 +271,51 @@ def run_ops_only(args):
     trj.lib()
     peaks = measured_peaks()
     steps = max(args.steps, 5)
-    print(json.dumps({"ops_only": True, "tree_attention": bench_tree_attention(trj, torch, peaks, steps, 3),
-                      "small_ops": bench_small_ops(trj, torch, peaks, steps, 3)}), flush=True)
+    out = {"ops_only": True}
+    if args.case in ("", "cfg2", "cfg3", "cfg4", "cfg5"):
+        out["tree_attention"] = bench_tree_attention(trj, torch, peaks, steps, 3, cpu=False, only=args.case)
+    if args.case in ("", "small"):
+        out["small_ops"] = bench_small_ops(trj, torch, peaks, steps, 3, cpu=False)
+    if args.case in ("", "gemm"):
+        out["prefill_gemm"] = bench_prefill_gemm(trj, torch, peaks, steps)
+    print(json.dumps(out), flush=True)
+
+
+def run_profile_step(args):
+    """A short, fixed launch sequence for a profiler: model set-up, prefill of the prompt, then `--steps` verification
+    steps (forward, arg-max + accept, compaction) launched one by one, without a CUDA graph.  Prints the number of
+    library launches before the first step and per step, so that a capture can skip to the steps."""
+    import torch
+    import synth
+    from synth.device import device_weights
+    import paper_2406_17404_b200 as trj
+    trj.lib()
+    torch.cuda.set_device(0)
+    dev = torch.device("cuda", 0)
+    cfg = synth.LLAMA7B if not args.layers else synth.LLAMA7B.with_layers(args.layers)
+    layers, glob = device_weights(cfg, 1234, dev)
+    model = trj.Model(cfg, layers, glob, max_batch=1, max_seq=PROMPT + 256, max_rows=trj.MAX_ROWS)
+    i32 = lambda a: torch.from_numpy(np.ascontiguousarray(a, dtype=np.int32)).to(dev)
+    prompt = synth.prompt(100, PROMPT, cfg.vocab)
+    first = model.prefill(i32(prompt))
+    ctx = np.concatenate([prompt, [int(first.item())]]).astype(np.int32)
+    draws = np.asarray(synth.noise_draws(0, 1, WIDTH + N_BRANCHES * BRANCH_LEN), np.int64)
+    window = ctx[np.asarray(synth.noise_draws(0, 0, WIDTH), np.int64) % len(ctx)]
+    tree = trj.build_tree(int(ctx[-1]), window, trj.retrieve(ctx, N_BRANCHES, BRANCH_LEN, draws[WIDTH:]))
+    d_tok, d_par, d_dep, d_off = i32(tree["tokens"]), i32(tree["parent"]), i32(tree["depth"]), i32([0, TREE_ROWS])
+    d_anc = torch.from_numpy(tree["anc"].view(np.int64)).to(dev)
+    seq0 = model.seq_len.clone()
+    torch.cuda.synchronize()
+    before = trj.launch_count()
+    for _ in range(args.steps):
+        model.seq_len.copy_(seq0)
+        out = model.verify_step(d_tok, d_par, d_dep, d_anc, d_off, max_rows=TREE_ROWS, max_len=PROMPT + TREE_ROWS)
+        acc = model.accept(d_tok, d_par, d_dep, d_off, out["node_argmax"])
+        model.compact_kv(acc["k_acc"], acc["path"])
+    torch.cuda.synchronize()
+    print(json.dumps({"profile_step": True, "layers": cfg.n_layers, "library_launches_before_the_steps": before,
+                      "library_launches_per_step": (trj.launch_count() - before) // max(args.steps, 1)}), flush=True)
+    model.close()
 
 
 def oracle_step_inputs(cfg, seed):
@@ -709,6 +754,20 @@ def run_ours(args, rank, world, local_rank):
                 "device_ms_per_step": gemm_ms_upper,
                 "duration_basis": "whole replayed step (upper bound)" if gemm_ms_upper == ms_step else "event brackets",
                 "bracketed_ms_per_step": gemm_ms_step}
+    if world == 1 and not args.no_timeline:
+        # the projections' own time inside the replayed step, from the clock-stamp build run as a child process
+        try:
+            child = subprocess.run([sys.executable, os.path.abspath(__file__), "--timeline", "--steps", "5"] +
+                                   (["--layers", str(args.layers)] if args.layers else []),
+                                   capture_output=True, text=True, timeout=600)
+            tl = json.loads(child.stdout.strip().splitlines()[-1])
+            roofline["kernel_ms_stamped"] = tl["projection_ms_per_step"]
+            roofline["achieved_stamped"] = tl["projection_gbs"]
+            roofline["frac_stamped"] = tl["projection_gbs"] / peaks["hbm_gbs"]
+            roofline["timeline_per_kernel_us"] = tl["per_kernel_us"]
+        except Exception as exc:                             # the headline numbers do not depend on this leg
+            roofline["kernel_ms_stamped"] = None
+            roofline["timeline_error"] = repr(exc)[:200]
     step_ms_prof = sum(v[0] for v in prof.values()) / args.steps
     breakdown = {k: {"ms_per_step": round(v[0] / args.steps, 4), "launches_per_step": v[1] // args.steps} for k, v in prof.items()}
 
@@ -756,6 +815,79 @@ def run_ours(args, rank, world, local_rank):
     model.close()
 
 
+def run_timeline(args):
+    """Per-kernel clock stamps of the replayed step, from the -DTRJ_TIMELINE build of the library (built here into a
+    second shared object; the default library carries no instrumentation).  For every per-layer kernel: the time
+    from the moment its first CTA is released by its predecessor to the end of its last CTA, and the gap to the next
+    release.  Prints one JSON line; `projection_ms_per_step` is the sum over the 129 projection launches."""
+    import torch
+    import synth
+    from synth.device import device_weights
+    from paper_2406_17404_b200 import build as trj_build
+    import paper_2406_17404_b200 as trj
+    trj.use_library(trj_build.build(timeline=True))
+    trj.lib()
+    torch.cuda.set_device(0)
+    dev = torch.device("cuda", 0)
+    cfg = synth.LLAMA7B if not args.layers else synth.LLAMA7B.with_layers(args.layers)
+    layers, glob = device_weights(cfg, 1234, dev)
+    model = trj.Model(cfg, layers, glob, max_batch=1, max_seq=PROMPT + 256, max_rows=trj.MAX_ROWS)
+    i32 = lambda a: torch.from_numpy(np.ascontiguousarray(a, dtype=np.int32)).to(dev)
+    prompt = synth.prompt(100, PROMPT, cfg.vocab)
+    first = model.prefill(i32(prompt))
+    ctx = np.concatenate([prompt, [int(first.item())]]).astype(np.int32)
+    draws = np.asarray(synth.noise_draws(0, 1, WIDTH + N_BRANCHES * BRANCH_LEN), np.int64)
+    window = ctx[np.asarray(synth.noise_draws(0, 0, WIDTH), np.int64) % len(ctx)]
+    tree = trj.build_tree(int(ctx[-1]), window, trj.retrieve(ctx, N_BRANCHES, BRANCH_LEN, draws[WIDTH:]))
+    d_tok, d_par, d_dep, d_off = i32(tree["tokens"]), i32(tree["parent"]), i32(tree["depth"]), i32([0, TREE_ROWS])
+    d_anc = torch.from_numpy(tree["anc"].view(np.int64)).to(dev)
+    seq0 = model.seq_len.clone()
+    pred = torch.empty(TREE_ROWS, dtype=torch.int32, device=dev)
+    acc = {"k_acc": torch.empty(1, dtype=torch.int32, device=dev), "bonus": torch.empty(1, dtype=torch.int32, device=dev),
+           "path": torch.empty(1, trj.PATH_STRIDE, dtype=torch.int32, device=dev)}
+
+    def step():
+        model.seq_len.copy_(seq0)
+        trj.timeline_reset()
+        model.verify_step(d_tok, d_par, d_dep, d_anc, d_off, max_rows=TREE_ROWS, max_len=PROMPT + TREE_ROWS, node_argmax=pred)
+        model.accept(d_tok, d_par, d_dep, d_off, pred, out=acc)
+        model.compact_kv(acc["k_acc"], acc["path"])
+    side = torch.cuda.Stream(device=dev)
+    with torch.cuda.stream(side):
+        for _ in range(2):
+            step()
+    torch.cuda.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph, stream=side):
+        step()
+    for _ in range(3):
+        graph.replay()
+    torch.cuda.synchronize()
+    dur = {k: [] for k in trj.TL_KINDS}
+    gap = {k: [] for k in trj.TL_KINDS}
+    span, proj = [], []
+    for _ in range(max(args.steps, 3)):
+        graph.replay()
+        torch.cuda.synchronize()
+        rec = trj.timeline_read()
+        events = sorted((int(b), int(e), k) for k, (bs, es) in rec.items() for b, e in zip(bs, es))
+        for i, (b, e, k) in enumerate(events):
+            dur[k].append((e - b) / 1e3)
+            if i + 1 < len(events):
+                gap[k].append((events[i + 1][0] - e) / 1e3)
+        span.append((max(e for _, e, _ in events) - min(b for b, _, _ in events)) / 1e6)
+        proj.append(sum(e - b for b, e, k in events if k == "gemm") / 1e6)
+    mean = lambda v: round(float(np.mean(v)), 3) if v else None
+    line = {"timeline": True, "layers": cfg.n_layers, "tree_rows": TREE_ROWS, "prefix": PROMPT,
+            "per_kernel_us": {k: {"launches_per_step": len(dur[k]) // max(args.steps, 3), "release_to_end": mean(dur[k]),
+                                  "gap_to_next_release": mean(gap[k])} for k in trj.TL_KINDS},
+            "projection_ms_per_step": mean(proj), "first_release_to_last_end_ms": mean(span),
+            "projection_bytes_per_step": gemm_bytes_per_step(cfg, TREE_ROWS),
+            "projection_gbs": round(gemm_bytes_per_step(cfg, TREE_ROWS) / (float(np.mean(proj)) / 1e3) / 1e9, 1)}
+    print(json.dumps(line), flush=True)
+    model.close()
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -765,7 +897,13 @@ def main():
     ap.add_argument("--layers", type=int, default=0, help="debug: fewer layers than the 7B shape (invalidates the number)")
     ap.add_argument("--no-pdl", action="store_true", help="launch the kernels fully serialised (comparison only)")
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-oracle baseline leg")
+    ap.add_argument("--no-timeline", action="store_true", help="skip the clock-stamp leg (a child process with the -DTRJ_TIMELINE build)")
     ap.add_argument("--no-attention", action="store_true", help="skip the op-level tree-attention leg")
+    ap.add_argument("--case", default="", help="with --ops-only: cfg2 | cfg3 | cfg4 | cfg5 | small | gemm (default: all)")
+    ap.add_argument("--profile-step", action="store_true",
+                    help="prefill + a few un-graphed verification steps and nothing else: a launch sequence for a profiler")
+    ap.add_argument("--timeline", action="store_true",
+                    help="per-kernel clock stamps of the replayed step from the -DTRJ_TIMELINE build (one JSON line)")
     ap.add_argument("--ops-only", action="store_true",
                     help="only the op-level legs (tree attention, arg-max + accept, compaction): a small run for profiling")
     args = ap.parse_args()
@@ -775,6 +913,14 @@ def main():
     if args.ops_only:
         if rank == 0:
             run_ops_only(args)
+        return
+    if args.timeline:
+        if rank == 0:
+            run_timeline(args)
+        return
+    if args.profile_step:
+        if rank == 0:
+            run_profile_step(args)
         return
     if args.impl == "reference":
         run_reference(args, rank, world)

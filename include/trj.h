@@ -454,6 +454,21 @@ trj_status trj_selftest_wait_expiry(int32_t* status, int32_t polls, void* stream
  * itself again (read with keep = 1 after each replay). */
 #define TRJ_PROF_CATEGORIES 6
 uint64_t   trj_launch_count(void);
+/* Clock stamps of the per-layer kernels.  Only a library built with -DTRJ_TIMELINE records them (the default
+ * build returns TRJ_EUNSUPPORTED from both calls and carries no instrumentation).  Every launch of a kind below
+ * records the time (ns, GPU global timer) at which its first CTA got past the wait for the previous kernel and the
+ * time at which its last CTA ended.  trj_timeline_reset clears the record (enqueued on `stream`);
+ * trj_timeline_read copies the launches of one kind since the last reset, in launch order, to begin_ns / end_ns
+ * (host, max_launches each) and their number to *n_launches; synchronise the device first. */
+#define TRJ_TL_RMSNORM   0   /* residual add + RMSNorm        */
+#define TRJ_TL_GEMM      1   /* projection                     */
+#define TRJ_TL_ROPE      2   /* rotary embedding + K/V append  */
+#define TRJ_TL_ATTENTION 3   /* tree attention                 */
+#define TRJ_TL_SWIGLU    4   /* SwiGLU                         */
+#define TRJ_TL_EMBED     5   /* embedding gather               */
+#define TRJ_TL_KINDS     6
+trj_status trj_timeline_reset(void* stream);
+trj_status trj_timeline_read(int32_t kind, int32_t max_launches, uint64_t* begin_ns, uint64_t* end_ns, int32_t* n_launches);
 /* Programmatic dependent launch (on by default): the kernels of a step are launched so that each may
  * be scheduled, and may prefetch weights, while its predecessor in the stream is still running.
  * trj_set_pdl(0) launches them fully serialised instead (for comparison).  Process-wide; set it

@@ -88,6 +88,8 @@ _SIGNATURES = {
     "trj_gemm": (_I, [_VP, _VP, _VP, _I, _I, _I, _I, _VP, _SZ, _VP]),
     "trj_device_status": (_I, [_VP, _I, _VP]),
     "trj_selftest_wait_expiry": (_I, [_VP, _I, _VP]),
+    "trj_timeline_reset": (_I, [_VP]),
+    "trj_timeline_read": (_I, [_I, _I, _U64P, _U64P, _I32P]),
     "trj_launch_count": (C.c_uint64, []),
     "trj_set_pdl": (None, [_I]),
     "trj_profile_enable": (_I, [_VP, _I]),
@@ -95,6 +97,33 @@ _SIGNATURES = {
 }
 PROF_CATEGORIES = ("elementwise", "gemm", "rope_kv", "attention", "argmax_accept", "compact")
 EXPORTS = tuple(_SIGNATURES)
+
+
+def use_library(path: str) -> None:
+    """Load another build of the library (the clock-stamp build) instead of the default one; call before lib()."""
+    global _lib, LIB_PATH
+    if _lib is not None:
+        raise RuntimeError("a library is already loaded")
+    LIB_PATH = path
+
+
+TL_KINDS = ("rmsnorm", "gemm", "rope_kv", "attention", "swiglu", "embed")
+
+
+def timeline_reset(stream=None) -> None:
+    """trj_timeline_reset (clock-stamp build only)."""
+    _check(lib().trj_timeline_reset(_stream(stream)))
+
+
+def timeline_read(max_launches: int = 512):
+    """trj_timeline_read for every kind: {kind: (begin_ns, end_ns)} as uint64 arrays in launch order."""
+    out = {}
+    for kind, name in enumerate(TL_KINDS):
+        b, e = np.zeros(max_launches, np.uint64), np.zeros(max_launches, np.uint64)
+        n = C.c_int32(0)
+        _check(lib().trj_timeline_read(kind, max_launches, b.ctypes.data_as(_U64P), e.ctypes.data_as(_U64P), C.byref(n)))
+        out[name] = (b[:n.value].copy(), e[:n.value].copy())
+    return out
 
 
 def lib() -> C.CDLL:

@@ -36,8 +36,19 @@ def _stale(target: str, deps) -> bool:
     return any(os.path.getmtime(d) > t for d in deps)
 
 
-def build(verbose: bool = False, force: bool = False) -> str:
-    """Compile every source under csrc/ and link libtrj.so; returns its path."""
+def build(verbose: bool = False, force: bool = False, timeline: bool = False) -> str:
+    """Compile every source under csrc/ and link libtrj.so; returns its path.  ``timeline=True`` builds a second
+    library, libtrj_timeline.so, with -DTRJ_TIMELINE (clock stamps in the per-layer kernels; measurement only)."""
+    global OBJ, LIB
+    if timeline:
+        saved = OBJ, LIB, list(NVCC_FLAGS)
+        OBJ, LIB = os.path.join(HERE, "_build_timeline"), os.path.join(HERE, "libtrj_timeline.so")
+        NVCC_FLAGS.append("-DTRJ_TIMELINE")
+        try:
+            return build(verbose, force)
+        finally:
+            OBJ, LIB = saved[0], saved[1]
+            NVCC_FLAGS[:] = saved[2]
     headers = [os.path.join(CSRC, f) for f in os.listdir(CSRC) if f.endswith((".h", ".cuh"))]
     headers.append(os.path.join(ROOT, "include", "trj.h"))
     if not force and not verbose and not _stale(LIB, [os.path.join(CSRC, s) for s in sources()] + headers):
@@ -70,4 +81,4 @@ def build(verbose: bool = False, force: bool = False) -> str:
 
 
 if __name__ == "__main__":
-    print(build(verbose="-v" in sys.argv, force="-f" in sys.argv))
+    print(build(verbose="-v" in sys.argv, force="-f" in sys.argv, timeline="--timeline" in sys.argv))

@@ -500,6 +500,35 @@ extern "C" trj_status trj_selftest_wait_expiry(int32_t* status, int32_t polls, v
     return TRJ_OK;
 }
 
+extern "C" trj_status trj_timeline_reset(void* stream) {
+#ifdef TRJ_TIMELINE
+    cudaStream_t st = (cudaStream_t)stream;
+    TRJ_CHECK_CUDA(timeline_reset_generic(st));
+    TRJ_CHECK_CUDA(timeline_reset_gemm(st));
+    TRJ_CHECK_CUDA(timeline_reset_attention(st));
+    return TRJ_OK;
+#else
+    (void)stream;
+    return fail(TRJ_EUNSUPPORTED, "timeline: this library was built without -DTRJ_TIMELINE");
+#endif
+}
+
+extern "C" trj_status trj_timeline_read(int32_t kind, int32_t max_launches, uint64_t* begin_ns, uint64_t* end_ns, int32_t* n_launches) {
+#ifdef TRJ_TIMELINE
+    TRJ_REQUIRE(begin_ns && end_ns && n_launches && max_launches >= 0, TRJ_EINVAL, "timeline_read: null pointer");
+    TRJ_REQUIRE(kind >= 0 && kind < TRJ_TL_KINDS, TRJ_EINVAL, "timeline_read: kind %d outside 0..%d", kind, TRJ_TL_KINDS - 1);
+    int n = kind == TRJ_TL_GEMM ? timeline_read_gemm(kind, max_launches, begin_ns, end_ns)
+          : kind == TRJ_TL_ATTENTION ? timeline_read_attention(kind, max_launches, begin_ns, end_ns)
+                                     : timeline_read_generic(kind, max_launches, begin_ns, end_ns);
+    TRJ_REQUIRE(n >= 0, TRJ_ECUDA, "timeline_read: copy from the device failed");
+    *n_launches = n;
+    return TRJ_OK;
+#else
+    (void)kind; (void)max_launches; (void)begin_ns; (void)end_ns; (void)n_launches;
+    return fail(TRJ_EUNSUPPORTED, "timeline: this library was built without -DTRJ_TIMELINE");
+#endif
+}
+
 extern "C" uint64_t trj_launch_count(void) { return launches_so_far(); }
 extern "C" void trj_set_pdl(int32_t on) { set_pdl(on != 0); }
 

@@ -18,6 +18,7 @@
 #include <mutex>
 #include "trj_internal.h"
 #include "sm100_common.cuh"
+#include "timeline.cuh"
 
 namespace trj {
 namespace {
@@ -311,6 +312,7 @@ __global__ void __launch_bounds__(at_threads(AT_SPLIT), 1) tree_attention_tc_ker
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
     pdl_launch_dependents();
+    TRJ_TL_DECL;
     if (threadIdx.x == 32) {                                 // have the tensor maps on their way before the first copy needs them
         asm volatile("prefetch.tensormap [%0];" ::"l"(&map_q) : "memory");
         asm volatile("prefetch.tensormap [%0];" ::"l"(&map_k) : "memory");
@@ -474,7 +476,7 @@ __global__ void __launch_bounds__(at_threads(AT_SPLIT), 1) tree_attention_tc_ker
             }
             const int total = w.S + w.rows;
             float m_ref = -INFINITY, l_sum = 0.f;
-            if (e == 0) pdl_wait();                          // the ancestor masks above are older than the chain
+            if (e == 0) { pdl_wait(); TRJ_TL_BEGIN(TRJ_TL_ATTENTION); }      // the ancestor masks above are older than the chain
             for (g = g0; g < g1 && ok; ++g) {
                 const int key0 = (w.t + (g - g0)) * AT_KEYS;
                 const bool edge = key0 + AT_KEYS > w.S;      // the tile reaches tree rows or the end of the keys
@@ -707,6 +709,10 @@ __global__ void __launch_bounds__(at_threads(AT_SPLIT), 1) tree_attention_tc_ker
     }
     if (warp == AT_W_MMA)
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(512u) : "memory");
+#ifdef TRJ_TIMELINE
+    if (threadIdx.x == 0 && u_begin >= u_end) tl_slot__ = ::trj::tl::begin(TRJ_TL_ATTENTION);   // a CTA without work never stamped its release
+#endif
+    TRJ_TL_END(TRJ_TL_ATTENTION);
 }
 
 // Merges the pieces of every (sequence, head) that more than one CTA worked on.  One CTA per
@@ -839,6 +845,11 @@ AtPlan at_plan(int32_t B, int32_t H, int32_t max_len) {
 }
 
 }  // namespace
+
+#ifdef TRJ_TIMELINE
+cudaError_t timeline_reset_attention(cudaStream_t st) { return tl::reset(st); }
+int timeline_read_attention(int kind, int max_launches, uint64_t* b, uint64_t* e) { return tl::read(kind, max_launches, b, e); }
+#endif
 
 int tree_attention_grid(int32_t B, int32_t H, int32_t max_len) { return at_plan(B, H, max_len).grid; }
 

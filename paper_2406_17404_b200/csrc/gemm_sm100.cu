@@ -20,6 +20,7 @@
 #include <algorithm>
 #include "trj_internal.h"
 #include "sm100_common.cuh"
+#include "timeline.cuh"
 
 namespace trj {
 namespace {
@@ -69,6 +70,7 @@ __global__ void __launch_bounds__(TC_THREADS, 2) gemm_tc_kernel(const __grid_con
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int per_tile = p.splits * p.m_blocks;              // items of one weight tile: block index fastest
     const int items = p.tiles * per_tile;
+    TRJ_TL_DECL;
 
     pdl_launch_dependents();
     if (threadIdx.x == 32) {                                 // have the tensor maps on their way before the first copy needs them
@@ -141,6 +143,7 @@ __global__ void __launch_bounds__(TC_THREADS, 2) gemm_tc_kernel(const __grid_con
                         for (int i = blockIdx.x; i < p.ahead_boxes; i += p.ahead_ctas)
                             tma_prefetch_l2_2d(&map_ahead, (i % p.ahead_kblocks) * TC_BK, (i / p.ahead_kblocks) * TC_BM);
                     pdl_wait();                              // activations come from the previous kernel
+                    TRJ_TL_BEGIN(TRJ_TL_GEMM);
                 }
             }
         }
@@ -216,6 +219,7 @@ __global__ void __launch_bounds__(TC_THREADS, 2) gemm_tc_kernel(const __grid_con
     }
     if (warp == 1)
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)(2 * p.acc_cols)) : "memory");
+    TRJ_TL_END(TRJ_TL_GEMM);
 }
 
 // y[i] = sum_s part[s][i], fixed order.
@@ -402,6 +406,11 @@ cudaError_t launch_gemm_tc(const void* x, const void* x_lo, const void* w, float
         (const float4*)workspace, (float4*)y, n4, p.splits);
     return cudaGetLastError();
 }
+
+#ifdef TRJ_TIMELINE
+cudaError_t timeline_reset_gemm(cudaStream_t st) { return tl::reset(st); }
+int timeline_read_gemm(int kind, int max_launches, uint64_t* b, uint64_t* e) { return tl::read(kind, max_launches, b, e); }
+#endif
 
 cudaError_t launch_wait_expiry_selftest(int* status, uint32_t polls, cudaStream_t st) {
     count_launch();

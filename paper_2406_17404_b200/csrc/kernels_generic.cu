@@ -5,6 +5,7 @@
 #include <mutex>
 #include <algorithm>
 #include "trj_internal.h"
+#include "timeline.cuh"
 
 namespace trj {
 namespace {
@@ -81,9 +82,11 @@ __global__ void embed_kernel(const T* __restrict__ embed, const int32_t* __restr
                              float* __restrict__ h, int d) {
     pdl_wait();                                  // the chain's fence: everything enqueued earlier is complete
     pdl_launch_dependents();                     // before any later kernel of the chain may start
+    TRJ_TL_DECL; TRJ_TL_BEGIN(TRJ_TL_EMBED);
     const int row = blockIdx.x;
     const T* src = embed + (size_t)tokens[row] * d;
     for (int c = threadIdx.x; c < d; c += blockDim.x) h[(size_t)row * d + c] = to_f(src[c]);
+    TRJ_TL_END(TRJ_TL_EMBED);
 }
 
 // ---------------------------------------------------------------- residual add + RMSNorm
@@ -130,6 +133,7 @@ __global__ void __launch_bounds__(RMS_THREADS) add_rmsnorm_vec_kernel(float* __r
                                                                      const float* __restrict__ gain, T* __restrict__ x,
                                                                      T* __restrict__ x_lo, int d, float eps) {
     pdl_prologue();
+    TRJ_TL_DECL; TRJ_TL_BEGIN(TRJ_TL_RMSNORM);
     __shared__ float red[32];
     const int row = blockIdx.x, n4 = d >> 2;
     float4 v[RMS_CHUNKS];
@@ -157,6 +161,10 @@ __global__ void __launch_bounds__(RMS_THREADS) add_rmsnorm_vec_kernel(float* __r
                             make_float4(v[k].x * inv * g.x, v[k].y * inv * g.y, v[k].z * inv * g.z, v[k].w * inv * g.w));
         }
     }
+#ifdef TRJ_TIMELINE
+    __syncthreads();
+#endif
+    TRJ_TL_END(TRJ_TL_RMSNORM);
 }
 
 template <typename T>
@@ -291,7 +299,8 @@ __global__ void __launch_bounds__(ROPE_THREADS) rope_kv_write_vec_kernel(const P
     const int half = D >> 1, HD = H * D, KD = Hkv * D, per_head = half >> 2;
     const int row = blockIdx.x, hh = blockIdx.y * heads_per_cta + (int)threadIdx.x / per_head;
     const int i = ((int)threadIdx.x % per_head) * 4;
-    if (hh >= H) return;
+    TRJ_TL_DECL;
+    if (hh >= H) return;                                     // never thread 0: a CTA's first thread has a head
     const int b = seq_of_row(row_off, B, row);
     const int local = row - row_off[b];
     const int pos = seq_len[b] + depth[row];
@@ -310,6 +319,7 @@ __global__ void __launch_bounds__(ROPE_THREADS) rope_kv_write_vec_kernel(const P
         sincosf((float)red, &sn[e], &cs[e]);
     }
     pdl_wait();
+    TRJ_TL_BEGIN(TRJ_TL_ROPE);
     float4 acc[6];                                           // q, k, v: first and second half of the head
 #pragma unroll
     for (int e = 0; e < 6; ++e) acc[e] = make_float4(0.f, 0.f, 0.f, 0.f);
@@ -340,11 +350,13 @@ __global__ void __launch_bounds__(ROPE_THREADS) rope_kv_write_vec_kernel(const P
     };
     store_split4<T>(q_out, nullptr, q_at, rot_lo(acc[0], acc[1]));
     store_split4<T>(q_out, nullptr, q_at + half, rot_hi(acc[0], acc[1]));
-    if (!has_kv) return;
-    store_split4<T>(k_slab, nullptr, cache_at, rot_lo(acc[2], acc[3]));
-    store_split4<T>(k_slab, nullptr, cache_at + half, rot_hi(acc[2], acc[3]));
-    store_split4<T>(v_slab, nullptr, cache_at, acc[4]);
-    store_split4<T>(v_slab, nullptr, cache_at + half, acc[5]);
+    if (has_kv) {
+        store_split4<T>(k_slab, nullptr, cache_at, rot_lo(acc[2], acc[3]));
+        store_split4<T>(k_slab, nullptr, cache_at + half, rot_hi(acc[2], acc[3]));
+        store_split4<T>(v_slab, nullptr, cache_at, acc[4]);
+        store_split4<T>(v_slab, nullptr, cache_at + half, acc[5]);
+    }
+    TRJ_TL_END(TRJ_TL_ROPE);                                 // thread 0's own stores; the others' end within the same few hundred ns
 }
 
 // ---------------------------------------------------------------- tree attention, one CTA per (row, head)
@@ -439,6 +451,7 @@ __global__ void swiglu_kernel(const Parts gu, T* __restrict__ act, T* __restrict
 template <typename T>
 __global__ void swiglu_vec_kernel(const Parts gu, T* __restrict__ act, T* __restrict__ act_lo, int rows, int f) {
     pdl_prologue();
+    TRJ_TL_DECL; TRJ_TL_BEGIN(TRJ_TL_SWIGLU);
     const int f4 = f >> 2;
     const size_t n4 = (size_t)rows * f4;
     for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n4; i += (size_t)gridDim.x * blockDim.x) {
@@ -448,6 +461,10 @@ __global__ void swiglu_vec_kernel(const Parts gu, T* __restrict__ act, T* __rest
                         make_float4(g.x / (1.f + expf(-g.x)) * u.x, g.y / (1.f + expf(-g.y)) * u.y,
                                     g.z / (1.f + expf(-g.z)) * u.z, g.w / (1.f + expf(-g.w)) * u.w));
     }
+#ifdef TRJ_TIMELINE
+    __syncthreads();
+#endif
+    TRJ_TL_END(TRJ_TL_SWIGLU);
 }
 
 // ---------------------------------------------------------------- arg-max + acceptance
@@ -759,6 +776,10 @@ static thread_local int t_chain_depth = 0;
 bool chain_active() { return t_chain_depth > 0 && pdl_enabled(); }
 ChainScope::ChainScope() { ++t_chain_depth; }
 ChainScope::~ChainScope() { --t_chain_depth; }
+#ifdef TRJ_TIMELINE
+cudaError_t timeline_reset_generic(cudaStream_t st) { return tl::reset(st); }
+int timeline_read_generic(int kind, int max_launches, uint64_t* b, uint64_t* e) { return tl::read(kind, max_launches, b, e); }
+#endif
 static std::atomic<uint64_t> g_launches{0};
 void count_launch() { g_launches.fetch_add(1, std::memory_order_relaxed); }
 uint64_t launches_so_far() { return g_launches.load(std::memory_order_relaxed); }

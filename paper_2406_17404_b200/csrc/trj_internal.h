@@ -67,6 +67,16 @@ cudaError_t launch_chain(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t
 }
 #endif
 
+// ---- optional clock stamps (builds with -DTRJ_TIMELINE): one table per translation unit that holds kernels
+#ifdef TRJ_TIMELINE
+cudaError_t timeline_reset_generic(cudaStream_t st);
+cudaError_t timeline_reset_gemm(cudaStream_t st);
+cudaError_t timeline_reset_attention(cudaStream_t st);
+int timeline_read_generic(int kind, int max_launches, uint64_t* begin_ns, uint64_t* end_ns);
+int timeline_read_gemm(int kind, int max_launches, uint64_t* begin_ns, uint64_t* end_ns);
+int timeline_read_attention(int kind, int max_launches, uint64_t* begin_ns, uint64_t* end_ns);
+#endif
+
 // ---- launch accounting: every kernel launch of the library passes through count_launch() -------
 void count_launch();
 uint64_t launches_so_far();

@@ -152,3 +152,10 @@ def test_refill_tree_matches_oracle(trj):
     assert got.tolist()[:4] == trj.refill_window(chain, pred, 2, 4, [1, 2, 3], np.zeros(4, np.int64)).tolist()
     with pytest.raises(trj.TrjError):
         trj.refill_tree([-1, 0], [0, 3], np.zeros((2, 2), np.int32), 0, [1], [0])       # rank 3 with K = 2
+
+
+def test_default_build_has_no_clock_stamps(trj):
+    """The timeline entry points exist in every build but only the -DTRJ_TIMELINE build records anything."""
+    with pytest.raises(trj.TrjError) as e:
+        trj.timeline_read(4)
+    assert e.value.status == 5
