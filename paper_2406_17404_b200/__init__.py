@@ -88,6 +88,7 @@ _SIGNATURES = {
     "trj_gemm": (_I, [_VP, _VP, _VP, _I, _I, _I, _I, _VP, _SZ, _VP]),
     "trj_device_status": (_I, [_VP, _I, _VP]),
     "trj_selftest_wait_expiry": (_I, [_VP, _I, _VP]),
+    "trj_debug_flags": (_I, [_I32P]),
     "trj_timeline_reset": (_I, [_VP]),
     "trj_timeline_read": (_I, [_I, _I, _U64P, _U64P, _I32P]),
     "trj_launch_count": (C.c_uint64, []),
@@ -105,6 +106,13 @@ def use_library(path: str) -> None:
     if _lib is not None:
         raise RuntimeError("a library is already loaded")
     LIB_PATH = path
+
+
+def debug_flags() -> int:
+    """trj_debug_flags (debug build only): index-check bits seen since the last call."""
+    f = C.c_int32(0)
+    _check(lib().trj_debug_flags(C.byref(f)))
+    return int(f.value)
 
 
 TL_KINDS = ("rmsnorm", "gemm", "rope_kv", "attention", "swiglu", "embed")

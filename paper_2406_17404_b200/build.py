@@ -36,14 +36,16 @@ def _stale(target: str, deps) -> bool:
     return any(os.path.getmtime(d) > t for d in deps)
 
 
-def build(verbose: bool = False, force: bool = False, timeline: bool = False) -> str:
+def build(verbose: bool = False, force: bool = False, timeline: bool = False, debug: bool = False) -> str:
     """Compile every source under csrc/ and link libtrj.so; returns its path.  ``timeline=True`` builds a second
-    library, libtrj_timeline.so, with -DTRJ_TIMELINE (clock stamps in the per-layer kernels; measurement only)."""
+    library, libtrj_timeline.so, with -DTRJ_TIMELINE (clock stamps in the per-layer kernels; measurement only);
+    ``debug=True`` builds libtrj_debug.so with -DTRJ_DEBUG (index checks in the kernels that address the cache)."""
     global OBJ, LIB
-    if timeline:
+    if timeline or debug:
+        tag = "timeline" if timeline else "debug"
         saved = OBJ, LIB, list(NVCC_FLAGS)
-        OBJ, LIB = os.path.join(HERE, "_build_timeline"), os.path.join(HERE, "libtrj_timeline.so")
-        NVCC_FLAGS.append("-DTRJ_TIMELINE")
+        OBJ, LIB = os.path.join(HERE, "_build_" + tag), os.path.join(HERE, "libtrj_%s.so" % tag)
+        NVCC_FLAGS.append("-DTRJ_TIMELINE" if timeline else "-DTRJ_DEBUG")
         try:
             return build(verbose, force)
         finally:
@@ -81,4 +83,5 @@ def build(verbose: bool = False, force: bool = False, timeline: bool = False) ->
 
 
 if __name__ == "__main__":
-    print(build(verbose="-v" in sys.argv, force="-f" in sys.argv, timeline="--timeline" in sys.argv))
+    print(build(verbose="-v" in sys.argv, force="-f" in sys.argv, timeline="--timeline" in sys.argv,
+                debug="--debug" in sys.argv))

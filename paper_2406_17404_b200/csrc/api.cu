@@ -500,6 +500,19 @@ extern "C" trj_status trj_selftest_wait_expiry(int32_t* status, int32_t polls, v
     return TRJ_OK;
 }
 
+extern "C" trj_status trj_debug_flags(int32_t* flags) {
+#ifdef TRJ_DEBUG
+    TRJ_REQUIRE(flags, TRJ_EINVAL, "debug_flags: null pointer");
+    int f = 0;
+    TRJ_CHECK_CUDA(debug_flags_read(&f));
+    *flags = f;
+    return TRJ_OK;
+#else
+    (void)flags;
+    return fail(TRJ_EUNSUPPORTED, "debug_flags: this library was built without -DTRJ_DEBUG");
+#endif
+}
+
 extern "C" trj_status trj_timeline_reset(void* stream) {
 #ifdef TRJ_TIMELINE
     cudaStream_t st = (cudaStream_t)stream;

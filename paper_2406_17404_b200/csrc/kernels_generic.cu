@@ -10,6 +10,17 @@
 namespace trj {
 namespace {
 
+// Index checks of the debug build (-DTRJ_DEBUG): a cache row index that a device-held length or path would push
+// outside the cache sets a bit in a flag word and the access is skipped; nothing traps.  The default build trusts
+// the caller's contract (seq_len[b] + rows <= max_seq) and carries none of this.
+#ifdef TRJ_DEBUG
+static __device__ int g_debug_flags;
+#define TRJ_DEBUG_CHECK(ok, bit) ((ok) ? true : (atomicOr(&g_debug_flags, (bit)), false))
+#else
+#define TRJ_DEBUG_CHECK(ok, bit) (true)
+#endif
+enum { DBG_ROPE_ROW = 1, DBG_COMPACT_ROW = 2, DBG_ATTENTION_LEN = 4 };
+
 template <typename T> __device__ __forceinline__ float to_f(T v);
 template <> __device__ __forceinline__ float to_f<float>(float v) { return v; }
 template <> __device__ __forceinline__ float to_f<__nv_bfloat16>(__nv_bfloat16 v) { return __bfloat162float(v); }
@@ -277,7 +288,7 @@ __global__ void rope_kv_write_kernel(const Parts qkv, const double* __restrict__
         }
         q_out[(size_t)row * HD + hh * D + i] = from_f<T>(qa * cs - qb * sn);
         q_out[(size_t)row * HD + hh * D + i + half] = from_f<T>(qb * cs + qa * sn);
-        if (!has_kv) continue;
+        if (!has_kv || !TRJ_DEBUG_CHECK(seq_len[b] + local < max_seq, DBG_ROPE_ROW)) continue;
         k_slab[cache_row + i] = from_f<T>(ka * cs - kb * sn);
         k_slab[cache_row + i + half] = from_f<T>(kb * cs + ka * sn);
         v_slab[cache_row + i] = from_f<T>(va);
@@ -350,7 +361,7 @@ __global__ void __launch_bounds__(ROPE_THREADS) rope_kv_write_vec_kernel(const P
     };
     store_split4<T>(q_out, nullptr, q_at, rot_lo(acc[0], acc[1]));
     store_split4<T>(q_out, nullptr, q_at + half, rot_hi(acc[0], acc[1]));
-    if (has_kv) {
+    if (has_kv && TRJ_DEBUG_CHECK(seq_len[b] + local < max_seq, DBG_ROPE_ROW)) {
         store_split4<T>(k_slab, nullptr, cache_at, rot_lo(acc[2], acc[3]));
         store_split4<T>(k_slab, nullptr, cache_at + half, rot_hi(acc[2], acc[3]));
         store_split4<T>(v_slab, nullptr, cache_at, acc[4]);
@@ -375,7 +386,7 @@ __global__ void __launch_bounds__(128) tree_attention_generic_kernel(
     const int b = seq_of_row(row_off, B, row);
     const int S = seq_len[b];
     const int rows_b = row_off[b + 1] - row_off[b];
-    const int total = S + rows_b;
+    const int total = TRJ_DEBUG_CHECK(S + rows_b <= max_seq, DBG_ATTENTION_LEN) ? S + rows_b : min(S + rows_b, max_seq);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int kvh = hh / (H / Hkv);              // grouped-query attention: the K/V head of this query head
     const T* kb = k_slab + ((size_t)b * Hkv + kvh) * max_seq * D;
@@ -740,12 +751,14 @@ __global__ void __launch_bounds__(256) compact_kernel(uint4* __restrict__ k_cach
         const int nj = min(COMPACT_BATCH, k - j0 + 1);
         for (int e = threadIdx.x; e < nj * row_vec; e += blockDim.x) {
             const int j = j0 + e / row_vec, c = e % row_vec;
-            stage[e] = slab[(size_t)(S + pb[j]) * row_vec + c];
+            if (TRJ_DEBUG_CHECK(pb[j] >= 0 && S + pb[j] < max_seq, DBG_COMPACT_ROW))
+                stage[e] = slab[(size_t)(S + pb[j]) * row_vec + c];
         }
         __syncthreads();
         for (int e = threadIdx.x; e < nj * row_vec; e += blockDim.x) {
             const int j = j0 + e / row_vec, c = e % row_vec;
-            slab[(size_t)(S + j) * row_vec + c] = stage[e];
+            if (TRJ_DEBUG_CHECK(pb[j] >= 0 && S + pb[j] < max_seq && S + j < max_seq, DBG_COMPACT_ROW))
+                slab[(size_t)(S + j) * row_vec + c] = stage[e];
         }
         __syncthreads();
     }
@@ -776,6 +789,15 @@ static thread_local int t_chain_depth = 0;
 bool chain_active() { return t_chain_depth > 0 && pdl_enabled(); }
 ChainScope::ChainScope() { ++t_chain_depth; }
 ChainScope::~ChainScope() { --t_chain_depth; }
+#ifdef TRJ_DEBUG
+cudaError_t debug_flags_read(int* flags) {
+    cudaError_t e = cudaDeviceSynchronize();
+    if (e == cudaSuccess) e = cudaMemcpyFromSymbol(flags, g_debug_flags, sizeof(int));
+    const int zero = 0;
+    if (e == cudaSuccess) e = cudaMemcpyToSymbol(g_debug_flags, &zero, sizeof(int));
+    return e;
+}
+#endif
 #ifdef TRJ_TIMELINE
 cudaError_t timeline_reset_generic(cudaStream_t st) { return tl::reset(st); }
 int timeline_read_generic(int kind, int max_launches, uint64_t* b, uint64_t* e) { return tl::read(kind, max_launches, b, e); }

@@ -77,6 +77,10 @@ int timeline_read_gemm(int kind, int max_launches, uint64_t* begin_ns, uint64_t*
 int timeline_read_attention(int kind, int max_launches, uint64_t* begin_ns, uint64_t* end_ns);
 #endif
 
+#ifdef TRJ_DEBUG
+cudaError_t debug_flags_read(int* flags);      // synchronises the device, returns and clears the index-check flags
+#endif
+
 // ---- launch accounting: every kernel launch of the library passes through count_launch() -------
 void count_launch();
 uint64_t launches_so_far();
