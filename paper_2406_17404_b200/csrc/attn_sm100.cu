@@ -15,6 +15,7 @@
 // otherwise it leaves (max, sum, O) in the workspace and a second kernel merges the pieces in a fixed
 // order.  Every wait on an mbarrier is bounded; on expiry the CTA records TRJ_ETIMEOUT and leaves.
 #include <cuda.h>
+#include <cstdlib>
 #include <mutex>
 #include "trj_internal.h"
 #include "sm100_common.cuh"
@@ -801,6 +802,7 @@ bool at_make_map(CUtensorMap* map, const void* base_ptr, size_t rows, size_t col
 
 constexpr int AT_MAX_GRID = 148;
 constexpr int AT_WHOLE_HEAD_TILES = 8;      // up to 1024 keys: heads are handled one by one when B == 1
+constexpr int AT_CLUSTER_MAX_TILES_DEFAULT = 1 << 20;
 
 // How many CTAs may share a head (as one thread-block cluster) when every head is handled on its own: the largest
 // of 4 and 2 for which all H clusters are resident at once, else 1.  Asked of the driver once per head count.
@@ -828,6 +830,19 @@ int at_cluster_size(int H) {
     return pick;
 }
 
+// Longest prefix (in key tiles) that is still given to clusters.  H clusters of 4 use 4 * H CTAs (128 of the 148 SMs
+// for 32 heads) and need no merge kernel; the contiguous-range shape uses every SM but pays for a second kernel and
+// for the pieces' round trip through memory, which only a long prefix repays.  TRJ_AT_CLUSTER_MAX_TILES overrides
+// the default (a tuning knob, read once).
+int at_cluster_max_tiles() {
+    static const int value = [] {
+        const char* e = getenv("TRJ_AT_CLUSTER_MAX_TILES");
+        const int v = e ? atoi(e) : 0;
+        return v > 0 ? v : AT_CLUSTER_MAX_TILES_DEFAULT;
+    }();
+    return value;
+}
+
 // Launch shape.  The host only knows an upper bound of the key count; CTAs whose range turns out empty do no work.
 struct AtPlan { int grid, cluster; bool merge_kernel; int split; };   // split: threads per query row in the softmax
 AtPlan at_plan(int32_t B, int32_t H, int32_t max_len) {
@@ -838,7 +853,7 @@ AtPlan at_plan(int32_t B, int32_t H, int32_t max_len) {
     // Where clusters do not fit, one CTA takes a whole head of up to AT_WHOLE_HEAD_TILES tiles.
     if (B == 1 && H <= AT_MAX_GRID) {
         const int c = tiles_bound >= 2 ? at_cluster_size(H) : 1;
-        if (c > 1 || tiles_bound <= AT_WHOLE_HEAD_TILES) return AtPlan{H * c, c, false, 2};
+        if ((c > 1 && tiles_bound <= at_cluster_max_tiles()) || tiles_bound <= AT_WHOLE_HEAD_TILES) return AtPlan{H * c, c, false, 2};
     }
     // contiguous ranges + merge kernel; batches of small trees leave row groups empty, so four threads share a row
     return AtPlan{(int)(units_bound < AT_MAX_GRID ? units_bound : AT_MAX_GRID), 1, true, B > 1 ? 4 : 2};

@@ -625,6 +625,23 @@ struct TopList {
         v[KMAX - 1] = -INFINITY; id[KMAX - 1] = 0x7fffffff;
     }
 };
+// Two entries (arg-max plus the runner-up that the margin needs): the same list without a branch, because this is
+// the arg-max of every verification step and 32 lanes that branch differently on every element cost more than the
+// selects do.
+template <>
+struct TopList<2> {
+    float v[2]; int id[2];
+    __device__ __forceinline__ void clear() { v[0] = v[1] = -INFINITY; id[0] = id[1] = 0x7fffffff; }
+    __device__ __forceinline__ void push(float x, int i) {
+        const bool b0 = x > v[0] || (x == v[0] && i < id[0]);
+        const bool b1 = x > v[1] || (x == v[1] && i < id[1]);
+        v[1] = b0 ? v[0] : (b1 ? x : v[1]);
+        id[1] = b0 ? id[0] : (b1 ? i : id[1]);
+        v[0] = b0 ? x : v[0];
+        id[0] = b0 ? i : id[0];
+    }
+    __device__ __forceinline__ void pop() { v[0] = v[1]; id[0] = id[1]; v[1] = -INFINITY; id[1] = 0x7fffffff; }
+};
 // KMAX rounds: the best head of the warp's 32 lists is taken out (ids are unique, so exactly one lane pops) and
 // handed to lane `round`; afterwards lane r < KMAX holds the warp's r-th best entry.
 template <int KMAX>
