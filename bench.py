@@ -272,7 +272,7 @@ def run_ops_only(args):
     peaks = measured_peaks()
     steps = max(args.steps, 5)
     out = {"ops_only": True}
-    if args.case in ("", "cfg2", "cfg3", "cfg4", "cfg5"):
+    if args.case == "" or args.case.startswith("cfg"):       # "cfg" alone: every attention case
         out["tree_attention"] = bench_tree_attention(trj, torch, peaks, steps, 3, cpu=False, only=args.case)
     if args.case in ("", "small"):
         out["small_ops"] = bench_small_ops(trj, torch, peaks, steps, 3, cpu=False)
@@ -899,7 +899,7 @@ def main():
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-oracle baseline leg")
     ap.add_argument("--no-timeline", action="store_true", help="skip the clock-stamp leg (a child process with the -DTRJ_TIMELINE build)")
     ap.add_argument("--no-attention", action="store_true", help="skip the op-level tree-attention leg")
-    ap.add_argument("--case", default="", help="with --ops-only: cfg2 | cfg3 | cfg4 | cfg5 | small | gemm (default: all)")
+    ap.add_argument("--case", default="", help="with --ops-only: cfg | cfg2 | cfg3 | cfg4 | cfg5 | small | gemm (default: all)")
     ap.add_argument("--profile-step", action="store_true",
                     help="prefill + a few un-graphed verification steps and nothing else: a launch sequence for a profiler")
     ap.add_argument("--timeline", action="store_true",

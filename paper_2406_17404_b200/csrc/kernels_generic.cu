@@ -517,15 +517,32 @@ __device__ void accept_sequence(const int32_t* tokens, const int32_t* parent, co
         s_pred[i] = __ldcg(pred + i);            // possibly written by other CTAs of this launch: read it from L2
     }
     __syncthreads();
-    if (threadIdx.x == 0) {
-        ok[0] = 1;
-        int best = 0, best_depth = 0;
-        for (int i = 1; i < rows; ++i) {
-            const int p = s_par[i];
-            const unsigned char o = ok[p] && s_tok[i] == s_pred[p];
-            ok[i] = o;
-            if (o && s_dep[i] > best_depth) { best = i; best_depth = s_dep[i]; }
+    // ok[i] = every row on the path root..i carries the token its parent predicted.  Pointer jumping: after round r a
+    // row has folded in the matches of its 2^r nearest ancestors, so ceil(log2(rows)) rounds replace a serial walk
+    // over the rows (the walk was the longest single piece of this kernel).
+    __shared__ short jump[2][TRJ_MAX_ROWS];
+    __shared__ unsigned char okb[2][TRJ_MAX_ROWS];
+    for (int i = threadIdx.x; i < rows; i += blockDim.x) {
+        const int p = s_par[i];
+        okb[0][i] = i == 0 || s_tok[i] == s_pred[p];
+        jump[0][i] = (short)(i == 0 ? 0 : p);
+    }
+    __syncthreads();
+    int cur = 0;
+    for (int span = 1; span < rows; span <<= 1, cur ^= 1) {
+        for (int i = threadIdx.x; i < rows; i += blockDim.x) {
+            const int j = jump[cur][i];
+            okb[cur ^ 1][i] = okb[cur][i] && okb[cur][j];
+            jump[cur ^ 1][i] = jump[cur][j];
         }
+        __syncthreads();
+    }
+    for (int i = threadIdx.x; i < rows; i += blockDim.x) ok[i] = okb[cur][i];
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        int best = 0, best_depth = 0;
+        for (int i = 1; i < rows; ++i)
+            if (ok[i] && s_dep[i] > best_depth) { best = i; best_depth = s_dep[i]; }
         *k_acc = best_depth;
         *bonus = s_pred[best];
         int node = best;
