@@ -484,6 +484,12 @@ trj_status trj_timeline_read(int32_t kind, int32_t max_launches, uint64_t* begin
  * trj_set_pdl(0) launches them fully serialised instead (for comparison).  Process-wide; set it
  * before the first step of a context, because a cached CUDA graph keeps the mode it was captured in. */
 void       trj_set_pdl(int32_t on);
+/* Fused projections (on by default): in bf16 models with head_dim 128 and at most 64 rows per call, the QKV projection
+ * applies the rotary embedding and appends K/V itself and the gate/up projection applies SwiGLU itself (one kernel
+ * each instead of two; the K ranges of a weight tile are summed inside a thread-block cluster).  trj_set_fused(0)
+ * runs projection and consumer as separate kernels instead (for comparison).  Process-wide; set it before the first
+ * step of a context, because a cached CUDA graph keeps the mode it was captured in. */
+void       trj_set_fused(int32_t on);
 trj_status trj_profile_enable(trj_ctx* ctx, int32_t on);
 trj_status trj_profile_read(trj_ctx* ctx, float* ms, int32_t* launches, int32_t keep);
 

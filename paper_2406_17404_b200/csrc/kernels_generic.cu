@@ -626,8 +626,9 @@ struct TopList {
 #pragma unroll
         for (int i = 0; i < KMAX; ++i) { v[i] = -INFINITY; id[i] = 0x7fffffff; }
     }
-    __device__ __forceinline__ void push(float x, int i) {
-        if (!(x > v[KMAX - 1] || (x == v[KMAX - 1] && i < id[KMAX - 1]))) return;
+    // not inlined: the insertion is long, a thread calls it for a minority of its elements, and a kernel whose code
+    // does not fit the instruction cache pays for every launch with fetches from L2 or DRAM
+    __device__ __noinline__ void insert(float x, int i) {
 #pragma unroll
         for (int s = KMAX - 1; s >= 1; --s) {
             const bool above = x > v[s - 1] || (x == v[s - 1] && i < id[s - 1]);    // the new entry goes above slot s - 1
@@ -635,6 +636,9 @@ struct TopList {
             else { v[s] = x; id[s] = i; return; }
         }
         v[0] = x; id[0] = i;
+    }
+    __device__ __forceinline__ void push(float x, int i) {
+        if (x > v[KMAX - 1] || (x == v[KMAX - 1] && i < id[KMAX - 1])) insert(x, i);
     }
     __device__ __forceinline__ void pop() {
 #pragma unroll
@@ -696,9 +700,9 @@ __global__ void __launch_bounds__(TOPK_THREADS) topk_accept_kernel(
     t.clear();
     constexpr int VEC = 16 / (int)sizeof(T);                 // elements per 16-byte load
     if (V % VEC == 0 && ((uintptr_t)logits % 16) == 0) {
-        // eight 16-byte loads are requested before the first of them is looked at: the row comes from L2 or HBM and
+        // four 16-byte loads are requested before the first of them is looked at: the row comes from L2 or HBM and
         // a CTA has nothing else to hide that latency with
-        constexpr int BATCH = 8;
+        constexpr int BATCH = 4;
         for (int v0 = threadIdx.x * VEC; v0 < V; v0 += BATCH * TOPK_THREADS * VEC) {
             uint4 raw[BATCH];
 #pragma unroll
@@ -819,6 +823,9 @@ __global__ void bump_len_kernel(int32_t* seq_len_b, int delta) { *seq_len_b += d
 static std::atomic<bool> g_pdl{true};
 bool pdl_enabled() { return g_pdl.load(std::memory_order_relaxed); }
 void set_pdl(bool on) { g_pdl.store(on, std::memory_order_relaxed); }
+static std::atomic<bool> g_fused{true};
+bool fused_enabled() { return g_fused.load(std::memory_order_relaxed); }
+void set_fused(bool on) { g_fused.store(on, std::memory_order_relaxed); }
 static thread_local int t_chain_depth = 0;
 bool chain_active() { return t_chain_depth > 0 && pdl_enabled(); }
 ChainScope::ChainScope() { ++t_chain_depth; }
