@@ -549,6 +549,8 @@ def run_ours(args, rank, world, local_rank):
     trj.lib()
     if args.no_pdl:
         trj.set_pdl(False)
+    if args.no_fused:
+        trj.set_fused(False)
     peaks = measured_peaks()
     cfg = synth.LLAMA7B if not args.layers else synth.LLAMA7B.with_layers(args.layers)
     layers, glob = device_weights(cfg, 1234 + rank, dev)
@@ -827,6 +829,8 @@ def run_timeline(args):
     import paper_2406_17404_b200 as trj
     trj.use_library(trj_build.build(timeline=True))
     trj.lib()
+    if args.no_fused:
+        trj.set_fused(False)
     torch.cuda.set_device(0)
     dev = torch.device("cuda", 0)
     cfg = synth.LLAMA7B if not args.layers else synth.LLAMA7B.with_layers(args.layers)
@@ -882,6 +886,7 @@ def run_timeline(args):
             "per_kernel_us": {k: {"launches_per_step": len(dur[k]) // max(args.steps, 3), "release_to_end": mean(dur[k]),
                                   "gap_to_next_release": mean(gap[k])} for k in trj.TL_KINDS},
             "projection_ms_per_step": mean(proj), "first_release_to_last_end_ms": mean(span),
+            "projection_ctas_per_sm_peak": trj.timeline_ctas_per_sm(),
             "projection_bytes_per_step": gemm_bytes_per_step(cfg, TREE_ROWS),
             "projection_gbs": round(gemm_bytes_per_step(cfg, TREE_ROWS) / (float(np.mean(proj)) / 1e3) / 1e9, 1)}
     print(json.dumps(line), flush=True)
@@ -896,6 +901,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--layers", type=int, default=0, help="debug: fewer layers than the 7B shape (invalidates the number)")
     ap.add_argument("--no-pdl", action="store_true", help="launch the kernels fully serialised (comparison only)")
+    ap.add_argument("--no-fused", action="store_true", help="projection and rotary / SwiGLU as separate kernels (comparison only)")
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-oracle baseline leg")
     ap.add_argument("--no-timeline", action="store_true", help="skip the clock-stamp leg (a child process with the -DTRJ_TIMELINE build)")
     ap.add_argument("--no-attention", action="store_true", help="skip the op-level tree-attention leg")

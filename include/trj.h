@@ -478,6 +478,9 @@ uint64_t   trj_launch_count(void);
 #define TRJ_TL_EMBED     5   /* embedding gather               */
 #define TRJ_TL_KINDS     6
 trj_status trj_timeline_reset(void* stream);
+/* Most CTAs of the plain projection kernel that were ever resident on one SM at the same time since the library was
+ * loaded (clock-stamp build only; synchronise the device first): shows whether two CTAs really share an SM. */
+trj_status trj_timeline_ctas_per_sm(int32_t* peak);
 trj_status trj_timeline_read(int32_t kind, int32_t max_launches, uint64_t* begin_ns, uint64_t* end_ns, int32_t* n_launches);
 /* Programmatic dependent launch (on by default): the kernels of a step are launched so that each may
  * be scheduled, and may prefetch weights, while its predecessor in the stream is still running.

@@ -91,6 +91,7 @@ _SIGNATURES = {
     "trj_debug_flags": (_I, [_I32P]),
     "trj_timeline_reset": (_I, [_VP]),
     "trj_timeline_read": (_I, [_I, _I, _U64P, _U64P, _I32P]),
+    "trj_timeline_ctas_per_sm": (_I, [_I32P]),
     "trj_launch_count": (C.c_uint64, []),
     "trj_set_pdl": (None, [_I]),
     "trj_set_fused": (None, [_I]),
@@ -133,6 +134,13 @@ def timeline_read(max_launches: int = 512):
         _check(lib().trj_timeline_read(kind, max_launches, b.ctypes.data_as(_U64P), e.ctypes.data_as(_U64P), C.byref(n)))
         out[name] = (b[:n.value].copy(), e[:n.value].copy())
     return out
+
+
+def timeline_ctas_per_sm() -> int:
+    """trj_timeline_ctas_per_sm (clock-stamp build only)."""
+    v = C.c_int32(0)
+    _check(lib().trj_timeline_ctas_per_sm(C.byref(v)))
+    return int(v.value)
 
 
 def lib() -> C.CDLL:

@@ -532,6 +532,7 @@ extern "C" trj_status trj_timeline_reset(void* stream) {
     cudaStream_t st = (cudaStream_t)stream;
     TRJ_CHECK_CUDA(timeline_reset_generic(st));
     TRJ_CHECK_CUDA(timeline_reset_gemm(st));
+    TRJ_CHECK_CUDA(timeline_reset_fused(st));
     TRJ_CHECK_CUDA(timeline_reset_attention(st));
     return TRJ_OK;
 #else
@@ -540,10 +541,38 @@ extern "C" trj_status trj_timeline_reset(void* stream) {
 #endif
 }
 
+extern "C" trj_status trj_timeline_ctas_per_sm(int32_t* peak) {
+#ifdef TRJ_TIMELINE
+    TRJ_REQUIRE(peak, TRJ_EINVAL, "timeline_ctas_per_sm: null pointer");
+    const int v = std::max(timeline_gemm_ctas_per_sm(), timeline_fused_ctas_per_sm());
+    TRJ_REQUIRE(v >= 0, TRJ_ECUDA, "timeline_ctas_per_sm: copy from the device failed");
+    *peak = v;
+    return TRJ_OK;
+#else
+    (void)peak;
+    return fail(TRJ_EUNSUPPORTED, "timeline: this library was built without -DTRJ_TIMELINE");
+#endif
+}
+
 extern "C" trj_status trj_timeline_read(int32_t kind, int32_t max_launches, uint64_t* begin_ns, uint64_t* end_ns, int32_t* n_launches) {
 #ifdef TRJ_TIMELINE
     TRJ_REQUIRE(begin_ns && end_ns && n_launches && max_launches >= 0, TRJ_EINVAL, "timeline_read: null pointer");
     TRJ_REQUIRE(kind >= 0 && kind < TRJ_TL_KINDS, TRJ_EINVAL, "timeline_read: kind %d outside 0..%d", kind, TRJ_TL_KINDS - 1);
+    if (kind == TRJ_TL_GEMM) {
+        // plain and fused projections keep separate records: the launches of both, in launch order
+        std::vector<uint64_t> b1(max_launches), e1(max_launches), b2(max_launches), e2(max_launches);
+        const int n1 = timeline_read_gemm(kind, max_launches, b1.data(), e1.data());
+        const int n2 = timeline_read_fused(kind, max_launches, b2.data(), e2.data());
+        TRJ_REQUIRE(n1 >= 0 && n2 >= 0, TRJ_ECUDA, "timeline_read: copy from the device failed");
+        std::vector<std::pair<uint64_t, uint64_t>> all;
+        for (int i = 0; i < n1; ++i) all.push_back({b1[i], e1[i]});
+        for (int i = 0; i < n2; ++i) all.push_back({b2[i], e2[i]});
+        std::sort(all.begin(), all.end());
+        const int n_all = std::min<int>((int)all.size(), max_launches);
+        for (int i = 0; i < n_all; ++i) { begin_ns[i] = all[i].first; end_ns[i] = all[i].second; }
+        *n_launches = n_all;
+        return TRJ_OK;
+    }
     int n = kind == TRJ_TL_GEMM ? timeline_read_gemm(kind, max_launches, begin_ns, end_ns)
           : kind == TRJ_TL_ATTENTION ? timeline_read_attention(kind, max_launches, begin_ns, end_ns)
                                      : timeline_read_generic(kind, max_launches, begin_ns, end_ns);

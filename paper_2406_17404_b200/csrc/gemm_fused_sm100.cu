@@ -121,6 +121,7 @@ __global__ void __launch_bounds__(FU_THREADS, 2) gemm_fused_kernel(const __grid_
     const int cluster_id = (int)blockIdx.x / C, n_clusters = (int)gridDim.x / C;
     const int kb0 = (int)((long long)rank * p.kblocks / C), kb1 = (int)((long long)(rank + 1) * p.kblocks / C);
     TRJ_TL_DECL;
+    TRJ_TL_ENTER();
 
     pdl_launch_dependents();
     if (threadIdx.x == 32) {
@@ -308,6 +309,7 @@ __global__ void __launch_bounds__(FU_THREADS, 2) gemm_fused_kernel(const __grid_
     asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
     if (warp == 1) tmem_dealloc(tmem_base, (uint32_t)(2 * p.acc_cols));
     TRJ_TL_END(TRJ_TL_GEMM);
+    TRJ_TL_LEAVE();
 }
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
@@ -342,35 +344,17 @@ cudaError_t fu_attributes() {
     static cudaError_t attr_err = cudaSuccess;
     std::call_once(once, [] {
         attr_err = cudaFuncSetAttribute(gemm_fused_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 112 * 1024);
+        // two CTAs of ~100 KB share an SM only if the SM's L1/shared split gives shared memory its maximum
+        if (attr_err == cudaSuccess)
+            attr_err = cudaFuncSetAttribute(gemm_fused_kernel, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
     });
     return attr_err;
 }
 
-// Clusters of `c` CTAs with `smem` bytes each that the device keeps resident at once (asked of the driver once per
-// size; whole clusters have to fit a GPC, so this is less than the CTA slots divided by c).
-int fu_max_clusters(int c, size_t smem) {
-    static std::mutex mu;
-    static int cached[FU_MAX_CLUSTER + 1] = {};
-    static size_t cached_smem[FU_MAX_CLUSTER + 1] = {};
-    std::lock_guard<std::mutex> lock(mu);
-    if (cached[c] > 0 && cached_smem[c] == smem) return cached[c];
-    int n = 0;
-    if (fu_attributes() == cudaSuccess) {
-        cudaLaunchConfig_t cfg = {};
-        cfg.gridDim = dim3(FU_CTAS / c * c); cfg.blockDim = dim3(FU_THREADS); cfg.dynamicSmemBytes = smem;
-        cudaLaunchAttribute attr[1];
-        attr[0].id = cudaLaunchAttributeClusterDimension;
-        attr[0].val.clusterDim.x = c; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
-        cfg.attrs = attr; cfg.numAttrs = 1;
-        if (cudaOccupancyMaxActiveClusters(&n, gemm_fused_kernel, &cfg) != cudaSuccess) n = 0;
-    }
-    (void)cudaGetLastError();
-    cached[c] = n > 0 ? n : -1; cached_smem[c] = smem;
-    return cached[c];
-}
-
-// Cluster size = number of K ranges: the one whose resident clusters are kept busiest over whole rounds of tiles and
-// cover most of the device, smaller on near ties; every range must keep at least four k-blocks.
+// Cluster size = number of K ranges: the one that keeps the 296 CTA slots (two per SM) busiest over whole rounds of
+// tiles, smaller on near ties; every range must keep at least four k-blocks.  (The occupancy calculator is of no help
+// here: it reports one CTA per SM for every kernel that allocates tensor memory, whereas two are resident in fact —
+// the clock-stamp build counts them.)
 struct FuPlan { bool ok; int cluster, clusters, stages, m_pad, n_mma, acc_cols; size_t smem; };
 FuPlan fu_plan(int M, int tiles, int K) {
     FuPlan pl{};
@@ -386,13 +370,11 @@ FuPlan fu_plan(int M, int tiles, int K) {
     pl.smem = pl.stages * stage + staging + 1024;
     double best = 0.0;
     for (int c = 2; c <= FU_MAX_CLUSTER && c * 4 <= kblocks; ++c) {
-        const int resident = fu_max_clusters(c, pl.smem);
-        if (resident <= 0) continue;
-        const int clusters = std::min(std::min(resident, FU_CTAS / c), tiles), rounds = (tiles + clusters - 1) / clusters;
+        const int clusters = std::min(FU_CTAS / c, tiles), rounds = (tiles + clusters - 1) / clusters;
         const double balance = (double)tiles * c / ((double)rounds * FU_CTAS);     // busy CTA slots over the kernel's span
         if (balance > best * 1.02) { best = balance; pl.cluster = c; pl.clusters = clusters; }
     }
-    pl.ok = pl.cluster >= 2 && best >= 0.75;
+    pl.ok = pl.cluster >= 2 && best >= 0.8;
     return pl;
 }
 
@@ -432,6 +414,12 @@ void fu_common(FuParams& p, const FuPlan& pl, int mode, int M, int N, int K, int
 bool fu_aligned(const void* a, const void* b, const void* c) { return (((uintptr_t)a | (uintptr_t)b | (uintptr_t)c) % 16) == 0; }
 
 }  // namespace
+
+#ifdef TRJ_TIMELINE
+cudaError_t timeline_reset_fused(cudaStream_t st) { return tl::reset(st); }
+int timeline_read_fused(int kind, int max_launches, uint64_t* b, uint64_t* e) { return tl::read(kind, max_launches, b, e); }
+int timeline_fused_ctas_per_sm() { return tl::sm_peak(); }
+#endif
 
 bool gemm_rope_fused_supported(int32_t M, int32_t H, int32_t Hkv, int32_t D, int32_t K, int32_t dtype) {
     return dtype == TRJ_BF16 && D == FU_BM && fu_encode_fn() != nullptr && fu_plan(M, H + 2 * Hkv, K).ok;

@@ -71,6 +71,7 @@ __global__ void __launch_bounds__(TC_THREADS, 2) gemm_tc_kernel(const __grid_con
     const int per_tile = p.splits * p.m_blocks;              // items of one weight tile: block index fastest
     const int items = p.tiles * per_tile;
     TRJ_TL_DECL;
+    TRJ_TL_ENTER();
 
     pdl_launch_dependents();
     if (threadIdx.x == 32) {                                 // have the tensor maps on their way before the first copy needs them
@@ -220,6 +221,7 @@ __global__ void __launch_bounds__(TC_THREADS, 2) gemm_tc_kernel(const __grid_con
     if (warp == 1)
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)(2 * p.acc_cols)) : "memory");
     TRJ_TL_END(TRJ_TL_GEMM);
+    TRJ_TL_LEAVE();
 }
 
 // y[i] = sum_s part[s][i], fixed order.
@@ -410,6 +412,7 @@ cudaError_t launch_gemm_tc(const void* x, const void* x_lo, const void* w, float
 #ifdef TRJ_TIMELINE
 cudaError_t timeline_reset_gemm(cudaStream_t st) { return tl::reset(st); }
 int timeline_read_gemm(int kind, int max_launches, uint64_t* b, uint64_t* e) { return tl::read(kind, max_launches, b, e); }
+int timeline_gemm_ctas_per_sm() { return tl::sm_peak(); }
 #endif
 
 cudaError_t launch_wait_expiry_selftest(int* status, uint32_t polls, cudaStream_t st) {

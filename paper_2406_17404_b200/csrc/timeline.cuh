@@ -14,11 +14,26 @@ constexpr int SLOTS = 512;        // launches of one kind between two resets
 struct Rec { unsigned long long begin_inv, end; unsigned int done, pad; };   // begin_inv = ~(earliest release): zero = none yet
 static __device__ Rec g_rec[KINDS][SLOTS];
 static __device__ unsigned int g_count[KINDS];
+static __device__ int g_sm_now[256];      // CTAs of this translation unit's projection kernels resident on each SM right now
+static __device__ int g_sm_peak;          // ... and the most that were ever resident on one SM at the same time
 
 __device__ __forceinline__ unsigned long long now() {
     unsigned long long t;
     asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
     return t;
+}
+// First and last thing a CTA does (one thread): how many CTAs of the kernel share an SM.
+__device__ __forceinline__ unsigned int smid() {
+    unsigned int s;
+    asm volatile("mov.u32 %0, %%smid;" : "=r"(s));
+    return s;
+}
+__device__ __forceinline__ void enter() { atomicMax(&g_sm_peak, atomicAdd(&g_sm_now[smid() & 255u], 1) + 1); }
+__device__ __forceinline__ void leave() { atomicSub(&g_sm_now[smid() & 255u], 1); }
+inline int sm_peak() {
+    int v = -1;
+    if (cudaMemcpyFromSymbol(&v, g_sm_peak, sizeof(int)) != cudaSuccess) return -1;
+    return v;
 }
 // One thread per CTA, right after the CTA's wait for the previous kernel.
 __device__ __forceinline__ unsigned int begin(int kind) {
@@ -56,10 +71,14 @@ inline int read(int kind, int max_launches, uint64_t* begin_ns, uint64_t* end_ns
 
 }  // namespace tl
 }  // namespace trj
+#define TRJ_TL_ENTER() do { if (threadIdx.x == 0) ::trj::tl::enter(); } while (0)
+#define TRJ_TL_LEAVE() do { if (threadIdx.x == 0) ::trj::tl::leave(); } while (0)
 #define TRJ_TL_DECL unsigned int tl_slot__ = 0
 #define TRJ_TL_BEGIN(kind) do { if (threadIdx.x == 0) tl_slot__ = ::trj::tl::begin(kind); } while (0)
 #define TRJ_TL_END(kind) do { if (threadIdx.x == 0) ::trj::tl::end(kind, tl_slot__); } while (0)
 #else
+#define TRJ_TL_ENTER()
+#define TRJ_TL_LEAVE()
 #define TRJ_TL_DECL
 #define TRJ_TL_BEGIN(kind)
 #define TRJ_TL_END(kind)

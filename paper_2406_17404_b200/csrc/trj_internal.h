@@ -74,6 +74,10 @@ cudaError_t timeline_reset_gemm(cudaStream_t st);
 cudaError_t timeline_reset_attention(cudaStream_t st);
 int timeline_read_generic(int kind, int max_launches, uint64_t* begin_ns, uint64_t* end_ns);
 int timeline_read_gemm(int kind, int max_launches, uint64_t* begin_ns, uint64_t* end_ns);
+cudaError_t timeline_reset_fused(cudaStream_t st);
+int timeline_read_fused(int kind, int max_launches, uint64_t* begin_ns, uint64_t* end_ns);
+int timeline_fused_ctas_per_sm();
+int timeline_gemm_ctas_per_sm();          // most CTAs of the plain projection kernel ever resident on one SM
 int timeline_read_attention(int kind, int max_launches, uint64_t* begin_ns, uint64_t* end_ns);
 #endif
 
