@@ -549,8 +549,6 @@ def run_ours(args, rank, world, local_rank):
     trj.lib()
     if args.no_pdl:
         trj.set_pdl(False)
-    if args.no_fused:
-        trj.set_fused(False)
     peaks = measured_peaks()
     cfg = synth.LLAMA7B if not args.layers else synth.LLAMA7B.with_layers(args.layers)
     layers, glob = device_weights(cfg, 1234 + rank, dev)
@@ -829,8 +827,6 @@ def run_timeline(args):
     import paper_2406_17404_b200 as trj
     trj.use_library(trj_build.build(timeline=True))
     trj.lib()
-    if args.no_fused:
-        trj.set_fused(False)
     torch.cuda.set_device(0)
     dev = torch.device("cuda", 0)
     cfg = synth.LLAMA7B if not args.layers else synth.LLAMA7B.with_layers(args.layers)
@@ -869,7 +865,7 @@ def run_timeline(args):
     torch.cuda.synchronize()
     dur = {k: [] for k in trj.TL_KINDS}
     gap = {k: [] for k in trj.TL_KINDS}
-    span, proj = [], []
+    span, proj, by_proj = [], [], {}
     for _ in range(max(args.steps, 3)):
         graph.replay()
         torch.cuda.synchronize()
@@ -879,12 +875,18 @@ def run_timeline(args):
             dur[k].append((e - b) / 1e3)
             if i + 1 < len(events):
                 gap[k].append((events[i + 1][0] - e) / 1e3)
+        gemms = [(e - b) / 1e3 for b, e, k in events if k == "gemm"]
+        if len(gemms) == 4 * cfg.n_layers + 1:               # QKV, output, gate/up, down per layer, then the LM head
+            for i, name in enumerate(("qkv", "o", "gate_up", "down")):
+                by_proj.setdefault(name, []).extend(gemms[i:-1:4])
+            by_proj.setdefault("lm_head", []).append(gemms[-1])
         span.append((max(e for _, e, _ in events) - min(b for b, _, _ in events)) / 1e6)
         proj.append(sum(e - b for b, e, k in events if k == "gemm") / 1e6)
     mean = lambda v: round(float(np.mean(v)), 3) if v else None
     line = {"timeline": True, "layers": cfg.n_layers, "tree_rows": TREE_ROWS, "prefix": PROMPT,
             "per_kernel_us": {k: {"launches_per_step": len(dur[k]) // max(args.steps, 3), "release_to_end": mean(dur[k]),
                                   "gap_to_next_release": mean(gap[k])} for k in trj.TL_KINDS},
+            "projection_us_by_kind": {k: mean(v) for k, v in by_proj.items()},
             "projection_ms_per_step": mean(proj), "first_release_to_last_end_ms": mean(span),
             "projection_ctas_per_sm_peak": trj.timeline_ctas_per_sm(),
             "projection_bytes_per_step": gemm_bytes_per_step(cfg, TREE_ROWS),
@@ -901,7 +903,6 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--layers", type=int, default=0, help="debug: fewer layers than the 7B shape (invalidates the number)")
     ap.add_argument("--no-pdl", action="store_true", help="launch the kernels fully serialised (comparison only)")
-    ap.add_argument("--no-fused", action="store_true", help="projection and rotary / SwiGLU as separate kernels (comparison only)")
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-oracle baseline leg")
     ap.add_argument("--no-timeline", action="store_true", help="skip the clock-stamp leg (a child process with the -DTRJ_TIMELINE build)")
     ap.add_argument("--no-attention", action="store_true", help="skip the op-level tree-attention leg")

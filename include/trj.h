@@ -478,8 +478,9 @@ uint64_t   trj_launch_count(void);
 #define TRJ_TL_EMBED     5   /* embedding gather               */
 #define TRJ_TL_KINDS     6
 trj_status trj_timeline_reset(void* stream);
-/* Most CTAs of the plain projection kernel that were ever resident on one SM at the same time since the library was
- * loaded (clock-stamp build only; synchronise the device first): shows whether two CTAs really share an SM. */
+/* Most CTAs of the projection kernel that were ever resident on one SM at the same time since the library was loaded
+ * (clock-stamp build only; synchronise the device first): shows that two CTAs really share an SM, which the occupancy
+ * calculator denies for a kernel that allocates tensor memory. */
 trj_status trj_timeline_ctas_per_sm(int32_t* peak);
 trj_status trj_timeline_read(int32_t kind, int32_t max_launches, uint64_t* begin_ns, uint64_t* end_ns, int32_t* n_launches);
 /* Programmatic dependent launch (on by default): the kernels of a step are launched so that each may
@@ -487,12 +488,6 @@ trj_status trj_timeline_read(int32_t kind, int32_t max_launches, uint64_t* begin
  * trj_set_pdl(0) launches them fully serialised instead (for comparison).  Process-wide; set it
  * before the first step of a context, because a cached CUDA graph keeps the mode it was captured in. */
 void       trj_set_pdl(int32_t on);
-/* Fused projections (on by default): in bf16 models with head_dim 128 and at most 64 rows per call, the QKV projection
- * applies the rotary embedding and appends K/V itself and the gate/up projection applies SwiGLU itself (one kernel
- * each instead of two; the K ranges of a weight tile are summed inside a thread-block cluster).  trj_set_fused(0)
- * runs projection and consumer as separate kernels instead (for comparison).  Process-wide; set it before the first
- * step of a context, because a cached CUDA graph keeps the mode it was captured in. */
-void       trj_set_fused(int32_t on);
 trj_status trj_profile_enable(trj_ctx* ctx, int32_t on);
 trj_status trj_profile_read(trj_ctx* ctx, float* ms, int32_t* launches, int32_t keep);
 

@@ -94,7 +94,6 @@ _SIGNATURES = {
     "trj_timeline_ctas_per_sm": (_I, [_I32P]),
     "trj_launch_count": (C.c_uint64, []),
     "trj_set_pdl": (None, [_I]),
-    "trj_set_fused": (None, [_I]),
     "trj_profile_enable": (_I, [_VP, _I]),
     "trj_profile_read": (_I, [_VP, C.POINTER(C.c_float), _I32P, _I]),
 }
@@ -170,11 +169,6 @@ def version() -> str:
 def set_pdl(on: bool) -> None:
     """trj_set_pdl: programmatic dependent launch of the step's kernels on (default) or off."""
     lib().trj_set_pdl(1 if on else 0)
-
-
-def set_fused(on: bool) -> None:
-    """trj_set_fused: projections with rotary embedding / SwiGLU folded in on (default) or off."""
-    lib().trj_set_fused(1 if on else 0)
 
 
 def launch_count() -> int:

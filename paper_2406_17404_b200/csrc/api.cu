@@ -330,10 +330,6 @@ trj_status forward(trj_ctx* ctx, void* k_cache, void* v_cache, int32_t b0, const
                          tree_attention_tc_supported(c.head_dim, c.dtype, bt.max_rows);
     const int attn_grid = attn_tc ? tree_attention_grid(bt.B, c.n_heads, bt.max_len) : ctx->sm_count;
     int* const gemm_status = ctx->dev_status, *const attn_status = ctx->dev_status + 1;
-    // the projections whose consumer is an element-wise map of a finished weight tile take the fused kernel when the
-    // shape allows it (few rows, bf16, head_dim 128); a fixed rule of the shape, not a fallback
-    const bool fuse_rope = fused_enabled() && ctx->x_lo && gemm_rope_fused_supported(M, c.n_heads, Hkv, c.head_dim, d, c.dtype);
-    const bool fuse_swiglu = fused_enabled() && ctx->x_lo && ctx->act_lo && gemm_swiglu_fused_supported(M, c.d_ff, d, c.dtype);
     constexpr size_t AHEAD_BYTES = (size_t)32 << 20;         // measured optimum on the 7B shape (16-40 MB are close)
     LAUNCH(PROF_ELEMENTWISE, launch_embed(ctx->embed, c.dtype, tokens, ctx->h, M, d, st));
     Parts pr{nullptr, 1, 0};                 // result of the latest projection, possibly in split-K pieces
@@ -342,15 +338,10 @@ trj_status forward(trj_ctx* ctx, void* k_cache, void* v_cache, int32_t b0, const
         char* v_slab = (char*)v_cache + ((size_t)l * c.max_batch + b0) * seq_stride;
         LAUNCH(PROF_ELEMENTWISE, launch_add_rmsnorm(ctx->h, pr, ctx->attn_norm[l], ctx->x, ctx->x_lo, c.dtype, M, d,
                                                     c.rms_eps, st));
-        if (fuse_rope) {
-            LAUNCH(PROF_GEMM, launch_gemm_rope_fused(ctx->x, ctx->x_lo, ctx->wqkv[l], d, ctx->inv_freq, depth, bt, ctx->q, k_slab,
-                                                     v_slab, c.n_heads, Hkv, c.max_seq, gemm_status, st));
-        } else {
-            LAUNCH(PROF_GEMM, launch_gemm(ctx->x, ctx->x_lo, ctx->wqkv[l], ctx->y, M, QKV, d, c.dtype, ctx->gemm_ws,
-                                          ctx->gemm_ws_bytes, st, &pr, nullptr, gemm_status));
-            LAUNCH(PROF_ROPE, launch_rope_kv_write(pr, ctx->inv_freq, depth, bt, ctx->q, k_slab, v_slab, c.dtype,
-                                                   c.n_heads, Hkv, c.head_dim, c.max_seq, st));
-        }
+        LAUNCH(PROF_GEMM, launch_gemm(ctx->x, ctx->x_lo, ctx->wqkv[l], ctx->y, M, QKV, d, c.dtype, ctx->gemm_ws,
+                                      ctx->gemm_ws_bytes, st, &pr, nullptr, gemm_status));
+        LAUNCH(PROF_ROPE, launch_rope_kv_write(pr, ctx->inv_freq, depth, bt, ctx->q, k_slab, v_slab, c.dtype,
+                                               c.n_heads, Hkv, c.head_dim, c.max_seq, st));
         // inside the decoder the attention result reaches the output projection as a bf16 pair, like every
         // other projection input
         if (!pieces) {
@@ -376,14 +367,9 @@ trj_status forward(trj_ctx* ctx, void* k_cache, void* v_cache, int32_t b0, const
                                       ctx->gemm_ws_bytes, st, &pr, &ahead, gemm_status));
         LAUNCH(PROF_ELEMENTWISE, launch_add_rmsnorm(ctx->h, pr, ctx->mlp_norm[l], ctx->x, ctx->x_lo, c.dtype, M, d,
                                                     c.rms_eps, st));
-        if (fuse_swiglu) {
-            LAUNCH(PROF_GEMM, launch_gemm_swiglu_fused(ctx->x, ctx->x_lo, ctx->w_gate_up[l], M, c.d_ff, d, ctx->act, ctx->act_lo,
-                                                       gemm_status, st));
-        } else {
-            LAUNCH(PROF_GEMM, launch_gemm(ctx->x, ctx->x_lo, ctx->w_gate_up[l], ctx->y, M, 2 * c.d_ff, d, c.dtype, ctx->gemm_ws,
-                                          ctx->gemm_ws_bytes, st, &pr, nullptr, gemm_status));
-            LAUNCH(PROF_ELEMENTWISE, launch_swiglu(pr, ctx->act, ctx->act_lo, c.dtype, M, c.d_ff, st));
-        }
+        LAUNCH(PROF_GEMM, launch_gemm(ctx->x, ctx->x_lo, ctx->w_gate_up[l], ctx->y, M, 2 * c.d_ff, d, c.dtype, ctx->gemm_ws,
+                                      ctx->gemm_ws_bytes, st, &pr, nullptr, gemm_status));
+        LAUNCH(PROF_ELEMENTWISE, launch_swiglu(pr, ctx->act, ctx->act_lo, c.dtype, M, c.d_ff, st));
         LAUNCH(PROF_GEMM, launch_gemm(ctx->act, ctx->act_lo, ctx->w_down[l], ctx->y, M, d, c.d_ff, c.dtype, ctx->gemm_ws,
                                       ctx->gemm_ws_bytes, st, &pr, nullptr, gemm_status));
     }
@@ -532,7 +518,6 @@ extern "C" trj_status trj_timeline_reset(void* stream) {
     cudaStream_t st = (cudaStream_t)stream;
     TRJ_CHECK_CUDA(timeline_reset_generic(st));
     TRJ_CHECK_CUDA(timeline_reset_gemm(st));
-    TRJ_CHECK_CUDA(timeline_reset_fused(st));
     TRJ_CHECK_CUDA(timeline_reset_attention(st));
     return TRJ_OK;
 #else
@@ -544,7 +529,7 @@ extern "C" trj_status trj_timeline_reset(void* stream) {
 extern "C" trj_status trj_timeline_ctas_per_sm(int32_t* peak) {
 #ifdef TRJ_TIMELINE
     TRJ_REQUIRE(peak, TRJ_EINVAL, "timeline_ctas_per_sm: null pointer");
-    const int v = std::max(timeline_gemm_ctas_per_sm(), timeline_fused_ctas_per_sm());
+    const int v = timeline_gemm_ctas_per_sm();
     TRJ_REQUIRE(v >= 0, TRJ_ECUDA, "timeline_ctas_per_sm: copy from the device failed");
     *peak = v;
     return TRJ_OK;
@@ -558,21 +543,6 @@ extern "C" trj_status trj_timeline_read(int32_t kind, int32_t max_launches, uint
 #ifdef TRJ_TIMELINE
     TRJ_REQUIRE(begin_ns && end_ns && n_launches && max_launches >= 0, TRJ_EINVAL, "timeline_read: null pointer");
     TRJ_REQUIRE(kind >= 0 && kind < TRJ_TL_KINDS, TRJ_EINVAL, "timeline_read: kind %d outside 0..%d", kind, TRJ_TL_KINDS - 1);
-    if (kind == TRJ_TL_GEMM) {
-        // plain and fused projections keep separate records: the launches of both, in launch order
-        std::vector<uint64_t> b1(max_launches), e1(max_launches), b2(max_launches), e2(max_launches);
-        const int n1 = timeline_read_gemm(kind, max_launches, b1.data(), e1.data());
-        const int n2 = timeline_read_fused(kind, max_launches, b2.data(), e2.data());
-        TRJ_REQUIRE(n1 >= 0 && n2 >= 0, TRJ_ECUDA, "timeline_read: copy from the device failed");
-        std::vector<std::pair<uint64_t, uint64_t>> all;
-        for (int i = 0; i < n1; ++i) all.push_back({b1[i], e1[i]});
-        for (int i = 0; i < n2; ++i) all.push_back({b2[i], e2[i]});
-        std::sort(all.begin(), all.end());
-        const int n_all = std::min<int>((int)all.size(), max_launches);
-        for (int i = 0; i < n_all; ++i) { begin_ns[i] = all[i].first; end_ns[i] = all[i].second; }
-        *n_launches = n_all;
-        return TRJ_OK;
-    }
     int n = kind == TRJ_TL_GEMM ? timeline_read_gemm(kind, max_launches, begin_ns, end_ns)
           : kind == TRJ_TL_ATTENTION ? timeline_read_attention(kind, max_launches, begin_ns, end_ns)
                                      : timeline_read_generic(kind, max_launches, begin_ns, end_ns);
@@ -587,7 +557,6 @@ extern "C" trj_status trj_timeline_read(int32_t kind, int32_t max_launches, uint
 
 extern "C" uint64_t trj_launch_count(void) { return launches_so_far(); }
 extern "C" void trj_set_pdl(int32_t on) { set_pdl(on != 0); }
-extern "C" void trj_set_fused(int32_t on) { set_fused(on != 0); }
 
 extern "C" trj_status trj_profile_enable(trj_ctx* ctx, int32_t on) {
     TRJ_REQUIRE(ctx, TRJ_EINVAL, "profile_enable: null context");

@@ -823,9 +823,6 @@ __global__ void bump_len_kernel(int32_t* seq_len_b, int delta) { *seq_len_b += d
 static std::atomic<bool> g_pdl{true};
 bool pdl_enabled() { return g_pdl.load(std::memory_order_relaxed); }
 void set_pdl(bool on) { g_pdl.store(on, std::memory_order_relaxed); }
-static std::atomic<bool> g_fused{true};
-bool fused_enabled() { return g_fused.load(std::memory_order_relaxed); }
-void set_fused(bool on) { g_fused.store(on, std::memory_order_relaxed); }
 static thread_local int t_chain_depth = 0;
 bool chain_active() { return t_chain_depth > 0 && pdl_enabled(); }
 ChainScope::ChainScope() { ++t_chain_depth; }

@@ -74,9 +74,6 @@ cudaError_t timeline_reset_gemm(cudaStream_t st);
 cudaError_t timeline_reset_attention(cudaStream_t st);
 int timeline_read_generic(int kind, int max_launches, uint64_t* begin_ns, uint64_t* end_ns);
 int timeline_read_gemm(int kind, int max_launches, uint64_t* begin_ns, uint64_t* end_ns);
-cudaError_t timeline_reset_fused(cudaStream_t st);
-int timeline_read_fused(int kind, int max_launches, uint64_t* begin_ns, uint64_t* end_ns);
-int timeline_fused_ctas_per_sm();
 int timeline_gemm_ctas_per_sm();          // most CTAs of the plain projection kernel ever resident on one SM
 int timeline_read_attention(int kind, int max_launches, uint64_t* begin_ns, uint64_t* end_ns);
 #endif
@@ -138,20 +135,6 @@ bool gemm_tc_shape(int32_t M, int32_t N, int32_t K, int32_t dtype);
 cudaError_t launch_gemm(const void* x, const void* x_lo, const void* w, float* y, int32_t M, int32_t N, int32_t K,
                         int32_t dtype, void* workspace, size_t workspace_bytes, cudaStream_t st, Parts* parts = nullptr,
                         const WeightPrefetch* ahead = nullptr, int* status = nullptr);
-
-// Projections with their consumer folded in (gemm_fused_sm100.cu): the K ranges of a weight tile are the CTAs of a
-// thread-block cluster, which add their partial sums through distributed shared memory and apply the consumer to the
-// finished tile.  bf16 models, at most 64 activation rows, head_dim 128 (rotary) / d_ff a multiple of 64 (SwiGLU);
-// `*_supported` says whether a shape takes this path, otherwise the projection and its consumer run as two kernels.
-bool fused_enabled();
-void set_fused(bool on);
-bool gemm_rope_fused_supported(int32_t M, int32_t H, int32_t Hkv, int32_t D, int32_t K, int32_t dtype);
-cudaError_t launch_gemm_rope_fused(const void* x, const void* x_lo, const void* wqkv, int32_t K, const double* inv_freq,
-                                   const int32_t* depth, const Batch& bt, void* q_out, void* k_slab, void* v_slab,
-                                   int32_t H, int32_t Hkv, int32_t max_seq, int* status, cudaStream_t st);
-bool gemm_swiglu_fused_supported(int32_t M, int32_t f, int32_t K, int32_t dtype);
-cudaError_t launch_gemm_swiglu_fused(const void* x, const void* x_lo, const void* w_gate_up, int32_t M, int32_t f, int32_t K,
-                                     void* act, void* act_lo, int* status, cudaStream_t st);
 
 // Rotary embedding of q and k at position seq_len[b] + depth[row]; q -> q_out [rows][H][D];
 // k, v -> cache rows seq_len[b] + local row of the layer slab [B][Hkv][max_seq][D].  The projection result has

@@ -238,48 +238,6 @@ def test_top_k_tree_template_decoding(trj):
     model.close()
 
 
-def test_fused_projections_agree_with_the_separate_kernels(trj):
-    """QKV projection + rotary embedding + K/V append as one kernel and gate/up projection + SwiGLU as one kernel
-    (K ranges summed inside a thread-block cluster) against the same steps as separate kernels: same arithmetic up to
-    the order of the fp32 partial sums, so logits agree to ~1e-4 and the bf16 cache rows are equal except where a
-    rounding fell the other way.  Both variants are compared with the oracle by the other tests of this file."""
-    cfg = synth.LLAMA7B.with_layers(2)
-    prompt = synth.prompt(21, 200, cfg.vocab)
-    parent = synth.random_tree(6, 33, 6, 3)
-    depth, anc = None, None
-    tokens = synth.prompt(22, 33, cfg.vocab)
-    res = {}
-    try:
-        for fused in (True, False):
-            trj.set_fused(fused)
-            model, _ = make_models(trj, cfg, 7, max_seq=384, max_rows=128)
-            depth, anc = trj.tree_from_parents(parent)
-            l0 = trj.launch_count()
-            model.prefill(i32(prompt))
-            out = model.verify_step(i32(tokens), i32(parent), i32(depth), anc_dev(anc), i32([0, 33]), max_rows=33,
-                                    max_len=233, want_logits=True)
-            torch.cuda.synchronize()
-            model.device_status()
-            res[fused] = (out["logits"].clone(), model.k_cache[:, 0, :, :233].clone(), model.v_cache[:, 0, :, :233].clone(),
-                          trj.launch_count() - l0)
-            model.close()
-    finally:
-        trj.set_fused(True)
-    (la, ka, va, na), (lb, kb, vb, nb) = res[True], res[False]
-    assert na < nb                                         # two launches fewer per layer
-    assert (la - lb).abs().max().item() <= 2e-3
-    for a, b in ((ka, kb), (va, vb)):
-        assert float((a != b).float().mean()) <= 0.02
-        assert (a.float() - b.float()).abs().max().item() <= 0.0625
-    # the fused path is deterministic: the same step again gives the same bits
-    model, _ = make_models(trj, cfg, 7, max_seq=384, max_rows=128)
-    model.prefill(i32(prompt))
-    again = model.verify_step(i32(tokens), i32(parent), i32(depth), anc_dev(anc), i32([0, 33]), max_rows=33, max_len=233,
-                              want_logits=True)
-    assert torch.equal(again["logits"], la)
-    model.close()
-
-
 def test_programmatic_launch_does_not_change_results(trj):
     """The chain's kernels start on chain-invariant data before their predecessor has finished (tensor maps, weights,
     batch geometry, cached K/V rows).  If any of that were data the predecessor still writes, the result would
