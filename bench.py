@@ -506,6 +506,42 @@ def bench_template_step(trj, torch, synth, model, cfg, prefix, side, steps):
             "what": "7B shape, prefix %d, 63-node template + retrieval path of 5 + root; random drafts" % prefix}
 
 
+def bench_llama3_step(trj, torch, synth, peaks, steps):
+    """The same verification step on the shape of the paper's main model family (Table 2): LLaMA-3-8B, grouped-query
+    attention with 8 K/V heads, 128 256-way vocabulary; 33-row trees behind a 512-token prompt, random drafts."""
+    from synth.device import device_weights
+    dev = torch.device("cuda", torch.cuda.current_device())
+    cfg = synth.LLAMA3_8B
+    layers, glob = device_weights(cfg, 4242, dev)
+    model = trj.Model(cfg, layers, glob, max_batch=1, max_seq=PROMPT + 256, max_rows=trj.MAX_ROWS)
+    i32 = lambda a: torch.from_numpy(np.ascontiguousarray(a, dtype=np.int32)).to(dev)
+    model.prefill(i32(synth.prompt(5, PROMPT, cfg.vocab)))
+    tree = trj.build_tree(17, synth.prompt(6, WIDTH, cfg.vocab), synth.prompt(7, N_BRANCHES * BRANCH_LEN, cfg.vocab).reshape(N_BRANCHES, BRANCH_LEN))
+    d_tok, d_par, d_dep, d_off = i32(tree["tokens"]), i32(tree["parent"]), i32(tree["depth"]), i32([0, TREE_ROWS])
+    d_anc = torch.from_numpy(tree["anc"].view(np.int64)).to(dev)
+    seq0 = model.seq_len.clone()
+    pred = torch.empty(TREE_ROWS, dtype=torch.int32, device=dev)
+    acc = {"k_acc": torch.empty(1, dtype=torch.int32, device=dev), "bonus": torch.empty(1, dtype=torch.int32, device=dev),
+           "path": torch.empty(1, trj.PATH_STRIDE, dtype=torch.int32, device=dev)}
+
+    def step():
+        model.seq_len.copy_(seq0)
+        model.verify_step(d_tok, d_par, d_dep, d_anc, d_off, max_rows=TREE_ROWS, max_len=PROMPT + TREE_ROWS, node_argmax=pred)
+        model.accept(d_tok, d_par, d_dep, d_off, pred, out=acc)
+        model.compact_kv(acc["k_acc"], acc["path"])
+    us = graph_us(torch, step, steps, 3)
+    model.device_status()
+    hd, kvd, d, f, v = cfg.n_heads * cfg.head_dim, cfg.kv_heads * cfg.head_dim, cfg.d_model, cfg.d_ff, cfg.vocab
+    weight_bytes = 2 * (cfg.n_layers * ((hd + 2 * kvd) * d + d * hd + 2 * f * d + d * f) + v * d)
+    model.close()
+    del layers, glob
+    torch.cuda.empty_cache()
+    return {"model": "LLaMA-3-8B shape (32 query / 8 K/V heads, d_ff 14336, vocabulary 128256), random init", "tree_rows": TREE_ROWS,
+            "prefix": PROMPT, "ms_per_step": us / 1e3, "draft_tokens_verified_per_s": DRAFTS / (us / 1e6),
+            "weight_bytes_per_step": weight_bytes, "weight_stream_gbs": round(weight_bytes / us / 1e3, 1),
+            "frac_of_" + peaks["source"] + "_peak_whole_step": round(weight_bytes / us / 1e3 / peaks["hbm_gbs"], 4)}
+
+
 def bench_prefill_gemm(trj, torch, peaks, steps):
     """The four projections of the 7B shape on prompt-sized row counts (the tensor-bound side of the projection
     kernel: 128 x 256 tiles), as a stand-alone op: TFLOP/s against the measured dense bf16 peak."""
@@ -806,6 +842,7 @@ def run_ours(args, rank, world, local_rank):
                            "note": "projections take bf16-pair activations: two tensor-core products per weight tile"}
         if not args.no_attention:
             line["prefill_gemm"] = bench_prefill_gemm(trj, torch, peaks, max(args.steps // 2, 5))
+            line["llama3_8b_step"] = bench_llama3_step(trj, torch, synth, peaks, max(args.steps // 2, 5))
         if not args.no_attention:
             line["tree_attention"] = bench_tree_attention(trj, torch, peaks, max(args.steps, 5), 3, cpu=not args.no_cpu)
             line["small_ops"] = bench_small_ops(trj, torch, peaks, max(args.steps, 5), 3, cpu=not args.no_cpu)

@@ -646,23 +646,6 @@ struct TopList {
         v[KMAX - 1] = -INFINITY; id[KMAX - 1] = 0x7fffffff;
     }
 };
-// Two entries (arg-max plus the runner-up that the margin needs): the same list without a branch, because this is
-// the arg-max of every verification step and 32 lanes that branch differently on every element cost more than the
-// selects do.
-template <>
-struct TopList<2> {
-    float v[2]; int id[2];
-    __device__ __forceinline__ void clear() { v[0] = v[1] = -INFINITY; id[0] = id[1] = 0x7fffffff; }
-    __device__ __forceinline__ void push(float x, int i) {
-        const bool b0 = x > v[0] || (x == v[0] && i < id[0]);
-        const bool b1 = x > v[1] || (x == v[1] && i < id[1]);
-        v[1] = b0 ? v[0] : (b1 ? x : v[1]);
-        id[1] = b0 ? id[0] : (b1 ? i : id[1]);
-        v[0] = b0 ? x : v[0];
-        id[0] = b0 ? i : id[0];
-    }
-    __device__ __forceinline__ void pop() { v[0] = v[1]; id[0] = id[1]; v[1] = -INFINITY; id[1] = 0x7fffffff; }
-};
 // KMAX rounds: the best head of the warp's 32 lists is taken out (ids are unique, so exactly one lane pops) and
 // handed to lane `round`; afterwards lane r < KMAX holds the warp's r-th best entry.
 template <int KMAX>
@@ -737,6 +720,80 @@ __global__ void __launch_bounds__(TOPK_THREADS) topk_accept_kernel(
         if (lane == 0) {
             node_argmax[row] = ci;
             if (margin) margin[row] = cv - second;
+            __threadfence();
+            const int b = seq_of_row(row_off, B, row);
+            const unsigned int need = (unsigned int)(row_off[b + 1] - row_off[b]);
+            const unsigned int got = atomicAdd(&tickets[b], 1u);
+            last_flag = (got + 1 == need) ? b : -1;
+            if (got + 1 == need) tickets[b] = 0;             // ready for the next call
+        }
+    }
+    __syncthreads();
+    const int b = last_flag;
+    if (b < 0 || !do_accept) return;
+    __threadfence();                                         // the other rows' predictions were written by other CTAs
+    const int r0 = row_off[b], rows = row_off[b + 1] - r0;
+    accept_sequence(tokens + r0, parent + r0, depth + r0, node_argmax + r0, rows,
+                    k_acc + b, path + (size_t)b * TRJ_PATH_STRIDE, bonus + b);
+}
+
+// The arg-max of every verification step (K = 1): one CTA per row, five instructions per element.  A thread scans its
+// elements in ascending id order, so "strictly larger" keeps the smallest id among equals; the runner-up value (for
+// the margin) is max(v2, min(v1, x)).  Threads, then warps, are merged with the full (value, id) order.
+template <typename T>
+__global__ void __launch_bounds__(TOPK_THREADS) argmax_row_accept_kernel(
+        const T* __restrict__ logits, int V, const int32_t* __restrict__ tokens,
+        const int32_t* __restrict__ parent, const int32_t* __restrict__ depth,
+        const int32_t* __restrict__ row_off, int B, int32_t* node_argmax,
+        float* __restrict__ margin, int32_t* __restrict__ k_acc, int32_t* __restrict__ path,
+        int32_t* __restrict__ bonus, int do_accept, unsigned int* tickets) {
+    pdl_prologue();
+    __shared__ Top red[TOPK_THREADS / 32];
+    __shared__ int last_flag;
+    const int row = blockIdx.x, warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const T* lr = logits + (size_t)row * V;
+    float v1 = -INFINITY, v2 = -INFINITY;
+    int i1 = 0x7fffffff;
+    auto look = [&](float x, int i) {
+        v2 = fmaxf(v2, fminf(v1, x));
+        i1 = x > v1 ? i : i1;
+        v1 = fmaxf(v1, x);
+    };
+    constexpr int VEC = 16 / (int)sizeof(T);
+    if (V % VEC == 0 && ((uintptr_t)logits % 16) == 0) {
+        constexpr int BATCH = 4;                             // four 16-byte loads in flight per thread
+        for (int v0 = threadIdx.x * VEC; v0 < V; v0 += BATCH * TOPK_THREADS * VEC) {
+            uint4 raw[BATCH];
+#pragma unroll
+            for (int j = 0; j < BATCH; ++j) {
+                const int v = v0 + j * TOPK_THREADS * VEC;
+                if (v < V) raw[j] = *reinterpret_cast<const uint4*>(lr + v);
+            }
+#pragma unroll
+            for (int j = 0; j < BATCH; ++j) {
+                const int v = v0 + j * TOPK_THREADS * VEC;
+                if (v < V) {
+                    const T* e = reinterpret_cast<const T*>(&raw[j]);
+#pragma unroll
+                    for (int i = 0; i < VEC; ++i) look(to_f(e[i]), v + i);
+                }
+            }
+        }
+    } else {
+        for (int v = threadIdx.x; v < V; v += TOPK_THREADS) look(to_f(lr[v]), v);
+    }
+    Top t{v1, i1, v2};
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) t = top_merge(t, top_shfl_xor(t, o));
+    if (lane == 0) red[warp] = t;
+    __syncthreads();
+    if (warp == 0) {
+        t = red[lane];
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) t = top_merge(t, top_shfl_xor(t, o));
+        if (lane == 0) {
+            node_argmax[row] = t.i1;
+            if (margin) margin[row] = t.v1 - t.v2;
             __threadfence();
             const int b = seq_of_row(row_off, B, row);
             const unsigned int need = (unsigned int)(row_off[b + 1] - row_off[b]);
@@ -967,11 +1024,12 @@ cudaError_t launch_topk_accept(const void* logits, int32_t dtype, int32_t V, int
     count_launch();
     cudaError_t launch_err = cudaSuccess;
     unsigned int* tickets = (unsigned int*)ws;
-    // the margin needs the runner-up, so the shortest list holds two entries
-    if (K <= 2) {
-        DISPATCH_T(dtype, launch_err = launch_chain(topk_accept_kernel<T, 2>, dim3(rows_total), dim3(TOPK_THREADS), 0, st,
-                                                    (const T*)logits, V, K, tokens, parent, depth, row_off, B, topk, node_argmax,
+    if (K == 1) {                                            // the step's arg-max: a kernel of its own, five instructions per element
+        DISPATCH_T(dtype, launch_err = launch_chain(argmax_row_accept_kernel<T>, dim3(rows_total), dim3(TOPK_THREADS), 0, st,
+                                                    (const T*)logits, V, tokens, parent, depth, row_off, B, node_argmax,
                                                     margin, k_acc, path, bonus, do_accept ? 1 : 0, tickets));
+        if (launch_err == cudaSuccess && topk)
+            launch_err = cudaMemcpyAsync(topk, node_argmax, sizeof(int32_t) * (size_t)rows_total, cudaMemcpyDeviceToDevice, st);
     } else {
         DISPATCH_T(dtype, launch_err = launch_chain(topk_accept_kernel<T, TRJ_MAX_TOPK>, dim3(rows_total), dim3(TOPK_THREADS), 0, st,
                                                     (const T*)logits, V, K, tokens, parent, depth, row_off, B, topk, node_argmax,
