@@ -66,7 +66,7 @@ class ClockSampler:
         try:
             self.file = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
             self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
-                                          "-lms", "100", "-i", str(self.index)], stdout=self.file, stderr=subprocess.DEVNULL)
+                                          "-lms", "50", "-i", str(self.index)], stdout=self.file, stderr=subprocess.DEVNULL)
         except Exception:
             self.proc = None
 
@@ -604,6 +604,10 @@ def run_ours(args, rank, world, local_rank):
     # here before any clock starts) is therefore planted into the first retrieved branch of every step, 0..3 tokens
     # of it, which puts the committed tokens per step at the 2-3 the paper reports.  The same lengths are used by
     # all three timed legs.
+    # clock samples run from here (a second or two of the same kernels before the first timed region, so that the
+    # sampler is up when it starts) to the end of the device loop
+    sampler = ClockSampler(local_rank)
+    sampler.start()
     truth = decode.tr_jacobi_generate(model, prompt, n_truth, 0, 0, 0, draw)
     abs_truth = np.concatenate([prompt, np.asarray(truth, np.int32)]).astype(np.int32)     # guess for position i
     take = planted_lengths(rank, n_host_steps + 2 * n_loop + 8)
@@ -665,9 +669,7 @@ def run_ours(args, rank, world, local_rank):
             dist.barrier()
         torch.cuda.synchronize()
 
-    sampler = ClockSampler(local_rank)
     barrier()
-    sampler.start()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     e0.record()
     for i in range(args.steps):

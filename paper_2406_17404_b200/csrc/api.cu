@@ -180,6 +180,7 @@ struct trj_ctx {
     void* argmax_ws; void* attn_ws; size_t attn_ws_bytes; void* gemm_ws; size_t gemm_ws_bytes;
     // chain-tree tables for prefill and the staging area of trj_step_host (device)
     int32_t* chain_depth; uint64_t* chain_anc; int32_t* chunk_row_off; int32_t* unit_row_off; int32_t* prefill_geo;
+    unsigned int* compact_tickets;   // device: one counter per sequence for the compaction kernel
     int32_t* loop_state;   // device: [0] step counter, [1] context-overflow flag of trj_decode_device
     int32_t* step_in;      // tokens | parent | depth | row_off(2) | pad -> anc
     int32_t* step_out;     // node_argmax | k_acc | bonus | path | device status words (projections, attention)
@@ -248,6 +249,7 @@ size_t carve(const trj_model_cfg& c, void* ws, trj_ctx* ctx) {
     int32_t* step_in = (int32_t*)cv.take<char>(STEP_IN_BYTES);
     int32_t* step_out = cv.take<int32_t>(STEP_OUT_INTS);
     int32_t* loop_state = cv.take<int32_t>(64);
+    unsigned int* compact_tickets = cv.take<unsigned int>(TRJ_MAX_BATCH);
     if (ctx) {
         ctx->h = h; ctx->y = y; ctx->logits = logits; ctx->x = x; ctx->q = q; ctx->act = act;
         ctx->x_lo = c.dtype == TRJ_BF16 ? x_lo : nullptr; ctx->act_lo = c.dtype == TRJ_BF16 ? act_lo : nullptr;
@@ -257,6 +259,7 @@ size_t carve(const trj_model_cfg& c, void* ws, trj_ctx* ctx) {
         ctx->chunk_row_off = chunk_row_off; ctx->unit_row_off = unit_row_off;
         ctx->step_in = step_in; ctx->step_out = step_out; ctx->loop_state = loop_state;
         ctx->dev_status = step_out + STEP_STATUS_AT;
+        ctx->compact_tickets = compact_tickets;
     }
     return cv.off;
 }
@@ -648,7 +651,7 @@ extern "C" trj_status trj_compact_kv(trj_ctx* ctx, void* k_cache, void* v_cache,
     cudaStream_t st = (cudaStream_t)stream;
     ChainScope chain;
     LAUNCH(PROF_COMPACT, launch_compact(k_cache, v_cache, c.n_layers, c.max_batch, B, kv_heads(c), c.max_seq, c.head_dim,
-                                        c.dtype, seq_len, k_acc, path, st));
+                                        c.dtype, seq_len, k_acc, path, st, ctx->compact_tickets));
     return TRJ_OK;
 }
 
@@ -700,7 +703,7 @@ trj_status enqueue_step(trj_ctx* ctx, void* k_cache, void* v_cache, int32_t* seq
     LAUNCH(PROF_ARGMAX, launch_topk_accept(ctx->logits, TRJ_F32, c.vocab, 1, d_tokens, d_parent, d_depth, d_off, 1, M, nullptr, d_pred,
                                            nullptr, d_k, d_path, d_bonus, true, ctx->argmax_ws, st));
     LAUNCH(PROF_COMPACT, launch_compact(k_cache, v_cache, c.n_layers, c.max_batch, 1, kv_heads(c), c.max_seq, c.head_dim,
-                                        c.dtype, seq_len, d_k, d_path, st));
+                                        c.dtype, seq_len, d_k, d_path, st, ctx->compact_tickets));
     TRJ_CHECK_CUDA(cudaMemcpyAsync(ctx->pin_out, ctx->step_out, sizeof(int32_t) * STEP_OUT_INTS, cudaMemcpyDeviceToHost, st));
     return TRJ_OK;
 }
@@ -870,7 +873,7 @@ extern "C" trj_status trj_decode_device(trj_ctx* ctx, void* k_cache, void* v_cac
         LAUNCH_ON(on, PROF_ARGMAX, launch_topk_accept(ctx->logits, TRJ_F32, c.vocab, 1, d_tokens, d_parent, d_depth, d_off, 1, M, nullptr,
                                                       d_pred, nullptr, d_k, d_path, d_bonus, true, ctx->argmax_ws, on));
         LAUNCH_ON(on, PROF_COMPACT, launch_compact(k_cache, v_cache, c.n_layers, c.max_batch, 1, kv_heads(c), c.max_seq, c.head_dim,
-                                                   c.dtype, seq_len, d_k, d_path, on));
+                                                   c.dtype, seq_len, d_k, d_path, on, ctx->compact_tickets));
         LAUNCH_ON(on, PROF_ELEMENTWISE, launch_commit_refill(d_tokens, d_parent, d_pred, M, d_k, d_path, d_bonus, context, capacity,
                                                              n_ctx, W, W + R * branch_len, draws, d_step, window, k_log, d_overflow, on));
         return TRJ_OK;

@@ -828,9 +828,9 @@ __global__ void accept_only_kernel(const int32_t* __restrict__ tokens, const int
 constexpr int COMPACT_BATCH = 16;
 __global__ void __launch_bounds__(256) compact_kernel(uint4* __restrict__ k_cache, uint4* __restrict__ v_cache,
                                                       int B_cache, int B, int H, int max_seq, int row_vec,
-                                                      const int32_t* __restrict__ seq_len,
+                                                      int32_t* seq_len,
                                                       const int32_t* __restrict__ k_acc,
-                                                      const int32_t* __restrict__ path) {
+                                                      const int32_t* __restrict__ path, unsigned int* tickets) {
     pdl_prologue();
     extern __shared__ uint4 stage[];             // [COMPACT_BATCH][row_vec]
     int idx = blockIdx.x;
@@ -838,8 +838,18 @@ __global__ void __launch_bounds__(256) compact_kernel(uint4* __restrict__ k_cach
     const int hh = idx % H; idx /= H;
     const int b = idx % B; const int l = idx / B;
     const int k = k_acc[b];
-    if (k <= 0) return;
     const int S = seq_len[b];
+    // With tickets the sequence's length is advanced here as well: every CTA has read it by the time it draws its
+    // ticket, so the CTA that draws the last one may write it (and leaves the ticket at zero for the next call).
+    auto finish = [&]() {
+        if (!tickets) return;
+        __syncthreads();
+        if (threadIdx.x == 0) {
+            const unsigned int per_seq = gridDim.x / (unsigned int)B;
+            if (atomicAdd(&tickets[b], 1u) + 1u == per_seq) { tickets[b] = 0; seq_len[b] = S + k + 1; }
+        }
+    };
+    if (k <= 0) { finish(); return; }
     uint4* slab = (kv ? v_cache : k_cache) + (((size_t)l * B_cache + b) * H + hh) * (size_t)max_seq * row_vec;
     const int32_t* pb = path + (size_t)b * TRJ_PATH_STRIDE;
     for (int j0 = 1; j0 <= k; j0 += COMPACT_BATCH) {
@@ -857,6 +867,7 @@ __global__ void __launch_bounds__(256) compact_kernel(uint4* __restrict__ k_cach
         }
         __syncthreads();
     }
+    finish();
 }
 
 __global__ void advance_len_kernel(int32_t* seq_len, const int32_t* k_acc, int B) {
@@ -1095,14 +1106,16 @@ cudaError_t launch_argmax_accept_static(const void* logits, int32_t dtype, int32
 
 cudaError_t launch_compact(void* k_cache, void* v_cache, int32_t L, int32_t B_cache, int32_t B, int32_t H,
                            int32_t max_seq, int32_t D, int32_t dtype, int32_t* seq_len,
-                           const int32_t* k_acc, const int32_t* path, cudaStream_t st) {
-    count_launch(); count_launch();
+                           const int32_t* k_acc, const int32_t* path, cudaStream_t st, unsigned int* tickets) {
+    count_launch();
     const int row_vec = (int)(D * dtype_size(dtype) / 16);
     const size_t smem = sizeof(uint4) * COMPACT_BATCH * row_vec;
     cudaError_t e = launch_chain(compact_kernel, dim3(L * B * H * 2), dim3(256), smem, st, (uint4*)k_cache, (uint4*)v_cache,
-                                 B_cache, B, H, max_seq, row_vec, (const int32_t*)seq_len, k_acc, path);
+                                 B_cache, B, H, max_seq, row_vec, seq_len, k_acc, path, tickets);
     if (e == cudaSuccess) e = cudaGetLastError();
-    if (e != cudaSuccess) return e;
+    if (e != cudaSuccess || tickets) return e;
+    // without a ticket array (the op-level call has no workspace) the lengths are advanced by a second kernel
+    count_launch();
     e = launch_chain(advance_len_kernel, dim3((B + 63) / 64), dim3(64), 0, st, seq_len, k_acc, B);
     return e != cudaSuccess ? e : cudaGetLastError();
 }

@@ -209,9 +209,11 @@ cudaError_t launch_argmax_accept_static(const void* logits, int32_t dtype, int32
                                         int32_t* node_argmax, float* margin, int32_t* k_acc, int32_t* path,
                                         int32_t* bonus, cudaStream_t st);
 
+// tickets (may be null): TRJ_MAX_BATCH zero-initialised counters; with them the lengths are advanced by the same
+// kernel (the CTA that finishes a sequence last), without them by a second launch.
 cudaError_t launch_compact(void* k_cache, void* v_cache, int32_t L, int32_t B_cache, int32_t B, int32_t H,
                            int32_t max_seq, int32_t D, int32_t dtype, int32_t* seq_len,
-                           const int32_t* k_acc, const int32_t* path, cudaStream_t st);
+                           const int32_t* k_acc, const int32_t* path, cudaStream_t st, unsigned int* tickets = nullptr);
 // row_off = {0, m} and seq_len[b] += delta: small bookkeeping used by prefill.
 cudaError_t launch_set_chunk(int32_t* row_off2, int32_t m, cudaStream_t st);
 // Geometry of a prefill chunk of m rows whose attention runs in n_sub pieces of `sub` rows (the last one of

@@ -238,6 +238,77 @@ def test_top_k_tree_template_decoding(trj):
     model.close()
 
 
+@pytest.mark.parametrize("cfg_name,n_seq,tol", [("tiny", 5, 1e-3), ("7b", 4, 2e-2)])
+def test_batched_verify_step(trj, cfg_name, n_seq, tol):
+    """A ragged batch through the model path: independent sequences with different prompts and trees of different
+    sizes in ONE verify_step / accept / compact_kv (the batched case of the configs, here with the whole decoder).
+    Every sequence is compared with the oracle run on that sequence alone: logits, predictions, accepted path,
+    committed cache rows and lengths."""
+    from oracle.model import verify_step as oracle_step
+    cfg = synth.TINY if cfg_name == "tiny" else synth.LLAMA7B.with_layers(2)
+    from paper_2406_17404_b200.decode import upload_weights
+    layers = [synth.layer_weights(cfg, 8, l) for l in range(cfg.n_layers)]
+    glob = synth.global_weights(cfg, 8)
+    dl, dg = upload_weights(cfg, layers, glob)
+    model = trj.Model(cfg, dl, dg, max_batch=n_seq, max_seq=256, max_rows=64)
+    f64 = lambda d: {k: np.asarray(v, np.float64) for k, v in d.items()}
+    dec = oracle.Decoder(cfg, [f64(l) for l in layers], f64(glob))
+    g = synth.stream(8, "batched")
+    prompts = [synth.prompt(80 + b, int(g.integers(20, 150)), cfg.vocab) for b in range(n_seq)]
+    rows = [int(g.integers(16, 65)) for _ in range(n_seq)]
+    parents = [synth.random_tree(90 + b, m, min(6, m - 1), 3) for b, m in enumerate(rows)]
+    # prompts go in one sequence at a time; the oracle keeps one cache per sequence
+    caches, roots = [], []
+    for b in range(n_seq):
+        first = int(model.prefill(i32(prompts[b]), b).item())
+        cache = dec.new_cache(256)
+        lg = dec.forward_rows(cache, prompts[b], synth.chain_parents(len(prompts[b])))
+        cache.seq_len = len(prompts[b])
+        root = int(oracle.node_argmax(lg[-1:])[0])
+        if oracle.top2_margin(lg[-1:])[0] >= MARGIN:
+            assert first == root
+        caches.append(cache); roots.append(root)
+    assert model.seq_len.tolist() == [len(p) for p in prompts]
+    # drafts: the root, then tokens planted so that some path is accepted (the oracle's own predictions of a first pass)
+    tokens = []
+    for b in range(n_seq):
+        t = synth.prompt(100 + b, rows[b], cfg.vocab); t[0] = roots[b]
+        probe = dec.new_cache(256); probe.k[:], probe.v[:], probe.seq_len = caches[b].k, caches[b].v, caches[b].seq_len
+        pred = oracle.node_argmax(dec.forward_rows(probe, t, parents[b]))
+        for i in range(1, rows[b]):                       # a row under the root's subtree carries its parent's prediction half the time
+            if g.random() < 0.5:
+                t[i] = pred[parents[b][i]]
+        tokens.append(t)
+    off = np.concatenate([[0], np.cumsum(rows)]).astype(np.int32)
+    dep_anc = [trj.tree_from_parents(p) for p in parents]
+    d_tok, d_par = i32(np.concatenate(tokens)), i32(np.concatenate(parents))
+    d_dep, d_anc, d_off = i32(np.concatenate([d for d, _ in dep_anc])), anc_dev(np.concatenate([a for _, a in dep_anc], 0)), i32(off)
+    max_len = max(len(p) + m for p, m in zip(prompts, rows))
+    out = model.verify_step(d_tok, d_par, d_dep, d_anc, d_off, max_rows=max(rows), max_len=max_len, want_logits=True, want_margin=True)
+    acc = model.accept(d_tok, d_par, d_dep, d_off, out["node_argmax"])
+    model.compact_kv(acc["k_acc"], acc["path"], batch=n_seq)
+    torch.cuda.synchronize()
+    model.device_status()
+    logits, pred = out["logits"].cpu().numpy(), out["node_argmax"].cpu().numpy()
+    for b in range(n_seq):
+        want = oracle_step(dec, caches[b], tokens[b], parents[b])
+        sl = slice(off[b], off[b + 1])
+        assert np.abs(logits[sl] - want["logits"]).max() <= tol, b
+        safe = oracle.top2_margin(want["logits"]) >= MARGIN
+        np.testing.assert_array_equal(pred[sl][safe], want["pred"][safe])
+        k = int(acc["k_acc"][b]); path = acc["path"][b, :k + 1].tolist()
+        assert (k, path, int(acc["bonus"][b])) == oracle.accept_path(tokens[b], parents[b], pred[sl])
+        if safe.all():
+            assert (k, path) == (want["k"], want["path"])
+            n = len(prompts[b]) + k + 1
+            assert int(model.seq_len[b]) == n == caches[b].seq_len
+            got = model.k_cache[:, b, :, :n].double().cpu().numpy()
+            lim = 1e-4 if cfg.dtype == "f32" else 0.07       # bf16 rows: equal up to a rounding that fell the other way
+            assert np.abs(got - caches[b].k[:, :, :n]).max() <= lim
+    assert int(acc["k_acc"].max()) >= 1
+    model.close()
+
+
 def test_programmatic_launch_does_not_change_results(trj):
     """The chain's kernels start on chain-invariant data before their predecessor has finished (tensor maps, weights,
     batch geometry, cached K/V rows).  If any of that were data the predecessor still writes, the result would
