@@ -37,10 +37,11 @@ DRAFTS = TREE_ROWS - 1                                   # 32 draft tokens per s
 PROMPT = 512
 METRIC = "draft_tokens_verified_per_s"
 UNIT = "tokens/s"
-# DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) of ALL 129 projection launches of one step, from
-# an ncu capture of the current projection kernel (profiles/gemm_tc_traffic_llama7b_33rows.md); set to None
-# whenever that kernel changes.
-GEMM_TRAFFIC_BYTES_PER_STEP = 13720706048 + 85961728
+# DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) of ALL 129 projection launches of one step, from an ncu
+# capture of the current projection kernel on a 4-layer model, scaled to 32 layers + the LM head: per layer 444.13 MB
+# (QKV 102.26, output 64.21 incl. 30 MB of gate/up weights that it prefetches and that ncu's serialised timing counts
+# again in the gate/up launch, gate/up 185.11, down 92.55), LM head 262.88 MB.  Set to None whenever that kernel changes.
+GEMM_TRAFFIC_BYTES_PER_STEP = int(32 * 444.13e6 + 262.88e6)
 
 
 def measured_peaks():

@@ -96,7 +96,22 @@ __global__ void embed_kernel(const T* __restrict__ embed, const int32_t* __restr
     TRJ_TL_DECL; TRJ_TL_BEGIN(TRJ_TL_EMBED);
     const int row = blockIdx.x;
     const T* src = embed + (size_t)tokens[row] * d;
-    for (int c = threadIdx.x; c < d; c += blockDim.x) h[(size_t)row * d + c] = to_f(src[c]);
+    constexpr int VEC = 16 / (int)sizeof(T);                 // elements per 16-byte load
+    if (d % VEC == 0 && ((uintptr_t)embed % 16) == 0 && ((uintptr_t)h % 16) == 0) {
+        // the table's rows are cold in HBM: few wide loads per thread, all in flight at once
+        for (int c = threadIdx.x * VEC; c < d; c += blockDim.x * VEC) {
+            const uint4 raw = *reinterpret_cast<const uint4*>(src + c);
+            const T* e = reinterpret_cast<const T*>(&raw);
+            float out[VEC];
+#pragma unroll
+            for (int i = 0; i < VEC; ++i) out[i] = to_f(e[i]);
+#pragma unroll
+            for (int i = 0; i < VEC; i += 4)
+                *reinterpret_cast<float4*>(h + (size_t)row * d + c + i) = make_float4(out[i], out[i + 1], out[i + 2], out[i + 3]);
+        }
+    } else {
+        for (int c = threadIdx.x; c < d; c += blockDim.x) h[(size_t)row * d + c] = to_f(src[c]);
+    }
     TRJ_TL_END(TRJ_TL_EMBED);
 }
 
@@ -155,7 +170,7 @@ __global__ void __launch_bounds__(RMS_THREADS) add_rmsnorm_vec_kernel(float* __r
         if (j < n4) {
             v[k] = reinterpret_cast<const float4*>(h + (size_t)row * d)[j];
             if (add.ptr) {
-                const float4 a = parts_at4(add, (size_t)row * n4 + j);
+                const float4 a = parts_at4_batched(add, (size_t)row * n4 + j);   // the pieces' loads overlap; same order of additions
                 v[k].x += a.x; v[k].y += a.y; v[k].z += a.z; v[k].w += a.w;
                 reinterpret_cast<float4*>(h + (size_t)row * d)[j] = v[k];
             }
