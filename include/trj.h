@@ -216,8 +216,8 @@ trj_status trj_argmax_accept(const void* logits, int32_t dtype, int32_t V,
 
 /* ------------------------------------------------------------------------
  * Top-K siblings (Appendix B: the tree template holds, as siblings, the K most
- * likely tokens of a draft position; what the tree gains "mainly depends on the
- * topK of the first draft token").
+ * likely tokens of a draft position; the candidates of the first draft position
+ * carry most of what the tree adds).
  *
  * trj_topk_accept is trj_argmax_accept that also returns, for every row, the ids
  * of its K largest logits, best first (larger logit first, equal logits by

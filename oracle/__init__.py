@@ -50,9 +50,9 @@ cannot change which tokens a greedy decoder commits, unless noted):
 * Refill (Section 3.3).  New root = bonus.  New window = the arg-max at the
   rows below the winner along its own branch (lowest-index child at every
   level), then ahead noise up to W tokens.
-* Top-K trees (Appendix B: the benefit of the tree "mainly depends on the
-  topK of the first draft token"; the 63-node template itself is third-party
-  and not printed).  A template is ``parent`` plus a rank per row: siblings
+* Top-K trees (Appendix B: most of the tree's benefit comes from the
+  candidates of the first draft position; the 63-node template itself is
+  third-party and not printed).  A template is ``parent`` plus a rank per row: siblings
   under one parent carry ranks 0, 1, 2, ... and hold the rank-th most likely
   token for their position; rows of negative rank form the retrieval path.
   The candidates for depth d come from the d-th row below the winner along

@@ -196,7 +196,12 @@ struct trj_ctx {
     std::vector<LoopGraph> loop_graphs;
     cudaStream_t cap_stream = nullptr; cudaEvent_t order_ev = nullptr; uint64_t steps_done = 0;
     DraftSource draft_src{nullptr, 0, nullptr}; int32_t draft_src_steps = 0;   // trj_set_draft_source
-    int32_t last_rows = 0, last_B = 0; const int32_t* last_row_off = nullptr;  // geometry of the latest trj_verify_step
+    int32_t last_rows = 0, last_B = 0; const int32_t* last_row_off = nullptr;  // geometry of the latest trj_verify_step    // the step a tensor-parallel rank is walking through segment by segment (trj_tp_begin .. trj_tp_finish)
+    struct TpStep {
+        bool open = false; int32_t next = 0; void* k_cache = nullptr; void* v_cache = nullptr;
+        Batch bt{}; const int32_t* tokens = nullptr; const int32_t* parent = nullptr; const int32_t* depth = nullptr;
+        const uint64_t* anc = nullptr; int32_t anc_words = 0;
+    } tp;
 };
 
 namespace {
@@ -315,14 +320,23 @@ void prof_end(trj_ctx* ctx, cudaStream_t st) {
         if (le__ != cudaSuccess) return fail(TRJ_ECUDA, "%s: %s", #expr, cudaGetErrorString(le__)); \
     } while (0)
 
-// One forward of the decoder over the rows of `bt`.  lm_first/lm_rows select which rows reach the
-// LM head (prefill only needs its last row).  b0 = first sequence of the cache the batch maps to.
-// `pieces` (prefill only): attention runs piece by piece, every piece a chain below all rows before it.
-trj_status forward(trj_ctx* ctx, void* k_cache, void* v_cache, int32_t b0, const Batch& bt,
-                   const int32_t* tokens, const int32_t* depth, const uint64_t* anc, int32_t anc_words,
-                   int32_t lm_first, int32_t lm_rows, cudaStream_t st, const SubChunks* pieces = nullptr) {
-    ChainScope chain;                        // the embedding below is the chain's fence
+// What one forward works on.  lm_first/lm_rows select which rows reach the LM head (prefill only needs its last
+// row).  b0 = first sequence of the cache the batch maps to.  `pieces` (prefill only): attention runs piece by
+// piece, every piece a chain below all rows before it.
+struct StepArgs {
+    void* k_cache; void* v_cache; int32_t b0; Batch bt;
+    const int32_t* tokens; const int32_t* depth; const uint64_t* anc; int32_t anc_words;
+    int32_t lm_first, lm_rows; const SubChunks* pieces;
+};
+
+// The decoder as 2 L + 1 segments: 2 l is the attention half of layer l (norm, QKV, rotary + cache write, tree
+// attention, output projection), 2 l + 1 its feed-forward half (norm, gate/up, SwiGLU, down projection), 2 L the
+// final norm and the LM head.  Every half ends in a projection whose result the next segment adds to the residual
+// stream; `pr` carries it from segment to segment, in split-K pieces unless `finish_last` asks for the last
+// segment's result as finished sums in ctx->y (what a tensor-parallel rank hands to the sum over ranks).
+trj_status run_segments(trj_ctx* ctx, const StepArgs& a, int s0, int s1, Parts& pr, bool finish_last, cudaStream_t st) {
     const trj_model_cfg& c = ctx->cfg;
+    const Batch& bt = a.bt;
     const int M = bt.rows_total, d = c.d_model, HD = c.n_heads * c.head_dim, Hkv = kv_heads(c);
     const int QKV = HD + 2 * Hkv * c.head_dim;
     const size_t es = dtype_size(c.dtype);
@@ -334,59 +348,77 @@ trj_status forward(trj_ctx* ctx, void* k_cache, void* v_cache, int32_t b0, const
     const int attn_grid = attn_tc ? tree_attention_grid(bt.B, c.n_heads, bt.max_len) : ctx->sm_count;
     int* const gemm_status = ctx->dev_status, *const attn_status = ctx->dev_status + 1;
     constexpr size_t AHEAD_BYTES = (size_t)32 << 20;         // measured optimum on the 7B shape (16-40 MB are close)
-    LAUNCH(PROF_ELEMENTWISE, launch_embed(ctx->embed, c.dtype, tokens, ctx->h, M, d, st));
-    Parts pr{nullptr, 1, 0};                 // result of the latest projection, possibly in split-K pieces
-    for (int l = 0; l < c.n_layers; ++l) {
-        char* k_slab = (char*)k_cache + ((size_t)l * c.max_batch + b0) * seq_stride;
-        char* v_slab = (char*)v_cache + ((size_t)l * c.max_batch + b0) * seq_stride;
-        LAUNCH(PROF_ELEMENTWISE, launch_add_rmsnorm(ctx->h, pr, ctx->attn_norm[l], ctx->x, ctx->x_lo, c.dtype, M, d,
-                                                    c.rms_eps, st));
-        LAUNCH(PROF_GEMM, launch_gemm(ctx->x, ctx->x_lo, ctx->wqkv[l], ctx->y, M, QKV, d, c.dtype, ctx->gemm_ws,
-                                      ctx->gemm_ws_bytes, st, &pr, nullptr, gemm_status));
-        LAUNCH(PROF_ROPE, launch_rope_kv_write(pr, ctx->inv_freq, depth, bt, ctx->q, k_slab, v_slab, c.dtype,
-                                               c.n_heads, Hkv, c.head_dim, c.max_seq, st));
-        // inside the decoder the attention result reaches the output projection as a bf16 pair, like every
-        // other projection input
-        if (!pieces) {
-            LAUNCH(PROF_ATTENTION, launch_tree_attention(ctx->q, k_slab, v_slab, anc, anc_words, bt, c.n_heads, Hkv, c.head_dim,
-                                                         c.max_seq, c.dtype, ctx->x, ctx->x_lo, ctx->attn_ws,
-                                                         ctx->attn_ws_bytes, st, attn_status));
-        } else {
-            for (int j = 0; j < pieces->n; ++j) {
-                const int mj = j + 1 < pieces->n ? pieces->sub : pieces->last_rows;
-                // piece j sees the rows of pieces 0..j-1 as cached rows, and those were written by this very chain
-                Batch bj{pieces->lens + j, j + 1 < pieces->n ? pieces->off_full : pieces->off_last, 1, mj, mj, bt.max_len, j == 0 ? 1 : 0};
-                const size_t off = (size_t)j * pieces->sub * HD * es;
-                LAUNCH(PROF_ATTENTION, launch_tree_attention((char*)ctx->q + off, k_slab, v_slab, anc, anc_words, bj, c.n_heads, Hkv,
-                                                             c.head_dim, c.max_seq, c.dtype, (char*)ctx->x + off,
-                                                             ctx->x_lo ? (char*)ctx->x_lo + off : nullptr, ctx->attn_ws,
-                                                             ctx->attn_ws_bytes, st, attn_status));
+    const SubChunks* pieces = a.pieces;
+    for (int s = s0; s < s1; ++s) {
+        const int l = s >> 1;
+        Parts* const out_parts = (finish_last && s == s1 - 1) ? nullptr : &pr;
+        if (s == 2 * c.n_layers) {
+            LAUNCH(PROF_ELEMENTWISE, launch_add_rmsnorm(ctx->h, pr, ctx->final_norm, ctx->x, ctx->x_lo, c.dtype, M, d,
+                                                        c.rms_eps, st));
+            if (a.lm_rows > 0) {
+                const size_t off = (size_t)a.lm_first * d * es;
+                // a verification step keeps every row's logits in place; prefill wants one row and gets it in row 0
+                float* lm_out = pieces ? ctx->logits : ctx->logits + (size_t)a.lm_first * c.vocab;
+                LAUNCH(PROF_GEMM, launch_gemm((char*)ctx->x + off, ctx->x_lo ? (char*)ctx->x_lo + off : nullptr, ctx->lm_head,
+                                              lm_out, a.lm_rows, c.vocab, d, c.dtype,
+                                              ctx->gemm_ws, ctx->gemm_ws_bytes, st, nullptr, nullptr, gemm_status));
             }
+        } else if ((s & 1) == 0) {
+            char* k_slab = (char*)a.k_cache + ((size_t)l * c.max_batch + a.b0) * seq_stride;
+            char* v_slab = (char*)a.v_cache + ((size_t)l * c.max_batch + a.b0) * seq_stride;
+            LAUNCH(PROF_ELEMENTWISE, launch_add_rmsnorm(ctx->h, pr, ctx->attn_norm[l], ctx->x, ctx->x_lo, c.dtype, M, d,
+                                                        c.rms_eps, st));
+            LAUNCH(PROF_GEMM, launch_gemm(ctx->x, ctx->x_lo, ctx->wqkv[l], ctx->y, M, QKV, d, c.dtype, ctx->gemm_ws,
+                                          ctx->gemm_ws_bytes, st, &pr, nullptr, gemm_status));
+            LAUNCH(PROF_ROPE, launch_rope_kv_write(pr, ctx->inv_freq, a.depth, bt, ctx->q, k_slab, v_slab, c.dtype,
+                                                   c.n_heads, Hkv, c.head_dim, c.max_seq, st));
+            // inside the decoder the attention result reaches the output projection as a bf16 pair, like every
+            // other projection input
+            if (!pieces) {
+                LAUNCH(PROF_ATTENTION, launch_tree_attention(ctx->q, k_slab, v_slab, a.anc, a.anc_words, bt, c.n_heads, Hkv, c.head_dim,
+                                                             c.max_seq, c.dtype, ctx->x, ctx->x_lo, ctx->attn_ws,
+                                                             ctx->attn_ws_bytes, st, attn_status));
+            } else {
+                for (int j = 0; j < pieces->n; ++j) {
+                    const int mj = j + 1 < pieces->n ? pieces->sub : pieces->last_rows;
+                    // piece j sees the rows of pieces 0..j-1 as cached rows, and those were written by this very chain
+                    Batch bj{pieces->lens + j, j + 1 < pieces->n ? pieces->off_full : pieces->off_last, 1, mj, mj, bt.max_len, j == 0 ? 1 : 0};
+                    const size_t off = (size_t)j * pieces->sub * HD * es;
+                    LAUNCH(PROF_ATTENTION, launch_tree_attention((char*)ctx->q + off, k_slab, v_slab, a.anc, a.anc_words, bj, c.n_heads, Hkv,
+                                                                 c.head_dim, c.max_seq, c.dtype, (char*)ctx->x + off,
+                                                                 ctx->x_lo ? (char*)ctx->x_lo + off : nullptr, ctx->attn_ws,
+                                                                 ctx->attn_ws_bytes, st, attn_status));
+                }
+            }
+            // While the attention kernel runs, HBM is nearly idle and the SMs it leaves free go to the first CTAs of
+            // the output projection, which only wait: they ask for the start of the gate/up weights into L2.
+            const WeightPrefetch ahead{ctx->w_gate_up[l], 2 * c.d_ff, d, AHEAD_BYTES, 2 * std::max(0, ctx->sm_count - attn_grid)};
+            LAUNCH(PROF_GEMM, launch_gemm(ctx->x, ctx->x_lo, ctx->wo[l], ctx->y, M, d, HD, c.dtype, ctx->gemm_ws,
+                                          ctx->gemm_ws_bytes, st, out_parts, &ahead, gemm_status));
+        } else {
+            LAUNCH(PROF_ELEMENTWISE, launch_add_rmsnorm(ctx->h, pr, ctx->mlp_norm[l], ctx->x, ctx->x_lo, c.dtype, M, d,
+                                                        c.rms_eps, st));
+            LAUNCH(PROF_GEMM, launch_gemm(ctx->x, ctx->x_lo, ctx->w_gate_up[l], ctx->y, M, 2 * c.d_ff, d, c.dtype, ctx->gemm_ws,
+                                          ctx->gemm_ws_bytes, st, &pr, nullptr, gemm_status));
+            LAUNCH(PROF_ELEMENTWISE, launch_swiglu(pr, ctx->act, ctx->act_lo, c.dtype, M, c.d_ff, st));
+            LAUNCH(PROF_GEMM, launch_gemm(ctx->act, ctx->act_lo, ctx->w_down[l], ctx->y, M, d, c.d_ff, c.dtype, ctx->gemm_ws,
+                                          ctx->gemm_ws_bytes, st, out_parts, nullptr, gemm_status));
         }
-        // While the attention kernel runs, HBM is nearly idle and the SMs it leaves free go to the first CTAs of
-        // the output projection, which only wait: they ask for the start of the gate/up weights into L2.
-        const WeightPrefetch ahead{ctx->w_gate_up[l], 2 * c.d_ff, d, AHEAD_BYTES, 2 * std::max(0, ctx->sm_count - attn_grid)};
-        LAUNCH(PROF_GEMM, launch_gemm(ctx->x, ctx->x_lo, ctx->wo[l], ctx->y, M, d, HD, c.dtype, ctx->gemm_ws,
-                                      ctx->gemm_ws_bytes, st, &pr, &ahead, gemm_status));
-        LAUNCH(PROF_ELEMENTWISE, launch_add_rmsnorm(ctx->h, pr, ctx->mlp_norm[l], ctx->x, ctx->x_lo, c.dtype, M, d,
-                                                    c.rms_eps, st));
-        LAUNCH(PROF_GEMM, launch_gemm(ctx->x, ctx->x_lo, ctx->w_gate_up[l], ctx->y, M, 2 * c.d_ff, d, c.dtype, ctx->gemm_ws,
-                                      ctx->gemm_ws_bytes, st, &pr, nullptr, gemm_status));
-        LAUNCH(PROF_ELEMENTWISE, launch_swiglu(pr, ctx->act, ctx->act_lo, c.dtype, M, c.d_ff, st));
-        LAUNCH(PROF_GEMM, launch_gemm(ctx->act, ctx->act_lo, ctx->w_down[l], ctx->y, M, d, c.d_ff, c.dtype, ctx->gemm_ws,
-                                      ctx->gemm_ws_bytes, st, &pr, nullptr, gemm_status));
-    }
-    LAUNCH(PROF_ELEMENTWISE, launch_add_rmsnorm(ctx->h, pr, ctx->final_norm, ctx->x, ctx->x_lo, c.dtype, M, d,
-                                                c.rms_eps, st));
-    if (lm_rows > 0) {
-        const size_t off = (size_t)lm_first * d * es;
-        // a verification step keeps every row's logits in place; prefill wants one row and gets it in row 0
-        float* lm_out = pieces ? ctx->logits : ctx->logits + (size_t)lm_first * c.vocab;
-        LAUNCH(PROF_GEMM, launch_gemm((char*)ctx->x + off, ctx->x_lo ? (char*)ctx->x_lo + off : nullptr, ctx->lm_head,
-                                      lm_out, lm_rows, c.vocab, d, c.dtype,
-                                      ctx->gemm_ws, ctx->gemm_ws_bytes, st, nullptr, nullptr, gemm_status));
+        if (!out_parts) pr = Parts{ctx->y, 1, 0};
     }
     return TRJ_OK;
+}
+
+// One forward of the decoder over the rows of `bt`: embedding, then every segment.
+trj_status forward(trj_ctx* ctx, void* k_cache, void* v_cache, int32_t b0, const Batch& bt,
+                   const int32_t* tokens, const int32_t* depth, const uint64_t* anc, int32_t anc_words,
+                   int32_t lm_first, int32_t lm_rows, cudaStream_t st, const SubChunks* pieces = nullptr) {
+    ChainScope chain;                        // the embedding below is the chain's fence
+    const trj_model_cfg& c = ctx->cfg;
+    LAUNCH(PROF_ELEMENTWISE, launch_embed(ctx->embed, c.dtype, tokens, ctx->h, bt.rows_total, c.d_model, st));
+    Parts pr{nullptr, 1, 0};                 // result of the latest projection, possibly in split-K pieces
+    const StepArgs a{k_cache, v_cache, b0, bt, tokens, depth, anc, anc_words, lm_first, lm_rows, pieces};
+    return run_segments(ctx, a, 0, 2 * c.n_layers + 1, pr, false, st);
 }
 
 trj_status check_step_args(const trj_ctx* ctx, int32_t B, int32_t rows_total, int32_t max_rows, int32_t max_len,
@@ -607,6 +639,74 @@ extern "C" trj_status trj_verify_step(trj_ctx* ctx, void* k_cache, void* v_cache
     ctx->last_rows = rows_total; ctx->last_row_off = row_off; ctx->last_B = B;
     if (logits)
         TRJ_CHECK_CUDA(cudaMemcpyAsync(logits, ctx->logits, sizeof(float) * (size_t)rows_total * ctx->cfg.vocab,
+                                       cudaMemcpyDeviceToDevice, st));
+    return TRJ_OK;
+}
+
+// ---- tensor-parallel stepping: one context per rank, each holding a slice of the heads and of the feed-forward
+// width.  Every half of a layer ends in a projection whose result is a partial sum over the rank's slice; the
+// caller adds the ranks' partial sums (the exchange buffer) between two segments.
+extern "C" int32_t trj_tp_segments(const trj_ctx* ctx) { return ctx ? 2 * ctx->cfg.n_layers + 1 : 0; }
+
+extern "C" trj_status trj_tp_begin(trj_ctx* ctx, void* k_cache, void* v_cache, const int32_t* seq_len,
+                                   const int32_t* tokens, const int32_t* parent, const int32_t* depth,
+                                   const uint64_t* anc, int32_t anc_words, const int32_t* row_off,
+                                   int32_t B, int32_t rows_total, int32_t max_rows, int32_t max_len, void* stream) {
+    trj_status s = check_step_args(ctx, B, rows_total, max_rows, max_len, anc_words);
+    if (s != TRJ_OK) return s;
+    TRJ_REQUIRE(k_cache && v_cache && seq_len && tokens && parent && depth && anc && row_off, TRJ_EINVAL, "tp_begin: null pointer");
+    cudaStream_t st = (cudaStream_t)stream;
+    ChainScope chain;
+    ctx->tp = trj_ctx::TpStep{};
+    LAUNCH(PROF_ELEMENTWISE, launch_embed(ctx->embed, ctx->cfg.dtype, tokens, ctx->h, rows_total, ctx->cfg.d_model, st));
+    ctx->tp.open = true; ctx->tp.next = 0; ctx->tp.k_cache = k_cache; ctx->tp.v_cache = v_cache;
+    ctx->tp.bt = Batch{seq_len, row_off, B, rows_total, max_rows, max_len};
+    ctx->tp.tokens = tokens; ctx->tp.parent = parent; ctx->tp.depth = depth; ctx->tp.anc = anc; ctx->tp.anc_words = anc_words;
+    return TRJ_OK;
+}
+
+extern "C" trj_status trj_tp_segment(trj_ctx* ctx, int32_t segment, void* stream) {
+    TRJ_REQUIRE(ctx, TRJ_EINVAL, "tp_segment: null context");
+    TRJ_REQUIRE(ctx->tp.open, TRJ_EINVAL, "tp_segment: no step begun");
+    const int32_t n_seg = 2 * ctx->cfg.n_layers + 1;
+    TRJ_REQUIRE(segment == ctx->tp.next && segment < n_seg, TRJ_EINVAL, "tp_segment: segment %d asked, %d is next of %d",
+                segment, ctx->tp.next, n_seg);
+    cudaStream_t st = (cudaStream_t)stream;
+    ChainScope chain;
+    const trj_ctx::TpStep& t = ctx->tp;
+    const StepArgs a{t.k_cache, t.v_cache, 0, t.bt, t.tokens, t.depth, t.anc, t.anc_words, 0, t.bt.rows_total, nullptr};
+    // what the previous segment left, summed over the ranks by the caller, sits in the exchange buffer
+    Parts pr = segment == 0 ? Parts{nullptr, 1, 0} : whole(ctx->y);
+    trj_status s = run_segments(ctx, a, segment, segment + 1, pr, segment + 1 < n_seg, st);
+    if (s != TRJ_OK) { ctx->tp.open = false; return s; }
+    ctx->tp.next = segment + 1;
+    return TRJ_OK;
+}
+
+extern "C" trj_status trj_tp_exchange_buffer(const trj_ctx* ctx, float** partial, size_t* count) {
+    TRJ_REQUIRE(ctx && partial && count, TRJ_EINVAL, "tp_exchange_buffer: null pointer");
+    TRJ_REQUIRE(ctx->tp.open, TRJ_EINVAL, "tp_exchange_buffer: no step begun");
+    *partial = ctx->y;
+    *count = (size_t)ctx->tp.bt.rows_total * ctx->cfg.d_model;
+    return TRJ_OK;
+}
+
+extern "C" trj_status trj_tp_finish(trj_ctx* ctx, int32_t* node_argmax, float* margin, float* logits, void* stream) {
+    TRJ_REQUIRE(ctx && node_argmax, TRJ_EINVAL, "tp_finish: null pointer");
+    const int32_t n_seg = 2 * ctx->cfg.n_layers + 1;
+    TRJ_REQUIRE(ctx->tp.open && ctx->tp.next == n_seg, TRJ_EINVAL, "tp_finish: %d of %d segments run",
+                ctx->tp.open ? ctx->tp.next : 0, n_seg);
+    cudaStream_t st = (cudaStream_t)stream;
+    ChainScope chain;
+    const trj_ctx::TpStep& t = ctx->tp;
+    const int32_t rows = t.bt.rows_total;
+    LAUNCH(PROF_ARGMAX, launch_topk_accept(ctx->logits, TRJ_F32, ctx->cfg.vocab, 1, t.tokens, t.parent, t.depth, t.bt.row_off, t.bt.B,
+                                           rows, nullptr, node_argmax, margin, nullptr, nullptr, nullptr, false,
+                                           ctx->argmax_ws, st));
+    ctx->last_rows = rows; ctx->last_row_off = t.bt.row_off; ctx->last_B = t.bt.B;
+    ctx->tp.open = false;
+    if (logits)
+        TRJ_CHECK_CUDA(cudaMemcpyAsync(logits, ctx->logits, sizeof(float) * (size_t)rows * ctx->cfg.vocab,
                                        cudaMemcpyDeviceToDevice, st));
     return TRJ_OK;
 }
