@@ -543,6 +543,50 @@ def bench_llama3_step(trj, torch, synth, peaks, steps):
             "frac_of_" + peaks["source"] + "_peak_whole_step": round(weight_bytes / us / 1e3 / peaks["hbm_gbs"], 4)}
 
 
+def bench_tp_rank(trj, torch, synth, peaks, steps):
+    """One rank's share of the 7B step when heads and feed-forward columns are split over 2, 4 or 8 ranks: every
+    segment, the arg-max, acceptance and compaction of a rank's slice, on this one GPU and WITHOUT the sums over
+    ranks that come between the segments (64 all-reduces of rows x d_model fp32 per step).  A lower bound on the
+    step time of a tensor-parallel job, not a measurement of one."""
+    from paper_2406_17404_b200 import tp
+    from synth.device import device_weights
+    dev = torch.device("cuda", torch.cuda.current_device())
+    i32 = lambda a: torch.from_numpy(np.ascontiguousarray(a, dtype=np.int32)).to(dev)
+    full = synth.LLAMA7B
+    tree = trj.build_tree(17, synth.prompt(6, WIDTH, full.vocab), synth.prompt(7, N_BRANCHES * BRANCH_LEN, full.vocab).reshape(N_BRANCHES, BRANCH_LEN))
+    d_tok, d_par, d_dep, d_off = i32(tree["tokens"]), i32(tree["parent"]), i32(tree["depth"]), i32([0, TREE_ROWS])
+    d_anc = torch.from_numpy(tree["anc"].view(np.int64)).to(dev)
+    out = {"exchange_bytes": TREE_ROWS * full.d_model * 4, "exchanges_per_step": 2 * full.n_layers, "ranks": {}}
+    for world in (2, 4, 8):
+        cfg = tp.shard_cfg(full, world)
+        layers, glob = device_weights(cfg, 777 + world, dev)       # a slice has the shape of a narrower model
+        model = trj.Model(cfg, layers, glob, max_batch=1, max_seq=PROMPT + 256, max_rows=trj.MAX_ROWS)
+        model.prefill(i32(synth.prompt(5, PROMPT, cfg.vocab)))
+        seq0 = model.seq_len.clone()
+        acc = {"k_acc": torch.empty(1, dtype=torch.int32, device=dev), "bonus": torch.empty(1, dtype=torch.int32, device=dev),
+               "path": torch.empty(1, trj.PATH_STRIDE, dtype=torch.int32, device=dev)}
+
+        def step():
+            model.seq_len.copy_(seq0)
+            model.tp_begin(d_tok, d_par, d_dep, d_anc, d_off, max_rows=TREE_ROWS, max_len=PROMPT + TREE_ROWS)
+            for sgm in range(model.tp_segments()):
+                model.tp_segment(sgm)
+            res = model.tp_finish()
+            model.accept(d_tok, d_par, d_dep, d_off, res["node_argmax"], out=acc)
+            model.compact_kv(acc["k_acc"], acc["path"])
+        us = graph_us(torch, step, steps, 3)
+        model.device_status()
+        hd, d, f, v = cfg.n_heads * cfg.head_dim, cfg.d_model, cfg.d_ff, cfg.vocab
+        weight_bytes = 2 * (cfg.n_layers * (3 * hd * d + d * hd + 2 * f * d + d * f) + v * d)
+        out["ranks"][str(world)] = {"ms_per_step_without_exchange": us / 1e3, "weight_bytes_per_rank": weight_bytes,
+                                    "weight_stream_gbs": round(weight_bytes / us / 1e3, 1),
+                                    "frac_of_" + peaks["source"] + "_peak": round(weight_bytes / us / 1e3 / peaks["hbm_gbs"], 4)}
+        model.close()
+        del layers, glob, model
+        torch.cuda.empty_cache()
+    return out
+
+
 def bench_prefill_gemm(trj, torch, peaks, steps):
     """The four projections of the 7B shape on prompt-sized row counts (the tensor-bound side of the projection
     kernel: 128 x 256 tiles), as a stand-alone op: TFLOP/s against the measured dense bf16 peak."""
@@ -846,6 +890,7 @@ def run_ours(args, rank, world, local_rank):
         if not args.no_attention:
             line["prefill_gemm"] = bench_prefill_gemm(trj, torch, peaks, max(args.steps // 2, 5))
             line["llama3_8b_step"] = bench_llama3_step(trj, torch, synth, peaks, max(args.steps // 2, 5))
+            line["tensor_parallel_rank"] = bench_tp_rank(trj, torch, synth, peaks, max(args.steps // 2, 5))
         if not args.no_attention:
             line["tree_attention"] = bench_tree_attention(trj, torch, peaks, max(args.steps, 5), 3, cpu=not args.no_cpu)
             line["small_ops"] = bench_small_ops(trj, torch, peaks, max(args.steps, 5), 3, cpu=not args.no_cpu)

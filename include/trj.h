@@ -322,6 +322,40 @@ trj_status trj_verify_step(trj_ctx* ctx, void* k_cache, void* v_cache, const int
                            int32_t B, int32_t rows_total, int32_t max_rows, int32_t max_len,
                            int32_t* node_argmax, float* margin, float* logits, void* stream);
 
+/* The same verification step (Section 3.3) for a decoder whose weights are
+ * split over several devices (the 70B models of Table 2 do not fit one): a rank's
+ * context is created from a cfg with n_heads / R query heads, n_kv_heads / R K/V
+ * heads and d_ff / R feed-forward columns, d_model and vocab whole, and from the
+ * matching slices of the weights: the rows of wqkv of its heads (its query
+ * heads, then its key heads, then its value heads), the columns of wo of its
+ * heads, its gate rows then its up rows of w_gate_up, its columns of w_down;
+ * embedding, norms and LM head whole.  Its cache holds its K/V heads only.
+ *
+ * The decoder is 2 * n_layers + 1 segments (trj_tp_segments): 2 l is the
+ * attention half of layer l, 2 l + 1 its feed-forward half, the last one the
+ * final norm and the LM head.  Every segment but the last leaves, in the
+ * exchange buffer (trj_tp_exchange_buffer: dev fp32 [rows_total][d_model], part
+ * of the workspace), this rank's partial sum of the half's output projection.
+ * The caller adds the buffers of all ranks, in place and to the same bits on
+ * every rank (an all-reduce on `stream`), before it runs the next segment, which
+ * adds the sum to the residual stream.  Order of calls: trj_tp_begin (checks as
+ * trj_verify_step, embeds the tokens), trj_tp_segment for 0, 1, 2, ... in this
+ * order (anything else: TRJ_EINVAL), trj_tp_finish (arg-max, margin and logits
+ * as trj_verify_step; every rank computes the same).  The pointers given to
+ * trj_tp_begin must stay valid until trj_tp_finish.  With R = 1 the sequence
+ * computes what trj_verify_step computes, up to the order of a few fp32
+ * additions (a half's split-K pieces are summed before they join the residual
+ * stream instead of one by one).  Launches only; all pointers
+ * dev except trj_tp_exchange_buffer's two results (host). */
+int32_t    trj_tp_segments(const trj_ctx* ctx);
+trj_status trj_tp_begin(trj_ctx* ctx, void* k_cache, void* v_cache, const int32_t* seq_len,
+                        const int32_t* tokens, const int32_t* parent, const int32_t* depth,
+                        const uint64_t* anc, int32_t anc_words, const int32_t* row_off,
+                        int32_t B, int32_t rows_total, int32_t max_rows, int32_t max_len, void* stream);
+trj_status trj_tp_segment(trj_ctx* ctx, int32_t segment, void* stream);
+trj_status trj_tp_exchange_buffer(const trj_ctx* ctx, float** partial, size_t* count);
+trj_status trj_tp_finish(trj_ctx* ctx, int32_t* node_argmax, float* margin, float* logits, void* stream);
+
 /* accept (Section 3.3): longest accepted path from node_argmax; see
  * trj_argmax_accept for the rule and the output layout.  All pointers dev. */
 trj_status trj_accept(trj_ctx* ctx, const int32_t* tokens, const int32_t* parent, const int32_t* depth,

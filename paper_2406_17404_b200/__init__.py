@@ -75,6 +75,11 @@ _SIGNATURES = {
     "trj_create": (_I, [C.POINTER(ModelCfg), C.POINTER(Weights), _VP, _SZ, C.POINTER(_VP)]),
     "trj_destroy": (_I, [_VP]),
     "trj_verify_step": (_I, [_VP, _VP, _VP, _VP, _VP, _VP, _VP, _VP, _I, _VP, _I, _I, _I, _I, _VP, _VP, _VP, _VP]),
+    "trj_tp_segments": (_I, [_VP]),
+    "trj_tp_begin": (_I, [_VP, _VP, _VP, _VP, _VP, _VP, _VP, _VP, _I, _VP, _I, _I, _I, _I, _VP]),
+    "trj_tp_segment": (_I, [_VP, _I, _VP]),
+    "trj_tp_exchange_buffer": (_I, [_VP, C.POINTER(_VP), C.POINTER(_SZ)]),
+    "trj_tp_finish": (_I, [_VP, _VP, _VP, _VP, _VP]),
     "trj_accept": (_I, [_VP, _VP, _VP, _VP, _VP, _I, _I, _VP, _VP, _VP, _VP, _VP]),
     "trj_compact_kv": (_I, [_VP, _VP, _VP, _VP, _I, _VP, _VP, _VP]),
     "trj_prefill": (_I, [_VP, _VP, _VP, _VP, _I, _VP, _I, _VP, _VP]),
@@ -546,6 +551,44 @@ class Model:
             _dev(anc, torch.int64, "anc"), anc.shape[1], _dev(row_off, torch.int32, "row_off"), batch, rows,
             max_rows, max_len, _dev(node_argmax), _dev(margin) if want_margin else None,
             _dev(logits) if want_logits else None, _stream(stream)))
+        return {"node_argmax": node_argmax, "margin": margin, "logits": logits}
+
+    # ---- tensor-parallel stepping: this context is one rank's slice of the decoder
+    def tp_segments(self) -> int:
+        return int(lib().trj_tp_segments(self._handle))
+
+    def tp_begin(self, tokens, parent, depth, anc, row_off, *, max_rows: int, max_len: int, stream=None) -> None:
+        """trj_tp_begin: the tensors must stay alive until tp_finish (kept on the object)."""
+        torch = _torch()
+        self._tp_keep = (tokens, parent, depth, anc, row_off)
+        _check(lib().trj_tp_begin(
+            self._handle, _dev(self.k_cache), _dev(self.v_cache), _dev(self.seq_len),
+            _dev(tokens, torch.int32, "tokens"), _dev(parent, torch.int32, "parent"), _dev(depth, torch.int32, "depth"),
+            _dev(anc, torch.int64, "anc"), anc.shape[1], _dev(row_off, torch.int32, "row_off"), row_off.numel() - 1,
+            tokens.numel(), max_rows, max_len, _stream(stream)))
+
+    def tp_segment(self, segment: int, stream=None) -> None:
+        _check(lib().trj_tp_segment(self._handle, int(segment), _stream(stream)))
+
+    def tp_exchange_tensor(self):
+        """trj_tp_exchange_buffer as a float32 tensor [rows, d_model] that aliases the workspace (no copy)."""
+        torch = _torch()
+        ptr, count = _VP(), _SZ()
+        _check(lib().trj_tp_exchange_buffer(self._handle, C.byref(ptr), C.byref(count)))
+        off = ptr.value - self.workspace.data_ptr()
+        if off < 0 or off + 4 * count.value > self.workspace.numel():
+            raise TrjError(1, "exchange buffer outside the workspace")
+        return self.workspace[off:off + 4 * count.value].view(torch.float32).view(-1, self.cfg.d_model)
+
+    def tp_finish(self, *, want_logits: bool = False, want_margin: bool = False, stream=None):
+        """trj_tp_finish: dict(node_argmax, margin | None, logits | None) as verify_step."""
+        torch = _torch()
+        rows = self._tp_keep[0].numel()
+        node_argmax = torch.empty(rows, dtype=torch.int32, device=self.device)
+        margin = torch.empty(rows, dtype=torch.float32, device=self.device) if want_margin else None
+        logits = torch.empty(rows, self.cfg.vocab, dtype=torch.float32, device=self.device) if want_logits else None
+        _check(lib().trj_tp_finish(self._handle, _dev(node_argmax), _dev(margin) if want_margin else None,
+                                   _dev(logits) if want_logits else None, _stream(stream)))
         return {"node_argmax": node_argmax, "margin": margin, "logits": logits}
 
     def node_topk(self, rows: int, k: int, out=None, stream=None):
