@@ -118,6 +118,7 @@ def gemm_bytes_per_step(cfg, rows):
 def graph_us(torch, fn, steps, warmup):
     """Average device time of one call of ``fn`` (a fixed launch sequence), replayed from a CUDA graph."""
     side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())        # what fn reads may still be in flight on the caller's stream
     with torch.cuda.stream(side):
         fn()
     torch.cuda.synchronize()
@@ -486,6 +487,7 @@ def bench_template_step(trj, torch, synth, model, cfg, prefix, side, steps):
         model.node_topk(m, 10, out=topk)
         model.accept(d_tok, d_par, d_dep, d_off, pred, out=acc)
         model.compact_kv(acc["k_acc"], acc["path"])
+    side.wait_stream(torch.cuda.current_stream())
     with torch.cuda.stream(side):
         step()
     torch.cuda.synchronize()
@@ -693,6 +695,7 @@ def run_ours(args, rank, world, local_rank):
             model.accept(d_tok, d_par, d_dep, d_off, pred, out=acc)
             model.compact_kv(acc["k_acc"], acc["path"])
         # the launch sequence of a step is fixed, so it is replayed from a CUDA graph (no host work per launch)
+        side.wait_stream(torch.cuda.current_stream())
         with torch.cuda.stream(side):
             for _ in range(2):
                 resident_step()
@@ -938,6 +941,7 @@ def run_timeline(args):
         model.accept(d_tok, d_par, d_dep, d_off, pred, out=acc)
         model.compact_kv(acc["k_acc"], acc["path"])
     side = torch.cuda.Stream(device=dev)
+    side.wait_stream(torch.cuda.current_stream())
     with torch.cuda.stream(side):
         for _ in range(2):
             step()

@@ -40,7 +40,7 @@ struct TcParams {
     int halves;         // 1: x only, 2: x and x_lo
     int n_mma;          // accumulator columns = m_pad * halves, a multiple of 16
     int acc_cols;       // TMEM columns of one accumulator buffer: power of two >= max(16, n_mma); two are allocated
-    int kblocks;        // K / 64
+    int kblocks;        // ceil(K / 64)
     int tiles, splits, stages;
     float* out;         // [splits][M][N]
     int* status;        // device word: 0, or TRJ_ETIMEOUT once a wait expired
@@ -287,7 +287,7 @@ int round_up(int x, int a) { return (x + a - 1) / a * a; }
 
 bool gemm_tc_supported(const void* x, const void* x_lo, const void* w, const float* y, int32_t M, int32_t N, int32_t K,
                        int32_t dtype) {
-    if (dtype != TRJ_BF16 || M < 1 || K < TC_BK || K % TC_BK != 0 || N < 4 || N % 4 != 0) return false;
+    if (dtype != TRJ_BF16 || M < 1 || K < TC_BK || K % 8 != 0 || N < 4 || N % 4 != 0) return false;
     if (((uintptr_t)x | (uintptr_t)x_lo | (uintptr_t)w | (uintptr_t)y) % 16 != 0) return false;
     return encode_fn() != nullptr;
 }
@@ -331,7 +331,7 @@ TcPlan tc_plan(int M, int N, int K, int halves, bool finished) {
     const int reach = (halves == 2 ? pl.m_pad : 0) + round_up(pl.m_pad, 16);
     pl.acc_cols = 16;
     while (pl.acc_cols < reach) pl.acc_cols *= 2;
-    pl.kblocks = K / TC_BK;
+    pl.kblocks = (K + TC_BK - 1) / TC_BK;      // a ragged last block reads zeros past K (both operands)
     pl.tiles = (N + TC_BM - 1) / TC_BM;
     pl.stage_bytes = TC_A_BYTES + (size_t)pl.n_mma * TC_BK * 2;
     // Two CTAs per SM (one's ramp and drain overlap the other's stream) when both fit: at least three stages in
@@ -353,7 +353,7 @@ TcPlan tc_plan(int M, int N, int K, int halves, bool finished) {
 
 // Workspace: a 256-byte header whose first word is the device status, then the split-K partial sums.
 size_t gemm_tc_workspace(int32_t M, int32_t N, int32_t K) {
-    if (K % TC_BK != 0 || K < TC_BK || M < 1) return 256;
+    if (K % 8 != 0 || K < TC_BK || M < 1) return 256;
     int s = 1;
     for (int halves = 1; halves <= 2; ++halves)
         for (int finished = 0; finished <= 1; ++finished) s = std::max(s, tc_plan(M, N, K, halves, finished != 0).splits);
@@ -381,13 +381,13 @@ cudaError_t launch_gemm_tc(const void* x, const void* x_lo, const void* w, float
     p.status = status;
     CUtensorMap map_w, map_x, map_xlo, map_ahead;
     p.ahead_boxes = 0; p.ahead_kblocks = 1; p.ahead_ctas = 0;
-    const bool want_ahead = ahead && ahead->ctas > 0 && ahead->w && ahead->K % TC_BK == 0 && ahead->K >= TC_BK &&
+    const bool want_ahead = ahead && ahead->ctas > 0 && ahead->w && ahead->K % 8 == 0 && ahead->K >= TC_BK &&
                             ((uintptr_t)ahead->w % 16) == 0;
     if (want_ahead) {
         if (!make_map(&map_ahead, ahead->w, ahead->N, ahead->K, TC_BM)) return cudaErrorInvalidValue;
-        const size_t all = (size_t)((ahead->N + TC_BM - 1) / TC_BM) * (ahead->K / TC_BK);
+        const size_t all = (size_t)((ahead->N + TC_BM - 1) / TC_BM) * ((ahead->K + TC_BK - 1) / TC_BK);
         const size_t asked = ahead->bytes / TC_A_BYTES;
-        p.ahead_kblocks = ahead->K / TC_BK;
+        p.ahead_kblocks = (ahead->K + TC_BK - 1) / TC_BK;
         p.ahead_boxes = (int)(asked < all ? asked : all);
         p.ahead_ctas = ahead->ctas;
     }
@@ -422,7 +422,7 @@ cudaError_t launch_wait_expiry_selftest(int* status, uint32_t polls, cudaStream_
 }
 
 bool gemm_tc_shape(int32_t M, int32_t N, int32_t K, int32_t dtype) {
-    return dtype == TRJ_BF16 && M >= 1 && K >= TC_BK && K % TC_BK == 0 && N >= 4 && N % 4 == 0;
+    return dtype == TRJ_BF16 && M >= 1 && K >= TC_BK && K % 8 == 0 && N >= 4 && N % 4 == 0;
 }
 
 cudaError_t launch_gemm(const void* x, const void* x_lo, const void* w, float* y, int32_t M, int32_t N, int32_t K,

@@ -116,7 +116,7 @@ cudaError_t launch_add_rmsnorm(float* h, const Parts& add, const float* gain, vo
 // y[M][N] fp32 = (x + x_lo)[M][K] . w[N][K]^T (x_lo may be null), plain shared-memory tiled FMA kernel.
 cudaError_t launch_gemm_simt(const void* x, const void* x_lo, const void* w, float* y, int32_t M, int32_t N,
                              int32_t K, int32_t dtype, cudaStream_t st);
-// tcgen05 / TMA projection kernel (gemm_sm100.cu): bf16, M <= 128 rows, K a multiple of 64.  The workspace
+// tcgen05 / TMA projection kernel (gemm_sm100.cu): bf16, K >= 64 and a multiple of 8 (rows of 16-byte multiples).  The workspace
 // (gemm_tc_workspace bytes, 256-byte aligned) starts with a status word that a device-side wait sets to
 // TRJ_ETIMEOUT if it expires; the rest holds split-K partial sums.
 bool gemm_tc_supported(const void* x, const void* x_lo, const void* w, const float* y, int32_t M, int32_t N, int32_t K,
@@ -125,7 +125,7 @@ size_t gemm_tc_workspace(int32_t M, int32_t N, int32_t K);
 cudaError_t launch_gemm_tc(const void* x, const void* x_lo, const void* w, float* y, int32_t M, int32_t N, int32_t K,
                            void* workspace, cudaStream_t st, Parts* parts, const WeightPrefetch* ahead = nullptr,
                            int* status = nullptr);
-// The tcgen05 kernel for every shape it is written for (bf16, K a multiple of 64, N a multiple of 4), the plain
+// The tcgen05 kernel for every shape it is written for (bf16, K >= 64 and a multiple of 8, N a multiple of 4), the plain
 // kernel for the rest (fp32 models, odd sizes).  A shape of the first kind whose workspace is too small or
 // misaligned is an error (cudaErrorInvalidValue), never a silent detour through the plain kernel.  With `parts`
 // non-null the split-K pieces are left unreduced in the workspace for the consumer to add (*parts says where);

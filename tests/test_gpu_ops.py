@@ -269,12 +269,14 @@ def test_compaction_long_chain_overlapping_ranges(trj):
 # ----------------------------------------------------------------------------- projection GEMM
 @pytest.mark.parametrize("dtype,m,n,k", [
     ("bf16", 33, 512, 4096), ("bf16", 1, 130, 688), ("f32", 11, 1376, 256), ("bf16", 128, 257, 1104), ("f32", 70, 64, 688),
-    # shapes the tcgen05 kernel takes: K % 64 == 0, N % 4 == 0, M <= 128; ragged N tiles, one k-block, deep split-K
+    # shapes the tcgen05 kernel takes: K >= 64, K % 8 == 0, N % 4 == 0; ragged N tiles, one k-block, deep split-K
     ("bf16", 48, 384, 64), ("bf16", 17, 132, 128), ("bf16", 33, 12288, 4096), ("bf16", 128, 4096, 11008),
     ("bf16", 1, 32000, 4096), ("bf16", 64, 22016, 4096), ("bf16", 16, 128, 8192), ("bf16", 100, 1000, 192),
     # more rows than one accumulator holds: row blocks (ragged last block, several K ranges, many blocks)
     ("bf16", 129, 512, 256), ("bf16", 257, 128, 64), ("bf16", 300, 260, 192), ("bf16", 512, 1024, 4096),
     ("bf16", 2048, 4096, 512), ("bf16", 1000, 384, 2048),
+    # K that ends inside a 64-wide block (both operands read zeros past K): an eighth of the 7B feed-forward width
+    ("bf16", 33, 4096, 1376), ("bf16", 7, 64, 72), ("bf16", 128, 512, 688), ("bf16", 300, 260, 200),
 ])
 def test_gemm(trj, dtype, m, n, k):
     g = synth.stream(m * n, "gemm")
