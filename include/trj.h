@@ -472,14 +472,15 @@ trj_status trj_gemm(const void* x, const void* w, float* y, int32_t M, int32_t N
 trj_status trj_device_status(trj_ctx* ctx, int32_t clear, void* stream);
 trj_status trj_selftest_wait_expiry(int32_t* status, int32_t polls, void* stream);
 
-/* Index checks of the debug build (no counterpart in the paper).  A library built with -DTRJ_DEBUG checks, inside
- * the kernels that index the cache with device-held lengths and paths (rotary + K/V append, the generic attention
- * kernel, compaction), that every cache row lies below max_seq; a row that does not sets a bit in a flag word and
- * the access is skipped (nothing traps).  trj_debug_flags synchronises the device, writes the bits seen since the
- * last call to *flags (host) and clears them: 1 a K/V append past the cache, 2 a compaction source or destination
- * past the cache or a negative path entry, 4 seq_len + rows beyond the cache in attention.  The default build
- * trusts the caller's contract (seq_len[b] + rows <= max_len <= max_seq), has none of these checks and returns
- * TRJ_EUNSUPPORTED. */
+/* Index checks (no counterpart in the paper).  The kernels that index the cache with device-held lengths and
+ * paths (rotary + K/V append, attention, compaction) never touch a row outside the cache: an access that a
+ * length or path breaking the caller's contract (seq_len[b] + rows <= max_len <= max_seq, path entries inside the
+ * tree) would push outside is skipped, lengths are brought inside the cache before they size a loop, and nothing
+ * traps; the result of such a step is unspecified.  A library built with -DTRJ_DEBUG also records which check
+ * fired: trj_debug_flags synchronises the device, writes the bits seen since the last call to *flags (host) and
+ * clears them: 1 a K/V append past the cache, 2 a compaction source or destination past the cache or a negative
+ * path entry, 4 seq_len + rows beyond the cache in the generic attention kernel.  The default build records
+ * nothing and returns TRJ_EUNSUPPORTED. */
 trj_status trj_debug_flags(int32_t* flags);
 
 /* ------------------------------------------------------------------------

@@ -255,9 +255,12 @@ __device__ __forceinline__ void build_sched(Sched& s, const AtParams& p) {
     int u = 0;
     s.row0[0] = p.row_off[0];
     for (int b = 0; b < p.B; ++b) {
-        s.S[b] = p.seq_len[b];
         s.row0[b + 1] = p.row_off[b + 1];
-        const int total = s.S[b] + (s.row0[b + 1] - s.row0[b]);
+        // a device-held length that breaks the caller's contract must not turn into a negative or unbounded tile
+        // count: it is brought inside the cache (the tensor maps read zeros past the cache's end anyway)
+        const int rows_b = min(max(s.row0[b + 1] - s.row0[b], 0), AT_ROWS);
+        s.S[b] = min(max(p.seq_len[b], 0), max(p.max_seq - rows_b, 0));
+        const int total = s.S[b] + rows_b;
         s.tiles[b] = (total + AT_KEYS - 1) / AT_KEYS;
         s.first[b] = u;
         u += s.tiles[b] * p.H;

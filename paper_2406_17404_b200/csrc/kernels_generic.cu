@@ -10,14 +10,15 @@
 namespace trj {
 namespace {
 
-// Index checks of the debug build (-DTRJ_DEBUG): a cache row index that a device-held length or path would push
-// outside the cache sets a bit in a flag word and the access is skipped; nothing traps.  The default build trusts
-// the caller's contract (seq_len[b] + rows <= max_seq) and carries none of this.
+// Index checks: a cache row index that a device-held length or path would push outside the cache is never
+// dereferenced: the access is skipped (one compare per row; the step's result is then unspecified, since the
+// caller's contract seq_len[b] + rows <= max_seq is broken, but no memory outside the cache is touched and nothing
+// traps).  The debug build (-DTRJ_DEBUG) also records which check fired in a flag word.
 #ifdef TRJ_DEBUG
 static __device__ int g_debug_flags;
 #define TRJ_DEBUG_CHECK(ok, bit) ((ok) ? true : (atomicOr(&g_debug_flags, (bit)), false))
 #else
-#define TRJ_DEBUG_CHECK(ok, bit) (true)
+#define TRJ_DEBUG_CHECK(ok, bit) (ok)
 #endif
 enum { DBG_ROPE_ROW = 1, DBG_COMPACT_ROW = 2, DBG_ATTENTION_LEN = 4 };
 
@@ -305,7 +306,7 @@ __global__ void rope_kv_write_kernel(const Parts qkv, const double* __restrict__
         }
         q_out[(size_t)row * HD + hh * D + i] = from_f<T>(qa * cs - qb * sn);
         q_out[(size_t)row * HD + hh * D + i + half] = from_f<T>(qb * cs + qa * sn);
-        if (!has_kv || !TRJ_DEBUG_CHECK(seq_len[b] + local < max_seq, DBG_ROPE_ROW)) continue;
+        if (!has_kv || !TRJ_DEBUG_CHECK((unsigned)(seq_len[b] + local) < (unsigned)max_seq, DBG_ROPE_ROW)) continue;
         k_slab[cache_row + i] = from_f<T>(ka * cs - kb * sn);
         k_slab[cache_row + i + half] = from_f<T>(kb * cs + ka * sn);
         v_slab[cache_row + i] = from_f<T>(va);
@@ -378,7 +379,7 @@ __global__ void __launch_bounds__(ROPE_THREADS) rope_kv_write_vec_kernel(const P
     };
     store_split4<T>(q_out, nullptr, q_at, rot_lo(acc[0], acc[1]));
     store_split4<T>(q_out, nullptr, q_at + half, rot_hi(acc[0], acc[1]));
-    if (has_kv && TRJ_DEBUG_CHECK(seq_len[b] + local < max_seq, DBG_ROPE_ROW)) {
+    if (has_kv && TRJ_DEBUG_CHECK((unsigned)(seq_len[b] + local) < (unsigned)max_seq, DBG_ROPE_ROW)) {
         store_split4<T>(k_slab, nullptr, cache_at, rot_lo(acc[2], acc[3]));
         store_split4<T>(k_slab, nullptr, cache_at + half, rot_hi(acc[2], acc[3]));
         store_split4<T>(v_slab, nullptr, cache_at, acc[4]);
@@ -401,9 +402,9 @@ __global__ void __launch_bounds__(128) tree_attention_generic_kernel(
     __shared__ float part_acc[4][D];
     const int row = blockIdx.x, hh = blockIdx.y;
     const int b = seq_of_row(row_off, B, row);
-    const int S = seq_len[b];
+    const int S = min(max(seq_len[b], 0), max_seq);      // a length outside the cache reads nothing outside it
     const int rows_b = row_off[b + 1] - row_off[b];
-    const int total = TRJ_DEBUG_CHECK(S + rows_b <= max_seq, DBG_ATTENTION_LEN) ? S + rows_b : min(S + rows_b, max_seq);
+    const int total = TRJ_DEBUG_CHECK(seq_len[b] >= 0 && S + rows_b <= max_seq, DBG_ATTENTION_LEN) ? S + rows_b : min(S + rows_b, max_seq);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int kvh = hh / (H / Hkv);              // grouped-query attention: the K/V head of this query head
     const T* kb = k_slab + ((size_t)b * Hkv + kvh) * max_seq * D;
@@ -854,7 +855,7 @@ __global__ void __launch_bounds__(256) compact_kernel(uint4* __restrict__ k_cach
     const int kv = idx & 1; idx >>= 1;
     const int hh = idx % H; idx /= H;
     const int b = idx % B; const int l = idx / B;
-    const int k = k_acc[b];
+    const int k = min(k_acc[b], TRJ_PATH_STRIDE - 1);    // a path holds at most TRJ_PATH_STRIDE rows
     const int S = seq_len[b];
     // With tickets the sequence's length is advanced here as well: every CTA has read it by the time it draws its
     // ticket, so the CTA that draws the last one may write it (and leaves the ticket at zero for the next call).
@@ -873,13 +874,13 @@ __global__ void __launch_bounds__(256) compact_kernel(uint4* __restrict__ k_cach
         const int nj = min(COMPACT_BATCH, k - j0 + 1);
         for (int e = threadIdx.x; e < nj * row_vec; e += blockDim.x) {
             const int j = j0 + e / row_vec, c = e % row_vec;
-            if (TRJ_DEBUG_CHECK(pb[j] >= 0 && S + pb[j] < max_seq, DBG_COMPACT_ROW))
+            if (TRJ_DEBUG_CHECK(pb[j] >= 0 && (unsigned)(S + pb[j]) < (unsigned)max_seq, DBG_COMPACT_ROW))
                 stage[e] = slab[(size_t)(S + pb[j]) * row_vec + c];
         }
         __syncthreads();
         for (int e = threadIdx.x; e < nj * row_vec; e += blockDim.x) {
             const int j = j0 + e / row_vec, c = e % row_vec;
-            if (TRJ_DEBUG_CHECK(pb[j] >= 0 && S + pb[j] < max_seq && S + j < max_seq, DBG_COMPACT_ROW))
+            if (TRJ_DEBUG_CHECK(pb[j] >= 0 && (unsigned)(S + pb[j]) < (unsigned)max_seq && (unsigned)(S + j) < (unsigned)max_seq, DBG_COMPACT_ROW))
                 slab[(size_t)(S + j) * row_vec + c] = stage[e];
         }
         __syncthreads();
