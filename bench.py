@@ -464,7 +464,7 @@ def whole_job_rate(world, units_per_rank, seconds):
     return world * units_per_rank / seconds
 
 
-def bench_template_step(trj, torch, synth, model, cfg, prefix, side, steps):
+def bench_template_step(trj, torch, synth, model, cfg, prefix, side, steps, context=None):
     """One verification step over a 69-row static template with top-K siblings (63 draft nodes + a retrieval path of
     5 + the root: the tree size the paper uses, Appendix B; the topology is a seeded stand-in): forward, per-row top-10,
     acceptance and compaction, replayed from a CUDA graph on the same model and cache."""
@@ -504,9 +504,39 @@ def bench_template_step(trj, torch, synth, model, cfg, prefix, side, steps):
     e1.record()
     torch.cuda.synchronize()
     ms = e0.elapsed_time(e1) / steps
-    return {"tree_rows": m, "draft_tokens_per_step": m - 1, "top_k": 10, "ms_per_step": ms,
-            "draft_tokens_verified_per_s": (m - 1) / (ms / 1e3),
-            "what": "7B shape, prefix %d, 63-node template + retrieval path of 5 + root; random drafts" % prefix}
+    out = {"tree_rows": m, "draft_tokens_per_step": m - 1, "top_k": 10, "ms_per_step": ms,
+           "draft_tokens_verified_per_s": (m - 1) / (ms / 1e3),
+           "what": "7B shape, prefix %d, 63-node template + retrieval path of 5 + root; random drafts" % prefix}
+    if context is not None:
+        # the whole loop on the device (tokens of the tree, retrieval, forward, top-K + acceptance, compaction, commit
+        # and refill from the top-K table): `steps` steps enqueued at once from the prompt's state, wall clock incl.
+        # the upload of the draws and the read-back of the committed tokens
+        n_retr = int((rank < 0).sum())
+        n0 = len(context)
+        per_step = int(depth.max()) + 1
+        draw = lambda st, n: synth.noise_draws(99, st, n)
+        host_ctx = np.zeros(n0 + steps * per_step, np.int32); host_ctx[:n0] = context
+        host_drafts = np.asarray(context, np.int32)[np.asarray(draw(0, m - 1), np.int64) % n0]
+        host_draws = np.stack([np.asarray(draw(st, m - 1 + n_retr), np.int64) for st in range(1, steps + 1)])
+        k_log = torch.zeros(steps, dtype=torch.int32, device=dev)
+
+        def loop():
+            model.seq_len.copy_(seq0)
+            d_ctx, d_n = i32(host_ctx), i32([n0])
+            d_drafts = i32(host_drafts)
+            d_draws = torch.from_numpy(host_draws).to(dev)
+            model.decode_device_tree(d_ctx, d_n, n0, parent, rank, 10, n_retr, d_drafts, d_draws, steps, k_log=k_log)
+            return d_ctx.cpu(), int(d_n.item())
+        loop()                                               # captures the step's graph
+        torch.cuda.synchronize()
+        t0 = time.perf_counter()
+        tokens_out, n_end = loop()
+        wall = time.perf_counter() - t0
+        model.device_status()
+        out["device_loop"] = {"ms_per_step": wall / steps * 1e3, "tokens_committed_per_step": (n_end - n0) / steps,
+                              "committed_tokens_per_s": (n_end - n0) / wall,
+                              "what": "trj_decode_device_tree: %d steps enqueued at once" % steps}
+    return out
 
 
 def bench_llama3_step(trj, torch, synth, peaks, steps):
@@ -879,7 +909,7 @@ def run_ours(args, rank, world, local_rank):
                                     "wall clock incl. uploading the draws and reading the tokens back" % args.steps},
             "roofline": roofline, "kernel_breakdown": breakdown, "profiled_step_ms": step_ms_prof}
     if world == 1:
-        line["paper_sized_tree"] = bench_template_step(trj, torch, synth, model, cfg, PROMPT, side, args.steps)
+        line["paper_sized_tree"] = bench_template_step(trj, torch, synth, model, cfg, PROMPT, side, args.steps, context=ctx0)
         # prefill of the 512-token prompt: the weights are streamed once (projections over all 512 rows at a time)
         model.seq_len.zero_()
         model.prefill(i32(prompt)); torch.cuda.synchronize()

@@ -437,6 +437,32 @@ trj_status trj_decode_device(trj_ctx* ctx, void* k_cache, void* v_cache, int32_t
                              int32_t R, int32_t branch_len, const int64_t* draws, int32_t n_steps,
                              int32_t* k_log, void* stream);
 
+/* The same loop over a static tree template with top-K siblings (Appendix B;
+ * template = parent [M] + rank [M] as for trj_refill_tree, HOST arrays; the rows
+ * of rank -1-j are one retrieval path of n_retrieved slots).  Per step, all on
+ * the device: the tree's tokens (root = the last committed token, the drafts
+ * the previous refill left, the retrieval path refreshed from the current
+ * context: slot j takes the j-th token after the most recent earlier occurrence
+ * of the context's last two tokens, then of its last token, else ahead noise),
+ * the verification forward, per-row top-K (K <= TRJ_MAX_TOPK) + acceptance, KV
+ * compaction, then commit and the refill rule of trj_refill_tree.
+ *   dev in/out: k_cache, v_cache, seq_len [1], context [capacity], *n_ctx as for
+ *               trj_decode_device; drafts [M - 1]: the draft tokens of rows
+ *               1 .. M-1 for the first step on entry (retrieval rows are
+ *               ignored), those for the next step on return
+ *   dev in    : draws [n_steps][M - 1 + n_retrieved] int64 >= 0: step i uses
+ *               row i, slots [0, M - 1) for its refill, the rest for the ahead
+ *               noise of its retrieval path
+ *   dev out   : k_log [n_steps] (may be null)
+ *   host      : parent, rank, n_ctx_now (every step commits at most the
+ *               template's depth + 1 tokens)
+ * Errors as trj_decode_device; a rank >= K or a retrieval slot >= n_retrieved
+ * is TRJ_EINVAL. */
+trj_status trj_decode_device_tree(trj_ctx* ctx, void* k_cache, void* v_cache, int32_t* seq_len, int32_t* context,
+                                  int32_t capacity, int32_t* n_ctx, int32_t n_ctx_now, const int32_t* parent,
+                                  const int32_t* rank, int32_t M, int32_t K, int32_t n_retrieved, int32_t* drafts,
+                                  const int64_t* draws, int32_t n_steps, int32_t* k_log, void* stream);
+
 /* An external source of drafts for trj_decode_device (Section 3.3: retrieved drafts get a path of their own; where
  * they are retrieved from is open).  stream [n] (dev int32) holds the source's guess for the token at context
  * position i in stream[i]; in step s of a later trj_decode_device call the first take[s] (dev int32 [n_steps],

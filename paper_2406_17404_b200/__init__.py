@@ -88,6 +88,7 @@ _SIGNATURES = {
     "trj_draft_tokens": (_I, [_VP, _VP, _VP, _I, _I, _I, _VP, _VP, _VP]),
     "trj_commit_refill": (_I, [_VP, _VP, _VP, _I, _VP, _VP, _VP, _VP, _I, _VP, _I, _VP, _VP, _VP, _VP]),
     "trj_decode_device": (_I, [_VP, _VP, _VP, _VP, _VP, _I, _VP, _I, _VP, _I, _I, _I, _VP, _I, _VP, _VP]),
+    "trj_decode_device_tree": (_I, [_VP, _VP, _VP, _VP, _VP, _I, _VP, _I, _I32P, _I32P, _I, _I, _I, _VP, _VP, _I, _VP, _VP]),
     "trj_set_draft_source": (_I, [_VP, _VP, _I, _VP, _I]),
     "trj_gemm_workspace": (_SZ, [_I, _I, _I]),
     "trj_gemm": (_I, [_VP, _VP, _VP, _I, _I, _I, _I, _VP, _SZ, _VP]),
@@ -632,6 +633,21 @@ class Model:
                                        _dev(window, torch.int32, "window") if w else None, w, n_branches, branch_len,
                                        _dev(draws, torch.int64, "draws"), int(n_steps),
                                        _dev(k_log, torch.int32, "k_log") if k_log is not None else None, _stream(stream)))
+
+    def decode_device_tree(self, context, n_ctx, n_ctx_now: int, parent, rank, top_k: int, n_retrieved: int, drafts,
+                           draws, n_steps: int, k_log=None, stream=None) -> None:
+        """trj_decode_device_tree: ``n_steps`` decode steps of sequence 0 over a static tree template with top-K
+        siblings, without the host in between.  parent / rank: host int arrays [M]; context int32 [capacity], n_ctx
+        int32 [1], drafts int32 [M - 1], draws int64 [n_steps, M - 1 + n_retrieved], k_log int32 [n_steps] or None:
+        CUDA tensors, updated in place."""
+        torch = _torch()
+        parent, rank = _i32(parent), _i32(rank)
+        _check(lib().trj_decode_device_tree(
+            self._handle, _dev(self.k_cache), _dev(self.v_cache), _dev(self.seq_len),
+            _dev(context, torch.int32, "context"), int(context.numel()), _dev(n_ctx, torch.int32, "n_ctx"), int(n_ctx_now),
+            _p32(parent), _p32(rank), len(parent), int(top_k), int(n_retrieved),
+            _dev(drafts, torch.int32, "drafts") if len(parent) > 1 else None, _dev(draws, torch.int64, "draws"), int(n_steps),
+            _dev(k_log, torch.int32, "k_log") if k_log is not None else None, _stream(stream)))
 
     def set_draft_source(self, stream=None, take=None) -> None:
         """trj_set_draft_source: ``stream`` int32 [n] guesses by context position, ``take`` int32 [n_steps] how many

@@ -182,6 +182,7 @@ struct trj_ctx {
     int32_t* chain_depth; uint64_t* chain_anc; int32_t* chunk_row_off; int32_t* unit_row_off; int32_t* prefill_geo;
     unsigned int* compact_tickets;   // device: one counter per sequence for the compaction kernel
     int32_t* loop_state;   // device: [0] step counter, [1] context-overflow flag of trj_decode_device
+    int32_t* loop_tree;    // device: rank [TRJ_MAX_ROWS] | retrieved tokens [TRJ_MAX_ROWS] | top-K table [TRJ_MAX_ROWS][TRJ_MAX_TOPK]
     int32_t* step_in;      // tokens | parent | depth | row_off(2) | pad -> anc
     int32_t* step_out;     // node_argmax | k_acc | bonus | path | device status words (projections, attention)
     int32_t* dev_status;   // the two status words at the end of step_out: TRJ_ETIMEOUT once a bounded wait expired
@@ -254,6 +255,7 @@ size_t carve(const trj_model_cfg& c, void* ws, trj_ctx* ctx) {
     int32_t* step_in = (int32_t*)cv.take<char>(STEP_IN_BYTES);
     int32_t* step_out = cv.take<int32_t>(STEP_OUT_INTS);
     int32_t* loop_state = cv.take<int32_t>(64);
+    int32_t* loop_tree = cv.take<int32_t>((size_t)TRJ_MAX_ROWS * (2 + TRJ_MAX_TOPK));
     unsigned int* compact_tickets = cv.take<unsigned int>(TRJ_MAX_BATCH);
     if (ctx) {
         ctx->h = h; ctx->y = y; ctx->logits = logits; ctx->x = x; ctx->q = q; ctx->act = act;
@@ -262,7 +264,7 @@ size_t carve(const trj_model_cfg& c, void* ws, trj_ctx* ctx) {
         ctx->gemm_ws = gemm_ws; ctx->gemm_ws_bytes = gemm_bytes;
         ctx->chain_depth = chain_depth; ctx->chain_anc = chain_anc; ctx->prefill_geo = prefill_geo;
         ctx->chunk_row_off = chunk_row_off; ctx->unit_row_off = unit_row_off;
-        ctx->step_in = step_in; ctx->step_out = step_out; ctx->loop_state = loop_state;
+        ctx->step_in = step_in; ctx->step_out = step_out; ctx->loop_state = loop_state; ctx->loop_tree = loop_tree;
         ctx->dev_status = step_out + STEP_STATUS_AT;
         ctx->compact_tickets = compact_tickets;
     }
@@ -916,6 +918,50 @@ extern "C" trj_status trj_set_draft_source(trj_ctx* ctx, const int32_t* stream, 
     return TRJ_OK;
 }
 
+namespace {
+
+// Runs n_steps of a device-resident decode loop whose single step `enqueue_one` puts on a stream.  The first step a
+// context ever runs is enqueued plainly (one-time set-up of the kernels happens outside any capture); so is
+// everything while profiling or without a capture stream.  Otherwise one step is captured once per key (every
+// pointer and size the step depends on) and the graph is launched once per step: the device step counter makes the
+// steps differ.
+template <typename EnqueueOne>
+trj_status run_device_loop(trj_ctx* ctx, const std::vector<uint64_t>& key, int32_t n_steps, EnqueueOne&& enqueue_one, cudaStream_t st) {
+    trj_status s = TRJ_OK;
+    int32_t done = 0;
+    const bool plain = ctx->prof_on || !ctx->cap_stream;
+    if (ctx->steps_done == 0 || plain) {
+        const int32_t n_plain = plain ? n_steps : 1;
+        for (; done < n_plain; ++done) {
+            s = enqueue_one(st);
+            if (s != TRJ_OK) return s;
+        }
+    }
+    if (done < n_steps) {
+        cudaGraphExec_t exec = nullptr;
+        for (const trj_ctx::LoopGraph& g : ctx->loop_graphs)
+            if (g.key == key) exec = g.exec;
+        if (!exec) {
+            cudaGraph_t graph = nullptr;
+            TRJ_CHECK_CUDA(cudaStreamBeginCapture(ctx->cap_stream, cudaStreamCaptureModeThreadLocal));
+            s = enqueue_one(ctx->cap_stream);
+            cudaError_t e = cudaStreamEndCapture(ctx->cap_stream, &graph);
+            if (s != TRJ_OK) { if (graph) cudaGraphDestroy(graph); return s; }
+            if (e != cudaSuccess) return fail(TRJ_ECUDA, "decode loop: graph capture: %s", cudaGetErrorString(e));
+            e = cudaGraphInstantiate(&exec, graph, 0);
+            cudaGraphDestroy(graph);
+            if (e != cudaSuccess) return fail(TRJ_ECUDA, "decode loop: graph instantiate: %s", cudaGetErrorString(e));
+            if (ctx->loop_graphs.size() >= 8) { cudaGraphExecDestroy(ctx->loop_graphs.front().exec); ctx->loop_graphs.erase(ctx->loop_graphs.begin()); }
+            ctx->loop_graphs.push_back({key, exec});
+        }
+        for (; done < n_steps; ++done) TRJ_CHECK_CUDA(cudaGraphLaunch(exec, st));
+    }
+    ctx->steps_done += n_steps;
+    return TRJ_OK;
+}
+
+}  // namespace
+
 extern "C" trj_status trj_decode_device(trj_ctx* ctx, void* k_cache, void* v_cache, int32_t* seq_len, int32_t* context,
                                         int32_t capacity, int32_t* n_ctx, int32_t n_ctx_now, int32_t* window, int32_t W,
                                         int32_t R, int32_t branch_len, const int64_t* draws, int32_t n_steps,
@@ -978,44 +1024,90 @@ extern "C" trj_status trj_decode_device(trj_ctx* ctx, void* k_cache, void* v_cac
                                                              n_ctx, W, W + R * branch_len, draws, d_step, window, k_log, d_overflow, on));
         return TRJ_OK;
     };
-    int32_t done = 0;
-    // The first step a context ever runs is enqueued plainly (one-time set-up of the kernels happens outside any
-    // capture); so is everything while profiling or without a capture stream.  Otherwise one step is captured once
-    // per key and the graph is launched once per step: the device step counter makes the steps differ.
-    const bool plain = ctx->prof_on || !ctx->cap_stream;
-    if (ctx->steps_done == 0 || plain) {
-        const int32_t n_plain = plain ? n_steps : 1;
-        for (; done < n_plain; ++done) {
-            s = enqueue_one(st);
-            if (s != TRJ_OK) return s;
-        }
-    }
-    if (done < n_steps) {
-        const std::vector<uint64_t> key = {(uint64_t)M, (uint64_t)tree_attention_grid(1, c.n_heads, (int32_t)max_len),
+    const std::vector<uint64_t> key_of_loop = {(uint64_t)0 /* window + branches */, (uint64_t)M, (uint64_t)tree_attention_grid(1, c.n_heads, (int32_t)max_len),
                                            (uint64_t)(uintptr_t)k_cache, (uint64_t)(uintptr_t)v_cache, (uint64_t)(uintptr_t)seq_len,
                                            (uint64_t)(uintptr_t)context, (uint64_t)capacity, (uint64_t)(uintptr_t)n_ctx,
                                            (uint64_t)(uintptr_t)window, (uint64_t)W, (uint64_t)R, (uint64_t)branch_len,
                                            (uint64_t)(uintptr_t)draws, (uint64_t)(uintptr_t)k_log, (uint64_t)max_len,
                                            (uint64_t)(uintptr_t)ctx->draft_src.stream, (uint64_t)ctx->draft_src.n,
                                            (uint64_t)(uintptr_t)ctx->draft_src.take};
-        cudaGraphExec_t exec = nullptr;
-        for (const trj_ctx::LoopGraph& g : ctx->loop_graphs)
-            if (g.key == key) exec = g.exec;
-        if (!exec) {
-            cudaGraph_t graph = nullptr;
-            TRJ_CHECK_CUDA(cudaStreamBeginCapture(ctx->cap_stream, cudaStreamCaptureModeThreadLocal));
-            s = enqueue_one(ctx->cap_stream);
-            cudaError_t e = cudaStreamEndCapture(ctx->cap_stream, &graph);
-            if (s != TRJ_OK) { if (graph) cudaGraphDestroy(graph); return s; }
-            if (e != cudaSuccess) return fail(TRJ_ECUDA, "decode_device: graph capture: %s", cudaGetErrorString(e));
-            e = cudaGraphInstantiate(&exec, graph, 0);
-            cudaGraphDestroy(graph);
-            if (e != cudaSuccess) return fail(TRJ_ECUDA, "decode_device: graph instantiate: %s", cudaGetErrorString(e));
-            if (ctx->loop_graphs.size() >= 8) { cudaGraphExecDestroy(ctx->loop_graphs.front().exec); ctx->loop_graphs.erase(ctx->loop_graphs.begin()); }
-            ctx->loop_graphs.push_back({key, exec});
-        }
-        for (; done < n_steps; ++done) TRJ_CHECK_CUDA(cudaGraphLaunch(exec, st));
-    }
-    ctx->steps_done += n_steps;
-    return TRJ_OK;
+    return run_device_loop(ctx, key_of_loop, n_steps, enqueue_one, st);
 }
+
+extern "C" trj_status trj_decode_device_tree(trj_ctx* ctx, void* k_cache, void* v_cache, int32_t* seq_len, int32_t* context,
+                                             int32_t capacity, int32_t* n_ctx, int32_t n_ctx_now, const int32_t* parent,
+                                             const int32_t* rank, int32_t M, int32_t K, int32_t n_retrieved, int32_t* drafts,
+                                             const int64_t* draws, int32_t n_steps, int32_t* k_log, void* stream) {
+    TRJ_REQUIRE(ctx, TRJ_EINVAL, "decode_device_tree: null context");
+    TRJ_REQUIRE(k_cache && v_cache && seq_len && context && n_ctx && parent && rank && draws, TRJ_EINVAL, "decode_device_tree: null pointer");
+    const trj_model_cfg& c = ctx->cfg;
+    TRJ_REQUIRE(M >= 1 && M <= c.max_rows && M <= TRJ_MAX_ROWS, TRJ_ECAPACITY, "decode_device_tree: %d tree rows outside 1..%d", M, c.max_rows);
+    TRJ_REQUIRE(M == 1 || drafts, TRJ_EINVAL, "decode_device_tree: null drafts");
+    TRJ_REQUIRE(K >= 1 && K <= TRJ_MAX_TOPK && K <= c.vocab, TRJ_EINVAL, "decode_device_tree: K = %d outside 1..%d", K, TRJ_MAX_TOPK);
+    TRJ_REQUIRE(n_retrieved >= 0 && n_retrieved < TRJ_MAX_ROWS && n_steps >= 0, TRJ_EINVAL, "decode_device_tree: bad sizes");
+    // the template on the host: depths, ancestor masks, and what the device kernels rely on without checking
+    int32_t* in = ctx->pin_in;
+    int32_t* h_parent = in + TRJ_MAX_ROWS, *h_depth = in + 2 * TRJ_MAX_ROWS, *h_off = in + 3 * TRJ_MAX_ROWS;
+    uint64_t* h_anc = (uint64_t*)(in + STEP_IN_INTS);
+    TRJ_REQUIRE(parent[0] == -1, TRJ_EINVAL, "decode_device_tree: row 0 must be the root");
+    for (int32_t i = 1; i < M; ++i)
+        TRJ_REQUIRE(parent[i] >= 0 && parent[i] < i, TRJ_EINVAL, "decode_device_tree: parent[%d] = %d is not an earlier row", i, parent[i]);
+    for (int32_t i = 0; i < M; ++i) h_parent[i] = parent[i];
+    trj_status s = tree_from_parents_impl(h_parent, M, 2, h_depth, h_anc);
+    if (s != TRJ_OK) return s;
+    int32_t deepest = 0;
+    for (int32_t i = 1; i < M; ++i) {
+        deepest = std::max(deepest, h_depth[i]);
+        TRJ_REQUIRE(rank[i] >= 0 ? rank[i] < K : -1 - rank[i] < n_retrieved, TRJ_EINVAL,
+                    "decode_device_tree: row %d has rank %d (K = %d, %d retrieval slots)", i, rank[i], K, n_retrieved);
+    }
+    const int32_t per_step = deepest + 1;        // a step commits at most the deepest path plus the bonus token
+    TRJ_REQUIRE(n_ctx_now >= 1, TRJ_EINVAL, "decode_device_tree: empty context");
+    TRJ_REQUIRE((int64_t)n_ctx_now + (int64_t)n_steps * per_step <= capacity, TRJ_ECAPACITY,
+                "decode_device_tree: context buffer of %d cannot take %d steps of up to %d tokens after %d", capacity, n_steps, per_step, n_ctx_now);
+    const int64_t max_len = (int64_t)n_ctx_now - 1 + (int64_t)n_steps * per_step + M;
+    TRJ_REQUIRE(max_len <= c.max_seq, TRJ_ECAPACITY, "decode_device_tree: up to %lld cache rows exceed max_seq %d", (long long)max_len, c.max_seq);
+    s = check_step_args(ctx, 1, M, M, (int32_t)max_len, 2);
+    if (s != TRJ_OK) return s;
+    if (n_steps == 0) return TRJ_OK;
+    cudaStream_t st = (cudaStream_t)stream;
+    h_off[0] = 0; h_off[1] = M;
+    // the ranks travel in the staging area's token slots (the tokens themselves are built on the device)
+    for (int32_t i = 0; i < M; ++i) in[i] = rank[i];
+    int32_t* d_rank = ctx->loop_tree, *d_retr = d_rank + TRJ_MAX_ROWS, *d_topk = d_retr + TRJ_MAX_ROWS;
+    TRJ_CHECK_CUDA(cudaMemcpyAsync(ctx->step_in, ctx->pin_in, STEP_IN_BYTES, cudaMemcpyHostToDevice, st));
+    TRJ_CHECK_CUDA(cudaMemcpyAsync(d_rank, ctx->step_in, sizeof(int32_t) * M, cudaMemcpyDeviceToDevice, st));
+    TRJ_CHECK_CUDA(cudaMemsetAsync(ctx->loop_state, 0, sizeof(int32_t) * 64, st));
+    // the pinned staging area is shared with trj_step_host: the copy must have left it before this call returns
+    TRJ_CHECK_CUDA(cudaEventRecord(ctx->order_ev, st));
+    TRJ_CHECK_CUDA(cudaEventSynchronize(ctx->order_ev));
+    int32_t* d_tokens = ctx->step_in, *d_parent = d_tokens + TRJ_MAX_ROWS, *d_depth = d_tokens + 2 * TRJ_MAX_ROWS;
+    int32_t* d_off = d_tokens + 3 * TRJ_MAX_ROWS;
+    uint64_t* d_anc = (uint64_t*)(d_tokens + STEP_IN_INTS);
+    int32_t* d_pred = ctx->step_out, *d_k = d_pred + TRJ_MAX_ROWS, *d_bonus = d_k + 1, *d_path = d_k + 2;
+    int32_t* d_step = ctx->loop_state, *d_overflow = ctx->loop_state + 1;
+    Batch bt{seq_len, d_off, 1, M, M, (int32_t)max_len};
+    auto enqueue_one = [&](cudaStream_t on) -> trj_status {
+        ChainScope chain;
+        LAUNCH_ON(on, PROF_ELEMENTWISE, launch_template_tokens(context, n_ctx, drafts, d_rank, M, n_retrieved, draws, d_step, d_tokens,
+                                                               d_retr, on));
+        trj_status fs = forward(ctx, k_cache, v_cache, 0, bt, d_tokens, d_depth, d_anc, 2, 0, M, on);
+        if (fs != TRJ_OK) return fs;
+        LAUNCH_ON(on, PROF_ARGMAX, launch_topk_accept(ctx->logits, TRJ_F32, c.vocab, K, d_tokens, d_parent, d_depth, d_off, 1, M, d_topk,
+                                                      d_pred, nullptr, d_k, d_path, d_bonus, true, ctx->argmax_ws, on));
+        LAUNCH_ON(on, PROF_COMPACT, launch_compact(k_cache, v_cache, c.n_layers, c.max_batch, 1, kv_heads(c), c.max_seq, c.head_dim,
+                                                   c.dtype, seq_len, d_k, d_path, on, ctx->compact_tickets));
+        LAUNCH_ON(on, PROF_ELEMENTWISE, launch_commit_refill_tree(d_tokens, d_parent, d_depth, d_rank, d_topk, K, M, d_k, d_path, d_bonus,
+                                                                  context, capacity, n_ctx, n_retrieved, draws, d_step, d_retr, drafts,
+                                                                  k_log, d_overflow, on));
+        return TRJ_OK;
+    };
+    const std::vector<uint64_t> key_of_loop = {(uint64_t)1 /* template */, (uint64_t)M, (uint64_t)K, (uint64_t)n_retrieved,
+                                               (uint64_t)tree_attention_grid(1, c.n_heads, (int32_t)max_len),
+                                               (uint64_t)(uintptr_t)k_cache, (uint64_t)(uintptr_t)v_cache, (uint64_t)(uintptr_t)seq_len,
+                                               (uint64_t)(uintptr_t)context, (uint64_t)capacity, (uint64_t)(uintptr_t)n_ctx,
+                                               (uint64_t)(uintptr_t)drafts, (uint64_t)(uintptr_t)draws, (uint64_t)(uintptr_t)k_log,
+                                               (uint64_t)max_len};
+    return run_device_loop(ctx, key_of_loop, n_steps, enqueue_one, st);
+}
+

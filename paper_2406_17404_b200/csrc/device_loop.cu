@@ -11,23 +11,9 @@ namespace {
 
 constexpr int MAX_BRANCHES = 64;          // R is bounded by the tree size (R * Lr < TRJ_MAX_ROWS)
 
-// tokens[0] = root (last committed token), tokens[1..W] = window, then R branches of Lr tokens: for each of the R
-// most recent earlier occurrences of the context's last two tokens (then of its last token), the Lr tokens that
-// followed; missing slots are ahead noise, context[draw % n].  `step` (may be null) selects this step's draws.
-// An external draft source (may be absent) overrides the start of branch 0: src.stream[i] is its guess for the token
-// at context position i, and step s takes src.take[s] of them, from position n on.
-__global__ void __launch_bounds__(32) draft_tokens_kernel(const int32_t* __restrict__ context, const int32_t* __restrict__ n_ctx,
-                                                          const int32_t* __restrict__ window, int W, int R, int Lr,
-                                                          const int64_t* __restrict__ draws, const int32_t* __restrict__ step,
-                                                          int32_t* __restrict__ tokens, const DraftSource src) {
-    pdl_prologue();
-    const int lane = threadIdx.x;
-    const int n = *n_ctx;
-    const int64_t* my_draws = draws + (step ? (size_t)*step * (size_t)(W + R * Lr) : 0);
-    if (lane == 0) tokens[0] = context[n - 1];
-    for (int i = lane; i < W; i += 32) tokens[1 + i] = window[i];
-    // every lane keeps the same list of follow positions (first index after a match), most recent match first
-    int follow[MAX_BRANCHES];
+// Prompt-lookup matches, by a whole warp: the positions that followed the R most recent earlier occurrences of the
+// context's last two tokens, then of its last token (no position twice).  Every lane ends up with the same list.
+__device__ __forceinline__ int find_follows(const int32_t* __restrict__ context, int n, int R, int* follow, int lane) {
     int nf = 0;
     for (int g = 2; g >= 1 && nf < R; --g) {
         if (n <= g) continue;
@@ -47,6 +33,27 @@ __global__ void __launch_bounds__(32) draft_tokens_kernel(const int32_t* __restr
             }
         }
     }
+    return nf;
+}
+
+// tokens[0] = root (last committed token), tokens[1..W] = window, then R branches of Lr tokens: for each of the R
+// most recent earlier occurrences of the context's last two tokens (then of its last token), the Lr tokens that
+// followed; missing slots are ahead noise, context[draw % n].  `step` (may be null) selects this step's draws.
+// An external draft source (may be absent) overrides the start of branch 0: src.stream[i] is its guess for the token
+// at context position i, and step s takes src.take[s] of them, from position n on.
+__global__ void __launch_bounds__(32) draft_tokens_kernel(const int32_t* __restrict__ context, const int32_t* __restrict__ n_ctx,
+                                                          const int32_t* __restrict__ window, int W, int R, int Lr,
+                                                          const int64_t* __restrict__ draws, const int32_t* __restrict__ step,
+                                                          int32_t* __restrict__ tokens, const DraftSource src) {
+    pdl_prologue();
+    const int lane = threadIdx.x;
+    const int n = *n_ctx;
+    const int64_t* my_draws = draws + (step ? (size_t)*step * (size_t)(W + R * Lr) : 0);
+    if (lane == 0) tokens[0] = context[n - 1];
+    for (int i = lane; i < W; i += 32) tokens[1 + i] = window[i];
+    // every lane keeps the same list of follow positions (first index after a match), most recent match first
+    int follow[MAX_BRANCHES];
+    const int nf = find_follows(context, n, R, follow, lane);
     for (int slot = lane; slot < R * Lr; slot += 32) {
         const int r = slot / Lr, j = slot % Lr;
         int32_t tok;
@@ -98,7 +105,106 @@ __global__ void __launch_bounds__(32) commit_refill_kernel(const int32_t* __rest
     }
 }
 
+// ---- static tree templates with top-K siblings (Appendix B) ----
+// The step's tree tokens: the root, the drafts the previous step's refill left, and the retrieval path (rows of rank
+// -1-j) refreshed from the current context: slot j takes the j-th token after the most recent earlier occurrence of
+// the context's last two tokens (then of its last token), or ahead noise context[draw % n] (Eq. 4).  The retrieved
+// tokens are kept in `retr` for the refill.  draws of step s: [0, M-1) refill, [M-1, M-1+n_retr) retrieval.
+__global__ void __launch_bounds__(32) template_tokens_kernel(const int32_t* __restrict__ context, const int32_t* __restrict__ n_ctx,
+                                                             const int32_t* __restrict__ drafts, const int32_t* __restrict__ rank,
+                                                             int M, int n_retr, const int64_t* __restrict__ draws,
+                                                             const int32_t* __restrict__ step, int32_t* __restrict__ tokens,
+                                                             int32_t* __restrict__ retr) {
+    pdl_prologue();
+    const int lane = threadIdx.x;
+    const int n = *n_ctx;
+    const int64_t* my_draws = draws + (size_t)*step * (size_t)(M - 1 + n_retr);
+    int follow[1];
+    const int nf = n_retr > 0 ? find_follows(context, n, 1, follow, lane) : 0;
+    for (int j = lane; j < n_retr; j += 32)
+        retr[j] = (nf > 0 && follow[0] + j < n) ? context[follow[0] + j] : context[(uint64_t)my_draws[M - 1 + j] % (uint64_t)n];
+    __syncwarp();
+    if (lane == 0) tokens[0] = context[n - 1];
+    for (int i = 1 + lane; i < M; i += 32) tokens[i] = rank[i] < 0 ? retr[-1 - rank[i]] : drafts[i - 1];
+}
+
+// After a step over a template: appends the accepted draft tokens and the bonus token to the context and writes the
+// next step's drafts.  Candidates for depth d come from the d-th row below the winner along its own path
+// (lowest-index child at every level): row i of depth d and rank r takes topk[that row][r]; depths the path does not
+// reach are ahead noise on the grown context; retrieval rows take this step's retrieved tokens.
+__global__ void __launch_bounds__(32) commit_refill_tree_kernel(const int32_t* __restrict__ tokens, const int32_t* __restrict__ parent,
+                                                                const int32_t* __restrict__ depth, const int32_t* __restrict__ rank,
+                                                                const int32_t* __restrict__ topk, int K, int M,
+                                                                const int32_t* __restrict__ k_acc, const int32_t* __restrict__ path,
+                                                                const int32_t* __restrict__ bonus, int32_t* __restrict__ context,
+                                                                int capacity, int32_t* __restrict__ n_ctx, int n_retr,
+                                                                const int64_t* __restrict__ draws, int32_t* __restrict__ step,
+                                                                const int32_t* __restrict__ retr, int32_t* __restrict__ drafts,
+                                                                int32_t* __restrict__ k_log, int32_t* __restrict__ overflow) {
+    pdl_prologue();
+    __shared__ int32_t below[TRJ_MAX_ROWS];
+    __shared__ int n_below_s;
+    const int lane = threadIdx.x;
+    const int n = *n_ctx, k = *k_acc;
+    const int s = *step;
+    const int64_t* my_draws = draws + (size_t)s * (size_t)(M - 1 + n_retr);
+    if (n + k + 1 > capacity) {
+        if (lane == 0 && overflow) *overflow = 1;
+        return;
+    }
+    for (int j = lane; j < k; j += 32) context[n + j] = tokens[path[j + 1]];
+    if (lane == 0) {
+        context[n + k] = *bonus;
+        int nb = 0;
+        for (int cur = path[k];;) {
+            int child = -1;
+            for (int c = cur + 1; c < M; ++c)
+                if (parent[c] == cur) { child = c; break; }
+            if (child < 0) break;
+            below[nb++] = child;
+            cur = child;
+        }
+        n_below_s = nb;
+    }
+    __syncwarp();
+    const int n_new = n + k + 1, n_below = n_below_s;
+    for (int i = 1 + lane; i < M; i += 32) {
+        const int r = rank[i];
+        int32_t tok;
+        if (r < 0) tok = retr[-1 - r];
+        else if (depth[i] <= n_below) tok = topk[(size_t)below[depth[i] - 1] * K + r];
+        else tok = context[(uint64_t)my_draws[i - 1] % (uint64_t)n_new];
+        drafts[i - 1] = tok;
+    }
+    __syncwarp();
+    if (lane == 0) {
+        *n_ctx = n_new;
+        if (k_log) k_log[s] = k;
+        *step = s + 1;
+    }
+}
+
 }  // namespace
+
+cudaError_t launch_template_tokens(const int32_t* context, const int32_t* n_ctx, const int32_t* drafts, const int32_t* rank,
+                                   int32_t M, int32_t n_retr, const int64_t* draws, const int32_t* step, int32_t* tokens,
+                                   int32_t* retr, cudaStream_t st) {
+    count_launch();
+    cudaError_t e = launch_chain(template_tokens_kernel, dim3(1), dim3(32), 0, st, context, n_ctx, drafts, rank, M, n_retr, draws, step,
+                                 tokens, retr);
+    return e != cudaSuccess ? e : cudaGetLastError();
+}
+
+cudaError_t launch_commit_refill_tree(const int32_t* tokens, const int32_t* parent, const int32_t* depth, const int32_t* rank,
+                                      const int32_t* topk, int32_t K, int32_t M, const int32_t* k_acc, const int32_t* path,
+                                      const int32_t* bonus, int32_t* context, int32_t capacity, int32_t* n_ctx, int32_t n_retr,
+                                      const int64_t* draws, int32_t* step, const int32_t* retr, int32_t* drafts, int32_t* k_log,
+                                      int32_t* overflow, cudaStream_t st) {
+    count_launch();
+    cudaError_t e = launch_chain(commit_refill_tree_kernel, dim3(1), dim3(32), 0, st, tokens, parent, depth, rank, topk, K, M, k_acc,
+                                 path, bonus, context, capacity, n_ctx, n_retr, draws, step, retr, drafts, k_log, overflow);
+    return e != cudaSuccess ? e : cudaGetLastError();
+}
 
 cudaError_t launch_draft_tokens(const int32_t* context, const int32_t* n_ctx, const int32_t* window, int32_t W, int32_t R,
                                 int32_t Lr, const int64_t* draws, const int32_t* step, int32_t* tokens, cudaStream_t st,

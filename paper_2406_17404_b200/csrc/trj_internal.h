@@ -178,6 +178,18 @@ cudaError_t launch_commit_refill(const int32_t* tokens, const int32_t* parent, c
                                  const int32_t* k_acc, const int32_t* path, const int32_t* bonus, int32_t* context,
                                  int32_t capacity, int32_t* n_ctx, int32_t W, int32_t draws_per_step, const int64_t* draws,
                                  int32_t* step, int32_t* window, int32_t* k_log, int32_t* overflow, cudaStream_t st);
+// The same two steps for a static tree template with top-K siblings (parent / depth / rank [M] on the device): the
+// tokens of a step (root, the drafts the previous refill left, the retrieval path refreshed from the context; the
+// retrieved tokens are kept in retr), and the commit + refill of the drafts from the per-row top-K table.  draws of
+// step s: draws[s][0 .. M-2] refill, draws[s][M-1 .. M-2+n_retr] retrieval.
+cudaError_t launch_template_tokens(const int32_t* context, const int32_t* n_ctx, const int32_t* drafts, const int32_t* rank,
+                                   int32_t M, int32_t n_retr, const int64_t* draws, const int32_t* step, int32_t* tokens,
+                                   int32_t* retr, cudaStream_t st);
+cudaError_t launch_commit_refill_tree(const int32_t* tokens, const int32_t* parent, const int32_t* depth, const int32_t* rank,
+                                      const int32_t* topk, int32_t K, int32_t M, const int32_t* k_acc, const int32_t* path,
+                                      const int32_t* bonus, int32_t* context, int32_t capacity, int32_t* n_ctx, int32_t n_retr,
+                                      const int64_t* draws, int32_t* step, const int32_t* retr, int32_t* drafts, int32_t* k_log,
+                                      int32_t* overflow, cudaStream_t st);
 
 // act[M][f] (dtype) = silu(gu[:, :f]) * gu[:, f:]
 cudaError_t launch_swiglu(const Parts& gu, void* act, void* act_lo, int32_t dtype, int32_t rows, int32_t f,

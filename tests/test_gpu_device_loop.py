@@ -232,3 +232,76 @@ def test_device_decode_loop_checks_capacity_on_the_host(trj):
     with pytest.raises(trj.TrjError):                       # 1 + 4 + 6 * 3 rows > max_rows 16
         model.decode_device(i32(np.zeros(400, np.int32)), d_n, 30, i32([1, 2, 3, 4]), 6, 3, i64(np.zeros((1, 22))), 1)
     model.close()
+
+
+def test_device_template_loop_equals_the_host_driven_loop_and_the_oracle(trj):
+    """A 69-row template with top-K siblings and a retrieval path (Appendix B), tiny fp32 model: the loop that stays
+    on the device (tokens, forward, top-K + acceptance, compaction, commit + refill from the top-K table) against
+    the host-driven loop over the same kernels (bit-exact: accepted counts, context, next drafts) and against the
+    oracle's template decoding (equal unless a near-tie fell the other way)."""
+    from paper_2406_17404_b200.decode import tr_jacobi_generate_tree
+    cfg = synth.TINY
+    model, dec = make_models(trj, cfg, 0, max_seq=512, max_rows=128)
+    prompt = synth.prompt(0, 64, cfg.vocab)
+    parent, rank = synth.tree_template(0)
+    m, top_k, n_retr, n_steps = len(parent), 10, 5, 12
+    draw = lambda s, n: synth.noise_draws(4, s, n)
+    # host-driven loop over the same kernels: its trace gives every step's accepted count and tokens
+    gtrace = []
+    tr_jacobi_generate_tree(model, prompt, 6 * n_steps, parent, rank, top_k, n_retr, draw, trace=gtrace)   # a step commits at most 6 tokens
+    assert len(gtrace) >= n_steps
+    gtrace = gtrace[:n_steps]
+    # the device loop from the same start
+    model.seq_len.zero_()
+    first = int(model.prefill(i32(prompt)).item())
+    committed = [int(t) for t in prompt] + [first]
+    depth = synth.node_depths(np.asarray(parent, np.int32))
+    capacity = len(committed) + n_steps * (int(depth.max()) + 1)
+    buf = np.zeros(capacity, np.int32); buf[:len(committed)] = committed
+    d_ctx, d_n = i32(buf), i32([len(committed)])
+    drafts = i32([committed[int(d) % len(committed)] for d in draw(0, m - 1)])
+    draws = i64(np.stack([np.asarray(draw(s, m - 1 + n_retr), np.int64) for s in range(1, n_steps + 1)]))
+    k_log = torch.full((n_steps,), -1, dtype=torch.int32, device="cuda")
+    model.decode_device_tree(d_ctx, d_n, len(committed), parent, rank, top_k, n_retr, drafts, draws, n_steps, k_log=k_log)
+    torch.cuda.synchronize()
+    model.device_status()
+    n_end = int(d_n[0])
+    got = d_ctx.cpu().numpy()[:n_end].tolist()
+    want_host = list(committed)
+    for rec in gtrace:
+        want_host += [int(rec["tokens"][r]) for r in rec["path"][1:]] + [rec["bonus"]]
+    assert k_log.cpu().tolist() == [rec["k_acc"] for rec in gtrace]
+    assert got == want_host
+    assert int(model.seq_len[0]) == n_end - 1
+    # the drafts left for the next step are what the host refill makes of the last step's top-K table
+    last = gtrace[-1]
+    retrieved = trj.retrieve(want_host[:len(want_host) - last["k_acc"] - 1], 1, n_retr, np.asarray(draw(n_steps, m - 1 + n_retr), np.int64)[m - 1:])[0]
+    want_drafts = trj.refill_tree(parent, rank, last["topk"], int(last["path"][-1]), want_host,
+                                  np.asarray(draw(n_steps, m - 1 + n_retr), np.int64)[:m - 1], retrieved)
+    np.testing.assert_array_equal(drafts.cpu().numpy(), want_drafts)
+    # and the oracle: greedy decoding commits the autoregressive tokens (Eq. 1)
+    want = oracle.autoregressive_greedy(dec, prompt, n_end - len(prompt))
+    if got[len(prompt):] != want:
+        trace = []
+        oracle.tr_jacobi_generate_tree(dec, prompt, n_end - len(prompt), parent, rank, top_k, n_retr, draw, trace=trace)
+        assert min(oracle.top2_margin(rec["logits"]).min() for rec in trace) < MARGIN
+    assert int(k_log.max()) >= 1
+    model.close()
+
+
+def test_device_template_loop_checks_the_template_on_the_host(trj):
+    cfg = synth.TINY
+    model, _ = make_models(trj, cfg, 0, max_seq=256, max_rows=32)
+    d_ctx, d_n = i32(np.zeros(200, np.int32)), i32([10])
+    drafts, draws = i32(np.zeros(3, np.int32)), i64(np.zeros((2, 4), np.int64))
+    good_parent, good_rank = [-1, 0, 0, 1], [0, 0, 1, -1]
+    for parent, rank, k, n_retr in (([-1, 0, 0, 3], good_rank, 2, 1),      # parent is not an earlier row
+                                   (good_parent, [0, 0, 2, -1], 2, 1),     # rank >= K
+                                   (good_parent, [0, 0, 1, -2], 2, 1),     # retrieval slot past n_retrieved
+                                   (good_parent, good_rank, 11, 1)):       # K past the limit
+        with pytest.raises(trj.TrjError):
+            model.decode_device_tree(d_ctx, d_n, 10, parent, rank, k, n_retr, drafts, draws, 2)
+    with pytest.raises(trj.TrjError):                                      # the context buffer cannot take the steps
+        model.decode_device_tree(i32(np.zeros(12, np.int32)), d_n, 10, good_parent, good_rank, 2, 1, drafts, draws, 2)
+    torch.cuda.synchronize()
+    model.close()
