@@ -38,8 +38,9 @@ struct TcParams {
     int block_rows;     // rows per block (the last block may hold fewer)
     int m_pad;          // rows of a block rounded up (8 with a lo half, else 16) = rows of the activation box
     int halves;         // 1: x only, 2: x and x_lo
-    int n_mma;          // accumulator columns = m_pad * halves, a multiple of 16
+    int n_mma;          // N of one product: m_pad * halves, or m_pad when the halves are summed in the accumulator; a multiple of 16
     int acc_cols;       // TMEM columns of one accumulator buffer: power of two >= max(16, n_mma); two are allocated
+    int pair_sum;       // hi and lo halves of a pair are two products into ONE accumulator (see tc_plan)
     int kblocks;        // ceil(K / 64)
     int tiles, splits, stages;
     float* out;         // [splits][M][N]
@@ -63,7 +64,7 @@ __global__ void __launch_bounds__(TC_THREADS, 2) gemm_tc_kernel(const __grid_con
     __shared__ int abort_flag;
 
     const uint32_t tiles_base = (smem_u32(smem_raw) + 1023u) & ~1023u;     // swizzled tiles need 1024-byte alignment
-    const uint32_t b_bytes = (uint32_t)p.n_mma * TC_BK * 2;
+    const uint32_t b_bytes = (uint32_t)(p.m_pad * p.halves) * TC_BK * 2;   // activation rows of a stage: hi tile, then lo tile
     const uint32_t stage_bytes = TC_A_BYTES + b_bytes;
     const uint32_t full0 = smem_u32(&bars[0]), empty0 = smem_u32(&bars[TC_MAX_STAGES]);
     const uint32_t acc_full0 = smem_u32(&bars[2 * TC_MAX_STAGES]), acc_empty0 = smem_u32(&bars[2 * TC_MAX_STAGES + 2]);
@@ -171,9 +172,19 @@ __global__ void __launch_bounds__(TC_THREADS, 2) gemm_tc_kernel(const __grid_con
                     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                     const uint32_t a_addr = tiles_base + s * stage_bytes;
                     const uint64_t a_desc = desc_kmajor_sw128(a_addr), b_desc = desc_kmajor_sw128(a_addr + TC_A_BYTES);
+                    if (!p.pair_sum) {
 #pragma unroll
-                    for (int kk = 0; kk < TC_BK / 16; ++kk)  // 16 bf16 = 32 bytes = 2 descriptor units per MMA
-                        umma_bf16(d_tmem, a_desc + 2 * kk, b_desc + 2 * kk, idesc, (i > 0 || kk > 0) ? 1u : 0u);
+                        for (int kk = 0; kk < TC_BK / 16; ++kk)  // 16 bf16 = 32 bytes = 2 descriptor units per MMA
+                            umma_bf16(d_tmem, a_desc + 2 * kk, b_desc + 2 * kk, idesc, (i > 0 || kk > 0) ? 1u : 0u);
+                    } else {
+                        // the low halves' tile lies m_pad rows of 128 bytes behind the high halves' tile
+                        const uint64_t lo_desc = desc_kmajor_sw128(a_addr + TC_A_BYTES + (uint32_t)p.m_pad * TC_BK * 2);
+#pragma unroll
+                        for (int kk = 0; kk < TC_BK / 16; ++kk) {
+                            umma_bf16(d_tmem, a_desc + 2 * kk, b_desc + 2 * kk, idesc, (i > 0 || kk > 0) ? 1u : 0u);
+                            umma_bf16(d_tmem, a_desc + 2 * kk, lo_desc + 2 * kk, idesc, 1u);
+                        }
+                    }
                     umma_commit(empty0 + 8 * s);             // frees the stage once these MMAs have read it
                 }
                 if (ok) umma_commit(acc_full0 + 8 * buf);    // accumulator of this item complete
@@ -199,12 +210,13 @@ __global__ void __launch_bounds__(TC_THREADS, 2) gemm_tc_kernel(const __grid_con
             for (int c0 = 0; c0 < p.m_pad; c0 += 8) {
                 float hi[8], lo[8];
                 tmem_ld8(taddr + c0, hi);
-                if (p.halves == 2) tmem_ld8(taddr + p.m_pad + c0, lo);
+                const bool two_halves = p.halves == 2 && !p.pair_sum;
+                if (two_halves) tmem_ld8(taddr + p.m_pad + c0, lo);
                 asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 #pragma unroll
                 for (int jj = 0; jj < 8; ++jj) {
                     const int m = row0 + c0 + jj;
-                    if (c0 + jj < p.block_rows && m < p.M && n < p.N) out[(size_t)m * p.N + n] = p.halves == 2 ? hi[jj] + lo[jj] : hi[jj];
+                    if (c0 + jj < p.block_rows && m < p.M && n < p.N) out[(size_t)m * p.N + n] = two_halves ? hi[jj] + lo[jj] : hi[jj];
                 }
             }
             asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
@@ -296,7 +308,7 @@ namespace {
 
 // Launch geometry of one projection.
 struct TcPlan {
-    int halves, m_blocks, block_rows, m_pad, n_mma, acc_cols, stages, grid_cap, tiles, kblocks, splits;
+    int halves, m_blocks, block_rows, m_pad, n_mma, acc_cols, stages, grid_cap, tiles, kblocks, splits, pair_sum;
     size_t stage_bytes;
 };
 
@@ -324,16 +336,24 @@ TcPlan tc_plan(int M, int N, int K, int halves, bool finished) {
     // an accumulator buffer holds 256 columns: 256 rows, or 128 rows as a hi + lo pair
     const int max_rows = halves == 2 ? 128 : 256, quantum = halves == 2 ? 8 : 16;
     pl.m_blocks = (M + max_rows - 1) / max_rows;
-    pl.block_rows = round_up((M + pl.m_blocks - 1) / pl.m_blocks, quantum);   // the lo box must start on a 1024-byte boundary: 8 rows
+    // A pair normally rides in one product whose accumulator holds the hi columns, then the lo columns, which the
+    // epilogue adds.  For 65-128 rows that accumulator would take 256 columns a buffer and leave room for one CTA per
+    // SM only; there the two halves are two products into the same 128 columns instead (twice the instructions and
+    // twice the shared-memory reads of the weight tile).
+    // Only where it buys the second CTA (three stages of both must fit: up to 80 rows); with one CTA per SM either
+    // way the single product is faster (96 rows: 4.9 against 5.8 ms per 7B step).
+    pl.pair_sum = (halves == 2 && pl.m_blocks == 1 && M > 64 &&
+                   3 * (TC_A_BYTES + (size_t)round_up(M, 16) * 2 * TC_BK * 2) <= 108 * 1024) ? 1 : 0;
+    pl.block_rows = round_up((M + pl.m_blocks - 1) / pl.m_blocks, pl.pair_sum ? 16 : quantum);   // the lo box must start on a 1024-byte boundary: 8 rows
     pl.m_pad = pl.block_rows;
-    pl.n_mma = pl.m_pad * halves;
+    pl.n_mma = pl.pair_sum ? pl.m_pad : pl.m_pad * halves;
     // the epilogue reads 8 columns at a time from each half, so a buffer must cover the last such read
-    const int reach = (halves == 2 ? pl.m_pad : 0) + round_up(pl.m_pad, 16);
+    const int reach = (halves == 2 && !pl.pair_sum ? pl.m_pad : 0) + round_up(pl.m_pad, 16);
     pl.acc_cols = 16;
     while (pl.acc_cols < reach) pl.acc_cols *= 2;
     pl.kblocks = (K + TC_BK - 1) / TC_BK;      // a ragged last block reads zeros past K (both operands)
     pl.tiles = (N + TC_BM - 1) / TC_BM;
-    pl.stage_bytes = TC_A_BYTES + (size_t)pl.n_mma * TC_BK * 2;
+    pl.stage_bytes = TC_A_BYTES + (size_t)pl.m_pad * halves * TC_BK * 2;
     // Two CTAs per SM (one's ramp and drain overlap the other's stream) when both fit: at least three stages in
     // ~108 KB each and both pairs of accumulator buffers in the 512 columns of tensor memory.  Otherwise one CTA
     // per SM with as deep a ring as shared memory allows.
@@ -375,7 +395,7 @@ cudaError_t launch_gemm_tc(const void* x, const void* x_lo, const void* w, float
     TcParams p;
     p.M = M; p.N = N; p.K = K;
     p.halves = pl.halves; p.m_blocks = pl.m_blocks; p.block_rows = pl.block_rows; p.m_pad = pl.m_pad;
-    p.n_mma = pl.n_mma; p.acc_cols = pl.acc_cols; p.kblocks = pl.kblocks; p.tiles = pl.tiles;
+    p.n_mma = pl.n_mma; p.acc_cols = pl.acc_cols; p.kblocks = pl.kblocks; p.tiles = pl.tiles; p.pair_sum = pl.pair_sum;
     p.splits = pl.splits; p.stages = pl.stages;
     p.out = p.splits > 1 ? (float*)workspace : y;
     p.status = status;
