@@ -619,6 +619,40 @@ def bench_tp_rank(trj, torch, synth, peaks, steps):
     return out
 
 
+def bench_batched_step(trj, torch, synth, cfg, layers, glob, peaks, steps, n_seq=8):
+    """The same verification step for `n_seq` independent sequences at once (each a 512-token prompt and a 33-row
+    tree): one forward over all rows, arg-max + acceptance per sequence, compaction of every cache.  The weights are
+    streamed once for all sequences, so this is the throughput side of the same kernels; not the headline metric."""
+    dev = torch.device("cuda", torch.cuda.current_device())
+    i32 = lambda a: torch.from_numpy(np.ascontiguousarray(a, dtype=np.int32)).to(dev)
+    model = trj.Model(cfg, layers, glob, max_batch=n_seq, max_seq=PROMPT + 64, max_rows=TREE_ROWS)
+    for b in range(n_seq):
+        model.prefill(i32(synth.prompt(300 + b, PROMPT, cfg.vocab)), b)
+    trees = [trj.build_tree(17 + b, synth.prompt(400 + b, WIDTH, cfg.vocab),
+                            synth.prompt(500 + b, N_BRANCHES * BRANCH_LEN, cfg.vocab).reshape(N_BRANCHES, BRANCH_LEN)) for b in range(n_seq)]
+    cat = lambda k: np.concatenate([t[k] for t in trees])
+    d_tok, d_par, d_dep = i32(cat("tokens")), i32(cat("parent")), i32(cat("depth"))
+    d_anc = torch.from_numpy(np.concatenate([t["anc"] for t in trees], 0).view(np.int64)).to(dev)
+    d_off = i32(np.arange(n_seq + 1) * TREE_ROWS)
+    rows = n_seq * TREE_ROWS
+    seq0 = model.seq_len.clone()
+    pred = torch.empty(rows, dtype=torch.int32, device=dev)
+    acc = {"k_acc": torch.empty(n_seq, dtype=torch.int32, device=dev), "bonus": torch.empty(n_seq, dtype=torch.int32, device=dev),
+           "path": torch.empty(n_seq, trj.PATH_STRIDE, dtype=torch.int32, device=dev)}
+
+    def step():
+        model.seq_len.copy_(seq0)
+        model.verify_step(d_tok, d_par, d_dep, d_anc, d_off, max_rows=TREE_ROWS, max_len=PROMPT + TREE_ROWS, node_argmax=pred)
+        model.accept(d_tok, d_par, d_dep, d_off, pred, out=acc)
+        model.compact_kv(acc["k_acc"], acc["path"], batch=n_seq)
+    us = graph_us(torch, step, steps, 3)
+    model.device_status()
+    model.close()
+    return {"sequences": n_seq, "tree_rows_each": TREE_ROWS, "prefix": PROMPT, "ms_per_step": us / 1e3,
+            "draft_tokens_verified_per_s": n_seq * DRAFTS / (us / 1e6),
+            "what": "%d independent sequences in one step (7B shape); random drafts" % n_seq}
+
+
 def bench_prefill_gemm(trj, torch, peaks, steps):
     """The four projections of the 7B shape on prompt-sized row counts (the tensor-bound side of the projection
     kernel: 128 x 256 tiles), as a stand-alone op: TFLOP/s against the measured dense bf16 peak."""
@@ -924,6 +958,7 @@ def run_ours(args, rank, world, local_rank):
             line["prefill_gemm"] = bench_prefill_gemm(trj, torch, peaks, max(args.steps // 2, 5))
             line["llama3_8b_step"] = bench_llama3_step(trj, torch, synth, peaks, max(args.steps // 2, 5))
             line["tensor_parallel_rank"] = bench_tp_rank(trj, torch, synth, peaks, max(args.steps // 2, 5))
+            line["batched_step"] = bench_batched_step(trj, torch, synth, cfg, layers, glob, peaks, max(args.steps // 2, 5))
         if not args.no_attention:
             line["tree_attention"] = bench_tree_attention(trj, torch, peaks, max(args.steps, 5), 3, cpu=not args.no_cpu)
             line["small_ops"] = bench_small_ops(trj, torch, peaks, max(args.steps, 5), 3, cpu=not args.no_cpu)
