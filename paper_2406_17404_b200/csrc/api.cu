@@ -182,6 +182,8 @@ struct trj_ctx {
     int32_t* chain_depth; uint64_t* chain_anc; int32_t* chunk_row_off; int32_t* unit_row_off; int32_t* prefill_geo;
     unsigned int* compact_tickets;   // device: one counter per sequence for the compaction kernel
     int32_t* loop_state;   // device: [0] step counter, [1] context-overflow flag of trj_decode_device
+    TopEntry* top_table; int32_t top_table_rows;   // arg-max candidates left by the LM head's epilogue, and how many rows it may hold
+    int32_t lm_table_rows = 0;   // rows whose candidates the latest forward left there (0: it wrote logits only)
     int32_t* loop_tree;    // device: rank [TRJ_MAX_ROWS] | retrieved tokens [TRJ_MAX_ROWS] | top-K table [TRJ_MAX_ROWS][TRJ_MAX_TOPK]
     int32_t* step_in;      // tokens | parent | depth | row_off(2) | pad -> anc
     int32_t* step_out;     // node_argmax | k_acc | bonus | path | device status words (projections, attention)
@@ -256,6 +258,8 @@ size_t carve(const trj_model_cfg& c, void* ws, trj_ctx* ctx) {
     int32_t* step_out = cv.take<int32_t>(STEP_OUT_INTS);
     int32_t* loop_state = cv.take<int32_t>(64);
     int32_t* loop_tree = cv.take<int32_t>((size_t)TRJ_MAX_ROWS * (2 + TRJ_MAX_TOPK));
+    const int top_rows = std::min(step_rows, 128);
+    TopEntry* top_table = cv.take<TopEntry>(gemm_top_table_entries(top_rows, c.vocab));
     unsigned int* compact_tickets = cv.take<unsigned int>(TRJ_MAX_BATCH);
     if (ctx) {
         ctx->h = h; ctx->y = y; ctx->logits = logits; ctx->x = x; ctx->q = q; ctx->act = act;
@@ -264,7 +268,7 @@ size_t carve(const trj_model_cfg& c, void* ws, trj_ctx* ctx) {
         ctx->gemm_ws = gemm_ws; ctx->gemm_ws_bytes = gemm_bytes;
         ctx->chain_depth = chain_depth; ctx->chain_anc = chain_anc; ctx->prefill_geo = prefill_geo;
         ctx->chunk_row_off = chunk_row_off; ctx->unit_row_off = unit_row_off;
-        ctx->step_in = step_in; ctx->step_out = step_out; ctx->loop_state = loop_state; ctx->loop_tree = loop_tree;
+        ctx->step_in = step_in; ctx->step_out = step_out; ctx->loop_state = loop_state; ctx->loop_tree = loop_tree; ctx->top_table = top_table; ctx->top_table_rows = top_rows;
         ctx->dev_status = step_out + STEP_STATUS_AT;
         ctx->compact_tickets = compact_tickets;
     }
@@ -329,6 +333,7 @@ struct StepArgs {
     void* k_cache; void* v_cache; int32_t b0; Batch bt;
     const int32_t* tokens; const int32_t* depth; const uint64_t* anc; int32_t anc_words;
     int32_t lm_first, lm_rows; const SubChunks* pieces;
+    int32_t lm_mode;   // 0: logits; 1: logits and the arg-max candidates of the epilogue; 2: the candidates only
 };
 
 // The decoder as 2 L + 1 segments: 2 l is the attention half of layer l (norm, QKV, rotary + cache write, tree
@@ -361,9 +366,16 @@ trj_status run_segments(trj_ctx* ctx, const StepArgs& a, int s0, int s1, Parts& 
                 const size_t off = (size_t)a.lm_first * d * es;
                 // a verification step keeps every row's logits in place; prefill wants one row and gets it in row 0
                 float* lm_out = pieces ? ctx->logits : ctx->logits + (size_t)a.lm_first * c.vocab;
+                // Eq. 1 needs every row's arg-max, not its logits: when the caller says so and the launch keeps all of
+                // a row's partial sums in one accumulator, the epilogue leaves one candidate per 32 outputs and the
+                // logits are written only if they are wanted as well
+                const bool table = a.lm_mode != 0 && !pieces && a.lm_first == 0 && a.lm_rows == M && M <= ctx->top_table_rows &&
+                                   gemm_top_table_ok(M, c.vocab, d, c.dtype, ctx->x_lo != nullptr);
+                const TopTable top{ctx->top_table, a.lm_mode == 2 ? 0 : 1};
+                ctx->lm_table_rows = table ? M : 0;
                 LAUNCH(PROF_GEMM, launch_gemm((char*)ctx->x + off, ctx->x_lo ? (char*)ctx->x_lo + off : nullptr, ctx->lm_head,
                                               lm_out, a.lm_rows, c.vocab, d, c.dtype,
-                                              ctx->gemm_ws, ctx->gemm_ws_bytes, st, nullptr, nullptr, gemm_status));
+                                              ctx->gemm_ws, ctx->gemm_ws_bytes, st, nullptr, nullptr, gemm_status, table ? &top : nullptr));
             }
         } else if ((s & 1) == 0) {
             char* k_slab = (char*)a.k_cache + ((size_t)l * c.max_batch + a.b0) * seq_stride;
@@ -414,13 +426,25 @@ trj_status run_segments(trj_ctx* ctx, const StepArgs& a, int s0, int s1, Parts& 
 // One forward of the decoder over the rows of `bt`: embedding, then every segment.
 trj_status forward(trj_ctx* ctx, void* k_cache, void* v_cache, int32_t b0, const Batch& bt,
                    const int32_t* tokens, const int32_t* depth, const uint64_t* anc, int32_t anc_words,
-                   int32_t lm_first, int32_t lm_rows, cudaStream_t st, const SubChunks* pieces = nullptr) {
+                   int32_t lm_first, int32_t lm_rows, cudaStream_t st, const SubChunks* pieces = nullptr, int32_t lm_mode = 0) {
     ChainScope chain;                        // the embedding below is the chain's fence
     const trj_model_cfg& c = ctx->cfg;
     LAUNCH(PROF_ELEMENTWISE, launch_embed(ctx->embed, c.dtype, tokens, ctx->h, bt.rows_total, c.d_model, st));
     Parts pr{nullptr, 1, 0};                 // result of the latest projection, possibly in split-K pieces
-    const StepArgs a{k_cache, v_cache, b0, bt, tokens, depth, anc, anc_words, lm_first, lm_rows, pieces};
+    const StepArgs a{k_cache, v_cache, b0, bt, tokens, depth, anc, anc_words, lm_first, lm_rows, pieces, lm_mode};
     return run_segments(ctx, a, 0, 2 * c.n_layers + 1, pr, false, st);
+}
+
+// Arg-max (and, when asked, acceptance) of the rows the latest forward scored: from the candidates the LM head's
+// epilogue left, or from the logits.
+cudaError_t step_argmax(trj_ctx* ctx, const int32_t* tokens, const int32_t* parent, const int32_t* depth, const int32_t* row_off,
+                        int32_t B, int32_t rows, int32_t* node_argmax, float* margin, int32_t* k_acc, int32_t* path, int32_t* bonus,
+                        bool do_accept, cudaStream_t st) {
+    if (ctx->lm_table_rows == rows)
+        return launch_argmax_table_accept(ctx->top_table, (int32_t)(gemm_top_table_entries(1, ctx->cfg.vocab)), tokens, parent, depth,
+                                          row_off, B, rows, node_argmax, margin, k_acc, path, bonus, do_accept, ctx->argmax_ws, st);
+    return launch_topk_accept(ctx->logits, TRJ_F32, ctx->cfg.vocab, 1, tokens, parent, depth, row_off, B, rows, nullptr, node_argmax,
+                              margin, k_acc, path, bonus, do_accept, ctx->argmax_ws, st);
 }
 
 trj_status check_step_args(const trj_ctx* ctx, int32_t B, int32_t rows_total, int32_t max_rows, int32_t max_len,
@@ -633,11 +657,11 @@ extern "C" trj_status trj_verify_step(trj_ctx* ctx, void* k_cache, void* v_cache
     cudaStream_t st = (cudaStream_t)stream;
     ChainScope chain;
     Batch bt{seq_len, row_off, B, rows_total, max_rows, max_len};
-    s = forward(ctx, k_cache, v_cache, 0, bt, tokens, depth, anc, anc_words, 0, rows_total, st);
+    // the logits stay materialised: the caller may ask for them here or for their top-K afterwards (trj_node_topk)
+    s = forward(ctx, k_cache, v_cache, 0, bt, tokens, depth, anc, anc_words, 0, rows_total, st, nullptr, 1);
     if (s != TRJ_OK) return s;
-    LAUNCH(PROF_ARGMAX, launch_topk_accept(ctx->logits, TRJ_F32, ctx->cfg.vocab, 1, tokens, parent, depth, row_off, B,
-                                           rows_total, nullptr, node_argmax, margin, nullptr, nullptr, nullptr, false,
-                                           ctx->argmax_ws, st));
+    LAUNCH(PROF_ARGMAX, step_argmax(ctx, tokens, parent, depth, row_off, B, rows_total, node_argmax, margin, nullptr, nullptr, nullptr,
+                                    false, st));
     ctx->last_rows = rows_total; ctx->last_row_off = row_off; ctx->last_B = B;
     if (logits)
         TRJ_CHECK_CUDA(cudaMemcpyAsync(logits, ctx->logits, sizeof(float) * (size_t)rows_total * ctx->cfg.vocab,
@@ -676,7 +700,7 @@ extern "C" trj_status trj_tp_segment(trj_ctx* ctx, int32_t segment, void* stream
     cudaStream_t st = (cudaStream_t)stream;
     ChainScope chain;
     const trj_ctx::TpStep& t = ctx->tp;
-    const StepArgs a{t.k_cache, t.v_cache, 0, t.bt, t.tokens, t.depth, t.anc, t.anc_words, 0, t.bt.rows_total, nullptr};
+    const StepArgs a{t.k_cache, t.v_cache, 0, t.bt, t.tokens, t.depth, t.anc, t.anc_words, 0, t.bt.rows_total, nullptr, 0};
     // what the previous segment left, summed over the ranks by the caller, sits in the exchange buffer
     Parts pr = segment == 0 ? Parts{nullptr, 1, 0} : whole(ctx->y);
     trj_status s = run_segments(ctx, a, segment, segment + 1, pr, segment + 1 < n_seg, st);
@@ -800,10 +824,9 @@ trj_status enqueue_step(trj_ctx* ctx, void* k_cache, void* v_cache, int32_t* seq
     uint64_t* d_anc = (uint64_t*)(d_tokens + STEP_IN_INTS);
     int32_t* d_pred = ctx->step_out, *d_k = d_pred + TRJ_MAX_ROWS, *d_bonus = d_k + 1, *d_path = d_k + 2;
     Batch bt{seq_len, d_off, 1, M, M, max_len};
-    trj_status s = forward(ctx, k_cache, v_cache, 0, bt, d_tokens, d_depth, d_anc, 2, 0, M, st);
+    trj_status s = forward(ctx, k_cache, v_cache, 0, bt, d_tokens, d_depth, d_anc, 2, 0, M, st, nullptr, 2);   // nobody reads this step's logits
     if (s != TRJ_OK) return s;
-    LAUNCH(PROF_ARGMAX, launch_topk_accept(ctx->logits, TRJ_F32, c.vocab, 1, d_tokens, d_parent, d_depth, d_off, 1, M, nullptr, d_pred,
-                                           nullptr, d_k, d_path, d_bonus, true, ctx->argmax_ws, st));
+    LAUNCH(PROF_ARGMAX, step_argmax(ctx, d_tokens, d_parent, d_depth, d_off, 1, M, d_pred, nullptr, d_k, d_path, d_bonus, true, st));
     LAUNCH(PROF_COMPACT, launch_compact(k_cache, v_cache, c.n_layers, c.max_batch, 1, kv_heads(c), c.max_seq, c.head_dim,
                                         c.dtype, seq_len, d_k, d_path, st, ctx->compact_tickets));
     TRJ_CHECK_CUDA(cudaMemcpyAsync(ctx->pin_out, ctx->step_out, sizeof(int32_t) * STEP_OUT_INTS, cudaMemcpyDeviceToHost, st));
@@ -1014,10 +1037,9 @@ extern "C" trj_status trj_decode_device(trj_ctx* ctx, void* k_cache, void* v_cac
         ChainScope chain;
         LAUNCH_ON(on, PROF_ELEMENTWISE, launch_draft_tokens(context, n_ctx, window, W, R, branch_len, draws, d_step, d_tokens, on,
                                                             ctx->draft_src));
-        trj_status fs = forward(ctx, k_cache, v_cache, 0, bt, d_tokens, d_depth, d_anc, 2, 0, M, on);
+        trj_status fs = forward(ctx, k_cache, v_cache, 0, bt, d_tokens, d_depth, d_anc, 2, 0, M, on, nullptr, 2);
         if (fs != TRJ_OK) return fs;
-        LAUNCH_ON(on, PROF_ARGMAX, launch_topk_accept(ctx->logits, TRJ_F32, c.vocab, 1, d_tokens, d_parent, d_depth, d_off, 1, M, nullptr,
-                                                      d_pred, nullptr, d_k, d_path, d_bonus, true, ctx->argmax_ws, on));
+        LAUNCH_ON(on, PROF_ARGMAX, step_argmax(ctx, d_tokens, d_parent, d_depth, d_off, 1, M, d_pred, nullptr, d_k, d_path, d_bonus, true, on));
         LAUNCH_ON(on, PROF_COMPACT, launch_compact(k_cache, v_cache, c.n_layers, c.max_batch, 1, kv_heads(c), c.max_seq, c.head_dim,
                                                    c.dtype, seq_len, d_k, d_path, on, ctx->compact_tickets));
         LAUNCH_ON(on, PROF_ELEMENTWISE, launch_commit_refill(d_tokens, d_parent, d_pred, M, d_k, d_path, d_bonus, context, capacity,

@@ -40,6 +40,8 @@ struct TcParams {
     int halves;         // 1: x only, 2: x and x_lo
     int n_mma;          // N of one product: m_pad * halves, or m_pad when the halves are summed in the accumulator; a multiple of 16
     int acc_cols;       // TMEM columns of one accumulator buffer: power of two >= max(16, n_mma); two are allocated
+    TopEntry* top;      // arg-max table of the epilogue (may be null); store_y == 0: the outputs themselves are not written
+    int store_y;
     int pair_sum;       // hi and lo halves of a pair are two products into ONE accumulator (see tc_plan)
     int kblocks;        // ceil(K / 64)
     int tiles, splits, stages;
@@ -54,6 +56,9 @@ using namespace sm100;
 // restricted to one K range (tile = item / splits, split = item % splits).  The TMA ring runs through item
 // boundaries, and the accumulator is double-buffered in TMEM so that the epilogue of one item overlaps the
 // loads and MMAs of the next.  Warp 0: TMA producer, warp 1: MMA issuer, warps 2-5: epilogue.
+// TOP: the epilogue also leaves arg-max candidates (the LM head of a verification step); the plain instantiation
+// carries none of that code (the epilogue's instruction schedule is on every projection's critical path).
+template <bool TOP>
 __global__ void __launch_bounds__(TC_THREADS, 2) gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w,
                                                                 const __grid_constant__ CUtensorMap map_x,
                                                                 const __grid_constant__ CUtensorMap map_xlo, const __grid_constant__ CUtensorMap map_ahead,
@@ -213,10 +218,43 @@ __global__ void __launch_bounds__(TC_THREADS, 2) gemm_tc_kernel(const __grid_con
                 const bool two_halves = p.halves == 2 && !p.pair_sum;
                 if (two_halves) tmem_ld8(taddr + p.m_pad + c0, lo);
                 asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+                if (!TOP || p.store_y) {
 #pragma unroll
-                for (int jj = 0; jj < 8; ++jj) {
-                    const int m = row0 + c0 + jj;
-                    if (c0 + jj < p.block_rows && m < p.M && n < p.N) out[(size_t)m * p.N + n] = two_halves ? hi[jj] + lo[jj] : hi[jj];
+                    for (int jj = 0; jj < 8; ++jj) {
+                        const int m = row0 + c0 + jj;
+                        if (c0 + jj < p.block_rows && m < p.M && n < p.N) out[(size_t)m * p.N + n] = two_halves ? hi[jj] + lo[jj] : hi[jj];
+                    }
+                }
+                if constexpr (TOP) {
+                    if (two_halves) {
+#pragma unroll
+                        for (int jj = 0; jj < 8; ++jj) hi[jj] += lo[jj];
+                    }
+                    // this warp's 32 outputs of every row: best value, its index (ties: the smaller index), runner-up
+                    float v1[8], v2[8];
+                    int i1[8];
+#pragma unroll
+                    for (int jj = 0; jj < 8; ++jj) { v1[jj] = n < p.N ? hi[jj] : -INFINITY; i1[jj] = n < p.N ? n : 0x7fffffff; v2[jj] = -INFINITY; }
+#pragma unroll
+                    for (int o = 16; o > 0; o >>= 1) {
+#pragma unroll
+                        for (int jj = 0; jj < 8; ++jj) {
+                            const float ov1 = __shfl_xor_sync(0xffffffffu, v1[jj], o), ov2 = __shfl_xor_sync(0xffffffffu, v2[jj], o);
+                            const int oi1 = __shfl_xor_sync(0xffffffffu, i1[jj], o);
+                            const bool mine = v1[jj] > ov1 || (v1[jj] == ov1 && i1[jj] < oi1);
+                            v2[jj] = fmaxf(mine ? ov1 : v1[jj], fmaxf(v2[jj], ov2));
+                            v1[jj] = mine ? v1[jj] : ov1;
+                            i1[jj] = mine ? i1[jj] : oi1;
+                        }
+                    }
+                    if (lane == 0) {
+#pragma unroll
+                        for (int jj = 0; jj < 8; ++jj) {
+                            const int m = row0 + c0 + jj;
+                            if (c0 + jj < p.block_rows && m < p.M)
+                                p.top[((size_t)m * p.tiles + tile) * 4 + q] = TopEntry{v1[jj], i1[jj], v2[jj]};
+                        }
+                    }
                 }
             }
             asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
@@ -381,13 +419,16 @@ size_t gemm_tc_workspace(int32_t M, int32_t N, int32_t K) {
 }
 
 cudaError_t launch_gemm_tc(const void* x, const void* x_lo, const void* w, float* y, int32_t M, int32_t N, int32_t K,
-                           void* workspace, cudaStream_t st, Parts* parts, const WeightPrefetch* ahead, int* status) {
+                           void* workspace, cudaStream_t st, Parts* parts, const WeightPrefetch* ahead, int* status,
+                           const TopTable* top) {
     if (!status) status = (int*)workspace;
     workspace = (char*)workspace + 256;
     static std::once_flag once;
     static cudaError_t attr_err = cudaSuccess;
     std::call_once(once, [] {
-        attr_err = cudaFuncSetAttribute(gemm_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024);
+        attr_err = cudaFuncSetAttribute(gemm_tc_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024);
+        if (attr_err == cudaSuccess)
+            attr_err = cudaFuncSetAttribute(gemm_tc_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024);
     });
     if (attr_err != cudaSuccess) return attr_err;
     const TcPlan pl = tc_plan(M, N, K, x_lo ? 2 : 1, parts == nullptr);
@@ -397,6 +438,11 @@ cudaError_t launch_gemm_tc(const void* x, const void* x_lo, const void* w, float
     p.halves = pl.halves; p.m_blocks = pl.m_blocks; p.block_rows = pl.block_rows; p.m_pad = pl.m_pad;
     p.n_mma = pl.n_mma; p.acc_cols = pl.acc_cols; p.kblocks = pl.kblocks; p.tiles = pl.tiles; p.pair_sum = pl.pair_sum;
     p.splits = pl.splits; p.stages = pl.stages;
+    p.top = nullptr; p.store_y = 1;
+    if (top) {                                               // the accumulator must hold finished sums of all rows
+        if (!top->entries || parts || pl.splits != 1 || pl.m_blocks != 1) return cudaErrorInvalidValue;
+        p.top = top->entries; p.store_y = top->store_y;
+    }
     p.out = p.splits > 1 ? (float*)workspace : y;
     p.status = status;
     CUtensorMap map_w, map_x, map_xlo, map_ahead;
@@ -417,8 +463,8 @@ cudaError_t launch_gemm_tc(const void* x, const void* x_lo, const void* w, float
     if (!want_ahead) map_ahead = map_w;                      // never used: no CTA asks
     count_launch();
     const int items = p.tiles * p.m_blocks * p.splits;
-    cudaError_t e = launch_chain(gemm_tc_kernel, dim3(items < pl.grid_cap ? items : pl.grid_cap), dim3(TC_THREADS),
-                                 p.stages * pl.stage_bytes + 1024, st, map_w, map_x, map_xlo, map_ahead, p);
+    cudaError_t e = launch_chain(p.top ? gemm_tc_kernel<true> : gemm_tc_kernel<false>, dim3(items < pl.grid_cap ? items : pl.grid_cap),
+                                 dim3(TC_THREADS), p.stages * pl.stage_bytes + 1024, st, map_w, map_x, map_xlo, map_ahead, p);
     if (e == cudaSuccess) e = cudaGetLastError();
     if (parts) *parts = Parts{p.out, p.splits, (size_t)M * N};
     if (e != cudaSuccess || p.splits == 1 || parts) return e;
@@ -441,19 +487,26 @@ cudaError_t launch_wait_expiry_selftest(int* status, uint32_t polls, cudaStream_
     return cudaGetLastError();
 }
 
+bool gemm_top_table_ok(int32_t M, int32_t N, int32_t K, int32_t dtype, bool pair) {
+    if (!gemm_tc_shape(M, N, K, dtype)) return false;
+    const TcPlan pl = tc_plan(M, N, K, pair ? 2 : 1, true);
+    return pl.splits == 1 && pl.m_blocks == 1 && pl.stages >= 2;
+}
+
 bool gemm_tc_shape(int32_t M, int32_t N, int32_t K, int32_t dtype) {
     return dtype == TRJ_BF16 && M >= 1 && K >= TC_BK && K % 8 == 0 && N >= 4 && N % 4 == 0;
 }
 
 cudaError_t launch_gemm(const void* x, const void* x_lo, const void* w, float* y, int32_t M, int32_t N, int32_t K,
                         int32_t dtype, void* workspace, size_t workspace_bytes, cudaStream_t st, Parts* parts,
-                        const WeightPrefetch* ahead, int* status) {
+                        const WeightPrefetch* ahead, int* status, const TopTable* top) {
     if (gemm_tc_shape(M, N, K, dtype)) {
         if (!workspace || workspace_bytes < gemm_tc_workspace(M, N, K) || ((uintptr_t)workspace % 256) != 0 ||
             !gemm_tc_supported(x, x_lo, w, y, M, N, K, dtype))
             return cudaErrorInvalidValue;
-        return launch_gemm_tc(x, x_lo, w, y, M, N, K, workspace, st, parts, ahead, status);
+        return launch_gemm_tc(x, x_lo, w, y, M, N, K, workspace, st, parts, ahead, status, top);
     }
+    if (top) return cudaErrorInvalidValue;                   // the caller asks gemm_top_table_ok first
     if (parts) *parts = whole(y);
     return launch_gemm_simt(x, x_lo, w, y, M, N, K, dtype, st);
 }

@@ -829,6 +829,47 @@ __global__ void __launch_bounds__(TOPK_THREADS) argmax_row_accept_kernel(
                     k_acc + b, path + (size_t)b * TRJ_PATH_STRIDE, bonus + b);
 }
 
+// Arg-max of every row from the candidates a projection's epilogue left (one per 32 outputs), then acceptance as above.
+__global__ void __launch_bounds__(128) argmax_table_accept_kernel(
+        const TopEntry* __restrict__ table, int per_row, const int32_t* __restrict__ tokens,
+        const int32_t* __restrict__ parent, const int32_t* __restrict__ depth,
+        const int32_t* __restrict__ row_off, int B, int32_t* node_argmax,
+        float* __restrict__ margin, int32_t* __restrict__ k_acc, int32_t* __restrict__ path,
+        int32_t* __restrict__ bonus, int do_accept, unsigned int* tickets) {
+    pdl_prologue();
+    __shared__ Top red[4];
+    __shared__ int last_flag;
+    const int row = blockIdx.x, warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const TopEntry* tr = table + (size_t)row * per_row;
+    Top t{-INFINITY, 0x7fffffff, -INFINITY};
+    for (int i = threadIdx.x; i < per_row; i += 128) {
+        const TopEntry e = tr[i];
+        t = top_merge(t, Top{e.v1, e.i1, e.v2});
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) t = top_merge(t, top_shfl_xor(t, o));
+    if (lane == 0) red[warp] = t;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        t = top_merge(top_merge(red[0], red[1]), top_merge(red[2], red[3]));
+        node_argmax[row] = t.i1;
+        if (margin) margin[row] = t.v1 - t.v2;
+        __threadfence();
+        const int b = seq_of_row(row_off, B, row);
+        const unsigned int need = (unsigned int)(row_off[b + 1] - row_off[b]);
+        const unsigned int got = atomicAdd(&tickets[b], 1u);
+        last_flag = (got + 1 == need) ? b : -1;
+        if (got + 1 == need) tickets[b] = 0;                 // ready for the next call
+    }
+    __syncthreads();
+    const int b = last_flag;
+    if (b < 0 || !do_accept) return;
+    __threadfence();                                         // the other rows' predictions were written by other CTAs
+    const int r0 = row_off[b], rows = row_off[b + 1] - r0;
+    accept_sequence(tokens + r0, parent + r0, depth + r0, node_argmax + r0, rows,
+                    k_acc + b, path + (size_t)b * TRJ_PATH_STRIDE, bonus + b);
+}
+
 __global__ void accept_only_kernel(const int32_t* __restrict__ tokens, const int32_t* __restrict__ parent,
                                    const int32_t* __restrict__ depth, const int32_t* __restrict__ row_off,
                                    const int32_t* __restrict__ node_argmax, int32_t* __restrict__ k_acc,
@@ -1065,6 +1106,17 @@ cudaError_t launch_topk_accept(const void* logits, int32_t dtype, int32_t V, int
                                                     margin, k_acc, path, bonus, do_accept ? 1 : 0, tickets));
     }
     return launch_err != cudaSuccess ? launch_err : cudaGetLastError();
+}
+
+cudaError_t launch_argmax_table_accept(const TopEntry* table, int32_t entries_per_row, const int32_t* tokens,
+                                       const int32_t* parent, const int32_t* depth, const int32_t* row_off, int32_t B,
+                                       int32_t rows_total, int32_t* node_argmax, float* margin, int32_t* k_acc,
+                                       int32_t* path, int32_t* bonus, bool do_accept, void* ws, cudaStream_t st) {
+    count_launch();
+    cudaError_t e = launch_chain(argmax_table_accept_kernel, dim3(rows_total), dim3(128), 0, st, table, entries_per_row, tokens,
+                                 parent, depth, row_off, B, node_argmax, margin, k_acc, path, bonus, do_accept ? 1 : 0,
+                                 (unsigned int*)ws);
+    return e != cudaSuccess ? e : cudaGetLastError();
 }
 
 // ---------------------------------------------------------------- arg-max + accept without a caller workspace

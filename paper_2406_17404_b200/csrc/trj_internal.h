@@ -107,6 +107,15 @@ struct WeightPrefetch { const void* w; int32_t N, K; size_t bytes; int32_t ctas;
 struct Parts { const float* ptr; int32_t splits; size_t stride; };
 inline Parts whole(const float* p) { return Parts{p, 1, 0}; }
 
+// Arg-max fused into a projection's epilogue (Eq. 1 needs every row's arg-max, not the logits): every epilogue warp
+// leaves, for every activation row, the best value, its output index (ties: the smaller index) and the runner-up value
+// among its 32 outputs of the tile.  Table layout: entry ((row * tiles + tile) * 4 + warp); tiles = ceil(N / 128).
+// Only for launches with one K range and one row block (gemm_top_table_ok); y is still written unless store_y == 0.
+struct TopEntry { float v1; int32_t i1; float v2; };
+struct TopTable { TopEntry* entries; int32_t store_y; };
+bool gemm_top_table_ok(int32_t M, int32_t N, int32_t K, int32_t dtype, bool pair);
+inline size_t gemm_top_table_entries(int32_t rows, int32_t N) { return (size_t)rows * ((N + 127) / 128) * 4; }
+
 cudaError_t launch_embed(const void* embed, int32_t dtype, const int32_t* tokens, float* h,
                          int32_t rows, int32_t d, cudaStream_t st);
 // h += add (when add != nullptr, h is updated in place); x = rmsnorm(h) * gain, stored as dtype.
@@ -124,7 +133,7 @@ bool gemm_tc_supported(const void* x, const void* x_lo, const void* w, const flo
 size_t gemm_tc_workspace(int32_t M, int32_t N, int32_t K);
 cudaError_t launch_gemm_tc(const void* x, const void* x_lo, const void* w, float* y, int32_t M, int32_t N, int32_t K,
                            void* workspace, cudaStream_t st, Parts* parts, const WeightPrefetch* ahead = nullptr,
-                           int* status = nullptr);
+                           int* status = nullptr, const TopTable* top = nullptr);
 // The tcgen05 kernel for every shape it is written for (bf16, K >= 64 and a multiple of 8, N a multiple of 4), the plain
 // kernel for the rest (fp32 models, odd sizes).  A shape of the first kind whose workspace is too small or
 // misaligned is an error (cudaErrorInvalidValue), never a silent detour through the plain kernel.  With `parts`
@@ -134,7 +143,7 @@ cudaError_t launch_gemm_tc(const void* x, const void* x_lo, const void* w, float
 bool gemm_tc_shape(int32_t M, int32_t N, int32_t K, int32_t dtype);
 cudaError_t launch_gemm(const void* x, const void* x_lo, const void* w, float* y, int32_t M, int32_t N, int32_t K,
                         int32_t dtype, void* workspace, size_t workspace_bytes, cudaStream_t st, Parts* parts = nullptr,
-                        const WeightPrefetch* ahead = nullptr, int* status = nullptr);
+                        const WeightPrefetch* ahead = nullptr, int* status = nullptr, const TopTable* top = nullptr);
 
 // Rotary embedding of q and k at position seq_len[b] + depth[row]; q -> q_out [rows][H][D];
 // k, v -> cache rows seq_len[b] + local row of the layer slab [B][Hkv][max_seq][D].  The projection result has
@@ -213,6 +222,13 @@ cudaError_t launch_topk_accept(const void* logits, int32_t dtype, int32_t V, int
                                const int32_t* row_off, int32_t B, int32_t rows_total, int32_t* topk,
                                int32_t* node_argmax, float* margin, int32_t* k_acc, int32_t* path,
                                int32_t* bonus, bool do_accept, void* ws, cudaStream_t st);
+
+// Arg-max + acceptance from the table a projection's epilogue left (gemm_top_table_entries): entries_per_row
+// candidates per row, merged with the full (value, index) order.
+cudaError_t launch_argmax_table_accept(const TopEntry* table, int32_t entries_per_row, const int32_t* tokens,
+                                       const int32_t* parent, const int32_t* depth, const int32_t* row_off, int32_t B,
+                                       int32_t rows_total, int32_t* node_argmax, float* margin, int32_t* k_acc,
+                                       int32_t* path, int32_t* bonus, bool do_accept, void* ws, cudaStream_t st);
 
 // Same kernel with its scratch in a file-scope device array of the library (no workspace argument).
 cudaError_t launch_argmax_accept_static(const void* logits, int32_t dtype, int32_t V,

@@ -188,6 +188,57 @@ def test_llama7b_shape_two_layers_paper_sized_trees(trj, width, r, lr):
     model.close()
 
 
+@pytest.mark.parametrize("cfg_name", ["small_bf16", "7b"])
+def test_argmax_from_the_lm_head_epilogue_ties_and_both_step_paths(trj, cfg_name):
+    """The step's arg-max comes from candidates the LM head's epilogue leaves (one per 32 vocabulary entries), the
+    logits being written only on request.  Rows of the LM head are duplicated so that logits tie bit for bit inside
+    a warp's 32 entries, across the warps of a tile and across tiles: the smaller id must win (Eq. 1 with the tie
+    rule) and the margin there is 0.  trj_verify_step (logits kept) and trj_step_host (no logits) must agree."""
+    from dataclasses import replace
+    from paper_2406_17404_b200.decode import upload_weights
+    cfg = replace(synth.TINY, dtype="bf16") if cfg_name == "small_bf16" else synth.LLAMA7B.with_layers(1)
+    layers = [synth.layer_weights(cfg, 5, l) for l in range(cfg.n_layers)]
+    glob = dict(synth.global_weights(cfg, 5))
+    lm = np.array(glob["lm_head"], np.float32)
+    lm[5] *= 16.0                                            # a row that wins for about half of the inputs (x16 is exact in bf16)
+    for dup in (6, 40, 133, cfg.vocab - 1):                  # same warp, next warp, next tile, last tile
+        lm[dup] = lm[5]
+    glob["lm_head"] = lm
+    dl, dg = upload_weights(cfg, layers, glob)
+    model = trj.Model(cfg, dl, dg, max_batch=1, max_seq=256, max_rows=64)
+    f64 = lambda d: {k: np.asarray(v, np.float64) for k, v in d.items()}
+    dec = oracle.Decoder(cfg, [f64(l) for l in layers], f64(glob))
+    prompt = synth.prompt(9, 40, cfg.vocab)
+    first = int(model.prefill(i32(prompt)).item())
+    cache = dec.new_cache(256)
+    dec.forward_rows(cache, prompt, synth.chain_parents(len(prompt)))
+    cache.seq_len = len(prompt)
+    window, branches = synth.prompt(10, 5, cfg.vocab), synth.prompt(11, 27, cfg.vocab).reshape(9, 3)
+    tree = trj.build_tree(first, window, branches)
+    m = len(tree["tokens"])
+    want_logits = dec.forward_rows(cache, tree["tokens"], tree["parent"])
+    want_pred = oracle.node_argmax(want_logits)
+    d_tok, d_par, d_dep, d_off = i32(tree["tokens"]), i32(tree["parent"]), i32(tree["depth"]), i32([0, m])
+    out = model.verify_step(d_tok, d_par, d_dep, anc_dev(tree["anc"]), d_off, max_rows=m, max_len=len(prompt) + m,
+                            want_logits=True, want_margin=True)
+    torch.cuda.synchronize()
+    model.device_status()
+    logits, pred, margin = out["logits"].cpu().numpy(), out["node_argmax"].cpu().numpy(), out["margin"].cpu().numpy()
+    # the kernel's own logits decide what its arg-max must be: bit-exact, ties to the smaller id
+    np.testing.assert_array_equal(pred, oracle.node_argmax(logits.astype(np.float64)))
+    np.testing.assert_array_equal(margin, oracle.top2_margin(logits.astype(np.float64)).astype(np.float32))
+    tied = np.isin(pred, [5, 6, 40, 133, cfg.vocab - 1])
+    assert tied.sum() >= 4 and (pred[tied] == 5).all() and (margin[tied] == 0).all()
+    assert (logits[:, 5] == logits[:, 133]).all()
+    safe = oracle.top2_margin(want_logits) >= MARGIN
+    np.testing.assert_array_equal(pred[safe | tied], want_pred[safe | tied])
+    # the path that never writes logits
+    host = model.step_host(first, window, branches, max_len=len(prompt) + m)
+    np.testing.assert_array_equal(host["node_argmax"], pred)
+    assert (host["k_acc"], host["path"].tolist(), host["bonus"]) == oracle.accept_path(tree["tokens"], tree["parent"], pred)
+    model.close()
+
+
 def test_grouped_query_tiny_fp32_16_steps(trj):
     """Grouped-query attention on the tiny fp32 shape (4 query heads over 2 K/V heads), generic kernels."""
     cfg = synth.TINY_GQA
