@@ -464,7 +464,7 @@ def whole_job_rate(world, units_per_rank, seconds):
     return world * units_per_rank / seconds
 
 
-def bench_template_step(trj, torch, synth, model, cfg, prefix, side, steps, context=None):
+def bench_template_step(trj, torch, synth, model, cfg, prefix, side, steps, context=None, truth=None, take=None):
     """One verification step over a 69-row static template with top-K siblings (63 draft nodes + a retrieval path of
     5 + the root: the tree size the paper uses, Appendix B; the topology is a seeded stand-in): forward, per-row top-10,
     acceptance and compaction, replayed from a CUDA graph on the same model and cache."""
@@ -519,6 +519,8 @@ def bench_template_step(trj, torch, synth, model, cfg, prefix, side, steps, cont
         host_drafts = np.asarray(context, np.int32)[np.asarray(draw(0, m - 1), np.int64) % n0]
         host_draws = np.stack([np.asarray(draw(st, m - 1 + n_retr), np.int64) for st in range(1, steps + 1)])
         k_log = torch.zeros(steps, dtype=torch.int32, device=dev)
+        if truth is not None:                                # the true continuation planted into the retrieval path, 0-3 tokens a step
+            model.set_draft_source(i32(truth), i32(np.asarray(take[:steps], np.int32)))
 
         def loop():
             model.seq_len.copy_(seq0)
@@ -533,9 +535,13 @@ def bench_template_step(trj, torch, synth, model, cfg, prefix, side, steps, cont
         tokens_out, n_end = loop()
         wall = time.perf_counter() - t0
         model.device_status()
+        model.set_draft_source(None)
         out["device_loop"] = {"ms_per_step": wall / steps * 1e3, "tokens_committed_per_step": (n_end - n0) / steps,
                               "committed_tokens_per_s": (n_end - n0) / wall,
-                              "what": "trj_decode_device_tree: %d steps enqueued at once" % steps}
+                              "what": "trj_decode_device_tree: %d steps enqueued at once; the true continuation planted "
+                                      "into 0-3 slots of the retrieval path per step" % steps}
+        if truth is not None:
+            out["device_loop"]["matches_autoregressive"] = bool((tokens_out.numpy()[:n_end] == np.asarray(truth)[:n_end]).all())
     return out
 
 
@@ -943,7 +949,7 @@ def run_ours(args, rank, world, local_rank):
                                     "wall clock incl. uploading the draws and reading the tokens back" % args.steps},
             "roofline": roofline, "kernel_breakdown": breakdown, "profiled_step_ms": step_ms_prof}
     if world == 1:
-        line["paper_sized_tree"] = bench_template_step(trj, torch, synth, model, cfg, PROMPT, side, args.steps, context=ctx0)
+        line["paper_sized_tree"] = bench_template_step(trj, torch, synth, model, cfg, PROMPT, side, args.steps, context=ctx0, truth=abs_truth, take=take)
         # prefill of the 512-token prompt: the weights are streamed once (projections over all 512 rows at a time)
         model.seq_len.zero_()
         model.prefill(i32(prompt)); torch.cuda.synchronize()

@@ -463,7 +463,8 @@ trj_status trj_decode_device_tree(trj_ctx* ctx, void* k_cache, void* v_cache, in
                                   const int32_t* rank, int32_t M, int32_t K, int32_t n_retrieved, int32_t* drafts,
                                   const int64_t* draws, int32_t n_steps, int32_t* k_log, void* stream);
 
-/* An external source of drafts for trj_decode_device (Section 3.3: retrieved drafts get a path of their own; where
+/* An external source of drafts for trj_decode_device and trj_decode_device_tree (there it feeds the start of the
+ * retrieval path instead of branch 0) (Section 3.3: retrieved drafts get a path of their own; where
  * they are retrieved from is open).  stream [n] (dev int32) holds the source's guess for the token at context
  * position i in stream[i]; in step s of a later trj_decode_device call the first take[s] (dev int32 [n_steps],
  * clipped to branch_len and to n) tokens of retrieved branch 0 come from stream, starting at the position after

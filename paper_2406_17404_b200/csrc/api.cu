@@ -1089,6 +1089,8 @@ extern "C" trj_status trj_decode_device_tree(trj_ctx* ctx, void* k_cache, void* 
                 "decode_device_tree: context buffer of %d cannot take %d steps of up to %d tokens after %d", capacity, n_steps, per_step, n_ctx_now);
     const int64_t max_len = (int64_t)n_ctx_now - 1 + (int64_t)n_steps * per_step + M;
     TRJ_REQUIRE(max_len <= c.max_seq, TRJ_ECAPACITY, "decode_device_tree: up to %lld cache rows exceed max_seq %d", (long long)max_len, c.max_seq);
+    TRJ_REQUIRE(!ctx->draft_src.stream || ctx->draft_src_steps >= n_steps, TRJ_ECAPACITY,
+                "decode_device_tree: the draft source covers %d steps, %d asked", ctx->draft_src_steps, n_steps);
     s = check_step_args(ctx, 1, M, M, (int32_t)max_len, 2);
     if (s != TRJ_OK) return s;
     if (n_steps == 0) return TRJ_OK;
@@ -1112,7 +1114,7 @@ extern "C" trj_status trj_decode_device_tree(trj_ctx* ctx, void* k_cache, void* 
     auto enqueue_one = [&](cudaStream_t on) -> trj_status {
         ChainScope chain;
         LAUNCH_ON(on, PROF_ELEMENTWISE, launch_template_tokens(context, n_ctx, drafts, d_rank, M, n_retrieved, draws, d_step, d_tokens,
-                                                               d_retr, on));
+                                                               d_retr, on, ctx->draft_src));
         trj_status fs = forward(ctx, k_cache, v_cache, 0, bt, d_tokens, d_depth, d_anc, 2, 0, M, on);
         if (fs != TRJ_OK) return fs;
         LAUNCH_ON(on, PROF_ARGMAX, launch_topk_accept(ctx->logits, TRJ_F32, c.vocab, K, d_tokens, d_parent, d_depth, d_off, 1, M, d_topk,
@@ -1129,7 +1131,8 @@ extern "C" trj_status trj_decode_device_tree(trj_ctx* ctx, void* k_cache, void* 
                                                (uint64_t)(uintptr_t)k_cache, (uint64_t)(uintptr_t)v_cache, (uint64_t)(uintptr_t)seq_len,
                                                (uint64_t)(uintptr_t)context, (uint64_t)capacity, (uint64_t)(uintptr_t)n_ctx,
                                                (uint64_t)(uintptr_t)drafts, (uint64_t)(uintptr_t)draws, (uint64_t)(uintptr_t)k_log,
-                                               (uint64_t)max_len};
+                                               (uint64_t)max_len, (uint64_t)(uintptr_t)ctx->draft_src.stream, (uint64_t)ctx->draft_src.n,
+                                               (uint64_t)(uintptr_t)ctx->draft_src.take};
     return run_device_loop(ctx, key_of_loop, n_steps, enqueue_one, st);
 }
 

@@ -114,15 +114,19 @@ __global__ void __launch_bounds__(32) template_tokens_kernel(const int32_t* __re
                                                              const int32_t* __restrict__ drafts, const int32_t* __restrict__ rank,
                                                              int M, int n_retr, const int64_t* __restrict__ draws,
                                                              const int32_t* __restrict__ step, int32_t* __restrict__ tokens,
-                                                             int32_t* __restrict__ retr) {
+                                                             int32_t* __restrict__ retr, const DraftSource src) {
     pdl_prologue();
     const int lane = threadIdx.x;
     const int n = *n_ctx;
     const int64_t* my_draws = draws + (size_t)*step * (size_t)(M - 1 + n_retr);
     int follow[1];
     const int nf = n_retr > 0 ? find_follows(context, n, 1, follow, lane) : 0;
-    for (int j = lane; j < n_retr; j += 32)
-        retr[j] = (nf > 0 && follow[0] + j < n) ? context[follow[0] + j] : context[(uint64_t)my_draws[M - 1 + j] % (uint64_t)n];
+    for (int j = lane; j < n_retr; j += 32) {
+        int32_t tok = (nf > 0 && follow[0] + j < n) ? context[follow[0] + j] : context[(uint64_t)my_draws[M - 1 + j] % (uint64_t)n];
+        // an external draft source (may be absent) overrides the start of the retrieval path, as it does for branch 0
+        if (src.stream && j < src.take[*step] && n + j < src.n) tok = src.stream[n + j];
+        retr[j] = tok;
+    }
     __syncwarp();
     if (lane == 0) tokens[0] = context[n - 1];
     for (int i = 1 + lane; i < M; i += 32) tokens[i] = rank[i] < 0 ? retr[-1 - rank[i]] : drafts[i - 1];
@@ -188,10 +192,10 @@ __global__ void __launch_bounds__(32) commit_refill_tree_kernel(const int32_t* _
 
 cudaError_t launch_template_tokens(const int32_t* context, const int32_t* n_ctx, const int32_t* drafts, const int32_t* rank,
                                    int32_t M, int32_t n_retr, const int64_t* draws, const int32_t* step, int32_t* tokens,
-                                   int32_t* retr, cudaStream_t st) {
+                                   int32_t* retr, cudaStream_t st, const DraftSource& src) {
     count_launch();
     cudaError_t e = launch_chain(template_tokens_kernel, dim3(1), dim3(32), 0, st, context, n_ctx, drafts, rank, M, n_retr, draws, step,
-                                 tokens, retr);
+                                 tokens, retr, src);
     return e != cudaSuccess ? e : cudaGetLastError();
 }
 

@@ -193,7 +193,7 @@ cudaError_t launch_commit_refill(const int32_t* tokens, const int32_t* parent, c
 // step s: draws[s][0 .. M-2] refill, draws[s][M-1 .. M-2+n_retr] retrieval.
 cudaError_t launch_template_tokens(const int32_t* context, const int32_t* n_ctx, const int32_t* drafts, const int32_t* rank,
                                    int32_t M, int32_t n_retr, const int64_t* draws, const int32_t* step, int32_t* tokens,
-                                   int32_t* retr, cudaStream_t st);
+                                   int32_t* retr, cudaStream_t st, const DraftSource& src = DraftSource{nullptr, 0, nullptr});
 cudaError_t launch_commit_refill_tree(const int32_t* tokens, const int32_t* parent, const int32_t* depth, const int32_t* rank,
                                       const int32_t* topk, int32_t K, int32_t M, const int32_t* k_acc, const int32_t* path,
                                       const int32_t* bonus, int32_t* context, int32_t capacity, int32_t* n_ctx, int32_t n_retr,

@@ -191,6 +191,44 @@ def test_device_decode_loop_with_an_external_draft_source(trj):
     model.close()
 
 
+def test_device_template_loop_with_an_external_draft_source(trj):
+    """The same source feeding the start of a template's retrieval path: step s accepts at least take[s] rows and the
+    loop commits the oracle's greedy tokens."""
+    cfg = synth.TINY
+    parent, rank = synth.tree_template(0)
+    m, top_k, n_retr, n_steps = len(parent), 10, 5, 10
+    model, dec = make_models(trj, cfg, 0, max_seq=512, max_rows=128)
+    prompt = synth.prompt(9, 64, cfg.vocab)
+    draw = lambda s, n: synth.noise_draws(9, s, n)
+    per_step = int(synth.node_depths(np.asarray(parent, np.int32)).max()) + 1
+    n_truth = n_steps * per_step + 2
+    truth = oracle.autoregressive_greedy(dec, prompt, n_truth)
+    take_host = np.asarray([s % 4 for s in range(n_steps)], np.int32)
+    model.seq_len.zero_()
+    first = int(model.prefill(i32(prompt)).item())
+    assert first == truth[0]
+    committed = [int(t) for t in prompt] + [first]
+    buf = np.zeros(len(prompt) + n_truth, np.int32); buf[:len(committed)] = committed
+    d_ctx, d_n = i32(buf), i32([len(committed)])
+    drafts = i32([committed[int(d) % len(committed)] for d in draw(0, m - 1)])
+    draws = i64(np.stack([np.asarray(draw(s, m - 1 + n_retr), np.int64) for s in range(1, n_steps + 1)]))
+    k_log = torch.full((n_steps,), -1, dtype=torch.int32, device="cuda")
+    model.set_draft_source(i32(np.concatenate([prompt, truth])), i32(take_host))
+    model.decode_device_tree(d_ctx, d_n, len(committed), parent, rank, top_k, n_retr, drafts, draws, n_steps, k_log=k_log)
+    torch.cuda.synchronize()
+    model.set_draft_source(None)
+    n_end = int(d_n[0])
+    got = d_ctx.cpu().numpy()[len(prompt):n_end].tolist()
+    if got != truth[:len(got)]:
+        cache = dec.new_cache(len(prompt) + n_truth + 1)
+        lg = dec.forward_rows(cache, list(prompt) + truth[:len(got)], list(range(-1, len(prompt) + len(got) - 1)))
+        assert oracle.top2_margin(lg[len(prompt) - 1:]).min() < MARGIN
+    else:
+        assert (k_log.cpu().numpy() >= take_host).all()
+        assert int(k_log.sum()) + n_steps == n_end - len(committed)
+    model.close()
+
+
 def test_device_decode_loop_7b_shape_equals_the_host_driven_loop(trj):
     """7B layer shape, 2 layers, bf16 (the tcgen05 kernels): the device-resident loop and the host-driven loop run the
     same kernels on the same inputs, so their committed tokens must be identical.  This checks the loop's plumbing on
