@@ -625,6 +625,32 @@ def bench_tp_rank(trj, torch, synth, peaks, steps):
     return out
 
 
+def bench_step_vs_rows(trj, torch, synth, model, cfg, prefix, steps):
+    """Verification step (forward + arg-max + acceptance + compaction) against the number of tree rows, on the same
+    model and cache: the projections stay weight-bound, so rows are cheap until the accumulators outgrow two CTAs per SM."""
+    dev = model.device
+    i32 = lambda a: torch.from_numpy(np.ascontiguousarray(a, dtype=np.int32)).to(dev)
+    seq0 = torch.full_like(model.seq_len, prefix)
+    out = {}
+    for m in (17, 33, 48, 64, 69, 80, 96, 128):
+        parent = synth.random_tree(3, m, min(8, m - 1), 4)
+        depth, anc = trj.tree_from_parents(parent)
+        d_tok, d_par, d_dep, d_off = i32(synth.prompt(77, m, cfg.vocab)), i32(parent), i32(depth), i32([0, m])
+        d_anc = torch.from_numpy(anc.view(np.int64)).to(dev)
+        pred = torch.empty(m, dtype=torch.int32, device=dev)
+        acc = {"k_acc": torch.empty(1, dtype=torch.int32, device=dev), "bonus": torch.empty(1, dtype=torch.int32, device=dev),
+               "path": torch.empty(1, trj.PATH_STRIDE, dtype=torch.int32, device=dev)}
+
+        def step():
+            model.seq_len.copy_(seq0)
+            model.verify_step(d_tok, d_par, d_dep, d_anc, d_off, max_rows=m, max_len=prefix + m, node_argmax=pred)
+            model.accept(d_tok, d_par, d_dep, d_off, pred, out=acc)
+            model.compact_kv(acc["k_acc"], acc["path"])
+        out[str(m)] = round(graph_us(torch, step, steps, 3) / 1e3, 4)
+    model.device_status()
+    return {"ms_per_step_by_tree_rows": out, "prefix": prefix, "what": "7B shape, random trees and drafts"}
+
+
 def bench_batched_step(trj, torch, synth, cfg, layers, glob, peaks, steps, n_seq=8):
     """The same verification step for `n_seq` independent sequences at once (each a 512-token prompt and a 33-row
     tree): one forward over all rows, arg-max + acceptance per sequence, compaction of every cache.  The weights are
@@ -964,6 +990,7 @@ def run_ours(args, rank, world, local_rank):
             line["prefill_gemm"] = bench_prefill_gemm(trj, torch, peaks, max(args.steps // 2, 5))
             line["llama3_8b_step"] = bench_llama3_step(trj, torch, synth, peaks, max(args.steps // 2, 5))
             line["tensor_parallel_rank"] = bench_tp_rank(trj, torch, synth, peaks, max(args.steps // 2, 5))
+            line["step_vs_rows"] = bench_step_vs_rows(trj, torch, synth, model, cfg, PROMPT, max(args.steps // 2, 5))
             line["batched_step"] = bench_batched_step(trj, torch, synth, cfg, layers, glob, peaks, max(args.steps // 2, 5))
         if not args.no_attention:
             line["tree_attention"] = bench_tree_attention(trj, torch, peaks, max(args.steps, 5), 3, cpu=not args.no_cpu)
