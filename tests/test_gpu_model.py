@@ -170,11 +170,11 @@ def test_llama7b_shape_two_layers_bf16(trj):
     model.close()
 
 
-@pytest.mark.parametrize("width,r,lr", [(8, 12, 5), (7, 12, 6)])
+@pytest.mark.parametrize("width,r,lr", [(8, 12, 5), (7, 12, 6), (7, 12, 10)])
 def test_llama7b_shape_two_layers_paper_sized_trees(trj, width, r, lr):
-    """The same decoder on trees of 69 and 80 rows (the paper verifies about 64 draft tokens per step): between 65 and
-    80 rows the projections add the two halves of a bf16 activation pair in the accumulator (two products per weight
-    tile) instead of side by side, which keeps two CTAs per SM."""
+    """The same decoder on trees of 69, 80 and 128 rows (the paper verifies about 64 draft tokens per step): between 65
+    and 80 rows the projections add the two halves of a bf16 activation pair in the accumulator (two products per
+    weight tile) instead of side by side, which keeps two CTAs per SM; 128 rows is the largest tree."""
     cfg = synth.LLAMA7B.with_layers(2)
     model, dec = make_models(trj, cfg, 3, max_seq=384, max_rows=128)
     prompt = synth.prompt(3, 40, cfg.vocab)
@@ -182,7 +182,7 @@ def test_llama7b_shape_two_layers_paper_sized_trees(trj, width, r, lr):
     trace = []
     oracle.tr_jacobi_generate(dec, prompt, 6, width, r, lr, draw, trace=trace)
     trace = trace[:3]
-    assert all(len(rec["tokens"]) == 1 + width + r * lr for rec in trace) and 64 < 1 + width + r * lr <= 80
+    assert all(len(rec["tokens"]) == 1 + width + r * lr for rec in trace) and 64 < 1 + width + r * lr <= 128
     stats = drive_with_oracle_trace(trj, model, prompt, trace, tol=2e-2)
     assert stats["rows"] > 150
     model.close()
