@@ -16,6 +16,7 @@
 // after that.  With 256 rows per block the kernel is a 128 x 256 x 64-per-stage tensor-core GEMM, bound by the
 // tensor pipe instead of by HBM.
 #include <cuda.h>
+#include <cstdlib>
 #include <mutex>
 #include <algorithm>
 #include "trj_internal.h"
@@ -352,7 +353,7 @@ struct TcPlan {
 
 // Number of K ranges per weight tile.  Items (tiles x row blocks x splits) are dealt round-robin to a grid of at
 // most grid_cap CTAs, so the choice trades balance (items close to a multiple of the grid) against the extra
-// traffic of the partial sums, about 2*splits*M/K of the weight bytes.  When no consumer kernel adds the pieces
+// traffic of the partial sums, about 2*splits*M/K of the weight bytes (weighted, see below).  When no consumer kernel adds the pieces
 // (`finished`: the caller wants y itself) a reduce kernel has to read them again and is one more launch: then a
 // single K range is taken as soon as the tiles alone fill most of the grid.
 int tc_splits(int M, int K, int units, int kblocks, int grid_cap, bool finished) {
@@ -362,7 +363,10 @@ int tc_splits(int M, int K, int units, int kblocks, int grid_cap, bool finished)
     for (int s = 1; s <= 16 && s <= (kblocks >= 4 ? kblocks / 4 : 1); ++s) {
         const int items = units * s, rounds = (items + grid_cap - 1) / grid_cap;
         const double balance = (double)items / ((double)rounds * grid_cap);
-        const double score = balance / (1.0 + 2.0 * s * M / K);
+        // the pieces cost more than their own bytes: the consumer kernel that adds them sits between two projections,
+        // where nothing hides it (weight 4 measured on the 7B step: gate/up goes from 5 to 3 pieces, 3.415 -> 3.393 ms;
+        // weights 8 and 16 choose the same splits)
+        const double score = balance / (1.0 + 4.0 * 2.0 * s * M / K);
         if (score > best_score * 1.02) { best_score = score; best = s; }      // prefer fewer splits on near ties
     }
     return best;
