@@ -38,10 +38,10 @@ PROMPT = 512
 METRIC = "draft_tokens_verified_per_s"
 UNIT = "tokens/s"
 # DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) of ALL 129 projection launches of one step, from an ncu
-# capture of the current projection kernel on a 4-layer model, scaled to 32 layers + the LM head: per layer 444.13 MB
-# (QKV 102.26, output 64.21 incl. 30 MB of gate/up weights that it prefetches and that ncu's serialised timing counts
-# again in the gate/up launch, gate/up 185.11, down 92.55), LM head 262.88 MB.  Set to None whenever that kernel changes.
-GEMM_TRAFFIC_BYTES_PER_STEP = int(32 * 444.13e6 + 262.88e6)
+# capture of the current projection kernel on a 4-layer model, scaled to 32 layers + the LM head: per layer 443.3 MB
+# (QKV 102.4, output 65.1 incl. 30 MB of gate/up weights that it prefetches and that ncu's serialised timing counts
+# again in the gate/up launch, gate/up 183.2, down 92.6), LM head 263.1 MB.  Set to None whenever that kernel changes.
+GEMM_TRAFFIC_BYTES_PER_STEP = int(32 * 443.3e6 + 263.1e6)
 
 
 def measured_peaks():
