@@ -5,6 +5,7 @@
 #include <new>
 #include <utility>
 #include <vector>
+#include <cstdlib>
 #include "trj_internal.h"
 
 using namespace trj;
@@ -354,7 +355,9 @@ trj_status run_segments(trj_ctx* ctx, const StepArgs& a, int s0, int s1, Parts& 
                          tree_attention_tc_supported(c.head_dim, c.dtype, bt.max_rows);
     const int attn_grid = attn_tc ? tree_attention_grid(bt.B, c.n_heads, bt.max_len) : ctx->sm_count;
     int* const gemm_status = ctx->dev_status, *const attn_status = ctx->dev_status + 1;
-    constexpr size_t AHEAD_BYTES = (size_t)32 << 20;         // measured optimum on the 7B shape (16-40 MB are close)
+    // measured on the 7B shape: 32-48 MB of the gate/up weights are worth 0.1 ms per step (16 MB: half of that, 64 MB:
+    // a quarter); 12-20 MB of the output projection's own weights on top another 0.012 ms, more of them cost again
+    constexpr size_t AHEAD_BYTES = (size_t)32 << 20, AHEAD_SELF_BYTES = (size_t)16 << 20;
     const SubChunks* pieces = a.pieces;
     for (int s = s0; s < s1; ++s) {
         const int l = s >> 1;
@@ -406,7 +409,7 @@ trj_status run_segments(trj_ctx* ctx, const StepArgs& a, int s0, int s1, Parts& 
             }
             // While the attention kernel runs, HBM is nearly idle and the SMs it leaves free go to the first CTAs of
             // the output projection, which only wait: they ask for the start of the gate/up weights into L2.
-            const WeightPrefetch ahead{ctx->w_gate_up[l], 2 * c.d_ff, d, AHEAD_BYTES, 2 * std::max(0, ctx->sm_count - attn_grid)};
+            const WeightPrefetch ahead{ctx->w_gate_up[l], 2 * c.d_ff, d, AHEAD_BYTES, 2 * std::max(0, ctx->sm_count - attn_grid), AHEAD_SELF_BYTES};
             LAUNCH(PROF_GEMM, launch_gemm(ctx->x, ctx->x_lo, ctx->wo[l], ctx->y, M, d, HD, c.dtype, ctx->gemm_ws,
                                           ctx->gemm_ws_bytes, st, out_parts, &ahead, gemm_status));
         } else {

@@ -48,6 +48,7 @@ struct TcParams {
     int tiles, splits, stages;
     float* out;         // [splits][M][N]
     int* status;        // device word: 0, or TRJ_ETIMEOUT once a wait expired
+    int self_boxes;     // [128 x 64] tiles of this projection's own weights that the early CTAs request into L2
     int ahead_boxes, ahead_kblocks, ahead_ctas;   // [128 x 64] tiles of a later projection's weights to request into L2
 };
 
@@ -147,9 +148,12 @@ __global__ void __launch_bounds__(TC_THREADS, 2) gemm_tc_kernel(const __grid_con
                 }
                 if (pass == 0) {
                     // CTAs that run while the previous kernel still does: a later projection's weights into L2
-                    if ((int)blockIdx.x < p.ahead_ctas)
+                    if ((int)blockIdx.x < p.ahead_ctas) {
+                        for (int i = blockIdx.x; i < p.self_boxes; i += p.ahead_ctas)      // this projection's own weights first
+                            tma_prefetch_l2_2d(&map_w, (i % p.kblocks) * TC_BK, (i / p.kblocks) * TC_BM);
                         for (int i = blockIdx.x; i < p.ahead_boxes; i += p.ahead_ctas)
                             tma_prefetch_l2_2d(&map_ahead, (i % p.ahead_kblocks) * TC_BK, (i / p.ahead_kblocks) * TC_BM);
+                    }
                     pdl_wait();                              // activations come from the previous kernel
                     TRJ_TL_BEGIN(TRJ_TL_GEMM);
                 }
@@ -455,7 +459,7 @@ cudaError_t launch_gemm_tc(const void* x, const void* x_lo, const void* w, float
     p.out = p.splits > 1 ? (float*)workspace : y;
     p.status = status;
     CUtensorMap map_w, map_x, map_xlo, map_ahead;
-    p.ahead_boxes = 0; p.ahead_kblocks = 1; p.ahead_ctas = 0;
+    p.ahead_boxes = 0; p.ahead_kblocks = 1; p.ahead_ctas = 0; p.self_boxes = 0;
     const bool want_ahead = ahead && ahead->ctas > 0 && ahead->w && ahead->K % 8 == 0 && ahead->K >= TC_BK &&
                             ((uintptr_t)ahead->w % 16) == 0;
     if (want_ahead) {
@@ -465,6 +469,8 @@ cudaError_t launch_gemm_tc(const void* x, const void* x_lo, const void* w, float
         p.ahead_kblocks = (ahead->K + TC_BK - 1) / TC_BK;
         p.ahead_boxes = (int)(asked < all ? asked : all);
         p.ahead_ctas = ahead->ctas;
+        const size_t own = (size_t)pl.tiles * pl.kblocks, want_self = ahead->self_bytes / TC_A_BYTES;
+        p.self_boxes = (int)(want_self < own ? want_self : own);
     }
     if (!make_map(&map_w, w, N, K, TC_BM) || !make_map(&map_x, x, M, K, p.m_pad) ||
         !make_map(&map_xlo, x_lo ? x_lo : x, M, K, p.m_pad))

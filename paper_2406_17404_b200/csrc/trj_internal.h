@@ -100,8 +100,9 @@ struct Batch {
 // Weights of a LATER projection that a projection kernel may ask for ahead of time.  When the kernel before a
 // projection leaves SMs free and HBM idle (the attention kernel of a decoding step does both), the projection's
 // first `ctas` CTAs get those SMs at once and spend their wait requesting the first `bytes` of `w` ([N][K] bf16)
-// into L2, so that the later projection starts from L2 instead of HBM.  ctas = 0: nothing is requested.
-struct WeightPrefetch { const void* w; int32_t N, K; size_t bytes; int32_t ctas; };
+// into L2, so that the later projection starts from L2 instead of HBM; before that they request the first
+// `self_bytes` of the projection's OWN weights the same way.  ctas = 0: nothing is requested.
+struct WeightPrefetch { const void* w; int32_t N, K; size_t bytes; int32_t ctas; size_t self_bytes; };
 
 // A projection result that may still be in split-K pieces: value(i) = sum over s < splits of ptr[s * stride + i].
 struct Parts { const float* ptr; int32_t splits; size_t stride; };
