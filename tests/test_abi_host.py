@@ -120,6 +120,14 @@ def test_device_entry_points_reject_bad_arguments_before_any_launch(trj):
     assert lib.trj_commit_refill(nul, nul, nul, 4, nul, nul, nul, nul, 10, nul, 2, nul, nul, nul, nul) == 1
     assert lib.trj_commit_refill(fake, fake, fake, 500, fake, fake, fake, fake, 10, fake, 2, fake, fake, nul, nul) == 2
     assert lib.trj_decode_device(nul, fake, fake, fake, fake, 10, fake, 1, fake, 4, 2, 3, fake, 1, nul, nul) == 1
+    i32p = lambda a: np.asarray(a, np.int32).ctypes.data_as(ctypes.POINTER(ctypes.c_int32))
+    assert lib.trj_decode_device_tree(nul, fake, fake, fake, fake, 10, fake, 1, i32p([-1, 0]), i32p([0, 0]), 2, 1, 0, fake, fake, 1, nul, nul) == 1
+    # the step of a rank that holds a slice of the weights: no context, no step
+    assert lib.trj_tp_segments(nul) == 0
+    assert lib.trj_tp_begin(nul, fake, fake, fake, fake, fake, fake, fake, 2, fake, 1, 1, 1, 1, nul) == 1
+    assert lib.trj_tp_segment(nul, 0, nul) == 1
+    assert lib.trj_tp_exchange_buffer(nul, nul, nul) == 1
+    assert lib.trj_tp_finish(nul, fake, nul, nul, nul) == 1
     cfg = trj.ModelCfg(2, 256, 4, 48, 688, 1024, 1e-5, 1e4, 0, 1, 256, 16)
     assert lib.trj_workspace_bytes(ctypes.byref(cfg)) == 0
     cfg = trj.ModelCfg(2, 256, 4, 64, 688, 1024, 1e-5, 1e4, 0, 1, 256, 300)
