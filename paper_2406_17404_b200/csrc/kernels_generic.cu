@@ -637,54 +637,27 @@ __global__ void __launch_bounds__(ARGMAX_THREADS) argmax_accept_kernel(
 // warp-wide arg-max over the lists' heads, and the first warp merges the 32 warp lists the same way.  The CTA that
 // finishes the last row of a sequence walks that sequence's tree.
 constexpr int TOPK_THREADS = 1024;
-template <int KMAX>
-struct TopList {
-    float v[KMAX]; int id[KMAX];
-    __device__ __forceinline__ void clear() {
+// Top-K (K <= TRJ_MAX_TOPK) of a row, value first and the smaller id among equals.  The row is taken in chunks of
+// 32 x 1024 elements that the CTA's threads hold in registers (element j * 1024 + t of the chunk in thread t).
+// Per chunk: (A) the 32 warp maxima; their K-th largest is a value that at least K elements of the chunk reach, so
+// together with the K-th value of the row's running list it is a threshold below which nothing can enter the list;
+// (B) every element at or above the threshold goes to a candidate buffer in shared memory (slots handed out by an
+// atomic counter: the order in the buffer is arbitrary, the selection below is not); (C) the first warp selects the K
+// best among the candidates and the running list by K rounds of a scan and a shuffle reduction.  Typically a few
+// dozen elements survive the threshold.  If more survive than the buffer holds (many equal values), the chunk is
+// done the slow way: K rounds of selection over all its elements, in every warp and then over the warps' lists.
+constexpr int TOPK_PER_THREAD = 32;
+constexpr int TOPK_CAND = 1024;
+__device__ __forceinline__ bool top_better(float v, int i, float w, int j) { return v > w || (v == w && i < j); }
+__device__ __forceinline__ void warp_best(float& bv, int& bi) {
 #pragma unroll
-        for (int i = 0; i < KMAX; ++i) { v[i] = -INFINITY; id[i] = 0x7fffffff; }
-    }
-    // not inlined: the insertion is long, a thread calls it for a minority of its elements, and a kernel whose code
-    // does not fit the instruction cache pays for every launch with fetches from L2 or DRAM
-    __device__ __noinline__ void insert(float x, int i) {
-#pragma unroll
-        for (int s = KMAX - 1; s >= 1; --s) {
-            const bool above = x > v[s - 1] || (x == v[s - 1] && i < id[s - 1]);    // the new entry goes above slot s - 1
-            if (above) { v[s] = v[s - 1]; id[s] = id[s - 1]; }
-            else { v[s] = x; id[s] = i; return; }
-        }
-        v[0] = x; id[0] = i;
-    }
-    __device__ __forceinline__ void push(float x, int i) {
-        if (x > v[KMAX - 1] || (x == v[KMAX - 1] && i < id[KMAX - 1])) insert(x, i);
-    }
-    __device__ __forceinline__ void pop() {
-#pragma unroll
-        for (int s = 0; s + 1 < KMAX; ++s) { v[s] = v[s + 1]; id[s] = id[s + 1]; }
-        v[KMAX - 1] = -INFINITY; id[KMAX - 1] = 0x7fffffff;
-    }
-};
-// KMAX rounds: the best head of the warp's 32 lists is taken out (ids are unique, so exactly one lane pops) and
-// handed to lane `round`; afterwards lane r < KMAX holds the warp's r-th best entry.
-template <int KMAX>
-__device__ __forceinline__ void warp_merge(TopList<KMAX>& t, float& out_v, int& out_id) {
-    const int lane = threadIdx.x & 31;
-    out_v = -INFINITY; out_id = 0x7fffffff;
-#pragma unroll 1
-    for (int r = 0; r < KMAX; ++r) {
-        float bv = t.v[0]; int bi = t.id[0];
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) {
-            const float ov = __shfl_xor_sync(0xffffffffu, bv, o);
-            const int oi = __shfl_xor_sync(0xffffffffu, bi, o);
-            if (ov > bv || (ov == bv && oi < bi)) { bv = ov; bi = oi; }
-        }
-        if (bi != 0x7fffffff && t.id[0] == bi) t.pop();
-        if (lane == r) { out_v = bv; out_id = bi; }
+    for (int o = 16; o > 0; o >>= 1) {
+        const float ov = __shfl_xor_sync(0xffffffffu, bv, o);
+        const int oi = __shfl_xor_sync(0xffffffffu, bi, o);
+        if (top_better(ov, oi, bv, bi)) { bv = ov; bi = oi; }
     }
 }
-
-template <typename T, int KMAX>
+template <typename T>
 __global__ void __launch_bounds__(TOPK_THREADS) topk_accept_kernel(
         const T* __restrict__ logits, int V, int K, const int32_t* __restrict__ tokens,
         const int32_t* __restrict__ parent, const int32_t* __restrict__ depth,
@@ -692,59 +665,136 @@ __global__ void __launch_bounds__(TOPK_THREADS) topk_accept_kernel(
         float* __restrict__ margin, int32_t* __restrict__ k_acc, int32_t* __restrict__ path,
         int32_t* __restrict__ bonus, int do_accept, unsigned int* tickets) {
     pdl_prologue();
-    __shared__ float warp_v[TOPK_THREADS / 32][KMAX];
-    __shared__ int warp_id[TOPK_THREADS / 32][KMAX];
+    __shared__ float cand_v[TOPK_CAND + TRJ_MAX_TOPK];             // candidates of the chunk, then the running list
+    __shared__ int cand_i[TOPK_CAND + TRJ_MAX_TOPK];
+    __shared__ float list_v[TOPK_THREADS / 32][TRJ_MAX_TOPK];      // slow path: the warps' sorted lists; [0] also: warp maxima
+    __shared__ int list_i[TOPK_THREADS / 32][TRJ_MAX_TOPK];
+    __shared__ float best_v[TRJ_MAX_TOPK];                          // the row's running list, sorted
+    __shared__ int best_i[TRJ_MAX_TOPK];
+    __shared__ float warp_max_v[TOPK_THREADS / 32];
+    __shared__ float thr;
+    __shared__ int cand_n;
     __shared__ int last_flag;
-    const int row = blockIdx.x, warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int row = blockIdx.x, tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const T* lr = logits + (size_t)row * V;
-    TopList<KMAX> t;
-    t.clear();
-    constexpr int VEC = 16 / (int)sizeof(T);                 // elements per 16-byte load
-    if (V % VEC == 0 && ((uintptr_t)logits % 16) == 0) {
-        // four 16-byte loads are requested before the first of them is looked at: the row comes from L2 or HBM and
-        // a CTA has nothing else to hide that latency with
-        constexpr int BATCH = 4;
-        for (int v0 = threadIdx.x * VEC; v0 < V; v0 += BATCH * TOPK_THREADS * VEC) {
-            uint4 raw[BATCH];
+    if (tid < TRJ_MAX_TOPK) { best_v[tid] = -INFINITY; best_i[tid] = 0x7fffffff; }
+    for (int base = 0; base < V; base += TOPK_PER_THREAD * TOPK_THREADS) {
+        float x[TOPK_PER_THREAD];
+        float tm = -INFINITY;
 #pragma unroll
-            for (int j = 0; j < BATCH; ++j) {
-                const int v = v0 + j * TOPK_THREADS * VEC;
-                if (v < V) raw[j] = *reinterpret_cast<const uint4*>(lr + v);
+        for (int j = 0; j < TOPK_PER_THREAD; ++j) {
+            const int id = base + j * TOPK_THREADS + tid;
+            x[j] = id < V ? to_f(lr[id]) : -INFINITY;
+            tm = fmaxf(tm, x[j]);
+        }
+        // (A) warp maxima, then the K-th largest of them (with multiplicity) in the first warp
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) tm = fmaxf(tm, __shfl_xor_sync(0xffffffffu, tm, o));
+        if (lane == 0) warp_max_v[warp] = tm;
+        __syncthreads();
+        if (warp == 0) {
+            float mine = warp_max_v[lane], kth = -INFINITY;
+            for (int r = 0; r < K; ++r) {
+                float m = mine;
+#pragma unroll
+                for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
+                kth = m;
+                const unsigned holders = __ballot_sync(0xffffffffu, mine == m);
+                if (lane == __ffs(holders) - 1) mine = -INFINITY;      // one holder gives its value up per round
             }
+            if (lane == 0) { thr = fmaxf(kth, best_v[K - 1]); cand_n = 0; }
+        }
+        __syncthreads();
+        // (B) candidates
+        const float t = thr;
 #pragma unroll
-            for (int j = 0; j < BATCH; ++j) {
-                const int v = v0 + j * TOPK_THREADS * VEC;
-                if (v < V) {
-                    const T* e = reinterpret_cast<const T*>(&raw[j]);
+        for (int j = 0; j < TOPK_PER_THREAD; ++j) {
+            const int id = base + j * TOPK_THREADS + tid;
+            if (id < V && x[j] >= t) {
+                const int slot = atomicAdd(&cand_n, 1);
+                if (slot < TOPK_CAND) { cand_v[slot] = x[j]; cand_i[slot] = id; }
+            }
+        }
+        __syncthreads();
+        const int n_cand = cand_n;                           // the same for every thread
+        if (n_cand <= TOPK_CAND) {
+            // (C) the first warp: K best of the candidates and the running list
+            if (warp == 0) {
+                if (lane < K) { cand_v[n_cand + lane] = best_v[lane]; cand_i[n_cand + lane] = best_i[lane]; }
+                __syncwarp();
+                const int n = n_cand + K;
+                float mv = -INFINITY;
+                int mi = 0x7fffffff;
+                for (int r = 0; r < K; ++r) {
+                    float bv = -INFINITY;
+                    int bi = 0x7fffffff, bs = -1;
+                    for (int e = lane; e < n; e += 32) {
+                        const float v = cand_v[e];
+                        const int i = cand_i[e];
+                        if (i != 0x7fffffff && top_better(v, i, bv, bi)) { bv = v; bi = i; bs = e; }
+                    }
+                    const int mine_i = bi;
+                    warp_best(bv, bi);
+                    if (bs >= 0 && mine_i == bi) cand_i[bs] = 0x7fffffff;     // taken (ids are unique: one lane owns it)
+                    __syncwarp();
+                    if (lane == r) { mv = bv; mi = bi; }
+                }
+                if (lane < K) { best_v[lane] = mv; best_i[lane] = mi; }
+            }
+        } else {
+            // slow path: K rounds over all elements of the chunk in every warp, then over the warps' lists
+            uint32_t taken = 0;
+            for (int r = 0; r < K; ++r) {
+                float bv = -INFINITY;
+                int bj = -1;
 #pragma unroll
-                    for (int i = 0; i < VEC; ++i) t.push(to_f(e[i]), v + i);
+                for (int j = 0; j < TOPK_PER_THREAD; ++j)    // ascending ids: "strictly larger" keeps the smallest id among equals
+                    if (!((taken >> j) & 1u) && x[j] > bv) { bv = x[j]; bj = j; }
+                int bi = bj >= 0 ? base + bj * TOPK_THREADS + tid : 0x7fffffff;
+                const int mine_i = bi;
+                warp_best(bv, bi);
+                if (bi == mine_i && bj >= 0) taken |= 1u << bj;
+                if (lane == 0) { list_v[warp][r] = bv; list_i[warp][r] = bi; }
+            }
+            __syncthreads();
+            if (warp == 0) {
+                int head = 0;
+                float mv = -INFINITY;
+                int mi = 0x7fffffff;
+                for (int r = 0; r < K; ++r) {
+                    float bv = head < K ? list_v[lane][head] : -INFINITY;
+                    int bi = head < K ? list_i[lane][head] : 0x7fffffff;
+                    const int mine_i = bi;
+                    warp_best(bv, bi);
+                    if (bi == mine_i && bi != 0x7fffffff) ++head;
+                    if (lane == r) { mv = bv; mi = bi; }
+                }
+                if (lane < K) { list_v[0][lane] = mv; list_i[0][lane] = mi; }
+                __syncwarp();
+                if (lane == 0) {                             // two sorted lists of K entries -> the K best
+                    float nv[TRJ_MAX_TOPK];
+                    int ni[TRJ_MAX_TOPK];
+                    int a = 0, c = 0;
+                    for (int r = 0; r < K; ++r) {
+                        if (top_better(list_v[0][a], list_i[0][a], best_v[c], best_i[c])) { nv[r] = list_v[0][a]; ni[r] = list_i[0][a]; ++a; }
+                        else { nv[r] = best_v[c]; ni[r] = best_i[c]; ++c; }
+                    }
+                    for (int r = 0; r < K; ++r) { best_v[r] = nv[r]; best_i[r] = ni[r]; }
                 }
             }
         }
-    } else {
-        for (int v = threadIdx.x; v < V; v += TOPK_THREADS) t.push(to_f(lr[v]), v);
+        __syncthreads();                                     // the buffers are rewritten by the next chunk
     }
-    float cv; int ci;
-    warp_merge<KMAX>(t, cv, ci);
-    if (lane < KMAX) { warp_v[warp][lane] = cv; warp_id[warp][lane] = ci; }
-    __syncthreads();
-    if (warp == 0) {
-        // lane w's list = warp w's merged list (already sorted)
-#pragma unroll
-        for (int i = 0; i < KMAX; ++i) { t.v[i] = warp_v[lane][i]; t.id[i] = warp_id[lane][i]; }
-        warp_merge<KMAX>(t, cv, ci);
-        if (lane < K && topk) topk[(size_t)row * K + lane] = ci;
-        const float second = __shfl_sync(0xffffffffu, cv, 1);
-        if (lane == 0) {
-            node_argmax[row] = ci;
-            if (margin) margin[row] = cv - second;
-            __threadfence();
-            const int b = seq_of_row(row_off, B, row);
-            const unsigned int need = (unsigned int)(row_off[b + 1] - row_off[b]);
-            const unsigned int got = atomicAdd(&tickets[b], 1u);
-            last_flag = (got + 1 == need) ? b : -1;
-            if (got + 1 == need) tickets[b] = 0;             // ready for the next call
-        }
+    if (tid < K && topk) topk[(size_t)row * K + tid] = best_i[tid];
+    if (tid == 0) {
+        node_argmax[row] = best_i[0];
+        if (margin) margin[row] = best_v[0] - best_v[K > 1 ? 1 : 0];
+        __threadfence();
+        const int b = seq_of_row(row_off, B, row);
+        const unsigned int need = (unsigned int)(row_off[b + 1] - row_off[b]);
+        const unsigned int got = atomicAdd(&tickets[b], 1u);
+        last_flag = (got + 1 == need) ? b : -1;
+        if (got + 1 == need) tickets[b] = 0;                 // ready for the next call
     }
     __syncthreads();
     const int b = last_flag;
@@ -1101,7 +1151,7 @@ cudaError_t launch_topk_accept(const void* logits, int32_t dtype, int32_t V, int
         if (launch_err == cudaSuccess && topk)
             launch_err = cudaMemcpyAsync(topk, node_argmax, sizeof(int32_t) * (size_t)rows_total, cudaMemcpyDeviceToDevice, st);
     } else {
-        DISPATCH_T(dtype, launch_err = launch_chain(topk_accept_kernel<T, TRJ_MAX_TOPK>, dim3(rows_total), dim3(TOPK_THREADS), 0, st,
+        DISPATCH_T(dtype, launch_err = launch_chain(topk_accept_kernel<T>, dim3(rows_total), dim3(TOPK_THREADS), 0, st,
                                                     (const T*)logits, V, K, tokens, parent, depth, row_off, B, topk, node_argmax,
                                                     margin, k_acc, path, bonus, do_accept ? 1 : 0, tickets));
     }

@@ -203,6 +203,30 @@ def test_topk_accept_against_oracle(trj, rows_list, vocab, k, dtype):
             assert res["path"][b, :kk + 1].tolist() == path and (res["path"][b, kk + 1:] == -1).all()
 
 
+@pytest.mark.parametrize("vocab,k", [(40000, 10), (128256, 7), (5000, 10)])
+def test_topk_with_thousands_of_equal_values(trj, vocab, k):
+    """Rows in which far more entries tie for the top than any candidate buffer holds (all equal; a plateau of 3 000
+    maxima; a few distinct values above a plateau; plateaus that straddle the 32 768-entry chunks): the K smallest ids
+    of the best values must come out, bit for bit as the oracle's total order (value first, then the smaller id)."""
+    g = synth.stream(vocab, "plateau")
+    rows = 6
+    logits = g.standard_normal((rows, vocab)).astype(np.float32)
+    logits[0, :] = 0.25                                                  # everything ties
+    top = g.choice(vocab, size=min(3000, vocab // 2), replace=False)
+    logits[1, top] = 9.0                                                 # a plateau of maxima
+    logits[2, top] = 9.0; logits[2, top[:3]] = [11.0, 10.0, 10.0]        # three above it, two of them tied
+    logits[3, -1500:] = 7.0; logits[3, :20] = 7.0                        # plateau at both ends of the row
+    logits[4, 32768 - 600:min(vocab, 32768 + 600)] = 8.0                 # plateau across a chunk boundary
+    parents = [synth.chain_parents(rows)]
+    tokens = synth.prompt(3, rows, vocab)
+    depth = np.concatenate([oracle.depths(p) for p in parents])
+    res = trj.topk_accept(to_dev(logits, "f32"), i32(tokens), i32(np.concatenate(parents)), i32(depth), i32([0, rows]), k)
+    torch.cuda.synchronize()
+    np.testing.assert_array_equal(res["topk"].cpu().numpy(), oracle.node_topk(logits, k))
+    np.testing.assert_array_equal(res["node_argmax"].cpu().numpy(), oracle.node_argmax(logits))
+    np.testing.assert_array_equal(res["margin"].cpu().numpy(), oracle.top2_margin(logits).astype(np.float32))
+
+
 def test_argmax_ties_go_to_the_smallest_id_and_workspace_is_reusable(trj):
     rows, vocab = 9, 4099
     logits = np.zeros((rows, vocab), np.float32)
