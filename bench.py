@@ -234,6 +234,14 @@ def bench_small_ops(trj, torch, peaks, steps, warmup, cpu=True):
     us = graph_us(torch, argmax_static_pass, steps, warmup) / n_arr
     out.append({"op": "argmax_accept_static (library-held scratch), same input", "us_per_launch": round(us, 2),
                 "algorithmic_bytes": nbytes, "hbm_gbs": round(nbytes / us / 1e3, 1)})
+    tk_ws = torch.zeros(trj.lib().trj_topk_accept_workspace(), dtype=torch.uint8, device="cuda")
+
+    def topk_pass():                                         # per-row top-10 + acceptance (templates with top-K siblings)
+        for a in range(n_arr):
+            trj.topk_accept(logits[a], tokens, d_parent, d_depth, off, 10, workspace=tk_ws)
+    us = graph_us(torch, topk_pass, steps, warmup) / n_arr
+    out.append({"op": "topk_accept K = 10, same input", "us_per_launch": round(us, 2), "algorithmic_bytes": nbytes,
+                "hbm_gbs": round(nbytes / us / 1e3, 1), "frac_of_" + peaks["source"] + "_peak": round(nbytes / us / 1e3 / peaks["hbm_gbs"], 4)})
     del logits
     # compaction: 32 layers x 32 heads x 128, k = 4 accepted rows of a 33-row tree behind a 512-row prefix
     n_layers, h, d, max_seq, k_acc = 32, 32, 128, 640, 4
