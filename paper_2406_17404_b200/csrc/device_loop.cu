@@ -13,23 +13,34 @@ constexpr int MAX_BRANCHES = 64;          // R is bounded by the tree size (R * 
 
 // Prompt-lookup matches, by a whole warp: the positions that followed the R most recent earlier occurrences of the
 // context's last two tokens, then of its last token (no position twice).  Every lane ends up with the same list.
+// The context is walked from its end in blocks of FOLLOW_BLOCK tokens that the warp first copies to shared memory
+// (32 independent loads per lane, one trip to L2 per block instead of one per 32 tokens).
+constexpr int FOLLOW_BLOCK = 1024;
 __device__ __forceinline__ int find_follows(const int32_t* __restrict__ context, int n, int R, int* follow, int lane) {
+    __shared__ int32_t blk[FOLLOW_BLOCK + 1];                // tokens lo .. lo + FOLLOW_BLOCK (one more: the pair's second token)
     int nf = 0;
     for (int g = 2; g >= 1 && nf < R; --g) {
         if (n <= g) continue;
         const int t0 = context[n - g], t1 = context[n - 1];          // g == 1: t0 == t1
-        for (int base = n - g - 1; base >= 0 && nf < R; base -= 32) {
-            const int p = base - lane;
-            bool match = false;
-            if (p >= 0) match = context[p] == t0 && (g == 1 || context[p + 1] == t1);
-            unsigned m = __ballot_sync(0xffffffffu, match);
-            while (m && nf < R) {                            // lane 0 holds the largest p: ascending lanes = descending p
-                const int l = __ffs(m) - 1;
-                m &= m - 1;
-                const int f = base - l + g;
-                bool seen = false;
-                for (int i = 0; i < nf; ++i) seen |= follow[i] == f;
-                if (!seen) follow[nf++] = f;
+        // candidate positions p = n - g - 1 down to 0
+        for (int hi = n - g - 1; hi >= 0 && nf < R; hi -= FOLLOW_BLOCK) {
+            const int lo = max(hi - FOLLOW_BLOCK + 1, 0);
+            __syncwarp();
+            for (int i = lo + lane; i <= hi + 1; i += 32) blk[i - lo] = context[i];      // hi + 1 <= n - g < n
+            __syncwarp();
+            for (int base = hi; base >= lo && nf < R; base -= 32) {
+                const int p = base - lane;
+                bool match = false;
+                if (p >= lo) match = blk[p - lo] == t0 && (g == 1 || blk[p - lo + 1] == t1);
+                unsigned m = __ballot_sync(0xffffffffu, match);
+                while (m && nf < R) {                        // lane 0 holds the largest p: ascending lanes = descending p
+                    const int l = __ffs(m) - 1;
+                    m &= m - 1;
+                    const int f = base - l + g;
+                    bool seen = false;
+                    for (int i = 0; i < nf; ++i) seen |= follow[i] == f;
+                    if (!seen) follow[nf++] = f;
+                }
             }
         }
     }
@@ -157,19 +168,26 @@ __global__ void __launch_bounds__(32) commit_refill_tree_kernel(const int32_t* _
         return;
     }
     for (int j = lane; j < k; j += 32) context[n + j] = tokens[path[j + 1]];
-    if (lane == 0) {
-        context[n + k] = *bonus;
-        int nb = 0;
-        for (int cur = path[k];;) {
-            int child = -1;
-            for (int c = cur + 1; c < M; ++c)
-                if (parent[c] == cur) { child = c; break; }
-            if (child < 0) break;
-            below[nb++] = child;
-            cur = child;
+    if (lane == 0) context[n + k] = *bonus;
+    // the rows below the winner along its own path: the lowest-index child at every level, found by the whole warp
+    // over a copy of the parent array in shared memory
+    __shared__ int32_t par_s[TRJ_MAX_ROWS];
+    for (int i = lane; i < M; i += 32) par_s[i] = parent[i];
+    __syncwarp();
+    int nb = 0;
+    for (int cur = path[k];;) {
+        int child = -1;
+        for (int c0 = cur + 1; c0 < M && child < 0; c0 += 32) {
+            const int c = c0 + lane;
+            const unsigned hit = __ballot_sync(0xffffffffu, c < M && par_s[c] == cur);
+            if (hit) child = c0 + __ffs(hit) - 1;
         }
-        n_below_s = nb;
+        if (child < 0) break;
+        if (lane == 0) below[nb] = child;
+        ++nb;
+        cur = child;
     }
+    if (lane == 0) n_below_s = nb;
     __syncwarp();
     const int n_new = n + k + 1, n_below = n_below_s;
     for (int i = 1 + lane; i < M; i += 32) {
