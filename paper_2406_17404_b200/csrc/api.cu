@@ -200,7 +200,8 @@ struct trj_ctx {
     std::vector<LoopGraph> loop_graphs;
     cudaStream_t cap_stream = nullptr; cudaEvent_t order_ev = nullptr; uint64_t steps_done = 0;
     DraftSource draft_src{nullptr, 0, nullptr}; int32_t draft_src_steps = 0;   // trj_set_draft_source
-    int32_t last_rows = 0, last_B = 0; const int32_t* last_row_off = nullptr;  // geometry of the latest trj_verify_step    // the step a tensor-parallel rank is walking through segment by segment (trj_tp_begin .. trj_tp_finish)
+    int32_t last_rows = 0, last_B = 0; const int32_t* last_row_off = nullptr;  // geometry of the latest trj_verify_step
+    // the step a tensor-parallel rank is walking through segment by segment (trj_tp_begin .. trj_tp_finish)
     struct TpStep {
         bool open = false; int32_t next = 0; void* k_cache = nullptr; void* v_cache = nullptr;
         Batch bt{}; const int32_t* tokens = nullptr; const int32_t* parent = nullptr; const int32_t* depth = nullptr;
@@ -214,7 +215,7 @@ namespace {
 // streamed once per chunk); attention runs inside a chunk in pieces of at most TRJ_MAX_ROWS rows, at most 16 of them.
 constexpr int PREFILL_CHUNK = 512;
 constexpr int PREFILL_MAX_SUB = 16;
-struct SubChunks { int n, sub, last_rows; const int32_t* lens; const int32_t* off_full; const int32_t* off_last; };
+struct SubChunks { int n, sub; const int32_t* lens; const int32_t* off_pieces; };
 
 constexpr int STEP_IN_INTS = 3 * TRJ_MAX_ROWS + 4;                       // + anc (2 words per row) after it
 constexpr int STEP_IN_BYTES = STEP_IN_INTS * 4 + TRJ_MAX_ROWS * 2 * 8;
@@ -241,7 +242,8 @@ size_t carve(const trj_model_cfg& c, void* ws, trj_ctx* ctx) {
     char* act_lo = cv.take<char>((size_t)rows * c.d_ff * es);
     double* inv_freq = cv.take<double>(c.head_dim / 2);
     char* argmax_ws = cv.take<char>(argmax_workspace_bytes(step_rows, c.max_batch));
-    const size_t attn_bytes = trj_tree_attention_workspace(step_rows, c.max_batch, c.n_heads, c.head_dim, c.max_seq);
+    // a prefill chunk's pieces are the sequences of one attention launch
+    const size_t attn_bytes = trj_tree_attention_workspace(rows, std::max(c.max_batch, PREFILL_MAX_SUB), c.n_heads, c.head_dim, c.max_seq);
     char* attn_ws = cv.take<char>(attn_bytes);
     // every row count a call may bring (the K split, hence the space for partial sums, is not monotone in it)
     size_t gemm_bytes = 256;
@@ -251,8 +253,8 @@ size_t carve(const trj_model_cfg& c, void* ws, trj_ctx* ctx) {
             gemm_bytes = std::max(gemm_bytes, gemm_tc_workspace(m, nk.first, nk.second));
     char* gemm_ws = cv.take<char>(gemm_bytes);
     int32_t* chain_depth = cv.take<int32_t>(PREFILL_CHUNK);
-    int32_t* prefill_geo = cv.take<int32_t>(PREFILL_MAX_SUB + 6);   // piece lengths, then three {0, n} row-offset pairs
-    uint64_t* chain_anc = cv.take<uint64_t>(TRJ_MAX_ROWS * 2);
+    int32_t* prefill_geo = cv.take<int32_t>(2 * PREFILL_MAX_SUB + 4);   // piece lengths, {0, m}, piece row offsets
+    uint64_t* chain_anc = cv.take<uint64_t>((size_t)PREFILL_CHUNK * 2);   // row i: the chain mask of row i % (rows of a piece)
     int32_t* chunk_row_off = cv.take<int32_t>(2);
     int32_t* unit_row_off = cv.take<int32_t>(2);
     int32_t* step_in = (int32_t*)cv.take<char>(STEP_IN_BYTES);
@@ -396,16 +398,12 @@ trj_status run_segments(trj_ctx* ctx, const StepArgs& a, int s0, int s1, Parts& 
                                                              c.max_seq, c.dtype, ctx->x, ctx->x_lo, ctx->attn_ws,
                                                              ctx->attn_ws_bytes, st, attn_status));
             } else {
-                for (int j = 0; j < pieces->n; ++j) {
-                    const int mj = j + 1 < pieces->n ? pieces->sub : pieces->last_rows;
-                    // piece j sees the rows of pieces 0..j-1 as cached rows, and those were written by this very chain
-                    Batch bj{pieces->lens + j, j + 1 < pieces->n ? pieces->off_full : pieces->off_last, 1, mj, mj, bt.max_len, j == 0 ? 1 : 0};
-                    const size_t off = (size_t)j * pieces->sub * HD * es;
-                    LAUNCH(PROF_ATTENTION, launch_tree_attention((char*)ctx->q + off, k_slab, v_slab, a.anc, a.anc_words, bj, c.n_heads, Hkv,
-                                                                 c.head_dim, c.max_seq, c.dtype, (char*)ctx->x + off,
-                                                                 ctx->x_lo ? (char*)ctx->x_lo + off : nullptr, ctx->attn_ws,
-                                                                 ctx->attn_ws_bytes, st, attn_status));
-                }
+                // the pieces of the chunk are the sequences of ONE launch: piece j sees the prompt so far plus the pieces
+                // before it as cached rows (all written by the rotary kernel above, inside this chain) of the same cache
+                Batch bj{pieces->lens, pieces->off_pieces, pieces->n, M, pieces->sub, bt.max_len, 0, 1};
+                LAUNCH(PROF_ATTENTION, launch_tree_attention(ctx->q, k_slab, v_slab, a.anc, a.anc_words, bj, c.n_heads, Hkv, c.head_dim,
+                                                             c.max_seq, c.dtype, ctx->x, ctx->x_lo, ctx->attn_ws,
+                                                             ctx->attn_ws_bytes, st, attn_status));
             }
             // While the attention kernel runs, HBM is nearly idle and the SMs it leaves free go to the first CTAs of
             // the output projection, which only wait: they ask for the start of the gate/up weights into L2.
@@ -506,13 +504,15 @@ extern "C" trj_status trj_create(const trj_model_cfg* cfg, const trj_weights* w,
     for (int i = 0; i < half; ++i) freq[i] = std::pow((double)cfg->rope_theta, -2.0 * i / cfg->head_dim);
     std::vector<int32_t> par(TRJ_MAX_ROWS), dep(TRJ_MAX_ROWS), long_dep(PREFILL_CHUNK);
     for (int i = 0; i < PREFILL_CHUNK; ++i) long_dep[i] = i;
-    std::vector<uint64_t> anc(TRJ_MAX_ROWS * 2);
+    std::vector<uint64_t> anc(TRJ_MAX_ROWS * 2), anc_long((size_t)PREFILL_CHUNK * 2);
     for (int i = 0; i < TRJ_MAX_ROWS; ++i) par[i] = i - 1;
     tree_from_parents_impl(par.data(), TRJ_MAX_ROWS, 2, dep.data(), anc.data());
+    const int piece_rows = std::min(cfg->max_rows, TRJ_MAX_ROWS);
+    for (int i = 0; i < PREFILL_CHUNK; ++i) { anc_long[2 * i] = anc[2 * (i % piece_rows)]; anc_long[2 * i + 1] = anc[2 * (i % piece_rows) + 1]; }
     const int32_t unit[2] = {0, 1};
     cudaError_t e = cudaMemcpy(ctx->inv_freq, freq.data(), sizeof(double) * half, cudaMemcpyHostToDevice);
     if (e == cudaSuccess) e = cudaMemcpy(ctx->chain_depth, long_dep.data(), sizeof(int32_t) * PREFILL_CHUNK, cudaMemcpyHostToDevice);
-    if (e == cudaSuccess) e = cudaMemcpy(ctx->chain_anc, anc.data(), sizeof(uint64_t) * TRJ_MAX_ROWS * 2, cudaMemcpyHostToDevice);
+    if (e == cudaSuccess) e = cudaMemcpy(ctx->chain_anc, anc_long.data(), sizeof(uint64_t) * PREFILL_CHUNK * 2, cudaMemcpyHostToDevice);
     if (e == cudaSuccess) e = cudaMemcpy(ctx->unit_row_off, unit, sizeof(unit), cudaMemcpyHostToDevice);
     if (e == cudaSuccess) e = cudaMallocHost((void**)&ctx->pin_in, STEP_IN_BYTES);
     if (e == cudaSuccess) e = cudaMallocHost((void**)&ctx->pin_out, sizeof(int32_t) * STEP_OUT_INTS);
@@ -794,14 +794,14 @@ extern "C" trj_status trj_prefill(trj_ctx* ctx, void* k_cache, void* v_cache, in
     cudaStream_t st = (cudaStream_t)stream;
     const int32_t sub = std::min(c.max_rows, TRJ_MAX_ROWS);                  // rows of an attention piece
     const int32_t chunk_cap = std::min(PREFILL_CHUNK, PREFILL_MAX_SUB * sub);
-    int32_t* lens = ctx->prefill_geo, *off_all = lens + PREFILL_MAX_SUB, *off_full = off_all + 2, *off_last = off_all + 4;
+    int32_t* lens = ctx->prefill_geo, *off_all = lens + PREFILL_MAX_SUB, *off_pieces = off_all + 2;
     for (int32_t done = 0; done < n; done += chunk_cap) {
         const int32_t m = std::min(chunk_cap, n - done);
         const bool last = done + m >= n;
-        const int32_t n_sub = (m + sub - 1) / sub, last_rows = m - (n_sub - 1) * sub;
-        TRJ_CHECK_CUDA(launch_prefill_geometry(seq_len + b, lens, n_sub, sub, m, last_rows, off_all, off_full, off_last, st));
+        const int32_t n_sub = (m + sub - 1) / sub;
+        TRJ_CHECK_CUDA(launch_prefill_geometry(seq_len + b, lens, n_sub, sub, m, off_all, off_pieces, st));
         Batch bt{seq_len + b, off_all, 1, m, sub, c.max_seq};
-        const SubChunks pieces{n_sub, sub, last_rows, lens, off_full, off_last};
+        const SubChunks pieces{n_sub, sub, lens, off_pieces};
         trj_status s = forward(ctx, k_cache, v_cache, b, bt, tokens + done, ctx->chain_depth, ctx->chain_anc, 2,
                                m - 1, last ? 1 : 0, st, &pieces);
         if (s != TRJ_OK) return s;

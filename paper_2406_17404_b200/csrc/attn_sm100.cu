@@ -54,6 +54,7 @@ struct AtParams {
     float scale_log2;            // log2(e) / sqrt(D)
     int cluster;                 // CTAs per thread-block cluster that share one head (1: no clusters)
     int early_ok;                // cache rows below seq_len are older than the chain: they may be fetched before the wait
+    int shared_cache;            // every sequence of the batch uses the cache of sequence 0 (pieces of one prompt chunk)
 };
 
 using namespace sm100;
@@ -373,7 +374,7 @@ __global__ void __launch_bounds__(at_threads(AT_SPLIT), 1) tree_attention_tc_ker
                 // the first segment's Q is requested by the MMA thread as soon as the previous kernel is done, so
                 // that it does not queue behind the cache tiles this thread asks for ahead of the wait
                 if (e > 0) { ok = load_q(); if (!ok) break; }
-                const int cache_row0 = (w.b * p.Hkv + w.h / p.group) * p.max_seq;
+                const int cache_row0 = ((p.shared_cache ? 0 : w.b) * p.Hkv + w.h / p.group) * p.max_seq;
                 const int old_tiles = w.S / AT_KEYS;          // tiles that hold cached rows only
                 for (int t = w.t; t < t_end && ok; ++t, ++g) {
                     for (int kv = 0; kv < 2 && ok; ++kv) {
@@ -898,14 +899,15 @@ cudaError_t launch_tree_attention_tc(const void* q, const void* k_slab, const vo
     if (attr_err != cudaSuccess) return attr_err;
     CUtensorMap map_q, map_k, map_v;
     if (!at_make_map(&map_q, q, (size_t)bt.rows_total, (size_t)H * AT_D) ||
-        !at_make_map(&map_k, k_slab, (size_t)bt.B * Hkv * max_seq, AT_D) ||
-        !at_make_map(&map_v, v_slab, (size_t)bt.B * Hkv * max_seq, AT_D))
+        !at_make_map(&map_k, k_slab, (size_t)(bt.shared_cache ? 1 : bt.B) * Hkv * max_seq, AT_D) ||
+        !at_make_map(&map_v, v_slab, (size_t)(bt.shared_cache ? 1 : bt.B) * Hkv * max_seq, AT_D))
         return cudaErrorInvalidValue;
     AtParams p;
     p.seq_len = bt.seq_len; p.row_off = bt.row_off; p.anc = anc; p.anc_words = anc_words;
     p.B = bt.B; p.H = H; p.max_seq = max_seq;
     p.Hkv = Hkv; p.group = H / Hkv;
     p.early_ok = bt.cached_rows_final;
+    p.shared_cache = bt.shared_cache;
     p.out = (__nv_bfloat16*)out;
     p.out_lo = (__nv_bfloat16*)out_lo;
     p.status = status ? status : (int*)workspace;

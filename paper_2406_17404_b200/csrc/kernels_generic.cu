@@ -395,7 +395,8 @@ template <typename T, int D>
 __global__ void __launch_bounds__(128) tree_attention_generic_kernel(
         const T* __restrict__ q, const T* __restrict__ k_slab, const T* __restrict__ v_slab,
         const uint64_t* __restrict__ anc, int anc_words, const int32_t* __restrict__ seq_len,
-        const int32_t* __restrict__ row_off, int B, int H, int Hkv, int max_seq, T* __restrict__ out, T* __restrict__ out_lo) {
+        const int32_t* __restrict__ row_off, int B, int H, int Hkv, int max_seq, T* __restrict__ out, T* __restrict__ out_lo,
+        int shared_cache) {
     constexpr int PER = D / 32;                  // output dims per lane
     __shared__ float qs[D];
     __shared__ float part_m[4], part_l[4];
@@ -407,8 +408,9 @@ __global__ void __launch_bounds__(128) tree_attention_generic_kernel(
     const int total = TRJ_DEBUG_CHECK(seq_len[b] >= 0 && S + rows_b <= max_seq, DBG_ATTENTION_LEN) ? S + rows_b : min(S + rows_b, max_seq);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int kvh = hh / (H / Hkv);              // grouped-query attention: the K/V head of this query head
-    const T* kb = k_slab + ((size_t)b * Hkv + kvh) * max_seq * D;
-    const T* vb = v_slab + ((size_t)b * Hkv + kvh) * max_seq * D;
+    const int cb = shared_cache ? 0 : b;         // pieces of one prompt chunk share the cache of sequence 0
+    const T* kb = k_slab + ((size_t)cb * Hkv + kvh) * max_seq * D;
+    const T* vb = v_slab + ((size_t)cb * Hkv + kvh) * max_seq * D;
     const uint64_t* mask = anc + (size_t)row * anc_words;
     for (int c = threadIdx.x; c < D; c += blockDim.x) qs[c] = to_f(q[((size_t)row * H + hh) * D + c]);
     __syncthreads();
@@ -985,12 +987,11 @@ __global__ void advance_len_kernel(int32_t* seq_len, const int32_t* k_acc, int B
     if (b < B) seq_len[b] += k_acc[b] + 1;
 }
 __global__ void set_chunk_kernel(int32_t* row_off2, int m) { row_off2[0] = 0; row_off2[1] = m; }
-__global__ void prefill_geometry_kernel(const int32_t* seq_len_b, int32_t* lens, int n_sub, int sub, int m, int last_rows,
-                                        int32_t* off_all, int32_t* off_full, int32_t* off_last) {
+__global__ void prefill_geometry_kernel(const int32_t* seq_len_b, int32_t* lens, int n_sub, int sub, int m, int32_t* off_all,
+                                        int32_t* off_pieces) {
     for (int j = threadIdx.x; j < n_sub; j += blockDim.x) lens[j] = *seq_len_b + j * sub;
-    if (threadIdx.x == 0) {
-        off_all[0] = 0; off_all[1] = m; off_full[0] = 0; off_full[1] = sub; off_last[0] = 0; off_last[1] = last_rows;
-    }
+    for (int j = threadIdx.x; j <= n_sub; j += blockDim.x) off_pieces[j] = min(j * sub, m);
+    if (threadIdx.x == 0) { off_all[0] = 0; off_all[1] = m; }
 }
 __global__ void bump_len_kernel(int32_t* seq_len_b, int delta) { *seq_len_b += delta; }
 
@@ -1084,7 +1085,7 @@ cudaError_t launch_tree_attention_generic(const void* q, const void* k_slab, con
 #define ATT(DD)                                                                                          \
     DISPATCH_T(dtype, tree_attention_generic_kernel<T, DD><<<grid, 128, 0, st>>>(                        \
                           (const T*)q, (const T*)k_slab, (const T*)v_slab, anc, anc_words, bt.seq_len,   \
-                          bt.row_off, bt.B, H, Hkv, max_seq, (T*)out, (T*)out_lo))
+                          bt.row_off, bt.B, H, Hkv, max_seq, (T*)out, (T*)out_lo, bt.shared_cache))
     if (D == 64) { ATT(64); }
     else if (D == 128) { ATT(128); }
     else return cudaErrorInvalidValue;
@@ -1246,9 +1247,9 @@ cudaError_t launch_set_chunk(int32_t* row_off2, int32_t m, cudaStream_t st) {
     return cudaGetLastError();
 }
 cudaError_t launch_prefill_geometry(const int32_t* seq_len_b, int32_t* lens, int32_t n_sub, int32_t sub, int32_t m,
-                                    int32_t last_rows, int32_t* off_all, int32_t* off_full, int32_t* off_last, cudaStream_t st) {
+                                    int32_t* off_all, int32_t* off_pieces, cudaStream_t st) {
     count_launch();
-    prefill_geometry_kernel<<<1, 32, 0, st>>>(seq_len_b, lens, n_sub, sub, m, last_rows, off_all, off_full, off_last);
+    prefill_geometry_kernel<<<1, 32, 0, st>>>(seq_len_b, lens, n_sub, sub, m, off_all, off_pieces);
     return cudaGetLastError();
 }
 cudaError_t launch_bump_len(int32_t* seq_len_b, int32_t delta, cudaStream_t st) {

@@ -95,6 +95,9 @@ struct Batch {
     // 1: every cache row below seq_len was written before the chain of kernels this batch is launched in began, so a
     // kernel may fetch such rows ahead of its wait for its predecessor; 0: some were written inside the chain
     int32_t cached_rows_final = 1;
+    // 1: every sequence of the batch reads and extends the cache of sequence 0 of the slab (the pieces of a prompt
+    // chunk: piece j is a "sequence" whose cached rows are the prompt so far plus the pieces before it)
+    int32_t shared_cache = 0;
 };
 
 // Weights of a LATER projection that a projection kernel may ask for ahead of time.  When the kernel before a
@@ -245,10 +248,10 @@ cudaError_t launch_compact(void* k_cache, void* v_cache, int32_t L, int32_t B_ca
                            const int32_t* k_acc, const int32_t* path, cudaStream_t st, unsigned int* tickets = nullptr);
 // row_off = {0, m} and seq_len[b] += delta: small bookkeeping used by prefill.
 cudaError_t launch_set_chunk(int32_t* row_off2, int32_t m, cudaStream_t st);
-// Geometry of a prefill chunk of m rows whose attention runs in n_sub pieces of `sub` rows (the last one of
-// last_rows): lens[j] = *seq_len_b + j * sub, off_all = {0, m}, off_full = {0, sub}, off_last = {0, last_rows}.
+// Geometry of a prefill chunk of m rows whose attention treats n_sub pieces of `sub` rows (the last one shorter) as
+// the sequences of one batch: lens[j] = *seq_len_b + j * sub, off_all = {0, m}, off_pieces[j] = min(j * sub, m).
 cudaError_t launch_prefill_geometry(const int32_t* seq_len_b, int32_t* lens, int32_t n_sub, int32_t sub, int32_t m,
-                                    int32_t last_rows, int32_t* off_all, int32_t* off_full, int32_t* off_last, cudaStream_t st);
+                                    int32_t* off_all, int32_t* off_pieces, cudaStream_t st);
 cudaError_t launch_bump_len(int32_t* seq_len_b, int32_t delta, cudaStream_t st);
 
 }  // namespace trj
